@@ -1,0 +1,539 @@
+// ema_oracle.cpp — plain CPU oracle for the memory-slice hot path.
+//
+// TEST INFRASTRUCTURE ONLY. This file is the slow, obviously-correct statement of what the
+// CUDA path must compute. It shares no code, header, table or helper with the CUDA library,
+// and the product never calls it: only the tests, the smoke check and the benchmark's CPU
+// baseline load it.
+//
+// What it states, and the passage of the paper each part follows:
+//   * O-alloc   — a memory slice keeps a mapping table per user and hands out capacity from
+//                 free memory first (Section 4, "Memory Slice", and Section 4.1: "first attempts
+//                 to allocate from free memory"); block ids apply uniformly to every layer
+//                 (Section 4.2.1, layer-major allocation).
+//   * O-gather  — data that lives in the peer's part of the slice is copied into a buffer of
+//                 one transferred chunk before the layer that reads it runs (Section 2.3 latency
+//                 window; Section 4.2.1 "prefetched in time"; Section 4.2.2 swap buffer;
+//                 Section 5.1 "prepares a directly accessible address").
+//   * O-attn    — the consumer of the prepared addresses: decode attention over a paged KV
+//                 cache. The paper inherits it from its serving engine (Section 6.1) and does
+//                 not define it; the definition used is softmax(scale * q K^T) V per query head,
+//                 with grouped-query head mapping g = h / (Hq / Hkv), in fp64.
+//   * O-reclaim — the lender regains capacity at once (Section 4.1, static-dynamic symmetry).
+//                 The paper does it by preempting the borrower; this build migrates the lent
+//                 blocks instead and rewrites the mapping tables (the variant the task fixes).
+//   * O-append  — one new token's K/V row written to its home block and to the staged copy.
+//
+// Parity pins (tests/test_oracle_*.py): paged == dense brute force; softmax row sums; closed
+// forms (n=1, equal keys, constant V, dominant key, score shift, token permutation); fp64
+// library attention; NaN-poisoned tails; tag round trips for gather; byte/logical-order
+// preservation for migration; allocator invariants under random operation sequences.
+// Bit-level agreement of the GPU attention with this file is "parity unpinned" beyond the
+// stated tolerance, by design: any result within tolerance is correct.
+//
+// Block layout (bytes): K plane [T][Hkv][D] bf16, then V plane [T][Hkv][D] bf16.
+// Arena layout: [layer][block id][block bytes].
+// Block-table entry (int32): e >= 0 -> local id e; e < 0 -> lent id ~e.
+// Resolved entry (int32):    e >= 0 -> local id e; e < 0 -> staging position ~e.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <map>
+#include <utility>
+#include <vector>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+enum Status : int {
+  OK = 0,
+  E_INVAL = -1,
+  E_NOSPC = -2,
+  E_STAGING = -3,
+  E_STATE = -7,
+};
+
+enum Tier : int { AUTO = 0, LOCAL = 1, LENT = 2 };
+
+struct Seq {
+  std::vector<int32_t> table;  // logical block -> entry
+  uint32_t len = 0;            // tokens
+};
+
+struct Owner {
+  int32_t seq = -1;
+  int32_t logical = -1;
+};
+
+struct State {
+  uint32_t num_layers = 0;
+  uint32_t block_tokens = 0;
+  uint64_t block_bytes = 0;
+  uint32_t local_blocks = 0;
+  uint32_t lent_cap = 0;   // current lent capacity (ids < lent_cap may be used)
+  uint32_t lent_phys = 0;  // physical size of the lent arena, in block ids
+  uint32_t ring_slots = 0;
+  uint32_t staging_cap = 0;  // blocks per ring slot
+  uint32_t max_seqs = 0;
+  uint32_t max_blocks_per_seq = 0;
+  // Free stacks: back() is the next id popped.
+  std::vector<int32_t> free_local;
+  std::vector<int32_t> free_lent;
+  // Order in which never-yet-lent ids are revealed is irrelevant: lend() pushes explicit ids.
+  std::map<int32_t, Seq> seqs;
+  std::vector<Owner> owner_local;
+  std::vector<Owner> owner_lent;
+};
+
+inline double bf16_to_double(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return static_cast<double>(f);
+}
+
+// Round-to-nearest-even conversion double -> bf16, through float.
+inline uint16_t double_to_bf16_rne(double x) {
+  float f = static_cast<float>(x);
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return static_cast<uint16_t>((u >> 16) | 0x40);
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;
+  return static_cast<uint16_t>(u >> 16);
+}
+
+inline uint32_t blocks_for(uint32_t len, uint32_t block_tokens) {
+  return (len + block_tokens - 1) / block_tokens;
+}
+
+}  // namespace
+
+extern "C" {
+
+// ------------------------------------------------------------------------------------------
+// O-alloc
+// ------------------------------------------------------------------------------------------
+
+// free orders: local_free_order has local_blocks ids, lent_free_order has lent_phys ids (a
+// permutation of the arena); NULL means identity. Pops return order[0], order[1], ...; the lent
+// stack initially holds only the ids < lent_blocks, in that order.
+void* oracle_create(uint32_t num_layers, uint32_t block_tokens, uint64_t block_bytes,
+                    uint32_t local_blocks, uint32_t lent_blocks, uint32_t lent_phys,
+                    uint32_t ring_slots, uint32_t staging_cap, uint32_t max_seqs,
+                    uint32_t max_blocks_per_seq, const uint32_t* local_free_order,
+                    const uint32_t* lent_free_order) {
+  if (lent_blocks > lent_phys || ring_slots == 0 || block_tokens == 0) return nullptr;
+  State* s = new State();
+  s->num_layers = num_layers;
+  s->block_tokens = block_tokens;
+  s->block_bytes = block_bytes;
+  s->local_blocks = local_blocks;
+  s->lent_cap = lent_blocks;
+  s->lent_phys = lent_phys;
+  s->ring_slots = ring_slots;
+  s->staging_cap = staging_cap;
+  s->max_seqs = max_seqs;
+  s->max_blocks_per_seq = max_blocks_per_seq;
+  s->owner_local.assign(local_blocks, Owner());
+  s->owner_lent.assign(lent_phys, Owner());
+  for (uint32_t k = local_blocks; k-- > 0;) {
+    s->free_local.push_back(static_cast<int32_t>(local_free_order ? local_free_order[k] : k));
+  }
+  for (uint32_t k = lent_phys; k-- > 0;) {
+    uint32_t id = lent_free_order ? lent_free_order[k] : k;
+    if (id < lent_blocks) s->free_lent.push_back(static_cast<int32_t>(id));
+  }
+  return s;
+}
+
+void oracle_destroy(void* h) { delete static_cast<State*>(h); }
+
+int oracle_alloc_blocks(void* h, int32_t seq, uint32_t n, int32_t hint, int32_t* out_entries) {
+  State* s = static_cast<State*>(h);
+  if (seq < 0 || hint < AUTO || hint > LENT) return E_INVAL;
+  auto it = s->seqs.find(seq);
+  const bool exists = it != s->seqs.end();
+  if (!exists && s->seqs.size() >= s->max_seqs) return E_INVAL;
+  const size_t have = exists ? it->second.table.size() : 0;
+  if (have + n > s->max_blocks_per_seq) return E_INVAL;
+  const size_t fl = s->free_local.size(), fr = s->free_lent.size();
+  if (hint == AUTO && n > fl + fr) return E_NOSPC;
+  if (hint == LOCAL && n > fl) return E_NOSPC;
+  if (hint == LENT && n > fr) return E_NOSPC;
+  Seq& q = s->seqs[seq];  // creates when absent
+  for (uint32_t k = 0; k < n; ++k) {
+    bool take_local = hint == LOCAL || (hint == AUTO && !s->free_local.empty());
+    int32_t entry;
+    if (take_local) {
+      int32_t id = s->free_local.back();
+      s->free_local.pop_back();
+      s->owner_local[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
+      entry = id;
+    } else {
+      int32_t id = s->free_lent.back();
+      s->free_lent.pop_back();
+      s->owner_lent[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
+      entry = ~id;
+    }
+    q.table.push_back(entry);
+    if (out_entries) out_entries[k] = entry;
+  }
+  return OK;
+}
+
+int oracle_set_seq_len(void* h, int32_t seq, uint32_t len) {
+  State* s = static_cast<State*>(h);
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return E_STATE;
+  if (len > static_cast<uint64_t>(it->second.table.size()) * s->block_tokens) return E_INVAL;
+  it->second.len = len;
+  return OK;
+}
+
+int oracle_free_seq(void* h, int32_t seq) {
+  State* s = static_cast<State*>(h);
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return E_STATE;
+  const std::vector<int32_t>& t = it->second.table;
+  for (size_t b = t.size(); b-- > 0;) {  // descending logical order
+    int32_t e = t[b];
+    if (e >= 0) {
+      s->free_local.push_back(e);
+      s->owner_local[e] = Owner();
+    } else {
+      s->free_lent.push_back(~e);
+      s->owner_lent[~e] = Owner();
+    }
+  }
+  s->seqs.erase(it);
+  return OK;
+}
+
+int oracle_get_block_table(void* h, int32_t seq, int32_t* out, uint32_t cap, uint32_t* n,
+                           uint32_t* len) {
+  State* s = static_cast<State*>(h);
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return E_STATE;
+  const std::vector<int32_t>& t = it->second.table;
+  if (n) *n = static_cast<uint32_t>(t.size());
+  if (len) *len = it->second.len;
+  if (out) {
+    if (cap < t.size()) return E_INVAL;
+    std::copy(t.begin(), t.end(), out);
+  }
+  return OK;
+}
+
+// Free stacks in pop order (first element = next id popped). which: 1 local, 2 lent.
+int oracle_get_free_stack(void* h, int32_t which, int32_t* out, uint32_t cap, uint32_t* n) {
+  State* s = static_cast<State*>(h);
+  const std::vector<int32_t>& st = which == LOCAL ? s->free_local : s->free_lent;
+  if (n) *n = static_cast<uint32_t>(st.size());
+  if (out) {
+    if (cap < st.size()) return E_INVAL;
+    for (size_t k = 0; k < st.size(); ++k) out[k] = st[st.size() - 1 - k];
+  }
+  return OK;
+}
+
+uint32_t oracle_lent_capacity(void* h) { return static_cast<State*>(h)->lent_cap; }
+uint32_t oracle_num_seqs(void* h) { return static_cast<uint32_t>(static_cast<State*>(h)->seqs.size()); }
+
+// ------------------------------------------------------------------------------------------
+// O-gather: resolve a batch's tables and copy every in-use lent block of `layer` into ring
+// slot (layer mod R), in canonical order: batch position, then logical index.
+// resolved is [nseq][max_blocks_per_seq] (entries past a sequence's in-use blocks are left as is).
+// lent_arena / staging may be NULL: then only the integer results are produced.
+// ------------------------------------------------------------------------------------------
+int oracle_gather(void* h, uint32_t layer, const int32_t* seqs, uint32_t nseq,
+                  const uint8_t* lent_arena, uint8_t* staging, int32_t* resolved, uint32_t* k_out) {
+  State* s = static_cast<State*>(h);
+  if (layer >= s->num_layers) return E_INVAL;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    if (s->seqs.find(seqs[i]) == s->seqs.end()) return E_STATE;
+    for (uint32_t j = 0; j < i; ++j)
+      if (seqs[j] == seqs[i]) return E_INVAL;
+  }
+  // Count first, so that an overflow is reported before any byte moves.
+  uint64_t total = 0;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    const Seq& q = s->seqs[seqs[i]];
+    uint32_t nb = blocks_for(q.len, s->block_tokens);
+    for (uint32_t b = 0; b < nb; ++b)
+      if (q.table[b] < 0) ++total;
+  }
+  if (total > s->staging_cap) return E_STAGING;
+  const uint64_t bb = s->block_bytes;
+  const uint64_t lent_layer = static_cast<uint64_t>(s->lent_phys) * bb;
+  const uint64_t slot_bytes = static_cast<uint64_t>(s->staging_cap) * bb;
+  const uint32_t slot = layer % s->ring_slots;
+  uint32_t k = 0;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    const Seq& q = s->seqs[seqs[i]];
+    uint32_t nb = blocks_for(q.len, s->block_tokens);
+    for (uint32_t b = 0; b < nb; ++b) {
+      int32_t e = q.table[b];
+      int32_t r;
+      if (e >= 0) {
+        r = e;
+      } else {
+        if (lent_arena && staging) {
+          const uint8_t* src = lent_arena + layer * lent_layer + static_cast<uint64_t>(~e) * bb;
+          uint8_t* dst = staging + slot * slot_bytes + static_cast<uint64_t>(k) * bb;
+          std::memcpy(dst, src, bb);
+        }
+        r = ~static_cast<int32_t>(k);
+        ++k;
+      }
+      if (resolved) resolved[static_cast<uint64_t>(i) * s->max_blocks_per_seq + b] = r;
+    }
+  }
+  if (k_out) *k_out = k;
+  return OK;
+}
+
+// The way back: every staged block of the batch is written to its home in the lent arena.
+int oracle_scatter(void* h, uint32_t layer, const int32_t* seqs, uint32_t nseq,
+                   const uint8_t* staging, uint8_t* lent_arena) {
+  State* s = static_cast<State*>(h);
+  if (layer >= s->num_layers) return E_INVAL;
+  const uint64_t bb = s->block_bytes;
+  const uint64_t lent_layer = static_cast<uint64_t>(s->lent_phys) * bb;
+  const uint64_t slot_bytes = static_cast<uint64_t>(s->staging_cap) * bb;
+  const uint32_t slot = layer % s->ring_slots;
+  uint32_t k = 0;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    auto it = s->seqs.find(seqs[i]);
+    if (it == s->seqs.end()) return E_STATE;
+    const Seq& q = it->second;
+    uint32_t nb = blocks_for(q.len, s->block_tokens);
+    for (uint32_t b = 0; b < nb; ++b) {
+      int32_t e = q.table[b];
+      if (e >= 0) continue;
+      std::memcpy(lent_arena + layer * lent_layer + static_cast<uint64_t>(~e) * bb,
+                  staging + slot * slot_bytes + static_cast<uint64_t>(k) * bb, bb);
+      ++k;
+    }
+  }
+  return OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// O-attn: decode attention read through resolved tables, fp64.
+//   q        [nseq][Hq][D] bf16 bit patterns
+//   local    base of this layer's local arena  [id][2][T][Hkv][D] bf16
+//   staging  base of this layer's ring slot    [pos][2][T][Hkv][D] bf16
+//   resolved [nseq][table_stride] ; lens [nseq]
+//   out      [nseq][Hq][D] double ; lse [nseq][Hq] double (may be NULL)
+// Tokens t >= len are excluded, not multiplied by zero.
+// ------------------------------------------------------------------------------------------
+int oracle_paged_attention(const uint16_t* q, const uint16_t* local, const uint16_t* staging,
+                           const int32_t* resolved, uint32_t table_stride, const uint32_t* lens,
+                           uint32_t nseq, uint32_t Hq, uint32_t Hkv, uint32_t D, uint32_t T,
+                           double sm_scale, double* out, double* lse) {
+  if (Hkv == 0 || Hq % Hkv != 0) return E_INVAL;
+  for (uint32_t i = 0; i < nseq; ++i)
+    if (lens[i] == 0) return E_INVAL;
+  const uint32_t G = Hq / Hkv;
+  const uint64_t plane = static_cast<uint64_t>(T) * Hkv * D;  // elements
+  const uint64_t block_elems = 2 * plane;
+  const int64_t npairs = static_cast<int64_t>(nseq) * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t pair = 0; pair < npairs; ++pair) {
+    const uint32_t i = static_cast<uint32_t>(pair / Hq);
+    const uint32_t hq = static_cast<uint32_t>(pair % Hq);
+    const uint32_t g = hq / G;
+    const uint32_t n = lens[i];
+    const uint16_t* qv = q + (static_cast<uint64_t>(i) * Hq + hq) * D;
+    std::vector<double> sc(n);
+    double m = -std::numeric_limits<double>::infinity();
+    for (uint32_t t = 0; t < n; ++t) {
+      int32_t e = resolved[static_cast<uint64_t>(i) * table_stride + t / T];
+      const uint16_t* blk = e >= 0 ? local + static_cast<uint64_t>(e) * block_elems
+                                   : staging + static_cast<uint64_t>(~e) * block_elems;
+      const uint16_t* krow = blk + (static_cast<uint64_t>(t % T) * Hkv + g) * D;
+      double acc = 0.0;
+      for (uint32_t d = 0; d < D; ++d) acc += bf16_to_double(qv[d]) * bf16_to_double(krow[d]);
+      sc[t] = sm_scale * acc;
+      if (sc[t] > m) m = sc[t];
+    }
+    double l = 0.0;
+    std::vector<double> o(D, 0.0);
+    for (uint32_t t = 0; t < n; ++t) {
+      int32_t e = resolved[static_cast<uint64_t>(i) * table_stride + t / T];
+      const uint16_t* blk = e >= 0 ? local + static_cast<uint64_t>(e) * block_elems
+                                   : staging + static_cast<uint64_t>(~e) * block_elems;
+      const uint16_t* vrow = blk + plane + (static_cast<uint64_t>(t % T) * Hkv + g) * D;
+      double p = std::exp(sc[t] - m);
+      l += p;
+      for (uint32_t d = 0; d < D; ++d) o[d] += p * bf16_to_double(vrow[d]);
+    }
+    double* od = out + (static_cast<uint64_t>(i) * Hq + hq) * D;
+    for (uint32_t d = 0; d < D; ++d) od[d] = o[d] / l;
+    if (lse) lse[static_cast<uint64_t>(i) * Hq + hq] = m + std::log(l);
+  }
+  return OK;
+}
+
+// Brute force on a dense, contiguous cache: K, V are [n][Hkv][D] bf16 for ONE sequence.
+// Also returns the normalised probabilities (probs [Hq][n], may be NULL) for the row-sum pin.
+int oracle_dense_attention(const uint16_t* q, const uint16_t* K, const uint16_t* V, uint32_t n,
+                           uint32_t Hq, uint32_t Hkv, uint32_t D, double sm_scale, double* out,
+                           double* lse, double* probs) {
+  if (n == 0 || Hkv == 0 || Hq % Hkv != 0) return E_INVAL;
+  const uint32_t G = Hq / Hkv;
+  for (uint32_t hq = 0; hq < Hq; ++hq) {
+    const uint32_t g = hq / G;
+    std::vector<double> sc(n);
+    double m = -std::numeric_limits<double>::infinity();
+    for (uint32_t t = 0; t < n; ++t) {
+      const uint16_t* krow = K + (static_cast<uint64_t>(t) * Hkv + g) * D;
+      double acc = 0.0;
+      for (uint32_t d = 0; d < D; ++d) acc += bf16_to_double(q[hq * D + d]) * bf16_to_double(krow[d]);
+      sc[t] = sm_scale * acc;
+      m = std::max(m, sc[t]);
+    }
+    double l = 0.0;
+    std::vector<double> o(D, 0.0);
+    for (uint32_t t = 0; t < n; ++t) {
+      const uint16_t* vrow = V + (static_cast<uint64_t>(t) * Hkv + g) * D;
+      double p = std::exp(sc[t] - m);
+      l += p;
+      for (uint32_t d = 0; d < D; ++d) o[d] += p * bf16_to_double(vrow[d]);
+    }
+    for (uint32_t d = 0; d < D; ++d) out[static_cast<uint64_t>(hq) * D + d] = o[d] / l;
+    if (lse) lse[hq] = m + std::log(l);
+    if (probs)
+      for (uint32_t t = 0; t < n; ++t) probs[static_cast<uint64_t>(hq) * n + t] = std::exp(sc[t] - m) / l;
+  }
+  return OK;
+}
+
+// Elementwise double -> bf16 (round to nearest even), for reporting.
+void oracle_to_bf16(const double* x, uint16_t* y, uint64_t n) {
+  for (uint64_t k = 0; k < n; ++k) y[k] = double_to_bf16_rne(x[k]);
+}
+
+// ------------------------------------------------------------------------------------------
+// O-reclaim: the lender takes the top `take` ids of the lent range; in-use blocks there move,
+// for every layer, to free local ids first and then to the smallest free lent id below the cut.
+// Arenas may be NULL (integer state only).
+// ------------------------------------------------------------------------------------------
+int oracle_reclaim(void* h, uint32_t take, uint8_t* local_arena, uint8_t* lent_arena,
+                   uint64_t* out_migrated) {
+  State* s = static_cast<State*>(h);
+  if (take > s->lent_cap) take = s->lent_cap;
+  const uint32_t cut = s->lent_cap - take;
+  std::vector<int32_t> victims;
+  for (uint32_t id = cut; id < s->lent_cap; ++id)
+    if (s->owner_lent[id].seq >= 0) victims.push_back(static_cast<int32_t>(id));
+  size_t free_below = 0;
+  for (int32_t id : s->free_lent)
+    if (static_cast<uint32_t>(id) < cut) ++free_below;
+  if (victims.size() > s->free_local.size() + free_below) return E_NOSPC;
+  // Free ids at or above the cut leave the stack; the others keep their relative order.
+  std::vector<int32_t> kept;
+  for (int32_t id : s->free_lent)
+    if (static_cast<uint32_t>(id) < cut) kept.push_back(id);
+  s->free_lent.swap(kept);
+  const uint64_t bb = s->block_bytes;
+  const uint64_t local_layer = static_cast<uint64_t>(s->local_blocks) * bb;
+  const uint64_t lent_layer = static_cast<uint64_t>(s->lent_phys) * bb;
+  for (int32_t v : victims) {
+    Owner own = s->owner_lent[v];
+    bool to_local = !s->free_local.empty();
+    int32_t dst;
+    if (to_local) {
+      dst = s->free_local.back();
+      s->free_local.pop_back();
+    } else {
+      auto mn = std::min_element(s->free_lent.begin(), s->free_lent.end());
+      dst = *mn;
+      s->free_lent.erase(mn);
+    }
+    if (local_arena && lent_arena) {
+      for (uint32_t l = 0; l < s->num_layers; ++l) {
+        const uint8_t* src = lent_arena + l * lent_layer + static_cast<uint64_t>(v) * bb;
+        uint8_t* d = to_local ? local_arena + l * local_layer + static_cast<uint64_t>(dst) * bb
+                              : lent_arena + l * lent_layer + static_cast<uint64_t>(dst) * bb;
+        std::memcpy(d, src, bb);
+      }
+    }
+    s->seqs[own.seq].table[own.logical] = to_local ? dst : ~dst;
+    if (to_local) s->owner_local[dst] = own; else s->owner_lent[dst] = own;
+    s->owner_lent[v] = Owner();
+  }
+  s->lent_cap = cut;
+  if (out_migrated) *out_migrated = victims.size();
+  return OK;
+}
+
+// The lender offers n more block ids: capacity grows, new ids pop in ascending order.
+int oracle_lend(void* h, uint32_t n) {
+  State* s = static_cast<State*>(h);
+  if (static_cast<uint64_t>(s->lent_cap) + n > s->lent_phys) return E_INVAL;
+  for (uint32_t k = n; k-- > 0;) s->free_lent.push_back(static_cast<int32_t>(s->lent_cap + k));
+  s->lent_cap += n;
+  return OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// O-append: token (len-1) of each sequence gets its K and V rows ([nseq][Hkv][D] bf16 each).
+// staging_slot, when not NULL, is the ring slot that currently holds `layer` for this batch:
+// rows whose home block is lent are written there too (position taken from the canonical order).
+// ------------------------------------------------------------------------------------------
+int oracle_append_kv(void* h, uint32_t layer, const int32_t* seqs, uint32_t nseq,
+                     const uint16_t* k_new, const uint16_t* v_new, uint32_t Hkv, uint32_t D,
+                     uint8_t* local_arena, uint8_t* lent_arena, uint8_t* staging_slot) {
+  State* s = static_cast<State*>(h);
+  if (layer >= s->num_layers) return E_INVAL;
+  const uint64_t bb = s->block_bytes;
+  const uint64_t row = static_cast<uint64_t>(Hkv) * D * 2;  // bytes of one token's K (or V) row
+  const uint64_t plane = static_cast<uint64_t>(s->block_tokens) * row;
+  if (2 * plane != bb) return E_INVAL;
+  const uint64_t local_layer = static_cast<uint64_t>(s->local_blocks) * bb;
+  const uint64_t lent_layer = static_cast<uint64_t>(s->lent_phys) * bb;
+  uint32_t k = 0;  // staging position counter, canonical order
+  for (uint32_t i = 0; i < nseq; ++i) {
+    auto it = s->seqs.find(seqs[i]);
+    if (it == s->seqs.end()) return E_STATE;
+    const Seq& q = it->second;
+    if (q.len == 0) return E_INVAL;
+    const uint32_t nb = blocks_for(q.len, s->block_tokens);
+    const uint32_t t = q.len - 1, b = t / s->block_tokens, r = t % s->block_tokens;
+    const uint8_t* ks = reinterpret_cast<const uint8_t*>(k_new) + i * row;
+    const uint8_t* vs = reinterpret_cast<const uint8_t*>(v_new) + i * row;
+    for (uint32_t bi = 0; bi < nb; ++bi) {
+      int32_t e = q.table[bi];
+      if (bi == b) {
+        uint8_t* home = e >= 0 ? local_arena + layer * local_layer + static_cast<uint64_t>(e) * bb
+                               : lent_arena + layer * lent_layer + static_cast<uint64_t>(~e) * bb;
+        std::memcpy(home + r * row, ks, row);
+        std::memcpy(home + plane + r * row, vs, row);
+        if (e < 0 && staging_slot) {
+          uint8_t* st = staging_slot + static_cast<uint64_t>(k) * bb;
+          std::memcpy(st + r * row, ks, row);
+          std::memcpy(st + plane + r * row, vs, row);
+        }
+      }
+      if (e < 0) ++k;
+    }
+  }
+  return OK;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+}  // extern "C"
