@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the memory-slice hot path: per-layer prefetch of lent KV blocks overlapped with
+paged GQA decode attention, on synthetic Llama-3-8B-shaped decode batches.
+
+    python bench.py --gpus N --steps K --warmup W            (one process per GPU under torchrun)
+    python bench.py --impl reference ...                      (the CPU oracle, timed as it stands)
+
+A step is one pass of the whole path over one batch: for every layer, the gather of that layer's
+lent blocks into the staging ring and the attention over the local arena plus the ring slot. The
+metric is decode tokens/s = sequences * steps / time. One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_27040_b200 import synth  # noqa: E402
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3_8b_decode", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--copy-kind", type=int, default=0)
+    ap.add_argument("--copy-ctas", type=int, default=0)
+    ap.add_argument("--decode-ctas", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (debugging)")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# Workload construction (device)
+# ---------------------------------------------------------------------------------------------
+class DeviceWorkload:
+    """Arenas, tables and query tensors of one workload on the current CUDA device."""
+
+    def __init__(self, wl: synth.Workload, seed: int, flags: int = 0, copy_kind: int = 0, copy_ctas: int = 0,
+                 decode_ctas: int = 0):
+        import torch
+        from paper_2609_27040_b200 import binding as B
+        self.wl, self.B = wl, B
+        self.pl = pl = synth.make_placement(wl, seed, slack_blocks=64)
+        shape = (2, wl.block_tokens, wl.num_kv_heads, wl.head_dim)
+        need = (wl.num_layers * (pl.local_blocks + pl.lent_blocks) + wl.ring_slots * pl.staging_blocks) * wl.block_bytes
+        free, _ = torch.cuda.mem_get_info()
+        if need > 0.92 * free:
+            raise RuntimeError(f"workload needs {need / 2**30:.1f} GiB, device has {free / 2**30:.1f} GiB free")
+        gen = torch.Generator(device="cuda").manual_seed(seed)
+        bf = torch.bfloat16
+        self.local = torch.empty((wl.num_layers, pl.local_blocks) + shape, device="cuda", dtype=bf)
+        self.lent = torch.empty((wl.num_layers, pl.lent_blocks) + shape, device="cuda", dtype=bf)
+        for l in range(wl.num_layers):          # N(0,1) bf16 KV, layer by layer
+            self.local[l].normal_(generator=gen)
+            self.lent[l].normal_(generator=gen)
+        self.staging = torch.zeros((wl.ring_slots, pl.staging_blocks) + shape, device="cuda", dtype=bf)
+        self.q = torch.empty((wl.num_layers, wl.batch, wl.num_q_heads, wl.head_dim), device="cuda", dtype=bf)
+        self.q.normal_(generator=gen)
+        self.out = torch.zeros_like(self.q)
+        self.main = torch.cuda.Stream()
+        self.side = torch.cuda.Stream(priority=-1)
+        torch.cuda.synchronize()
+        self.max_blocks = int(max(len(h) for h in pl.hints)) + 4
+        self.s = B.Slice(wl.num_layers, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks,
+                         local=self.local, lent=self.lent, staging=self.staging, ring_slots=wl.ring_slots,
+                         max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks, flags=flags,
+                         local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order,
+                         copy_kind=copy_kind, copy_ctas=copy_ctas, decode_ctas=decode_ctas)
+        t0 = time.perf_counter()
+        for i, hints in enumerate(pl.hints):
+            for h in hints:
+                rc, _ = self.s.slice_alloc_blocks(i, 1, int(h))
+                assert rc == 0, rc
+            assert self.s.slice_set_seq_len(i, int(pl.lengths[i])) == 0
+        self.alloc_s = time.perf_counter() - t0
+        self.seqs = np.arange(wl.batch, dtype=np.int32)
+        self.scale = 1.0 / float(np.sqrt(wl.head_dim))
+        # algorithmic bytes
+        self.tokens = int(pl.lengths.sum())
+        self.attn_bytes_layer = (self.tokens * wl.kv_bytes_per_token + 2 * wl.batch * wl.num_q_heads * wl.head_dim * 2
+                                 + 4 * pl.total_blocks)
+        self.pref_bytes_layer = 2 * pl.staging_blocks * wl.block_bytes + 4 * pl.staging_blocks
+        self.step_bytes = wl.num_layers * (self.attn_bytes_layer + self.pref_bytes_layer)
+
+    def step(self, wrap=True, host_io=None):
+        if host_io is None:
+            rc = self.s.slice_decode_step(self.seqs, self.q, self.wl.num_q_heads, self.scale, self.out, False, wrap,
+                                          self.main, self.side)
+        else:
+            qh, oh = host_io
+            rc = self.s.slice_decode_step(self.seqs, qh, self.wl.num_q_heads, self.scale, oh, True, wrap,
+                                          self.main, self.side)
+        if rc != 0:
+            raise RuntimeError(f"slice_decode_step: {self.B.slice_strerror(rc)}")
+
+    def timed(self, steps, wrap=True, host_io=None):
+        """K steps between CUDA events on the launching stream; both streams are joined at the end."""
+        import torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(self.main)
+        for _ in range(steps):
+            self.step(wrap, host_io)
+        self.main.wait_stream(self.side)
+        e1.record(self.main)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3
+
+
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed regions run."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", uuid], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL,
+                                         text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+def oracle_layer_sample(wl: synth.Workload, seed: int, nseq: int, repeats: int):
+    """Times the oracle (gather + fp64 paged attention) on one layer of the first `nseq` sequences
+    of the workload, host data drawn with the same placement rule. Returns (seconds per repeat,
+    sample tokens, threads)."""
+    import oracle
+    pl = synth.make_placement(wl, seed, slack_blocks=64)
+    sub = list(range(min(nseq, wl.batch)))
+    n_local = sum(int((pl.hints[i] == synth.LOCAL).sum()) for i in sub)
+    n_lent = sum(int((pl.hints[i] == synth.LENT).sum()) for i in sub)
+    max_blocks = int(max(len(pl.hints[i]) for i in sub)) + 1
+    orc = oracle.OracleSlice(1, wl.block_tokens, wl.block_bytes, n_local, n_lent, n_lent, 1, max(n_lent, 1),
+                             max_seqs=len(sub), max_blocks_per_seq=max_blocks)
+    for i in sub:
+        for h in pl.hints[i]:
+            assert orc.alloc_blocks(i, 1, int(h))[0] == 0
+        assert orc.set_seq_len(i, int(pl.lengths[i])) == 0
+    rng = np.random.default_rng(seed)
+    shape = (2, wl.block_tokens, wl.num_kv_heads, wl.head_dim)
+    local = synth.normal_bf16_bits(rng, (1, n_local) + shape)
+    lent = synth.normal_bf16_bits(rng, (1, max(n_lent, 1)) + shape)
+    staging = np.zeros((1, max(n_lent, 1)) + shape, np.uint16)
+    q = synth.normal_bf16_bits(rng, (len(sub), wl.num_q_heads, wl.head_dim))
+    lens = np.asarray([pl.lengths[i] for i in sub], np.uint32)
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        rc, resolved, k = orc.gather(0, sub, lent, staging)
+        assert rc == 0
+        rc, out, _ = oracle.paged_attention(q, local[0], staging[0], resolved, lens, wl.num_q_heads, wl.num_kv_heads,
+                                            wl.head_dim, wl.block_tokens, 1.0 / np.sqrt(wl.head_dim), want_lse=False)
+        assert rc == 0
+        times.append(time.perf_counter() - t0)
+    return times, int(lens.sum()), oracle.num_threads()
+
+
+def oracle_tokens_per_s(wl, seconds_per_layer_sample, sample_tokens, total_tokens):
+    """Scales one sampled layer to a full step: time grows with tokens and with layers."""
+    step_s = seconds_per_layer_sample * (total_tokens / sample_tokens) * wl.num_layers
+    return wl.batch / step_s
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    nseq = min(8, wl.batch)
+    pl = synth.make_placement(wl, args.seed, slack_blocks=64)
+    total_tokens = int(pl.lengths.sum())
+    times, sample_tokens, threads = oracle_layer_sample(wl, args.seed, nseq, args.warmup + args.steps)
+    timed = times[args.warmup:]
+    per = sum(timed) / len(timed)
+    value = oracle_tokens_per_s(wl, per, sample_tokens, total_tokens)
+    sample = (f"each step = oracle gather + fp64 paged attention of 1 layer over the first {nseq} of {wl.batch} "
+              f"sequences ({sample_tokens} of {total_tokens} tokens), scaled by tokens and by {wl.num_layers} layers")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": per * (total_tokens / sample_tokens) * wl.num_layers * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.num_layers, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_27040_b200 import binding as B
+    from paper_2609_27040_b200 import build as build_mod
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build_mod.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    # Replicas only: every rank runs the same workload shape on its own GPU with its own seed.
+    w = DeviceWorkload(wl, args.seed + rank, copy_kind=args.copy_kind, copy_ctas=args.copy_ctas,
+                       decode_ctas=args.decode_ctas)
+    wrap = not args.no_wrap
+    for _ in range(max(args.warmup, 3)):
+        w.step(wrap)
+    torch.cuda.synchronize()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid).replace("GPU-", ""))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: device-resident inputs ----
+    st0 = w.s.slice_stats()
+    barrier()
+    t = w.timed(args.steps, wrap)
+    barrier()
+    st1 = w.s.slice_stats()
+    launches = st1["kernel_launches"] - st0["kernel_launches"]
+
+    # ---- end to end: pinned host q in, out back, every step ----
+    qh = w.q.cpu().pin_memory()
+    oh = torch.zeros_like(qh).pin_memory()
+    for _ in range(3):
+        w.step(wrap, (qh, oh))
+    barrier()
+    e2e_steps = max(3, min(args.steps, 50))
+    t_e2e = w.timed(e2e_steps, wrap, (qh, oh))
+    barrier()
+    io_bytes = qh.numel() * qh.element_size()
+
+    if world > 1:
+        tt = torch.tensor([t, t_e2e / e2e_steps], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t, t_e2e_step = float(tt[0]), float(tt[1])
+        ll = torch.tensor([launches], device="cuda", dtype=torch.int64)
+        dist.all_reduce(ll)
+        launches = int(ll[0])
+    else:
+        t_e2e_step = t_e2e / e2e_steps
+
+    # ---- per-layer kernel times inside the pipelined pass (profile events), rank 0 ----
+    roof = None
+    extra = {}
+    if rank == 0:
+        del w
+        torch.cuda.empty_cache()
+        wp = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, copy_kind=args.copy_kind, copy_ctas=args.copy_ctas,
+                            decode_ctas=args.decode_ctas)
+        for _ in range(3):
+            wp.step(wrap)
+        attn_us, pref_us, stall_us, layer_us = [], [], [], []
+        for _ in range(max(3, min(args.steps, 20))):
+            wp.step(wrap)
+            tm = wp.s.slice_layer_times().astype(np.float64)     # synchronises
+            attn_us.append(tm[:, 4] - tm[:, 2])                  # attention kernel proper
+            pref_us.append(tm[:, 1] - tm[:, 0])
+            prev_end = np.concatenate(([tm[0, 2]], tm[:-1, 3]))  # end of the previous layer's attention
+            stall_us.append(np.maximum(0.0, tm[:, 1] - prev_end))
+            layer_us.append(tm[:, 3] - prev_end)
+        attn = float(np.nanmean(np.stack(attn_us)))
+        pref = float(np.nanmean(np.stack(pref_us)))
+        stall = float(np.nanmean(np.stack(stall_us)[:, 1:]))
+        layer = float(np.nanmean(np.stack(layer_us)[:, 1:]))
+        peak, peak_src = measured_peaks()
+        achieved = wp.attn_bytes_layer / (attn * 1e-6) / 1e9
+        combined = wp.step_bytes * args.steps / t / 1e9
+        roof = {"bound": "hbm", "kernel": "paged_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": f"of {peak_src}",
+                "note": "attention kernel timed inside the pipelined pass, where the concurrent gather takes its "
+                        "share of HBM; 'combined' counts attention + gather bytes over the step time",
+                "combined": {"achieved": combined, "frac": combined / peak, "frac_of_nominal_8TBs": combined / NOMINAL_HBM_GBS},
+                "algorithmic_bytes_per_launch": wp.attn_bytes_layer}
+        extra = {"attn_us_per_layer": attn, "prefetch_us_per_layer": pref, "stall_us_per_layer": stall,
+                 "layer_us": layer, "stall_frac_of_attention": stall / attn if attn else None,
+                 "alloc_seconds_setup": wp.alloc_s}
+        # attention alone (no concurrent gather): the kernel's own roofline
+        for _ in range(2):
+            wp.step(False)
+        iso = []
+        for l in range(wl.num_layers):
+            assert wp.s.prefetch_layer(l, wp.seqs, wp.side) == 0
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(wp.main)
+            assert wp.s.paged_decode(l, wp.seqs, wp.q[l], wl.num_q_heads, wp.scale, wp.out[l], None, wp.main) == 0
+            e1.record(wp.main)
+            torch.cuda.synchronize()
+            iso.append(e0.elapsed_time(e1) * 1e3)
+        iso_us = float(np.mean(iso[1:] if len(iso) > 1 else iso))
+        roof["isolated"] = {"achieved": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9, "us_per_layer": iso_us,
+                            "frac": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak,
+                            "includes": "attention kernel + merge kernel, no concurrent gather"}
+        step_bytes, tokens, pl_blocks, k_blocks = wp.step_bytes, wp.tokens, wp.pl.total_blocks, wp.pl.staging_blocks
+        del wp
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        oracle.build()
+        nseq = wl.batch
+        times, sample_tokens, threads = oracle_layer_sample(wl, args.seed, nseq, 3)
+        per = min(times)
+        cpu = {"value": oracle_tokens_per_s(wl, per, sample_tokens, tokens), "unit": UNIT, "cores": threads,
+               "kind": "oracle",
+               "sample": f"oracle gather + fp64 paged attention of 1 layer over the first {nseq} of {wl.batch} sequences "
+                         f"({sample_tokens} of {tokens} tokens, best of 3), scaled by tokens and by {wl.num_layers} layers"}
+
+    value = wl.batch * world * args.steps / t
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": t / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.num_layers, "q_heads": wl.num_q_heads,
+                   "kv_heads": wl.num_kv_heads, "head_dim": wl.head_dim, "block_tokens": wl.block_tokens,
+                   "len_range": [wl.len_lo, wl.len_hi], "lent_fraction": wl.lent_fraction, "ring_slots": wl.ring_slots,
+                   "tokens_in_batch": tokens, "blocks": pl_blocks, "lent_blocks": k_blocks,
+                   "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "inputs larger than L2: every step streams %.1f GB of KV" % (step_bytes / 1e9)},
+        "hbm_gbs_combined": step_bytes * world * args.steps / t / 1e9,
+        "roofline": roof, "cpu_baseline": cpu,
+        "e2e": {"value": wl.batch * world / t_e2e_step, "unit": UNIT, "h2d_bytes_per_step": io_bytes,
+                "d2h_bytes_per_step": io_bytes, "ms_per_step": t_e2e_step * 1e3},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    line.update(extra)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.layers or args.batch:
+        import dataclasses
+        wl = dataclasses.replace(wl, num_layers=args.layers or wl.num_layers, batch=args.batch or wl.batch)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,217 @@
+/* emaslice.h — C ABI of libemaslice.so: the memory-slice hot path on one B200 (sm_100a).
+ *
+ * A memory slice (paper, Section 4) is a segment shared by two GPUs; a user's data may sit in its
+ * own part ("local") or in the part the peer contributed ("lent"). Before a layer runs, the slice
+ * side prepares a directly accessible address and prefetches the data (Section 5.1), inside the
+ * latency window between two uses of the same layer (Section 2.3); the lender can take its memory
+ * back at any time (Section 4.1). On one GPU the lent part is a separate arena that only the
+ * prefetch, write-back, append and reclaim kernels touch; attention reads the local arena and the
+ * staging ring only.
+ *
+ * Conventions
+ *   - No exception, abort or print crosses this boundary. Every call returns a status code
+ *     (0 = OK, negative = error, see slice_strerror). A failing call leaves tables, free lists and
+ *     capacities unchanged.
+ *   - "device pointer": memory the GPU can address (HBM; for the lent arena optionally mapped
+ *     pinned host memory). "host pointer": ordinary host memory. The caller owns every buffer it
+ *     passes; arenas and staging must outlive the slice and be 256-byte aligned.
+ *   - Streams are cudaStream_t values passed as void*. prefetch_layer, paged_decode,
+ *     slice_append_kv, slice_writeback_layer and slice_reclaim enqueue work and return; the
+ *     library orders them with its own events (attention of a layer waits for that layer's
+ *     prefetch; a prefetch into a ring slot waits for the attention that last read the slot;
+ *     reclaim waits for everything outstanding and invalidates what is staged).
+ *   - One caller thread per slice.
+ *
+ * Data layout
+ *   block      = K plane [block_tokens][num_kv_heads][head_dim] bf16, then the V plane of the
+ *                same shape: 2*16*8*128*2 = 65 536 bytes for the shapes used here.
+ *   arena      = [layer][block id][block]; byte address = base + layer*layer_stride
+ *                + id*block_stride (strides 0 select the dense default).
+ *   staging    = [ring slot][position][block], dense.
+ *   table entry (int32): e >= 0 is local id e; e < 0 is lent id ~e. Block ids are the same for
+ *                every layer (Section 4.2.1: allocation "applied uniformly across all layers").
+ *   resolved entry (int32): e >= 0 is local id e; e < 0 is staging position ~e.
+ *   Supported shapes: head_dim 128, block_tokens 16, num_kv_heads 1..8, bf16,
+ *   num_q_heads = G * num_kv_heads with G in 1..8.
+ */
+#ifndef EMASLICE_H_
+#define EMASLICE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ema_slice slice_t; /* opaque; the library owns metadata, events and work lists */
+
+enum {
+  SLICE_OK = 0,
+  SLICE_EINVAL = -1,   /* bad id, shape, pointer or argument                                   */
+  SLICE_ENOSPC = -2,   /* not enough free blocks: capacity beyond the local part is not
+                          guaranteed (Section 5.1); the caller preempts and retries             */
+  SLICE_ESTAGING = -3, /* the batch's lent blocks exceed a ring slot                            */
+  SLICE_ESTALE = -4,   /* paged_decode of a layer whose prefetch for this batch is not valid     */
+  SLICE_ECUDA = -5,    /* a CUDA call failed; slice_stats reports the code                       */
+  SLICE_ETIMEOUT = -6, /* a bounded device-side wait expired (reported through slice_stats)      */
+  SLICE_ESTATE = -7    /* unknown sequence, double free                                          */
+};
+
+enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
+
+enum {
+  SLICE_FLAG_PROFILE = 1u,     /* record timing events per layer (slice_layer_times)            */
+  SLICE_FLAG_NULL_DEVICE = 4u  /* tables only: no CUDA call is made, no kernel is launched       */
+};
+
+typedef struct {
+  uint32_t num_layers, num_kv_heads, head_dim, block_tokens;
+  uint32_t dtype;                 /* 0 = bf16 */
+  uint32_t local_blocks;          /* local capacity in block ids                                 */
+  uint32_t lent_blocks;           /* lent capacity now; changes with slice_reclaim / slice_lend  */
+  uint32_t lent_blocks_physical;  /* size of the lent arena in block ids (>= lent_blocks)        */
+  uint32_t ring_slots;            /* staging ring depth R >= 1; layer l uses slot l mod R        */
+  uint32_t staging_blocks_per_slot;
+  uint32_t max_seqs, max_blocks_per_seq;
+  uint32_t lent_kind;             /* 0 = device HBM arena, 1 = mapped pinned-host arena          */
+  uint32_t flags;                 /* SLICE_FLAG_*                                                */
+  void* local_base;               /* device pointers, caller-owned (may be NULL with NULL_DEVICE) */
+  void* lent_base;
+  void* staging_base;
+  uint64_t local_layer_stride, local_block_stride; /* bytes; 0 = dense                          */
+  uint64_t lent_layer_stride, lent_block_stride;
+  const uint32_t* local_free_order; /* host; optional pop order of local ids (a permutation of
+                                       0..local_blocks-1); NULL = ascending                      */
+  const uint32_t* lent_free_order;  /* host; optional permutation of 0..lent_blocks_physical-1;
+                                       ids >= lent_blocks are skipped at creation                */
+  uint32_t decode_ctas;           /* 0 = one per SM; CTAs of the attention kernel                */
+  uint32_t copy_ctas;             /* 0 = default; CTAs of the gather / migration kernel          */
+  uint32_t copy_kind;             /* 0 = default, 1 = vector load/store kernel, 2 = bulk-copy ring */
+  uint32_t reserved;
+} slice_config_t;
+
+typedef struct {
+  uint32_t local_used, local_free, lent_used, lent_free, lent_capacity, num_seqs;
+  uint64_t prefetch_calls, prefetched_blocks, prefetched_bytes;
+  uint64_t decode_calls, decode_tokens;
+  uint64_t reclaims, migrated_blocks, migrated_bytes;
+  uint64_t plans_built;          /* how often tables were re-resolved for a batch               */
+  uint64_t kernel_launches;      /* kernels of this library launched so far                     */
+  int32_t last_cuda_error;       /* cudaError_t of the last failed CUDA call, 0 if none         */
+  int32_t device_status;         /* 0, or SLICE_ETIMEOUT if a kernel gave up a bounded wait
+                                    (read back by slice_stats; the call synchronises nothing)   */
+} slice_stats_t;
+
+/* Section 4 (memory slice with a mapping table per user). Creates the allocator state and the
+ * device-side work lists. cfg and the free orders are host pointers, read during the call only.
+ * out receives the handle. Errors: EINVAL (shape unsupported, NULL arena without NULL_DEVICE,
+ * lent_blocks > lent_blocks_physical, ring_slots == 0), ECUDA. */
+int slice_create(const slice_config_t* cfg, slice_t** out);
+
+/* Frees what slice_create made after waiting for the slice's outstanding work. */
+int slice_destroy(slice_t* s);
+
+/* Section 4.1: "first attempts to allocate from free memory" — appends n logical blocks to
+ * sequence seq (created when absent). AUTO takes free local ids first and the lent part only when
+ * local memory is exhausted; LOCAL / LENT force a tier (seeded placements). out_entries (host, n
+ * entries, may be NULL) receives the new table entries. Errors: ENOSPC (nothing changes), EINVAL
+ * (negative seq, bad hint, more than max_seqs sequences or max_blocks_per_seq blocks). */
+int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t tier_hint, int32_t* out_entries);
+
+/* Sets the number of valid tokens of seq; len <= block_tokens * allocated blocks.
+ * Errors: ESTATE (unknown seq), EINVAL. */
+int slice_set_seq_len(slice_t* s, int32_t seq, uint32_t len);
+
+/* Completion or preemption of a request (Section 4.1): its blocks return to the free lists, in
+ * descending logical order. Errors: ESTATE. */
+int slice_free_seq(slice_t* s, int32_t seq);
+
+/* Copies the block table of seq to out (host, cap entries; may be NULL to query). n and len
+ * (host, may be NULL) receive the number of blocks and tokens. Errors: ESTATE, EINVAL (cap). */
+int slice_get_block_table(slice_t* s, int32_t seq, int32_t* out, uint32_t cap, uint32_t* n, uint32_t* len);
+
+/* Test hook: free list of a tier (1 local, 2 lent) in pop order. */
+int slice_get_free_stack(slice_t* s, int32_t tier, int32_t* out, uint32_t cap, uint32_t* n);
+
+/* Sections 2.3, 4.2.1, 5.1: prefetch before use. For layer `layer` and the batch seqs[0..nseq)
+ * (host array of distinct sequence ids), every in-use lent block is copied, in batch order then
+ * logical order, from the lent arena into ring slot (layer mod R) at consecutive positions; the
+ * batch's resolved table maps each lent block to its position. Enqueued on side_stream after the
+ * attention that last read the slot. Errors: EINVAL, ESTATE, ESTAGING (before any copy), ECUDA. */
+int prefetch_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* side_stream);
+
+/* The consumer of the prepared addresses (Section 5.1); the paper takes the attention kernel from
+ * its serving engine (Section 6.1) and does not define it. Computes, for each sequence i of the
+ * batch and query head h (KV head h / G): out = softmax(sm_scale * q K^T) V over tokens
+ * 0..len-1, read through the resolved table from the local arena and the ring slot of `layer`.
+ *   q, out  device, [nseq][num_q_heads][128] bf16;  lse_or_null device, [nseq][num_q_heads] f32
+ *           (natural-log sum of exponentials of the scaled scores).
+ * Arithmetic: bf16 products, f32 accumulation and softmax, bf16 result (nearest even).
+ * Enqueued on stream after the layer's prefetch. Errors: EINVAL (shape, zero-length sequence,
+ * G > 8), ESTATE, ESTALE (batch has lent blocks and the slot does not hold a valid prefetch of
+ * this layer for this batch and table state), ECUDA. */
+int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
+                 uint32_t num_q_heads, float sm_scale, void* out, float* lse_or_null, void* stream);
+
+/* Section 4.1: the lender regains capacity immediately. The paper reclaims by preempting the
+ * borrower's requests; this entry migrates instead. The top `take_blocks` ids of the lent range
+ * (UINT32_MAX = all) leave the slice; in-use blocks there move, for every layer, to free local ids
+ * first and then to the smallest free lent ids below the cut; tables and free lists are rewritten
+ * and everything staged becomes invalid. out_n_migrated (host, may be NULL) receives the number of
+ * block ids moved. The copy is enqueued on stream after all outstanding work of the slice; later
+ * calls on other streams wait for it. Errors: ENOSPC (no room; nothing changes), ECUDA. */
+int slice_reclaim(slice_t* s, uint32_t take_blocks, uint64_t* out_n_migrated, void* stream);
+
+/* The lender offers n more block ids (the share of a slice is renegotiated at run time,
+ * Section 1 / 4.1). New ids are handed out in ascending order. Errors: EINVAL (beyond arena). */
+int slice_lend(slice_t* s, uint32_t n_blocks);
+
+/* One new token per sequence (the caller has already grown len and allocated a block where
+ * needed): writes K and V rows of token len-1 for `layer` into the home block and, when the home is
+ * lent and the layer is validly staged for this batch, into the staged copy too.
+ *   k_new, v_new  device, [nseq][num_kv_heads][128] bf16. */
+int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* k_new,
+                    const void* v_new, void* stream);
+
+/* The way back (swap-out direction of Section 4): every staged block of the batch's layer is
+ * written from its ring slot to its home in the lent arena. Requires a valid prefetch of the
+ * layer for this batch (ESTALE otherwise). */
+int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* stream);
+
+/* One pass of the whole path over a batch: for every layer, prefetch of layer l+1 on side_stream
+ * overlapped with attention of layer l on stream (cyclic: the last layer's attention overlaps the
+ * prefetch of layer 0 for the next pass when wrap_prefetch != 0).
+ *   q, out: [num_layers][nseq][num_q_heads][128] bf16; device pointers when io_on_host == 0.
+ *   With io_on_host != 0 they are host pointers (pinned for asynchronous copies): q is copied to the
+ *   device and out back to the host on `stream`, inside the call's enqueued work, through device
+ *   buffers the library allocates on first use. */
+int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t num_q_heads,
+                      float sm_scale, void* out, int32_t io_on_host, int32_t wrap_prefetch,
+                      void* stream, void* side_stream);
+
+/* Counters and capacities (host struct). */
+int slice_stats(slice_t* s, slice_stats_t* out);
+
+/* Test hook: resolved table of the batch, as [nseq][max_blocks_per_seq] int32 on the host (entries
+ * past a sequence's in-use blocks are left untouched); k receives the number of staged blocks. */
+int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* out, uint32_t cap, uint32_t* k);
+
+/* With SLICE_FLAG_PROFILE: after synchronising, returns for each layer of the most recent pass
+ * five times in microseconds relative to the pass's first event: prefetch start, prefetch end,
+ * attention start, attention end (after the merge), end of the attention kernel proper (before the
+ * merge) (host, [num_layers][5] floats; NaN where not recorded). */
+int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers);
+
+/* Low-level copy used by the prefetch microbenchmark: n blocks of block_bytes (a multiple of 16
+ * bytes, 16-byte aligned addresses) are copied dst_base + dst_idx[i]*block_bytes <-
+ * src_base + src_idx[i]*block_bytes. Index arrays and bases are device pointers; dst_idx or src_idx
+ * may be NULL for the identity. kind: 0 default, 1 vector load/store, 2 bulk-copy ring. */
+int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_base, const int32_t* src_idx,
+                      uint32_t n, uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream);
+
+const char* slice_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMASLICE_H_ */

@@ -1,0 +1,91 @@
+// kernels.h — launch interface between the host side of libemaslice (slice.cpp) and its CUDA
+// kernels (copy_kernels.cu, decode_kernels.cu). Internal to the library; not part of the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ema {
+
+// Value written to the device status word when a bounded wait expires.
+constexpr int kDevTimeout = -6;
+
+// One batched block copy: item i moves block_bytes from src(entry src_entry[i]) to
+// dst(entry dst_entry[i]) for each of nlayers layers. An entry e >= 0 addresses id e of base[0],
+// e < 0 addresses id ~e of base[1]. A NULL entry array means entry i = i.
+struct CopyDesc {
+  const uint8_t* src_base[2];
+  uint8_t* dst_base[2];
+  uint64_t src_block_stride[2];
+  uint64_t dst_block_stride[2];
+  uint64_t src_layer_stride[2];
+  uint64_t dst_layer_stride[2];
+  const int32_t* src_entry;
+  const int32_t* dst_entry;
+  uint32_t n;
+  uint32_t nlayers;
+  uint64_t block_bytes;  // multiple of 16
+  int* status;
+};
+
+enum CopyKind : uint32_t { kCopyDefault = 0, kCopyVector = 1, kCopyBulk = 2 };
+
+// Launches one copy kernel on `stream`. ctas == 0 picks a default grid. Returns the CUDA error.
+cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num_sms, cudaStream_t stream);
+
+// Work of one attention CTA range: blocks [blk_begin, blk_end) of batch position seq_idx.
+struct Segment {
+  uint32_t seq_idx;
+  uint32_t blk_begin;
+  uint32_t blk_end;
+  uint32_t flat_begin;  // index of blk_begin in the batch's flat block list
+};
+
+struct DecodeParams {
+  const uint8_t* local_layer;  // base of this layer's local arena
+  uint64_t local_block_stride;
+  const uint8_t* slot_base;    // ring slot that holds this layer's staged blocks
+  uint64_t block_bytes;
+  const int32_t* resolved;     // flat resolved table of the batch
+  const uint32_t* lens;        // [nseq] tokens
+  const Segment* segs;
+  const uint32_t* cta_seg_off; // [ncta + 1]
+  const uint32_t* seq_seg_off; // [nseq + 1] (merge)
+  const void* q;               // [nseq][Hq][128] bf16
+  void* out;                   // [nseq][Hq][128] bf16
+  float* lse;                  // [nseq][Hq] or NULL
+  float* part_o;               // [nsegs][Hq][128] unnormalised partial outputs
+  float* part_ml;              // [nsegs][Hq][2]   running max (log2 domain) and sum
+  uint32_t nseq, nsegs, ncta;
+  uint32_t Hq, Hkv, G;
+  float scale_log2;            // sm_scale * log2(e)
+  int* status;
+};
+
+// Shared memory the attention kernel needs for Hkv KV heads (0 if unsupported).
+size_t decode_smem_bytes(uint32_t Hkv);
+// One-time per-process opt-in to large dynamic shared memory.
+cudaError_t decode_setup();
+// Attention over the batch's segments (partials), then the merge of the partials: two launches.
+cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_merge(const DecodeParams& p, cudaStream_t stream);
+
+struct AppendParams {
+  uint8_t* local_layer;        // this layer's local arena
+  uint64_t local_block_stride;
+  uint8_t* lent_layer;         // this layer's lent arena
+  uint64_t lent_block_stride;
+  uint8_t* slot_base;          // ring slot holding the layer, or NULL when not staged
+  uint64_t block_bytes;
+  const int32_t* home_entry;   // [nseq] table entry of the block holding token len-1
+  const int32_t* stage_pos;    // [nseq] staging position of that block, or -1
+  const uint32_t* lens;        // [nseq]
+  const void* k_new;           // [nseq][Hkv][128] bf16
+  const void* v_new;
+  uint32_t nseq;
+  uint32_t row_bytes;          // Hkv * 128 * 2
+  uint32_t block_tokens;
+};
+cudaError_t launch_append(const AppendParams& p, cudaStream_t stream);
+
+}  // namespace ema

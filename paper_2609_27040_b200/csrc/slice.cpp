@@ -1,0 +1,1052 @@
+// slice.cpp — host side of libemaslice: the slice arena allocator (block tables, free lists,
+// local/lent split), batch plans (resolved tables, copy lists, attention work partition), the
+// stream/event pipeline that overlaps a layer's prefetch with the previous layer's attention,
+// the reclaim planner, and the C ABI declared in include/emaslice.h.
+#include "../../include/emaslice.h"
+#include "kernels.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+namespace {
+
+using ema::Segment;
+
+constexpr int kNumPlans = 4;
+constexpr uint32_t kBlockTokens = 16;
+constexpr uint32_t kHeadDim = 128;
+
+struct Seq {
+  std::vector<int32_t> table;
+  uint32_t len = 0;
+};
+
+struct Owner {
+  int32_t seq = -1;
+  int32_t logical = -1;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// A batch plan: everything about a batch that does not depend on the layer.
+struct Plan {
+  bool valid = false;
+  uint64_t serial = 0;   // unique id of this plan
+  uint64_t version = 0;  // table version it was built from
+  std::vector<int32_t> seqs;
+  uint32_t nseq = 0, total_blocks = 0, k = 0, nsegs = 0, ncta = 0;
+  uint64_t tokens = 0;
+  // byte offsets inside the plan buffer
+  size_t off_resolved = 0, off_lens = 0, off_copy_src = 0, off_segs = 0, off_cta_seg = 0, off_seq_seg = 0,
+         off_home = 0, off_stage_pos = 0, bytes = 0;
+  // host copies for the test hook
+  std::vector<uint32_t> blk_off;
+  uint8_t* host = nullptr;  // pinned (or plain in null-device mode)
+  uint8_t* dev = nullptr;
+  size_t cap = 0;
+  bool uploaded = false;
+  cudaEvent_t ev_uploaded = nullptr;
+  cudaEvent_t ev_used_main = nullptr, ev_used_side = nullptr;
+  bool used_main = false, used_side = false;
+};
+
+struct SlotState {
+  bool valid = false;
+  uint32_t layer = 0;
+  uint64_t plan_serial = 0;
+  bool pref_recorded = false, attn_recorded = false;
+  cudaEvent_t pref_done = nullptr, attn_done = nullptr;
+};
+
+struct StreamEpoch {
+  cudaStream_t stream;
+  uint64_t epoch;
+};
+
+}  // namespace
+
+struct ema_slice {
+  slice_config_t cfg{};
+  bool null_dev = false, profile = false;
+  uint64_t block_bytes = 0;
+  uint64_t local_ls = 0, local_bs = 0, lent_ls = 0, lent_bs = 0, slot_bytes = 0;
+  int num_sms = 148;
+  uint32_t ncta_decode = 148;
+  // allocator
+  std::vector<int32_t> free_local, free_lent;  // back() pops next
+  std::unordered_map<int32_t, Seq> seqs;
+  std::vector<Owner> owner_local, owner_lent;
+  uint32_t lent_cap = 0;
+  uint64_t version = 1;
+  // plans and slots
+  Plan plans[kNumPlans];
+  int next_plan = 0;
+  uint64_t plan_serial = 0;
+  std::vector<SlotState> slots;
+  // device scratch
+  float* part_o = nullptr;
+  float* part_ml = nullptr;
+  uint32_t part_hq = 0;
+  int* dev_status = nullptr;
+  int* host_status = nullptr;  // pinned
+  // reclaim
+  int32_t* reclaim_host = nullptr;
+  int32_t* reclaim_dev = nullptr;
+  cudaEvent_t reclaim_done = nullptr;
+  bool reclaim_recorded = false;
+  uint64_t reclaim_epoch = 0;
+  std::vector<StreamEpoch> streams;
+  cudaEvent_t append_done = nullptr;
+  bool append_pending = false;
+  cudaEvent_t ev_tmp = nullptr;
+  // host io staging for slice_decode_step
+  void* io_q = nullptr;
+  void* io_out = nullptr;
+  size_t io_bytes = 0;
+  // profiling
+  std::vector<cudaEvent_t> prof;  // [layer][5]
+  std::vector<uint8_t> prof_set;
+  cudaEvent_t prof_base = nullptr;
+  bool prof_base_set = false;
+  slice_stats_t st{};
+};
+
+namespace {
+
+#define CU(s, call)                                   \
+  do {                                                \
+    cudaError_t e__ = (call);                         \
+    if (e__ != cudaSuccess) {                         \
+      (s)->st.last_cuda_error = static_cast<int>(e__); \
+      return SLICE_ECUDA;                             \
+    }                                                 \
+  } while (0)
+
+inline uint32_t blocks_for(uint32_t len) { return (len + kBlockTokens - 1) / kBlockTokens; }
+
+int ensure_stream(ema_slice* s, cudaStream_t stream) {
+  if (s->null_dev) return SLICE_OK;
+  for (auto& se : s->streams) {
+    if (se.stream == stream) {
+      if (se.epoch < s->reclaim_epoch) {
+        CU(s, cudaStreamWaitEvent(stream, s->reclaim_done, 0));
+        se.epoch = s->reclaim_epoch;
+      }
+      return SLICE_OK;
+    }
+  }
+  if (s->reclaim_recorded) CU(s, cudaStreamWaitEvent(stream, s->reclaim_done, 0));
+  s->streams.push_back(StreamEpoch{stream, s->reclaim_epoch});
+  return SLICE_OK;
+}
+
+size_t plan_capacity(const ema_slice* s) {
+  const slice_config_t& c = s->cfg;
+  size_t b = 0;
+  b += align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved (upper bound)
+  b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // lens
+  b += align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src
+  b += align_up((static_cast<size_t>(c.max_seqs) + s->ncta_decode + 1) * sizeof(Segment), 256);
+  b += align_up((static_cast<size_t>(s->ncta_decode) + 1) * 4, 256);                // cta_seg_off
+  b += align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // seq_seg_off
+  b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                      // home, stage_pos
+  return b;
+}
+
+// Validates a batch: known, distinct sequences. Returns OK or the error.
+int check_batch(ema_slice* s, const int32_t* seqs, uint32_t nseq) {
+  if (!seqs && nseq) return SLICE_EINVAL;
+  if (nseq == 0 || nseq > s->cfg.max_seqs) return SLICE_EINVAL;
+  for (uint32_t i = 0; i < nseq; ++i)
+    if (s->seqs.find(seqs[i]) == s->seqs.end()) return SLICE_ESTATE;
+  if (nseq > 1) {
+    std::vector<int32_t> tmp(seqs, seqs + nseq);
+    std::sort(tmp.begin(), tmp.end());
+    if (std::adjacent_find(tmp.begin(), tmp.end()) != tmp.end()) return SLICE_EINVAL;
+  }
+  return SLICE_OK;
+}
+
+// Finds or builds the plan of a batch for the current table version.
+int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
+  if (!seqs || nseq == 0) return SLICE_EINVAL;
+  for (Plan& p : s->plans) {
+    if (p.valid && p.version == s->version && p.nseq == nseq &&
+        std::memcmp(p.seqs.data(), seqs, nseq * sizeof(int32_t)) == 0) {
+      *out = &p;
+      return SLICE_OK;
+    }
+  }
+  int rc = check_batch(s, seqs, nseq);
+  if (rc != SLICE_OK) return rc;
+  // Size the batch before touching a plan buffer.
+  uint64_t total_blocks = 0, k = 0, tokens = 0;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    const Seq& q = s->seqs[seqs[i]];
+    const uint32_t nb = blocks_for(q.len);
+    total_blocks += nb;
+    tokens += q.len;
+    for (uint32_t b = 0; b < nb; ++b)
+      if (q.table[b] < 0) ++k;
+  }
+  if (k > s->cfg.staging_blocks_per_slot) return SLICE_ESTAGING;
+
+  Plan& p = s->plans[s->next_plan];
+  s->next_plan = (s->next_plan + 1) % kNumPlans;
+  if (!s->null_dev) {
+    // The previous upload from this host buffer must have left it.
+    if (p.uploaded) CU(s, cudaEventSynchronize(p.ev_uploaded));
+  }
+  p.valid = false;
+  p.serial = ++s->plan_serial;
+  p.version = s->version;
+  p.seqs.assign(seqs, seqs + nseq);
+  p.nseq = nseq;
+  p.total_blocks = static_cast<uint32_t>(total_blocks);
+  p.k = static_cast<uint32_t>(k);
+  p.tokens = tokens;
+  p.uploaded = false;
+
+  // Attention work partition: equal contiguous ranges of the flat block list, one per CTA.
+  const uint32_t ncta = s->ncta_decode;
+  uint32_t per = static_cast<uint32_t>((total_blocks + ncta - 1) / ncta);
+  if (per == 0) per = 1;
+  const uint32_t used_cta = static_cast<uint32_t>((total_blocks + per - 1) / per);
+  p.ncta = used_cta;
+
+  size_t off = 0;
+  p.off_resolved = off;
+  off += align_up(static_cast<size_t>(total_blocks) * 4, 256);
+  p.off_lens = off;
+  off += align_up(static_cast<size_t>(nseq) * 4, 256);
+  p.off_copy_src = off;
+  off += align_up(static_cast<size_t>(k) * 4, 256);
+  p.off_segs = off;
+  off += align_up((static_cast<size_t>(nseq) + used_cta + 1) * sizeof(Segment), 256);
+  p.off_cta_seg = off;
+  off += align_up((static_cast<size_t>(used_cta) + 1) * 4, 256);
+  p.off_seq_seg = off;
+  off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
+  p.off_home = off;
+  off += align_up(static_cast<size_t>(nseq) * 4, 256);
+  p.off_stage_pos = off;
+  off += align_up(static_cast<size_t>(nseq) * 4, 256);
+  p.bytes = off;
+  if (off > p.cap) return SLICE_EINVAL;  // cannot happen: capacity is sized from the maxima
+
+  int32_t* resolved = reinterpret_cast<int32_t*>(p.host + p.off_resolved);
+  uint32_t* lens = reinterpret_cast<uint32_t*>(p.host + p.off_lens);
+  int32_t* copy_src = reinterpret_cast<int32_t*>(p.host + p.off_copy_src);
+  Segment* segs = reinterpret_cast<Segment*>(p.host + p.off_segs);
+  uint32_t* cta_seg = reinterpret_cast<uint32_t*>(p.host + p.off_cta_seg);
+  uint32_t* seq_seg = reinterpret_cast<uint32_t*>(p.host + p.off_seq_seg);
+  int32_t* home = reinterpret_cast<int32_t*>(p.host + p.off_home);
+  int32_t* stage_pos = reinterpret_cast<int32_t*>(p.host + p.off_stage_pos);
+
+  p.blk_off.resize(nseq + 1);
+  uint32_t flat = 0, kk = 0, nsegs = 0, cta = 0;
+  cta_seg[0] = 0;
+  for (uint32_t i = 0; i < nseq; ++i) {
+    const Seq& q = s->seqs[seqs[i]];
+    const uint32_t nb = blocks_for(q.len);
+    p.blk_off[i] = flat;
+    lens[i] = q.len;
+    seq_seg[i] = nsegs;
+    home[i] = 0;
+    stage_pos[i] = -1;
+    const uint32_t last_b = q.len ? (q.len - 1) / kBlockTokens : 0;
+    uint32_t b = 0;
+    while (b < nb) {
+      // this CTA's range is [cta*per, (cta+1)*per) in flat block indices
+      const uint32_t cta_end = (cta + 1) * per;
+      const uint32_t take = std::min(nb - b, cta_end - flat);
+      segs[nsegs++] = Segment{i, b, b + take, flat};
+      for (uint32_t j = 0; j < take; ++j) {
+        const int32_t e = q.table[b + j];
+        int32_t r = e;
+        if (e < 0) {
+          copy_src[kk] = e;  // negative entry: tier 1 (lent arena), id ~e
+          r = ~static_cast<int32_t>(kk);
+          ++kk;
+        }
+        resolved[flat + j] = r;
+        if (q.len && b + j == last_b) {
+          home[i] = e;
+          stage_pos[i] = e < 0 ? ~r : -1;
+        }
+      }
+      b += take;
+      flat += take;
+      if (flat == cta_end) {
+        ++cta;
+        cta_seg[cta] = nsegs;
+      }
+    }
+  }
+  p.blk_off[nseq] = flat;
+  seq_seg[nseq] = nsegs;
+  if (cta < used_cta) cta_seg[used_cta] = nsegs;  // last, partly filled range
+  p.nsegs = nsegs;
+  p.valid = true;  // used_main / used_side stay: they guard the device buffer, not the plan
+  s->st.plans_built++;
+  *out = &p;
+  return SLICE_OK;
+}
+
+// Uploads the plan on `stream` if nobody has yet; otherwise makes `stream` wait for the upload.
+int plan_on_stream(ema_slice* s, Plan* p, cudaStream_t stream, bool is_side) {
+  if (s->null_dev) return SLICE_OK;
+  if (!p->uploaded) {
+    // The device buffer may still be read by kernels of the plan that lived here before.
+    if (p->used_main) CU(s, cudaStreamWaitEvent(stream, p->ev_used_main, 0));
+    if (p->used_side) CU(s, cudaStreamWaitEvent(stream, p->ev_used_side, 0));
+    CU(s, cudaMemcpyAsync(p->dev, p->host, p->bytes, cudaMemcpyHostToDevice, stream));
+    CU(s, cudaEventRecord(p->ev_uploaded, stream));
+    p->uploaded = true;
+  } else {
+    CU(s, cudaStreamWaitEvent(stream, p->ev_uploaded, 0));
+  }
+  (void)is_side;
+  return SLICE_OK;
+}
+
+int mark_used(ema_slice* s, Plan* p, cudaStream_t stream, bool is_side) {
+  if (s->null_dev) return SLICE_OK;
+  if (is_side) {
+    CU(s, cudaEventRecord(p->ev_used_side, stream));
+    p->used_side = true;
+  } else {
+    CU(s, cudaEventRecord(p->ev_used_main, stream));
+    p->used_main = true;
+  }
+  return SLICE_OK;
+}
+
+void invalidate_staged(ema_slice* s) {
+  for (auto& sl : s->slots) sl.valid = false;
+}
+
+void bump_version(ema_slice* s) { ++s->version; }
+
+int prof_record(ema_slice* s, uint32_t layer, int which, cudaStream_t stream) {
+  if (!s->profile || s->null_dev) return SLICE_OK;
+  CU(s, cudaEventRecord(s->prof[layer * 5 + which], stream));
+  s->prof_set[layer * 5 + which] = 1;
+  return SLICE_OK;
+}
+
+int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
+  int rc = ensure_stream(s, side);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, side, true);
+  if (rc) return rc;
+  const uint32_t slot = layer % s->cfg.ring_slots;
+  SlotState& sl = s->slots[slot];
+  if (!s->null_dev) {
+    if (sl.attn_recorded) CU(s, cudaStreamWaitEvent(side, sl.attn_done, 0));
+    if (s->append_pending) CU(s, cudaStreamWaitEvent(side, s->append_done, 0));
+    rc = prof_record(s, layer, 0, side);
+    if (rc) return rc;
+    if (p->k) {
+      ema::CopyDesc d{};
+      d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base);
+      d.src_block_stride[0] = d.src_block_stride[1] = s->lent_bs;
+      d.src_layer_stride[0] = d.src_layer_stride[1] = 0;
+      d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+      d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
+      d.dst_block_stride[0] = d.dst_block_stride[1] = s->block_bytes;
+      d.src_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
+      d.dst_entry = nullptr;
+      d.n = p->k;
+      d.nlayers = 1;
+      d.block_bytes = s->block_bytes;
+      d.status = s->dev_status;
+      const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+      CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, side));
+      s->st.kernel_launches++;
+    }
+    rc = prof_record(s, layer, 1, side);
+    if (rc) return rc;
+    CU(s, cudaEventRecord(sl.pref_done, side));
+    sl.pref_recorded = true;
+    rc = mark_used(s, p, side, true);
+    if (rc) return rc;
+  }
+  sl.valid = true;
+  sl.layer = layer;
+  sl.plan_serial = p->serial;
+  s->st.prefetch_calls++;
+  s->st.prefetched_blocks += p->k;
+  s->st.prefetched_bytes += static_cast<uint64_t>(p->k) * s->block_bytes;
+  return SLICE_OK;
+}
+
+int ensure_partials(ema_slice* s, uint32_t Hq) {
+  if (s->null_dev || Hq <= s->part_hq) return SLICE_OK;
+  if (s->part_o) {
+    CU(s, cudaDeviceSynchronize());
+    cudaFree(s->part_o);
+    cudaFree(s->part_ml);
+    s->part_o = s->part_ml = nullptr;
+  }
+  const size_t nseg = static_cast<size_t>(s->cfg.max_seqs) + s->ncta_decode + 1;
+  CU(s, cudaMalloc(&s->part_o, nseg * Hq * kHeadDim * sizeof(float)));
+  CU(s, cudaMalloc(&s->part_ml, nseg * Hq * 2 * sizeof(float)));
+  s->part_hq = Hq;
+  return SLICE_OK;
+}
+
+int do_decode(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out,
+              float* lse, cudaStream_t stream) {
+  const uint32_t Hkv = s->cfg.num_kv_heads;
+  if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
+  if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
+  const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
+  for (uint32_t i = 0; i < p->nseq; ++i)
+    if (lens[i] == 0) return SLICE_EINVAL;
+  const uint32_t slot = layer % s->cfg.ring_slots;
+  SlotState& sl = s->slots[slot];
+  if (p->k && !(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
+  int rc = ensure_stream(s, stream);
+  if (rc) return rc;
+  rc = ensure_partials(s, Hq);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, stream, false);
+  if (rc) return rc;
+  if (!s->null_dev) {
+    if (p->k && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    rc = prof_record(s, layer, 2, stream);
+    if (rc) return rc;
+    ema::DecodeParams d{};
+    d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
+    d.local_block_stride = s->local_bs;
+    d.slot_base = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
+    d.block_bytes = s->block_bytes;
+    d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
+    d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
+    d.segs = reinterpret_cast<const Segment*>(p->dev + p->off_segs);
+    d.cta_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_seg);
+    d.seq_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_seq_seg);
+    d.q = q;
+    d.out = out;
+    d.lse = lse;
+    d.part_o = s->part_o;
+    d.part_ml = s->part_ml;
+    d.nseq = p->nseq;
+    d.nsegs = p->nsegs;
+    d.ncta = p->ncta;
+    d.Hq = Hq;
+    d.Hkv = Hkv;
+    d.G = Hq / Hkv;
+    d.scale_log2 = sm_scale * 1.4426950408889634f;
+    d.status = s->dev_status;
+    CU(s, ema::launch_decode(d, stream));
+    rc = prof_record(s, layer, 4, stream);
+    if (rc) return rc;
+    CU(s, ema::launch_merge(d, stream));
+    s->st.kernel_launches += 2;
+    rc = prof_record(s, layer, 3, stream);
+    if (rc) return rc;
+    // The slot may be refilled once this attention has read it.
+    CU(s, cudaEventRecord(sl.attn_done, stream));
+    sl.attn_recorded = true;
+    rc = mark_used(s, p, stream, false);
+    if (rc) return rc;
+  }
+  s->st.decode_calls++;
+  s->st.decode_tokens += p->tokens;
+  return SLICE_OK;
+}
+
+void destroy_impl(ema_slice* s) {
+  if (!s->null_dev) {
+    cudaDeviceSynchronize();
+    for (Plan& p : s->plans) {
+      if (p.host) cudaFreeHost(p.host);
+      if (p.dev) cudaFree(p.dev);
+      if (p.ev_uploaded) cudaEventDestroy(p.ev_uploaded);
+      if (p.ev_used_main) cudaEventDestroy(p.ev_used_main);
+      if (p.ev_used_side) cudaEventDestroy(p.ev_used_side);
+    }
+    for (auto& sl : s->slots) {
+      if (sl.pref_done) cudaEventDestroy(sl.pref_done);
+      if (sl.attn_done) cudaEventDestroy(sl.attn_done);
+    }
+    for (auto e : s->prof)
+      if (e) cudaEventDestroy(e);
+    if (s->prof_base) cudaEventDestroy(s->prof_base);
+    if (s->part_o) cudaFree(s->part_o);
+    if (s->part_ml) cudaFree(s->part_ml);
+    if (s->dev_status) cudaFree(s->dev_status);
+    if (s->host_status) cudaFreeHost(s->host_status);
+    if (s->reclaim_host) cudaFreeHost(s->reclaim_host);
+    if (s->reclaim_dev) cudaFree(s->reclaim_dev);
+    if (s->reclaim_done) cudaEventDestroy(s->reclaim_done);
+    if (s->append_done) cudaEventDestroy(s->append_done);
+    if (s->ev_tmp) cudaEventDestroy(s->ev_tmp);
+    if (s->io_q) cudaFree(s->io_q);
+    if (s->io_out) cudaFree(s->io_out);
+  } else {
+    for (Plan& p : s->plans) delete[] p.host;
+  }
+  delete s;
+}
+
+}  // namespace
+
+extern "C" {
+
+int slice_create(const slice_config_t* cfg, slice_t** out) {
+  if (!cfg || !out) return SLICE_EINVAL;
+  *out = nullptr;
+  const bool null_dev = (cfg->flags & SLICE_FLAG_NULL_DEVICE) != 0;
+  if (cfg->head_dim != kHeadDim || cfg->block_tokens != kBlockTokens || cfg->dtype != 0) return SLICE_EINVAL;
+  if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
+  if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
+  if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
+  if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
+    return SLICE_EINVAL;
+  const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
+  if (!null_dev) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(cfg->local_base) | reinterpret_cast<uintptr_t>(cfg->lent_base) |
+                        reinterpret_cast<uintptr_t>(cfg->staging_base);
+    if (a & 255u) return SLICE_EINVAL;
+  }
+  const uint64_t strides[4] = {cfg->local_layer_stride, cfg->local_block_stride, cfg->lent_layer_stride,
+                               cfg->lent_block_stride};
+  for (uint64_t v : strides)
+    if (v & 255u) return SLICE_EINVAL;
+  // free orders must be permutations
+  auto is_perm = [](const uint32_t* o, uint32_t n) {
+    if (!o) return true;
+    std::vector<uint8_t> seen(n, 0);
+    for (uint32_t k = 0; k < n; ++k) {
+      if (o[k] >= n || seen[o[k]]) return false;
+      seen[o[k]] = 1;
+    }
+    return true;
+  };
+  if (!is_perm(cfg->local_free_order, cfg->local_blocks) || !is_perm(cfg->lent_free_order, cfg->lent_blocks_physical))
+    return SLICE_EINVAL;
+
+  ema_slice* s = new (std::nothrow) ema_slice();
+  if (!s) return SLICE_EINVAL;
+  s->cfg = *cfg;
+  s->cfg.local_free_order = s->cfg.lent_free_order = nullptr;
+  s->null_dev = null_dev;
+  s->profile = (cfg->flags & SLICE_FLAG_PROFILE) != 0;
+  s->block_bytes = bb;
+  s->local_bs = cfg->local_block_stride ? cfg->local_block_stride : bb;
+  s->local_ls = cfg->local_layer_stride ? cfg->local_layer_stride : bb * cfg->local_blocks;
+  s->lent_bs = cfg->lent_block_stride ? cfg->lent_block_stride : bb;
+  s->lent_ls = cfg->lent_layer_stride ? cfg->lent_layer_stride : bb * cfg->lent_blocks_physical;
+  s->slot_bytes = bb * cfg->staging_blocks_per_slot;
+  s->lent_cap = cfg->lent_blocks;
+  s->owner_local.assign(cfg->local_blocks, Owner());
+  s->owner_lent.assign(cfg->lent_blocks_physical, Owner());
+  for (uint32_t k = cfg->local_blocks; k-- > 0;)
+    s->free_local.push_back(static_cast<int32_t>(cfg->local_free_order ? cfg->local_free_order[k] : k));
+  for (uint32_t k = cfg->lent_blocks_physical; k-- > 0;) {
+    const uint32_t id = cfg->lent_free_order ? cfg->lent_free_order[k] : k;
+    if (id < cfg->lent_blocks) s->free_lent.push_back(static_cast<int32_t>(id));
+  }
+  s->slots.resize(cfg->ring_slots);
+
+  int rc = SLICE_OK;
+  auto fail = [&](int code) {
+    destroy_impl(s);
+    return code;
+  };
+  if (!null_dev) {
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(SLICE_ECUDA);
+    s->num_sms = prop.multiProcessorCount;
+    if (ema::decode_setup() != cudaSuccess) return fail(SLICE_ECUDA);
+  }
+  s->ncta_decode = cfg->decode_ctas ? cfg->decode_ctas : static_cast<uint32_t>(s->num_sms);
+  const size_t cap = plan_capacity(s);
+  for (Plan& p : s->plans) {
+    p.cap = cap;
+    if (null_dev) {
+      p.host = new (std::nothrow) uint8_t[cap];
+      if (!p.host) return fail(SLICE_EINVAL);
+    } else {
+      if (cudaMallocHost(reinterpret_cast<void**>(&p.host), cap) != cudaSuccess) return fail(SLICE_ECUDA);
+      if (cudaMalloc(reinterpret_cast<void**>(&p.dev), cap) != cudaSuccess) return fail(SLICE_ECUDA);
+      if (cudaEventCreateWithFlags(&p.ev_uploaded, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&p.ev_used_main, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&p.ev_used_side, cudaEventDisableTiming) != cudaSuccess)
+        return fail(SLICE_ECUDA);
+    }
+  }
+  if (!null_dev) {
+    for (auto& sl : s->slots) {
+      if (cudaEventCreateWithFlags(&sl.pref_done, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&sl.attn_done, cudaEventDisableTiming) != cudaSuccess)
+        return fail(SLICE_ECUDA);
+    }
+    if (cudaMalloc(reinterpret_cast<void**>(&s->dev_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaMemset(s->dev_status, 0, 256) != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaMallocHost(reinterpret_cast<void**>(&s->host_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
+    *s->host_status = 0;
+    const size_t rl = static_cast<size_t>(std::max(cfg->lent_blocks_physical, 1u)) * 2 * sizeof(int32_t);
+    if (cudaMallocHost(reinterpret_cast<void**>(&s->reclaim_host), rl) != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaMalloc(reinterpret_cast<void**>(&s->reclaim_dev), rl) != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaEventCreateWithFlags(&s->reclaim_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->append_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&s->ev_tmp, cudaEventDisableTiming) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+    if (s->profile) {
+      s->prof.assign(static_cast<size_t>(cfg->num_layers) * 5, nullptr);
+      s->prof_set.assign(static_cast<size_t>(cfg->num_layers) * 5, 0);
+      for (auto& e : s->prof)
+        if (cudaEventCreate(&e) != cudaSuccess) return fail(SLICE_ECUDA);
+      if (cudaEventCreate(&s->prof_base) != cudaSuccess) return fail(SLICE_ECUDA);
+    }
+  }
+  (void)rc;
+  *out = s;
+  return SLICE_OK;
+}
+
+int slice_destroy(slice_t* s) {
+  if (!s) return SLICE_EINVAL;
+  destroy_impl(s);
+  return SLICE_OK;
+}
+
+int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t hint, int32_t* out_entries) {
+  if (!s || seq < 0 || hint < SLICE_TIER_AUTO || hint > SLICE_TIER_LENT) return SLICE_EINVAL;
+  auto it = s->seqs.find(seq);
+  const bool exists = it != s->seqs.end();
+  if (!exists && s->seqs.size() >= s->cfg.max_seqs) return SLICE_EINVAL;
+  const size_t have = exists ? it->second.table.size() : 0;
+  if (have + n > s->cfg.max_blocks_per_seq) return SLICE_EINVAL;
+  const size_t fl = s->free_local.size(), fr = s->free_lent.size();
+  if (hint == SLICE_TIER_AUTO && n > fl + fr) return SLICE_ENOSPC;
+  if (hint == SLICE_TIER_LOCAL && n > fl) return SLICE_ENOSPC;
+  if (hint == SLICE_TIER_LENT && n > fr) return SLICE_ENOSPC;
+  Seq& q = s->seqs[seq];
+  for (uint32_t k = 0; k < n; ++k) {
+    const bool local = hint == SLICE_TIER_LOCAL || (hint == SLICE_TIER_AUTO && !s->free_local.empty());
+    std::vector<int32_t>& stack = local ? s->free_local : s->free_lent;
+    const int32_t id = stack.back();
+    stack.pop_back();
+    (local ? s->owner_local : s->owner_lent)[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
+    const int32_t entry = local ? id : ~id;
+    q.table.push_back(entry);
+    if (out_entries) out_entries[k] = entry;
+  }
+  bump_version(s);
+  return SLICE_OK;
+}
+
+int slice_set_seq_len(slice_t* s, int32_t seq, uint32_t len) {
+  if (!s) return SLICE_EINVAL;
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return SLICE_ESTATE;
+  if (len > static_cast<uint64_t>(it->second.table.size()) * kBlockTokens) return SLICE_EINVAL;
+  if (it->second.len != len) {
+    it->second.len = len;
+    bump_version(s);
+  }
+  return SLICE_OK;
+}
+
+int slice_free_seq(slice_t* s, int32_t seq) {
+  if (!s) return SLICE_EINVAL;
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return SLICE_ESTATE;
+  const std::vector<int32_t>& t = it->second.table;
+  for (size_t b = t.size(); b-- > 0;) {
+    const int32_t e = t[b];
+    if (e >= 0) {
+      s->free_local.push_back(e);
+      s->owner_local[e] = Owner();
+    } else {
+      s->free_lent.push_back(~e);
+      s->owner_lent[~e] = Owner();
+    }
+  }
+  s->seqs.erase(it);
+  bump_version(s);
+  return SLICE_OK;
+}
+
+int slice_get_block_table(slice_t* s, int32_t seq, int32_t* out, uint32_t cap, uint32_t* n, uint32_t* len) {
+  if (!s) return SLICE_EINVAL;
+  auto it = s->seqs.find(seq);
+  if (it == s->seqs.end()) return SLICE_ESTATE;
+  const std::vector<int32_t>& t = it->second.table;
+  if (n) *n = static_cast<uint32_t>(t.size());
+  if (len) *len = it->second.len;
+  if (out) {
+    if (cap < t.size()) return SLICE_EINVAL;
+    std::copy(t.begin(), t.end(), out);
+  }
+  return SLICE_OK;
+}
+
+int slice_get_free_stack(slice_t* s, int32_t tier, int32_t* out, uint32_t cap, uint32_t* n) {
+  if (!s || (tier != SLICE_TIER_LOCAL && tier != SLICE_TIER_LENT)) return SLICE_EINVAL;
+  const std::vector<int32_t>& st = tier == SLICE_TIER_LOCAL ? s->free_local : s->free_lent;
+  if (n) *n = static_cast<uint32_t>(st.size());
+  if (out) {
+    if (cap < st.size()) return SLICE_EINVAL;
+    for (size_t k = 0; k < st.size(); ++k) out[k] = st[st.size() - 1 - k];
+  }
+  return SLICE_OK;
+}
+
+int prefetch_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* side_stream) {
+  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  return do_prefetch(s, layer, p, static_cast<cudaStream_t>(side_stream));
+}
+
+int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t num_q_heads,
+                 float sm_scale, void* out, float* lse_or_null, void* stream) {
+  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  return do_decode(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream));
+}
+
+int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* stream_v) {
+  if (!s) return SLICE_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (take > s->lent_cap) take = s->lent_cap;
+  const uint32_t cut = s->lent_cap - take;
+  std::vector<int32_t> victims;
+  for (uint32_t id = cut; id < s->lent_cap; ++id)
+    if (s->owner_lent[id].seq >= 0) victims.push_back(static_cast<int32_t>(id));
+  std::vector<int32_t> below;  // free lent ids under the cut
+  for (int32_t id : s->free_lent)
+    if (static_cast<uint32_t>(id) < cut) below.push_back(id);
+  if (victims.size() > s->free_local.size() + below.size()) return SLICE_ENOSPC;
+
+  // Plan first: destinations in ascending victim order, local ids before lent ids.
+  const size_t n_local = std::min(victims.size(), s->free_local.size());
+  const size_t n_lent = victims.size() - n_local;
+  std::vector<int32_t> sorted_below(below);
+  std::sort(sorted_below.begin(), sorted_below.end());
+  std::vector<int32_t> dst(victims.size());
+  for (size_t k = 0; k < n_local; ++k) dst[k] = s->free_local[s->free_local.size() - 1 - k];
+  for (size_t k = 0; k < n_lent; ++k) dst[n_local + k] = ~sorted_below[k];
+
+  if (!s->null_dev && !victims.empty()) {
+    // Everything outstanding on the slice's streams must finish before blocks move.
+    int rc = ensure_stream(s, stream);
+    if (rc) return rc;
+    if (s->reclaim_recorded) CU(s, cudaEventSynchronize(s->reclaim_done));  // list buffer reuse
+    for (auto& se : s->streams) {
+      if (se.stream == stream) continue;
+      CU(s, cudaEventRecord(s->ev_tmp, se.stream));
+      CU(s, cudaStreamWaitEvent(stream, s->ev_tmp, 0));
+    }
+    const size_t n = victims.size();
+    for (size_t k = 0; k < n; ++k) {
+      s->reclaim_host[k] = ~victims[k];
+      s->reclaim_host[n + k] = dst[k];
+    }
+    CU(s, cudaMemcpyAsync(s->reclaim_dev, s->reclaim_host, 2 * n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    ema::CopyDesc d{};
+    d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base);
+    d.src_block_stride[0] = d.src_block_stride[1] = s->lent_bs;
+    d.src_layer_stride[0] = d.src_layer_stride[1] = s->lent_ls;
+    d.dst_base[0] = static_cast<uint8_t*>(s->cfg.local_base);
+    d.dst_block_stride[0] = s->local_bs;
+    d.dst_layer_stride[0] = s->local_ls;
+    d.dst_base[1] = static_cast<uint8_t*>(s->cfg.lent_base);
+    d.dst_block_stride[1] = s->lent_bs;
+    d.dst_layer_stride[1] = s->lent_ls;
+    d.src_entry = s->reclaim_dev;
+    d.dst_entry = s->reclaim_dev + n;
+    d.n = static_cast<uint32_t>(n);
+    d.nlayers = s->cfg.num_layers;
+    d.block_bytes = s->block_bytes;
+    d.status = s->dev_status;
+    const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+    CU(s, ema::launch_copy(d, kind, 0, s->num_sms, stream));
+    s->st.kernel_launches++;
+    CU(s, cudaEventRecord(s->reclaim_done, stream));
+    s->reclaim_recorded = true;
+    ++s->reclaim_epoch;
+    for (auto& se : s->streams)
+      if (se.stream == stream) se.epoch = s->reclaim_epoch;
+  }
+
+  // Commit the integer state.
+  std::vector<int32_t> kept;
+  for (int32_t id : s->free_lent)
+    if (static_cast<uint32_t>(id) < cut) kept.push_back(id);
+  s->free_lent.swap(kept);
+  for (size_t k = 0; k < victims.size(); ++k) {
+    const int32_t v = victims[k];
+    const Owner own = s->owner_lent[v];
+    if (k < n_local) {
+      s->free_local.pop_back();
+      s->owner_local[dst[k]] = own;
+    } else {
+      const int32_t id = ~dst[k];
+      s->free_lent.erase(std::find(s->free_lent.begin(), s->free_lent.end(), id));
+      s->owner_lent[id] = own;
+    }
+    s->seqs[own.seq].table[own.logical] = dst[k];
+    s->owner_lent[v] = Owner();
+  }
+  s->lent_cap = cut;
+  bump_version(s);
+  invalidate_staged(s);
+  s->st.reclaims++;
+  s->st.migrated_blocks += victims.size();
+  s->st.migrated_bytes += static_cast<uint64_t>(victims.size()) * s->block_bytes * s->cfg.num_layers;
+  if (out_n_migrated) *out_n_migrated = victims.size();
+  return SLICE_OK;
+}
+
+int slice_lend(slice_t* s, uint32_t n) {
+  if (!s) return SLICE_EINVAL;
+  if (static_cast<uint64_t>(s->lent_cap) + n > s->cfg.lent_blocks_physical) return SLICE_EINVAL;
+  for (uint32_t k = n; k-- > 0;) s->free_lent.push_back(static_cast<int32_t>(s->lent_cap + k));
+  s->lent_cap += n;
+  return SLICE_OK;
+}
+
+int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* k_new,
+                    const void* v_new, void* stream_v) {
+  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  if (!s->null_dev && (!k_new || !v_new)) return SLICE_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
+  for (uint32_t i = 0; i < nseq; ++i)
+    if (lens[i] == 0) return SLICE_EINVAL;
+  if (s->null_dev) return SLICE_OK;
+  rc = ensure_stream(s, stream);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, stream, false);
+  if (rc) return rc;
+  const uint32_t slot = layer % s->cfg.ring_slots;
+  SlotState& sl = s->slots[slot];
+  const bool staged = sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
+  if (staged && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  ema::AppendParams a{};
+  a.local_layer = static_cast<uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
+  a.local_block_stride = s->local_bs;
+  a.lent_layer = static_cast<uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  a.lent_block_stride = s->lent_bs;
+  a.slot_base = staged ? static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes : nullptr;
+  a.block_bytes = s->block_bytes;
+  a.home_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_home);
+  a.stage_pos = reinterpret_cast<const int32_t*>(p->dev + p->off_stage_pos);
+  a.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
+  a.k_new = k_new;
+  a.v_new = v_new;
+  a.nseq = nseq;
+  a.row_bytes = s->cfg.num_kv_heads * kHeadDim * 2;
+  a.block_tokens = kBlockTokens;
+  CU(s, ema::launch_append(a, stream));
+  s->st.kernel_launches++;
+  CU(s, cudaEventRecord(s->append_done, stream));
+  s->append_pending = true;
+  return mark_used(s, p, stream, false);
+}
+
+int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* stream_v) {
+  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  const uint32_t slot = layer % s->cfg.ring_slots;
+  SlotState& sl = s->slots[slot];
+  if (!(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
+  if (s->null_dev || p->k == 0) return SLICE_OK;
+  rc = ensure_stream(s, stream);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, stream, false);
+  if (rc) return rc;
+  if (sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  ema::CopyDesc d{};
+  d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
+  d.src_block_stride[0] = d.src_block_stride[1] = s->block_bytes;
+  d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  d.dst_block_stride[0] = d.dst_block_stride[1] = s->lent_bs;
+  d.src_entry = nullptr;
+  d.dst_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
+  d.n = p->k;
+  d.nlayers = 1;
+  d.block_bytes = s->block_bytes;
+  d.status = s->dev_status;
+  const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+  CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, stream));
+  s->st.kernel_launches++;
+  // A later prefetch of this layer reads the lent arena: it must see the written blocks.
+  CU(s, cudaEventRecord(s->append_done, stream));
+  s->append_pending = true;
+  return mark_used(s, p, stream, false);
+}
+
+int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
+                      void* out, int32_t io_on_host, int32_t wrap, void* stream_v, void* side_v) {
+  if (!s) return SLICE_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v), side = static_cast<cudaStream_t>(side_v);
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  const uint32_t L = s->cfg.num_layers, R = s->cfg.ring_slots;
+  const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
+  const uint8_t* qd = static_cast<const uint8_t*>(q);
+  uint8_t* od = static_cast<uint8_t*>(out);
+  if (s->profile && !s->null_dev) {
+    std::fill(s->prof_set.begin(), s->prof_set.end(), 0);
+    CU(s, cudaEventRecord(s->prof_base, stream));
+    s->prof_base_set = true;
+  }
+  if (io_on_host && !s->null_dev) {
+    if (!q || !out) return SLICE_EINVAL;
+    const size_t need = per_layer * L;
+    if (need > s->io_bytes) {
+      CU(s, cudaDeviceSynchronize());
+      if (s->io_q) cudaFree(s->io_q);
+      if (s->io_out) cudaFree(s->io_out);
+      s->io_q = s->io_out = nullptr;
+      s->io_bytes = 0;
+      CU(s, cudaMalloc(&s->io_q, need));
+      CU(s, cudaMalloc(&s->io_out, need));
+      s->io_bytes = need;
+    }
+    rc = ensure_stream(s, stream);
+    if (rc) return rc;
+    CU(s, cudaMemcpyAsync(s->io_q, q, need, cudaMemcpyHostToDevice, stream));
+    qd = static_cast<const uint8_t*>(s->io_q);
+    od = static_cast<uint8_t*>(s->io_out);
+  }
+  auto staged = [&](uint32_t layer) {
+    const SlotState& sl = s->slots[layer % R];
+    return sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
+  };
+  if (p->k && !staged(0)) {
+    rc = do_prefetch(s, 0, p, side);
+    if (rc) return rc;
+  }
+  for (uint32_t l = 0; l < L; ++l) {
+    // Layer-boundary check (Section 4.2.2): trigger the next transfer before computing this layer.
+    if (p->k) {
+      if (l + 1 < L) {
+        if (!staged(l + 1)) {
+          rc = do_prefetch(s, l + 1, p, side);
+          if (rc) return rc;
+        }
+      } else if (wrap && L > 1) {
+        rc = do_prefetch(s, 0, p, side);
+        if (rc) return rc;
+      }
+    }
+    rc = do_decode(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream);
+    if (rc) return rc;
+  }
+  if (io_on_host && !s->null_dev)
+    CU(s, cudaMemcpyAsync(out, s->io_out, per_layer * L, cudaMemcpyDeviceToHost, stream));
+  return SLICE_OK;
+}
+
+int slice_stats(slice_t* s, slice_stats_t* out) {
+  if (!s || !out) return SLICE_EINVAL;
+  s->st.local_free = static_cast<uint32_t>(s->free_local.size());
+  s->st.local_used = s->cfg.local_blocks - s->st.local_free;
+  s->st.lent_free = static_cast<uint32_t>(s->free_lent.size());
+  s->st.lent_used = s->lent_cap - s->st.lent_free;
+  s->st.lent_capacity = s->lent_cap;
+  s->st.num_seqs = static_cast<uint32_t>(s->seqs.size());
+  if (!s->null_dev && s->dev_status) {
+    // A plain blocking copy of one word: reports what finished kernels have recorded.
+    int v = 0;
+    if (cudaMemcpy(&v, s->dev_status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess) s->st.device_status = v;
+  }
+  *out = s->st;
+  return SLICE_OK;
+}
+
+int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* out, uint32_t cap, uint32_t* k) {
+  if (!s) return SLICE_EINVAL;
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  if (k) *k = p->k;
+  if (out) {
+    const uint32_t stride = s->cfg.max_blocks_per_seq;
+    if (static_cast<uint64_t>(cap) < static_cast<uint64_t>(nseq) * stride) return SLICE_EINVAL;
+    const int32_t* resolved = reinterpret_cast<const int32_t*>(p->host + p->off_resolved);
+    for (uint32_t i = 0; i < nseq; ++i)
+      for (uint32_t f = p->blk_off[i]; f < p->blk_off[i + 1]; ++f)
+        out[static_cast<size_t>(i) * stride + (f - p->blk_off[i])] = resolved[f];
+  }
+  return SLICE_OK;
+}
+
+int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers) {
+  if (!s || !out || !s->profile || s->null_dev || !s->prof_base_set) return SLICE_EINVAL;
+  if (cap_layers < s->cfg.num_layers) return SLICE_EINVAL;
+  CU(s, cudaDeviceSynchronize());
+  for (uint32_t i = 0; i < s->cfg.num_layers * 5; ++i) {
+    out[i] = std::numeric_limits<float>::quiet_NaN();
+    if (!s->prof_set[i]) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, s->prof_base, s->prof[i]) == cudaSuccess) out[i] = ms * 1000.f;
+  }
+  return SLICE_OK;
+}
+
+int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_base, const int32_t* src_idx, uint32_t n,
+                      uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream) {
+  if (!dst_base || !src_base || (block_bytes & 15u) || block_bytes == 0 || kind > 2) return SLICE_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(dst_base) | reinterpret_cast<uintptr_t>(src_base)) & 15u) return SLICE_EINVAL;
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return SLICE_ECUDA;
+  }
+  ema::CopyDesc d{};
+  d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(src_base);
+  d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(dst_base);
+  d.src_block_stride[0] = d.src_block_stride[1] = block_bytes;
+  d.dst_block_stride[0] = d.dst_block_stride[1] = block_bytes;
+  d.src_entry = src_idx;
+  d.dst_entry = dst_idx;
+  d.n = n;
+  d.nlayers = 1;
+  d.block_bytes = block_bytes;
+  d.status = nullptr;
+  return ema::launch_copy(d, kind, ctas, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SLICE_OK : SLICE_ECUDA;
+}
+
+const char* slice_strerror(int code) {
+  switch (code) {
+    case SLICE_OK: return "ok";
+    case SLICE_EINVAL: return "invalid argument";
+    case SLICE_ENOSPC: return "not enough free blocks";
+    case SLICE_ESTAGING: return "batch exceeds the staging slot";
+    case SLICE_ESTALE: return "layer is not validly staged for this batch";
+    case SLICE_ECUDA: return "CUDA call failed";
+    case SLICE_ETIMEOUT: return "bounded device wait expired";
+    case SLICE_ESTATE: return "unknown sequence or bad state";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

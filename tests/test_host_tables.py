@@ -1,0 +1,157 @@
+"""Host logic of the CUDA library, run without a GPU in its tables-only mode: the library's
+allocator, resolved tables, staging order and reclaim planning must agree bit for bit with the
+oracle's integer state machine; the shared object must export every entry point the header
+declares."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_27040_b200 import binding as B
+from paper_2609_27040_b200 import build as build_mod
+from paper_2609_27040_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+
+
+def _null_slice(L, Hkv, local, lent, phys, cap, max_seqs, max_blocks, lo=None, ro=None, ring=2):
+    return B.Slice(L, Hkv, local, lent, cap, lent_blocks_physical=phys, ring_slots=ring, max_seqs=max_seqs,
+                   max_blocks_per_seq=max_blocks, flags=B.FLAG_NULL_DEVICE, local_free_order=lo,
+                   lent_free_order=ro)
+
+
+def test_library_exports_every_declared_entry_point():
+    with open(os.path.join(ROOT, "include", "emaslice.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    declared = set(re.findall(r"\b(?:int|const char\*)\s+(\w+)\s*\(", text))
+    assert declared == set(B.EXPORTS)
+    lib = C.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_config_struct_matches_header_size():
+    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 4 uint32
+    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 4 * 4
+
+
+def test_create_rejects_bad_configs():
+    with pytest.raises(B.SliceError):
+        _null_slice(1, 9, 4, 4, 4, 4, 4, 4)                       # more than 8 KV heads
+    with pytest.raises(B.SliceError):
+        _null_slice(1, 8, 4, 5, 4, 4, 4, 4)                       # lent capacity beyond the arena
+    with pytest.raises(B.SliceError):
+        _null_slice(1, 8, 4, 4, 4, 4, 4, 4, ring=0)
+    with pytest.raises(B.SliceError):
+        _null_slice(1, 8, 4, 4, 4, 4, 4, 4, lo=np.array([0, 0, 1, 2], np.uint32))   # not a permutation
+    with pytest.raises(B.SliceError):
+        B.Slice(1, 8, 4, 4, 4)                                     # device mode needs arenas
+
+
+def _same_state(s: B.Slice, o: oracle.OracleSlice, live):
+    for q in live:
+        rc1, t1, l1 = s.slice_get_block_table(q)
+        rc2, t2, l2 = o.block_table(q)
+        assert rc1 == rc2 == 0 and l1 == l2 and t1.tolist() == t2.tolist()
+    assert s.slice_get_free_stack(B.TIER_LOCAL).tolist() == o.free_stack(oracle.LOCAL).tolist()
+    assert s.slice_get_free_stack(B.TIER_LENT).tolist() == o.free_stack(oracle.LENT).tolist()
+    st = s.slice_stats()
+    assert st["lent_capacity"] == o.lent_capacity and st["num_seqs"] == o.num_seqs
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_random_ops_match_oracle_state_machine(seed):
+    rng = np.random.default_rng(seed)
+    LB, RB, PH, CAP = 24, 14, 20, 12
+    lo, ro = synth.free_order(rng, LB), synth.free_order(rng, PH)
+    s = _null_slice(2, 8, LB, RB, PH, CAP, 6, 9, lo, ro)
+    o = oracle.OracleSlice(2, 16, 65536, LB, RB, PH, 2, CAP, max_seqs=6, max_blocks_per_seq=9,
+                           local_free_order=lo, lent_free_order=ro)
+    live = set()
+    for step in range(3000):
+        op = int(rng.integers(0, 12))
+        if op < 5:
+            q, n, hint = int(rng.integers(0, 8)), int(rng.integers(0, 5)), int(rng.integers(0, 3))
+            rc1, e1 = s.slice_alloc_blocks(q, n, hint)
+            rc2, e2 = o.alloc_blocks(q, n, hint)
+            assert rc1 == rc2
+            if rc1 == 0:
+                assert e1.tolist() == e2.tolist()
+                live.add(q)
+        elif op == 5 and live:
+            q = int(rng.choice(sorted(live)))
+            nb = len(o.block_table(q)[1])
+            ln = int(rng.integers(0, nb * 16 + 3))
+            assert s.slice_set_seq_len(q, ln) == o.set_seq_len(q, ln)
+        elif op == 6:
+            q = int(rng.integers(0, 8))
+            rc1, rc2 = s.slice_free_seq(q), o.free_seq(q)
+            assert rc1 == rc2
+            live.discard(q)
+        elif op == 7:
+            take = int(rng.integers(0, 6))
+            rc1, m1 = s.slice_reclaim(take)
+            rc2, m2 = o.reclaim(take, None, None)
+            assert rc1 == rc2 and (rc1 != 0 or m1 == m2)
+        elif op == 8:
+            n = int(rng.integers(0, 4))
+            assert s.slice_lend(n) == o.lend(n)
+        elif live:
+            # resolved tables and staging order of a random batch
+            batch = [int(x) for x in rng.permutation(sorted(live))[: int(rng.integers(1, len(live) + 1))]]
+            rc2, r2, k2 = o.gather(int(rng.integers(0, 2)), batch, None, None)
+            rc1, r1, k1 = s.slice_get_resolved(batch)
+            assert rc1 == rc2
+            if rc1 == 0:
+                assert k1 == k2 and (r1 == r2).all()
+        _same_state(s, o, live)
+    s.close()
+
+
+def test_error_codes_and_unchanged_state():
+    s = _null_slice(2, 8, 4, 4, 4, 2, 4, 8)
+    assert s.slice_alloc_blocks(0, 3, B.TIER_LENT)[0] == B.OK
+    assert s.slice_set_seq_len(0, 48) == B.OK
+    assert s.prefetch_layer(0, [0]) == B.ESTAGING                  # three lent blocks, slot holds two
+    assert s.slice_set_seq_len(0, 20) == B.OK
+    assert s.paged_decode(0, [0], None, 8, 1.0, None) == B.ESTALE   # nothing staged yet
+    assert s.prefetch_layer(0, [0]) == B.OK
+    assert s.paged_decode(0, [0], None, 8, 1.0, None) == B.OK       # tables-only mode: no launch
+    assert s.paged_decode(1, [0], None, 8, 1.0, None) == B.ESTALE   # other layer not staged
+    assert s.prefetch_layer(2, [0]) == B.EINVAL
+    assert s.prefetch_layer(0, [0, 0]) == B.EINVAL
+    assert s.prefetch_layer(0, [7]) == B.ESTATE
+    assert s.paged_decode(0, [0], None, 12, 1.0, None) == B.EINVAL  # 12 query heads over 8 KV heads
+    assert s.slice_set_seq_len(0, 21) == B.OK                       # tables changed: staged copy is stale
+    assert s.paged_decode(0, [0], None, 8, 1.0, None) == B.ESTALE
+    assert s.prefetch_layer(0, [0]) == B.OK
+    rc, mig = s.slice_reclaim(B.TAKE_ALL)
+    assert rc == B.OK and mig == 3
+    assert s.paged_decode(0, [0], None, 8, 1.0, None) == B.OK       # all local now: nothing to stage
+    assert s.slice_get_block_table(0)[1].tolist() == [0, 1, 2]
+    assert s.slice_free_seq(0) == B.OK and s.slice_free_seq(0) == B.ESTATE
+    assert B.slice_strerror(B.ENOSPC) == "not enough free blocks"
+    s.close()
+
+
+def test_decode_step_drives_the_layer_pipeline_in_tables_only_mode():
+    s = _null_slice(4, 8, 8, 8, 8, 4, 4, 8)
+    s.slice_alloc_blocks(0, 2, B.TIER_LENT)
+    s.slice_alloc_blocks(0, 1, B.TIER_LOCAL)
+    s.slice_set_seq_len(0, 40)
+    assert s.slice_decode_step([0], None, 8, 1.0, None) == B.OK
+    st = s.slice_stats()
+    # four layers prefetched, plus layer 0 again for the next pass (cyclic order)
+    assert st["prefetch_calls"] == 5 and st["decode_calls"] == 4 and st["plans_built"] == 1
+    assert s.slice_decode_step([0], None, 8, 1.0, None, wrap_prefetch=False) == B.OK
+    st = s.slice_stats()
+    assert st["prefetch_calls"] == 8 and st["decode_calls"] == 8   # layer 0 was already staged
+    s.close()
