@@ -37,7 +37,8 @@ __host__ __device__ constexpr uint32_t stage_bytes(uint32_t Hkv) { return 2 * kT
 
 struct SegState {
   float m0, m1;  // running max of the two heads this thread owns (MMA path) / of the head (ALU path)
-  float l0, l1;  // running sums (per-thread partial)
+  float l0, l1;  // running sums of the weights as used in P*V (per-thread partial)
+  float e0, e1;  // running sums of the unrounded weights, for the log-sum-exp
 };
 
 // ------------------------------------------------------------------------------------------
@@ -82,6 +83,8 @@ __device__ __forceinline__ void tile_mma(uint32_t stage_addr, uint32_t pitch, ui
   // The sums use the rounded weights, so the result stays a convex combination of V rows.
   st.l0 = st.l0 * al0 + __uint_as_float(p01 << 16) + __uint_as_float(p23 << 16);
   st.l1 = st.l1 * al1 + __uint_as_float(p01 & 0xffff0000u) + __uint_as_float(p23 & 0xffff0000u);
+  st.e0 = st.e0 * al0 + (p0 + p2);
+  st.e1 = st.e1 * al1 + (p1 + p3);
   const uint32_t pb0 = ptx::movmatrix_trans(p01);  // P^T rows = tokens 0..7
   const uint32_t pb1 = ptx::movmatrix_trans(p23);  // tokens 8..15
   // V^T fragment addresses: matrix mj covers tokens (mj>>1)*8.., dims (mj&1)*8..
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__(288, 1) paged_decode_kernel(const DecodeParams
   for (uint32_t sgi = seg0; sgi < seg1; ++sgi) {
     const Segment sg = p.segs[sgi];
     const uint32_t len = p.lens[sg.seq_idx];
-    SegState st{kNegInf, kNegInf, 0.f, 0.f};
+    SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
     bool ok = true;
     if constexpr (kMma) {
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
@@ -244,11 +247,13 @@ __global__ void __launch_bounds__(288, 1) paged_decode_kernel(const DecodeParams
       for (int sh = 4; sh <= 16; sh <<= 1) {
         st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
         st.l1 += __shfl_xor_sync(0xffffffffu, st.l1, sh);
+        st.e0 += __shfl_xor_sync(0xffffffffu, st.e0, sh);
+        st.e1 += __shfl_xor_sync(0xffffffffu, st.e1, sh);
       }
       const uint32_t r0 = lane >> 2;
       const uint32_t h0 = 2 * tig, h1 = h0 + 1;
       float* po = p.part_o + (static_cast<uint64_t>(sgi) * p.Hq + g * G) * kD;
-      float* pml = p.part_ml + (static_cast<uint64_t>(sgi) * p.Hq + g * G) * 2;
+      float* pml = p.part_ml + (static_cast<uint64_t>(sgi) * p.Hq + g * G) * 4;
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
         const uint32_t d = mt * 16 + r0;
@@ -263,12 +268,14 @@ __global__ void __launch_bounds__(288, 1) paged_decode_kernel(const DecodeParams
       }
       if (r0 == 0) {
         if (h0 < G) {
-          pml[h0 * 2] = st.m0;
-          pml[h0 * 2 + 1] = st.l0;
+          pml[h0 * 4] = st.m0;
+          pml[h0 * 4 + 1] = st.l0;
+          pml[h0 * 4 + 2] = st.e0;
         }
         if (h1 < G) {
-          pml[h1 * 2] = st.m1;
-          pml[h1 * 2 + 1] = st.l1;
+          pml[h1 * 4] = st.m1;
+          pml[h1 * 4 + 1] = st.l1;
+          pml[h1 * 4 + 2] = st.e1;
         }
       }
     } else {
@@ -302,9 +309,10 @@ __global__ void __launch_bounds__(288, 1) paged_decode_kernel(const DecodeParams
       float* po = p.part_o + (static_cast<uint64_t>(sgi) * p.Hq + g) * kD;
       *reinterpret_cast<float4*>(po + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
       if (lane == 0) {
-        float* pml = p.part_ml + (static_cast<uint64_t>(sgi) * p.Hq + g) * 2;
+        float* pml = p.part_ml + (static_cast<uint64_t>(sgi) * p.Hq + g) * 4;
         pml[0] = st.m0;
         pml[1] = st.l0;
+        pml[2] = st.l0;
       }
     }
   }
@@ -318,13 +326,14 @@ __global__ void __launch_bounds__(128) merge_partials_kernel(const DecodeParams 
   const uint32_t i = w / p.Hq, h = w % p.Hq;
   const uint32_t s0 = p.seq_seg_off[i], s1 = p.seq_seg_off[i + 1];
   float M = kNegInf;
-  for (uint32_t s = s0; s < s1; ++s) M = fmaxf(M, p.part_ml[(static_cast<uint64_t>(s) * p.Hq + h) * 2]);
-  float l = 0.f;
+  for (uint32_t s = s0; s < s1; ++s) M = fmaxf(M, p.part_ml[(static_cast<uint64_t>(s) * p.Hq + h) * 4]);
+  float l = 0.f, le = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (uint32_t s = s0; s < s1; ++s) {
-    const float* ml = p.part_ml + (static_cast<uint64_t>(s) * p.Hq + h) * 2;
+    const float* ml = p.part_ml + (static_cast<uint64_t>(s) * p.Hq + h) * 4;
     const float wgt = ptx::exp2_approx(ml[0] - M);
     l += ml[1] * wgt;
+    le += ml[2] * wgt;
     const float4 v = *reinterpret_cast<const float4*>(p.part_o + (static_cast<uint64_t>(s) * p.Hq + h) * kD + lane * 4);
     acc.x = fmaf(v.x, wgt, acc.x);
     acc.y = fmaf(v.y, wgt, acc.y);
@@ -337,7 +346,7 @@ __global__ void __launch_bounds__(128) merge_partials_kernel(const DecodeParams 
   uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(i) * p.Hq + h) * kD +
                                         lane * 4);
   *dst = make_uint2(lo, hi);
-  if (p.lse && lane == 0) p.lse[static_cast<uint64_t>(i) * p.Hq + h] = (M + log2f(l)) * 0.6931471805599453f;
+  if (p.lse && lane == 0) p.lse[static_cast<uint64_t>(i) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
 }
 
 // One CTA per sequence: the new token's K and V rows go to the home block and the staged copy.

@@ -55,7 +55,7 @@ struct DecodeParams {
   void* out;                   // [nseq][Hq][128] bf16
   float* lse;                  // [nseq][Hq] or NULL
   float* part_o;               // [nsegs][Hq][128] unnormalised partial outputs
-  float* part_ml;              // [nsegs][Hq][2]   running max (log2 domain) and sum
+  float* part_ml;              // [nsegs][Hq][4]   max (log2 domain), sum as used, exact sum, pad
   uint32_t nseq, nsegs, ncta;
   uint32_t Hq, Hkv, G;
   float scale_log2;            // sm_scale * log2(e)

@@ -396,7 +396,7 @@ int ensure_partials(ema_slice* s, uint32_t Hq) {
   }
   const size_t nseg = static_cast<size_t>(s->cfg.max_seqs) + s->ncta_decode + 1;
   CU(s, cudaMalloc(&s->part_o, nseg * Hq * kHeadDim * sizeof(float)));
-  CU(s, cudaMalloc(&s->part_ml, nseg * Hq * 2 * sizeof(float)));
+  CU(s, cudaMalloc(&s->part_ml, nseg * Hq * 4 * sizeof(float)));
   s->part_hq = Hq;
   return SLICE_OK;
 }
@@ -950,12 +950,17 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
           rc = do_prefetch(s, l + 1, p, side);
           if (rc) return rc;
         }
-      } else if (wrap && L > 1) {
+      } else if (wrap && L > 1 && (L - 1) % R != 0) {
         rc = do_prefetch(s, 0, p, side);
         if (rc) return rc;
       }
     }
     rc = do_decode(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream);
+    if (rc) return rc;
+  }
+  if (p->k && wrap && L > 1 && (L - 1) % R == 0) {
+    // The last layer shares its ring slot with layer 0: refill it only after that attention.
+    rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
   }
   if (io_on_host && !s->null_dev)

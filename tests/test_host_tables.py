@@ -155,3 +155,16 @@ def test_decode_step_drives_the_layer_pipeline_in_tables_only_mode():
     st = s.slice_stats()
     assert st["prefetch_calls"] == 8 and st["decode_calls"] == 8   # layer 0 was already staged
     s.close()
+
+
+def test_decode_step_with_a_shared_ring_slot_for_first_and_last_layer():
+    """Five layers on a ring of two: the last layer and layer 0 share slot 0, so the prefetch of
+    layer 0 for the next pass may only follow the last attention."""
+    s = _null_slice(5, 8, 8, 8, 8, 4, 4, 8)
+    s.slice_alloc_blocks(0, 2, B.TIER_LENT)
+    s.slice_set_seq_len(0, 20)
+    for _ in range(3):
+        assert s.slice_decode_step([0], None, 8, 1.0, None) == B.OK
+    st = s.slice_stats()
+    assert st["decode_calls"] == 15 and st["prefetch_calls"] == 16
+    s.close()
