@@ -51,6 +51,19 @@ def parse_args():
     return ap.parse_args()
 
 
+def profile_traffic(wl):
+    """DRAM bytes per launch of the attention kernel from the committed ncu summary (same per-launch
+    work as the benchmark's: one layer of the full batch); None for other workloads."""
+    path = os.path.join(ROOT, "profiles", "paged_decode_kernel_llama3_8b_batch64_ncu_full.md")
+    if wl.name != "llama3_8b_decode" or wl.batch != 64 or not os.path.exists(path):
+        return None
+    with open(path) as f:
+        for line in f:
+            if line.strip().startswith("traffic_bytes_per_launch:"):
+                return int(line.split(":")[1])
+    return None
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -349,23 +362,37 @@ def run_ours(args, wl):
         extra = {"attn_us_per_layer": attn, "prefetch_us_per_layer": pref, "stall_us_per_layer": stall,
                  "layer_us": layer, "stall_frac_of_attention": stall / attn if attn else None,
                  "alloc_seconds_setup": wp.alloc_s}
-        # attention alone (no concurrent gather): the kernel's own roofline
+        # On-demand ablation: the same pass with prefetch and attention serialised on ONE stream
+        # (no overlap). Its profile events give each kernel's duration without a concurrent kernel.
         for _ in range(2):
-            wp.step(False)
-        iso = []
-        for l in range(wl.num_layers):
-            assert wp.s.prefetch_layer(l, wp.seqs, wp.side) == 0
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            assert wp.s.slice_decode_step(wp.seqs, wp.q, wl.num_q_heads, wp.scale, wp.out, False, wrap, wp.main, wp.main) == 0
+        iso_attn, iso_pref, iso_merge = [], [], []
+        reps = max(3, min(args.steps, 10))
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_serial = 0.0
+        for _ in range(reps):
             e0.record(wp.main)
-            assert wp.s.paged_decode(l, wp.seqs, wp.q[l], wl.num_q_heads, wp.scale, wp.out[l], None, wp.main) == 0
+            assert wp.s.slice_decode_step(wp.seqs, wp.q, wl.num_q_heads, wp.scale, wp.out, False, wrap, wp.main, wp.main) == 0
             e1.record(wp.main)
-            torch.cuda.synchronize()
-            iso.append(e0.elapsed_time(e1) * 1e3)
-        iso_us = float(np.mean(iso[1:] if len(iso) > 1 else iso))
-        roof["isolated"] = {"achieved": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9, "us_per_layer": iso_us,
+            tm = wp.s.slice_layer_times().astype(np.float64)
+            t_serial += e0.elapsed_time(e1) / 1e3
+            iso_attn.append(tm[:, 4] - tm[:, 2])
+            iso_merge.append(tm[:, 3] - tm[:, 4])
+            iso_pref.append(tm[:, 1] - tm[:, 0])
+        iso_us = float(np.nanmean(np.stack(iso_attn)))
+        iso_pref_us = float(np.nanmean(np.stack(iso_pref)))
+        roof["isolated"] = {"achieved": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9, "us_per_launch": iso_us,
                             "frac": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak,
-                            "includes": "attention kernel + merge kernel, no concurrent gather"}
+                            "what": "same kernel with no concurrent gather (serialised pass)"}
+        roof["traffic"] = profile_traffic(wl)
+        extra["gather_kernel_isolated"] = {"us_per_launch": iso_pref_us, "algorithmic_bytes": wp.pref_bytes_layer,
+                                           "achieved_gbs": wp.pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9,
+                                           "frac": wp.pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9 / peak}
+        extra["merge_us_per_launch"] = float(np.nanmean(np.stack(iso_merge)))
+        extra["ablation_serialised_prefetch"] = {"tokens_per_s": wl.batch * reps / t_serial,
+                                                 "ms_per_step": t_serial / reps * 1e3,
+                                                 "note": "on-demand variant: prefetch not overlapped with attention"}
         step_bytes, tokens, pl_blocks, k_blocks = wp.step_bytes, wp.tokens, wp.pl.total_blocks, wp.pl.staging_blocks
         del wp
         torch.cuda.empty_cache()
