@@ -54,7 +54,8 @@ enum {
   SLICE_ESTALE = -4,   /* paged_decode of a layer whose prefetch for this batch is not valid     */
   SLICE_ECUDA = -5,    /* a CUDA call failed; slice_stats reports the code                       */
   SLICE_ETIMEOUT = -6, /* a bounded device-side wait expired (reported through slice_stats)      */
-  SLICE_ESTATE = -7    /* unknown sequence, double free                                          */
+  SLICE_ESTATE = -7,   /* unknown sequence, double free                                          */
+  SLICE_ESCRATCH = -8  /* paged_decode_noalloc: the batch needs more than the static scratch array */
 };
 
 enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
@@ -152,6 +153,28 @@ int prefetch_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nse
  * this layer for this batch and table state), ECUDA. */
 int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
                  uint32_t num_q_heads, float sm_scale, void* out, float* lse_or_null, void* stream);
+
+/* The paper has no counterpart to this entry point; it exists for callers that must not cause a
+ * device memory allocation when they run attention. paged_decode obtains its split-KV scratch from
+ * cudaMalloc on its first call (and again if a later call needs more). That is unusable for a server
+ * that gave every byte of the GPU to its KV-cache pool at start-up, for a decode loop that cannot
+ * tolerate the device-wide synchronisation an allocation brings, and under rules that forbid
+ * allocator calls once initialisation is over. paged_decode_noalloc takes the same arguments,
+ * computes the same result and orders itself on the streams the same way, but keeps the scratch in a
+ * static device array built into the library: 8 MiB per GPU, held by every GPU that loads the
+ * library until the process exits. It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   Limit: (segments of the batch) * num_q_heads * 528 bytes (rounded up to 256-byte pieces) must
+ *   fit in 8 MiB, where segments <= nseq + attention CTAs; larger requests return SLICE_ESCRATCH
+ *   and change nothing.
+ *   First call on a device: looks up the array's device address (one-time set-up for that device,
+ *   done with that device current). Make that first call outside any stream capture.
+ *   Sharing: all calls, from every slice in the process, use the one array, and it keeps the last
+ *   call's contents (nothing in it needs clearing: each call overwrites what it later reads). Two
+ *   calls whose kernels may overlap on the GPU (different streams without an ordering between them)
+ *   race on it; issue them on one stream or order them with events.
+ * Errors: as paged_decode, plus SLICE_ESCRATCH. */
+int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
+                         uint32_t num_q_heads, float sm_scale, void* out, float* lse_or_null, void* stream);
 
 /* Section 4.1: the lender regains capacity immediately. The paper reclaims by preempting the
  * borrower's requests; this entry migrates instead. The top `take_blocks` ids of the lent range

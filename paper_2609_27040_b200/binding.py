@@ -16,7 +16,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libemaslice.so")
 
-OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE = 0, -1, -2, -3, -4, -5, -6, -7
+OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
 FLAG_PROFILE, FLAG_NULL_DEVICE = 1, 4
 COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
@@ -26,7 +26,7 @@ EXPORTS = [
     "slice_create", "slice_destroy", "slice_alloc_blocks", "slice_set_seq_len", "slice_free_seq",
     "slice_get_block_table", "slice_get_free_stack", "prefetch_layer", "paged_decode", "slice_reclaim",
     "slice_lend", "slice_append_kv", "slice_writeback_layer", "slice_decode_step", "slice_stats",
-    "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror",
+    "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc",
 ]
 
 
@@ -81,6 +81,7 @@ def lib() -> C.CDLL:
         L.slice_get_free_stack.argtypes = [vp, i32, vp, u32, vp]
         L.prefetch_layer.argtypes = [vp, u32, vp, u32, vp]
         L.paged_decode.argtypes = [vp, u32, vp, u32, vp, u32, C.c_float, vp, vp, vp]
+        L.paged_decode_noalloc.argtypes = [vp, u32, vp, u32, vp, u32, C.c_float, vp, vp, vp]
         L.slice_reclaim.argtypes = [vp, u32, vp, vp]
         L.slice_lend.argtypes = [vp, u32]
         L.slice_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, vp]
@@ -217,6 +218,15 @@ class Slice:
         sq = _seqs(seqs)
         return lib().paged_decode(self._h, layer, _ptr(sq), len(sq), _ptr(q), num_q_heads, sm_scale,
                                   _ptr(out), _ptr(lse), _stream(stream))
+
+    def paged_decode_noalloc(self, layer: int, seqs, q, num_q_heads: int, sm_scale: float, out, lse=None,
+                             stream=None) -> int:
+        """paged_decode for callers that must not allocate device memory: same arguments and result,
+        scratch in the library's static 8 MiB device array (see include/emaslice.h for the limit, the
+        one-time set-up on the first call per device, and the rule against overlapping calls)."""
+        sq = _seqs(seqs)
+        return lib().paged_decode_noalloc(self._h, layer, _ptr(sq), len(sq), _ptr(q), num_q_heads, sm_scale,
+                                          _ptr(out), _ptr(lse), _stream(stream))
 
     def slice_reclaim(self, take_blocks: int = TAKE_ALL, stream=None):
         mig = C.c_uint64(0)

@@ -70,6 +70,12 @@ cudaError_t decode_setup();
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const DecodeParams& p, cudaStream_t stream);
 
+// noalloc.cu: the same two launches with the partials in a static device array (part_o / part_ml
+// of p are ignored). static_scratch_needed() > static_scratch_bytes() must be rejected by the caller.
+size_t static_scratch_bytes();
+size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq);
+cudaError_t launch_decode_static(DecodeParams p, cudaStream_t stream);
+
 struct AppendParams {
   uint8_t* local_layer;        // this layer's local arena
   uint64_t local_block_stride;

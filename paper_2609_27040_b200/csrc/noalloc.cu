@@ -1,0 +1,75 @@
+// noalloc.cu — attention launch whose split-KV scratch lives in a static device array.
+//
+// paged_decode keeps the partial results of its split-KV segments in a buffer that it obtains from
+// cudaMalloc the first time it is called (and again when a later call needs a larger one). Some
+// callers must not trigger a device allocation at that point: a serving engine that has handed
+// all of the GPU's memory to its KV-cache pool at start-up (a late cudaMalloc would fail), a
+// latency-critical decode loop that cannot afford the device-wide synchronisation an allocation
+// implies, or code running under a policy that forbids allocator calls after initialisation.
+// For them this file provides the same two launches with the scratch placed in a file-scope
+// `static __device__` array of fixed size.
+//
+// The array occupies kStaticScratchBytes on every GPU that loads the library, until the process
+// exits. In host code the array's name is only a host-side stand-in, not a device address, so the
+// address handed to the kernels is looked up with cudaGetSymbolAddress: once per device, on the
+// first call made with that device current. All calls share the one array and it keeps whatever the
+// last call left in it; two calls whose kernels overlap on the GPU would race on it.
+#include "kernels.h"
+
+namespace {
+
+constexpr size_t kStaticScratchBytes = 8u << 20;  // 8 MiB per GPU
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device addresses of g_static_scratch, filled in lazily per device.
+void* g_scratch_addr[kMaxDevices] = {};
+
+inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+namespace ema {
+
+size_t static_scratch_bytes() { return kStaticScratchBytes; }
+
+size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq) {
+  const size_t o_bytes = static_cast<size_t>(nsegs) * Hq * 128 * sizeof(float);
+  const size_t ml_bytes = static_cast<size_t>(nsegs) * Hq * 4 * sizeof(float);
+  return align256(o_bytes) + align256(ml_bytes);
+}
+
+// Set-up for the device that is current: resolves and caches the array's device address.
+cudaError_t static_scratch_address(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+// Attention + merge with the partials in the static array. Nothing in the array has to start at
+// zero: every segment writes its (max, sums, output) rows before the merge reads them, and the
+// merge reads only the rows of this launch's segments. The caller has checked the size.
+cudaError_t launch_decode_static(DecodeParams p, cudaStream_t stream) {
+  void* base = nullptr;
+  cudaError_t e = static_scratch_address(&base);
+  if (e != cudaSuccess) return e;
+  if (static_scratch_needed(p.nsegs, p.Hq) > kStaticScratchBytes) return cudaErrorInvalidValue;
+  const size_t o_bytes = align256(static_cast<size_t>(p.nsegs) * p.Hq * 128 * sizeof(float));
+  p.part_o = static_cast<float*>(base);
+  p.part_ml = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + o_bytes);
+  e = launch_decode(p, stream);
+  if (e != cudaSuccess) return e;
+  return launch_merge(p, stream);
+}
+
+}  // namespace ema

@@ -463,6 +463,59 @@ int do_decode(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq,
   return SLICE_OK;
 }
 
+// Same checks, ordering and launches as do_decode, but the split-KV partials go to the library's
+// static device array: no device memory is obtained or released anywhere on this path.
+int do_decode_static(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out,
+                     float* lse, cudaStream_t stream) {
+  const uint32_t Hkv = s->cfg.num_kv_heads;
+  if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
+  if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
+  const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
+  for (uint32_t i = 0; i < p->nseq; ++i)
+    if (lens[i] == 0) return SLICE_EINVAL;
+  if (ema::static_scratch_needed(p->nsegs, Hq) > ema::static_scratch_bytes()) return SLICE_ESCRATCH;
+  const uint32_t slot = layer % s->cfg.ring_slots;
+  SlotState& sl = s->slots[slot];
+  if (p->k && !(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
+  int rc = ensure_stream(s, stream);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, stream, false);
+  if (rc) return rc;
+  if (!s->null_dev) {
+    if (p->k && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    ema::DecodeParams d{};
+    d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
+    d.local_block_stride = s->local_bs;
+    d.slot_base = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
+    d.block_bytes = s->block_bytes;
+    d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
+    d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
+    d.segs = reinterpret_cast<const Segment*>(p->dev + p->off_segs);
+    d.cta_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_seg);
+    d.seq_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_seq_seg);
+    d.q = q;
+    d.out = out;
+    d.lse = lse;
+    d.nseq = p->nseq;
+    d.nsegs = p->nsegs;
+    d.ncta = p->ncta;
+    d.Hq = Hq;
+    d.Hkv = Hkv;
+    d.G = Hq / Hkv;
+    d.scale_log2 = sm_scale * 1.4426950408889634f;
+    d.status = s->dev_status;
+    CU(s, ema::launch_decode_static(d, stream));
+    s->st.kernel_launches += 2;
+    CU(s, cudaEventRecord(sl.attn_done, stream));
+    sl.attn_recorded = true;
+    rc = mark_used(s, p, stream, false);
+    if (rc) return rc;
+  }
+  s->st.decode_calls++;
+  s->st.decode_tokens += p->tokens;
+  return SLICE_OK;
+}
+
 void destroy_impl(ema_slice* s) {
   if (!s->null_dev) {
     cudaDeviceSynchronize();
@@ -719,6 +772,15 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
   return do_decode(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream));
+}
+
+int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
+                         uint32_t num_q_heads, float sm_scale, void* out, float* lse_or_null, void* stream) {
+  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  Plan* p = nullptr;
+  int rc = get_plan(s, seqs, nseq, &p);
+  if (rc) return rc;
+  return do_decode_static(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream));
 }
 
 int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* stream_v) {
@@ -1050,6 +1112,7 @@ const char* slice_strerror(int code) {
     case SLICE_ECUDA: return "CUDA call failed";
     case SLICE_ETIMEOUT: return "bounded device wait expired";
     case SLICE_ESTATE: return "unknown sequence or bad state";
+    case SLICE_ESCRATCH: return "request exceeds the static scratch array";
     default: return "unknown status";
   }
 }
