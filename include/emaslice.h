@@ -85,9 +85,14 @@ typedef struct {
                                        0..local_blocks-1); NULL = ascending                      */
   const uint32_t* lent_free_order;  /* host; optional permutation of 0..lent_blocks_physical-1;
                                        ids >= lent_blocks are skipped at creation                */
-  uint32_t decode_ctas;           /* 0 = one per SM; CTAs of the attention kernel                */
-  uint32_t copy_ctas;             /* 0 = default; CTAs of the gather / migration kernel          */
+  uint32_t decode_ctas;           /* 0 = one per SM; CTAs of the layer (attention) kernel        */
+  uint32_t copy_ctas;             /* 0 = default; CTAs of the stand-alone gather / migration kernel */
   uint32_t copy_kind;             /* 0 = default, 1 = vector load/store kernel, 2 = bulk-copy ring */
+  uint32_t pipeline_mode;         /* slice_decode_step: 0 = fused (attention of layer l and gather of
+                                     layer l+1 in one launch, one stream), 1 = two kernels on two
+                                     streams ordered by events                                   */
+  uint32_t dynamic_pct;           /* share of the attention blocks handed out dynamically to even out
+                                     SMs: 0 = default (20), 1..99 percent, 100 = fully static     */
   uint32_t reserved;
 } slice_config_t;
 
@@ -148,6 +153,8 @@ int prefetch_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nse
  *   q, out  device, [nseq][num_q_heads][128] bf16;  lse_or_null device, [nseq][num_q_heads] f32
  *           (natural-log sum of exponentials of the scaled scores).
  * Arithmetic: bf16 products, f32 accumulation and softmax, bf16 result (nearest even).
+ * The split-KV partials are merged inside the same launch. Calls on one slice must not overlap on
+ * the GPU (they share the partial buffers): issue them on one stream or order them.
  * Enqueued on stream after the layer's prefetch. Errors: EINVAL (shape, zero-length sequence,
  * G > 8), ESTATE, ESTALE (batch has lent blocks and the slot does not hold a valid prefetch of
  * this layer for this batch and table state), ECUDA. */
@@ -163,13 +170,15 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
  * computes the same result and orders itself on the streams the same way, but keeps the scratch in a
  * static device array built into the library: 8 MiB per GPU, held by every GPU that loads the
  * library until the process exits. It calls no cudaMalloc, cudaFree or other allocating routine.
- *   Limit: (segments of the batch) * num_q_heads * 528 bytes (rounded up to 256-byte pieces) must
- *   fit in 8 MiB, where segments <= nseq + attention CTAs; larger requests return SLICE_ESCRATCH
+ *   Limit: (work items of the batch) * num_q_heads * 528 bytes plus 4 bytes per (sequence, KV head),
+ *   rounded up to 256-byte pieces, must fit in 8 MiB (a work item is a run of blocks of one sequence;
+ *   there are about nseq + CTAs + a few hundred of them); larger requests return SLICE_ESCRATCH
  *   and change nothing.
  *   First call on a device: looks up the array's device address (one-time set-up for that device,
  *   done with that device current). Make that first call outside any stream capture.
  *   Sharing: all calls, from every slice in the process, use the one array, and it keeps the last
- *   call's contents (nothing in it needs clearing: each call overwrites what it later reads). Two
+ *   call's contents (its counters are cleared on the stream before every launch; the partial rows
+ *   need no clearing: each call overwrites what it later reads). Two
  *   calls whose kernels may overlap on the GPU (different streams without an ordering between them)
  *   race on it; issue them on one stream or order them with events.
  * Errors: as paged_decode, plus SLICE_ESCRATCH. */
@@ -201,9 +210,12 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
  * layer for this batch (ESTALE otherwise). */
 int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* stream);
 
-/* One pass of the whole path over a batch: for every layer, prefetch of layer l+1 on side_stream
- * overlapped with attention of layer l on stream (cyclic: the last layer's attention overlaps the
- * prefetch of layer 0 for the next pass when wrap_prefetch != 0).
+/* One pass of the whole path over a batch: for every layer, the prefetch of layer l+1 overlapped
+ * with the attention of layer l (cyclic: the last layer's attention overlaps the prefetch of layer 0
+ * for the next pass when wrap_prefetch != 0). With pipeline_mode 0 and a ring of at least two slots
+ * both run inside one kernel launch per layer on `stream` (side_stream is not used); with
+ * pipeline_mode 1 the gather kernel runs on side_stream and the attention kernel on stream, ordered
+ * by events.
  *   q, out: [num_layers][nseq][num_q_heads][128] bf16; device pointers when io_on_host == 0.
  *   With io_on_host != 0 they are host pointers (pinned for asynchronous copies): q is copied to the
  *   device and out back to the host on `stream`, inside the call's enqueued work, through device
@@ -224,6 +236,14 @@ int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* 
  * attention start, attention end (after the merge), end of the attention kernel proper (before the
  * merge) (host, [num_layers][5] floats; NaN where not recorded). */
 int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers);
+
+/* With SLICE_FLAG_PROFILE: per-CTA times (GPU nanosecond timer) of the most recent launch of each
+ * layer's kernel, as [num_layers][ctas_per_layer][words_per_cta] uint64 on the host; unused entries
+ * are 0. which = 0: layer kernel, 4 words (start, end of the CTA's attention work, end of its copy
+ * work, SM id); which = 1: stand-alone gather kernel, 2 words (start, end). out may be NULL to query
+ * the two sizes. Synchronises the device. */
+int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entries, uint32_t* ctas_per_layer,
+                    uint32_t* words_per_cta);
 
 /* Low-level copy used by the prefetch microbenchmark: n blocks of block_bytes (a multiple of 16
  * bytes, 16-byte aligned addresses) are copied dst_base + dst_idx[i]*block_bytes <-

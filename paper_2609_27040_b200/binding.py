@@ -26,7 +26,7 @@ EXPORTS = [
     "slice_create", "slice_destroy", "slice_alloc_blocks", "slice_set_seq_len", "slice_free_seq",
     "slice_get_block_table", "slice_get_free_stack", "prefetch_layer", "paged_decode", "slice_reclaim",
     "slice_lend", "slice_append_kv", "slice_writeback_layer", "slice_decode_step", "slice_stats",
-    "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc",
+    "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc", "slice_cta_trace",
 ]
 
 
@@ -41,7 +41,8 @@ class SliceConfig(C.Structure):
         ("local_layer_stride", C.c_uint64), ("local_block_stride", C.c_uint64),
         ("lent_layer_stride", C.c_uint64), ("lent_block_stride", C.c_uint64),
         ("local_free_order", C.c_void_p), ("lent_free_order", C.c_void_p),
-        ("decode_ctas", C.c_uint32), ("copy_ctas", C.c_uint32), ("copy_kind", C.c_uint32), ("reserved", C.c_uint32),
+        ("decode_ctas", C.c_uint32), ("copy_ctas", C.c_uint32), ("copy_kind", C.c_uint32),
+        ("pipeline_mode", C.c_uint32), ("dynamic_pct", C.c_uint32), ("reserved", C.c_uint32),
     ]
 
 
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
         L.slice_stats.argtypes = [vp, C.POINTER(SliceStats)]
         L.slice_get_resolved.argtypes = [vp, vp, u32, vp, u32, vp]
         L.slice_layer_times.argtypes = [vp, vp, u32]
+        L.slice_cta_trace.argtypes = [vp, i32, vp, u64, vp, vp]
         L.slice_copy_blocks.argtypes = [vp, vp, vp, vp, u32, u64, u32, u32, vp]
         L.slice_strerror.argtypes = [C.c_int]
         L.slice_strerror.restype = C.c_char_p
@@ -138,7 +140,8 @@ class Slice:
                  lent_blocks_physical: Optional[int] = None, ring_slots: int = 2, max_seqs: int = 256,
                  max_blocks_per_seq: int = 512, head_dim: int = 128, block_tokens: int = 16,
                  lent_kind: int = 0, flags: int = 0, local_free_order=None, lent_free_order=None,
-                 decode_ctas: int = 0, copy_ctas: int = 0, copy_kind: int = 0,
+                 decode_ctas: int = 0, copy_ctas: int = 0, copy_kind: int = 0, pipeline_mode: int = 0,
+                 dynamic_pct: int = 0,
                  local_layer_stride: int = 0, local_block_stride: int = 0,
                  lent_layer_stride: int = 0, lent_block_stride: int = 0):
         cfg = SliceConfig()
@@ -156,6 +159,7 @@ class Slice:
         self._ro = None if lent_free_order is None else np.ascontiguousarray(lent_free_order, np.uint32)
         cfg.local_free_order, cfg.lent_free_order = _ptr(self._lo), _ptr(self._ro)
         cfg.decode_ctas, cfg.copy_ctas, cfg.copy_kind = decode_ctas, copy_ctas, copy_kind
+        cfg.pipeline_mode, cfg.dynamic_pct = pipeline_mode, dynamic_pct
         self.cfg = cfg
         self._keep = (local, lent, staging)       # arenas must outlive the slice
         h = C.c_void_p()
@@ -273,6 +277,21 @@ class Slice:
         if rc != OK:
             raise SliceError(rc, "slice_layer_times")
         return out
+
+
+def _cta_trace(self, which: int) -> np.ndarray:
+    per, words = C.c_uint32(0), C.c_uint32(0)
+    rc = lib().slice_cta_trace(self._h, which, None, 0, C.byref(per), C.byref(words))
+    if rc != OK:
+        raise SliceError(rc, "slice_cta_trace")
+    out = np.zeros((self.num_layers, per.value, words.value), np.uint64)
+    rc = lib().slice_cta_trace(self._h, which, _ptr(out), out.size, C.byref(per), C.byref(words))
+    if rc != OK:
+        raise SliceError(rc, "slice_cta_trace")
+    return out
+
+
+Slice.slice_cta_trace = _cta_trace
 
 
 def slice_copy_blocks(dst, dst_idx, src, src_idx, n: int, block_bytes: int, kind: int = 0, ctas: int = 0,

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libemaslice.so")
-SOURCES = ["slice.cpp", "copy_kernels.cu", "decode_kernels.cu", "noalloc.cu"]
-HEADERS = ["kernels.h", "ptx.cuh", os.path.join("..", "..", "include", "emaslice.h")]
+SOURCES = ["slice.cpp", "copy_kernels.cu", "layer_kernel.cu", "noalloc.cu"]
+HEADERS = ["kernels.h", "ptx.cuh", "attention_tiles.cuh", os.path.join("..", "..", "include", "emaslice.h")]
 
 
 def _nvcc() -> str:

@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(kVecThreads) copy_blocks_vector(const CopyDesc
   const uint32_t vecs = static_cast<uint32_t>(d.block_bytes >> 4);
   const uint32_t pieces = (vecs + kPieceVecs - 1) / kPieceVecs;
   const uint64_t total = static_cast<uint64_t>(d.n) * d.nlayers * pieces;
+  if (d.trace && threadIdx.x == 0) d.trace[2 * blockIdx.x] = ptx::global_timer_ns();
   for (uint64_t w = blockIdx.x; w < total; w += gridDim.x) {
     const uint32_t piece = static_cast<uint32_t>(w % pieces);
     const uint64_t bi = w / pieces;
@@ -55,6 +56,7 @@ __global__ void __launch_bounds__(kVecThreads) copy_blocks_vector(const CopyDesc
       if (v < vecs) dst[v] = r[j];
     }
   }
+  if (d.trace && threadIdx.x == 0) d.trace[2 * blockIdx.x + 1] = ptx::global_timer_ns();
 }
 
 // Bulk ring: stage = 16 KB; kLoadsAhead loads in flight, the remaining stages drain as stores.

@@ -34,10 +34,11 @@ namespace ema {
 
 size_t static_scratch_bytes() { return kStaticScratchBytes; }
 
-size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq) {
+size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq, uint32_t nseq, uint32_t Hkv) {
   const size_t o_bytes = static_cast<size_t>(nsegs) * Hq * 128 * sizeof(float);
   const size_t ml_bytes = static_cast<size_t>(nsegs) * Hq * 4 * sizeof(float);
-  return align256(o_bytes) + align256(ml_bytes);
+  const size_t cnt_bytes = (kLaunchCounters + static_cast<size_t>(nseq) * Hkv) * sizeof(uint32_t);
+  return align256(o_bytes) + align256(ml_bytes) + align256(cnt_bytes);
 }
 
 // Set-up for the device that is current: resolves and caches the array's device address.
@@ -56,20 +57,26 @@ cudaError_t static_scratch_address(void** out) {
   return cudaSuccess;
 }
 
-// Attention + merge with the partials in the static array. Nothing in the array has to start at
-// zero: every segment writes its (max, sums, output) rows before the merge reads them, and the
-// merge reads only the rows of this launch's segments. The caller has checked the size.
-cudaError_t launch_decode_static(DecodeParams p, cudaStream_t stream) {
+// The layer kernel with its partials and counters in the static array. The partial rows need no
+// clearing (every work item writes its row before the merging warp reads it, and only this
+// launch's rows are read); the work and arrival counters must start at zero and may hold anything
+// after an earlier call that failed, so they are cleared on the stream before every launch.
+cudaError_t launch_layer_static(LayerParams p, cudaStream_t stream) {
   void* base = nullptr;
   cudaError_t e = static_scratch_address(&base);
   if (e != cudaSuccess) return e;
-  if (static_scratch_needed(p.nsegs, p.Hq) > kStaticScratchBytes) return cudaErrorInvalidValue;
+  if (static_scratch_needed(p.nsegs, p.Hq, p.nseq, p.Hkv) > kStaticScratchBytes) return cudaErrorInvalidValue;
   const size_t o_bytes = align256(static_cast<size_t>(p.nsegs) * p.Hq * 128 * sizeof(float));
-  p.part_o = static_cast<float*>(base);
-  p.part_ml = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + o_bytes);
-  e = launch_decode(p, stream);
+  const size_t ml_bytes = align256(static_cast<size_t>(p.nsegs) * p.Hq * 4 * sizeof(float));
+  const size_t cnt_bytes = (kLaunchCounters + static_cast<size_t>(p.nseq) * p.Hkv) * sizeof(uint32_t);
+  unsigned char* b = static_cast<unsigned char*>(base);
+  p.part_o = reinterpret_cast<float*>(b);
+  p.part_ml = reinterpret_cast<float*>(b + o_bytes);
+  p.launch_cnt = reinterpret_cast<uint32_t*>(b + o_bytes + ml_bytes);
+  p.merge_cnt = p.launch_cnt + kLaunchCounters;
+  e = cudaMemsetAsync(p.launch_cnt, 0, cnt_bytes, stream);
   if (e != cudaSuccess) return e;
-  return launch_merge(p, stream);
+  return launch_layer(p, stream);
 }
 
 }  // namespace ema

@@ -1,7 +1,7 @@
 // slice.cpp — host side of libemaslice: the slice arena allocator (block tables, free lists,
-// local/lent split), batch plans (resolved tables, copy lists, attention work partition), the
-// stream/event pipeline that overlaps a layer's prefetch with the previous layer's attention,
-// the reclaim planner, and the C ABI declared in include/emaslice.h.
+// local/lent split), batch plans (resolved tables, copy lists, attention work items), the layer
+// pipeline (fused: attention of layer l and gather of layer l+1 in one launch; or two streams with
+// events), the reclaim planner, and the C ABI declared in include/emaslice.h.
 #include "../../include/emaslice.h"
 #include "kernels.h"
 
@@ -15,11 +15,15 @@
 
 namespace {
 
-using ema::Segment;
+using ema::WorkItem;
 
 constexpr int kNumPlans = 4;
+constexpr int kMaxGuards = 4;
 constexpr uint32_t kBlockTokens = 16;
 constexpr uint32_t kHeadDim = 128;
+constexpr uint32_t kTraceCopyCtas = 2048;
+constexpr uint32_t kDefaultDynamicPct = 20;
+constexpr uint32_t kDynChunkMax = 8, kDynChunkMin = 2;
 
 struct Seq {
   std::vector<int32_t> table;
@@ -39,20 +43,24 @@ struct Plan {
   uint64_t serial = 0;   // unique id of this plan
   uint64_t version = 0;  // table version it was built from
   std::vector<int32_t> seqs;
-  uint32_t nseq = 0, total_blocks = 0, k = 0, nsegs = 0, ncta = 0;
+  uint32_t nseq = 0, total_blocks = 0, k = 0, nsegs = 0, grid = 0;
+  uint32_t n_static = 0, n_dyn = 0;
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
-  size_t off_resolved = 0, off_lens = 0, off_copy_src = 0, off_segs = 0, off_cta_seg = 0, off_seq_seg = 0,
+  size_t off_resolved = 0, off_lens = 0, off_copy_src = 0, off_items = 0, off_cta_item = 0, off_seq_seg = 0,
          off_home = 0, off_stage_pos = 0, bytes = 0;
-  // host copies for the test hook
-  std::vector<uint32_t> blk_off;
-  uint8_t* host = nullptr;  // pinned (or plain in null-device mode)
+  std::vector<uint32_t> blk_off;  // host copy for the test hook
+  uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
   uint8_t* dev = nullptr;
   size_t cap = 0;
   bool uploaded = false;
   cudaEvent_t ev_uploaded = nullptr;
-  cudaEvent_t ev_used_main = nullptr, ev_used_side = nullptr;
-  bool used_main = false, used_side = false;
+  cudaStream_t upload_stream = nullptr;
+  // Guards of the device buffer: recorded on every known stream when the plan can no longer be
+  // used; the next upload into the buffer waits for them.
+  cudaEvent_t guard[kMaxGuards] = {};
+  int n_guard = 0;
+  bool guarded = true;
 };
 
 struct SlotState {
@@ -60,6 +68,7 @@ struct SlotState {
   uint32_t layer = 0;
   uint64_t plan_serial = 0;
   bool pref_recorded = false, attn_recorded = false;
+  cudaStream_t pref_stream = nullptr, attn_stream = nullptr;
   cudaEvent_t pref_done = nullptr, attn_done = nullptr;
 };
 
@@ -76,7 +85,8 @@ struct ema_slice {
   uint64_t block_bytes = 0;
   uint64_t local_ls = 0, local_bs = 0, lent_ls = 0, lent_bs = 0, slot_bytes = 0;
   int num_sms = 148;
-  uint32_t ncta_decode = 148;
+  uint32_t ncta = 148;
+  uint32_t dynamic_pct = kDefaultDynamicPct;
   // allocator
   std::vector<int32_t> free_local, free_lent;  // back() pops next
   std::unordered_map<int32_t, Seq> seqs;
@@ -91,9 +101,9 @@ struct ema_slice {
   // device scratch
   float* part_o = nullptr;
   float* part_ml = nullptr;
-  uint32_t part_hq = 0;
+  size_t part_rows = 0;         // partial rows (segments * query heads) currently allocated
+  uint32_t* cnt_dev = nullptr;  // [num_layers][kLaunchCounters], then merge counters [max_seqs * Hkv]
   int* dev_status = nullptr;
-  int* host_status = nullptr;  // pinned
   // reclaim
   int32_t* reclaim_host = nullptr;
   int32_t* reclaim_dev = nullptr;
@@ -103,6 +113,7 @@ struct ema_slice {
   std::vector<StreamEpoch> streams;
   cudaEvent_t append_done = nullptr;
   bool append_pending = false;
+  cudaStream_t append_stream = nullptr;
   cudaEvent_t ev_tmp = nullptr;
   // host io staging for slice_decode_step
   void* io_q = nullptr;
@@ -113,22 +124,29 @@ struct ema_slice {
   std::vector<uint8_t> prof_set;
   cudaEvent_t prof_base = nullptr;
   bool prof_base_set = false;
+  unsigned long long* trace_layer = nullptr;  // [layer][ncta][4]
+  unsigned long long* trace_copy = nullptr;   // [layer][kTraceCopyCtas][2]
   slice_stats_t st{};
 };
 
 namespace {
 
-#define CU(s, call)                                   \
-  do {                                                \
-    cudaError_t e__ = (call);                         \
-    if (e__ != cudaSuccess) {                         \
+#define CU(s, call)                                    \
+  do {                                                 \
+    cudaError_t e__ = (call);                          \
+    if (e__ != cudaSuccess) {                          \
       (s)->st.last_cuda_error = static_cast<int>(e__); \
-      return SLICE_ECUDA;                             \
-    }                                                 \
+      return SLICE_ECUDA;                              \
+    }                                                  \
   } while (0)
 
 inline uint32_t blocks_for(uint32_t len) { return (len + kBlockTokens - 1) / kBlockTokens; }
 
+inline bool multi_stream(const ema_slice* s) { return s->streams.size() > 1; }
+
+// Registers a stream with the slice. A stream seen for the first time waits for everything the
+// slice has enqueued on the streams it already knows (from then on per-operation events order the
+// streams); every stream waits once for the latest reclaim.
 int ensure_stream(ema_slice* s, cudaStream_t stream) {
   if (s->null_dev) return SLICE_OK;
   for (auto& se : s->streams) {
@@ -140,9 +158,19 @@ int ensure_stream(ema_slice* s, cudaStream_t stream) {
       return SLICE_OK;
     }
   }
+  for (auto& se : s->streams) {
+    CU(s, cudaEventRecord(s->ev_tmp, se.stream));
+    CU(s, cudaStreamWaitEvent(stream, s->ev_tmp, 0));
+  }
   if (s->reclaim_recorded) CU(s, cudaStreamWaitEvent(stream, s->reclaim_done, 0));
   s->streams.push_back(StreamEpoch{stream, s->reclaim_epoch});
   return SLICE_OK;
+}
+
+size_t max_items(const ema_slice* s) {
+  const slice_config_t& c = s->cfg;
+  const size_t blocks = static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq;
+  return 2 * static_cast<size_t>(c.max_seqs) + s->ncta + blocks * std::min(s->dynamic_pct, 100u) / 100 / kDynChunkMin + 8;
 }
 
 size_t plan_capacity(const ema_slice* s) {
@@ -151,8 +179,8 @@ size_t plan_capacity(const ema_slice* s) {
   b += align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved (upper bound)
   b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // lens
   b += align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src
-  b += align_up((static_cast<size_t>(c.max_seqs) + s->ncta_decode + 1) * sizeof(Segment), 256);
-  b += align_up((static_cast<size_t>(s->ncta_decode) + 1) * 4, 256);                // cta_seg_off
+  b += align_up(max_items(s) * sizeof(WorkItem), 256);                              // items
+  b += align_up((static_cast<size_t>(s->ncta) + 1) * 4, 256);                       // cta_item_off
   b += align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // seq_seg_off
   b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                      // home, stage_pos
   return b;
@@ -160,7 +188,6 @@ size_t plan_capacity(const ema_slice* s) {
 
 // Validates a batch: known, distinct sequences. Returns OK or the error.
 int check_batch(ema_slice* s, const int32_t* seqs, uint32_t nseq) {
-  if (!seqs && nseq) return SLICE_EINVAL;
   if (nseq == 0 || nseq > s->cfg.max_seqs) return SLICE_EINVAL;
   for (uint32_t i = 0; i < nseq; ++i)
     if (s->seqs.find(seqs[i]) == s->seqs.end()) return SLICE_ESTATE;
@@ -169,6 +196,23 @@ int check_batch(ema_slice* s, const int32_t* seqs, uint32_t nseq) {
     std::sort(tmp.begin(), tmp.end());
     if (std::adjacent_find(tmp.begin(), tmp.end()) != tmp.end()) return SLICE_EINVAL;
   }
+  return SLICE_OK;
+}
+
+// Records the guards of a plan's device buffer on every known stream: all uses of the plan have
+// been enqueued by now, so a later upload into the buffer only has to wait for these events.
+int guard_plan(ema_slice* s, Plan& p) {
+  if (s->null_dev || p.guarded) return SLICE_OK;
+  p.n_guard = 0;
+  if (s->streams.size() > static_cast<size_t>(kMaxGuards)) {
+    CU(s, cudaDeviceSynchronize());
+  } else {
+    for (auto& se : s->streams) {
+      CU(s, cudaEventRecord(p.guard[p.n_guard], se.stream));
+      ++p.n_guard;
+    }
+  }
+  p.guarded = true;
   return SLICE_OK;
 }
 
@@ -196,12 +240,18 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   }
   if (k > s->cfg.staging_blocks_per_slot) return SLICE_ESTAGING;
 
+  // Plans of older table versions can never be used again: guard their buffers now.
+  for (Plan& old : s->plans)
+    if (old.valid && old.version != s->version) {
+      rc = guard_plan(s, old);
+      if (rc) return rc;
+      old.valid = false;
+    }
   Plan& p = s->plans[s->next_plan];
   s->next_plan = (s->next_plan + 1) % kNumPlans;
-  if (!s->null_dev) {
-    // The previous upload from this host buffer must have left it.
-    if (p.uploaded) CU(s, cudaEventSynchronize(p.ev_uploaded));
-  }
+  rc = guard_plan(s, p);  // still current (same version, other batch): guard at recycling time
+  if (rc) return rc;
+  if (!s->null_dev && p.uploaded) CU(s, cudaEventSynchronize(p.ev_uploaded));  // host buffer is free again
   p.valid = false;
   p.serial = ++s->plan_serial;
   p.version = s->version;
@@ -212,24 +262,39 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   p.tokens = tokens;
   p.uploaded = false;
 
-  // Attention work partition: equal contiguous ranges of the flat block list, one per CTA.
-  const uint32_t ncta = s->ncta_decode;
-  uint32_t per = static_cast<uint32_t>((total_blocks + ncta - 1) / ncta);
+  // Attention work items. The flat block list (batch order) is cut into a static region, split
+  // evenly over the CTAs, and a dynamic tail of small chunks that CTAs pull as they run dry; the
+  // chunks shrink towards the end so that all SMs finish together. Items never cross a sequence.
+  const uint32_t ncta = s->ncta;
+  const uint32_t total = p.total_blocks;
+  uint32_t static_total = total;
+  if (s->dynamic_pct < 100 && total >= 4 * ncta)
+    static_total = static_cast<uint32_t>(static_cast<uint64_t>(total) * (100 - s->dynamic_pct) / 100);
+  uint32_t per = (static_total + ncta - 1) / ncta;
   if (per == 0) per = 1;
-  const uint32_t used_cta = static_cast<uint32_t>((total_blocks + per - 1) / per);
-  p.ncta = used_cta;
+  std::vector<uint32_t> cuts;  // flat positions where a new item starts (besides sequence starts)
+  for (uint32_t c = per; c < static_total; c += per) cuts.push_back(c);
+  if (static_total < total) {
+    uint32_t pos = static_total;
+    while (pos < total) {
+      cuts.push_back(pos);
+      const uint32_t rem = total - pos;
+      const uint32_t c = std::max(kDynChunkMin, std::min(kDynChunkMax, rem / ncta));
+      pos += std::min(c, rem);
+    }
+  }
 
   size_t off = 0;
   p.off_resolved = off;
-  off += align_up(static_cast<size_t>(total_blocks) * 4, 256);
+  off += align_up(static_cast<size_t>(total) * 4, 256);
   p.off_lens = off;
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.off_copy_src = off;
   off += align_up(static_cast<size_t>(k) * 4, 256);
-  p.off_segs = off;
-  off += align_up((static_cast<size_t>(nseq) + used_cta + 1) * sizeof(Segment), 256);
-  p.off_cta_seg = off;
-  off += align_up((static_cast<size_t>(used_cta) + 1) * 4, 256);
+  p.off_items = off;
+  off += align_up((cuts.size() + nseq + 1) * sizeof(WorkItem), 256);
+  p.off_cta_item = off;
+  off += align_up((static_cast<size_t>(ncta) + 1) * 4, 256);
   p.off_seq_seg = off;
   off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
   p.off_home = off;
@@ -242,30 +307,37 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   int32_t* resolved = reinterpret_cast<int32_t*>(p.host + p.off_resolved);
   uint32_t* lens = reinterpret_cast<uint32_t*>(p.host + p.off_lens);
   int32_t* copy_src = reinterpret_cast<int32_t*>(p.host + p.off_copy_src);
-  Segment* segs = reinterpret_cast<Segment*>(p.host + p.off_segs);
-  uint32_t* cta_seg = reinterpret_cast<uint32_t*>(p.host + p.off_cta_seg);
+  WorkItem* items = reinterpret_cast<WorkItem*>(p.host + p.off_items);
+  uint32_t* cta_item = reinterpret_cast<uint32_t*>(p.host + p.off_cta_item);
   uint32_t* seq_seg = reinterpret_cast<uint32_t*>(p.host + p.off_seq_seg);
   int32_t* home = reinterpret_cast<int32_t*>(p.host + p.off_home);
   int32_t* stage_pos = reinterpret_cast<int32_t*>(p.host + p.off_stage_pos);
 
   p.blk_off.resize(nseq + 1);
-  uint32_t flat = 0, kk = 0, nsegs = 0, cta = 0;
-  cta_seg[0] = 0;
+  uint32_t flat = 0, kk = 0, nitems = 0;
+  size_t ci = 0;  // next cut
   for (uint32_t i = 0; i < nseq; ++i) {
     const Seq& q = s->seqs[seqs[i]];
     const uint32_t nb = blocks_for(q.len);
     p.blk_off[i] = flat;
     lens[i] = q.len;
-    seq_seg[i] = nsegs;
+    seq_seg[i] = nitems;
     home[i] = 0;
     stage_pos[i] = -1;
     const uint32_t last_b = q.len ? (q.len - 1) / kBlockTokens : 0;
     uint32_t b = 0;
     while (b < nb) {
-      // this CTA's range is [cta*per, (cta+1)*per) in flat block indices
-      const uint32_t cta_end = (cta + 1) * per;
-      const uint32_t take = std::min(nb - b, cta_end - flat);
-      segs[nsegs++] = Segment{i, b, b + take, flat};
+      while (ci < cuts.size() && cuts[ci] <= flat) ++ci;
+      const uint32_t until = ci < cuts.size() ? cuts[ci] : total;
+      const uint32_t take = std::min(nb - b, until - flat);
+      WorkItem& it = items[nitems];
+      it.seq_idx = i;
+      it.blk_begin = b;
+      it.blk_end = b + take;
+      it.flat_begin = flat;
+      it.seg_id = nitems;
+      it.pad[0] = it.pad[1] = it.pad[2] = 0;
+      ++nitems;
       for (uint32_t j = 0; j < take; ++j) {
         const int32_t e = q.table[b + j];
         int32_t r = e;
@@ -282,47 +354,44 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
       }
       b += take;
       flat += take;
-      if (flat == cta_end) {
-        ++cta;
-        cta_seg[cta] = nsegs;
-      }
     }
   }
   p.blk_off[nseq] = flat;
-  seq_seg[nseq] = nsegs;
-  if (cta < used_cta) cta_seg[used_cta] = nsegs;  // last, partly filled range
-  p.nsegs = nsegs;
-  p.valid = true;  // used_main / used_side stay: they guard the device buffer, not the plan
+  seq_seg[nseq] = nitems;
+  p.nsegs = nitems;
+  // Items are in flat order: the static ones come first, grouped by owning CTA.
+  uint32_t n_static = 0;
+  while (n_static < nitems && items[n_static].flat_begin < static_total) ++n_static;
+  p.n_static = n_static;
+  p.n_dyn = nitems - n_static;
+  uint32_t it_idx = 0;
+  for (uint32_t c = 0; c < ncta; ++c) {
+    const uint64_t lo = static_cast<uint64_t>(c) * per;
+    while (it_idx < n_static && items[it_idx].flat_begin < lo) ++it_idx;
+    cta_item[c] = it_idx;
+  }
+  cta_item[ncta] = n_static;
+  const uint32_t used_static = static_cast<uint32_t>((static_total + per - 1) / per);
+  p.grid = (p.n_dyn || p.k) ? ncta : std::max(used_static, 1u);
+  p.guarded = false;
+  p.valid = true;
   s->st.plans_built++;
   *out = &p;
   return SLICE_OK;
 }
 
 // Uploads the plan on `stream` if nobody has yet; otherwise makes `stream` wait for the upload.
-int plan_on_stream(ema_slice* s, Plan* p, cudaStream_t stream, bool is_side) {
+int plan_on_stream(ema_slice* s, Plan* p, cudaStream_t stream) {
   if (s->null_dev) return SLICE_OK;
   if (!p->uploaded) {
-    // The device buffer may still be read by kernels of the plan that lived here before.
-    if (p->used_main) CU(s, cudaStreamWaitEvent(stream, p->ev_used_main, 0));
-    if (p->used_side) CU(s, cudaStreamWaitEvent(stream, p->ev_used_side, 0));
+    for (int g = 0; g < p->n_guard; ++g) CU(s, cudaStreamWaitEvent(stream, p->guard[g], 0));
+    p->n_guard = 0;
     CU(s, cudaMemcpyAsync(p->dev, p->host, p->bytes, cudaMemcpyHostToDevice, stream));
     CU(s, cudaEventRecord(p->ev_uploaded, stream));
     p->uploaded = true;
-  } else {
+    p->upload_stream = stream;
+  } else if (p->upload_stream != stream) {
     CU(s, cudaStreamWaitEvent(stream, p->ev_uploaded, 0));
-  }
-  (void)is_side;
-  return SLICE_OK;
-}
-
-int mark_used(ema_slice* s, Plan* p, cudaStream_t stream, bool is_side) {
-  if (s->null_dev) return SLICE_OK;
-  if (is_side) {
-    CU(s, cudaEventRecord(p->ev_used_side, stream));
-    p->used_side = true;
-  } else {
-    CU(s, cudaEventRecord(p->ev_used_main, stream));
-    p->used_main = true;
   }
   return SLICE_OK;
 }
@@ -340,42 +409,42 @@ int prof_record(ema_slice* s, uint32_t layer, int which, cudaStream_t stream) {
   return SLICE_OK;
 }
 
-int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
-  int rc = ensure_stream(s, side);
-  if (rc) return rc;
-  rc = plan_on_stream(s, p, side, true);
-  if (rc) return rc;
+bool staged(const ema_slice* s, uint32_t layer, const Plan* p) {
+  const SlotState& sl = s->slots[layer % s->cfg.ring_slots];
+  return sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
+}
+
+// Describes the gather of `layer`'s lent blocks into its ring slot.
+void fill_gather(const ema_slice* s, uint32_t layer, const Plan* p, ema::CopyDesc& d) {
   const uint32_t slot = layer % s->cfg.ring_slots;
-  SlotState& sl = s->slots[slot];
+  d = ema::CopyDesc{};
+  d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  d.src_block_stride[0] = d.src_block_stride[1] = s->lent_bs;
+  d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
+  d.dst_block_stride[0] = d.dst_block_stride[1] = s->block_bytes;
+  d.src_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
+  d.dst_entry = nullptr;
+  d.n = p->k;
+  d.nlayers = 1;
+  d.block_bytes = s->block_bytes;
+  d.status = s->dev_status;
+}
+
+// Ordering before a write into ring slot `sl` on `stream`: after the attention that last read
+// it, and after the last append / write-back (which may have written the blocks to be read).
+int order_before_slot_write(ema_slice* s, SlotState& sl, cudaStream_t stream) {
+  if (sl.attn_recorded && sl.attn_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.attn_done, 0));
+  if (s->append_pending && s->append_stream != stream) CU(s, cudaStreamWaitEvent(stream, s->append_done, 0));
+  return SLICE_OK;
+}
+
+int note_slot_written(ema_slice* s, SlotState& sl, uint32_t layer, const Plan* p, cudaStream_t stream) {
   if (!s->null_dev) {
-    if (sl.attn_recorded) CU(s, cudaStreamWaitEvent(side, sl.attn_done, 0));
-    if (s->append_pending) CU(s, cudaStreamWaitEvent(side, s->append_done, 0));
-    rc = prof_record(s, layer, 0, side);
-    if (rc) return rc;
-    if (p->k) {
-      ema::CopyDesc d{};
-      d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base);
-      d.src_block_stride[0] = d.src_block_stride[1] = s->lent_bs;
-      d.src_layer_stride[0] = d.src_layer_stride[1] = 0;
-      d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
-      d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
-      d.dst_block_stride[0] = d.dst_block_stride[1] = s->block_bytes;
-      d.src_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
-      d.dst_entry = nullptr;
-      d.n = p->k;
-      d.nlayers = 1;
-      d.block_bytes = s->block_bytes;
-      d.status = s->dev_status;
-      const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
-      CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, side));
-      s->st.kernel_launches++;
+    if (multi_stream(s)) {
+      CU(s, cudaEventRecord(sl.pref_done, stream));
+      sl.pref_recorded = true;
     }
-    rc = prof_record(s, layer, 1, side);
-    if (rc) return rc;
-    CU(s, cudaEventRecord(sl.pref_done, side));
-    sl.pref_recorded = true;
-    rc = mark_used(s, p, side, true);
-    if (rc) return rc;
+    sl.pref_stream = stream;
   }
   sl.valid = true;
   sl.layer = layer;
@@ -386,133 +455,137 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
   return SLICE_OK;
 }
 
-int ensure_partials(ema_slice* s, uint32_t Hq) {
-  if (s->null_dev || Hq <= s->part_hq) return SLICE_OK;
+// Stand-alone gather of one layer (the copy kernel), used by prefetch_layer and to prime the ring.
+int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
+  int rc = ensure_stream(s, side);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, side);
+  if (rc) return rc;
+  SlotState& sl = s->slots[layer % s->cfg.ring_slots];
+  if (!s->null_dev) {
+    rc = order_before_slot_write(s, sl, side);
+    if (rc) return rc;
+    rc = prof_record(s, layer, 0, side);
+    if (rc) return rc;
+    if (p->k) {
+      ema::CopyDesc d;
+      fill_gather(s, layer, p, d);
+      if (s->trace_copy && (s->cfg.copy_ctas ? s->cfg.copy_ctas : s->num_sms * 8u) <= kTraceCopyCtas)
+        d.trace = s->trace_copy + static_cast<size_t>(layer) * kTraceCopyCtas * 2;
+      const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+      CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, side));
+      s->st.kernel_launches++;
+    }
+    rc = prof_record(s, layer, 1, side);
+    if (rc) return rc;
+  }
+  return note_slot_written(s, sl, layer, p, side);
+}
+
+int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t nsegs) {
+  const size_t rows = static_cast<size_t>(nsegs) * Hq;
+  if (s->null_dev || rows <= s->part_rows) return SLICE_OK;
   if (s->part_o) {
     CU(s, cudaDeviceSynchronize());
     cudaFree(s->part_o);
     cudaFree(s->part_ml);
     s->part_o = s->part_ml = nullptr;
+    s->part_rows = 0;
   }
-  const size_t nseg = static_cast<size_t>(s->cfg.max_seqs) + s->ncta_decode + 1;
-  CU(s, cudaMalloc(&s->part_o, nseg * Hq * kHeadDim * sizeof(float)));
-  CU(s, cudaMalloc(&s->part_ml, nseg * Hq * 4 * sizeof(float)));
-  s->part_hq = Hq;
+  const size_t want = rows + rows / 4 + 64;  // head room: lengths grow from step to step
+  CU(s, cudaMalloc(&s->part_o, want * kHeadDim * sizeof(float)));
+  CU(s, cudaMalloc(&s->part_ml, want * 4 * sizeof(float)));
+  s->part_rows = want;
   return SLICE_OK;
 }
 
-int do_decode(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out,
-              float* lse, cudaStream_t stream) {
+// One launch of the layer kernel: attention of `layer` and, when next_layer >= 0, the gather of
+// next_layer's lent blocks into its ring slot (which must differ from layer's slot).
+int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out, float* lse,
+             cudaStream_t stream, int next_layer, bool static_scratch, bool counters_zeroed) {
   const uint32_t Hkv = s->cfg.num_kv_heads;
+  const uint32_t R = s->cfg.ring_slots;
   if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
   if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
   const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
   for (uint32_t i = 0; i < p->nseq; ++i)
     if (lens[i] == 0) return SLICE_EINVAL;
-  const uint32_t slot = layer % s->cfg.ring_slots;
+  if (static_scratch && ema::static_scratch_needed(p->nsegs, Hq, p->nseq, Hkv) > ema::static_scratch_bytes())
+    return SLICE_ESCRATCH;
+  const uint32_t slot = layer % R;
   SlotState& sl = s->slots[slot];
-  if (p->k && !(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
+  if (p->k && !staged(s, layer, p)) return SLICE_ESTALE;
+  const bool gather = next_layer >= 0 && p->k > 0;
+  if (next_layer >= 0 && static_cast<uint32_t>(next_layer) % R == slot) return SLICE_EINVAL;
   int rc = ensure_stream(s, stream);
   if (rc) return rc;
-  rc = ensure_partials(s, Hq);
+  if (!static_scratch) {
+    rc = ensure_partials(s, Hq, p->nsegs);
+    if (rc) return rc;
+  }
+  rc = plan_on_stream(s, p, stream);
   if (rc) return rc;
-  rc = plan_on_stream(s, p, stream, false);
-  if (rc) return rc;
+  SlotState* nsl = next_layer >= 0 ? &s->slots[static_cast<uint32_t>(next_layer) % R] : nullptr;
   if (!s->null_dev) {
-    if (p->k && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    if (p->k && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    if (gather) {
+      rc = order_before_slot_write(s, *nsl, stream);
+      if (rc) return rc;
+    }
+    uint32_t* launch_cnt = s->cnt_dev + static_cast<size_t>(layer) * ema::kLaunchCounters;
+    if (!static_scratch && !counters_zeroed)
+      CU(s, cudaMemsetAsync(launch_cnt, 0, ema::kLaunchCounters * sizeof(uint32_t), stream));
     rc = prof_record(s, layer, 2, stream);
     if (rc) return rc;
-    ema::DecodeParams d{};
+    ema::LayerParams d{};
     d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
     d.local_block_stride = s->local_bs;
     d.slot_base = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
     d.block_bytes = s->block_bytes;
     d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
     d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
-    d.segs = reinterpret_cast<const Segment*>(p->dev + p->off_segs);
-    d.cta_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_seg);
+    d.items = reinterpret_cast<const WorkItem*>(p->dev + p->off_items);
+    d.cta_item_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_item);
+    d.dyn_begin = p->n_static;
+    d.n_dyn = p->n_dyn;
     d.seq_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_seq_seg);
     d.q = q;
     d.out = out;
     d.lse = lse;
     d.part_o = s->part_o;
     d.part_ml = s->part_ml;
+    d.launch_cnt = launch_cnt;
+    d.merge_cnt = s->cnt_dev + static_cast<size_t>(s->cfg.num_layers) * ema::kLaunchCounters;
     d.nseq = p->nseq;
     d.nsegs = p->nsegs;
-    d.ncta = p->ncta;
+    d.ncta = p->grid;
     d.Hq = Hq;
     d.Hkv = Hkv;
     d.G = Hq / Hkv;
     d.scale_log2 = sm_scale * 1.4426950408889634f;
+    d.has_attention = 1;
+    if (gather) fill_gather(s, static_cast<uint32_t>(next_layer), p, d.copy);
     d.status = s->dev_status;
-    CU(s, ema::launch_decode(d, stream));
+    if (s->trace_layer) d.trace = s->trace_layer + static_cast<size_t>(layer) * s->ncta * 4;
+    if (static_scratch)
+      CU(s, ema::launch_layer_static(d, stream));
+    else
+      CU(s, ema::launch_layer(d, stream));
+    s->st.kernel_launches++;
     rc = prof_record(s, layer, 4, stream);
     if (rc) return rc;
-    CU(s, ema::launch_merge(d, stream));
-    s->st.kernel_launches += 2;
     rc = prof_record(s, layer, 3, stream);
     if (rc) return rc;
     // The slot may be refilled once this attention has read it.
-    CU(s, cudaEventRecord(sl.attn_done, stream));
-    sl.attn_recorded = true;
-    rc = mark_used(s, p, stream, false);
-    if (rc) return rc;
+    if (multi_stream(s)) {
+      CU(s, cudaEventRecord(sl.attn_done, stream));
+      sl.attn_recorded = true;
+    }
+    sl.attn_stream = stream;
   }
   s->st.decode_calls++;
   s->st.decode_tokens += p->tokens;
-  return SLICE_OK;
-}
-
-// Same checks, ordering and launches as do_decode, but the split-KV partials go to the library's
-// static device array: no device memory is obtained or released anywhere on this path.
-int do_decode_static(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out,
-                     float* lse, cudaStream_t stream) {
-  const uint32_t Hkv = s->cfg.num_kv_heads;
-  if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
-  if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
-  const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
-  for (uint32_t i = 0; i < p->nseq; ++i)
-    if (lens[i] == 0) return SLICE_EINVAL;
-  if (ema::static_scratch_needed(p->nsegs, Hq) > ema::static_scratch_bytes()) return SLICE_ESCRATCH;
-  const uint32_t slot = layer % s->cfg.ring_slots;
-  SlotState& sl = s->slots[slot];
-  if (p->k && !(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
-  int rc = ensure_stream(s, stream);
-  if (rc) return rc;
-  rc = plan_on_stream(s, p, stream, false);
-  if (rc) return rc;
-  if (!s->null_dev) {
-    if (p->k && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
-    ema::DecodeParams d{};
-    d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
-    d.local_block_stride = s->local_bs;
-    d.slot_base = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
-    d.block_bytes = s->block_bytes;
-    d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
-    d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
-    d.segs = reinterpret_cast<const Segment*>(p->dev + p->off_segs);
-    d.cta_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_seg);
-    d.seq_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_seq_seg);
-    d.q = q;
-    d.out = out;
-    d.lse = lse;
-    d.nseq = p->nseq;
-    d.nsegs = p->nsegs;
-    d.ncta = p->ncta;
-    d.Hq = Hq;
-    d.Hkv = Hkv;
-    d.G = Hq / Hkv;
-    d.scale_log2 = sm_scale * 1.4426950408889634f;
-    d.status = s->dev_status;
-    CU(s, ema::launch_decode_static(d, stream));
-    s->st.kernel_launches += 2;
-    CU(s, cudaEventRecord(sl.attn_done, stream));
-    sl.attn_recorded = true;
-    rc = mark_used(s, p, stream, false);
-    if (rc) return rc;
-  }
-  s->st.decode_calls++;
-  s->st.decode_tokens += p->tokens;
+  if (next_layer >= 0) return note_slot_written(s, *nsl, static_cast<uint32_t>(next_layer), p, stream);
   return SLICE_OK;
 }
 
@@ -523,8 +596,8 @@ void destroy_impl(ema_slice* s) {
       if (p.host) cudaFreeHost(p.host);
       if (p.dev) cudaFree(p.dev);
       if (p.ev_uploaded) cudaEventDestroy(p.ev_uploaded);
-      if (p.ev_used_main) cudaEventDestroy(p.ev_used_main);
-      if (p.ev_used_side) cudaEventDestroy(p.ev_used_side);
+      for (auto g : p.guard)
+        if (g) cudaEventDestroy(g);
     }
     for (auto& sl : s->slots) {
       if (sl.pref_done) cudaEventDestroy(sl.pref_done);
@@ -533,10 +606,12 @@ void destroy_impl(ema_slice* s) {
     for (auto e : s->prof)
       if (e) cudaEventDestroy(e);
     if (s->prof_base) cudaEventDestroy(s->prof_base);
+    if (s->trace_layer) cudaFree(s->trace_layer);
+    if (s->trace_copy) cudaFree(s->trace_copy);
     if (s->part_o) cudaFree(s->part_o);
     if (s->part_ml) cudaFree(s->part_ml);
+    if (s->cnt_dev) cudaFree(s->cnt_dev);
     if (s->dev_status) cudaFree(s->dev_status);
-    if (s->host_status) cudaFreeHost(s->host_status);
     if (s->reclaim_host) cudaFreeHost(s->reclaim_host);
     if (s->reclaim_dev) cudaFree(s->reclaim_dev);
     if (s->reclaim_done) cudaEventDestroy(s->reclaim_done);
@@ -562,6 +637,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 1 || cfg->dynamic_pct > 100) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
@@ -593,6 +669,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   s->cfg.local_free_order = s->cfg.lent_free_order = nullptr;
   s->null_dev = null_dev;
   s->profile = (cfg->flags & SLICE_FLAG_PROFILE) != 0;
+  s->dynamic_pct = cfg->dynamic_pct ? cfg->dynamic_pct : kDefaultDynamicPct;
   s->block_bytes = bb;
   s->local_bs = cfg->local_block_stride ? cfg->local_block_stride : bb;
   s->local_ls = cfg->local_layer_stride ? cfg->local_layer_stride : bb * cfg->local_blocks;
@@ -610,19 +687,18 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   }
   s->slots.resize(cfg->ring_slots);
 
-  int rc = SLICE_OK;
   auto fail = [&](int code) {
     destroy_impl(s);
     return code;
   };
   if (!null_dev) {
     int dev = 0;
-    cudaDeviceProp prop;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(SLICE_ECUDA);
-    s->num_sms = prop.multiProcessorCount;
-    if (ema::decode_setup() != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+    if (ema::layer_setup() != cudaSuccess) return fail(SLICE_ECUDA);
   }
-  s->ncta_decode = cfg->decode_ctas ? cfg->decode_ctas : static_cast<uint32_t>(s->num_sms);
+  s->ncta = cfg->decode_ctas ? cfg->decode_ctas : static_cast<uint32_t>(s->num_sms);
   const size_t cap = plan_capacity(s);
   for (Plan& p : s->plans) {
     p.cap = cap;
@@ -632,10 +708,9 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     } else {
       if (cudaMallocHost(reinterpret_cast<void**>(&p.host), cap) != cudaSuccess) return fail(SLICE_ECUDA);
       if (cudaMalloc(reinterpret_cast<void**>(&p.dev), cap) != cudaSuccess) return fail(SLICE_ECUDA);
-      if (cudaEventCreateWithFlags(&p.ev_uploaded, cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&p.ev_used_main, cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&p.ev_used_side, cudaEventDisableTiming) != cudaSuccess)
-        return fail(SLICE_ECUDA);
+      if (cudaEventCreateWithFlags(&p.ev_uploaded, cudaEventDisableTiming) != cudaSuccess) return fail(SLICE_ECUDA);
+      for (auto& g : p.guard)
+        if (cudaEventCreateWithFlags(&g, cudaEventDisableTiming) != cudaSuccess) return fail(SLICE_ECUDA);
     }
   }
   if (!null_dev) {
@@ -646,8 +721,11 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     }
     if (cudaMalloc(reinterpret_cast<void**>(&s->dev_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
     if (cudaMemset(s->dev_status, 0, 256) != cudaSuccess) return fail(SLICE_ECUDA);
-    if (cudaMallocHost(reinterpret_cast<void**>(&s->host_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
-    *s->host_status = 0;
+    const size_t cnt_words = static_cast<size_t>(cfg->num_layers) * ema::kLaunchCounters +
+                             static_cast<size_t>(cfg->max_seqs) * cfg->num_kv_heads;
+    if (cudaMalloc(reinterpret_cast<void**>(&s->cnt_dev), cnt_words * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(s->cnt_dev, 0, cnt_words * sizeof(uint32_t)) != cudaSuccess)
+      return fail(SLICE_ECUDA);
     const size_t rl = static_cast<size_t>(std::max(cfg->lent_blocks_physical, 1u)) * 2 * sizeof(int32_t);
     if (cudaMallocHost(reinterpret_cast<void**>(&s->reclaim_host), rl) != cudaSuccess) return fail(SLICE_ECUDA);
     if (cudaMalloc(reinterpret_cast<void**>(&s->reclaim_dev), rl) != cudaSuccess) return fail(SLICE_ECUDA);
@@ -661,9 +739,14 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
       for (auto& e : s->prof)
         if (cudaEventCreate(&e) != cudaSuccess) return fail(SLICE_ECUDA);
       if (cudaEventCreate(&s->prof_base) != cudaSuccess) return fail(SLICE_ECUDA);
+      const size_t tl = static_cast<size_t>(cfg->num_layers) * s->ncta * 4 * sizeof(unsigned long long);
+      const size_t tc = static_cast<size_t>(cfg->num_layers) * kTraceCopyCtas * 2 * sizeof(unsigned long long);
+      if (cudaMalloc(reinterpret_cast<void**>(&s->trace_layer), tl) != cudaSuccess ||
+          cudaMalloc(reinterpret_cast<void**>(&s->trace_copy), tc) != cudaSuccess ||
+          cudaMemset(s->trace_layer, 0, tl) != cudaSuccess || cudaMemset(s->trace_copy, 0, tc) != cudaSuccess)
+        return fail(SLICE_ECUDA);
     }
   }
-  (void)rc;
   *out = s;
   return SLICE_OK;
 }
@@ -771,7 +854,8 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
   Plan* p = nullptr;
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
-  return do_decode(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream));
+  return do_layer(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream), -1, false,
+                  false);
 }
 
 int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
@@ -780,7 +864,8 @@ int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32
   Plan* p = nullptr;
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
-  return do_decode_static(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream));
+  return do_layer(s, layer, p, q, num_q_heads, sm_scale, out, lse_or_null, static_cast<cudaStream_t>(stream), -1, true,
+                  false);
 }
 
 int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* stream_v) {
@@ -898,18 +983,18 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   if (s->null_dev) return SLICE_OK;
   rc = ensure_stream(s, stream);
   if (rc) return rc;
-  rc = plan_on_stream(s, p, stream, false);
+  rc = plan_on_stream(s, p, stream);
   if (rc) return rc;
   const uint32_t slot = layer % s->cfg.ring_slots;
   SlotState& sl = s->slots[slot];
-  const bool staged = sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
-  if (staged && sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  const bool is_staged = staged(s, layer, p);
+  if (is_staged && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
   ema::AppendParams a{};
   a.local_layer = static_cast<uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
   a.local_block_stride = s->local_bs;
   a.lent_layer = static_cast<uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
   a.lent_block_stride = s->lent_bs;
-  a.slot_base = staged ? static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes : nullptr;
+  a.slot_base = is_staged ? static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes : nullptr;
   a.block_bytes = s->block_bytes;
   a.home_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_home);
   a.stage_pos = reinterpret_cast<const int32_t*>(p->dev + p->off_stage_pos);
@@ -921,9 +1006,10 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   a.block_tokens = kBlockTokens;
   CU(s, ema::launch_append(a, stream));
   s->st.kernel_launches++;
-  CU(s, cudaEventRecord(s->append_done, stream));
-  s->append_pending = true;
-  return mark_used(s, p, stream, false);
+  if (multi_stream(s)) CU(s, cudaEventRecord(s->append_done, stream));
+  s->append_pending = multi_stream(s);
+  s->append_stream = stream;
+  return SLICE_OK;
 }
 
 int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* stream_v) {
@@ -934,13 +1020,13 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   if (rc) return rc;
   const uint32_t slot = layer % s->cfg.ring_slots;
   SlotState& sl = s->slots[slot];
-  if (!(sl.valid && sl.layer == layer && sl.plan_serial == p->serial)) return SLICE_ESTALE;
+  if (!staged(s, layer, p)) return SLICE_ESTALE;
   if (s->null_dev || p->k == 0) return SLICE_OK;
   rc = ensure_stream(s, stream);
   if (rc) return rc;
-  rc = plan_on_stream(s, p, stream, false);
+  rc = plan_on_stream(s, p, stream);
   if (rc) return rc;
-  if (sl.pref_recorded) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  if (sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
   ema::CopyDesc d{};
   d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
   d.src_block_stride[0] = d.src_block_stride[1] = s->block_bytes;
@@ -956,9 +1042,10 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, stream));
   s->st.kernel_launches++;
   // A later prefetch of this layer reads the lent arena: it must see the written blocks.
-  CU(s, cudaEventRecord(s->append_done, stream));
-  s->append_pending = true;
-  return mark_used(s, p, stream, false);
+  if (multi_stream(s)) CU(s, cudaEventRecord(s->append_done, stream));
+  s->append_pending = multi_stream(s);
+  s->append_stream = stream;
+  return SLICE_OK;
 }
 
 int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
@@ -969,9 +1056,15 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
   const uint32_t L = s->cfg.num_layers, R = s->cfg.ring_slots;
+  const bool fused = s->cfg.pipeline_mode == 0 && R >= 2;
+  if (fused) side = stream;
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
   const uint8_t* qd = static_cast<const uint8_t*>(q);
   uint8_t* od = static_cast<uint8_t*>(out);
+  if (!s->null_dev) {
+    rc = ensure_stream(s, stream);
+    if (rc) return rc;
+  }
   if (s->profile && !s->null_dev) {
     std::fill(s->prof_set.begin(), s->prof_set.end(), 0);
     CU(s, cudaEventRecord(s->prof_base, stream));
@@ -990,37 +1083,39 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       CU(s, cudaMalloc(&s->io_out, need));
       s->io_bytes = need;
     }
-    rc = ensure_stream(s, stream);
-    if (rc) return rc;
     CU(s, cudaMemcpyAsync(s->io_q, q, need, cudaMemcpyHostToDevice, stream));
     qd = static_cast<const uint8_t*>(s->io_q);
     od = static_cast<uint8_t*>(s->io_out);
   }
-  auto staged = [&](uint32_t layer) {
-    const SlotState& sl = s->slots[layer % R];
-    return sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
-  };
-  if (p->k && !staged(0)) {
+  if (!s->null_dev)  // the work counters of all layers, cleared once per pass
+    CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * ema::kLaunchCounters * sizeof(uint32_t), stream));
+  if (p->k && !staged(s, 0, p)) {
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
   }
   for (uint32_t l = 0; l < L; ++l) {
-    // Layer-boundary check (Section 4.2.2): trigger the next transfer before computing this layer.
+    // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.
+    int next = -1;
     if (p->k) {
-      if (l + 1 < L) {
-        if (!staged(l + 1)) {
-          rc = do_prefetch(s, l + 1, p, side);
-          if (rc) return rc;
-        }
-      } else if (wrap && L > 1 && (L - 1) % R != 0) {
-        rc = do_prefetch(s, 0, p, side);
+      if (l + 1 < L)
+        next = static_cast<int>(l + 1);
+      else if (wrap && L > 1 && (L - 1) % R != 0)
+        next = 0;
+      if (next >= 0 && staged(s, static_cast<uint32_t>(next), p)) next = -1;
+    }
+    if (fused) {
+      rc = do_layer(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream, next, false, true);
+      if (rc) return rc;
+    } else {
+      if (next >= 0) {
+        rc = do_prefetch(s, static_cast<uint32_t>(next), p, side);
         if (rc) return rc;
       }
+      rc = do_layer(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream, -1, false, true);
+      if (rc) return rc;
     }
-    rc = do_decode(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream);
-    if (rc) return rc;
   }
-  if (p->k && wrap && L > 1 && (L - 1) % R == 0) {
+  if (p->k && wrap && L > 1 && (L - 1) % R == 0 && !staged(s, 0, p)) {
     // The last layer shares its ring slot with layer 0: refill it only after that attention.
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
@@ -1061,6 +1156,21 @@ int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* 
       for (uint32_t f = p->blk_off[i]; f < p->blk_off[i + 1]; ++f)
         out[static_cast<size_t>(i) * stride + (f - p->blk_off[i])] = resolved[f];
   }
+  return SLICE_OK;
+}
+
+int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entries, uint32_t* ctas_per_layer,
+                    uint32_t* words_per_cta) {
+  if (!s || !s->profile || s->null_dev || (which != 0 && which != 1)) return SLICE_EINVAL;
+  const uint32_t per = which == 0 ? s->ncta : kTraceCopyCtas;
+  const uint32_t words = which == 0 ? 4 : 2;
+  if (ctas_per_layer) *ctas_per_layer = per;
+  if (words_per_cta) *words_per_cta = words;
+  if (!out) return SLICE_OK;
+  const uint64_t n = static_cast<uint64_t>(s->cfg.num_layers) * per * words;
+  if (cap_entries < n) return SLICE_EINVAL;
+  CU(s, cudaDeviceSynchronize());
+  CU(s, cudaMemcpy(out, which == 0 ? s->trace_layer : s->trace_copy, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
   return SLICE_OK;
 }
 

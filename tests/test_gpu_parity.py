@@ -89,10 +89,11 @@ def test_both_gather_kernels_are_bit_exact(kind):
 
 
 def test_small_decode_grid_and_many_segments():
-    """Few CTAs: each walks many segments; many CTAs per sequence: many partials to merge."""
+    """Few CTAs: each walks many work items; a large dynamic share: many partials to merge; a
+    fully static split: no dynamic items at all."""
     sc = Scenario(GQA4, 6)
-    for ctas in (3, 64):
-        g = _gpu(sc, decode_ctas=ctas)
+    for ctas, dyn in ((3, 0), (64, 0), (2, 60), (7, 100), (0, 90)):
+        g = _gpu(sc, decode_ctas=ctas, dynamic_pct=dyn)
         for layer in range(sc.L):
             _check_layer(sc, g, layer)
 
@@ -251,10 +252,13 @@ def test_copy_blocks_matches_index_select(kind, n, bb):
     assert torch.equal(dst2, src[src_idx.long()])
 
 
-def test_decode_step_pipeline_matches_oracle_for_every_layer():
-    wl = synth.Workload("pipe", 5, 32, 8, 7, 100, 1200, 0.4)
+@pytest.mark.parametrize("mode,layers,dyn", [(0, 5, 0), (1, 5, 0), (0, 4, 50), (1, 4, 100)])
+def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, dyn):
+    """Both pipelines (fused: attention + next layer's gather in one launch; two streams with
+    events), odd and even layer counts on a ring of two, three passes each."""
+    wl = synth.Workload("pipe", layers, 32, 8, 7, 100, 1200, 0.4)
     sc = Scenario(wl, 9)
-    g = _gpu(sc, flags=B.FLAG_PROFILE)
+    g = _gpu(sc, flags=B.FLAG_PROFILE, pipeline_mode=mode, dynamic_pct=dyn, decode_ctas=12)
     seqs = np.asarray(sc.seq_ids, np.int32)
     for rep in range(3):
         g.out.zero_()
@@ -271,6 +275,18 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer():
         assert ok, (layer, max_abs)
     times = g.s.slice_layer_times()
     assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
+    trace = g.s.slice_cta_trace(0)
+    assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 1] >= trace[:, :, 0]).all()
+    # the staged bytes left in the ring are the oracle's
+    from tests.gpu_helpers import to_host
+    for slot in range(wl.ring_slots):
+        layer = [l for l in range(sc.L) if l % wl.ring_slots == slot][-1]
+        if slot == 0 and (sc.L - 1) % wl.ring_slots != 0:
+            layer = 0          # refilled with layer 0 for the next pass
+        if slot == 0 and (sc.L - 1) % wl.ring_slots == 0:
+            layer = 0          # shared slot: refilled after the last attention
+        rc, _, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+        assert (to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
     # host buffers: the same call with pinned host q/out
     qh = g.q.cpu().pin_memory()
     oh = torch.zeros_like(qh).pin_memory()
