@@ -61,7 +61,8 @@ enum {
 enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
 
 enum {
-  SLICE_FLAG_PROFILE = 1u,     /* record timing events per layer (slice_layer_times)            */
+  SLICE_FLAG_PROFILE = 1u,     /* record timing events per layer (slice_layer_times) and CTA traces */
+  SLICE_FLAG_TRACE = 2u,       /* per-CTA traces only (slice_cta_trace), no timing events         */
   SLICE_FLAG_NULL_DEVICE = 4u  /* tables only: no CUDA call is made, no kernel is launched       */
 };
 
@@ -91,8 +92,9 @@ typedef struct {
   uint32_t pipeline_mode;         /* slice_decode_step: 0 = fused (attention of layer l and gather of
                                      layer l+1 in one launch, one stream), 1 = two kernels on two
                                      streams ordered by events                                   */
-  uint32_t dynamic_pct;           /* share of the attention blocks handed out dynamically to even out
-                                     SMs: 0 = default (20), 1..99 percent, 100 = fully static     */
+  uint32_t static_split;          /* attention work split: 0 = each CTA owns a range of blocks and idle
+                                     CTAs steal from the ranges with most left (default); 1 = static
+                                     ranges only                                                  */
   uint32_t reserved;
 } slice_config_t;
 
@@ -170,9 +172,10 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
  * computes the same result and orders itself on the streams the same way, but keeps the scratch in a
  * static device array built into the library: 8 MiB per GPU, held by every GPU that loads the
  * library until the process exits. It calls no cudaMalloc, cudaFree or other allocating routine.
- *   Limit: (work items of the batch) * num_q_heads * 528 bytes plus 4 bytes per (sequence, KV head),
- *   rounded up to 256-byte pieces, must fit in 8 MiB (a work item is a run of blocks of one sequence;
- *   there are about nseq + CTAs + a few hundred of them); larger requests return SLICE_ESCRATCH
+ *   Limit: this entry point splits the work statically (no stealing between CTAs), which needs one
+ *   partial slot per (sequence, CTA range it touches) plus one per sequence, i.e. at most
+ *   2 * nseq + CTAs slots; slots * num_q_heads * 528 bytes plus about 4 bytes per (sequence, KV head)
+ *   and 8 per CTA must fit in 8 MiB; larger requests return SLICE_ESCRATCH
  *   and change nothing.
  *   First call on a device: looks up the array's device address (one-time set-up for that device,
  *   done with that device current). Make that first call outside any stream capture.

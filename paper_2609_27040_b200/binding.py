@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libemaslice.so")
 
 OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
-FLAG_PROFILE, FLAG_NULL_DEVICE = 1, 4
+FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE = 1, 2, 4
 COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
 TAKE_ALL = 0xFFFFFFFF
 
@@ -42,7 +42,7 @@ class SliceConfig(C.Structure):
         ("lent_layer_stride", C.c_uint64), ("lent_block_stride", C.c_uint64),
         ("local_free_order", C.c_void_p), ("lent_free_order", C.c_void_p),
         ("decode_ctas", C.c_uint32), ("copy_ctas", C.c_uint32), ("copy_kind", C.c_uint32),
-        ("pipeline_mode", C.c_uint32), ("dynamic_pct", C.c_uint32), ("reserved", C.c_uint32),
+        ("pipeline_mode", C.c_uint32), ("static_split", C.c_uint32), ("reserved", C.c_uint32),
     ]
 
 
@@ -141,7 +141,7 @@ class Slice:
                  max_blocks_per_seq: int = 512, head_dim: int = 128, block_tokens: int = 16,
                  lent_kind: int = 0, flags: int = 0, local_free_order=None, lent_free_order=None,
                  decode_ctas: int = 0, copy_ctas: int = 0, copy_kind: int = 0, pipeline_mode: int = 0,
-                 dynamic_pct: int = 0,
+                 static_split: int = 0,
                  local_layer_stride: int = 0, local_block_stride: int = 0,
                  lent_layer_stride: int = 0, lent_block_stride: int = 0):
         cfg = SliceConfig()
@@ -159,7 +159,7 @@ class Slice:
         self._ro = None if lent_free_order is None else np.ascontiguousarray(lent_free_order, np.uint32)
         cfg.local_free_order, cfg.lent_free_order = _ptr(self._lo), _ptr(self._ro)
         cfg.decode_ctas, cfg.copy_ctas, cfg.copy_kind = decode_ctas, copy_ctas, copy_kind
-        cfg.pipeline_mode, cfg.dynamic_pct = pipeline_mode, dynamic_pct
+        cfg.pipeline_mode, cfg.static_split = pipeline_mode, static_split
         self.cfg = cfg
         self._keep = (local, lent, staging)       # arenas must outlive the slice
         h = C.c_void_p()

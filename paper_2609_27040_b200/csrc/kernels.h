@@ -35,21 +35,17 @@ enum CopyKind : uint32_t { kCopyDefault = 0, kCopyVector = 1, kCopyBulk = 2 };
 // Launches one copy kernel on `stream`. ctas == 0 picks a default grid. Returns the CUDA error.
 cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num_sms, cudaStream_t stream);
 
-// One unit of attention work: blocks [blk_begin, blk_end) of batch position seq_idx. Its partial
-// result goes to slot seg_id (slots of one sequence are contiguous).
-struct WorkItem {
-  uint32_t seq_idx;
-  uint32_t blk_begin;
-  uint32_t blk_end;
-  uint32_t flat_begin;  // index of blk_begin in the batch's flat resolved table
-  uint32_t seg_id;
-  uint32_t pad[3];
-};
-
-// Device counters of one layer-kernel launch (must be zero when the kernel starts).
-//   [0] next dynamic attention item, [1] next copy unit; merge_cnt[seq * Hkv + g] counts the
-//   finished segments of a (sequence, KV head) and is reset by the warp that merges.
-constexpr uint32_t kLaunchCounters = 16;  // uint32 words reserved per launch for [0], [1]
+// Device counters of one layer-kernel launch; the whole block must be zero when the kernel
+// starts. Layout in uint32 words:
+//   [0, 16)                         launch words: [1] = next copy unit
+//   [16, 16 + 2*ncta)               one 64-bit claim word per CTA range: blocks claimed from the front
+//                                   (low half, by the owner) and from the back (high half, by thieves)
+//   [.., + nseq)                    partial slots handed out per sequence
+//   [.., + nseq*Hkv)                blocks finished per (sequence, KV head)
+constexpr uint32_t kLaunchCounters = 16;
+inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
+  return kLaunchCounters + 2 * static_cast<size_t>(ncta) + nseq + static_cast<size_t>(nseq) * Hkv;
+}
 
 struct LayerParams {
   // attention of one layer over one batch
@@ -57,20 +53,22 @@ struct LayerParams {
   uint64_t local_block_stride;
   const uint8_t* slot_base;     // ring slot that holds this layer's staged blocks
   uint64_t block_bytes;
-  const int32_t* resolved;      // flat resolved table of the batch
+  const int32_t* resolved;      // flat resolved table of the batch (batch order, then block order)
   const uint32_t* lens;         // [nseq] tokens
-  const WorkItem* items;        // static items grouped by CTA, then the dynamic items
-  const uint32_t* cta_item_off; // [ncta + 1] static items of each CTA
-  uint32_t dyn_begin, n_dyn;    // dynamic items: items[dyn_begin .. dyn_begin + n_dyn)
-  const uint32_t* seq_seg_off;  // [nseq + 1] partial slots of each sequence
+  const uint32_t* blk_seq;      // [total_blocks] batch position of each flat block
+  const uint32_t* blk_off;      // [nseq + 1] first flat block of each sequence
+  const uint32_t* seq_slot_base;// [nseq + 1] first partial slot of each sequence
+  uint32_t total_blocks;
+  uint32_t per;                 // blocks per CTA range; range c = [c*per, min((c+1)*per, total))
+  uint32_t used_cta;            // number of non-empty ranges
+  uint32_t allow_steal;         // 0: every range is processed by its owner only
   const void* q;                // [nseq][Hq][128] bf16
   void* out;                    // [nseq][Hq][128] bf16
   float* lse;                   // [nseq][Hq] or NULL
-  float* part_o;                // [nsegs][Hq][128] unnormalised partial outputs
-  float* part_ml;               // [nsegs][Hq][4]   max (log2 domain), sum as used, exact sum, pad
-  uint32_t* launch_cnt;         // [kLaunchCounters] zeroed before the launch
-  uint32_t* merge_cnt;          // [nseq * Hkv] zero between launches
-  uint32_t nseq, nsegs, ncta;
+  float* part_o;                // [slots][Hq][128] unnormalised partial outputs
+  float* part_ml;               // [slots][Hq][4]   max (log2 domain), sum as used, exact sum, pad
+  uint32_t* counters;           // layer_counter_words(), zeroed before the launch
+  uint32_t nseq, ncta;
   uint32_t Hq, Hkv, G;
   float scale_log2;             // sm_scale * log2(e)
   uint32_t has_attention;       // 0: copy work only
@@ -88,11 +86,11 @@ cudaError_t layer_setup();
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream);
 
 // noalloc.cu: the same launch with partials and counters in a static device array (part_o,
-// part_ml, launch_cnt, merge_cnt of p are ignored). static_scratch_needed() >
-// static_scratch_bytes() must be rejected by the caller.
+// part_ml, counters of p are ignored). static_scratch_needed() > static_scratch_bytes() must be
+// rejected by the caller.
 size_t static_scratch_bytes();
-size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq, uint32_t nseq, uint32_t Hkv);
-cudaError_t launch_layer_static(LayerParams p, cudaStream_t stream);
+size_t static_scratch_needed(uint32_t slots, uint32_t Hq, uint32_t nseq, uint32_t Hkv, uint32_t ncta);
+cudaError_t launch_layer_static(LayerParams p, uint32_t slots, cudaStream_t stream);
 
 struct AppendParams {
   uint8_t* local_layer;        // this layer's local arena

@@ -5,20 +5,30 @@
 // overlap for the whole duration of the layer, with no second kernel to co-schedule, no merge launch
 // and no cross-stream event between layers. With copy.n == 0 it is the plain attention kernel.
 //
+// Work distribution. The batch's blocks, flattened in batch order, are cut into one contiguous range
+// per CTA. A CTA claims blocks from the FRONT of its own range, eight at a time; a CTA whose range is
+// used up steals from the BACK of the range with the most unclaimed blocks (a quarter of what is
+// left, at least two blocks). Both kinds of claim are one atomicAdd on the range's packed 64-bit word
+// (front count | back count), so they can never overlap. SMs stream at visibly different rates
+// (position on the die, mixed read/write traffic), and stealing keeps all of them busy to the end.
+// A CTA keeps one running softmax state per "run" = consecutive claims that belong to the same
+// sequence, so the number of partial results stays close to the number of (CTA, sequence) pairs.
+//
 // Roles inside a CTA (warps):
-//   * producer warp: streams KV blocks of the CTA's work items into a shared-memory ring of half
-//     blocks (K plane / V plane, 16 token rows of Hkv*256 B, each row padded by 16 B so ldmatrix is
+//   * producer warp: claims work and streams KV blocks into a shared-memory ring of half blocks
+//     (K plane / V plane, 16 token rows of Hkv*256 B, each row padded by 16 B so ldmatrix is
 //     bank-conflict free) with untiled TMA bulk copies (cp.async.bulk, one row per lane), completion
-//     by mbarrier expect-tx. Work items: a static share per CTA, then items pulled from a shared
-//     dynamic pool (atomic counter), which evens out SMs that stream at different rates.
+//     by mbarrier expect-tx; a small descriptor queue tells the consumers what each unit is.
 //   * one consumer warp per KV head: tile products on tensor cores when the GQA group is >= 2
 //     (mma.sync m16n8k16 bf16, swapped form), f32 FMAs when G == 1; online softmax with warp
-//     shuffles. Each item emits a partial (max, sums, unnormalised output); the warp that
-//     delivers the last partial of a (sequence, KV head) merges them and writes bf16 (no waiting:
-//     a per-(sequence, head) arrival counter decides).
+//     shuffles. A finished run writes (max, sums, unnormalised output) to a partial slot and adds its
+//     block count to the (sequence, KV head) counter; the warp whose addition completes the sequence
+//     notes a merge; when the CTA's streaming is over its consumer warps share out the noted
+//     merges (the ring is shared by all consumer warps, so a warp that stopped to merge earlier
+//     would stall the whole CTA).
 //   * copy warp: one thread moves 16 KB pieces lent arena -> shared ring -> staging slot with TMA
 //     bulk copies (global->shared on an mbarrier, shared->global in bulk async-groups), pulling
-//     64 KB units from a second atomic counter. No SM lane touches the copied bytes.
+//     64 KB units from an atomic counter. No SM lane touches the copied bytes.
 // Every mbarrier wait is bounded; on expiry the role records SLICE_ETIMEOUT in the status word,
 // gives its own copies in flight a bounded chance to land and returns.
 // HBM-bound: algorithmic bytes per launch = sum_s len_s * 2*Hkv*128*2 (+ q, out, table)
@@ -36,16 +46,27 @@ constexpr int kNA = 4;                     // attention ring: half-block stages
 constexpr int kNC = 5;                     // copy ring: 16 KB stages
 constexpr int kCopyLoadsAhead = 3;         // loads in flight; the other stages drain as stores
 constexpr uint32_t kCopyChunk = 16384;
-constexpr int kQueue = 8;                  // item descriptors in flight (> kNA / 2 + 1)
+constexpr int kQueue = 8;                  // unit descriptors in flight (> kNA / 2 + 1)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
+constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRowPad = 16;
+constexpr uint32_t kOwnChunk = 8;          // blocks an owner claims at a time
+constexpr uint32_t kStealMin = 2, kStealMax = 16;
+constexpr uint32_t kMq = 64;               // merges a CTA can note for the end of its streaming
+constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
 __host__ __device__ constexpr uint32_t row_pitch(uint32_t Hkv) { return row_bytes(Hkv) + kRowPad; }
 __host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_pitch(Hkv); }
 
-struct ItemDesc {
-  uint32_t seq_idx, blk_begin, blk_end, seg_id;
+// A unit: blocks [blk_begin, blk_end) of batch position seq_idx. slot carries the run's partial
+// slot and the kNewRun flag when the unit starts a new run.
+struct UnitDesc {
+  uint32_t seq_idx, blk_begin, blk_end, slot;
+};
+
+struct Claim {
+  uint32_t b, e;  // flat blocks [b, e); empty when b >= e
 };
 
 struct Smem {
@@ -54,22 +75,24 @@ struct Smem {
   uint64_t* att_full;   // [kNA]
   uint64_t* att_empty;  // [kNA]
   uint64_t* copy_full;  // [kNC]
-  ItemDesc* queue;      // [kQueue]
+  UnitDesc* queue;      // [kQueue]
   uint8_t** copy_dst;   // [kNC]
   uint32_t* copy_len;   // [kNC]
+  uint32_t* mq;         // merge list: [kMq] entries, then count, unused, consumer warps done
 };
 
-// Bookkeeping area behind the two rings: 16 mbarrier slots, the item queue, the copy ring's
+// Bookkeeping area behind the two rings: 16 mbarrier slots, the unit queue, the copy ring's
 // destination pointers and lengths; every part 16-byte aligned.
 constexpr size_t kBarBytes = 16 * sizeof(uint64_t);
-constexpr size_t kQueueBytes = kQueue * sizeof(ItemDesc);
+constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
 constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
+constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
 static_assert(2 * kNA + kNC <= 16 && kNC <= 8, "bookkeeping area too small");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
   return static_cast<size_t>(kNA) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
-         kQueueBytes + kCopyDstBytes + kCopyLenBytes;
+         kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv) {
@@ -80,11 +103,20 @@ __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv) {
   s.att_full = reinterpret_cast<uint64_t*>(p);
   s.att_empty = s.att_full + kNA;
   s.copy_full = s.att_empty + kNA;
-  s.queue = reinterpret_cast<ItemDesc*>(p + kBarBytes);
+  s.queue = reinterpret_cast<UnitDesc*>(p + kBarBytes);
   s.copy_dst = reinterpret_cast<uint8_t**>(p + kBarBytes + kQueueBytes);
   s.copy_len = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes);
+  s.mq = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes);
   return s;
 }
+
+__device__ __forceinline__ unsigned long long* range_words(const LayerParams& p) {
+  return reinterpret_cast<unsigned long long*>(p.counters + kLaunchCounters);
+}
+__device__ __forceinline__ uint32_t* seq_counts(const LayerParams& p) {
+  return p.counters + kLaunchCounters + 2 * p.ncta;
+}
+__device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p) { return seq_counts(p) + p.nseq; }
 
 __device__ __forceinline__ const uint8_t* copy_src(const CopyDesc& d, uint32_t i, uint32_t layer) {
   const int32_t e = d.src_entry ? d.src_entry[i] : static_cast<int32_t>(i);
@@ -109,14 +141,17 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t rb = row_bytes(Hkv), pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t plane_bytes = kT * rb;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
-  uint32_t hs = 0, nq = 0;
+  unsigned long long* rw = range_words(p);
+  uint32_t* seq_count = seq_counts(p);
+  uint32_t hs = 0, nq = 0, cur_seq = kSentinel, nruns = 0, nclaims = 0;
   bool ok = true;
 
-  auto stream_item = [&](const WorkItem& it) {
-    const uint32_t nb = it.blk_end - it.blk_begin;
+  // Streams blocks [bb, be) of batch position seq (flat index of bb: flat) as one unit.
+  auto stream_unit = [&](uint32_t seq, uint32_t bb, uint32_t be, uint32_t flat, uint32_t slot_flag) {
+    const uint32_t nb = be - bb;
     for (uint32_t b0 = 0; b0 < nb && ok; b0 += 32) {
       const uint32_t cnt = min(32u, nb - b0);
-      const int32_t my = lane < cnt ? p.resolved[it.flat_begin + b0 + lane] : 0;
+      const int32_t my = lane < cnt ? p.resolved[flat + b0 + lane] : 0;
       for (uint32_t j = 0; j < cnt && ok; ++j) {
         const int32_t e = __shfl_sync(0xffffffffu, my, j);
         const uint8_t* src = e >= 0 ? p.local_layer + static_cast<uint64_t>(e) * p.local_block_stride
@@ -130,7 +165,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
           if (lane == 0) {
             if (b0 + j == 0 && plane == 0) {
-              sm.queue[nq % kQueue] = ItemDesc{it.seq_idx, it.blk_begin, it.blk_end, it.seg_id};
+              sm.queue[nq % kQueue] = UnitDesc{seq, bb, be, slot_flag};
               ++nq;
             }
             ptx::mbar_arrive_expect_tx(full, plane_bytes);
@@ -144,20 +179,108 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     }
   };
 
-  auto fetch_dynamic = [&]() -> uint32_t {
-    uint32_t j = 0;
-    if (lane == 0) j = atomicAdd(&p.launch_cnt[0], 1u);
-    return __shfl_sync(0xffffffffu, j, 0);
+  // Streams a claimed flat range, one unit per sequence it touches. A unit that belongs to another
+  // sequence than the previous one starts a new run and takes the next partial slot of its sequence.
+  auto stream_claim = [&](Claim c) {
+    ++nclaims;
+    uint32_t pos = c.b;
+    while (pos < c.e && ok) {
+      const uint32_t seq = p.blk_seq[pos];
+      const uint32_t seq_lo = p.blk_off[seq], seq_hi = p.blk_off[seq + 1];
+      const uint32_t ue = min(c.e, seq_hi);
+      uint32_t slot_flag = 0;
+      if (seq != cur_seq) {
+        uint32_t k = 0;
+        if (lane == 0) k = atomicAdd(&seq_count[seq], 1u);
+        k = __shfl_sync(0xffffffffu, k, 0);
+        const uint32_t base = p.seq_slot_base[seq], cap = p.seq_slot_base[seq + 1] - base;
+        if (k >= cap) {  // cannot happen with the host's sizing; never write outside the slots
+          if (lane == 0 && p.status) atomicExch(p.status, kDevTimeout - 1);
+          k = cap - 1;
+        }
+        slot_flag = (base + k) | kNewRun;
+        cur_seq = seq;
+        ++nruns;
+      }
+      stream_unit(seq, pos - seq_lo, ue - seq_lo, pos, slot_flag);
+      pos = ue;
+    }
   };
 
-  const uint32_t s0 = p.cta_item_off[blockIdx.x], s1 = p.cta_item_off[blockIdx.x + 1];
-  for (uint32_t i = s0; i < s1 && ok; ++i) stream_item(p.items[i]);
-  if (ok && p.n_dyn) {
-    uint32_t next = fetch_dynamic();
-    while (ok && next < p.n_dyn) {
-      const WorkItem cur = p.items[p.dyn_begin + next];
-      next = fetch_dynamic();  // one ahead: the atomic's latency hides behind this item's blocks
-      stream_item(cur);
+  auto range_len = [&](uint32_t c) { return min(p.per, p.total_blocks - c * p.per); };
+
+  // The owner's claims shrink as its range runs out (a quarter of what the last claim saw left),
+  // so that little claimed-but-unprocessed work is hidden from thieves near the end.
+  uint32_t own_left = 0xFFFFFFFFu;
+  auto claim_front = [&](uint32_t c) -> Claim {
+    const uint32_t want = min(kOwnChunk, max(1u, own_left / 4));
+    unsigned long long old = 0;
+    if (lane == 0) old = atomicAdd(&rw[c], static_cast<unsigned long long>(want));
+    old = __shfl_sync(0xffffffffu, old, 0);
+    const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
+    const uint32_t len = range_len(c);
+    const uint32_t avail_end = b < len ? len - b : 0;
+    if (f >= avail_end) return Claim{0, 0};
+    const uint32_t e = min(f + want, avail_end);
+    own_left = avail_end - e;
+    return Claim{c * p.per + f, c * p.per + e};
+  };
+
+  auto steal = [&]() -> Claim {
+    for (int attempt = 0; attempt < 16; ++attempt) {
+      uint32_t best_rem = 0, best_v = 0;
+      for (uint32_t v = lane; v < p.used_cta; v += 32) {
+        const unsigned long long w = __ldcg(&rw[v]);
+        const uint32_t f = static_cast<uint32_t>(w), b = static_cast<uint32_t>(w >> 32);
+        const uint32_t len = range_len(v);
+        const uint32_t rem = f + b < len ? len - f - b : 0;
+        if (rem > best_rem) {
+          best_rem = rem;
+          best_v = v;
+        }
+      }
+#pragma unroll
+      for (int sh = 16; sh >= 1; sh >>= 1) {
+        const uint32_t r = __shfl_xor_sync(0xffffffffu, best_rem, sh);
+        const uint32_t vv = __shfl_xor_sync(0xffffffffu, best_v, sh);
+        if (r > best_rem || (r == best_rem && vv < best_v)) {
+          best_rem = r;
+          best_v = vv;
+        }
+      }
+      if (best_rem == 0) return Claim{0, 0};
+      const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / 4));
+      unsigned long long old = 0;
+      if (lane == 0) old = atomicAdd(&rw[best_v], static_cast<unsigned long long>(amount) << 32);
+      old = __shfl_sync(0xffffffffu, old, 0);
+      const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
+      const uint32_t len = range_len(best_v);
+      const uint32_t hi = b < len ? len - b : 0;  // end of what was unclaimed before this steal
+      const uint32_t lo_avail = min(f, hi);
+      if (hi > lo_avail) {
+        const uint32_t lo = hi - lo_avail > amount ? hi - amount : lo_avail;
+        return Claim{best_v * p.per + lo, best_v * p.per + hi};
+      }
+    }
+    return Claim{0, 0};
+  };
+
+  // Own range first (claims run one ahead of the streaming, so the atomic's latency is hidden) ...
+  if (blockIdx.x < p.used_cta) {
+    Claim cur = claim_front(blockIdx.x);
+    while (cur.b < cur.e && ok) {
+      const Claim nxt = claim_front(blockIdx.x);
+      stream_claim(cur);
+      cur = nxt;
+    }
+  }
+  // ... then the back of whichever range has most left.
+  if (ok && p.allow_steal) {
+    Claim cur = steal();
+    while (cur.b < cur.e && ok) {
+      const Claim nxt = steal();
+      stream_claim(cur);
+      cur = nxt;
     }
   }
   if (ok) {
@@ -166,10 +289,11 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
     ok = __all_sync(0xffffffffu, ok);
     if (ok && lane == 0) {
-      sm.queue[nq % kQueue] = ItemDesc{kSentinel, 0, 0, 0};
+      sm.queue[nq % kQueue] = UnitDesc{kSentinel, 0, 0, 0};
       ptx::mbar_arrive(ptx::smem_u32(&sm.att_full[stg]));
     }
   }
+  if (p.trace && lane == 0) p.trace[4 * blockIdx.x + 3] |= (static_cast<unsigned long long>(nruns) << 16) | (static_cast<unsigned long long>(nclaims) << 32);
   if (!ok) {
     // Bounded second chance for copies already issued, so that none lands after the CTA is gone.
     const uint32_t from = hs > static_cast<uint32_t>(kNA) ? hs - kNA : 0;
@@ -179,141 +303,315 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// merge by the last-arriving warp of a (sequence, KV head)
+// merge of a (sequence, KV head): n partial slots starting at s0, all kG query heads at once.
+// Lane groups of 32/kG lanes own one head each; a lane owns 4*kG consecutive dims of that head.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void finish_segment(const LayerParams& p, uint32_t seq, uint32_t g) {
+template <int kG>
+__device__ __forceinline__ void merge_heads(const LayerParams& p, uint32_t seq, uint32_t g, uint32_t s0, uint32_t n) {
+  constexpr uint32_t kLph = 32 / kG;  // lanes per head
+  constexpr int kU = 16 / kG;         // partials in flight per round (16 float4 loads per lane)
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t hh = lane / kLph, j = lane % kLph;
+  const uint32_t h = g * kG + hh;
+  const float* mlh = p.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
+  const float* poh = p.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + j * 4 * kG;
+  const uint64_t ml_step = static_cast<uint64_t>(p.Hq) * 4, po_step = static_cast<uint64_t>(p.Hq) * kD;
+  float M = kNegInf;
+  for (uint32_t s = j; s < n; s += kLph) M = fmaxf(M, __ldcg(mlh + s * ml_step));
+#pragma unroll
+  for (uint32_t sh = 1; sh < kLph; sh <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+  float l = 0.f, le = 0.f;
+  for (uint32_t s = j; s < n; s += kLph) {
+    const float4 ml = __ldcg(reinterpret_cast<const float4*>(mlh + s * ml_step));
+    const float w = ptx::exp2_approx(ml.x - M);
+    l += ml.y * w;
+    le += ml.z * w;
+  }
+#pragma unroll
+  for (uint32_t sh = 1; sh < kLph; sh <<= 1) {
+    l += __shfl_xor_sync(0xffffffffu, l, sh);
+    le += __shfl_xor_sync(0xffffffffu, le, sh);
+  }
+  float4 acc[kG];
+#pragma unroll
+  for (int k = 0; k < kG; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (uint32_t sb = 0; sb < n; sb += kU) {
+    float4 v[kU][kG];
+    float m[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const bool in = sb + u < n;
+      m[u] = in ? __ldcg(mlh + (sb + u) * ml_step) : kNegInf;
+#pragma unroll
+      for (int k = 0; k < kG; ++k)
+        v[u][k] = in ? __ldcg(reinterpret_cast<const float4*>(poh + (sb + u) * po_step + 4 * k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const float w = ptx::exp2_approx(m[u] - M);
+#pragma unroll
+      for (int k = 0; k < kG; ++k) {
+        acc[k].x = fmaf(v[u][k].x, w, acc[k].x);
+        acc[k].y = fmaf(v[u][k].y, w, acc[k].y);
+        acc[k].z = fmaf(v[u][k].z, w, acc[k].z);
+        acc[k].w = fmaf(v[u][k].w, w, acc[k].w);
+      }
+    }
+  }
+  const float inv = 1.f / l;
+  uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
+                                        j * 4 * kG);
+#pragma unroll
+  for (int k = 0; k < kG; ++k)
+    dst[k] = make_uint2(ptx::pack_bf16x2(acc[k].x * inv, acc[k].y * inv), ptx::pack_bf16x2(acc[k].z * inv, acc[k].w * inv));
+  if (p.lse && j == 0) p.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
+}
+
+// The same for any group size, one head after the other (group sizes that are not a power of two).
+__device__ __forceinline__ void merge_heads_serial(const LayerParams& p, uint32_t seq, uint32_t g, uint32_t s0, uint32_t n) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t G = p.G;
+  for (uint32_t hh = 0; hh < G; ++hh) {
+    const uint32_t h = g * G + hh;
+    const float* mlh = p.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
+    const float* poh = p.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + lane * 4;
+    const uint64_t ml_step = static_cast<uint64_t>(p.Hq) * 4, po_step = static_cast<uint64_t>(p.Hq) * kD;
+    float M = kNegInf, l = 0.f, le = 0.f;
+    for (uint32_t s = lane; s < n; s += 32) M = fmaxf(M, __ldcg(mlh + s * ml_step));
+#pragma unroll
+    for (int sh = 1; sh <= 16; sh <<= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+    for (uint32_t s = lane; s < n; s += 32) {
+      const float4 ml = __ldcg(reinterpret_cast<const float4*>(mlh + s * ml_step));
+      const float w = ptx::exp2_approx(ml.x - M);
+      l += ml.y * w;
+      le += ml.z * w;
+    }
+#pragma unroll
+    for (int sh = 1; sh <= 16; sh <<= 1) {
+      l += __shfl_xor_sync(0xffffffffu, l, sh);
+      le += __shfl_xor_sync(0xffffffffu, le, sh);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (uint32_t s = 0; s < n; ++s) {
+      const float w = ptx::exp2_approx(__ldcg(mlh + s * ml_step) - M);
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(poh + s * po_step));
+      acc.x = fmaf(v.x, w, acc.x);
+      acc.y = fmaf(v.y, w, acc.y);
+      acc.z = fmaf(v.z, w, acc.z);
+      acc.w = fmaf(v.w, w, acc.w);
+    }
+    const float inv = 1.f / l;
+    uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
+                                          lane * 4);
+    *dst = make_uint2(ptx::pack_bf16x2(acc.x * inv, acc.y * inv), ptx::pack_bf16x2(acc.z * inv, acc.w * inv));
+    if (p.lse && lane == 0) p.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// end of a run: count its blocks; the warp that completes a (sequence, KV head) merges
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t seq, uint32_t g) {
+  const uint32_t s0 = p.seq_slot_base[seq];
+  const uint32_t n = __ldcg(&seq_counts(p)[seq]);
+  switch (p.G) {
+    case 1: merge_heads<1>(p, seq, g, s0, n); break;
+    case 2: merge_heads<2>(p, seq, g, s0, n); break;
+    case 4: merge_heads<4>(p, seq, g, s0, n); break;
+    case 8: merge_heads<8>(p, seq, g, s0, n); break;
+    default: merge_heads_serial(p, seq, g, s0, n); break;
+  }
+}
+
+// A consumer warp that completes a (sequence, KV head) only notes the merge in a CTA-local list:
+// the ring is shared by all consumer warps, so a warp that stopped to merge would stall the whole
+// CTA. Almost every sequence completes in the last microseconds of the kernel anyway (all ranges
+// finish together), and then all consumer warps of the CTA work through the list in parallel.
+__device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm, uint32_t seq, uint32_t g,
+                                           uint32_t blocks) {
   const uint32_t lane = threadIdx.x & 31u;
   __threadfence();
   __syncwarp();
   uint32_t old = 0;
-  if (lane == 0) old = atomicAdd(&p.merge_cnt[seq * p.Hkv + g], 1u);
+  if (lane == 0) old = atomicAdd(&merge_counts(p)[seq * p.Hkv + g], blocks);
   old = __shfl_sync(0xffffffffu, old, 0);
-  const uint32_t s0 = p.seq_seg_off[seq], s1 = p.seq_seg_off[seq + 1];
-  if (old + 1 != s1 - s0) return;
+  if (old + blocks != p.blk_off[seq + 1] - p.blk_off[seq]) return;
   __threadfence();
-  const uint32_t G = p.G;
-  for (uint32_t hh = 0; hh < G; ++hh) {
-    const uint32_t h = g * G + hh;
-    float M = kNegInf;
-    for (uint32_t s = s0; s < s1; ++s) M = fmaxf(M, __ldcg(p.part_ml + (static_cast<uint64_t>(s) * p.Hq + h) * 4));
-    float l = 0.f, le = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (uint32_t s = s0; s < s1; ++s) {
-      const float4 ml = __ldcg(reinterpret_cast<const float4*>(p.part_ml + (static_cast<uint64_t>(s) * p.Hq + h) * 4));
-      const float wgt = ptx::exp2_approx(ml.x - M);
-      l += ml.y * wgt;
-      le += ml.z * wgt;
-      const float4 v =
-          __ldcg(reinterpret_cast<const float4*>(p.part_o + (static_cast<uint64_t>(s) * p.Hq + h) * kD + lane * 4));
-      acc.x = fmaf(v.x, wgt, acc.x);
-      acc.y = fmaf(v.y, wgt, acc.y);
-      acc.z = fmaf(v.z, wgt, acc.z);
-      acc.w = fmaf(v.w, wgt, acc.w);
-    }
-    const float inv = 1.f / l;
-    const uint32_t lo = ptx::pack_bf16x2(acc.x * inv, acc.y * inv);
-    const uint32_t hi = ptx::pack_bf16x2(acc.z * inv, acc.w * inv);
-    uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
-                                          lane * 4);
-    *dst = make_uint2(lo, hi);
-    if (p.lse && lane == 0) p.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
+  uint32_t t = kMq;
+  if (lane == 0) {
+    t = atomicAdd(&sm.mq[kMq], 1u);
+    if (t < kMq) sm.mq[t] = (seq << 4) | g;
   }
-  if (lane == 0) p.merge_cnt[seq * p.Hkv + g] = 0;  // ready for the next launch
+  t = __shfl_sync(0xffffffffu, t, 0);
+  if (t >= kMq) merge_one(p, seq, g);  // list full: merge right away
+}
+
+// After the CTA's streaming: consumer warp w takes list entries w, w + Hkv, ...
+__device__ __forceinline__ void drain_merges(const LayerParams& p, const Smem& sm, uint32_t w) {
+  const uint32_t lane = threadIdx.x & 31u;
+  if (lane == 0) {
+    __threadfence_block();
+    atomicAdd(&sm.mq[kMq + 2], 1u);
+    // All consumer warps of the CTA must have noted their last merge before the list is read.
+    const uint64_t t0 = ptx::global_timer_ns();
+    while (*reinterpret_cast<volatile uint32_t*>(&sm.mq[kMq + 2]) < p.Hkv) {
+      if (ptx::global_timer_ns() - t0 > 2000000000ull) break;
+      __nanosleep(64);
+    }
+  }
+  __syncwarp();
+  const uint32_t n = min(*reinterpret_cast<volatile uint32_t*>(&sm.mq[kMq]), kMq);
+  __threadfence();
+  for (uint32_t i = w; i < n; i += p.Hkv) {
+    const uint32_t v = *reinterpret_cast<volatile uint32_t*>(&sm.mq[i]);
+    merge_one(p, v >> 4, v & 15u);
+  }
+}
+
+// Waits for the next half-stage; false when the bounded wait expired anywhere in the warp.
+__device__ __forceinline__ bool wait_stage(const LayerParams& p, const Smem& sm, uint32_t hs) {
+  const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[hs % kNA]), (hs / kNA) & 1u, p.status, kDevTimeout);
+  return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void release_stage(const Smem& sm, uint32_t hs) {
+  __syncwarp();
+  if ((threadIdx.x & 31u) == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[hs % kNA]));
 }
 
 // ---------------------------------------------------------------------------------------------
-// consumer warp (= KV head g)
+// consumer warp (= KV head g), tensor-core tiles
 // ---------------------------------------------------------------------------------------------
-template <bool kMma>
-__device__ void consumer_role(const LayerParams& p, const Smem& sm, uint32_t g) {
+__device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv, G = p.G;
   const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
-  uint32_t hs = 0, nseg = 0;
-  for (;;) {
-    {
-      const uint32_t stg = hs % kNA;
-      const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[stg]), (hs / kNA) & 1u, p.status, kDevTimeout);
-      if (!__all_sync(0xffffffffu, ok)) return;
+  const uint32_t n = lane >> 2, tig = lane & 3u, r0 = lane >> 2;
+  uint32_t hs = 0, nunit = 0;
+  bool have_run = false;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, len = 0;
+  SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+  uint32_t qf[8][2];
+  float o[8][4];
+
+  auto emit = [&]() {
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
+      st.l1 += __shfl_xor_sync(0xffffffffu, st.l1, sh);
+      st.e0 += __shfl_xor_sync(0xffffffffu, st.e0, sh);
+      st.e1 += __shfl_xor_sync(0xffffffffu, st.e1, sh);
     }
-    const ItemDesc it = sm.queue[nseg % kQueue];
-    if (it.seq_idx == kSentinel) break;
-    ++nseg;
-    const uint32_t len = p.lens[it.seq_idx];
-    SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
-    if constexpr (kMma) {
+    const uint32_t h0 = 2 * tig, h1 = h0 + 1;
+    float* po = p.part_o + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * kD;
+    float* pml = p.part_ml + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * 4;
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      const uint32_t d = mt * 16 + r0;
+      if (h0 < G) {
+        po[h0 * kD + d] = o[mt][0];
+        po[h0 * kD + d + 8] = o[mt][2];
+      }
+      if (h1 < G) {
+        po[h1 * kD + d] = o[mt][1];
+        po[h1 * kD + d + 8] = o[mt][3];
+      }
+    }
+    if (r0 == 0) {
+      if (h0 < G) *reinterpret_cast<float4*>(pml + h0 * 4) = make_float4(st.m0, st.l0, st.e0, 0.f);
+      if (h1 < G) *reinterpret_cast<float4*>(pml + h1 * 4) = make_float4(st.m1, st.l1, st.e1, 0.f);
+    }
+    finish_run(p, sm, run_seq, g, run_blocks);
+  };
+
+  for (;;) {
+    if (!wait_stage(p, sm, hs)) return;
+    const UnitDesc it = sm.queue[nunit % kQueue];
+    const bool end = it.seq_idx == kSentinel;
+    if (end || (it.slot & kNewRun)) {
+      if (have_run) emit();
+      if (end) break;
+      have_run = true;
+      run_seq = it.seq_idx;
+      run_slot = it.slot & ~kNewRun;
+      run_blocks = 0;
+      len = p.lens[run_seq];
+      st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
-      uint32_t qf[8][2];
-      const uint32_t n = lane >> 2, tig = lane & 3u;
       const uint32_t* qrow =
-          reinterpret_cast<const uint32_t*>(qg + (static_cast<uint64_t>(it.seq_idx) * p.Hq + g * G + (n < G ? n : 0)) * kD);
+          reinterpret_cast<const uint32_t*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g * G + (n < G ? n : 0)) * kD);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         qf[ks][0] = n < G ? qrow[ks * 8 + tig] : 0u;
         qf[ks][1] = n < G ? qrow[ks * 8 + tig + 4] : 0u;
       }
-      float o[8][4];
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
-      for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
-        uint32_t stg = hs % kNA;
-        if (b != it.blk_begin) {
-          const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[stg]), (hs / kNA) & 1u, p.status, kDevTimeout);
-          if (!__all_sync(0xffffffffu, ok)) return;
-        }
-        const uint32_t valid = min(kT, len - b * kT);
-        uint32_t pb0, pb1;
-        float al0, al1;
-        tile_mma_scores(ring + stg * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[stg]));
-        ++hs;
-        stg = hs % kNA;
-        {
-          const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[stg]), (hs / kNA) & 1u, p.status, kDevTimeout);
-          if (!__all_sync(0xffffffffu, ok)) return;
-        }
-        tile_mma_pv(ring + stg * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[stg]));
-        ++hs;
-      }
+    }
+    ++nunit;
+    for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
+      if (b != it.blk_begin && !wait_stage(p, sm, hs)) return;
+      const uint32_t valid = min(kT, len - b * kT);
+      uint32_t pb0, pb1;
+      float al0, al1;
+      tile_mma_scores(ring + (hs % kNA) * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
+      release_stage(sm, hs);
+      ++hs;
+      if (!wait_stage(p, sm, hs)) return;
+      tile_mma_pv(ring + (hs % kNA) * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
+      release_stage(sm, hs);
+      ++hs;
+    }
+    run_blocks += it.blk_end - it.blk_begin;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// consumer warp (= KV head = query head g), f32 tiles for G == 1
+// ---------------------------------------------------------------------------------------------
+__device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t Hkv = p.Hkv;
+  const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
+  const uint32_t head_off = g * kD * 2;
+  const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
+  const uint32_t half = lane & 1u;
+  uint32_t hs = 0, nunit = 0;
+  bool have_run = false;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, len = 0;
+  SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+  float qh[64];  // this lane's half (64 dims) of q as f32
+  float o[4] = {0.f, 0.f, 0.f, 0.f};
+
+  auto emit = [&]() {
 #pragma unroll
-      for (int sh = 4; sh <= 16; sh <<= 1) {
-        st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
-        st.l1 += __shfl_xor_sync(0xffffffffu, st.l1, sh);
-        st.e0 += __shfl_xor_sync(0xffffffffu, st.e0, sh);
-        st.e1 += __shfl_xor_sync(0xffffffffu, st.e1, sh);
-      }
-      const uint32_t r0 = lane >> 2;
-      const uint32_t h0 = 2 * tig, h1 = h0 + 1;
-      float* po = p.part_o + (static_cast<uint64_t>(it.seg_id) * p.Hq + g * G) * kD;
-      float* pml = p.part_ml + (static_cast<uint64_t>(it.seg_id) * p.Hq + g * G) * 4;
-#pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
-        const uint32_t d = mt * 16 + r0;
-        if (h0 < G) {
-          po[h0 * kD + d] = o[mt][0];
-          po[h0 * kD + d + 8] = o[mt][2];
-        }
-        if (h1 < G) {
-          po[h1 * kD + d] = o[mt][1];
-          po[h1 * kD + d + 8] = o[mt][3];
-        }
-      }
-      if (r0 == 0) {
-        if (h0 < G) *reinterpret_cast<float4*>(pml + h0 * 4) = make_float4(st.m0, st.l0, st.e0, 0.f);
-        if (h1 < G) *reinterpret_cast<float4*>(pml + h1 * 4) = make_float4(st.m1, st.l1, st.e1, 0.f);
-      }
-    } else {
-      // G == 1: query head = KV head. Lane keeps its half (64 dims) of q in registers as f32.
-      float qh[64];
-      const uint32_t half = lane & 1u;
+    for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
+    float* po = p.part_o + (static_cast<uint64_t>(run_slot) * p.Hq + g) * kD;
+    *reinterpret_cast<float4*>(po + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
+    if (lane == 0)
+      *reinterpret_cast<float4*>(p.part_ml + (static_cast<uint64_t>(run_slot) * p.Hq + g) * 4) =
+          make_float4(st.m0, st.l0, st.l0, 0.f);
+    finish_run(p, sm, run_seq, g, run_blocks);
+  };
+
+  for (;;) {
+    if (!wait_stage(p, sm, hs)) return;
+    const UnitDesc it = sm.queue[nunit % kQueue];
+    const bool end = it.seq_idx == kSentinel;
+    if (end || (it.slot & kNewRun)) {
+      if (have_run) emit();
+      if (end) break;
+      have_run = true;
+      run_seq = it.seq_idx;
+      run_slot = it.slot & ~kNewRun;
+      run_blocks = 0;
+      len = p.lens[run_seq];
+      st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
       const uint4* qrow =
-          reinterpret_cast<const uint4*>(qg + (static_cast<uint64_t>(it.seq_idx) * p.Hq + g) * kD + half * 64);
+          reinterpret_cast<const uint4*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g) * kD + half * 64);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const uint4 v = qrow[c];
@@ -324,38 +622,22 @@ __device__ void consumer_role(const LayerParams& p, const Smem& sm, uint32_t g) 
           qh[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
         }
       }
-      float o[4] = {0.f, 0.f, 0.f, 0.f};
-      for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
-        uint32_t stg = hs % kNA;
-        if (b != it.blk_begin) {
-          const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[stg]), (hs / kNA) & 1u, p.status, kDevTimeout);
-          if (!__all_sync(0xffffffffu, ok)) return;
-        }
-        const uint32_t valid = min(kT, len - b * kT);
-        float pw, al;
-        tile_alu_scores(sm.att_ring + stg * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[stg]));
-        ++hs;
-        stg = hs % kNA;
-        {
-          const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[stg]), (hs / kNA) & 1u, p.status, kDevTimeout);
-          if (!__all_sync(0xffffffffu, ok)) return;
-        }
-        tile_alu_pv(sm.att_ring + stg * hsb, pitch, head_off, valid, pw, al, o);
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[stg]));
-        ++hs;
-      }
-#pragma unroll
-      for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
-      float* po = p.part_o + (static_cast<uint64_t>(it.seg_id) * p.Hq + g) * kD;
-      *reinterpret_cast<float4*>(po + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
-      if (lane == 0)
-        *reinterpret_cast<float4*>(p.part_ml + (static_cast<uint64_t>(it.seg_id) * p.Hq + g) * 4) =
-            make_float4(st.m0, st.l0, st.l0, 0.f);
+      o[0] = o[1] = o[2] = o[3] = 0.f;
     }
-    finish_segment(p, it.seq_idx, g);
+    ++nunit;
+    for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
+      if (b != it.blk_begin && !wait_stage(p, sm, hs)) return;
+      const uint32_t valid = min(kT, len - b * kT);
+      float pw, al;
+      tile_alu_scores(sm.att_ring + (hs % kNA) * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
+      release_stage(sm, hs);
+      ++hs;
+      if (!wait_stage(p, sm, hs)) return;
+      tile_alu_pv(sm.att_ring + (hs % kNA) * hsb, pitch, head_off, valid, pw, al, o);
+      release_stage(sm, hs);
+      ++hs;
+    }
+    run_blocks += it.blk_end - it.blk_begin;
   }
 }
 
@@ -377,7 +659,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   // Issues the load of the next 16 KB piece, pulling a new 64 KB unit when the current one is used up.
   auto issue_next = [&]() -> bool {
     if (piece == pieces) {
-      const uint32_t unit = atomicAdd(&p.launch_cnt[1], 1u);
+      const uint32_t unit = atomicAdd(&p.counters[1], 1u);
       if (unit >= n_units) return false;
       const uint32_t i = unit % d.n, layer = unit / d.n;
       src_blk = copy_src(d, i, layer);
@@ -438,11 +720,20 @@ __global__ void __launch_bounds__(320, 1) slice_layer_kernel(const LayerParams p
       ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), p.Hkv);
     }
     for (int s = 0; s < kNC; ++s) ptx::mbar_init(ptx::smem_u32(&sm.copy_full[s]), 1);
+    for (uint32_t s = 0; s < kMq; ++s) sm.mq[s] = kMqEmpty;
+    sm.mq[kMq] = sm.mq[kMq + 1] = sm.mq[kMq + 2] = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
   if (warp < p.Hkv) {
-    if (p.has_attention) consumer_role<kMma>(p, sm, warp);
+    if (p.has_attention) {
+      if constexpr (kMma)
+        consumer_mma(p, sm, warp);
+      else
+        consumer_alu(p, sm, warp);
+      __syncwarp();
+      drain_merges(p, sm, warp);
+    }
     if (p.trace && warp == 0 && lane == 0) p.trace[4 * blockIdx.x + 1] = ptx::global_timer_ns();
   } else if (warp == p.Hkv) {
     if (p.has_attention) producer_role(p, sm);

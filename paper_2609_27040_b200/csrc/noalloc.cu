@@ -34,10 +34,10 @@ namespace ema {
 
 size_t static_scratch_bytes() { return kStaticScratchBytes; }
 
-size_t static_scratch_needed(uint32_t nsegs, uint32_t Hq, uint32_t nseq, uint32_t Hkv) {
-  const size_t o_bytes = static_cast<size_t>(nsegs) * Hq * 128 * sizeof(float);
-  const size_t ml_bytes = static_cast<size_t>(nsegs) * Hq * 4 * sizeof(float);
-  const size_t cnt_bytes = (kLaunchCounters + static_cast<size_t>(nseq) * Hkv) * sizeof(uint32_t);
+size_t static_scratch_needed(uint32_t slots, uint32_t Hq, uint32_t nseq, uint32_t Hkv, uint32_t ncta) {
+  const size_t o_bytes = static_cast<size_t>(slots) * Hq * 128 * sizeof(float);
+  const size_t ml_bytes = static_cast<size_t>(slots) * Hq * 4 * sizeof(float);
+  const size_t cnt_bytes = layer_counter_words(ncta, nseq, Hkv) * sizeof(uint32_t);
   return align256(o_bytes) + align256(ml_bytes) + align256(cnt_bytes);
 }
 
@@ -61,20 +61,19 @@ cudaError_t static_scratch_address(void** out) {
 // clearing (every work item writes its row before the merging warp reads it, and only this
 // launch's rows are read); the work and arrival counters must start at zero and may hold anything
 // after an earlier call that failed, so they are cleared on the stream before every launch.
-cudaError_t launch_layer_static(LayerParams p, cudaStream_t stream) {
+cudaError_t launch_layer_static(LayerParams p, uint32_t slots, cudaStream_t stream) {
   void* base = nullptr;
   cudaError_t e = static_scratch_address(&base);
   if (e != cudaSuccess) return e;
-  if (static_scratch_needed(p.nsegs, p.Hq, p.nseq, p.Hkv) > kStaticScratchBytes) return cudaErrorInvalidValue;
-  const size_t o_bytes = align256(static_cast<size_t>(p.nsegs) * p.Hq * 128 * sizeof(float));
-  const size_t ml_bytes = align256(static_cast<size_t>(p.nsegs) * p.Hq * 4 * sizeof(float));
-  const size_t cnt_bytes = (kLaunchCounters + static_cast<size_t>(p.nseq) * p.Hkv) * sizeof(uint32_t);
+  if (static_scratch_needed(slots, p.Hq, p.nseq, p.Hkv, p.ncta) > kStaticScratchBytes) return cudaErrorInvalidValue;
+  const size_t o_bytes = align256(static_cast<size_t>(slots) * p.Hq * 128 * sizeof(float));
+  const size_t ml_bytes = align256(static_cast<size_t>(slots) * p.Hq * 4 * sizeof(float));
+  const size_t cnt_bytes = layer_counter_words(p.ncta, p.nseq, p.Hkv) * sizeof(uint32_t);
   unsigned char* b = static_cast<unsigned char*>(base);
   p.part_o = reinterpret_cast<float*>(b);
   p.part_ml = reinterpret_cast<float*>(b + o_bytes);
-  p.launch_cnt = reinterpret_cast<uint32_t*>(b + o_bytes + ml_bytes);
-  p.merge_cnt = p.launch_cnt + kLaunchCounters;
-  e = cudaMemsetAsync(p.launch_cnt, 0, cnt_bytes, stream);
+  p.counters = reinterpret_cast<uint32_t*>(b + o_bytes + ml_bytes);
+  e = cudaMemsetAsync(p.counters, 0, cnt_bytes, stream);
   if (e != cudaSuccess) return e;
   return launch_layer(p, stream);
 }

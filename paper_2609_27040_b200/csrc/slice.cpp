@@ -15,15 +15,12 @@
 
 namespace {
 
-using ema::WorkItem;
-
 constexpr int kNumPlans = 4;
 constexpr int kMaxGuards = 4;
 constexpr uint32_t kBlockTokens = 16;
 constexpr uint32_t kHeadDim = 128;
 constexpr uint32_t kTraceCopyCtas = 2048;
-constexpr uint32_t kDefaultDynamicPct = 20;
-constexpr uint32_t kDynChunkMax = 8, kDynChunkMin = 2;
+constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must match the kernel)
 
 struct Seq {
   std::vector<int32_t> table;
@@ -43,12 +40,13 @@ struct Plan {
   uint64_t serial = 0;   // unique id of this plan
   uint64_t version = 0;  // table version it was built from
   std::vector<int32_t> seqs;
-  uint32_t nseq = 0, total_blocks = 0, k = 0, nsegs = 0, grid = 0;
-  uint32_t n_static = 0, n_dyn = 0;
+  uint32_t nseq = 0, total_blocks = 0, k = 0;
+  uint32_t per = 1, used_cta = 0;        // attention ranges: range c = [c*per, min((c+1)*per, total))
+  uint32_t slots = 0, slots_static = 0;  // partial slots with / without work stealing
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
-  size_t off_resolved = 0, off_lens = 0, off_copy_src = 0, off_items = 0, off_cta_item = 0, off_seq_seg = 0,
-         off_home = 0, off_stage_pos = 0, bytes = 0;
+  size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_blk_off = 0, off_slot_base = 0,
+         off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
   uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
   uint8_t* dev = nullptr;
@@ -81,12 +79,13 @@ struct StreamEpoch {
 
 struct ema_slice {
   slice_config_t cfg{};
-  bool null_dev = false, profile = false;
+  bool null_dev = false, profile = false, trace = false;
   uint64_t block_bytes = 0;
   uint64_t local_ls = 0, local_bs = 0, lent_ls = 0, lent_bs = 0, slot_bytes = 0;
   int num_sms = 148;
   uint32_t ncta = 148;
-  uint32_t dynamic_pct = kDefaultDynamicPct;
+  bool steal = true;
+  size_t cnt_stride = 0;  // uint32 words of device counters per layer
   // allocator
   std::vector<int32_t> free_local, free_lent;  // back() pops next
   std::unordered_map<int32_t, Seq> seqs;
@@ -167,22 +166,14 @@ int ensure_stream(ema_slice* s, cudaStream_t stream) {
   return SLICE_OK;
 }
 
-size_t max_items(const ema_slice* s) {
-  const slice_config_t& c = s->cfg;
-  const size_t blocks = static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq;
-  return 2 * static_cast<size_t>(c.max_seqs) + s->ncta + blocks * std::min(s->dynamic_pct, 100u) / 100 / kDynChunkMin + 8;
-}
-
 size_t plan_capacity(const ema_slice* s) {
   const slice_config_t& c = s->cfg;
   size_t b = 0;
-  b += align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved (upper bound)
-  b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // lens
-  b += align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src
-  b += align_up(max_items(s) * sizeof(WorkItem), 256);                              // items
-  b += align_up((static_cast<size_t>(s->ncta) + 1) * 4, 256);                       // cta_item_off
-  b += align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // seq_seg_off
-  b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                      // home, stage_pos
+  b += 2 * align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved, blk_seq (upper bound)
+  b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                              // lens
+  b += align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);               // copy_src
+  b += 3 * align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // blk_off, slot bases
+  b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos
   return b;
 }
 
@@ -262,40 +253,32 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   p.tokens = tokens;
   p.uploaded = false;
 
-  // Attention work items. The flat block list (batch order) is cut into a static region, split
-  // evenly over the CTAs, and a dynamic tail of small chunks that CTAs pull as they run dry; the
-  // chunks shrink towards the end so that all SMs finish together. Items never cross a sequence.
+  // Attention work: the flat block list (batch order) is cut into one contiguous range per CTA.
+  // Inside the kernel a CTA claims blocks from the front of its range and, once that is used up,
+  // steals from the back of other ranges; a run of claims within one sequence yields one partial.
+  // Partial slots per sequence are sized for the worst case: every steal takes at least kStealMin
+  // blocks, except one clipped steal and one clipped owner claim per range.
   const uint32_t ncta = s->ncta;
   const uint32_t total = p.total_blocks;
-  uint32_t static_total = total;
-  if (s->dynamic_pct < 100 && total >= 4 * ncta)
-    static_total = static_cast<uint32_t>(static_cast<uint64_t>(total) * (100 - s->dynamic_pct) / 100);
-  uint32_t per = (static_total + ncta - 1) / ncta;
+  uint32_t per = (total + ncta - 1) / ncta;
   if (per == 0) per = 1;
-  std::vector<uint32_t> cuts;  // flat positions where a new item starts (besides sequence starts)
-  for (uint32_t c = per; c < static_total; c += per) cuts.push_back(c);
-  if (static_total < total) {
-    uint32_t pos = static_total;
-    while (pos < total) {
-      cuts.push_back(pos);
-      const uint32_t rem = total - pos;
-      const uint32_t c = std::max(kDynChunkMin, std::min(kDynChunkMax, rem / ncta));
-      pos += std::min(c, rem);
-    }
-  }
+  p.per = per;
+  p.used_cta = (total + per - 1) / per;
 
   size_t off = 0;
   p.off_resolved = off;
+  off += align_up(static_cast<size_t>(total) * 4, 256);
+  p.off_blk_seq = off;
   off += align_up(static_cast<size_t>(total) * 4, 256);
   p.off_lens = off;
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.off_copy_src = off;
   off += align_up(static_cast<size_t>(k) * 4, 256);
-  p.off_items = off;
-  off += align_up((cuts.size() + nseq + 1) * sizeof(WorkItem), 256);
-  p.off_cta_item = off;
-  off += align_up((static_cast<size_t>(ncta) + 1) * 4, 256);
-  p.off_seq_seg = off;
+  p.off_blk_off = off;
+  off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
+  p.off_slot_base = off;
+  off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
+  p.off_slot_base_static = off;
   off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
   p.off_home = off;
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
@@ -305,74 +288,54 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   if (off > p.cap) return SLICE_EINVAL;  // cannot happen: capacity is sized from the maxima
 
   int32_t* resolved = reinterpret_cast<int32_t*>(p.host + p.off_resolved);
+  uint32_t* blk_seq = reinterpret_cast<uint32_t*>(p.host + p.off_blk_seq);
   uint32_t* lens = reinterpret_cast<uint32_t*>(p.host + p.off_lens);
   int32_t* copy_src = reinterpret_cast<int32_t*>(p.host + p.off_copy_src);
-  WorkItem* items = reinterpret_cast<WorkItem*>(p.host + p.off_items);
-  uint32_t* cta_item = reinterpret_cast<uint32_t*>(p.host + p.off_cta_item);
-  uint32_t* seq_seg = reinterpret_cast<uint32_t*>(p.host + p.off_seq_seg);
+  uint32_t* blk_off = reinterpret_cast<uint32_t*>(p.host + p.off_blk_off);
+  uint32_t* slot_base = reinterpret_cast<uint32_t*>(p.host + p.off_slot_base);
+  uint32_t* slot_base_static = reinterpret_cast<uint32_t*>(p.host + p.off_slot_base_static);
   int32_t* home = reinterpret_cast<int32_t*>(p.host + p.off_home);
   int32_t* stage_pos = reinterpret_cast<int32_t*>(p.host + p.off_stage_pos);
 
   p.blk_off.resize(nseq + 1);
-  uint32_t flat = 0, kk = 0, nitems = 0;
-  size_t ci = 0;  // next cut
+  uint32_t flat = 0, kk = 0, slots = 0, slots_static = 0;
   for (uint32_t i = 0; i < nseq; ++i) {
     const Seq& q = s->seqs[seqs[i]];
     const uint32_t nb = blocks_for(q.len);
-    p.blk_off[i] = flat;
+    p.blk_off[i] = blk_off[i] = flat;
     lens[i] = q.len;
-    seq_seg[i] = nitems;
+    slot_base[i] = slots;
+    slot_base_static[i] = slots_static;
+    if (nb) {
+      const uint32_t ranges = (flat + nb - 1) / per - flat / per + 1;
+      slots += nb / kStealMin + 2 * ranges + 2;
+      slots_static += ranges + 1;
+    }
     home[i] = 0;
     stage_pos[i] = -1;
     const uint32_t last_b = q.len ? (q.len - 1) / kBlockTokens : 0;
-    uint32_t b = 0;
-    while (b < nb) {
-      while (ci < cuts.size() && cuts[ci] <= flat) ++ci;
-      const uint32_t until = ci < cuts.size() ? cuts[ci] : total;
-      const uint32_t take = std::min(nb - b, until - flat);
-      WorkItem& it = items[nitems];
-      it.seq_idx = i;
-      it.blk_begin = b;
-      it.blk_end = b + take;
-      it.flat_begin = flat;
-      it.seg_id = nitems;
-      it.pad[0] = it.pad[1] = it.pad[2] = 0;
-      ++nitems;
-      for (uint32_t j = 0; j < take; ++j) {
-        const int32_t e = q.table[b + j];
-        int32_t r = e;
-        if (e < 0) {
-          copy_src[kk] = e;  // negative entry: tier 1 (lent arena), id ~e
-          r = ~static_cast<int32_t>(kk);
-          ++kk;
-        }
-        resolved[flat + j] = r;
-        if (q.len && b + j == last_b) {
-          home[i] = e;
-          stage_pos[i] = e < 0 ? ~r : -1;
-        }
+    for (uint32_t b = 0; b < nb; ++b) {
+      const int32_t e = q.table[b];
+      int32_t r = e;
+      if (e < 0) {
+        copy_src[kk] = e;  // negative entry: tier 1 (lent arena), id ~e
+        r = ~static_cast<int32_t>(kk);
+        ++kk;
       }
-      b += take;
-      flat += take;
+      resolved[flat] = r;
+      blk_seq[flat] = i;
+      if (b == last_b) {
+        home[i] = e;
+        stage_pos[i] = e < 0 ? ~r : -1;
+      }
+      ++flat;
     }
   }
-  p.blk_off[nseq] = flat;
-  seq_seg[nseq] = nitems;
-  p.nsegs = nitems;
-  // Items are in flat order: the static ones come first, grouped by owning CTA.
-  uint32_t n_static = 0;
-  while (n_static < nitems && items[n_static].flat_begin < static_total) ++n_static;
-  p.n_static = n_static;
-  p.n_dyn = nitems - n_static;
-  uint32_t it_idx = 0;
-  for (uint32_t c = 0; c < ncta; ++c) {
-    const uint64_t lo = static_cast<uint64_t>(c) * per;
-    while (it_idx < n_static && items[it_idx].flat_begin < lo) ++it_idx;
-    cta_item[c] = it_idx;
-  }
-  cta_item[ncta] = n_static;
-  const uint32_t used_static = static_cast<uint32_t>((static_total + per - 1) / per);
-  p.grid = (p.n_dyn || p.k) ? ncta : std::max(used_static, 1u);
+  p.blk_off[nseq] = blk_off[nseq] = flat;
+  slot_base[nseq] = slots;
+  slot_base_static[nseq] = slots_static;
+  p.slots = std::max(slots, 1u);
+  p.slots_static = std::max(slots_static, 1u);
   p.guarded = false;
   p.valid = true;
   s->st.plans_built++;
@@ -482,8 +445,8 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
   return note_slot_written(s, sl, layer, p, side);
 }
 
-int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t nsegs) {
-  const size_t rows = static_cast<size_t>(nsegs) * Hq;
+int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots) {
+  const size_t rows = static_cast<size_t>(slots) * Hq;
   if (s->null_dev || rows <= s->part_rows) return SLICE_OK;
   if (s->part_o) {
     CU(s, cudaDeviceSynchronize());
@@ -510,7 +473,8 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
   for (uint32_t i = 0; i < p->nseq; ++i)
     if (lens[i] == 0) return SLICE_EINVAL;
-  if (static_scratch && ema::static_scratch_needed(p->nsegs, Hq, p->nseq, Hkv) > ema::static_scratch_bytes())
+  if (static_scratch &&
+      ema::static_scratch_needed(p->slots_static, Hq, p->nseq, Hkv, s->ncta) > ema::static_scratch_bytes())
     return SLICE_ESCRATCH;
   const uint32_t slot = layer % R;
   SlotState& sl = s->slots[slot];
@@ -520,7 +484,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   int rc = ensure_stream(s, stream);
   if (rc) return rc;
   if (!static_scratch) {
-    rc = ensure_partials(s, Hq, p->nsegs);
+    rc = ensure_partials(s, Hq, p->slots);
     if (rc) return rc;
   }
   rc = plan_on_stream(s, p, stream);
@@ -532,9 +496,9 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
       rc = order_before_slot_write(s, *nsl, stream);
       if (rc) return rc;
     }
-    uint32_t* launch_cnt = s->cnt_dev + static_cast<size_t>(layer) * ema::kLaunchCounters;
+    uint32_t* counters = s->cnt_dev + static_cast<size_t>(layer) * s->cnt_stride;
     if (!static_scratch && !counters_zeroed)
-      CU(s, cudaMemsetAsync(launch_cnt, 0, ema::kLaunchCounters * sizeof(uint32_t), stream));
+      CU(s, cudaMemsetAsync(counters, 0, s->cnt_stride * sizeof(uint32_t), stream));
     rc = prof_record(s, layer, 2, stream);
     if (rc) return rc;
     ema::LayerParams d{};
@@ -544,21 +508,23 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
     d.block_bytes = s->block_bytes;
     d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
     d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
-    d.items = reinterpret_cast<const WorkItem*>(p->dev + p->off_items);
-    d.cta_item_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_cta_item);
-    d.dyn_begin = p->n_static;
-    d.n_dyn = p->n_dyn;
-    d.seq_seg_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_seq_seg);
+    d.blk_seq = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_seq);
+    d.blk_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_off);
+    // Without stealing a sequence needs one slot per range it touches: the compact layout.
+    const bool steal = s->steal && !static_scratch;
+    d.seq_slot_base = reinterpret_cast<const uint32_t*>(p->dev + (steal ? p->off_slot_base : p->off_slot_base_static));
+    d.total_blocks = p->total_blocks;
+    d.per = p->per;
+    d.used_cta = p->used_cta;
+    d.allow_steal = steal ? 1u : 0u;
     d.q = q;
     d.out = out;
     d.lse = lse;
     d.part_o = s->part_o;
     d.part_ml = s->part_ml;
-    d.launch_cnt = launch_cnt;
-    d.merge_cnt = s->cnt_dev + static_cast<size_t>(s->cfg.num_layers) * ema::kLaunchCounters;
+    d.counters = counters;
     d.nseq = p->nseq;
-    d.nsegs = p->nsegs;
-    d.ncta = p->grid;
+    d.ncta = s->ncta;
     d.Hq = Hq;
     d.Hkv = Hkv;
     d.G = Hq / Hkv;
@@ -568,7 +534,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
     d.status = s->dev_status;
     if (s->trace_layer) d.trace = s->trace_layer + static_cast<size_t>(layer) * s->ncta * 4;
     if (static_scratch)
-      CU(s, ema::launch_layer_static(d, stream));
+      CU(s, ema::launch_layer_static(d, p->slots_static, stream));
     else
       CU(s, ema::launch_layer(d, stream));
     s->st.kernel_launches++;
@@ -637,7 +603,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 1 || cfg->dynamic_pct > 100) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 1 || cfg->static_split > 1) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
@@ -669,7 +635,8 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   s->cfg.local_free_order = s->cfg.lent_free_order = nullptr;
   s->null_dev = null_dev;
   s->profile = (cfg->flags & SLICE_FLAG_PROFILE) != 0;
-  s->dynamic_pct = cfg->dynamic_pct ? cfg->dynamic_pct : kDefaultDynamicPct;
+  s->trace = s->profile || (cfg->flags & SLICE_FLAG_TRACE) != 0;
+  s->steal = cfg->static_split == 0;
   s->block_bytes = bb;
   s->local_bs = cfg->local_block_stride ? cfg->local_block_stride : bb;
   s->local_ls = cfg->local_layer_stride ? cfg->local_layer_stride : bb * cfg->local_blocks;
@@ -721,8 +688,8 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     }
     if (cudaMalloc(reinterpret_cast<void**>(&s->dev_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
     if (cudaMemset(s->dev_status, 0, 256) != cudaSuccess) return fail(SLICE_ECUDA);
-    const size_t cnt_words = static_cast<size_t>(cfg->num_layers) * ema::kLaunchCounters +
-                             static_cast<size_t>(cfg->max_seqs) * cfg->num_kv_heads;
+    s->cnt_stride = align_up(ema::layer_counter_words(s->ncta, cfg->max_seqs, cfg->num_kv_heads), 64);
+    const size_t cnt_words = static_cast<size_t>(cfg->num_layers) * s->cnt_stride;
     if (cudaMalloc(reinterpret_cast<void**>(&s->cnt_dev), cnt_words * sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(s->cnt_dev, 0, cnt_words * sizeof(uint32_t)) != cudaSuccess)
       return fail(SLICE_ECUDA);
@@ -739,6 +706,8 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
       for (auto& e : s->prof)
         if (cudaEventCreate(&e) != cudaSuccess) return fail(SLICE_ECUDA);
       if (cudaEventCreate(&s->prof_base) != cudaSuccess) return fail(SLICE_ECUDA);
+    }
+    if (s->trace) {
       const size_t tl = static_cast<size_t>(cfg->num_layers) * s->ncta * 4 * sizeof(unsigned long long);
       const size_t tc = static_cast<size_t>(cfg->num_layers) * kTraceCopyCtas * 2 * sizeof(unsigned long long);
       if (cudaMalloc(reinterpret_cast<void**>(&s->trace_layer), tl) != cudaSuccess ||
@@ -1088,7 +1057,7 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
     od = static_cast<uint8_t*>(s->io_out);
   }
   if (!s->null_dev)  // the work counters of all layers, cleared once per pass
-    CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * ema::kLaunchCounters * sizeof(uint32_t), stream));
+    CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * s->cnt_stride * sizeof(uint32_t), stream));
   if (p->k && !staged(s, 0, p)) {
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
@@ -1161,7 +1130,7 @@ int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* 
 
 int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entries, uint32_t* ctas_per_layer,
                     uint32_t* words_per_cta) {
-  if (!s || !s->profile || s->null_dev || (which != 0 && which != 1)) return SLICE_EINVAL;
+  if (!s || !s->trace || s->null_dev || (which != 0 && which != 1)) return SLICE_EINVAL;
   const uint32_t per = which == 0 ? s->ncta : kTraceCopyCtas;
   const uint32_t words = which == 0 ? 4 : 2;
   if (ctas_per_layer) *ctas_per_layer = per;

@@ -89,11 +89,11 @@ def test_both_gather_kernels_are_bit_exact(kind):
 
 
 def test_small_decode_grid_and_many_segments():
-    """Few CTAs: each walks many work items; a large dynamic share: many partials to merge; a
-    fully static split: no dynamic items at all."""
+    """Few CTAs: each walks many sequences; many CTAs: most have no range of their own and only
+    steal; static split: no stealing at all."""
     sc = Scenario(GQA4, 6)
-    for ctas, dyn in ((3, 0), (64, 0), (2, 60), (7, 100), (0, 90)):
-        g = _gpu(sc, decode_ctas=ctas, dynamic_pct=dyn)
+    for ctas, static in ((3, 0), (64, 0), (2, 1), (7, 1), (0, 0), (0, 1)):
+        g = _gpu(sc, decode_ctas=ctas, static_split=static)
         for layer in range(sc.L):
             _check_layer(sc, g, layer)
 
@@ -252,13 +252,13 @@ def test_copy_blocks_matches_index_select(kind, n, bb):
     assert torch.equal(dst2, src[src_idx.long()])
 
 
-@pytest.mark.parametrize("mode,layers,dyn", [(0, 5, 0), (1, 5, 0), (0, 4, 50), (1, 4, 100)])
-def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, dyn):
+@pytest.mark.parametrize("mode,layers,static", [(0, 5, 0), (1, 5, 0), (0, 4, 1), (1, 4, 1)])
+def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, static):
     """Both pipelines (fused: attention + next layer's gather in one launch; two streams with
     events), odd and even layer counts on a ring of two, three passes each."""
     wl = synth.Workload("pipe", layers, 32, 8, 7, 100, 1200, 0.4)
     sc = Scenario(wl, 9)
-    g = _gpu(sc, flags=B.FLAG_PROFILE, pipeline_mode=mode, dynamic_pct=dyn, decode_ctas=12)
+    g = _gpu(sc, flags=B.FLAG_PROFILE, pipeline_mode=mode, static_split=static, decode_ctas=12)
     seqs = np.asarray(sc.seq_ids, np.int32)
     for rep in range(3):
         g.out.zero_()
@@ -292,7 +292,16 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, dyn):
     oh = torch.zeros_like(qh).pin_memory()
     assert g.s.slice_decode_step(seqs, qh, sc.Hq, float(sc.sm_scale), oh, True, True, g.main, g.side) == B.OK
     torch.cuda.synchronize()
-    assert torch.equal(oh, g.out.cpu())
+    # same inputs, same result up to the rounding of a different work split (stealing is not
+    # deterministic): compare with the oracle again rather than bit for bit
+    outh = oh.view(torch.bfloat16).double().numpy()
+    for layer in range(sc.L):
+        rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+        _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % wl.ring_slots], resolved,
+                                           sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+        assert attention_close(outh[layer], ref, ATOL, RTOL)[0]
+    if static:
+        assert torch.equal(oh, g.out.cpu())     # static split: bit-identical from run to run
 
 
 def test_llama8b_shapes_sampled_parity():
