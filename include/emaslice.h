@@ -89,9 +89,11 @@ typedef struct {
   uint32_t decode_ctas;           /* 0 = one per SM; CTAs of the layer (attention) kernel        */
   uint32_t copy_ctas;             /* 0 = default; CTAs of the stand-alone gather / migration kernel */
   uint32_t copy_kind;             /* 0 = default, 1 = vector load/store kernel, 2 = bulk-copy ring */
-  uint32_t pipeline_mode;         /* slice_decode_step: 0 = fused (attention of layer l and gather of
-                                     layer l+1 in one launch, one stream), 1 = two kernels on two
-                                     streams ordered by events                                   */
+  uint32_t pipeline_mode;         /* slice_decode_step: 0 = one persistent launch for the whole pass
+                                     (attention of layer l overlapped with the gather of layer l+1,
+                                     soft layer boundaries; falls back to 2 when the shape does not
+                                     allow it), 1 = two kernels on two streams ordered by events,
+                                     2 = one fused launch per layer                              */
   uint32_t static_split;          /* attention work split: 0 = each CTA owns a range of blocks and idle
                                      CTAs steal from the ranges with most left (default); 1 = static
                                      ranges only                                                  */
@@ -215,10 +217,10 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
 
 /* One pass of the whole path over a batch: for every layer, the prefetch of layer l+1 overlapped
  * with the attention of layer l (cyclic: the last layer's attention overlaps the prefetch of layer 0
- * for the next pass when wrap_prefetch != 0). With pipeline_mode 0 and a ring of at least two slots
- * both run inside one kernel launch per layer on `stream` (side_stream is not used); with
- * pipeline_mode 1 the gather kernel runs on side_stream and the attention kernel on stream, ordered
- * by events.
+ * for the next pass when wrap_prefetch != 0). With pipeline_mode 0 or 2 and a ring of at least two
+ * slots both run inside the same kernel on `stream` (side_stream is not used): one launch for the
+ * whole pass (mode 0) or one per layer (mode 2); with pipeline_mode 1 the gather kernel runs on
+ * side_stream and the attention kernel on stream, ordered by events.
  *   q, out: [num_layers][nseq][num_q_heads][128] bf16; device pointers when io_on_host == 0.
  *   With io_on_host != 0 they are host pointers (pinned for asynchronous copies): q is copied to the
  *   device and out back to the host on `stream`, inside the call's enqueued work, through device

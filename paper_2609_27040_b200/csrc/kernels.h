@@ -35,23 +35,32 @@ enum CopyKind : uint32_t { kCopyDefault = 0, kCopyVector = 1, kCopyBulk = 2 };
 // Launches one copy kernel on `stream`. ctas == 0 picks a default grid. Returns the CUDA error.
 cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num_sms, cudaStream_t stream);
 
-// Device counters of one layer-kernel launch; the whole block must be zero when the kernel
-// starts. Layout in uint32 words:
-//   [0, 16)                         launch words: [1] = next copy unit
-//   [16, 16 + 2*ncta)               one 64-bit claim word per CTA range: blocks claimed from the front
-//                                   (low half, by the owner) and from the back (high half, by thieves)
-//   [.., + nseq)                    partial slots handed out per sequence
-//   [.., + nseq*Hkv)                blocks finished per (sequence, KV head)
+// Device counters of ONE layer inside a layer-kernel launch; the whole block must be zero when the
+// kernel starts. Layout in uint32 words:
+//   [0, 16)                 launch words: [1] next copy unit of the gather issued during this layer,
+//                           [2] attention work finished (blocks x KV heads), [3] gathered blocks of
+//                           THIS layer that have landed in its ring slot, [4] merges finished
+//   [16, 16 + 2*ncta)       one 64-bit claim word per CTA range: blocks claimed from the front (low
+//                           half, by the owner) and from the back (high half, by thieves)
+//   [.., + nseq)            partial slots handed out per sequence
+//   [.., + nseq*Hkv)        blocks finished per (sequence, KV head)
 constexpr uint32_t kLaunchCounters = 16;
+constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntGathered = 3, kCntMerged = 4;
+constexpr uint32_t kMaxStepLayers = 128;
 inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
   return kLaunchCounters + 2 * static_cast<size_t>(ncta) + nseq + static_cast<size_t>(nseq) * Hkv;
 }
 
+// Parameters of one launch of the layer kernel. It covers layers first_layer .. first_layer +
+// num_layers - 1 of one batch; pointers refer to first_layer and the strides lead to the next layer.
 struct LayerParams {
-  // attention of one layer over one batch
-  const uint8_t* local_layer;   // base of this layer's local arena
+  const uint8_t* local_layer;   // local arena of first_layer
+  uint64_t local_layer_stride;
   uint64_t local_block_stride;
-  const uint8_t* slot_base;     // ring slot that holds this layer's staged blocks
+  const uint8_t* staging_base;  // ring: layer l is staged in slot l % ring_slots
+  uint64_t slot_bytes;
+  uint32_t ring_slots;
+  uint32_t first_layer, num_layers;
   uint64_t block_bytes;
   const int32_t* resolved;      // flat resolved table of the batch (batch order, then block order)
   const uint32_t* lens;         // [nseq] tokens
@@ -62,27 +71,39 @@ struct LayerParams {
   uint32_t per;                 // blocks per CTA range; range c = [c*per, min((c+1)*per, total))
   uint32_t used_cta;            // number of non-empty ranges
   uint32_t allow_steal;         // 0: every range is processed by its owner only
-  const void* q;                // [nseq][Hq][128] bf16
-  void* out;                    // [nseq][Hq][128] bf16
-  float* lse;                   // [nseq][Hq] or NULL
-  float* part_o;                // [slots][Hq][128] unnormalised partial outputs
-  float* part_ml;               // [slots][Hq][4]   max (log2 domain), sum as used, exact sum, pad
-  uint32_t* counters;           // layer_counter_words(), zeroed before the launch
+  const void* q;                // first_layer's [nseq][Hq][128] bf16
+  void* out;
+  uint64_t io_layer_stride;     // bytes from one layer's q / out to the next
+  float* lse;                   // [nseq][Hq] or NULL (single-layer launches only)
+  float* part_o;                // [slots][Hq][128] unnormalised partial outputs; layers alternate
+  float* part_ml;               // [slots][Hq][4]   between two such buffers (stride below)
+  uint64_t part_o_stride, part_ml_stride;  // floats between the two buffers (0: single layer)
+  uint32_t* counters;           // first_layer's layer_counter_words(), all zeroed before the launch
+  uint64_t counters_stride;     // words from one layer's counters to the next
   uint32_t nseq, ncta;
   uint32_t Hq, Hkv, G;
   float scale_log2;             // sm_scale * log2(e)
-  uint32_t has_attention;       // 0: copy work only
-  // optional gather of another layer's lent blocks in the same launch (copy.n == 0: none)
-  CopyDesc copy;
+  // Gather issued while layer first_layer + i is attended to: target layer (or -1), and the layer of
+  // this launch whose attention must be complete before the target's ring slot may be overwritten
+  // (-1: ordered by the stream already).
+  const uint8_t* lent_base;     // lent arena of layer 0
+  uint64_t lent_layer_stride, lent_block_stride;
+  const int32_t* copy_src;      // [copy_n] lent entries in staging order
+  uint32_t copy_n;
+  int16_t gather_target[kMaxStepLayers];
+  int16_t gather_after[kMaxStepLayers];
   int* status;
-  unsigned long long* trace;    // optional [ncta][4]: start, attention end, copy end, SM id
+  unsigned long long* trace;    // optional, per layer [ncta][4]: start, attention end, copy end, info
+  uint64_t trace_stride;        // words from one layer's trace to the next
 };
 
 // Shared memory the layer kernel needs for Hkv KV heads (0 if unsupported).
 size_t layer_smem_bytes(uint32_t Hkv);
 // One-time per-process opt-in to large dynamic shared memory.
 cudaError_t layer_setup();
-// Attention (+ fused gather, + merge by the last-arriving warp): ONE launch.
+// Attention (+ fused gather, + merges) of num_layers layers: ONE launch. Launches that span several
+// layers contain bounded waits between CTAs and are therefore launched cooperatively (all CTAs
+// resident).
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream);
 
 // noalloc.cu: the same launch with partials and counters in a static device array (part_o,

@@ -1,18 +1,20 @@
-// layer_kernel.cu — the fused per-layer kernel of the memory-slice hot path:
+// layer_kernel.cu — the fused kernel of the memory-slice hot path. One persistent launch (one CTA
+// per SM) covers one layer or a whole pass over all layers of a batch:
 //   paged GQA decode attention of layer l  (split-KV flash decoding, merge included)
-//   + prefetch gather of layer l+1's lent blocks into the other ring slot
-// in ONE persistent launch (one CTA per SM), so the two streams of HBM traffic share every SM and
-// overlap for the whole duration of the layer, with no second kernel to co-schedule, no merge launch
-// and no cross-stream event between layers. With copy.n == 0 it is the plain attention kernel.
+//   + prefetch gather of layer l+1's lent blocks into the other ring slot,
+// so the two streams of HBM traffic share every SM for the whole duration of a layer, with no second
+// kernel to co-schedule, no merge launch and no cross-stream event. When the launch spans several
+// layers, layer boundaries are soft: a CTA that runs out of work in layer l moves on to layer l+1
+// while others finish l, so tails, merges and ramp-up overlap with streaming instead of leaving HBM
+// idle once per layer.
 //
 // Work distribution. The batch's blocks, flattened in batch order, are cut into one contiguous range
-// per CTA. A CTA claims blocks from the FRONT of its own range, eight at a time; a CTA whose range is
-// used up steals from the BACK of the range with the most unclaimed blocks (a quarter of what is
-// left, at least two blocks). Both kinds of claim are one atomicAdd on the range's packed 64-bit word
-// (front count | back count), so they can never overlap. SMs stream at visibly different rates
-// (position on the die, mixed read/write traffic), and stealing keeps all of them busy to the end.
-// A CTA keeps one running softmax state per "run" = consecutive claims that belong to the same
-// sequence, so the number of partial results stays close to the number of (CTA, sequence) pairs.
+// per CTA (the same for every layer). A CTA claims blocks from the FRONT of its own range; a CTA
+// whose range is used up steals from the BACK of the range with the most unclaimed blocks. Both
+// kinds of claim are one atomicAdd on the range's packed 64-bit word (front count | back count), so
+// they can never overlap. SMs stream at visibly different rates (position on the die, mixed
+// read/write traffic); stealing keeps all of them busy. A CTA keeps one running softmax state per
+// "run" = consecutive claims within one sequence, so partial results stay few.
 //
 // Roles inside a CTA (warps):
 //   * producer warp: claims work and streams KV blocks into a shared-memory ring of half blocks
@@ -23,19 +25,29 @@
 //     (mma.sync m16n8k16 bf16, swapped form), f32 FMAs when G == 1; online softmax with warp
 //     shuffles. A finished run writes (max, sums, unnormalised output) to a partial slot and adds its
 //     block count to the (sequence, KV head) counter; the warp whose addition completes the sequence
-//     notes a merge; when the CTA's streaming is over its consumer warps share out the noted
-//     merges (the ring is shared by all consumer warps, so a warp that stopped to merge earlier
-//     would stall the whole CTA).
+//     queues a merge request (the ring is shared by all consumer warps, so a warp that stopped to
+//     merge would stall the whole CTA).
+//   * merge warp: serves the CTA's merge requests; consumer warps join it once their streaming is
+//     over.
 //   * copy warp: one thread moves 16 KB pieces lent arena -> shared ring -> staging slot with TMA
 //     bulk copies (global->shared on an mbarrier, shared->global in bulk async-groups), pulling
 //     64 KB units from an atomic counter. No SM lane touches the copied bytes.
-// Every mbarrier wait is bounded; on expiry the role records SLICE_ETIMEOUT in the status word,
-// gives its own copies in flight a bounded chance to land and returns.
-// HBM-bound: algorithmic bytes per launch = sum_s len_s * 2*Hkv*128*2 (+ q, out, table)
+//
+// Waits. Inside a CTA everything is mbarriers. Between CTAs there are three waits, only in launches
+// that span several layers (which are launched cooperatively, so every CTA is resident): staged
+// blocks of layer l are read only after all of l's gathered blocks have landed; a ring slot is
+// overwritten only after the attention of the layer that last used it is complete; a partial
+// buffer (two alternate) is reused only after the merges of the layer before last are done. They
+// wait on counters that earlier layers' work increments, never on later work, so they cannot form a
+// cycle. Every wait, mbarrier or counter, is bounded (about two seconds): on expiry the role records
+// SLICE_ETIMEOUT in the status word, gives its own copies in flight a bounded chance to land and
+// returns.
+// HBM-bound: algorithmic bytes per layer = sum_s len_s * 2*Hkv*128*2 (+ q, out, table)
 // + 2 * block_bytes per gathered block.
 #include "attention_tiles.cuh"
 #include "kernels.h"
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 namespace ema {
@@ -50,19 +62,20 @@ constexpr int kQueue = 8;                  // unit descriptors in flight (> kNA 
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRowPad = 16;
-constexpr uint32_t kOwnChunk = 8;          // blocks an owner claims at a time
+constexpr uint32_t kOwnChunk = 8;          // most blocks an owner claims at a time
 constexpr uint32_t kStealMin = 2, kStealMax = 16;
-constexpr uint32_t kMq = 64;               // merges a CTA can note for the end of its streaming
+constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
+constexpr uint64_t kWaitNs = 2000000000ull;
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
 __host__ __device__ constexpr uint32_t row_pitch(uint32_t Hkv) { return row_bytes(Hkv) + kRowPad; }
 __host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_pitch(Hkv); }
 
-// A unit: blocks [blk_begin, blk_end) of batch position seq_idx. slot carries the run's partial
-// slot and the kNewRun flag when the unit starts a new run.
+// A unit: blocks [blk_begin, blk_end) of batch position seq_idx in layer `layer`. slot carries the
+// run's partial slot and the kNewRun flag when the unit starts a new run.
 struct UnitDesc {
-  uint32_t seq_idx, blk_begin, blk_end, slot;
+  uint32_t seq_idx, blk_begin, blk_end, slot, layer, pad0, pad1, pad2;
 };
 
 struct Claim {
@@ -78,11 +91,10 @@ struct Smem {
   UnitDesc* queue;      // [kQueue]
   uint8_t** copy_dst;   // [kNC]
   uint32_t* copy_len;   // [kNC]
-  uint32_t* mq;         // merge list: [kMq] entries, then count, unused, consumer warps done
+  uint32_t* mq;         // merge queue: [kMq] entries, then tail, head, consumer warps done
 };
 
-// Bookkeeping area behind the two rings: 16 mbarrier slots, the unit queue, the copy ring's
-// destination pointers and lengths; every part 16-byte aligned.
+// Bookkeeping area behind the two rings; every part 16-byte aligned.
 constexpr size_t kBarBytes = 16 * sizeof(uint64_t);
 constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
@@ -110,26 +122,32 @@ __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv) {
   return s;
 }
 
-__device__ __forceinline__ unsigned long long* range_words(const LayerParams& p) {
-  return reinterpret_cast<unsigned long long*>(p.counters + kLaunchCounters);
+// Per-layer pieces of the parameter block; li = layer - first_layer.
+__device__ __forceinline__ uint32_t* layer_counters(const LayerParams& p, uint32_t li) {
+  return p.counters + li * p.counters_stride;
 }
-__device__ __forceinline__ uint32_t* seq_counts(const LayerParams& p) {
-  return p.counters + kLaunchCounters + 2 * p.ncta;
+__device__ __forceinline__ unsigned long long* range_words(const LayerParams& p, uint32_t li) {
+  return reinterpret_cast<unsigned long long*>(layer_counters(p, li) + kLaunchCounters);
 }
-__device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p) { return seq_counts(p) + p.nseq; }
+__device__ __forceinline__ uint32_t* seq_counts(const LayerParams& p, uint32_t li) {
+  return layer_counters(p, li) + kLaunchCounters + 2 * p.ncta;
+}
+__device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p, uint32_t li) { return seq_counts(p, li) + p.nseq; }
+__device__ __forceinline__ float* part_o_of(const LayerParams& p, uint32_t li) { return p.part_o + (li & 1u) * p.part_o_stride; }
+__device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) { return p.part_ml + (li & 1u) * p.part_ml_stride; }
 
-__device__ __forceinline__ const uint8_t* copy_src(const CopyDesc& d, uint32_t i, uint32_t layer) {
-  const int32_t e = d.src_entry ? d.src_entry[i] : static_cast<int32_t>(i);
-  const int t = e < 0;
-  const uint32_t id = t ? static_cast<uint32_t>(~e) : static_cast<uint32_t>(e);
-  return d.src_base[t] + layer * d.src_layer_stride[t] + id * d.src_block_stride[t];
-}
-
-__device__ __forceinline__ uint8_t* copy_dst(const CopyDesc& d, uint32_t i, uint32_t layer) {
-  const int32_t e = d.dst_entry ? d.dst_entry[i] : static_cast<int32_t>(i);
-  const int t = e < 0;
-  const uint32_t id = t ? static_cast<uint32_t>(~e) : static_cast<uint32_t>(e);
-  return d.dst_base[t] + layer * d.dst_layer_stride[t] + id * d.dst_block_stride[t];
+// Bounded wait until a device counter written by other CTAs reaches `target`.
+__device__ __forceinline__ bool wait_counter(const uint32_t* cnt, uint32_t target, int* status) {
+  if (__ldcg(cnt) >= target) return true;
+  const uint64_t t0 = ptx::global_timer_ns();
+  while (__ldcg(cnt) < target) {
+    if (ptx::global_timer_ns() - t0 > kWaitNs) {
+      if (status) atomicExch(status, kDevTimeout);
+      return false;
+    }
+    __nanosleep(128);
+  }
+  return true;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -141,146 +159,182 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t rb = row_bytes(Hkv), pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t plane_bytes = kT * rb;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
-  unsigned long long* rw = range_words(p);
-  uint32_t* seq_count = seq_counts(p);
-  uint32_t hs = 0, nq = 0, cur_seq = kSentinel, nruns = 0, nclaims = 0;
+  uint32_t hs = 0, nq = 0;
   bool ok = true;
 
-  // Streams blocks [bb, be) of batch position seq (flat index of bb: flat) as one unit.
-  auto stream_unit = [&](uint32_t seq, uint32_t bb, uint32_t be, uint32_t flat, uint32_t slot_flag) {
-    const uint32_t nb = be - bb;
-    for (uint32_t b0 = 0; b0 < nb && ok; b0 += 32) {
-      const uint32_t cnt = min(32u, nb - b0);
-      const int32_t my = lane < cnt ? p.resolved[flat + b0 + lane] : 0;
-      for (uint32_t j = 0; j < cnt && ok; ++j) {
-        const int32_t e = __shfl_sync(0xffffffffu, my, j);
-        const uint8_t* src = e >= 0 ? p.local_layer + static_cast<uint64_t>(e) * p.local_block_stride
-                                    : p.slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
-#pragma unroll
-        for (uint32_t plane = 0; plane < 2; ++plane, ++hs) {
-          const uint32_t stg = hs % kNA;
-          ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) return;
-          const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
-          if (lane == 0) {
-            if (b0 + j == 0 && plane == 0) {
-              sm.queue[nq % kQueue] = UnitDesc{seq, bb, be, slot_flag};
-              ++nq;
-            }
-            ptx::mbar_arrive_expect_tx(full, plane_bytes);
+  for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
+    const uint32_t layer = p.first_layer + li;
+    const uint8_t* local_layer = p.local_layer + li * p.local_layer_stride;
+    const uint8_t* slot_base = p.staging_base + (layer % p.ring_slots) * p.slot_bytes;
+    unsigned long long* rw = range_words(p, li);
+    uint32_t* seq_count = seq_counts(p, li);
+    uint32_t cur_seq = kSentinel, nruns = 0, nclaims = 0;
+    // Staged blocks of this layer may be read once its gather (issued during the previous layer of
+    // this launch) has landed completely; the first layer's gather precedes the launch in stream order.
+    bool staged_ok = li == 0 || p.gather_target[li - 1] != static_cast<int16_t>(layer);
+    if (p.trace && lane == 0) p.trace[li * p.trace_stride + 4 * blockIdx.x] = ptx::global_timer_ns();
+    // The partial buffer of this layer's parity was last used two layers ago: its merges must be done.
+    if (li >= 2) {
+      ok = wait_counter(layer_counters(p, li - 2) + kCntMerged, p.nseq * Hkv, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+    }
+
+    // Streams blocks [bb, be) of batch position seq (flat index of bb: flat) as one unit.
+    auto stream_unit = [&](uint32_t seq, uint32_t bb, uint32_t be, uint32_t flat, uint32_t slot_flag) {
+      const uint32_t nb = be - bb;
+      for (uint32_t b0 = 0; b0 < nb && ok; b0 += 32) {
+        const uint32_t cnt = min(32u, nb - b0);
+        const int32_t my = lane < cnt ? p.resolved[flat + b0 + lane] : 0;
+        for (uint32_t j = 0; j < cnt && ok; ++j) {
+          const int32_t e = __shfl_sync(0xffffffffu, my, j);
+          if (e < 0 && !staged_ok) {
+            ok = wait_counter(layer_counters(p, li) + kCntGathered, p.copy_n, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            staged_ok = true;
           }
-          __syncwarp();
-          if (lane < kT)
-            ptx::bulk_g2s(ring + stg * hsb + lane * pitch, src + plane * plane_bytes + static_cast<uint64_t>(lane) * rb,
-                          rb, full);
-        }
-      }
-    }
-  };
-
-  // Streams a claimed flat range, one unit per sequence it touches. A unit that belongs to another
-  // sequence than the previous one starts a new run and takes the next partial slot of its sequence.
-  auto stream_claim = [&](Claim c) {
-    ++nclaims;
-    uint32_t pos = c.b;
-    while (pos < c.e && ok) {
-      const uint32_t seq = p.blk_seq[pos];
-      const uint32_t seq_lo = p.blk_off[seq], seq_hi = p.blk_off[seq + 1];
-      const uint32_t ue = min(c.e, seq_hi);
-      uint32_t slot_flag = 0;
-      if (seq != cur_seq) {
-        uint32_t k = 0;
-        if (lane == 0) k = atomicAdd(&seq_count[seq], 1u);
-        k = __shfl_sync(0xffffffffu, k, 0);
-        const uint32_t base = p.seq_slot_base[seq], cap = p.seq_slot_base[seq + 1] - base;
-        if (k >= cap) {  // cannot happen with the host's sizing; never write outside the slots
-          if (lane == 0 && p.status) atomicExch(p.status, kDevTimeout - 1);
-          k = cap - 1;
-        }
-        slot_flag = (base + k) | kNewRun;
-        cur_seq = seq;
-        ++nruns;
-      }
-      stream_unit(seq, pos - seq_lo, ue - seq_lo, pos, slot_flag);
-      pos = ue;
-    }
-  };
-
-  auto range_len = [&](uint32_t c) { return min(p.per, p.total_blocks - c * p.per); };
-
-  // The owner's claims shrink as its range runs out (a quarter of what the last claim saw left),
-  // so that little claimed-but-unprocessed work is hidden from thieves near the end.
-  uint32_t own_left = 0xFFFFFFFFu;
-  auto claim_front = [&](uint32_t c) -> Claim {
-    const uint32_t want = min(kOwnChunk, max(1u, own_left / 4));
-    unsigned long long old = 0;
-    if (lane == 0) old = atomicAdd(&rw[c], static_cast<unsigned long long>(want));
-    old = __shfl_sync(0xffffffffu, old, 0);
-    const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
-    const uint32_t len = range_len(c);
-    const uint32_t avail_end = b < len ? len - b : 0;
-    if (f >= avail_end) return Claim{0, 0};
-    const uint32_t e = min(f + want, avail_end);
-    own_left = avail_end - e;
-    return Claim{c * p.per + f, c * p.per + e};
-  };
-
-  auto steal = [&]() -> Claim {
-    for (int attempt = 0; attempt < 16; ++attempt) {
-      uint32_t best_rem = 0, best_v = 0;
-      for (uint32_t v = lane; v < p.used_cta; v += 32) {
-        const unsigned long long w = __ldcg(&rw[v]);
-        const uint32_t f = static_cast<uint32_t>(w), b = static_cast<uint32_t>(w >> 32);
-        const uint32_t len = range_len(v);
-        const uint32_t rem = f + b < len ? len - f - b : 0;
-        if (rem > best_rem) {
-          best_rem = rem;
-          best_v = v;
-        }
-      }
+          const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
+                                      : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
 #pragma unroll
-      for (int sh = 16; sh >= 1; sh >>= 1) {
-        const uint32_t r = __shfl_xor_sync(0xffffffffu, best_rem, sh);
-        const uint32_t vv = __shfl_xor_sync(0xffffffffu, best_v, sh);
-        if (r > best_rem || (r == best_rem && vv < best_v)) {
-          best_rem = r;
-          best_v = vv;
+          for (uint32_t plane = 0; plane < 2; ++plane, ++hs) {
+            const uint32_t stg = hs % kNA;
+            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
+            if (lane == 0) {
+              if (b0 + j == 0 && plane == 0) {
+                sm.queue[nq % kQueue] = UnitDesc{seq, bb, be, slot_flag, li, 0, 0, 0};
+                ++nq;
+              }
+              ptx::mbar_arrive_expect_tx(full, plane_bytes);
+            }
+            __syncwarp();
+            if (lane < kT)
+              ptx::bulk_g2s(ring + stg * hsb + lane * pitch,
+                            src + plane * plane_bytes + static_cast<uint64_t>(lane) * rb, rb, full);
+          }
         }
       }
-      if (best_rem == 0) return Claim{0, 0};
-      const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / 4));
+    };
+
+    // Streams a claimed flat range, one unit per sequence it touches. A unit of another sequence
+    // than the previous one starts a new run and takes the next partial slot of its sequence.
+    auto stream_claim = [&](Claim c) {
+      ++nclaims;
+      uint32_t pos = c.b;
+      while (pos < c.e && ok) {
+        const uint32_t seq = p.blk_seq[pos];
+        const uint32_t seq_lo = p.blk_off[seq], seq_hi = p.blk_off[seq + 1];
+        const uint32_t ue = min(c.e, seq_hi);
+        uint32_t slot_flag = 0;
+        if (seq != cur_seq) {
+          // With stealing, slots are handed out in arrival order; with the static split a
+          // sequence's slot is the index of the range among those it touches, so the merge order,
+          // and with it every bit of the result, is the same from run to run.
+          uint32_t k = 0;
+          if (p.allow_steal) {
+            if (lane == 0) k = atomicAdd(&seq_count[seq], 1u);
+            k = __shfl_sync(0xffffffffu, k, 0);
+          } else {
+            k = blockIdx.x - seq_lo / p.per;
+          }
+          const uint32_t base = p.seq_slot_base[seq], cap = p.seq_slot_base[seq + 1] - base;
+          if (k >= cap) {  // cannot happen with the host's sizing; never write outside the slots
+            if (lane == 0 && p.status) atomicExch(p.status, kDevTimeout - 1);
+            k = cap - 1;
+          }
+          slot_flag = (base + k) | kNewRun;
+          cur_seq = seq;
+          ++nruns;
+        }
+        stream_unit(seq, pos - seq_lo, ue - seq_lo, pos, slot_flag);
+        pos = ue;
+      }
+    };
+
+    auto range_len = [&](uint32_t c) { return min(p.per, p.total_blocks - c * p.per); };
+
+    // The owner's claims shrink as its range runs out (a quarter of what the last claim saw left),
+    // so that little claimed-but-unprocessed work is hidden from thieves near the end.
+    uint32_t own_left = 0xFFFFFFFFu;
+    auto claim_front = [&](uint32_t c) -> Claim {
+      const uint32_t want = min(kOwnChunk, max(1u, own_left / 4));
       unsigned long long old = 0;
-      if (lane == 0) old = atomicAdd(&rw[best_v], static_cast<unsigned long long>(amount) << 32);
+      if (lane == 0) old = atomicAdd(&rw[c], static_cast<unsigned long long>(want));
       old = __shfl_sync(0xffffffffu, old, 0);
       const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
-      const uint32_t len = range_len(best_v);
-      const uint32_t hi = b < len ? len - b : 0;  // end of what was unclaimed before this steal
-      const uint32_t lo_avail = min(f, hi);
-      if (hi > lo_avail) {
-        const uint32_t lo = hi - lo_avail > amount ? hi - amount : lo_avail;
-        return Claim{best_v * p.per + lo, best_v * p.per + hi};
+      const uint32_t len = range_len(c);
+      const uint32_t avail_end = b < len ? len - b : 0;
+      if (f >= avail_end) return Claim{0, 0};
+      const uint32_t e = min(f + want, avail_end);
+      own_left = avail_end - e;
+      return Claim{c * p.per + f, c * p.per + e};
+    };
+
+    auto steal = [&]() -> Claim {
+      for (int attempt = 0; attempt < 16; ++attempt) {
+        uint32_t best_rem = 0, best_v = 0;
+        for (uint32_t v = lane; v < p.used_cta; v += 32) {
+          const unsigned long long w = __ldcg(&rw[v]);
+          const uint32_t f = static_cast<uint32_t>(w), b = static_cast<uint32_t>(w >> 32);
+          const uint32_t len = range_len(v);
+          const uint32_t rem = f + b < len ? len - f - b : 0;
+          if (rem > best_rem) {
+            best_rem = rem;
+            best_v = v;
+          }
+        }
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) {
+          const uint32_t r = __shfl_xor_sync(0xffffffffu, best_rem, sh);
+          const uint32_t vv = __shfl_xor_sync(0xffffffffu, best_v, sh);
+          if (r > best_rem || (r == best_rem && vv < best_v)) {
+            best_rem = r;
+            best_v = vv;
+          }
+        }
+        if (best_rem == 0) return Claim{0, 0};
+        const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / 4));
+        unsigned long long old = 0;
+        if (lane == 0) old = atomicAdd(&rw[best_v], static_cast<unsigned long long>(amount) << 32);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
+        const uint32_t len = range_len(best_v);
+        const uint32_t hi = b < len ? len - b : 0;  // end of what was unclaimed before this steal
+        const uint32_t lo_avail = min(f, hi);
+        if (hi > lo_avail) {
+          const uint32_t lo = hi - lo_avail > amount ? hi - amount : lo_avail;
+          return Claim{best_v * p.per + lo, best_v * p.per + hi};
+        }
+      }
+      return Claim{0, 0};
+    };
+
+    // Own range first (claims run one ahead of the streaming, so the atomic's latency is hidden) ...
+    if (blockIdx.x < p.used_cta) {
+      Claim cur = claim_front(blockIdx.x);
+      while (cur.b < cur.e && ok) {
+        const Claim nxt = claim_front(blockIdx.x);
+        stream_claim(cur);
+        cur = nxt;
       }
     }
-    return Claim{0, 0};
-  };
-
-  // Own range first (claims run one ahead of the streaming, so the atomic's latency is hidden) ...
-  if (blockIdx.x < p.used_cta) {
-    Claim cur = claim_front(blockIdx.x);
-    while (cur.b < cur.e && ok) {
-      const Claim nxt = claim_front(blockIdx.x);
-      stream_claim(cur);
-      cur = nxt;
+    // ... then the back of whichever range has most left.
+    if (ok && p.allow_steal) {
+      Claim cur = steal();
+      while (cur.b < cur.e && ok) {
+        const Claim nxt = steal();
+        stream_claim(cur);
+        cur = nxt;
+      }
     }
-  }
-  // ... then the back of whichever range has most left.
-  if (ok && p.allow_steal) {
-    Claim cur = steal();
-    while (cur.b < cur.e && ok) {
-      const Claim nxt = steal();
-      stream_claim(cur);
-      cur = nxt;
+    if (p.trace && lane == 0) {
+      uint32_t smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      p.trace[li * p.trace_stride + 4 * blockIdx.x + 3] =
+          smid | (static_cast<unsigned long long>(nruns) << 16) | (static_cast<unsigned long long>(nclaims) << 32);
     }
   }
   if (ok) {
@@ -289,11 +343,10 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
     ok = __all_sync(0xffffffffu, ok);
     if (ok && lane == 0) {
-      sm.queue[nq % kQueue] = UnitDesc{kSentinel, 0, 0, 0};
+      sm.queue[nq % kQueue] = UnitDesc{kSentinel, 0, 0, 0, 0, 0, 0, 0};
       ptx::mbar_arrive(ptx::smem_u32(&sm.att_full[stg]));
     }
   }
-  if (p.trace && lane == 0) p.trace[4 * blockIdx.x + 3] |= (static_cast<unsigned long long>(nruns) << 16) | (static_cast<unsigned long long>(nclaims) << 32);
   if (!ok) {
     // Bounded second chance for copies already issued, so that none lands after the CTA is gone.
     const uint32_t from = hs > static_cast<uint32_t>(kNA) ? hs - kNA : 0;
@@ -303,18 +356,26 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// merge of a (sequence, KV head): n partial slots starting at s0, all kG query heads at once.
-// Lane groups of 32/kG lanes own one head each; a lane owns 4*kG consecutive dims of that head.
+// merge of a (layer, sequence, KV head): n partial slots starting at s0, all kG query heads at
+// once. Lane groups of 32/kG lanes own one head each; a lane owns 4*kG consecutive dims.
 // ---------------------------------------------------------------------------------------------
+struct MergeCtx {
+  const float* part_o;
+  const float* part_ml;
+  void* out;
+  float* lse;
+};
+
 template <int kG>
-__device__ __forceinline__ void merge_heads(const LayerParams& p, uint32_t seq, uint32_t g, uint32_t s0, uint32_t n) {
+__device__ __forceinline__ void merge_heads(const LayerParams& p, const MergeCtx& c, uint32_t seq, uint32_t g,
+                                            uint32_t s0, uint32_t n) {
   constexpr uint32_t kLph = 32 / kG;  // lanes per head
   constexpr int kU = 16 / kG;         // partials in flight per round (16 float4 loads per lane)
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t hh = lane / kLph, j = lane % kLph;
   const uint32_t h = g * kG + hh;
-  const float* mlh = p.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
-  const float* poh = p.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + j * 4 * kG;
+  const float* mlh = c.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
+  const float* poh = c.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + j * 4 * kG;
   const uint64_t ml_step = static_cast<uint64_t>(p.Hq) * 4, po_step = static_cast<uint64_t>(p.Hq) * kD;
   float M = kNegInf;
   for (uint32_t s = j; s < n; s += kLph) M = fmaxf(M, __ldcg(mlh + s * ml_step));
@@ -359,22 +420,23 @@ __device__ __forceinline__ void merge_heads(const LayerParams& p, uint32_t seq, 
     }
   }
   const float inv = 1.f / l;
-  uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
+  uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
                                         j * 4 * kG);
 #pragma unroll
   for (int k = 0; k < kG; ++k)
     dst[k] = make_uint2(ptx::pack_bf16x2(acc[k].x * inv, acc[k].y * inv), ptx::pack_bf16x2(acc[k].z * inv, acc[k].w * inv));
-  if (p.lse && j == 0) p.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
+  if (c.lse && j == 0) c.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
 }
 
 // The same for any group size, one head after the other (group sizes that are not a power of two).
-__device__ __forceinline__ void merge_heads_serial(const LayerParams& p, uint32_t seq, uint32_t g, uint32_t s0, uint32_t n) {
+__device__ __forceinline__ void merge_heads_serial(const LayerParams& p, const MergeCtx& c, uint32_t seq, uint32_t g,
+                                                   uint32_t s0, uint32_t n) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t G = p.G;
   for (uint32_t hh = 0; hh < G; ++hh) {
     const uint32_t h = g * G + hh;
-    const float* mlh = p.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
-    const float* poh = p.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + lane * 4;
+    const float* mlh = c.part_ml + (static_cast<uint64_t>(s0) * p.Hq + h) * 4;
+    const float* poh = c.part_o + (static_cast<uint64_t>(s0) * p.Hq + h) * kD + lane * 4;
     const uint64_t ml_step = static_cast<uint64_t>(p.Hq) * 4, po_step = static_cast<uint64_t>(p.Hq) * kD;
     float M = kNegInf, l = 0.f, le = 0.f;
     for (uint32_t s = lane; s < n; s += 32) M = fmaxf(M, __ldcg(mlh + s * ml_step));
@@ -401,70 +463,93 @@ __device__ __forceinline__ void merge_heads_serial(const LayerParams& p, uint32_
       acc.w = fmaf(v.w, w, acc.w);
     }
     const float inv = 1.f / l;
-    uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
+    uint2* dst = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(c.out) + (static_cast<uint64_t>(seq) * p.Hq + h) * kD +
                                           lane * 4);
     *dst = make_uint2(ptx::pack_bf16x2(acc.x * inv, acc.y * inv), ptx::pack_bf16x2(acc.z * inv, acc.w * inv));
-    if (p.lse && lane == 0) p.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
+    if (c.lse && lane == 0) c.lse[static_cast<uint64_t>(seq) * p.Hq + h] = (M + log2f(le)) * 0.6931471805599453f;
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// end of a run: count its blocks; the warp that completes a (sequence, KV head) merges
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t seq, uint32_t g) {
+__device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uint32_t seq, uint32_t g) {
+  MergeCtx c;
+  c.part_o = part_o_of(p, li);
+  c.part_ml = part_ml_of(p, li);
+  c.out = static_cast<uint8_t*>(p.out) + li * p.io_layer_stride;
+  c.lse = p.lse;
   const uint32_t s0 = p.seq_slot_base[seq];
-  const uint32_t n = __ldcg(&seq_counts(p)[seq]);
+  const uint32_t n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
+                                   : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
   switch (p.G) {
-    case 1: merge_heads<1>(p, seq, g, s0, n); break;
-    case 2: merge_heads<2>(p, seq, g, s0, n); break;
-    case 4: merge_heads<4>(p, seq, g, s0, n); break;
-    case 8: merge_heads<8>(p, seq, g, s0, n); break;
-    default: merge_heads_serial(p, seq, g, s0, n); break;
+    case 1: merge_heads<1>(p, c, seq, g, s0, n); break;
+    case 2: merge_heads<2>(p, c, seq, g, s0, n); break;
+    case 4: merge_heads<4>(p, c, seq, g, s0, n); break;
+    case 8: merge_heads<8>(p, c, seq, g, s0, n); break;
+    default: merge_heads_serial(p, c, seq, g, s0, n); break;
+  }
+  __syncwarp();
+  if ((threadIdx.x & 31u) == 0) {
+    __threadfence();
+    atomicAdd(layer_counters(p, li) + kCntMerged, 1u);
   }
 }
 
-// A consumer warp that completes a (sequence, KV head) only notes the merge in a CTA-local list:
-// the ring is shared by all consumer warps, so a warp that stopped to merge would stall the whole
-// CTA. Almost every sequence completes in the last microseconds of the kernel anyway (all ranges
-// finish together), and then all consumer warps of the CTA work through the list in parallel.
-__device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm, uint32_t seq, uint32_t g,
+// End of a run: count its blocks; the warp that completes a (sequence, KV head) queues the merge
+// for the merge warp, and merges itself only when the queue is nearly full.
+__device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm, uint32_t li, uint32_t seq, uint32_t g,
                                            uint32_t blocks) {
   const uint32_t lane = threadIdx.x & 31u;
   __threadfence();
   __syncwarp();
   uint32_t old = 0;
-  if (lane == 0) old = atomicAdd(&merge_counts(p)[seq * p.Hkv + g], blocks);
+  if (lane == 0) {
+    old = atomicAdd(&merge_counts(p, li)[seq * p.Hkv + g], blocks);
+    atomicAdd(layer_counters(p, li) + kCntAttnDone, blocks);
+  }
   old = __shfl_sync(0xffffffffu, old, 0);
   if (old + blocks != p.blk_off[seq + 1] - p.blk_off[seq]) return;
   __threadfence();
-  uint32_t t = kMq;
+  volatile uint32_t* mq = sm.mq;
+  uint32_t queued = 0;
   if (lane == 0) {
-    t = atomicAdd(&sm.mq[kMq], 1u);
-    if (t < kMq) sm.mq[t] = (seq << 4) | g;
-  }
-  t = __shfl_sync(0xffffffffu, t, 0);
-  if (t >= kMq) merge_one(p, seq, g);  // list full: merge right away
-}
-
-// After the CTA's streaming: consumer warp w takes list entries w, w + Hkv, ...
-__device__ __forceinline__ void drain_merges(const LayerParams& p, const Smem& sm, uint32_t w) {
-  const uint32_t lane = threadIdx.x & 31u;
-  if (lane == 0) {
-    __threadfence_block();
-    atomicAdd(&sm.mq[kMq + 2], 1u);
-    // All consumer warps of the CTA must have noted their last merge before the list is read.
-    const uint64_t t0 = ptx::global_timer_ns();
-    while (*reinterpret_cast<volatile uint32_t*>(&sm.mq[kMq + 2]) < p.Hkv) {
-      if (ptx::global_timer_ns() - t0 > 2000000000ull) break;
-      __nanosleep(64);
+    // Up to Hkv warps may pass this check at once, hence the margin.
+    if (static_cast<int32_t>(mq[kMq] - mq[kMq + 1]) < static_cast<int32_t>(kMq - 8)) {
+      const uint32_t t = atomicAdd(&sm.mq[kMq], 1u);
+      const uint64_t t0 = ptx::global_timer_ns();
+      while (mq[t % kMq] != kMqEmpty && ptx::global_timer_ns() - t0 < kWaitNs) __nanosleep(64);
+      mq[t % kMq] = (li << 24) | (seq << 4) | g;
+      queued = 1;
     }
   }
-  __syncwarp();
-  const uint32_t n = min(*reinterpret_cast<volatile uint32_t*>(&sm.mq[kMq]), kMq);
-  __threadfence();
-  for (uint32_t i = w; i < n; i += p.Hkv) {
-    const uint32_t v = *reinterpret_cast<volatile uint32_t*>(&sm.mq[i]);
-    merge_one(p, v >> 4, v & 15u);
+  queued = __shfl_sync(0xffffffffu, queued, 0);
+  if (!queued) merge_one(p, li, seq, g);
+}
+
+// Serves the merge queue until every consumer warp of the CTA has finished and no request is left.
+// Run by the merge warp from the start and by each consumer warp once its streaming is over.
+__device__ void merge_role(const LayerParams& p, const Smem& sm) {
+  const uint32_t lane = threadIdx.x & 31u;
+  volatile uint32_t* mq = sm.mq;
+  for (;;) {
+    uint32_t v = kMqEmpty;
+    if (lane == 0) {
+      const uint32_t h = atomicAdd(&sm.mq[kMq + 1], 1u);
+      const uint64_t t0 = ptx::global_timer_ns();
+      for (;;) {
+        v = mq[h % kMq];
+        if (v != kMqEmpty) {
+          mq[h % kMq] = kMqEmpty;
+          break;
+        }
+        // No request will ever get this ticket once all consumers are done and the tail is behind it.
+        if (mq[kMq + 2] == p.Hkv && static_cast<int32_t>(mq[kMq] - h) <= 0) break;
+        if (ptx::global_timer_ns() - t0 > 2 * kWaitNs) break;  // a consumer that gave up never reports in
+        __nanosleep(128);
+      }
+    }
+    v = __shfl_sync(0xffffffffu, v, 0);
+    if (v == kMqEmpty) return;
+    __threadfence();
+    merge_one(p, v >> 24, (v >> 4) & 0xFFFFFu, v & 15u);
   }
 }
 
@@ -488,11 +573,10 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
-  const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
   const uint32_t n = lane >> 2, tig = lane & 3u, r0 = lane >> 2;
   uint32_t hs = 0, nunit = 0;
   bool have_run = false;
-  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, len = 0;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
   uint32_t qf[8][2];
   float o[8][4];
@@ -506,8 +590,8 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       st.e1 += __shfl_xor_sync(0xffffffffu, st.e1, sh);
     }
     const uint32_t h0 = 2 * tig, h1 = h0 + 1;
-    float* po = p.part_o + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * kD;
-    float* pml = p.part_ml + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * 4;
+    float* po = part_o_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * kD;
+    float* pml = part_ml_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g * G) * 4;
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
       const uint32_t d = mt * 16 + r0;
@@ -524,7 +608,7 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       if (h0 < G) *reinterpret_cast<float4*>(pml + h0 * 4) = make_float4(st.m0, st.l0, st.e0, 0.f);
       if (h1 < G) *reinterpret_cast<float4*>(pml + h1 * 4) = make_float4(st.m1, st.l1, st.e1, 0.f);
     }
-    finish_run(p, sm, run_seq, g, run_blocks);
+    finish_run(p, sm, run_li, run_seq, g, run_blocks);
   };
 
   for (;;) {
@@ -537,10 +621,13 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       have_run = true;
       run_seq = it.seq_idx;
       run_slot = it.slot & ~kNewRun;
+      run_li = it.layer;
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
+      const __nv_bfloat16* qg =
+          reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
       const uint32_t* qrow =
           reinterpret_cast<const uint32_t*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g * G + (n < G ? n : 0)) * kD);
 #pragma unroll
@@ -577,11 +664,10 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t Hkv = p.Hkv;
   const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
-  const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q);
   const uint32_t half = lane & 1u;
   uint32_t hs = 0, nunit = 0;
   bool have_run = false;
-  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, len = 0;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
   float qh[64];  // this lane's half (64 dims) of q as f32
   float o[4] = {0.f, 0.f, 0.f, 0.f};
@@ -589,12 +675,12 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   auto emit = [&]() {
 #pragma unroll
     for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
-    float* po = p.part_o + (static_cast<uint64_t>(run_slot) * p.Hq + g) * kD;
+    float* po = part_o_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g) * kD;
     *reinterpret_cast<float4*>(po + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
     if (lane == 0)
-      *reinterpret_cast<float4*>(p.part_ml + (static_cast<uint64_t>(run_slot) * p.Hq + g) * 4) =
+      *reinterpret_cast<float4*>(part_ml_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g) * 4) =
           make_float4(st.m0, st.l0, st.l0, 0.f);
-    finish_run(p, sm, run_seq, g, run_blocks);
+    finish_run(p, sm, run_li, run_seq, g, run_blocks);
   };
 
   for (;;) {
@@ -607,9 +693,12 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       have_run = true;
       run_seq = it.seq_idx;
       run_slot = it.slot & ~kNewRun;
+      run_li = it.layer;
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+      const __nv_bfloat16* qg =
+          reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
       const uint4* qrow =
           reinterpret_cast<const uint4*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g) * kD + half * 64);
 #pragma unroll
@@ -642,79 +731,103 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// copy warp (one thread)
+// copy warp (one thread): the gathers issued during each layer of the launch
 // ---------------------------------------------------------------------------------------------
 __device__ void copy_role(const LayerParams& p, const Smem& sm) {
-  const CopyDesc& d = p.copy;
-  const uint32_t n_units = d.n * d.nlayers;
-  const uint32_t pieces = static_cast<uint32_t>((d.block_bytes + kCopyChunk - 1) / kCopyChunk);
+  const uint32_t pieces = static_cast<uint32_t>((p.block_bytes + kCopyChunk - 1) / kCopyChunk);
   const uint32_t ring = ptx::smem_u32(sm.copy_ring);
   const uint64_t pol = ptx::policy_evict_first();
-  uint32_t piece = pieces;  // forces a unit fetch
-  const uint8_t* src_blk = nullptr;
-  uint8_t* dst_blk = nullptr;
-  uint32_t issued = 0, done = 0;
-  bool more = true, ok = true;
-
-  // Issues the load of the next 16 KB piece, pulling a new 64 KB unit when the current one is used up.
-  auto issue_next = [&]() -> bool {
-    if (piece == pieces) {
-      const uint32_t unit = atomicAdd(&p.counters[1], 1u);
-      if (unit >= n_units) return false;
-      const uint32_t i = unit % d.n, layer = unit / d.n;
-      src_blk = copy_src(d, i, layer);
-      dst_blk = copy_dst(d, i, layer);
-      piece = 0;
+  uint32_t issued = 0, done = 0;  // pieces over the whole launch: stages and barrier phases continue
+  bool ok = true;
+  for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
+    const int32_t target = p.gather_target[li];
+    if (target < 0 || p.copy_n == 0) continue;
+    // The target's ring slot was last read by an earlier layer of this launch: wait for its attention.
+    const int32_t after = p.gather_after[li];
+    if (after >= 0) {
+      ok = wait_counter(layer_counters(p, static_cast<uint32_t>(after) - p.first_layer) + kCntAttnDone,
+                        p.total_blocks * p.Hkv, p.status);
+      if (!ok) break;
     }
-    const uint64_t off = static_cast<uint64_t>(piece) * kCopyChunk;
-    const uint64_t left = d.block_bytes - off;
-    const uint32_t bytes = left < kCopyChunk ? static_cast<uint32_t>(left) : kCopyChunk;
-    const uint32_t stg = issued % kNC;
-    sm.copy_dst[stg] = dst_blk + off;
-    sm.copy_len[stg] = bytes;
-    const uint32_t bar = ptx::smem_u32(&sm.copy_full[stg]);
-    ptx::mbar_arrive_expect_tx(bar, bytes);
-    ptx::bulk_g2s_hint(ring + stg * kCopyChunk, src_blk + off, bytes, bar, pol);
-    ++piece;
-    ++issued;
-    return true;
-  };
+    const uint8_t* src_layer = p.lent_base + static_cast<uint64_t>(target) * p.lent_layer_stride;
+    uint8_t* dst_slot = const_cast<uint8_t*>(p.staging_base) + (static_cast<uint32_t>(target) % p.ring_slots) * p.slot_bytes;
+    uint32_t* ticket = layer_counters(p, li) + kCntCopyTicket;
+    // Landed blocks are reported to the target layer's counter when the target is in this launch.
+    const bool report = static_cast<uint32_t>(target) > p.first_layer && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
+    uint32_t* landed = report ? layer_counters(p, static_cast<uint32_t>(target) - p.first_layer) + kCntGathered : nullptr;
+    uint32_t piece = pieces;  // forces a unit fetch
+    const uint8_t* src_blk = nullptr;
+    uint8_t* dst_blk = nullptr;
+    const uint32_t first_piece = issued;  // this layer's pieces are [first_piece, issued)
+    uint32_t reported = 0;                // units of this layer already reported as landed
+    bool more = true;
 
-  while (issued < static_cast<uint32_t>(kCopyLoadsAhead) && more) more = issue_next();
-  while (done < issued) {
-    const uint32_t stg = done % kNC;
-    ok = ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[stg]), (done / kNC) & 1u, p.status, kDevTimeout);
-    if (!ok) break;
-    ptx::bulk_s2g(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg]);
-    ptx::bulk_commit();
-    ++done;
-    if (more) {
-      // The stage about to be refilled was last read by the store of piece issued - kNC.
-      ptx::bulk_wait_read<kNC - kCopyLoadsAhead>();
-      more = issue_next();
+    // Issues the load of the next 16 KB piece, pulling a new 64 KB unit when the current one is used up.
+    auto issue_next = [&]() -> bool {
+      if (piece == pieces) {
+        const uint32_t unit = atomicAdd(ticket, 1u);
+        if (unit >= p.copy_n) return false;
+        const int32_t e = p.copy_src[unit];
+        src_blk = src_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
+        dst_blk = dst_slot + static_cast<uint64_t>(unit) * p.block_bytes;
+        piece = 0;
+      }
+      const uint64_t off = static_cast<uint64_t>(piece) * kCopyChunk;
+      const uint64_t left = p.block_bytes - off;
+      const uint32_t bytes = left < kCopyChunk ? static_cast<uint32_t>(left) : kCopyChunk;
+      const uint32_t stg = issued % kNC;
+      sm.copy_dst[stg] = dst_blk + off;
+      sm.copy_len[stg] = bytes;
+      const uint32_t bar = ptx::smem_u32(&sm.copy_full[stg]);
+      ptx::mbar_arrive_expect_tx(bar, bytes);
+      ptx::bulk_g2s_hint(ring + stg * kCopyChunk, src_blk + off, bytes, bar, pol);
+      ++piece;
+      ++issued;
+      return true;
+    };
+    // Reports the units all of whose pieces are among the first `complete` stored pieces of this layer.
+    auto report_landed = [&](uint32_t complete) {
+      if (!landed) return;
+      const uint32_t units = complete / pieces;
+      if (units > reported) {
+        __threadfence();
+        atomicAdd(landed, units - reported);
+        reported = units;
+      }
+    };
+
+    while (issued - done < static_cast<uint32_t>(kCopyLoadsAhead) && more) more = issue_next();
+    while (done < issued) {
+      const uint32_t stg = done % kNC;
+      ok = ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[stg]), (done / kNC) & 1u, p.status, kDevTimeout);
+      if (!ok) break;
+      ptx::bulk_s2g(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg]);
+      ptx::bulk_commit();
+      ++done;
+      // All but the newest kNC - kCopyLoadsAhead stores are complete after this wait: their stages
+      // may be refilled and their bytes are in global memory.
+      ptx::bulk_wait_all<kNC - kCopyLoadsAhead>();
+      const uint32_t stored = done - first_piece;
+      report_landed(stored > static_cast<uint32_t>(kNC - kCopyLoadsAhead) ? stored - (kNC - kCopyLoadsAhead) : 0);
+      if (more) more = issue_next();
     }
+    ptx::bulk_wait_all<0>();
+    if (ok) report_landed(done - first_piece);
+    if (p.trace) p.trace[li * p.trace_stride + 4 * blockIdx.x + 2] = ptx::global_timer_ns();
   }
   if (!ok) {
     for (uint32_t k = done; k < issued; ++k)
       ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[k % kNC]), (k / kNC) & 1u, nullptr, 0);
+    ptx::bulk_wait_all<0>();
   }
-  ptx::bulk_wait_all<0>();
 }
 
 template <bool kMma>
-__global__ void __launch_bounds__(320, 1) slice_layer_kernel(const LayerParams p) {
+__global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   const Smem sm = carve(smem_raw, p.Hkv);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
   if (threadIdx.x == 0) {
-    if (p.trace) {
-      uint32_t smid;
-      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      p.trace[4 * blockIdx.x] = ptx::global_timer_ns();
-      p.trace[4 * blockIdx.x + 1] = 0;
-      p.trace[4 * blockIdx.x + 2] = 0;
-      p.trace[4 * blockIdx.x + 3] = smid;
-    }
     for (int s = 0; s < kNA; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sm.att_full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), p.Hkv);
@@ -726,22 +839,25 @@ __global__ void __launch_bounds__(320, 1) slice_layer_kernel(const LayerParams p
   }
   __syncthreads();
   if (warp < p.Hkv) {
-    if (p.has_attention) {
-      if constexpr (kMma)
-        consumer_mma(p, sm, warp);
-      else
-        consumer_alu(p, sm, warp);
-      __syncwarp();
-      drain_merges(p, sm, warp);
+    if constexpr (kMma)
+      consumer_mma(p, sm, warp);
+    else
+      consumer_alu(p, sm, warp);
+    __syncwarp();
+    if (p.trace && warp == 0 && lane == 0)
+      p.trace[(p.num_layers - 1) * p.trace_stride + 4 * blockIdx.x + 1] = ptx::global_timer_ns();
+    if (lane == 0) {
+      __threadfence_block();
+      atomicAdd(&sm.mq[kMq + 2], 1u);  // this consumer warp queues no more merges
     }
-    if (p.trace && warp == 0 && lane == 0) p.trace[4 * blockIdx.x + 1] = ptx::global_timer_ns();
+    __syncwarp();
+    merge_role(p, sm);
   } else if (warp == p.Hkv) {
-    if (p.has_attention) producer_role(p, sm);
+    producer_role(p, sm);
   } else if (warp == p.Hkv + 1) {
-    if (lane == 0 && p.copy.n) {
-      copy_role(p, sm);
-      if (p.trace) p.trace[4 * blockIdx.x + 2] = ptx::global_timer_ns();
-    }
+    if (lane == 0) copy_role(p, sm);
+  } else if (warp == p.Hkv + 2) {
+    merge_role(p, sm);
   }
 }
 
@@ -788,7 +904,14 @@ cudaError_t layer_setup() {
 
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
   const size_t smem = layer_smem_bytes(p.Hkv);
-  const unsigned threads = (p.Hkv + 2) * 32;
+  const unsigned threads = (p.Hkv + 3) * 32;
+  if (p.num_layers > 1) {
+    // CTAs wait for one another across layers: all of them must be resident.
+    void* args[] = {const_cast<LayerParams*>(&p)};
+    const void* fn = p.G == 1 ? reinterpret_cast<const void*>(slice_layer_kernel<false>)
+                              : reinterpret_cast<const void*>(slice_layer_kernel<true>);
+    return cudaLaunchCooperativeKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
+  }
   if (p.G == 1)
     slice_layer_kernel<false><<<p.ncta, threads, smem, stream>>>(p);
   else

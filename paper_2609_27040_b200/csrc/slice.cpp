@@ -445,8 +445,10 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
   return note_slot_written(s, sl, layer, p, side);
 }
 
-int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots) {
-  const size_t rows = static_cast<size_t>(slots) * Hq;
+// Room for `buffers` partial buffers of slots * Hq rows each (a pass over all layers alternates
+// between two).
+int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots, uint32_t buffers = 1) {
+  const size_t rows = static_cast<size_t>(slots) * Hq * buffers;
   if (s->null_dev || rows <= s->part_rows) return SLICE_OK;
   if (s->part_o) {
     CU(s, cudaDeviceSynchronize());
@@ -460,6 +462,54 @@ int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots) {
   CU(s, cudaMalloc(&s->part_ml, want * 4 * sizeof(float)));
   s->part_rows = want;
   return SLICE_OK;
+}
+
+// Fields of the layer kernel's parameters that do not depend on how many layers a launch spans.
+void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_t first_layer, uint32_t num_layers,
+                 const void* q, void* out, uint32_t Hq, float sm_scale, bool steal) {
+  const uint32_t Hkv = s->cfg.num_kv_heads;
+  d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + first_layer * s->local_ls;
+  d.local_layer_stride = s->local_ls;
+  d.local_block_stride = s->local_bs;
+  d.staging_base = static_cast<const uint8_t*>(s->cfg.staging_base);
+  d.slot_bytes = s->slot_bytes;
+  d.ring_slots = s->cfg.ring_slots;
+  d.first_layer = first_layer;
+  d.num_layers = num_layers;
+  d.block_bytes = s->block_bytes;
+  d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
+  d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
+  d.blk_seq = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_seq);
+  d.blk_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_off);
+  // Without stealing a sequence needs one slot per range it touches: the compact layout.
+  d.seq_slot_base = reinterpret_cast<const uint32_t*>(p->dev + (steal ? p->off_slot_base : p->off_slot_base_static));
+  d.total_blocks = p->total_blocks;
+  d.per = p->per;
+  d.used_cta = p->used_cta;
+  d.allow_steal = steal ? 1u : 0u;
+  d.q = q;
+  d.out = out;
+  d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
+  d.lse = nullptr;
+  d.part_o = s->part_o;
+  d.part_ml = s->part_ml;
+  d.part_o_stride = d.part_ml_stride = 0;
+  d.counters_stride = s->cnt_stride;
+  d.nseq = p->nseq;
+  d.ncta = s->ncta;
+  d.Hq = Hq;
+  d.Hkv = Hkv;
+  d.G = Hq / Hkv;
+  d.scale_log2 = sm_scale * 1.4426950408889634f;
+  d.lent_base = static_cast<const uint8_t*>(s->cfg.lent_base);
+  d.lent_layer_stride = s->lent_ls;
+  d.lent_block_stride = s->lent_bs;
+  d.copy_src = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
+  d.copy_n = p->k;
+  for (uint32_t i = 0; i < ema::kMaxStepLayers; ++i) d.gather_target[i] = d.gather_after[i] = -1;
+  d.status = s->dev_status;
+  d.trace = s->trace_layer ? s->trace_layer + static_cast<size_t>(first_layer) * s->ncta * 4 : nullptr;
+  d.trace_stride = static_cast<uint64_t>(s->ncta) * 4;
 }
 
 // One launch of the layer kernel: attention of `layer` and, when next_layer >= 0, the gather of
@@ -502,37 +552,11 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
     rc = prof_record(s, layer, 2, stream);
     if (rc) return rc;
     ema::LayerParams d{};
-    d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
-    d.local_block_stride = s->local_bs;
-    d.slot_base = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
-    d.block_bytes = s->block_bytes;
-    d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
-    d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
-    d.blk_seq = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_seq);
-    d.blk_off = reinterpret_cast<const uint32_t*>(p->dev + p->off_blk_off);
-    // Without stealing a sequence needs one slot per range it touches: the compact layout.
-    const bool steal = s->steal && !static_scratch;
-    d.seq_slot_base = reinterpret_cast<const uint32_t*>(p->dev + (steal ? p->off_slot_base : p->off_slot_base_static));
-    d.total_blocks = p->total_blocks;
-    d.per = p->per;
-    d.used_cta = p->used_cta;
-    d.allow_steal = steal ? 1u : 0u;
-    d.q = q;
-    d.out = out;
+    fill_common(s, p, d, layer, 1, q, out, Hq, sm_scale, s->steal && !static_scratch);
     d.lse = lse;
-    d.part_o = s->part_o;
-    d.part_ml = s->part_ml;
     d.counters = counters;
-    d.nseq = p->nseq;
-    d.ncta = s->ncta;
-    d.Hq = Hq;
-    d.Hkv = Hkv;
-    d.G = Hq / Hkv;
-    d.scale_log2 = sm_scale * 1.4426950408889634f;
-    d.has_attention = 1;
-    if (gather) fill_gather(s, static_cast<uint32_t>(next_layer), p, d.copy);
-    d.status = s->dev_status;
-    if (s->trace_layer) d.trace = s->trace_layer + static_cast<size_t>(layer) * s->ncta * 4;
+    d.gather_target[0] = gather ? static_cast<int16_t>(next_layer) : static_cast<int16_t>(-1);
+    d.gather_after[0] = -1;  // the slot's last reader precedes this launch in stream order
     if (static_scratch)
       CU(s, ema::launch_layer_static(d, p->slots_static, stream));
     else
@@ -552,6 +576,101 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   s->st.decode_calls++;
   s->st.decode_tokens += p->tokens;
   if (next_layer >= 0) return note_slot_written(s, *nsl, static_cast<uint32_t>(next_layer), p, stream);
+  return SLICE_OK;
+}
+
+// One launch for a whole pass: attention of every layer, each overlapped with the gather of the next
+// layer's lent blocks, layer boundaries soft (see layer_kernel.cu). The caller has primed layer 0.
+int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out, cudaStream_t stream,
+            bool wrap) {
+  const uint32_t Hkv = s->cfg.num_kv_heads, L = s->cfg.num_layers, R = s->cfg.ring_slots;
+  if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
+  if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
+  const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
+  for (uint32_t i = 0; i < p->nseq; ++i)
+    if (lens[i] == 0) return SLICE_EINVAL;
+  if (p->k && !staged(s, 0, p)) return SLICE_ESTALE;
+  // Plan the gathers by following what each ring slot will hold.
+  std::vector<int64_t> holds(R, -1);
+  for (uint32_t r = 0; r < R; ++r)
+    if (s->slots[r].valid && s->slots[r].plan_serial == p->serial) holds[r] = s->slots[r].layer;
+  int16_t target[ema::kMaxStepLayers], after[ema::kMaxStepLayers];
+  uint32_t n_gathers = 0;
+  for (uint32_t l = 0; l < L; ++l) {
+    target[l] = after[l] = -1;
+    if (!p->k) continue;
+    int64_t t = -1;
+    if (l + 1 < L)
+      t = l + 1;
+    else if (wrap && L > 1 && (L - 1) % R != 0)
+      t = 0;
+    if (t < 0 || holds[t % R] == t) continue;  // nothing to fetch, or the slot still holds that layer
+    target[l] = static_cast<int16_t>(t);
+    for (int64_t j = static_cast<int64_t>(l) - 1; j >= 0; --j)
+      if (j % R == t % R) {
+        after[l] = static_cast<int16_t>(j);
+        break;
+      }
+    holds[t % R] = t;
+    ++n_gathers;
+  }
+  int rc = ensure_stream(s, stream);
+  if (rc) return rc;
+  rc = ensure_partials(s, Hq, p->slots, 2);
+  if (rc) return rc;
+  rc = plan_on_stream(s, p, stream);
+  if (rc) return rc;
+  if (!s->null_dev) {
+    for (uint32_t r = 0; r < R; ++r) {
+      SlotState& sl = s->slots[r];
+      if (p->k && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+      rc = order_before_slot_write(s, sl, stream);
+      if (rc) return rc;
+    }
+    for (uint32_t l = 0; l < L; ++l) {
+      rc = prof_record(s, l, 2, stream);
+      if (rc) return rc;
+    }
+    ema::LayerParams d{};
+    fill_common(s, p, d, 0, L, q, out, Hq, sm_scale, s->steal);
+    d.counters = s->cnt_dev;
+    const size_t rows = s->part_rows / 2;
+    d.part_o_stride = rows * kHeadDim;
+    d.part_ml_stride = rows * 4;
+    for (uint32_t l = 0; l < L; ++l) {
+      d.gather_target[l] = target[l];
+      d.gather_after[l] = after[l];
+    }
+    CU(s, ema::launch_layer(d, stream));
+    s->st.kernel_launches++;
+    for (uint32_t l = 0; l < L; ++l) {
+      rc = prof_record(s, l, 4, stream);
+      if (rc) return rc;
+      rc = prof_record(s, l, 3, stream);
+      if (rc) return rc;
+    }
+  }
+  for (uint32_t r = 0; r < R; ++r) {
+    SlotState& sl = s->slots[r];
+    if (!s->null_dev) {
+      if (multi_stream(s)) {
+        CU(s, cudaEventRecord(sl.attn_done, stream));
+        CU(s, cudaEventRecord(sl.pref_done, stream));
+        sl.attn_recorded = sl.pref_recorded = true;
+      }
+      sl.attn_stream = sl.pref_stream = stream;
+    }
+    if (holds[r] >= 0) {
+      sl.valid = true;
+      sl.layer = static_cast<uint32_t>(holds[r]);
+      sl.plan_serial = p->serial;
+    }
+  }
+  s->st.decode_calls += L;
+  s->st.decode_tokens += p->tokens * L;
+  s->st.prefetch_calls += n_gathers;
+  s->st.prefetched_blocks += static_cast<uint64_t>(n_gathers) * p->k;
+  s->st.prefetched_bytes += static_cast<uint64_t>(n_gathers) * p->k * s->block_bytes;
   return SLICE_OK;
 }
 
@@ -603,7 +722,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 1 || cfg->static_split > 1) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 2 || cfg->static_split > 1) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
@@ -1025,7 +1144,10 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
   const uint32_t L = s->cfg.num_layers, R = s->cfg.ring_slots;
-  const bool fused = s->cfg.pipeline_mode == 0 && R >= 2;
+  // Mode 0: one launch for the whole pass when the shape allows it, else one launch per layer.
+  const bool step = s->cfg.pipeline_mode == 0 && R >= 2 && L >= 2 && L <= ema::kMaxStepLayers &&
+                    s->ncta <= static_cast<uint32_t>(s->num_sms);
+  const bool fused = s->cfg.pipeline_mode != 1 && R >= 2;
   if (fused) side = stream;
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
   const uint8_t* qd = static_cast<const uint8_t*>(q);
@@ -1062,7 +1184,11 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
   }
-  for (uint32_t l = 0; l < L; ++l) {
+  if (step) {
+    rc = do_step(s, p, qd, Hq, sm_scale, od, stream, wrap != 0);
+    if (rc) return rc;
+  }
+  for (uint32_t l = 0; l < L && !step; ++l) {
     // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.
     int next = -1;
     if (p->k) {

@@ -252,10 +252,10 @@ def test_copy_blocks_matches_index_select(kind, n, bb):
     assert torch.equal(dst2, src[src_idx.long()])
 
 
-@pytest.mark.parametrize("mode,layers,static", [(0, 5, 0), (1, 5, 0), (0, 4, 1), (1, 4, 1)])
+@pytest.mark.parametrize("mode,layers,static", [(0, 5, 0), (0, 4, 1), (0, 4, 0), (1, 5, 0), (1, 4, 1), (2, 5, 0), (2, 4, 1)])
 def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, static):
-    """Both pipelines (fused: attention + next layer's gather in one launch; two streams with
-    events), odd and even layer counts on a ring of two, three passes each."""
+    """All three pipelines (0: one persistent launch per pass; 1: two streams with events; 2: one
+    fused launch per layer), odd and even layer counts on a ring of two, three passes each."""
     wl = synth.Workload("pipe", layers, 32, 8, 7, 100, 1200, 0.4)
     sc = Scenario(wl, 9)
     g = _gpu(sc, flags=B.FLAG_PROFILE, pipeline_mode=mode, static_split=static, decode_ctas=12)
@@ -276,7 +276,7 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
     times = g.s.slice_layer_times()
     assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
     trace = g.s.slice_cta_trace(0)
-    assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 1] >= trace[:, :, 0]).all()
+    assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 0] > 0).all()      # every CTA visited every layer
     # the staged bytes left in the ring are the oracle's
     from tests.gpu_helpers import to_host
     for slot in range(wl.ring_slots):
