@@ -44,6 +44,10 @@ def parse_args():
     ap.add_argument("--copy-kind", type=int, default=0)
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--decode-ctas", type=int, default=0)
+    ap.add_argument("--pipeline-mode", type=int, default=0,
+                    help="0 one persistent launch per pass, 1 two streams with events, 2 one fused launch per layer")
+    ap.add_argument("--static-split", type=int, default=0, help="1: no work stealing between CTAs")
+    ap.add_argument("--no-ablations", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
@@ -51,16 +55,17 @@ def parse_args():
     return ap.parse_args()
 
 
-def profile_traffic(wl):
-    """DRAM bytes per launch of the attention kernel from the committed ncu summary (same per-launch
-    work as the benchmark's: one layer of the full batch); None for other workloads."""
-    path = os.path.join(ROOT, "profiles", "paged_decode_kernel_llama3_8b_batch64_ncu_full.md")
-    if wl.name != "llama3_8b_decode" or wl.batch != 64 or not os.path.exists(path):
+def profile_traffic(wl, mode):
+    """DRAM bytes per launch of the layer kernel from the committed ncu summary. The capture ran the
+    full batch on 2 layers; traffic grows in proportion to the layers a launch spans, so it is scaled
+    by layers. None for other workloads or pipelines."""
+    path = os.path.join(ROOT, "profiles", "slice_layer_kernel_llama3_8b_batch64_ncu.md")
+    if wl.name != "llama3_8b_decode" or wl.batch != 64 or mode != 0 or not os.path.exists(path):
         return None
     with open(path) as f:
         for line in f:
-            if line.strip().startswith("traffic_bytes_per_launch:"):
-                return int(line.split(":")[1])
+            if line.strip().startswith("traffic_bytes_per_layer:"):
+                return int(line.split(":")[1]) * wl.num_layers
     return None
 
 
@@ -79,7 +84,7 @@ class DeviceWorkload:
     """Arenas, tables and query tensors of one workload on the current CUDA device."""
 
     def __init__(self, wl: synth.Workload, seed: int, flags: int = 0, copy_kind: int = 0, copy_ctas: int = 0,
-                 decode_ctas: int = 0):
+                 decode_ctas: int = 0, pipeline_mode: int = 0, static_split: int = 0):
         import torch
         from paper_2609_27040_b200 import binding as B
         self.wl, self.B = wl, B
@@ -108,7 +113,8 @@ class DeviceWorkload:
                          local=self.local, lent=self.lent, staging=self.staging, ring_slots=wl.ring_slots,
                          max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks, flags=flags,
                          local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order,
-                         copy_kind=copy_kind, copy_ctas=copy_ctas, decode_ctas=decode_ctas)
+                         copy_kind=copy_kind, copy_ctas=copy_ctas, decode_ctas=decode_ctas,
+                         pipeline_mode=pipeline_mode, static_split=static_split)
         t0 = time.perf_counter()
         for i, hints in enumerate(pl.hints):
             for h in hints:
@@ -285,8 +291,9 @@ def run_ours(args, wl):
     B.lib()
 
     # Replicas only: every rank runs the same workload shape on its own GPU with its own seed.
-    w = DeviceWorkload(wl, args.seed + rank, copy_kind=args.copy_kind, copy_ctas=args.copy_ctas,
-                       decode_ctas=args.decode_ctas)
+    kw = dict(copy_kind=args.copy_kind, copy_ctas=args.copy_ctas, decode_ctas=args.decode_ctas,
+              static_split=args.static_split)
+    w = DeviceWorkload(wl, args.seed + rank, pipeline_mode=args.pipeline_mode, **kw)
     wrap = not args.no_wrap
     for _ in range(max(args.warmup, 3)):
         w.step(wrap)
@@ -327,75 +334,103 @@ def run_ours(args, wl):
     else:
         t_e2e_step = t_e2e / e2e_steps
 
-    # ---- per-layer kernel times inside the pipelined pass (profile events), rank 0 ----
+    # ---- the dominant kernel inside the pipelined pass (profile events + per-CTA trace), rank 0 ----
     roof = None
     extra = {}
     if rank == 0:
+        step_bytes, tokens, pl_blocks, k_blocks = w.step_bytes, w.tokens, w.pl.total_blocks, w.pl.staging_blocks
+        attn_bytes_layer, pref_bytes_layer = w.attn_bytes_layer, w.pref_bytes_layer
         del w
         torch.cuda.empty_cache()
-        wp = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, copy_kind=args.copy_kind, copy_ctas=args.copy_ctas,
-                            decode_ctas=args.decode_ctas)
+        peak, peak_src = measured_peaks()
+        L = wl.num_layers
+        reps = max(3, min(args.steps, 20))
+        wp = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, pipeline_mode=args.pipeline_mode, **kw)
         for _ in range(3):
             wp.step(wrap)
-        attn_us, pref_us, stall_us, layer_us = [], [], [], []
-        for _ in range(max(3, min(args.steps, 20))):
-            wp.step(wrap)
-            tm = wp.s.slice_layer_times().astype(np.float64)     # synchronises
-            attn_us.append(tm[:, 4] - tm[:, 2])                  # attention kernel proper
-            pref_us.append(tm[:, 1] - tm[:, 0])
-            prev_end = np.concatenate(([tm[0, 2]], tm[:-1, 3]))  # end of the previous layer's attention
-            stall_us.append(np.maximum(0.0, tm[:, 1] - prev_end))
-            layer_us.append(tm[:, 3] - prev_end)
-        attn = float(np.nanmean(np.stack(attn_us)))
-        pref = float(np.nanmean(np.stack(pref_us)))
-        stall = float(np.nanmean(np.stack(stall_us)[:, 1:]))
-        layer = float(np.nanmean(np.stack(layer_us)[:, 1:]))
-        peak, peak_src = measured_peaks()
-        achieved = wp.attn_bytes_layer / (attn * 1e-6) / 1e9
-        combined = wp.step_bytes * args.steps / t / 1e9
-        roof = {"bound": "hbm", "kernel": "paged_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": f"of {peak_src}",
-                "note": "attention kernel timed inside the pipelined pass, where the concurrent gather takes its "
-                        "share of HBM; 'combined' counts attention + gather bytes over the step time",
-                "combined": {"achieved": combined, "frac": combined / peak, "frac_of_nominal_8TBs": combined / NOMINAL_HBM_GBS},
-                "algorithmic_bytes_per_launch": wp.attn_bytes_layer}
-        extra = {"attn_us_per_layer": attn, "prefetch_us_per_layer": pref, "stall_us_per_layer": stall,
-                 "layer_us": layer, "stall_frac_of_attention": stall / attn if attn else None,
-                 "alloc_seconds_setup": wp.alloc_s}
-        # On-demand ablation: the same pass with prefetch and attention serialised on ONE stream
-        # (no overlap). Its profile events give each kernel's duration without a concurrent kernel.
-        for _ in range(2):
-            assert wp.s.slice_decode_step(wp.seqs, wp.q, wl.num_q_heads, wp.scale, wp.out, False, wrap, wp.main, wp.main) == 0
-        iso_attn, iso_pref, iso_merge = [], [], []
-        reps = max(3, min(args.steps, 10))
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t_serial = 0.0
+        kernel_us, stall_mean, stall_max, launches_per_step = [], [], [], None
         for _ in range(reps):
-            e0.record(wp.main)
-            assert wp.s.slice_decode_step(wp.seqs, wp.q, wl.num_q_heads, wp.scale, wp.out, False, wrap, wp.main, wp.main) == 0
-            e1.record(wp.main)
-            tm = wp.s.slice_layer_times().astype(np.float64)
-            t_serial += e0.elapsed_time(e1) / 1e3
-            iso_attn.append(tm[:, 4] - tm[:, 2])
-            iso_merge.append(tm[:, 3] - tm[:, 4])
-            iso_pref.append(tm[:, 1] - tm[:, 0])
-        iso_us = float(np.nanmean(np.stack(iso_attn)))
-        iso_pref_us = float(np.nanmean(np.stack(iso_pref)))
-        roof["isolated"] = {"achieved": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9, "us_per_launch": iso_us,
-                            "frac": wp.attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak,
-                            "what": "same kernel with no concurrent gather (serialised pass)"}
-        roof["traffic"] = profile_traffic(wl)
-        extra["gather_kernel_isolated"] = {"us_per_launch": iso_pref_us, "algorithmic_bytes": wp.pref_bytes_layer,
-                                           "achieved_gbs": wp.pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9,
-                                           "frac": wp.pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9 / peak}
-        extra["merge_us_per_launch"] = float(np.nanmean(np.stack(iso_merge)))
-        extra["ablation_serialised_prefetch"] = {"tokens_per_s": wl.batch * reps / t_serial,
-                                                 "ms_per_step": t_serial / reps * 1e3,
-                                                 "note": "on-demand variant: prefetch not overlapped with attention"}
-        step_bytes, tokens, pl_blocks, k_blocks = wp.step_bytes, wp.tokens, wp.pl.total_blocks, wp.pl.staging_blocks
+            k0 = wp.s.slice_stats()["kernel_launches"]
+            wp.step(wrap)
+            tm = wp.s.slice_layer_times().astype(np.float64)         # synchronises
+            launches_per_step = wp.s.slice_stats()["kernel_launches"] - k0
+            if args.pipeline_mode == 0:
+                kernel_us.append(float(tm[L - 1, 3] - tm[0, 2]))     # one launch spans the pass
+            else:
+                kernel_us.append(float(np.nansum(tm[:, 4] - tm[:, 2])))
+            tr = wp.s.slice_cta_trace(0).astype(np.float64)
+            wait_us = tr[:, :, 1] / 1e3                               # [layer][cta] ns the attention waited
+            stall_mean.append(wait_us[1:].mean())
+            stall_max.append(wait_us[1:].max(axis=1).mean())
+        kernel_s = float(np.mean(kernel_us)) * 1e-6
+        algo = step_bytes if args.pipeline_mode != 1 else L * attn_bytes_layer
+        achieved = algo / kernel_s / 1e9
+        combined = step_bytes * args.steps / t / 1e9
+        name = {0: "slice_layer_kernel (one launch per pass: attention + gather of every layer)",
+                1: "slice_layer_kernel (attention only; gather in copy_blocks_vector on a second stream)",
+                2: "slice_layer_kernel (one launch per layer: attention + gather of the next layer)"}[args.pipeline_mode]
+        roof = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": profile_traffic(wl, args.pipeline_mode),
+                "peak_source": f"of {peak_src}", "launches_per_step": launches_per_step,
+                "launch_us": kernel_s * 1e6 / max(launches_per_step, 1) if args.pipeline_mode != 1 else None,
+                "algorithmic_bytes_per_launch": algo // max(launches_per_step, 1) if args.pipeline_mode != 1 else attn_bytes_layer,
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "combined_over_step_time": {"achieved": combined, "frac": combined / peak,
+                                            "frac_of_nominal_8TBs": combined / NOMINAL_HBM_GBS}}
+        attn_layer_us = kernel_s * 1e6 / L
+        extra = {"layer_us": attn_layer_us, "stall_us_per_layer": float(np.mean(stall_mean)),
+                 "stall_us_per_layer_worst_cta": float(np.mean(stall_max)),
+                 "stall_frac_of_layer": float(np.mean(stall_mean)) / attn_layer_us,
+                 "stall_definition": "time a CTA's attention waits for the layer's prefetched blocks (device timer), "
+                                     "mean over CTAs and layers; worst_cta = mean over layers of the slowest CTA",
+                 "alloc_seconds_setup": wp.alloc_s}
         del wp
         torch.cuda.empty_cache()
+        if not args.no_ablations:
+            # Other pipelines on the same workload: one fused launch per layer; two kernels on two
+            # streams; and the on-demand variant (gather and attention serialised on one stream), whose
+            # profile events also give each kernel's duration with nothing running beside it.
+            abl = {}
+            for label, mode in (("fused_launch_per_layer", 2), ("two_streams", 1)):
+                if mode == args.pipeline_mode:
+                    continue
+                wa = DeviceWorkload(wl, args.seed, pipeline_mode=mode, **kw)
+                for _ in range(3):
+                    wa.step(wrap)
+                ta = wa.timed(reps, wrap)
+                abl[label] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
+                              "hbm_gbs_combined": step_bytes * reps / ta / 1e9}
+                del wa
+                torch.cuda.empty_cache()
+            ws = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, pipeline_mode=1, **kw)
+            for _ in range(2):
+                assert ws.s.slice_decode_step(ws.seqs, ws.q, wl.num_q_heads, ws.scale, ws.out, False, wrap, ws.main, ws.main) == 0
+            iso_attn, iso_pref = [], []
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t_serial = 0.0
+            for _ in range(max(3, reps // 2)):
+                e0.record(ws.main)
+                assert ws.s.slice_decode_step(ws.seqs, ws.q, wl.num_q_heads, ws.scale, ws.out, False, wrap, ws.main, ws.main) == 0
+                e1.record(ws.main)
+                tm = ws.s.slice_layer_times().astype(np.float64)
+                t_serial += e0.elapsed_time(e1) / 1e3
+                iso_attn.append(tm[:, 4] - tm[:, 2])
+                iso_pref.append(tm[:, 1] - tm[:, 0])
+            n_ser = max(3, reps // 2)
+            iso_us, iso_pref_us = float(np.nanmean(np.stack(iso_attn))), float(np.nanmean(np.stack(iso_pref)))
+            abl["serialised_prefetch"] = {"tokens_per_s": wl.batch * n_ser / t_serial, "ms_per_step": t_serial / n_ser * 1e3,
+                                          "note": "on-demand variant: prefetch not overlapped with attention"}
+            extra["ablations"] = abl
+            extra["kernels_alone"] = {
+                "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
+                                                "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
+                                                "frac": attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak},
+                "copy_blocks_vector_gather": {"us_per_launch": iso_pref_us, "algorithmic_bytes": pref_bytes_layer,
+                                              "achieved_gbs": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9,
+                                              "frac": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9 / peak}}
+            del ws
+            torch.cuda.empty_cache()
     clocks = sampler.stop()
 
     if rank != 0:
@@ -424,7 +459,7 @@ def run_ours(args, wl):
                    "kv_heads": wl.num_kv_heads, "head_dim": wl.head_dim, "block_tokens": wl.block_tokens,
                    "len_range": [wl.len_lo, wl.len_hi], "lent_fraction": wl.lent_fraction, "ring_slots": wl.ring_slots,
                    "tokens_in_batch": tokens, "blocks": pl_blocks, "lent_blocks": k_blocks,
-                   "parallelism": "replicas" if world > 1 else "single",
+                   "parallelism": "replicas" if world > 1 else "single", "pipeline_mode": args.pipeline_mode,
                    "l2": "inputs larger than L2: every step streams %.1f GB of KV" % (step_bytes / 1e9)},
         "hbm_gbs_combined": step_bytes * world * args.steps / t / 1e9,
         "roofline": roof, "cpu_baseline": cpu,

@@ -244,8 +244,9 @@ int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers);
 
 /* With SLICE_FLAG_PROFILE: per-CTA times (GPU nanosecond timer) of the most recent launch of each
  * layer's kernel, as [num_layers][ctas_per_layer][words_per_cta] uint64 on the host; unused entries
- * are 0. which = 0: layer kernel, 4 words (start, end of the CTA's attention work, end of its copy
- * work, SM id); which = 1: stand-alone gather kernel, 2 words (start, end). out may be NULL to query
+ * are 0. which = 0: layer kernel, 4 words (time the CTA started on the layer, nanoseconds its
+ * attention waited for the layer's prefetched blocks, end of the copy work it did during the layer,
+ * SM id | runs << 16 | claims << 32); which = 1: stand-alone gather kernel, 2 words (start, end). out may be NULL to query
  * the two sizes. Synchronises the device. */
 int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entries, uint32_t* ctas_per_layer,
                     uint32_t* words_per_cta);

@@ -38,14 +38,13 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
 // Device counters of ONE layer inside a layer-kernel launch; the whole block must be zero when the
 // kernel starts. Layout in uint32 words:
 //   [0, 16)                 launch words: [1] next copy unit of the gather issued during this layer,
-//                           [2] attention work finished (blocks x KV heads), [3] gathered blocks of
-//                           THIS layer that have landed in its ring slot, [4] merges finished
+//                           [2] attention work finished (blocks x KV heads), [4] merges finished
 //   [16, 16 + 2*ncta)       one 64-bit claim word per CTA range: blocks claimed from the front (low
 //                           half, by the owner) and from the back (high half, by thieves)
 //   [.., + nseq)            partial slots handed out per sequence
 //   [.., + nseq*Hkv)        blocks finished per (sequence, KV head)
 constexpr uint32_t kLaunchCounters = 16;
-constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntGathered = 3, kCntMerged = 4;
+constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntMerged = 4;
 constexpr uint32_t kMaxStepLayers = 128;
 inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
   return kLaunchCounters + 2 * static_cast<size_t>(ncta) + nseq + static_cast<size_t>(nseq) * Hkv;
@@ -89,11 +88,15 @@ struct LayerParams {
   const uint8_t* lent_base;     // lent arena of layer 0
   uint64_t lent_layer_stride, lent_block_stride;
   const int32_t* copy_src;      // [copy_n] lent entries in staging order
+  const uint32_t* copy_order;   // [copy_n] staging positions in the order they are gathered
   uint32_t copy_n;
+  uint32_t* ready;              // [ring_slots][ready_stride] per staged position: epoch of the layer
+  uint32_t ready_stride;        //   whose block has landed there (multi-layer launches)
+  uint32_t epoch_base;          // epoch of first_layer; layer l has epoch_base + (l - first_layer)
   int16_t gather_target[kMaxStepLayers];
   int16_t gather_after[kMaxStepLayers];
   int* status;
-  unsigned long long* trace;    // optional, per layer [ncta][4]: start, attention end, copy end, info
+  unsigned long long* trace;    // optional, per layer [ncta][4]: start, ns waited for the gather, copy end, info
   uint64_t trace_stride;        // words from one layer's trace to the next
 };
 

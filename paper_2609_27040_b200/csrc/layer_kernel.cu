@@ -54,11 +54,13 @@ namespace ema {
 
 namespace {
 
-constexpr int kNA = 4;                     // attention ring: half-block stages
+constexpr uint32_t kNAFused = 4;           // attention ring (half-block stages) beside a copy ring
+constexpr uint32_t kNAAlone = 6;           // ... and when the launch gathers nothing: the copy ring's memory too
+constexpr uint32_t kNAMax = 6;
 constexpr int kNC = 5;                     // copy ring: 16 KB stages
 constexpr int kCopyLoadsAhead = 3;         // loads in flight; the other stages drain as stores
 constexpr uint32_t kCopyChunk = 16384;
-constexpr int kQueue = 8;                  // unit descriptors in flight (> kNA / 2 + 1)
+constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAMax / 2 + 1)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRowPad = 16;
@@ -83,10 +85,11 @@ struct Claim {
 };
 
 struct Smem {
+  uint32_t na;          // attention ring stages in use
   uint8_t* att_ring;
   uint8_t* copy_ring;
-  uint64_t* att_full;   // [kNA]
-  uint64_t* att_empty;  // [kNA]
+  uint64_t* att_full;   // [kNAMax]
+  uint64_t* att_empty;  // [kNAMax]
   uint64_t* copy_full;  // [kNC]
   UnitDesc* queue;      // [kQueue]
   uint8_t** copy_dst;   // [kNC]
@@ -95,26 +98,28 @@ struct Smem {
 };
 
 // Bookkeeping area behind the two rings; every part 16-byte aligned.
-constexpr size_t kBarBytes = 16 * sizeof(uint64_t);
+constexpr size_t kBarBytes = 24 * sizeof(uint64_t);
 constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
 constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
 constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
-static_assert(2 * kNA + kNC <= 16 && kNC <= 8, "bookkeeping area too small");
+static_assert(2 * kNAMax + kNC <= 24 && kNC <= 8, "bookkeeping area too small");
+static_assert(kNAFused * 33024 + kNC * 16384 >= kNAAlone * 33024, "the deeper ring must fit in the fused layout");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
-  return static_cast<size_t>(kNA) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
+  return static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes;
 }
 
-__device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv) {
+__device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
   Smem s;
+  s.na = gathers ? kNAFused : kNAAlone;
   s.att_ring = base;
-  s.copy_ring = base + static_cast<size_t>(kNA) * half_stage_bytes(Hkv);
+  s.copy_ring = base + static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv);
   uint8_t* p = s.copy_ring + static_cast<size_t>(kNC) * kCopyChunk;
   s.att_full = reinterpret_cast<uint64_t*>(p);
-  s.att_empty = s.att_full + kNA;
-  s.copy_full = s.att_empty + kNA;
+  s.att_empty = s.att_full + kNAMax;
+  s.copy_full = s.att_empty + kNAMax;
   s.queue = reinterpret_cast<UnitDesc*>(p + kBarBytes);
   s.copy_dst = reinterpret_cast<uint8_t**>(p + kBarBytes + kQueueBytes);
   s.copy_len = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes);
@@ -135,6 +140,20 @@ __device__ __forceinline__ uint32_t* seq_counts(const LayerParams& p, uint32_t l
 __device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p, uint32_t li) { return seq_counts(p, li) + p.nseq; }
 __device__ __forceinline__ float* part_o_of(const LayerParams& p, uint32_t li) { return p.part_o + (li & 1u) * p.part_o_stride; }
 __device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) { return p.part_ml + (li & 1u) * p.part_ml_stride; }
+
+// Bounded wait until a device word written by another CTA equals `value`.
+__device__ __forceinline__ bool wait_counter_eq(const uint32_t* word, uint32_t value, int* status) {
+  if (__ldcg(word) == value) return true;
+  const uint64_t t0 = ptx::global_timer_ns();
+  while (__ldcg(word) != value) {
+    if (ptx::global_timer_ns() - t0 > kWaitNs) {
+      if (status) atomicExch(status, kDevTimeout);
+      return false;
+    }
+    __nanosleep(64);
+  }
+  return true;
+}
 
 // Bounded wait until a device counter written by other CTAs reaches `target`.
 __device__ __forceinline__ bool wait_counter(const uint32_t* cnt, uint32_t target, int* status) {
@@ -169,10 +188,17 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     unsigned long long* rw = range_words(p, li);
     uint32_t* seq_count = seq_counts(p, li);
     uint32_t cur_seq = kSentinel, nruns = 0, nclaims = 0;
-    // Staged blocks of this layer may be read once its gather (issued during the previous layer of
-    // this launch) has landed completely; the first layer's gather precedes the launch in stream order.
-    bool staged_ok = li == 0 || p.gather_target[li - 1] != static_cast<int16_t>(layer);
-    if (p.trace && lane == 0) p.trace[li * p.trace_stride + 4 * blockIdx.x] = ptx::global_timer_ns();
+    // A staged block of this layer may be read once the gather issued during the previous layer of
+    // this launch has landed it (per-position ready flags carrying the layer's epoch); the first
+    // layer's gather precedes the launch in stream order, as does any gather the host skipped.
+    const bool check_ready = li > 0 && p.gather_target[li - 1] == static_cast<int16_t>(layer);
+    const uint32_t* ready = p.ready + static_cast<size_t>(layer % p.ring_slots) * p.ready_stride;
+    const uint32_t epoch = p.epoch_base + li;
+    uint64_t waited_ns = 0;
+    if (p.trace && lane == 0) {
+      p.trace[li * p.trace_stride + 4 * blockIdx.x] = ptx::global_timer_ns();
+      p.trace[li * p.trace_stride + 4 * blockIdx.x + 1] = 0;
+    }
     // The partial buffer of this layer's parity was last used two layers ago: its merges must be done.
     if (li >= 2) {
       ok = wait_counter(layer_counters(p, li - 2) + kCntMerged, p.nseq * Hkv, p.status);
@@ -186,20 +212,25 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       for (uint32_t b0 = 0; b0 < nb && ok; b0 += 32) {
         const uint32_t cnt = min(32u, nb - b0);
         const int32_t my = lane < cnt ? p.resolved[flat + b0 + lane] : 0;
+        // Ready flags of this batch of blocks, fetched together (a flag that is not there yet is
+        // polled below).
+        uint32_t my_ready = epoch;
+        if (check_ready && lane < cnt && my < 0) my_ready = __ldcg(ready + static_cast<uint32_t>(~my));
         for (uint32_t j = 0; j < cnt && ok; ++j) {
           const int32_t e = __shfl_sync(0xffffffffu, my, j);
-          if (e < 0 && !staged_ok) {
-            ok = wait_counter(layer_counters(p, li) + kCntGathered, p.copy_n, p.status);
+          if (check_ready && e < 0 && __shfl_sync(0xffffffffu, my_ready, j) != epoch) {
+            const uint64_t w0 = ptx::global_timer_ns();
+            ok = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
-            staged_ok = true;
+            waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
           }
           const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
                                       : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
 #pragma unroll
           for (uint32_t plane = 0; plane < 2; ++plane, ++hs) {
-            const uint32_t stg = hs % kNA;
-            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
+            const uint32_t stg = hs % sm.na;
+            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / sm.na) & 1u) ^ 1u, p.status, kDevTimeout);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
             const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
@@ -333,14 +364,15 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     if (p.trace && lane == 0) {
       uint32_t smid;
       asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      p.trace[li * p.trace_stride + 4 * blockIdx.x + 1] = waited_ns;
       p.trace[li * p.trace_stride + 4 * blockIdx.x + 3] =
           smid | (static_cast<unsigned long long>(nruns) << 16) | (static_cast<unsigned long long>(nclaims) << 32);
     }
   }
   if (ok) {
     // End marker: a descriptor with no data behind it.
-    const uint32_t stg = hs % kNA;
-    ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / kNA) & 1u) ^ 1u, p.status, kDevTimeout);
+    const uint32_t stg = hs % sm.na;
+    ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / sm.na) & 1u) ^ 1u, p.status, kDevTimeout);
     ok = __all_sync(0xffffffffu, ok);
     if (ok && lane == 0) {
       sm.queue[nq % kQueue] = UnitDesc{kSentinel, 0, 0, 0, 0, 0, 0, 0};
@@ -349,9 +381,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   }
   if (!ok) {
     // Bounded second chance for copies already issued, so that none lands after the CTA is gone.
-    const uint32_t from = hs > static_cast<uint32_t>(kNA) ? hs - kNA : 0;
+    const uint32_t from = hs > sm.na ? hs - sm.na : 0;
     for (uint32_t k = from; k < hs; ++k)
-      ptx::mbar_wait(ptx::smem_u32(&sm.att_full[k % kNA]), (k / kNA) & 1u, nullptr, 0);
+      ptx::mbar_wait(ptx::smem_u32(&sm.att_full[k % sm.na]), (k / sm.na) & 1u, nullptr, 0);
   }
 }
 
@@ -555,13 +587,13 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm) {
 
 // Waits for the next half-stage; false when the bounded wait expired anywhere in the warp.
 __device__ __forceinline__ bool wait_stage(const LayerParams& p, const Smem& sm, uint32_t hs) {
-  const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[hs % kNA]), (hs / kNA) & 1u, p.status, kDevTimeout);
+  const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[hs % sm.na]), (hs / sm.na) & 1u, p.status, kDevTimeout);
   return __all_sync(0xffffffffu, ok);
 }
 
 __device__ __forceinline__ void release_stage(const Smem& sm, uint32_t hs) {
   __syncwarp();
-  if ((threadIdx.x & 31u) == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[hs % kNA]));
+  if ((threadIdx.x & 31u) == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[hs % sm.na]));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -644,11 +676,11 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       const uint32_t valid = min(kT, len - b * kT);
       uint32_t pb0, pb1;
       float al0, al1;
-      tile_mma_scores(ring + (hs % kNA) * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
+      tile_mma_scores(ring + (hs % sm.na) * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
       release_stage(sm, hs);
       ++hs;
       if (!wait_stage(p, sm, hs)) return;
-      tile_mma_pv(ring + (hs % kNA) * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
+      tile_mma_pv(ring + (hs % sm.na) * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
       release_stage(sm, hs);
       ++hs;
     }
@@ -718,11 +750,11 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       if (b != it.blk_begin && !wait_stage(p, sm, hs)) return;
       const uint32_t valid = min(kT, len - b * kT);
       float pw, al;
-      tile_alu_scores(sm.att_ring + (hs % kNA) * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
+      tile_alu_scores(sm.att_ring + (hs % sm.na) * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
       release_stage(sm, hs);
       ++hs;
       if (!wait_stage(p, sm, hs)) return;
-      tile_alu_pv(sm.att_ring + (hs % kNA) * hsb, pitch, head_off, valid, pw, al, o);
+      tile_alu_pv(sm.att_ring + (hs % sm.na) * hsb, pitch, head_off, valid, pw, al, o);
       release_stage(sm, hs);
       ++hs;
     }
@@ -752,9 +784,13 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     const uint8_t* src_layer = p.lent_base + static_cast<uint64_t>(target) * p.lent_layer_stride;
     uint8_t* dst_slot = const_cast<uint8_t*>(p.staging_base) + (static_cast<uint32_t>(target) % p.ring_slots) * p.slot_bytes;
     uint32_t* ticket = layer_counters(p, li) + kCntCopyTicket;
-    // Landed blocks are reported to the target layer's counter when the target is in this launch.
+    // A landed block is announced by writing the target layer's epoch to its position's ready flag
+    // (only when the target is attended to later in this launch).
     const bool report = static_cast<uint32_t>(target) > p.first_layer && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
-    uint32_t* landed = report ? layer_counters(p, static_cast<uint32_t>(target) - p.first_layer) + kCntGathered : nullptr;
+    uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
+    const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
+    uint32_t my_pos[16];                  // positions of this thread's most recent units
+    uint32_t my_units = 0;                // units of this layer taken by this thread
     uint32_t piece = pieces;  // forces a unit fetch
     const uint8_t* src_blk = nullptr;
     uint8_t* dst_blk = nullptr;
@@ -767,9 +803,12 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       if (piece == pieces) {
         const uint32_t unit = atomicAdd(ticket, 1u);
         if (unit >= p.copy_n) return false;
-        const int32_t e = p.copy_src[unit];
+        const uint32_t pos = p.copy_order[unit];
+        const int32_t e = p.copy_src[pos];
         src_blk = src_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
-        dst_blk = dst_slot + static_cast<uint64_t>(unit) * p.block_bytes;
+        dst_blk = dst_slot + static_cast<uint64_t>(pos) * p.block_bytes;
+        my_pos[my_units % 16] = pos;
+        ++my_units;
         piece = 0;
       }
       const uint64_t off = static_cast<uint64_t>(piece) * kCopyChunk;
@@ -787,12 +826,11 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     };
     // Reports the units all of whose pieces are among the first `complete` stored pieces of this layer.
     auto report_landed = [&](uint32_t complete) {
-      if (!landed) return;
+      if (!ready) return;
       const uint32_t units = complete / pieces;
       if (units > reported) {
         __threadfence();
-        atomicAdd(landed, units - reported);
-        reported = units;
+        for (; reported < units; ++reported) ready[my_pos[reported % 16]] = epoch;
       }
     };
 
@@ -825,10 +863,13 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
 template <bool kMma>
 __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  const Smem sm = carve(smem_raw, p.Hkv);
+  bool gathers = false;
+  if (p.copy_n)
+    for (uint32_t li = 0; li < p.num_layers; ++li) gathers |= p.gather_target[li] >= 0;
+  const Smem sm = carve(smem_raw, p.Hkv, gathers);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kNA; ++s) {
+    for (uint32_t s = 0; s < kNAMax; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sm.att_full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), p.Hkv);
     }
@@ -844,8 +885,6 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     else
       consumer_alu(p, sm, warp);
     __syncwarp();
-    if (p.trace && warp == 0 && lane == 0)
-      p.trace[(p.num_layers - 1) * p.trace_stride + 4 * blockIdx.x + 1] = ptx::global_timer_ns();
     if (lane == 0) {
       __threadfence_block();
       atomicAdd(&sm.mq[kMq + 2], 1u);  // this consumer warp queues no more merges

@@ -45,7 +45,7 @@ struct Plan {
   uint32_t slots = 0, slots_static = 0;  // partial slots with / without work stealing
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
-  size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_blk_off = 0, off_slot_base = 0,
+  size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_blk_off = 0, off_slot_base = 0,
          off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
   uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
@@ -101,7 +101,9 @@ struct ema_slice {
   float* part_o = nullptr;
   float* part_ml = nullptr;
   size_t part_rows = 0;         // partial rows (segments * query heads) currently allocated
-  uint32_t* cnt_dev = nullptr;  // [num_layers][kLaunchCounters], then merge counters [max_seqs * Hkv]
+  uint32_t* cnt_dev = nullptr;  // [num_layers][cnt_stride] device counters of the layer kernel
+  uint32_t* ready_dev = nullptr;  // [ring_slots][staging_blocks_per_slot] ready flags (epochs)
+  uint32_t epoch = 1;
   int* dev_status = nullptr;
   // reclaim
   int32_t* reclaim_host = nullptr;
@@ -171,7 +173,7 @@ size_t plan_capacity(const ema_slice* s) {
   size_t b = 0;
   b += 2 * align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved, blk_seq (upper bound)
   b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                              // lens
-  b += align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);               // copy_src
+  b += 2 * align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src, copy_order
   b += 3 * align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // blk_off, slot bases
   b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos
   return b;
@@ -274,6 +276,8 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.off_copy_src = off;
   off += align_up(static_cast<size_t>(k) * 4, 256);
+  p.off_copy_order = off;
+  off += align_up(static_cast<size_t>(k) * 4, 256);
   p.off_blk_off = off;
   off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
   p.off_slot_base = off;
@@ -291,7 +295,9 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   uint32_t* blk_seq = reinterpret_cast<uint32_t*>(p.host + p.off_blk_seq);
   uint32_t* lens = reinterpret_cast<uint32_t*>(p.host + p.off_lens);
   int32_t* copy_src = reinterpret_cast<int32_t*>(p.host + p.off_copy_src);
+  uint32_t* copy_order = reinterpret_cast<uint32_t*>(p.host + p.off_copy_order);
   uint32_t* blk_off = reinterpret_cast<uint32_t*>(p.host + p.off_blk_off);
+  std::vector<uint32_t> pos_range(k), pos_rank(k), range_staged(p.used_cta + 1, 0);
   uint32_t* slot_base = reinterpret_cast<uint32_t*>(p.host + p.off_slot_base);
   uint32_t* slot_base_static = reinterpret_cast<uint32_t*>(p.host + p.off_slot_base_static);
   int32_t* home = reinterpret_cast<int32_t*>(p.host + p.off_home);
@@ -320,6 +326,8 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
       if (e < 0) {
         copy_src[kk] = e;  // negative entry: tier 1 (lent arena), id ~e
         r = ~static_cast<int32_t>(kk);
+        pos_range[kk] = flat / per;
+        pos_rank[kk] = range_staged[flat / per]++;
         ++kk;
       }
       resolved[flat] = r;
@@ -336,6 +344,17 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   slot_base_static[nseq] = slots_static;
   p.slots = std::max(slots, 1u);
   p.slots_static = std::max(slots_static, 1u);
+  // Order in which the fused kernel gathers the staged positions: the first staged block of every
+  // CTA range, then the second of every range, ... A CTA reads its range front to back, so what it
+  // needs first lands first and what lands last is needed last.
+  {
+    uint32_t max_rank = 0;
+    for (uint32_t c = 0; c < p.used_cta; ++c) max_rank = std::max(max_rank, range_staged[c]);
+    std::vector<uint32_t> start(max_rank + 1, 0);
+    for (uint32_t j = 0; j < kk; ++j) ++start[pos_rank[j] + 1];
+    for (uint32_t r = 0; r < max_rank; ++r) start[r + 1] += start[r];
+    for (uint32_t j = 0; j < kk; ++j) copy_order[start[pos_rank[j]]++] = j;  // positions ascend within a rank
+  }
   p.guarded = false;
   p.valid = true;
   s->st.plans_built++;
@@ -505,7 +524,11 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.lent_layer_stride = s->lent_ls;
   d.lent_block_stride = s->lent_bs;
   d.copy_src = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
+  d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order);
   d.copy_n = p->k;
+  d.ready = s->ready_dev;
+  d.ready_stride = s->cfg.staging_blocks_per_slot;
+  d.epoch_base = 0;
   for (uint32_t i = 0; i < ema::kMaxStepLayers; ++i) d.gather_target[i] = d.gather_after[i] = -1;
   d.status = s->dev_status;
   d.trace = s->trace_layer ? s->trace_layer + static_cast<size_t>(first_layer) * s->ncta * 4 : nullptr;
@@ -634,6 +657,8 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     ema::LayerParams d{};
     fill_common(s, p, d, 0, L, q, out, Hq, sm_scale, s->steal);
     d.counters = s->cnt_dev;
+    d.epoch_base = s->epoch;
+    s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / 2;
     d.part_o_stride = rows * kHeadDim;
     d.part_ml_stride = rows * 4;
@@ -696,6 +721,7 @@ void destroy_impl(ema_slice* s) {
     if (s->part_o) cudaFree(s->part_o);
     if (s->part_ml) cudaFree(s->part_ml);
     if (s->cnt_dev) cudaFree(s->cnt_dev);
+    if (s->ready_dev) cudaFree(s->ready_dev);
     if (s->dev_status) cudaFree(s->dev_status);
     if (s->reclaim_host) cudaFreeHost(s->reclaim_host);
     if (s->reclaim_dev) cudaFree(s->reclaim_dev);
@@ -811,6 +837,9 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     const size_t cnt_words = static_cast<size_t>(cfg->num_layers) * s->cnt_stride;
     if (cudaMalloc(reinterpret_cast<void**>(&s->cnt_dev), cnt_words * sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(s->cnt_dev, 0, cnt_words * sizeof(uint32_t)) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+    const size_t rd = static_cast<size_t>(cfg->ring_slots) * std::max(cfg->staging_blocks_per_slot, 1u) * sizeof(uint32_t);
+    if (cudaMalloc(reinterpret_cast<void**>(&s->ready_dev), rd) != cudaSuccess || cudaMemset(s->ready_dev, 0, rd) != cudaSuccess)
       return fail(SLICE_ECUDA);
     const size_t rl = static_cast<size_t>(std::max(cfg->lent_blocks_physical, 1u)) * 2 * sizeof(int32_t);
     if (cudaMallocHost(reinterpret_cast<void**>(&s->reclaim_host), rl) != cudaSuccess) return fail(SLICE_ECUDA);
