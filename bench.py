@@ -101,7 +101,7 @@ class DeviceWorkload:
         for l in range(wl.num_layers):          # N(0,1) bf16 KV, layer by layer
             self.local[l].normal_(generator=gen)
             self.lent[l].normal_(generator=gen)
-        self.staging = torch.zeros((wl.ring_slots, pl.staging_blocks) + shape, device="cuda", dtype=bf)
+        self.staging = torch.zeros((wl.ring_slots, max(pl.staging_blocks, 1)) + shape, device="cuda", dtype=bf)
         self.q = torch.empty((wl.num_layers, wl.batch, wl.num_q_heads, wl.head_dim), device="cuda", dtype=bf)
         self.q.normal_(generator=gen)
         self.out = torch.zeros_like(self.q)

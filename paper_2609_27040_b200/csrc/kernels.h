@@ -70,6 +70,7 @@ struct LayerParams {
   uint32_t per;                 // blocks per CTA range; range c = [c*per, min((c+1)*per, total))
   uint32_t used_cta;            // number of non-empty ranges
   uint32_t allow_steal;         // 0: every range is processed by its owner only
+  uint32_t own_chunk;           // most blocks an owner claims at a time
   const void* q;                // first_layer's [nseq][Hq][128] bf16
   void* out;
   uint64_t io_layer_stride;     // bytes from one layer's q / out to the next

@@ -64,7 +64,6 @@ constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAM
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRowPad = 16;
-constexpr uint32_t kOwnChunk = 8;          // most blocks an owner claims at a time
 constexpr uint32_t kStealMin = 2, kStealMax = 16;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
@@ -78,6 +77,18 @@ __host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return k
 // run's partial slot and the kNewRun flag when the unit starts a new run.
 struct UnitDesc {
   uint32_t seq_idx, blk_begin, blk_end, slot, layer, pad0, pad1, pad2;
+};
+
+// Position in the attention ring: stage index and the parity of its current use, advanced without
+// divisions (the ring depth is a run-time value).
+struct RingPos {
+  uint32_t stg = 0, phase = 0;
+  __device__ __forceinline__ void advance(uint32_t na) {
+    if (++stg == na) {
+      stg = 0;
+      phase ^= 1u;
+    }
+  }
 };
 
 struct Claim {
@@ -179,6 +190,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t plane_bytes = kT * rb;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   uint32_t hs = 0, nq = 0;
+  RingPos pos;
   bool ok = true;
 
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
@@ -228,9 +240,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
                                       : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
 #pragma unroll
-          for (uint32_t plane = 0; plane < 2; ++plane, ++hs) {
-            const uint32_t stg = hs % sm.na;
-            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / sm.na) & 1u) ^ 1u, p.status, kDevTimeout);
+          for (uint32_t plane = 0; plane < 2; ++plane, ++hs, pos.advance(sm.na)) {
+            const uint32_t stg = pos.stg;
+            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
             const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
@@ -291,7 +303,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     // so that little claimed-but-unprocessed work is hidden from thieves near the end.
     uint32_t own_left = 0xFFFFFFFFu;
     auto claim_front = [&](uint32_t c) -> Claim {
-      const uint32_t want = min(kOwnChunk, max(1u, own_left / 4));
+      const uint32_t want = min(p.own_chunk, max(1u, own_left / 4));
       unsigned long long old = 0;
       if (lane == 0) old = atomicAdd(&rw[c], static_cast<unsigned long long>(want));
       old = __shfl_sync(0xffffffffu, old, 0);
@@ -371,8 +383,8 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   }
   if (ok) {
     // End marker: a descriptor with no data behind it.
-    const uint32_t stg = hs % sm.na;
-    ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), ((hs / sm.na) & 1u) ^ 1u, p.status, kDevTimeout);
+    const uint32_t stg = pos.stg;
+    ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
     ok = __all_sync(0xffffffffu, ok);
     if (ok && lane == 0) {
       sm.queue[nq % kQueue] = UnitDesc{kSentinel, 0, 0, 0, 0, 0, 0, 0};
@@ -586,14 +598,14 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm) {
 }
 
 // Waits for the next half-stage; false when the bounded wait expired anywhere in the warp.
-__device__ __forceinline__ bool wait_stage(const LayerParams& p, const Smem& sm, uint32_t hs) {
-  const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[hs % sm.na]), (hs / sm.na) & 1u, p.status, kDevTimeout);
+__device__ __forceinline__ bool wait_stage(const LayerParams& p, const Smem& sm, const RingPos& pos) {
+  const bool ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_full[pos.stg]), pos.phase, p.status, kDevTimeout);
   return __all_sync(0xffffffffu, ok);
 }
 
-__device__ __forceinline__ void release_stage(const Smem& sm, uint32_t hs) {
+__device__ __forceinline__ void release_stage(const Smem& sm, const RingPos& pos) {
   __syncwarp();
-  if ((threadIdx.x & 31u) == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[hs % sm.na]));
+  if ((threadIdx.x & 31u) == 0) ptx::mbar_arrive(ptx::smem_u32(&sm.att_empty[pos.stg]));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -606,7 +618,8 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t head_off = g * kD * 2;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   const uint32_t n = lane >> 2, tig = lane & 3u, r0 = lane >> 2;
-  uint32_t hs = 0, nunit = 0;
+  uint32_t nunit = 0;
+  RingPos pos;
   bool have_run = false;
   uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
@@ -644,7 +657,7 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   };
 
   for (;;) {
-    if (!wait_stage(p, sm, hs)) return;
+    if (!wait_stage(p, sm, pos)) return;
     const UnitDesc it = sm.queue[nunit % kQueue];
     const bool end = it.seq_idx == kSentinel;
     if (end || (it.slot & kNewRun)) {
@@ -672,17 +685,17 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
     }
     ++nunit;
     for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
-      if (b != it.blk_begin && !wait_stage(p, sm, hs)) return;
+      if (b != it.blk_begin && !wait_stage(p, sm, pos)) return;
       const uint32_t valid = min(kT, len - b * kT);
       uint32_t pb0, pb1;
       float al0, al1;
-      tile_mma_scores(ring + (hs % sm.na) * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
-      release_stage(sm, hs);
-      ++hs;
-      if (!wait_stage(p, sm, hs)) return;
-      tile_mma_pv(ring + (hs % sm.na) * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
-      release_stage(sm, hs);
-      ++hs;
+      tile_mma_scores(ring + pos.stg * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      if (!wait_stage(p, sm, pos)) return;
+      tile_mma_pv(ring + pos.stg * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
+      release_stage(sm, pos);
+      pos.advance(sm.na);
     }
     run_blocks += it.blk_end - it.blk_begin;
   }
@@ -697,7 +710,8 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
   const uint32_t half = lane & 1u;
-  uint32_t hs = 0, nunit = 0;
+  uint32_t nunit = 0;
+  RingPos pos;
   bool have_run = false;
   uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
@@ -716,7 +730,7 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   };
 
   for (;;) {
-    if (!wait_stage(p, sm, hs)) return;
+    if (!wait_stage(p, sm, pos)) return;
     const UnitDesc it = sm.queue[nunit % kQueue];
     const bool end = it.seq_idx == kSentinel;
     if (end || (it.slot & kNewRun)) {
@@ -747,16 +761,16 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
     }
     ++nunit;
     for (uint32_t b = it.blk_begin; b < it.blk_end; ++b) {
-      if (b != it.blk_begin && !wait_stage(p, sm, hs)) return;
+      if (b != it.blk_begin && !wait_stage(p, sm, pos)) return;
       const uint32_t valid = min(kT, len - b * kT);
       float pw, al;
-      tile_alu_scores(sm.att_ring + (hs % sm.na) * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
-      release_stage(sm, hs);
-      ++hs;
-      if (!wait_stage(p, sm, hs)) return;
-      tile_alu_pv(sm.att_ring + (hs % sm.na) * hsb, pitch, head_off, valid, pw, al, o);
-      release_stage(sm, hs);
-      ++hs;
+      tile_alu_scores(sm.att_ring + pos.stg * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      if (!wait_stage(p, sm, pos)) return;
+      tile_alu_pv(sm.att_ring + pos.stg * hsb, pitch, head_off, valid, pw, al, o);
+      release_stage(sm, pos);
+      pos.advance(sm.na);
     }
     run_blocks += it.blk_end - it.blk_begin;
   }

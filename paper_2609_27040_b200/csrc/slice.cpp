@@ -21,6 +21,7 @@ constexpr uint32_t kBlockTokens = 16;
 constexpr uint32_t kHeadDim = 128;
 constexpr uint32_t kTraceCopyCtas = 2048;
 constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must match the kernel)
+constexpr uint32_t kOwnChunk = 8;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
   std::vector<int32_t> table;
@@ -506,6 +507,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.per = p->per;
   d.used_cta = p->used_cta;
   d.allow_steal = steal ? 1u : 0u;
+  d.own_chunk = kOwnChunk;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
