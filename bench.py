@@ -358,6 +358,14 @@ def run_ours(args, wl):
                 kernel_us.append(float(tm[L - 1, 3] - tm[0, 2]))     # one launch spans the pass
             else:
                 kernel_us.append(float(np.nansum(tm[:, 4] - tm[:, 2])))
+        del wp
+        torch.cuda.empty_cache()
+        # per-CTA device-timer trace in a pass of its own (the trace costs a few per cent)
+        wp = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=args.pipeline_mode, **kw)
+        for _ in range(3):
+            wp.step(wrap)
+        for _ in range(max(3, reps // 2)):
+            wp.step(wrap)
             tr = wp.s.slice_cta_trace(0).astype(np.float64)
             wait_us = tr[:, :, 1] / 1e3                               # [layer][cta] ns the attention waited
             stall_mean.append(wait_us[1:].mean())

@@ -61,8 +61,8 @@ enum {
 enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
 
 enum {
-  SLICE_FLAG_PROFILE = 1u,     /* record timing events per layer (slice_layer_times) and CTA traces */
-  SLICE_FLAG_TRACE = 2u,       /* per-CTA traces only (slice_cta_trace), no timing events         */
+  SLICE_FLAG_PROFILE = 1u,     /* record timing events around the kernels (slice_layer_times)     */
+  SLICE_FLAG_TRACE = 2u,       /* per-CTA device-timer traces (slice_cta_trace)                    */
   SLICE_FLAG_NULL_DEVICE = 4u  /* tables only: no CUDA call is made, no kernel is launched       */
 };
 
@@ -97,7 +97,9 @@ typedef struct {
   uint32_t static_split;          /* attention work split: 0 = each CTA owns a range of blocks and idle
                                      CTAs steal from the ranges with most left (default); 1 = static
                                      ranges only                                                  */
-  uint32_t reserved;
+  uint32_t claim_blocks;          /* most KV blocks a CTA claims from its own range at a time
+                                     (0 = default); smaller claims leave more for idle CTAs to
+                                     steal, larger ones cost fewer atomics                       */
 } slice_config_t;
 
 typedef struct {
@@ -239,7 +241,8 @@ int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* 
 /* With SLICE_FLAG_PROFILE: after synchronising, returns for each layer of the most recent pass
  * five times in microseconds relative to the pass's first event: prefetch start, prefetch end,
  * attention start, attention end (after the merge), end of the attention kernel proper (before the
- * merge) (host, [num_layers][5] floats; NaN where not recorded). */
+ * merge) (host, [num_layers][5] floats; NaN where not recorded). A pass done in one launch records
+ * only the attention start of layer 0 and the two end times of the last layer. */
 int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers);
 
 /* With SLICE_FLAG_PROFILE: per-CTA times (GPU nanosecond timer) of the most recent launch of each

@@ -62,12 +62,14 @@ constexpr int kCopyLoadsAhead = 3;         // loads in flight; the other stages 
 constexpr uint32_t kCopyChunk = 16384;
 constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAMax / 2 + 1)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
+constexpr uint32_t kFlush = 0xFFFFFFFEu;   // descriptor without data: close the open run now
 constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRowPad = 16;
 constexpr uint32_t kStealMin = 2, kStealMax = 16;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
 constexpr uint64_t kWaitNs = 2000000000ull;
+constexpr uint32_t kOwnCache = 2048;       // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
 __host__ __device__ constexpr uint32_t row_pitch(uint32_t Hkv) { return row_bytes(Hkv) + kRowPad; }
@@ -95,6 +97,12 @@ struct Claim {
   uint32_t b, e;  // flat blocks [b, e); empty when b >= e
 };
 
+// The sequence the producer is in: batch position, its flat blocks [lo, hi), and the end of the
+// next sequence's blocks (fetched ahead).
+struct Cursor {
+  uint32_t seq, lo, hi, nhi;
+};
+
 struct Smem {
   uint32_t na;          // attention ring stages in use
   uint8_t* att_ring;
@@ -106,6 +114,7 @@ struct Smem {
   uint8_t** copy_dst;   // [kNC]
   uint32_t* copy_len;   // [kNC]
   uint32_t* mq;         // merge queue: [kMq] entries, then tail, head, consumer warps done
+  int32_t* own_res;     // [kOwnCache] resolved entries of the CTA's own range
 };
 
 // Bookkeeping area behind the two rings; every part 16-byte aligned.
@@ -114,12 +123,13 @@ constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
 constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
 constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
+constexpr size_t kOwnBytes = kOwnCache * sizeof(int32_t);
 static_assert(2 * kNAMax + kNC <= 24 && kNC <= 8, "bookkeeping area too small");
 static_assert(kNAFused * 33024 + kNC * 16384 >= kNAAlone * 33024, "the deeper ring must fit in the fused layout");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
   return static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
-         kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes;
+         kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
@@ -135,6 +145,7 @@ __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers)
   s.copy_dst = reinterpret_cast<uint8_t**>(p + kBarBytes + kQueueBytes);
   s.copy_len = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes);
   s.mq = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes);
+  s.own_res = reinterpret_cast<int32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes);
   return s;
 }
 
@@ -193,6 +204,23 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   RingPos pos;
   bool ok = true;
 
+  // What is the same in every layer of the launch: the own range, its resolved entries (copied to
+  // shared memory as far as they fit) and the sequence its first block belongs to.
+  const bool owner = blockIdx.x < p.used_cta;
+  const uint32_t r0 = owner ? blockIdx.x * p.per : 0;
+  const uint32_t r1 = owner ? min(r0 + p.per, p.total_blocks) : 0;
+  const uint32_t ncache = min(r1 - r0, kOwnCache);
+  const uint32_t own_chunk = min(p.own_chunk & 0xFFu, 32u);
+  for (uint32_t i = lane; i < ncache; i += 32) sm.own_res[i] = p.resolved[r0 + i];
+  __syncwarp();
+  Cursor first{kSentinel, 0, 0, 0};
+  if (owner) {
+    first.seq = p.blk_seq[r0];
+    first.lo = p.blk_off[first.seq];
+    first.hi = p.blk_off[first.seq + 1];
+    first.nhi = p.blk_off[min(first.seq + 2, p.nseq)];
+  }
+
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
     const uint32_t layer = p.first_layer + li;
     const uint8_t* local_layer = p.local_layer + li * p.local_layer_stride;
@@ -200,6 +228,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     unsigned long long* rw = range_words(p, li);
     uint32_t* seq_count = seq_counts(p, li);
     uint32_t cur_seq = kSentinel, nruns = 0, nclaims = 0;
+    Cursor cur = first;
     // A staged block of this layer may be read once the gather issued during the previous layer of
     // this launch has landed it (per-position ready flags carrying the layer's epoch); the first
     // layer's gather precedes the launch in stream order, as does any gather the host skipped.
@@ -218,59 +247,40 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       if (!ok) break;
     }
 
-    // Streams blocks [bb, be) of batch position seq (flat index of bb: flat) as one unit.
-    auto stream_unit = [&](uint32_t seq, uint32_t bb, uint32_t be, uint32_t flat, uint32_t slot_flag) {
-      const uint32_t nb = be - bb;
-      for (uint32_t b0 = 0; b0 < nb && ok; b0 += 32) {
-        const uint32_t cnt = min(32u, nb - b0);
-        const int32_t my = lane < cnt ? p.resolved[flat + b0 + lane] : 0;
-        // Ready flags of this batch of blocks, fetched together (a flag that is not there yet is
-        // polled below).
-        uint32_t my_ready = epoch;
-        if (check_ready && lane < cnt && my < 0) my_ready = __ldcg(ready + static_cast<uint32_t>(~my));
-        for (uint32_t j = 0; j < cnt && ok; ++j) {
-          const int32_t e = __shfl_sync(0xffffffffu, my, j);
-          if (check_ready && e < 0 && __shfl_sync(0xffffffffu, my_ready, j) != epoch) {
-            const uint64_t w0 = ptx::global_timer_ns();
-            ok = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
-            waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
-          }
-          const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
-                                      : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
-#pragma unroll
-          for (uint32_t plane = 0; plane < 2; ++plane, ++hs, pos.advance(sm.na)) {
-            const uint32_t stg = pos.stg;
-            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
-            const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
-            if (lane == 0) {
-              if (b0 + j == 0 && plane == 0) {
-                sm.queue[nq % kQueue] = UnitDesc{seq, bb, be, slot_flag, li, 0, 0, 0};
-                ++nq;
-              }
-              ptx::mbar_arrive_expect_tx(full, plane_bytes);
-            }
-            __syncwarp();
-            if (lane < kT)
-              ptx::bulk_g2s(ring + stg * hsb + lane * pitch,
-                            src + plane * plane_bytes + static_cast<uint64_t>(lane) * rb, rb, full);
-          }
-        }
+    // Moves the sequence cursor to the sequence that holds flat block `at`. Walking into the next
+    // sequence costs no load that is waited for (its end was fetched when the cursor last moved);
+    // anywhere else (a stolen claim) the sequence is looked up, `hint` being blk_seq[at] if the
+    // caller has fetched it already.
+    auto seek = [&](uint32_t at, uint32_t hint) {
+      if (at >= cur.lo && at < cur.hi) return;
+      if (at == cur.hi && cur.seq != kSentinel && cur.seq + 1 < p.nseq && at < cur.nhi) {
+        ++cur.seq;
+        cur.lo = cur.hi;
+        cur.hi = cur.nhi;
+        cur.nhi = p.blk_off[min(cur.seq + 2, p.nseq)];
+        return;
       }
+      cur.seq = hint != kSentinel ? hint : p.blk_seq[at];
+      cur.lo = p.blk_off[cur.seq];
+      cur.hi = p.blk_off[cur.seq + 1];
+      cur.nhi = p.blk_off[min(cur.seq + 2, p.nseq)];
     };
 
-    // Streams a claimed flat range, one unit per sequence it touches. A unit of another sequence
-    // than the previous one starts a new run and takes the next partial slot of its sequence.
-    auto stream_claim = [&](Claim c) {
+    // Streams a claim of at most 32 flat blocks, one unit per sequence it touches. Lane j holds the
+    // resolved entry of block c.b + j in `my` and, when have_rdy, the ready flag it read for it. A
+    // unit of another sequence than the previous one starts a new run and takes the next partial
+    // slot of its sequence.
+    auto stream_claim = [&](Claim c, int32_t my, uint32_t rdy, bool have_rdy, uint32_t hint) {
       ++nclaims;
-      uint32_t pos = c.b;
-      while (pos < c.e && ok) {
-        const uint32_t seq = p.blk_seq[pos];
-        const uint32_t seq_lo = p.blk_off[seq], seq_hi = p.blk_off[seq + 1];
-        const uint32_t ue = min(c.e, seq_hi);
+      if (!have_rdy) {
+        rdy = epoch;
+        if (check_ready && lane < c.e - c.b && my < 0) rdy = __ldcg(ready + static_cast<uint32_t>(~my));
+      }
+      uint32_t at = c.b;
+      while (at < c.e && ok) {
+        seek(at, at == c.b ? hint : kSentinel);
+        const uint32_t seq = cur.seq, seq_lo = cur.lo;
+        const uint32_t ue = min(c.e, cur.hi);
         uint32_t slot_flag = 0;
         if (seq != cur_seq) {
           // With stealing, slots are handed out in arrival order; with the static split a
@@ -292,30 +302,79 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           cur_seq = seq;
           ++nruns;
         }
-        stream_unit(seq, pos - seq_lo, ue - seq_lo, pos, slot_flag);
-        pos = ue;
+        for (uint32_t blk = at; blk < ue && ok; ++blk) {
+          const uint32_t j = blk - c.b;
+          const int32_t e = __shfl_sync(0xffffffffu, my, j);
+          if (check_ready && e < 0 && __shfl_sync(0xffffffffu, rdy, j) != epoch) {
+            const uint64_t w0 = ptx::global_timer_ns();
+            ok = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
+          }
+          const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
+                                      : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
+#pragma unroll
+          for (uint32_t plane = 0; plane < 2; ++plane, ++hs, pos.advance(sm.na)) {
+            const uint32_t stg = pos.stg;
+            ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
+            if (lane == 0) {
+              if (blk == at && plane == 0) {
+                sm.queue[nq % kQueue] = UnitDesc{seq, at - seq_lo, ue - seq_lo, slot_flag, li, 0, 0, 0};
+                ++nq;
+              }
+              ptx::mbar_arrive_expect_tx(full, plane_bytes);
+            }
+            __syncwarp();
+            if (lane < kT)
+              ptx::bulk_g2s(ring + stg * hsb + lane * pitch,
+                            src + plane * plane_bytes + static_cast<uint64_t>(lane) * rb, rb, full);
+          }
+        }
+        at = ue;
       }
     };
 
     auto range_len = [&](uint32_t c) { return min(p.per, p.total_blocks - c * p.per); };
 
-    // The owner's claims shrink as its range runs out (a quarter of what the last claim saw left),
-    // so that little claimed-but-unprocessed work is hidden from thieves near the end.
-    uint32_t own_left = 0xFFFFFFFFu;
-    auto claim_front = [&](uint32_t c) -> Claim {
-      const uint32_t want = min(p.own_chunk, max(1u, own_left / 4));
-      unsigned long long old = 0;
-      if (lane == 0) old = atomicAdd(&rw[c], static_cast<unsigned long long>(want));
-      old = __shfl_sync(0xffffffffu, old, 0);
+    // Claims from the front of the own range are split in two: the atomic is issued before the
+    // current claim is streamed and its answer is read afterwards, so its latency costs nothing.
+    // Claims shrink as the range runs out (a quarter of what the last claim saw left), so that
+    // little claimed-but-unprocessed work is hidden from thieves near the end.
+    uint32_t own_left = 0xFFFFFFFFu, pend_want = 0;
+    unsigned long long pend_old = 0;
+    auto issue_front = [&]() {
+      pend_want = min(own_chunk, max(1u, own_left / 4));
+      if (lane == 0) pend_old = atomicAdd(&rw[blockIdx.x], static_cast<unsigned long long>(pend_want));
+    };
+    auto resolve_front = [&]() -> Claim {
+      const unsigned long long old = __shfl_sync(0xffffffffu, pend_old, 0);
       const uint32_t f = static_cast<uint32_t>(old), b = static_cast<uint32_t>(old >> 32);
-      const uint32_t len = range_len(c);
+      const uint32_t len = r1 - r0;
       const uint32_t avail_end = b < len ? len - b : 0;
       if (f >= avail_end) return Claim{0, 0};
-      const uint32_t e = min(f + want, avail_end);
+      const uint32_t e = min(f + pend_want, avail_end);
       own_left = avail_end - e;
-      return Claim{c * p.per + f, c * p.per + e};
+      return Claim{r0 + f, r0 + e};
+    };
+    // Entries of n own blocks from flat block b on and, when they come from the shared-memory copy
+    // (no load to wait for), their ready flags as well.
+    auto prefetch_own = [&](uint32_t b, uint32_t n, int32_t& my, uint32_t& rdy, bool& have) {
+      have = b + n - r0 <= ncache;
+      my = 0;
+      if (lane < n) my = have ? sm.own_res[b + lane - r0] : p.resolved[b + lane];
+      rdy = epoch;
+      if (have && check_ready && lane < n && my < 0) rdy = __ldcg(ready + static_cast<uint32_t>(~my));
     };
 
+    // Before the last layer of a launch a CTA that is out of own work does better to start on the
+    // next layer than to compete for another range's last blocks: it steals only from ranges that
+    // are well behind.
+    const uint32_t thr = (p.own_chunk >> 8) & 0xFFu, steal_div = ((p.own_chunk >> 16) & 0xFFu) ? ((p.own_chunk >> 16) & 0xFFu) : 4u;
+    const uint32_t steal_floor = li + 1 < p.num_layers ? max(thr, 1u) : 1u;
     auto steal = [&]() -> Claim {
       for (int attempt = 0; attempt < 16; ++attempt) {
         uint32_t best_rem = 0, best_v = 0;
@@ -338,8 +397,8 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
             best_v = vv;
           }
         }
-        if (best_rem == 0) return Claim{0, 0};
-        const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / 4));
+        if (best_rem < steal_floor) return Claim{0, 0};
+        const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / steal_div));
         unsigned long long old = 0;
         if (lane == 0) old = atomicAdd(&rw[best_v], static_cast<unsigned long long>(amount) << 32);
         old = __shfl_sync(0xffffffffu, old, 0);
@@ -355,22 +414,56 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       return Claim{0, 0};
     };
 
-    // Own range first (claims run one ahead of the streaming, so the atomic's latency is hidden) ...
-    if (blockIdx.x < p.used_cta) {
-      Claim cur = claim_front(blockIdx.x);
-      while (cur.b < cur.e && ok) {
-        const Claim nxt = claim_front(blockIdx.x);
-        stream_claim(cur);
-        cur = nxt;
+    // Own range first. While a claim is streamed, the next claim's atomic is in flight and the
+    // entries and ready flags of the blocks it will start with (it begins where this one ends)
+    // are fetched, so a new claim does not leave the ring dry.
+    if (owner) {
+      issue_front();
+      Claim c = resolve_front();
+      int32_t my = 0;
+      uint32_t rdy = 0;
+      bool have = false;
+      if (c.b < c.e) prefetch_own(c.b, c.e - c.b, my, rdy, have);
+      while (c.b < c.e && ok) {
+        issue_front();
+        int32_t my_n = 0;
+        uint32_t rdy_n = 0;
+        bool have_n = false;
+        prefetch_own(c.e, min(pend_want, r1 - c.e), my_n, rdy_n, have_n);
+        stream_claim(c, my, rdy, have, kSentinel);
+        c = resolve_front();
+        my = my_n;
+        rdy = rdy_n;
+        have = have_n;
       }
     }
-    // ... then the back of whichever range has most left.
+    // ... then the back of whichever range has most left (the next steal, its entries and its
+    // sequence are fetched before the current one is streamed).
     if (ok && p.allow_steal) {
-      Claim cur = steal();
-      while (cur.b < cur.e && ok) {
+      Claim c = steal();
+      while (c.b < c.e && ok) {
+        const int32_t my = lane < c.e - c.b ? p.resolved[c.b + lane] : 0;
+        const uint32_t hint = p.blk_seq[c.b];
         const Claim nxt = steal();
-        stream_claim(cur);
-        cur = nxt;
+        stream_claim(c, my, 0, false, hint);
+        c = nxt;
+      }
+    }
+    // A run left open at the end of a layer would be closed only by this CTA's next unit, and a CTA
+    // may find nothing to claim in the following layers while every CTA waits for this layer's
+    // merges: close it now with a descriptor that has no data behind it.
+    if (ok && cur_seq != kSentinel && li + 1 < p.num_layers) {
+      const uint32_t stg = pos.stg;
+      ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        if (lane == 0) {
+          sm.queue[nq % kQueue] = UnitDesc{kFlush, 0, 0, 0, li, 0, 0, 0};
+          ++nq;
+          ptx::mbar_arrive(ptx::smem_u32(&sm.att_full[stg]));
+        }
+        ++hs;
+        pos.advance(sm.na);
       }
     }
     if (p.trace && lane == 0) {
@@ -659,6 +752,14 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   for (;;) {
     if (!wait_stage(p, sm, pos)) return;
     const UnitDesc it = sm.queue[nunit % kQueue];
+    if (it.seq_idx == kFlush) {
+      if (have_run) emit();
+      have_run = false;
+      ++nunit;
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      continue;
+    }
     const bool end = it.seq_idx == kSentinel;
     if (end || (it.slot & kNewRun)) {
       if (have_run) emit();
@@ -732,6 +833,14 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   for (;;) {
     if (!wait_stage(p, sm, pos)) return;
     const UnitDesc it = sm.queue[nunit % kQueue];
+    if (it.seq_idx == kFlush) {
+      if (have_run) emit();
+      have_run = false;
+      ++nunit;
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      continue;
+    }
     const bool end = it.seq_idx == kSentinel;
     if (end || (it.slot & kNewRun)) {
       if (have_run) emit();

@@ -507,7 +507,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.per = p->per;
   d.used_cta = p->used_cta;
   d.allow_steal = steal ? 1u : 0u;
-  d.own_chunk = kOwnChunk;
+  d.own_chunk = s->cfg.claim_blocks ? s->cfg.claim_blocks : kOwnChunk;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
@@ -652,10 +652,8 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
       rc = order_before_slot_write(s, sl, stream);
       if (rc) return rc;
     }
-    for (uint32_t l = 0; l < L; ++l) {
-      rc = prof_record(s, l, 2, stream);
-      if (rc) return rc;
-    }
+    rc = prof_record(s, 0, 2, stream);  // the launch spans the pass: start of layer 0 ...
+    if (rc) return rc;
     ema::LayerParams d{};
     fill_common(s, p, d, 0, L, q, out, Hq, sm_scale, s->steal);
     d.counters = s->cnt_dev;
@@ -670,12 +668,10 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     }
     CU(s, ema::launch_layer(d, stream));
     s->st.kernel_launches++;
-    for (uint32_t l = 0; l < L; ++l) {
-      rc = prof_record(s, l, 4, stream);
-      if (rc) return rc;
-      rc = prof_record(s, l, 3, stream);
-      if (rc) return rc;
-    }
+    rc = prof_record(s, L - 1, 4, stream);  // ... and end of the last layer
+    if (rc) return rc;
+    rc = prof_record(s, L - 1, 3, stream);
+    if (rc) return rc;
   }
   for (uint32_t r = 0; r < R; ++r) {
     SlotState& sl = s->slots[r];
@@ -782,7 +778,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   s->cfg.local_free_order = s->cfg.lent_free_order = nullptr;
   s->null_dev = null_dev;
   s->profile = (cfg->flags & SLICE_FLAG_PROFILE) != 0;
-  s->trace = s->profile || (cfg->flags & SLICE_FLAG_TRACE) != 0;
+  s->trace = (cfg->flags & SLICE_FLAG_TRACE) != 0;
   s->steal = cfg->static_split == 0;
   s->block_bytes = bb;
   s->local_bs = cfg->local_block_stride ? cfg->local_block_stride : bb;

@@ -258,7 +258,7 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
     fused launch per layer), odd and even layer counts on a ring of two, three passes each."""
     wl = synth.Workload("pipe", layers, 32, 8, 7, 100, 1200, 0.4)
     sc = Scenario(wl, 9)
-    g = _gpu(sc, flags=B.FLAG_PROFILE, pipeline_mode=mode, static_split=static, decode_ctas=12)
+    g = _gpu(sc, flags=B.FLAG_PROFILE | B.FLAG_TRACE, pipeline_mode=mode, static_split=static, decode_ctas=12)
     seqs = np.asarray(sc.seq_ids, np.int32)
     for rep in range(3):
         g.out.zero_()
@@ -274,7 +274,10 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
         ok, max_abs, _ = attention_close(out[layer], ref, ATOL, RTOL)
         assert ok, (layer, max_abs)
     times = g.s.slice_layer_times()
-    assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
+    if mode == 0:
+        assert np.isfinite(times[0, 2]) and times[-1, 3] >= times[0, 2]      # one launch spans the pass
+    else:
+        assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
     trace = g.s.slice_cta_trace(0)
     assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 0] > 0).all()      # every CTA visited every layer
     # the staged bytes left in the ring are the oracle's
@@ -304,25 +307,26 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
         assert torch.equal(oh, g.out.cpu())     # static split: bit-identical from run to run
 
 
-def test_llama8b_shapes_sampled_parity():
-    """Full batch and lengths of the Llama-3-8B-shaped workload on two layers, in the launch
-    configuration the benchmark times; sampled (sequence, head) outputs are recomputed by the
-    oracle's dense brute force from blocks copied back to the host."""
-    wl = synth.WORKLOADS["llama3_8b_decode"]
-    L = 2
+@pytest.mark.parametrize("name,L", [("llama3_8b_decode", 4), ("llama3_70b_decode", 3)])
+def test_full_batch_shapes_sampled_parity(name, L):
+    """Full batch and lengths of the Llama-3-8B- and 70B-shaped workloads on a few layers, in the
+    launch configuration the benchmark times (one persistent launch per pass, 148 CTAs, work
+    stealing); integer results and staged bytes are compared in full, attention on sampled
+    sequences recomputed by the oracle's dense brute force from blocks copied back to the host."""
+    wl = synth.WORKLOADS[name]
     pl = synth.make_placement(wl, 0, slack_blocks=64)
     gen = torch.Generator(device="cuda").manual_seed(0)
     shape = (2, wl.block_tokens, wl.num_kv_heads, wl.head_dim)
-    local = torch.randn((L, pl.local_blocks) + shape, device="cuda", generator=gen, dtype=torch.float32).to(torch.bfloat16)
-    lent = torch.randn((L, pl.lent_blocks) + shape, device="cuda", generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    local = torch.empty((L, pl.local_blocks) + shape, device="cuda", dtype=torch.bfloat16).normal_(generator=gen)
+    lent = torch.empty((L, pl.lent_blocks) + shape, device="cuda", dtype=torch.bfloat16).normal_(generator=gen)
     staging = torch.zeros((2, pl.staging_blocks) + shape, device="cuda", dtype=torch.bfloat16)
-    q = torch.randn((L, wl.batch, wl.num_q_heads, wl.head_dim), device="cuda", generator=gen).to(torch.bfloat16)
+    q = torch.empty((L, wl.batch, wl.num_q_heads, wl.head_dim), device="cuda", dtype=torch.bfloat16).normal_(generator=gen)
     out = torch.zeros_like(q)
     s = B.Slice(L, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks, local=local, lent=lent,
-                staging=staging, max_seqs=wl.batch, max_blocks_per_seq=256,
+                staging=staging, max_seqs=wl.batch, max_blocks_per_seq=520,
                 local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
     orc = oracle.OracleSlice(L, 16, wl.block_bytes, pl.local_blocks, pl.lent_blocks, pl.lent_blocks, 2,
-                             pl.staging_blocks, max_seqs=wl.batch, max_blocks_per_seq=256,
+                             pl.staging_blocks, max_seqs=wl.batch, max_blocks_per_seq=520,
                              local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
     for i, hints in enumerate(pl.hints):
         for h in hints:
@@ -341,15 +345,15 @@ def test_llama8b_shapes_sampled_parity():
     rc2, res_gpu, k_gpu = s.slice_get_resolved(seqs)
     assert rc == rc2 == 0 and k == k_gpu == pl.staging_blocks and (resolved == res_gpu).all()
     # staged bytes in full for the layer still resident in each slot (device-side comparison)
-    # slot 0 holds layer 0 again (cyclic prefetch for the next pass), slot 1 holds layer 1
-    for layer, slot in ((0, 0), (1, 1)):
+    # slot 0 holds layer 0 again (cyclic prefetch for the next pass), slot 1 the last odd layer
+    for layer, slot in ((0, 0), (L - 1 if (L - 1) % 2 else L - 2, 1)):
         ids = torch.tensor([~int(e) for i in range(wl.batch) for e in orc.block_table(i)[1][: synth.blocks_for(pl.lengths[i])]
                             if e < 0], device="cuda")
         assert torch.equal(staging[slot, :k], lent[layer].index_select(0, ids))
     # sampled attention parity: shortest, longest and seeded random sequences, a few heads each
     rng = np.random.default_rng(0)
     order = np.argsort(pl.lengths)
-    sample = {int(order[0]), int(order[-1])} | {int(x) for x in rng.choice(wl.batch, 6, replace=False)}
+    sample = {int(order[0]), int(order[-1])} | {int(x) for x in rng.choice(wl.batch, 4, replace=False)}
     G = wl.num_q_heads // wl.num_kv_heads
     for layer in range(L):
         for i in sorted(sample):
