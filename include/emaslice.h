@@ -100,6 +100,13 @@ typedef struct {
   uint32_t claim_blocks;          /* most KV blocks a CTA claims from its own range at a time
                                      (0 = default); smaller claims leave more for idle CTAs to
                                      steal, larger ones cost fewer atomics                       */
+  uint32_t steal_floor;           /* persistent pass (pipeline_mode 0): before the last layer an idle
+                                     CTA steals only from a range with at least this many blocks
+                                     left, and otherwise starts on the next layer. 0 = default (a
+                                     third of a range); 1 = steal down to the last block, which
+                                     keeps all CTAs in step: almost no CTA ever waits for
+                                     prefetched data, at a lower overall rate                    */
+  uint32_t reserved;
 } slice_config_t;
 
 typedef struct {

@@ -210,7 +210,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t r0 = owner ? blockIdx.x * p.per : 0;
   const uint32_t r1 = owner ? min(r0 + p.per, p.total_blocks) : 0;
   const uint32_t ncache = min(r1 - r0, kOwnCache);
-  const uint32_t own_chunk = min(p.own_chunk & 0xFFu, 32u);
+  const uint32_t own_chunk = min(p.own_chunk, 32u);
   for (uint32_t i = lane; i < ncache; i += 32) sm.own_res[i] = p.resolved[r0 + i];
   __syncwarp();
   Cursor first{kSentinel, 0, 0, 0};
@@ -373,8 +373,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     // Before the last layer of a launch a CTA that is out of own work does better to start on the
     // next layer than to compete for another range's last blocks: it steals only from ranges that
     // are well behind.
-    const uint32_t thr = (p.own_chunk >> 8) & 0xFFu, steal_div = ((p.own_chunk >> 16) & 0xFFu) ? ((p.own_chunk >> 16) & 0xFFu) : 4u;
-    const uint32_t steal_floor = li + 1 < p.num_layers ? max(thr, 1u) : 1u;
+    // Keeping all CTAs in step would cost more (every layer would end in a scramble for crumbs,
+    // with the rings running dry) than the lead it takes away.
+    const uint32_t steal_floor = li + 1 < p.num_layers ? max(p.steal_floor, 1u) : 1u;
     auto steal = [&]() -> Claim {
       for (int attempt = 0; attempt < 16; ++attempt) {
         uint32_t best_rem = 0, best_v = 0;
@@ -398,7 +399,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           }
         }
         if (best_rem < steal_floor) return Claim{0, 0};
-        const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / steal_div));
+        const uint32_t amount = min(kStealMax, max(kStealMin, best_rem / 4));
         unsigned long long old = 0;
         if (lane == 0) old = atomicAdd(&rw[best_v], static_cast<unsigned long long>(amount) << 32);
         old = __shfl_sync(0xffffffffu, old, 0);

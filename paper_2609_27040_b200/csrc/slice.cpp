@@ -21,7 +21,8 @@ constexpr uint32_t kBlockTokens = 16;
 constexpr uint32_t kHeadDim = 128;
 constexpr uint32_t kTraceCopyCtas = 2048;
 constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must match the kernel)
-constexpr uint32_t kOwnChunk = 8;  // most blocks a CTA claims from its own range at a time
+constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a range, at least this
+constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
   std::vector<int32_t> table;
@@ -507,7 +508,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.per = p->per;
   d.used_cta = p->used_cta;
   d.allow_steal = steal ? 1u : 0u;
-  d.own_chunk = s->cfg.claim_blocks ? s->cfg.claim_blocks : kOwnChunk;
+  d.own_chunk = s->cfg.claim_blocks ? std::min(s->cfg.claim_blocks, 32u) : kOwnChunk;
+  d.steal_floor = s->cfg.steal_floor ? s->cfg.steal_floor : std::max(kStealFloorMin, p->per / 3);
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;

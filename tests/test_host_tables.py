@@ -40,7 +40,7 @@ def test_library_exports_every_declared_entry_point():
 
 def test_config_struct_matches_header_size():
     # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 6 uint32
-    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 6 * 4
+    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 8 * 4
 
 
 def test_create_rejects_bad_configs():
