@@ -25,6 +25,13 @@
  * Data layout
  *   block      = K plane [block_tokens][num_kv_heads][head_dim] bf16, then the V plane of the
  *                same shape: 2*16*8*128*2 = 65 536 bytes for the shapes used here.
+ *                Storage order inside a token row: within every aligned 128 bytes of row r, the
+ *                16-byte unit u (8 bf16) is stored at unit u ^ (r & 7). The permutation is its own
+ *                inverse; slice_append_kv writes it, paged_decode reads it, and the copy paths
+ *                (prefetch, write-back, reclaim) move whole blocks and never look inside. It lets a
+ *                plane go from HBM to shared memory as ONE linear bulk copy and still be read by
+ *                ldmatrix without bank conflicts. A caller that fills blocks itself applies the
+ *                same permutation (the Python binding has kv_block_swizzle for it).
  *   arena      = [layer][block id][block]; byte address = base + layer*layer_stride
  *                + id*block_stride (strides 0 select the dense default).
  *   staging    = [ring slot][position][block], dense.

@@ -132,6 +132,22 @@ def _seqs(seqs) -> np.ndarray:
     return np.ascontiguousarray(seqs, np.int32)
 
 
+def kv_block_swizzle(x):
+    """Converts KV rows between canonical order and the block format's storage order (and back: the
+    permutation is its own inverse). `x` is a numpy array or torch tensor of 16-bit elements whose
+    last three dimensions are [16 token rows][num_kv_heads][128]; within every 128 bytes of token
+    row r, the 16-byte unit u moves to unit u ^ (r & 7). Returns a new array."""
+    shape = tuple(x.shape)
+    if len(shape) < 3 or shape[-3] != 16 or shape[-1] != 128:
+        raise ValueError(f"expected [..., 16, num_kv_heads, 128], got {shape}")
+    v = x.reshape(shape[:-3] + (16, shape[-2] * 2, 8, 8))
+    out = v.copy() if isinstance(v, np.ndarray) else v.clone()
+    for k in range(1, 8):
+        perm = [u ^ k for u in range(8)]
+        out[..., k::8, :, :, :] = v[..., k::8, :, perm, :]
+    return out.reshape(shape)
+
+
 class Slice:
     """Owner of one ``slice_t`` handle. Methods are named after the C entry points and return the
     status code (plus outputs); ``check=True`` turns a non-zero status into SliceError."""

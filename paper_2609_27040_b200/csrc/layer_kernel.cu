@@ -64,7 +64,7 @@ constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAM
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kFlush = 0xFFFFFFFEu;   // descriptor without data: close the open run now
 constexpr uint32_t kNewRun = 0x80000000u;
-constexpr uint32_t kRowPad = 16;
+constexpr uint32_t kRingAlign = 128;
 constexpr uint32_t kStealMin = 2, kStealMax = 16;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
@@ -72,8 +72,7 @@ constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kOwnCache = 2048;       // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
-__host__ __device__ constexpr uint32_t row_pitch(uint32_t Hkv) { return row_bytes(Hkv) + kRowPad; }
-__host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_pitch(Hkv); }
+__host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_bytes(Hkv); }
 
 // A unit: blocks [blk_begin, blk_end) of batch position seq_idx in layer `layer`. slot carries the
 // run's partial slot and the kNewRun flag when the unit starts a new run.
@@ -125,16 +124,17 @@ constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
 constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
 constexpr size_t kOwnBytes = kOwnCache * sizeof(int32_t);
 static_assert(2 * kNAMax + kNC <= 24 && kNC <= 8, "bookkeeping area too small");
-static_assert(kNAFused * 33024 + kNC * 16384 >= kNAAlone * 33024, "the deeper ring must fit in the fused layout");
+static_assert(kNAFused * 32768 + kNC * 16384 >= kNAAlone * 32768, "the deeper ring must fit in the fused layout");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
-  return static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
+  return kRingAlign + static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
   Smem s;
   s.na = gathers ? kNAFused : kNAAlone;
+  base += (kRingAlign - (ptx::smem_u32(base) & (kRingAlign - 1))) & (kRingAlign - 1);
   s.att_ring = base;
   s.copy_ring = base + static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv);
   uint8_t* p = s.copy_ring + static_cast<size_t>(kNC) * kCopyChunk;
@@ -197,8 +197,8 @@ __device__ __forceinline__ bool wait_counter(const uint32_t* cnt, uint32_t targe
 __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv;
-  const uint32_t rb = row_bytes(Hkv), pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
-  const uint32_t plane_bytes = kT * rb;
+  const uint32_t hsb = half_stage_bytes(Hkv);
+  const uint32_t plane_bytes = hsb;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   uint32_t hs = 0, nq = 0;
   RingPos pos;
@@ -326,12 +326,16 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
                 sm.queue[nq % kQueue] = UnitDesc{seq, at - seq_lo, ue - seq_lo, slot_flag, li, 0, 0, 0};
                 ++nq;
               }
+              // The stage was last read through the generic proxy (ldmatrix / ld.shared of the
+              // consumer warps, ordered before this point by the empty barrier); the bulk copy writes
+              // it through the asynchronous proxy. Without this fence the copy can overtake those
+              // reads: seen as rare wrong V tiles in launches spanning several layers.
+              ptx::fence_proxy_async();
               ptx::mbar_arrive_expect_tx(full, plane_bytes);
+              // One request per plane: an SM streams far faster through few large bulk copies than
+              // through many small ones.
+              ptx::bulk_g2s(ring + stg * hsb, src + plane * plane_bytes, plane_bytes, full);
             }
-            __syncwarp();
-            if (lane < kT)
-              ptx::bulk_g2s(ring + stg * hsb + lane * pitch,
-                            src + plane * plane_bytes + static_cast<uint64_t>(lane) * rb, rb, full);
           }
         }
         at = ue;
@@ -708,7 +712,7 @@ __device__ __forceinline__ void release_stage(const Smem& sm, const RingPos& pos
 __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv, G = p.G;
-  const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
+  const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   const uint32_t n = lane >> 2, tig = lane & 3u, r0 = lane >> 2;
@@ -791,11 +795,11 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       const uint32_t valid = min(kT, len - b * kT);
       uint32_t pb0, pb1;
       float al0, al1;
-      tile_mma_scores(ring + pos.stg * hsb, pitch, head_off, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
+      tile_mma_scores(ring + pos.stg * hsb + head_off, rb, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
       release_stage(sm, pos);
       pos.advance(sm.na);
       if (!wait_stage(p, sm, pos)) return;
-      tile_mma_pv(ring + pos.stg * hsb, pitch, head_off, valid, pb0, pb1, al0, al1, o);
+      tile_mma_pv(ring + pos.stg * hsb + head_off, rb, valid, pb0, pb1, al0, al1, o);
       release_stage(sm, pos);
       pos.advance(sm.na);
     }
@@ -809,7 +813,7 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
 __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv;
-  const uint32_t pitch = row_pitch(Hkv), hsb = half_stage_bytes(Hkv);
+  const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
   const uint32_t head_off = g * kD * 2;
   const uint32_t half = lane & 1u;
   uint32_t nunit = 0;
@@ -874,11 +878,11 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       if (b != it.blk_begin && !wait_stage(p, sm, pos)) return;
       const uint32_t valid = min(kT, len - b * kT);
       float pw, al;
-      tile_alu_scores(sm.att_ring + pos.stg * hsb, pitch, head_off, valid, qh, p.scale_log2, st, pw, al);
+      tile_alu_scores(sm.att_ring + pos.stg * hsb + head_off, rb, valid, qh, p.scale_log2, st, pw, al);
       release_stage(sm, pos);
       pos.advance(sm.na);
       if (!wait_stage(p, sm, pos)) return;
-      tile_alu_pv(sm.att_ring + pos.stg * hsb, pitch, head_off, valid, pw, al, o);
+      tile_alu_pv(sm.att_ring + pos.stg * hsb + head_off, rb, valid, pw, al, o);
       release_stage(sm, pos);
       pos.advance(sm.na);
     }
@@ -1042,11 +1046,12 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   const uint4* vs = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(p.v_new) + static_cast<uint64_t>(i) * p.row_bytes);
   for (uint32_t v = threadIdx.x; v < vecs; v += blockDim.x) {
     const uint4 kv = ks[v], vv = vs[v];
-    reinterpret_cast<uint4*>(home + r * p.row_bytes)[v] = kv;
-    reinterpret_cast<uint4*>(home + plane + r * p.row_bytes)[v] = vv;
+    const uint32_t w = (v & ~7u) | ((v & 7u) ^ (r & 7u));  // the block format's swizzle of 16-byte units
+    reinterpret_cast<uint4*>(home + r * p.row_bytes)[w] = kv;
+    reinterpret_cast<uint4*>(home + plane + r * p.row_bytes)[w] = vv;
     if (staged) {
-      reinterpret_cast<uint4*>(staged + r * p.row_bytes)[v] = kv;
-      reinterpret_cast<uint4*>(staged + plane + r * p.row_bytes)[v] = vv;
+      reinterpret_cast<uint4*>(staged + r * p.row_bytes)[w] = kv;
+      reinterpret_cast<uint4*>(staged + plane + r * p.row_bytes)[w] = vv;
     }
   }
 }

@@ -508,7 +508,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.per = p->per;
   d.used_cta = p->used_cta;
   d.allow_steal = steal ? 1u : 0u;
-  d.own_chunk = s->cfg.claim_blocks ? std::min(s->cfg.claim_blocks, 32u) : kOwnChunk;
+  d.own_chunk = s->cfg.claim_blocks ? s->cfg.claim_blocks : kOwnChunk;
   d.steal_floor = s->cfg.steal_floor ? s->cfg.steal_floor : std::max(kStealFloorMin, p->per / 3);
   d.q = q;
   d.out = out;

@@ -18,12 +18,23 @@ def to_host(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy().view(np.uint16)
 
 
+def kv_to_dev(a: np.ndarray) -> torch.Tensor:
+    """KV blocks [..., 2, 16, Hkv, 128] in canonical order (as the oracle reads them) -> device tensor
+    in the library's block format."""
+    return to_dev(B.kv_block_swizzle(a))
+
+
+def kv_to_host(t: torch.Tensor) -> np.ndarray:
+    """Device KV blocks in the library's block format -> canonical order on the host."""
+    return B.kv_block_swizzle(to_host(t))
+
+
 class GpuScenario:
     def __init__(self, sc: Scenario, **kw):
         self.sc = sc
-        self.local = to_dev(sc.local)
-        self.lent = to_dev(sc.lent)
-        self.staging = to_dev(sc.staging)
+        self.local = kv_to_dev(sc.local)
+        self.lent = kv_to_dev(sc.lent)
+        self.staging = kv_to_dev(sc.staging)
         self.q = to_dev(sc.q)
         self.out = torch.zeros_like(self.q)
         self.lse = torch.zeros((sc.L, sc.nseq, sc.Hq), dtype=torch.float32, device="cuda")

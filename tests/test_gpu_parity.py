@@ -54,8 +54,8 @@ def _check_layer(sc, g, layer, seqs=None, check_bytes=True):
     assert (res_gpu == resolved).all()
     slot = layer % sc.wl.ring_slots
     if check_bytes and k:
-        from tests.gpu_helpers import to_host
-        got = to_host(g.staging[slot, :k])
+        from tests.gpu_helpers import kv_to_host, to_host
+        got = kv_to_host(g.staging[slot, :k])
         assert (got == sc.staging[slot, :k]).all()          # bit-exact gather
     lens = np.asarray([int(sc.pl.lengths[i]) for i in seqs], np.uint32)
     rc, ref, ref_lse = oracle.paged_attention(sc.q[layer][pos], sc.local[layer], sc.staging[slot], resolved, lens,
@@ -122,7 +122,7 @@ def test_single_token_output_is_the_value_row_exactly():
         assert g.s.prefetch_layer(0, sc.seq_ids, g.side) == B.OK
         assert g.s.paged_decode(0, sc.seq_ids, g.q[0], sc.Hq, float(sc.sm_scale), g.out[0], None, g.main) == B.OK
         torch.cuda.synchronize()
-        from tests.gpu_helpers import to_host
+        from tests.gpu_helpers import kv_to_host, to_host
         out = to_host(g.out[0])
         G = sc.Hq // sc.Hkv
         for pos, i in enumerate(sc.seq_ids):
@@ -134,7 +134,7 @@ def test_single_token_output_is_the_value_row_exactly():
 def test_reclaim_migration_is_bit_exact_and_attention_survives():
     sc = Scenario(GQA4, 7, slack=96, lent_extra_physical=3)
     g = _gpu(sc)
-    from tests.gpu_helpers import to_host
+    from tests.gpu_helpers import kv_to_host, to_host
     first = {}
     for layer in range(sc.L):
         _check_layer(sc, g, layer)
@@ -145,7 +145,7 @@ def test_reclaim_migration_is_bit_exact_and_attention_survives():
     assert rc == rc2 == 0 and mig == mig2 and mig > 0
     torch.cuda.synchronize()
     g.tables_equal_oracle()
-    local_gpu, lent_gpu = to_host(g.local), to_host(g.lent)
+    local_gpu, lent_gpu = kv_to_host(g.local), kv_to_host(g.lent)
     for i in sc.seq_ids:
         _, tab, _ = sc.orc.block_table(i)
         for l in range(sc.L):
@@ -163,7 +163,7 @@ def test_reclaim_migration_is_bit_exact_and_attention_survives():
     assert rc == rc2 == 0 and mig == mig2
     torch.cuda.synchronize()
     g.tables_equal_oracle()
-    assert (to_host(g.local) == sc.local).all()
+    assert (kv_to_host(g.local) == sc.local).all()
     assert g.s.slice_stats()["lent_capacity"] == 0
     for layer in range(sc.L):
         max_abs, _ = _check_layer(sc, g, layer)
@@ -183,7 +183,7 @@ def test_append_kv_writes_home_and_staged_copy():
     wl = synth.Workload("app", 2, 32, 8, 4, 17, 90, 0.5)
     sc = Scenario(wl, 5, slack=8)
     g = _gpu(sc)
-    from tests.gpu_helpers import to_dev, to_host
+    from tests.gpu_helpers import kv_to_host, to_dev, to_host
     rng = np.random.default_rng(12)
     for step in range(3):
         for i in sc.seq_ids:
@@ -206,15 +206,15 @@ def test_append_kv_writes_home_and_staged_copy():
             assert g.s.slice_append_kv(layer, sc.seq_ids, kd, vd, g.main) == B.OK
             torch.cuda.synchronize()
             k = g.s.slice_get_resolved(sc.seq_ids)[2]
-            assert (to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
+            assert (kv_to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
             _check_layer(sc, g, layer)       # re-prefetches (already staged plan) and attends
-        assert (to_host(g.local) == sc.local).all() and (to_host(g.lent) == sc.lent).all()
+        assert (kv_to_host(g.local) == sc.local).all() and (kv_to_host(g.lent) == sc.lent).all()
 
 
 def test_writeback_round_trip():
     sc = Scenario(GQA4, 8)
     g = _gpu(sc)
-    from tests.gpu_helpers import to_host
+    from tests.gpu_helpers import kv_to_host, to_host
     keep = sc.lent.copy()
     for layer in range(sc.L):
         assert g.s.prefetch_layer(layer, sc.seq_ids, g.side) == B.OK
@@ -228,7 +228,7 @@ def test_writeback_round_trip():
                     g.lent[layer, ~e].zero_()
         assert g.s.slice_writeback_layer(layer, sc.seq_ids, g.main) == B.OK
         torch.cuda.synchronize()
-    assert (to_host(g.lent) == keep).all()
+    assert (kv_to_host(g.lent) == keep).all()
     assert g.s.slice_writeback_layer(0, sc.seq_ids[:2], g.main) == B.ESTALE
 
 
@@ -281,7 +281,7 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
     trace = g.s.slice_cta_trace(0)
     assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 0] > 0).all()      # every CTA visited every layer
     # the staged bytes left in the ring are the oracle's
-    from tests.gpu_helpers import to_host
+    from tests.gpu_helpers import kv_to_host, to_host
     for slot in range(wl.ring_slots):
         layer = [l for l in range(sc.L) if l % wl.ring_slots == slot][-1]
         if slot == 0 and (sc.L - 1) % wl.ring_slots != 0:
@@ -289,7 +289,7 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
         if slot == 0 and (sc.L - 1) % wl.ring_slots == 0:
             layer = 0          # shared slot: refilled after the last attention
         rc, _, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
-        assert (to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
+        assert (kv_to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
     # host buffers: the same call with pinned host q/out
     qh = g.q.cpu().pin_memory()
     oh = torch.zeros_like(qh).pin_memory()
@@ -360,6 +360,7 @@ def test_full_batch_shapes_sampled_parity(name, L):
             n = int(pl.lengths[i])
             tab = orc.block_table(i)[1][: synth.blocks_for(n)]
             blocks = torch.stack([local[layer, e] if e >= 0 else lent[layer, ~e] for e in tab.tolist()])
+            blocks = B.kv_block_swizzle(blocks)          # block format -> canonical token rows
             K = blocks[:, 0].reshape(-1, wl.num_kv_heads, wl.head_dim)[:n].contiguous()
             V = blocks[:, 1].reshape(-1, wl.num_kv_heads, wl.head_dim)[:n].contiguous()
             Kh = K.view(torch.int16).cpu().numpy().view(np.uint16)
