@@ -110,7 +110,8 @@ typedef struct {
   uint32_t steal_floor;           /* persistent pass (pipeline_mode 0): before the last layer an idle
                                      CTA steals only from a range with at least this many blocks
                                      left, and otherwise starts on the next layer. 0 = default (a
-                                     third of a range); 1 = steal down to the last block, which
+                                     third of a range; 8 blocks in the last layer of a launch and
+                                     in single-layer launches); 1 = steal down to the last block, which
                                      keeps all CTAs in step: almost no CTA ever waits for
                                      prefetched data, at a lower overall rate                    */
   uint32_t reserved;

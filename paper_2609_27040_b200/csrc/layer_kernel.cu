@@ -378,10 +378,12 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
 
     // Before the last layer of a launch a CTA that is out of own work does better to start on the
     // next layer than to compete for another range's last blocks: it steals only from ranges that
-    // are well behind.
+    // are well behind. In the last layer the floor is lower but not 1: stealing the last few blocks
+    // of a range costs more (latency of the claim, one more partial and a longer merge at the very
+    // end of the launch) than the slower SM needs to finish them.
     // Keeping all CTAs in step would cost more (every layer would end in a scramble for crumbs,
     // with the rings running dry) than the lead it takes away.
-    const uint32_t steal_floor = li + 1 < p.num_layers ? max(p.steal_floor, 1u) : 1u;
+    const uint32_t steal_floor = max(li + 1 < p.num_layers ? p.steal_floor : p.steal_floor_last, 1u);
     auto steal = [&]() -> Claim {
       for (int attempt = 0; attempt < 16; ++attempt) {
         uint32_t best_rem = 0, best_v = 0;

@@ -22,6 +22,7 @@ constexpr uint32_t kHeadDim = 128;
 constexpr uint32_t kTraceCopyCtas = 2048;
 constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must match the kernel)
 constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a range, at least this
+constexpr uint32_t kStealFloorLast = 8; // default steal floor in the last layer of a launch
 constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
@@ -510,6 +511,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.allow_steal = steal ? 1u : 0u;
   d.own_chunk = s->cfg.claim_blocks ? s->cfg.claim_blocks : kOwnChunk;
   d.steal_floor = s->cfg.steal_floor ? s->cfg.steal_floor : std::max(kStealFloorMin, p->per / 3);
+  d.steal_floor_last = s->cfg.steal_floor ? std::min(s->cfg.steal_floor, kStealFloorLast) : kStealFloorLast;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
