@@ -168,3 +168,22 @@ def test_decode_step_with_a_shared_ring_slot_for_first_and_last_layer():
     st = s.slice_stats()
     assert st["decode_calls"] == 15 and st["prefetch_calls"] == 16
     s.close()
+
+
+def test_kv_block_swizzle_is_the_documented_self_inverse_permutation():
+    """Block format of include/emaslice.h: within every 128 bytes of token row r, 16-byte unit u is
+    stored at unit u ^ (r & 7); applying it twice gives the rows back."""
+    rng = np.random.default_rng(3)
+    x = rng.integers(0, 65536, size=(3, 2, 16, 4, 128), dtype=np.uint16)
+    y = B.kv_block_swizzle(x)
+    assert y.shape == x.shape and (B.kv_block_swizzle(y) == x).all()
+    rows_x = x.reshape(3, 2, 16, -1)       # 4 heads * 128 bf16 = 1024 B per row = 8 windows of 128 B
+    rows_y = y.reshape(3, 2, 16, -1)
+    for r in range(16):
+        for w in range(8):
+            for u in range(8):
+                src = rows_x[..., r, w * 64 + u * 8: w * 64 + u * 8 + 8]
+                dst = rows_y[..., r, w * 64 + (u ^ (r & 7)) * 8: w * 64 + (u ^ (r & 7)) * 8 + 8]
+                assert (src == dst).all()
+    with pytest.raises(ValueError):
+        B.kv_block_swizzle(np.zeros((15, 4, 128), np.uint16))
