@@ -239,9 +239,14 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
  * whole pass (mode 0) or one per layer (mode 2); with pipeline_mode 1 the gather kernel runs on
  * side_stream and the attention kernel on stream, ordered by events.
  *   q, out: [num_layers][nseq][num_q_heads][128] bf16; device pointers when io_on_host == 0.
- *   With io_on_host != 0 they are host pointers (pinned for asynchronous copies): q is copied to the
- *   device and out back to the host on `stream`, inside the call's enqueued work, through device
- *   buffers the library allocates on first use. */
+ *   With io_on_host != 0 they are host pointers. Pageable memory: q is copied to the device and out
+ *   back to the host on `stream`, inside the call's enqueued work, through device buffers the
+ *   library allocates on first use. Pinned memory: the kernels write out straight into it (every
+ *   finished row goes to the host while the pass goes on; complete when the work enqueued on
+ *   `stream` is), and when one launch covers the pass q is brought in behind the running kernel on
+ *   a copy stream of the library's own, a few layers per copy, each copy followed by an arrival
+ *   flag that the kernel checks (bounded wait, SLICE_ETIMEOUT through slice_stats) before it reads
+ *   that layer's rows. The caller must not change q before the work enqueued on `stream` is done. */
 int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t num_q_heads,
                       float sm_scale, void* out, int32_t io_on_host, int32_t wrap_prefetch,
                       void* stream, void* side_stream);

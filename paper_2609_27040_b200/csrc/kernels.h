@@ -76,6 +76,9 @@ struct LayerParams {
   const void* q;                // first_layer's [nseq][Hq][128] bf16
   void* out;
   uint64_t io_layer_stride;     // bytes from one layer's q / out to the next
+  const uint32_t* q_ready;      // optional: q arrives while the launch runs; layer l's rows may be read once
+  uint32_t q_ready_epoch;       //   q_ready[l / q_ready_layers] == q_ready_epoch (written by the copy that brought them)
+  uint32_t q_ready_layers;
   float* lse;                   // [nseq][Hq] or NULL (single-layer launches only)
   float* part_o;                // [slots][Hq][128] unnormalised partial outputs; layers alternate
   float* part_ml;               // [slots][Hq][4]   between two such buffers (stride below)

@@ -723,7 +723,7 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
   uint32_t nunit = 0;
   RingPos pos;
   bool have_run = false;
-  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0, q_upto = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
   uint32_t qf[8][2];
   float o[8][4];
@@ -780,6 +780,10 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+      if (run_li >= q_upto) {  // q may still be on its way from the host: wait for this layer's chunk
+        if (p.q_ready && !wait_counter_eq(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+      }
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
       const __nv_bfloat16* qg =
           reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
@@ -787,8 +791,8 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
           reinterpret_cast<const uint32_t*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g * G + (n < G ? n : 0)) * kD);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
-        qf[ks][0] = n < G ? qrow[ks * 8 + tig] : 0u;
-        qf[ks][1] = n < G ? qrow[ks * 8 + tig + 4] : 0u;
+        qf[ks][0] = n < G ? __ldcg(qrow + ks * 8 + tig) : 0u;
+        qf[ks][1] = n < G ? __ldcg(qrow + ks * 8 + tig + 4) : 0u;
       }
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
@@ -823,7 +827,7 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   uint32_t nunit = 0;
   RingPos pos;
   bool have_run = false;
-  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0, q_upto = 0;
   SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
   float qh[64];  // this lane's half (64 dims) of q as f32
   float o[4] = {0.f, 0.f, 0.f, 0.f};
@@ -861,13 +865,17 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+      if (run_li >= q_upto) {
+        if (p.q_ready && !wait_counter_eq(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+      }
       const __nv_bfloat16* qg =
           reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
       const uint4* qrow =
           reinterpret_cast<const uint4*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g) * kD + half * 64);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
-        const uint4 v = qrow[c];
+        const uint4 v = __ldcg(qrow + c);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {

@@ -123,6 +123,16 @@ struct ema_slice {
   void* io_q = nullptr;
   void* io_out = nullptr;
   size_t io_bytes = 0;
+  // q streamed in behind a running pass: copy stream, per-chunk arrival flags, their epoch (pinned
+  // host word the flag copies read), and the event after which io_q may be overwritten.
+  cudaStream_t io_stream = nullptr;
+  uint32_t* q_flags_dev = nullptr;
+  uint32_t* q_epoch_host = nullptr;
+  uint32_t q_epoch = 0;
+  cudaEvent_t io_q_free = nullptr;
+  bool io_q_busy = false;
+  const uint32_t* step_q_ready = nullptr;  // set for the pass being enqueued
+  uint32_t step_q_layers = 0;
   // profiling
   std::vector<cudaEvent_t> prof;  // [layer][5]
   std::vector<uint8_t> prof_set;
@@ -661,6 +671,9 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     ema::LayerParams d{};
     fill_common(s, p, d, 0, L, q, out, Hq, sm_scale, s->steal);
     d.counters = s->cnt_dev;
+    d.q_ready = s->step_q_ready;
+    d.q_ready_epoch = s->q_epoch;
+    d.q_ready_layers = s->step_q_layers ? s->step_q_layers : 1;
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / 2;
@@ -732,6 +745,10 @@ void destroy_impl(ema_slice* s) {
     if (s->ev_tmp) cudaEventDestroy(s->ev_tmp);
     if (s->io_q) cudaFree(s->io_q);
     if (s->io_out) cudaFree(s->io_out);
+    if (s->q_flags_dev) cudaFree(s->q_flags_dev);
+    if (s->q_epoch_host) cudaFreeHost(s->q_epoch_host);
+    if (s->io_q_free) cudaEventDestroy(s->io_q_free);
+    if (s->io_stream) cudaStreamDestroy(s->io_stream);
   } else {
     for (Plan& p : s->plans) delete[] p.host;
   }
@@ -1186,6 +1203,8 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
   const uint8_t* qd = static_cast<const uint8_t*>(q);
   uint8_t* od = static_cast<uint8_t*>(out);
+  bool out_mapped = false;
+  s->step_q_ready = nullptr;
   if (!s->null_dev) {
     rc = ensure_stream(s, stream);
     if (rc) return rc;
@@ -1208,9 +1227,51 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       CU(s, cudaMalloc(&s->io_out, need));
       s->io_bytes = need;
     }
-    CU(s, cudaMemcpyAsync(s->io_q, q, need, cudaMemcpyHostToDevice, stream));
     qd = static_cast<const uint8_t*>(s->io_q);
     od = static_cast<uint8_t*>(s->io_out);
+    cudaPointerAttributes aq{};
+    const bool q_pinned = cudaPointerGetAttributes(&aq, q) == cudaSuccess && aq.type == cudaMemoryTypeHost;
+    if (!q_pinned) cudaGetLastError();
+    if (step && q_pinned) {
+      // One launch covers the pass: bring q in behind it, a few layers per copy on a stream of its
+      // own, each copy followed by a 4-byte copy that sets the chunk's arrival flag; the kernel
+      // reads a layer's rows only after its flag shows this pass's epoch (bounded wait).
+      if (!s->io_stream) {
+        CU(s, cudaStreamCreateWithFlags(&s->io_stream, cudaStreamNonBlocking));
+        CU(s, cudaMalloc(reinterpret_cast<void**>(&s->q_flags_dev), ema::kMaxStepLayers * sizeof(uint32_t)));
+        CU(s, cudaMemset(s->q_flags_dev, 0, ema::kMaxStepLayers * sizeof(uint32_t)));
+        CU(s, cudaMallocHost(reinterpret_cast<void**>(&s->q_epoch_host), 64 * sizeof(uint32_t)));
+        CU(s, cudaEventCreateWithFlags(&s->io_q_free, cudaEventDisableTiming));
+      }
+      if (s->io_q_busy) CU(s, cudaStreamWaitEvent(s->io_stream, s->io_q_free, 0));
+      // everything enqueued on `stream` so far (earlier passes, the reallocation above) comes first
+      CU(s, cudaEventRecord(s->ev_tmp, stream));
+      CU(s, cudaStreamWaitEvent(s->io_stream, s->ev_tmp, 0));
+      const uint32_t per_flag = 4;
+      ++s->q_epoch;
+      uint32_t* epoch_word = s->q_epoch_host + (s->q_epoch % 64);  // a slot of its own while copies of it are in flight
+      *epoch_word = s->q_epoch;
+      for (uint32_t l0 = 0; l0 < L; l0 += per_flag) {
+        const size_t bytes = per_layer * std::min(per_flag, L - l0);
+        CU(s, cudaMemcpyAsync(static_cast<uint8_t*>(s->io_q) + l0 * per_layer, static_cast<const uint8_t*>(q) + l0 * per_layer, bytes,
+                              cudaMemcpyHostToDevice, s->io_stream));
+        CU(s, cudaMemcpyAsync(s->q_flags_dev + l0 / per_flag, epoch_word, sizeof(uint32_t), cudaMemcpyHostToDevice, s->io_stream));
+      }
+      s->step_q_ready = s->q_flags_dev;
+      s->step_q_layers = per_flag;
+    } else {
+      CU(s, cudaMemcpyAsync(s->io_q, q, need, cudaMemcpyHostToDevice, stream));
+    }
+    // Pinned (mapped) host memory can be written by the kernels themselves: the merges then store
+    // each finished row straight to the host while the pass goes on, and no copy follows the pass.
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, out) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+) {
+      od = static_cast<uint8_t*>(attr.devicePointer);
+      out_mapped = true;
+    } else {
+      cudaGetLastError();  // a pageable pointer is not an error here
+    }
   }
   if (!s->null_dev)  // the work counters of all layers, cleared once per pass
     CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * s->cnt_stride * sizeof(uint32_t), stream));
@@ -1249,7 +1310,14 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
   }
-  if (io_on_host && !s->null_dev)
+  if (s->step_q_ready) {
+    // io_q may be overwritten once this pass is done; a later non-streamed use of io_q on `stream`
+    // is ordered by the stream itself.
+    CU(s, cudaEventRecord(s->io_q_free, stream));
+    s->io_q_busy = true;
+    s->step_q_ready = nullptr;
+  }
+  if (io_on_host && !s->null_dev && !out_mapped)
     CU(s, cudaMemcpyAsync(out, s->io_out, per_layer * L, cudaMemcpyDeviceToHost, stream));
   return SLICE_OK;
 }

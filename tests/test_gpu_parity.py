@@ -305,6 +305,22 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
         assert attention_close(outh[layer], ref, ATOL, RTOL)[0]
     if static:
         assert torch.equal(oh, g.out.cpu())     # static split: bit-identical from run to run
+    # two passes back to back without a synchronisation in between (the second pass's q copies must
+    # not overtake the first pass's reads), then pageable host memory (plain copies on the stream)
+    oh.zero_()
+    for _ in range(2):
+        assert g.s.slice_decode_step(seqs, qh, sc.Hq, float(sc.sm_scale), oh, True, True, g.main, g.side) == B.OK
+    qp, op = g.q.cpu(), torch.zeros_like(g.q).cpu()
+    assert g.s.slice_decode_step(seqs, qp, sc.Hq, float(sc.sm_scale), op, True, True, g.main, g.side) == B.OK
+    torch.cuda.synchronize()
+    g.device_ok()
+    for o2 in (oh, op):
+        o2 = o2.view(torch.bfloat16).double().numpy()
+        for layer in range(sc.L):
+            rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+            _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % wl.ring_slots], resolved,
+                                               sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert attention_close(o2[layer], ref, ATOL, RTOL)[0]
 
 
 @pytest.mark.parametrize("name,L", [("llama3_8b_decode", 4), ("llama3_70b_decode", 3)])
