@@ -1265,8 +1265,7 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
     // Pinned (mapped) host memory can be written by the kernels themselves: the merges then store
     // each finished row straight to the host while the pass goes on, and no copy follows the pass.
     cudaPointerAttributes attr{};
-    if (cudaPointerGetAttributes(&attr, out) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
-) {
+    if (cudaPointerGetAttributes(&attr, out) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer) {
       od = static_cast<uint8_t*>(attr.devicePointer);
       out_mapped = true;
     } else {
