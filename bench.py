@@ -270,6 +270,25 @@ def run_reference(args, wl):
 
 
 # ---------------------------------------------------------------------------------------------
+def reduce_over_ranks(t: float, t_e2e_step: float, launches: int, world: int, device: str):
+    """Replicas only: the job's time is the slowest rank's (max over ranks, for the device-resident
+    and the end-to-end figure alike), its launch count the sum. No other exchange between ranks."""
+    if world <= 1:
+        return t, t_e2e_step, launches
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor([t, t_e2e_step], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ll = torch.tensor([launches], device=device, dtype=torch.int64)
+    dist.all_reduce(ll)
+    return float(tt[0]), float(tt[1]), int(ll[0])
+
+
+def job_value(batch: int, world: int, steps: int, t: float) -> float:
+    """Whole-job tokens/s: every replica decodes `batch` tokens per step; t is the max over ranks."""
+    return batch * world * steps / t
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -324,15 +343,7 @@ def run_ours(args, wl):
     barrier()
     io_bytes = qh.numel() * qh.element_size()
 
-    if world > 1:
-        tt = torch.tensor([t, t_e2e / e2e_steps], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t, t_e2e_step = float(tt[0]), float(tt[1])
-        ll = torch.tensor([launches], device="cuda", dtype=torch.int64)
-        dist.all_reduce(ll)
-        launches = int(ll[0])
-    else:
-        t_e2e_step = t_e2e / e2e_steps
+    t, t_e2e_step, launches = reduce_over_ranks(t, t_e2e / e2e_steps, launches, world, "cuda")
 
     # ---- the dominant kernel inside the pipelined pass (profile events + per-CTA trace), rank 0 ----
     roof = None
@@ -499,7 +510,7 @@ def run_ours(args, wl):
                "sample": f"oracle gather + fp64 paged attention of 1 layer over the first {nseq} of {wl.batch} sequences "
                          f"({sample_tokens} of {tokens} tokens, best of 3), scaled by tokens and by {wl.num_layers} layers"}
 
-    value = wl.batch * world * args.steps / t
+    value = job_value(wl.batch, world, args.steps, t)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": t / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
