@@ -98,6 +98,31 @@ def test_small_decode_grid_and_many_segments():
             _check_layer(sc, g, layer)
 
 
+def test_ranges_longer_than_the_cached_table_and_multi_layer_pass():
+    """One or two CTAs over ~2 500 blocks: a range is longer than the 2 048 table entries a CTA keeps
+    in shared memory, so the tail of the range reads its entries from global memory; claims of 16
+    blocks cross the boundary. Checked per layer and as one launch over both layers."""
+    wl = synth.Workload("long", 2, 4, 2, 5, 7000, 8200, 0.45)
+    sc = Scenario(wl, 11)
+    assert sum(synth.blocks_for(int(n)) for n in sc.lengths()) > 2300
+    for ctas, static in ((1, 0), (2, 1)):
+        g = _gpu(sc, decode_ctas=ctas, static_split=static)
+        for layer in range(sc.L):
+            _check_layer(sc, g, layer)
+        seqs = np.array(sc.seq_ids, np.int32)
+        g.out.zero_()
+        assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
+        torch.cuda.synchronize()
+        g.device_ok()
+        from tests.gpu_helpers import to_host
+        got = g.out.view(torch.bfloat16).double().cpu().numpy()
+        for layer in range(sc.L):
+            rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+            _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % wl.ring_slots], resolved,
+                                               sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert attention_close(got[layer], ref, ATOL, RTOL)[0]
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
