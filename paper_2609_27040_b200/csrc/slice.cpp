@@ -1296,12 +1296,19 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       rc = do_layer(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream, next, false, true);
       if (rc) return rc;
     } else {
-      if (next >= 0) {
+      // A ring of one slot: the next layer's data goes where this layer's is, so the prefetch can
+      // only follow the attention (no overlap; the slot-reuse event orders the two streams).
+      const bool same_slot = next >= 0 && static_cast<uint32_t>(next) % R == l % R;
+      if (next >= 0 && !same_slot) {
         rc = do_prefetch(s, static_cast<uint32_t>(next), p, side);
         if (rc) return rc;
       }
       rc = do_layer(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream, -1, false, true);
       if (rc) return rc;
+      if (same_slot) {
+        rc = do_prefetch(s, static_cast<uint32_t>(next), p, side);
+        if (rc) return rc;
+      }
     }
   }
   if (p->k && wrap && L > 1 && (L - 1) % R == 0 && !staged(s, 0, p)) {

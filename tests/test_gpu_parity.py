@@ -123,6 +123,28 @@ def test_ranges_longer_than_the_cached_table_and_multi_layer_pass():
             assert attention_close(got[layer], ref, ATOL, RTOL)[0]
 
 
+@pytest.mark.parametrize("ring,mode", [(1, 0), (1, 1), (3, 0), (3, 1), (3, 2), (4, 0)])
+def test_other_ring_depths(ring, mode):
+    """A ring of one slot cannot overlap anything (every prefetch waits for the attention that reads
+    the slot); rings of three and four slots change which layer a slot holds and which attention a
+    gather has to wait for. Two passes (the second starts from what the first left staged), 5 layers."""
+    wl = synth.Workload("ring", 5, 16, 4, 6, 40, 900, 0.4, ring_slots=ring)
+    sc = Scenario(wl, 21)
+    g = _gpu(sc, pipeline_mode=mode, decode_ctas=12)
+    seqs = np.array(sc.seq_ids, np.int32)
+    for _ in range(2):
+        g.out.zero_()
+        assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
+        torch.cuda.synchronize()
+        g.device_ok()
+        got = g.out.view(torch.bfloat16).double().cpu().numpy()
+        for layer in range(sc.L):
+            rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+            _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % ring], resolved,
+                                               sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert attention_close(got[layer], ref, ATOL, RTOL)[0], (ring, mode, layer)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)

@@ -187,3 +187,22 @@ def test_kv_block_swizzle_is_the_documented_self_inverse_permutation():
                 assert (src == dst).all()
     with pytest.raises(ValueError):
         B.kv_block_swizzle(np.zeros((15, 4, 128), np.uint16))
+
+
+@pytest.mark.parametrize("ring,calls", [(1, 11), (2, 11), (3, 10), (4, 8)])
+def test_decode_step_plans_prefetches_for_any_ring_depth(ring, calls):
+    """Tables-only mode: two passes over 5 layers succeed for every pipeline and ring depth (a ring
+    of one slot prefetches after the attention that reads the slot), and the number of prefetches
+    follows from which layers are still staged when the second pass starts."""
+    for mode in (0, 1, 2):
+        s = B.Slice(5, 4, 64, 64, 64, lent_blocks_physical=64, ring_slots=ring, max_seqs=8, max_blocks_per_seq=64,
+                    flags=B.FLAG_NULL_DEVICE, pipeline_mode=mode)
+        for i in range(3):
+            for b in range(10):
+                assert s.slice_alloc_blocks(i, 1, B.TIER_LENT if b % 2 else B.TIER_LOCAL)[0] == B.OK
+            assert s.slice_set_seq_len(i, 150) == B.OK
+        seqs = np.arange(3, dtype=np.int32)
+        for _ in range(2):
+            assert s.slice_decode_step(seqs, None, 16, 0.1, None, False, True, None, None) == B.OK
+        assert s.slice_stats()["prefetch_calls"] == calls
+        s.slice_destroy()
