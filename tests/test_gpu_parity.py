@@ -145,6 +145,45 @@ def test_other_ring_depths(ring, mode):
             assert attention_close(got[layer], ref, ATOL, RTOL)[0], (ring, mode, layer)
 
 
+def _step_matches_oracle(sc, g, passes=2):
+    seqs = np.array(sc.seq_ids, np.int32)
+    ring = sc.wl.ring_slots
+    for _ in range(passes):
+        g.out.zero_()
+        assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
+        torch.cuda.synchronize()
+        g.device_ok()
+        got = g.out.view(torch.bfloat16).double().cpu().numpy()
+        for layer in range(sc.L):
+            rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+            _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % ring], resolved,
+                                               sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert attention_close(got[layer], ref, ATOL, RTOL)[0], layer
+
+
+@pytest.mark.parametrize("case", ["130_layers", "more_ctas_than_sms", "nothing_lent", "everything_lent", "one_sequence"])
+def test_decode_step_corner_shapes(case):
+    """Shapes at the edges of what one persistent launch covers: more layers than a launch spans and
+    more CTAs than SMs (both fall back to one launch per layer), no lent block at all (nothing to
+    gather, no staging read), every block lent (attention reads the ring only), a single sequence
+    (most CTAs own nothing)."""
+    kw = {}
+    if case == "130_layers":
+        wl = synth.Workload(case, 130, 2, 1, 2, 20, 60, 0.5)
+    elif case == "more_ctas_than_sms":
+        wl = synth.Workload(case, 3, 8, 4, 6, 300, 2500, 0.4)
+        kw["decode_ctas"] = 200
+    elif case == "nothing_lent":
+        wl = synth.Workload(case, 4, 8, 4, 5, 30, 700, 0.0)
+    elif case == "everything_lent":
+        wl = synth.Workload(case, 4, 8, 4, 5, 30, 700, 1.0)
+    else:
+        wl = synth.Workload(case, 4, 16, 4, 1, 3000, 3000, 0.4)
+    sc = Scenario(wl, 17)
+    g = _gpu(sc, **kw)
+    _step_matches_oracle(sc, g)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
