@@ -184,6 +184,41 @@ def test_decode_step_corner_shapes(case):
     _step_matches_oracle(sc, g)
 
 
+def test_many_different_batches_rotate_the_plan_buffers():
+    """More distinct batches (subsets and orders of the sequences) than the library has plan buffers,
+    enqueued back to back without synchronising, then each result checked: a plan buffer must not
+    be rewritten while a launch that reads it is still in flight."""
+    wl = synth.Workload("plans", 3, 16, 4, 8, 50, 1500, 0.4)
+    sc = Scenario(wl, 23)
+    g = _gpu(sc, decode_ctas=24)
+    ids = list(sc.seq_ids)
+    rng = np.random.default_rng(2)
+    batches = [ids, ids[::2], ids[1::2], ids[::-1], ids[:3], ids[3:], [ids[5], ids[0], ids[6]], ids[2:7]]
+    batches += [list(rng.permutation(ids)[: int(rng.integers(1, 9))]) for _ in range(6)]
+    outs = []
+    pos = {i: n for n, i in enumerate(ids)}
+    for bt in batches:
+        seqs = np.array(bt, np.int32)
+        rows = torch.tensor([pos[i] for i in bt], device="cuda")
+        q = g.q.index_select(1, rows).contiguous()
+        out = torch.zeros_like(q)
+        assert g.s.slice_decode_step(seqs, q, sc.Hq, float(sc.sm_scale), out, False, True, g.main, g.side) == B.OK
+        outs.append((bt, q, out))
+    torch.cuda.synchronize()
+    g.device_ok()
+    lens_all = sc.lengths()
+    for bt, q, out in outs:
+        got = out.view(torch.bfloat16).double().cpu().numpy()
+        qh = q.cpu().numpy().view(np.uint16)
+        lens = np.array([lens_all[pos[i]] for i in bt], np.uint32)
+        for layer in range(sc.L):
+            rc, resolved, k = sc.orc.gather(layer, bt, sc.lent, sc.staging)
+            assert rc == 0
+            _, ref, _ = oracle.paged_attention(qh[layer], sc.local[layer], sc.staging[layer % wl.ring_slots], resolved, lens,
+                                               sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert attention_close(got[layer], ref, ATOL, RTOL)[0], (bt, layer)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
