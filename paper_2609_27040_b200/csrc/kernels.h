@@ -73,6 +73,7 @@ struct LayerParams {
   uint32_t own_chunk;           // most blocks an owner claims at a time
   uint32_t steal_floor;         // before the launch's last layer: least a range must have left to be stolen from
   uint32_t steal_floor_last;    // the same in the launch's last layer
+  uint32_t merge_inline;        // 1: the warp that completes a (sequence, KV head) merges it itself
   const void* q;                // first_layer's [nseq][Hq][128] bf16
   void* out;
   uint64_t io_layer_stride;     // bytes from one layer's q / out to the next

@@ -657,8 +657,10 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
   volatile uint32_t* mq = sm.mq;
   uint32_t queued = 0;
   if (lane == 0) {
-    // Up to Hkv warps may pass this check at once, hence the margin.
-    if (static_cast<int32_t>(mq[kMq] - mq[kMq + 1]) < static_cast<int32_t>(kMq - 8)) {
+    // Up to Hkv warps may pass this check at once, hence the margin. When a layer is short
+    // (merge_inline) the merges are the critical path: the Hkv warps that finish a sequence together
+    // merge side by side instead of leaving Hkv merges in a row to the merge warp.
+    if (!p.merge_inline && static_cast<int32_t>(mq[kMq] - mq[kMq + 1]) < static_cast<int32_t>(kMq - 8)) {
       const uint32_t t = atomicAdd(&sm.mq[kMq], 1u);
       const uint64_t t0 = ptx::global_timer_ns();
       while (mq[t % kMq] != kMqEmpty && ptx::global_timer_ns() - t0 < kWaitNs) __nanosleep(64);

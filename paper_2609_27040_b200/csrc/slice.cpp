@@ -23,6 +23,8 @@ constexpr uint32_t kTraceCopyCtas = 2048;
 constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must match the kernel)
 constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a range, at least this
 constexpr uint32_t kStealFloorLast = 8; // default steal floor in the last layer of a launch
+constexpr uint32_t kInlineMergePer = 48; // ranges up to this many blocks: consumer warps merge in line
+constexpr uint32_t kMinPer = 8;          // least blocks per CTA range: fewer CTAs rather than more partials
 constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
@@ -275,8 +277,7 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   // blocks, except one clipped steal and one clipped owner claim per range.
   const uint32_t ncta = s->ncta;
   const uint32_t total = p.total_blocks;
-  uint32_t per = (total + ncta - 1) / ncta;
-  if (per == 0) per = 1;
+  uint32_t per = std::max((total + ncta - 1) / ncta, kMinPer);
   p.per = per;
   p.used_cta = (total + per - 1) / per;
 
@@ -522,6 +523,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.own_chunk = s->cfg.claim_blocks ? s->cfg.claim_blocks : kOwnChunk;
   d.steal_floor = s->cfg.steal_floor ? s->cfg.steal_floor : std::max(kStealFloorMin, p->per / 3);
   d.steal_floor_last = s->cfg.steal_floor ? std::min(s->cfg.steal_floor, kStealFloorLast) : kStealFloorLast;
+  // A layer of a few dozen blocks per CTA lasts less than the merges of one sequence done in a row.
+  d.merge_inline = p->per <= kInlineMergePer ? 1u : 0u;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
