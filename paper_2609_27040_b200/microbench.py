@@ -131,9 +131,139 @@ def reclaim_bench(args):
         del local, lent, before
 
 
+def growth_bench(args):
+    """Bursty KV growth at serving size: Poisson arrivals, one token per sequence per step, blocks
+    allocated as sequences grow (local first, then lent), finished sequences freed, the lender taking
+    2-8 GB back every 200 steps and lending it again 100 steps later; on ENOSPC the most recently
+    admitted sequence is preempted. Every step = one append per layer + one decode pass (one launch).
+    KV contents are whatever the arenas hold (random): only shapes and placement matter for timing."""
+    import time
+    import torch
+    from paper_2609_27040_b200 import binding as B, synth
+    Lr, Hq, Hkv, max_batch = 32, 32, 8, 256
+    total_ids = int(args.arena_gb * 2**30 / (Lr * BLOCK_BYTES))
+    local_blocks = int(total_ids * 0.6)
+    lent_blocks = total_ids - local_blocks
+    shape = (2, 16, Hkv, 128)
+    local = torch.empty((Lr, local_blocks) + shape, dtype=torch.bfloat16, device="cuda")
+    lent = torch.empty((Lr, lent_blocks) + shape, dtype=torch.bfloat16, device="cuda")
+    for l in range(Lr):
+        local[l].normal_()
+        lent[l].normal_()
+    staging = torch.zeros((2, lent_blocks) + shape, dtype=torch.bfloat16, device="cuda")
+    max_blocks = (2048 + 8192) // 16 + 2
+    s = B.Slice(Lr, Hkv, local_blocks, lent_blocks, lent_blocks, local=local, lent=lent, staging=staging, max_seqs=max_batch,
+                max_blocks_per_seq=max_blocks)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    q = torch.empty((Lr, max_batch, Hq, 128), dtype=torch.bfloat16, device="cuda").normal_()
+    out = torch.zeros_like(q)
+    knew = torch.empty((max_batch, Hkv, 128), dtype=torch.bfloat16, device="cuda").normal_()
+    rng = np.random.default_rng(args.seed)
+    arrivals = synth.bursty_arrivals(args.seed, args.steps)
+    by_step = {}
+    for a in arrivals:
+        by_step.setdefault(a.step, []).append(a)
+    waiting, active, length, remaining = [], [], {}, {}
+    next_id = taken = tokens = preempted = enospc = 0
+    alloc_s = 0.0
+    reclaims, lent_frac = [], []
+    scale = 1.0 / float(np.sqrt(128))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    e0.record(main)
+    for t in range(args.steps):
+        waiting += by_step.get(t, [])
+        t_a = time.perf_counter()
+        while waiting and len(active) < max_batch:
+            a = waiting[0]
+            need = synth.blocks_for(a.prompt_len)
+            rc, _ = s.slice_alloc_blocks(next_id, need, B.TIER_AUTO)
+            if rc == B.ENOSPC:               # a failing call changes nothing: the request keeps waiting
+                break
+            assert rc == 0, rc
+            assert s.slice_set_seq_len(next_id, a.prompt_len) == 0
+            waiting.pop(0)
+            active.append(next_id)
+            length[next_id], remaining[next_id] = a.prompt_len, a.output_len
+            next_id += 1
+        if t and t % 200 == 0:
+            take = int(rng.uniform(2, 8) * 2**30 / (Lr * BLOCK_BYTES))
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            r0.record(main)
+            rc, mig = s.slice_reclaim(take, main)
+            while rc == B.ENOSPC and active:  # no room for the blocks in use up there: preempt and retry
+                victim = active.pop()
+                assert s.slice_free_seq(victim) == 0
+                del length[victim], remaining[victim]
+                preempted += 1
+                rc, mig = s.slice_reclaim(take, main)
+            r1.record(main)
+            r1.synchronize()
+            if rc == 0:
+                taken = take
+                reclaims.append({"step": t, "take_ids": take, "migrated_ids": int(mig), "ms": round(r0.elapsed_time(r1), 3),
+                                 "gbs": round(2 * mig * Lr * BLOCK_BYTES / r0.elapsed_time(r1) / 1e6, 1)})
+            else:
+                reclaims.append({"step": t, "take_ids": take, "rc": rc})
+        if t % 200 == 100 and taken:
+            assert s.slice_lend(taken) == 0
+            taken = 0
+        for i in list(active):
+            if i not in length:
+                continue
+            if length[i] % 16 == 0:
+                while s.slice_alloc_blocks(i, 1, B.TIER_AUTO)[0] != 0:
+                    enospc += 1
+                    victim = active[-1]
+                    assert s.slice_free_seq(victim) == 0
+                    active.remove(victim)
+                    del length[victim], remaining[victim]
+                    preempted += 1
+                    if victim == i:
+                        break
+                if i not in length:
+                    continue
+            length[i] += 1
+            assert s.slice_set_seq_len(i, length[i]) == 0
+        alloc_s += time.perf_counter() - t_a
+        if not active:
+            continue
+        seqs = np.array(active, np.int32)
+        n = len(active)
+        for layer in range(Lr):
+            assert s.slice_append_kv(layer, seqs, knew[:n], knew[:n], main) == 0
+        assert s.slice_decode_step(seqs, q[:, :n].contiguous() if n != max_batch else q, Hq, scale, out[:, :n].contiguous() if n != max_batch else out,
+                                   False, True, main, side) == 0
+        tokens += n
+        if t % 50 == 0:
+            st = s.slice_stats()             # reads the device status word: synchronises
+            lent_frac.append(round(st["lent_used"] / max(st["lent_used"] + st["local_used"], 1), 3))
+        for i in list(active):
+            remaining[i] -= 1
+            if remaining[i] <= 0:
+                assert s.slice_free_seq(i) == 0
+                active.remove(i)
+                del length[i], remaining[i]
+    e1.record(main)
+    e1.synchronize()
+    wall = time.perf_counter() - wall0
+    st = s.slice_stats()
+    print(json.dumps({"case": "bursty_growth", "steps": args.steps, "arena_gb": args.arena_gb, "block_ids": total_ids,
+                      "decoded_tokens": tokens, "tokens_per_s": round(tokens / wall, 1), "wall_s": round(wall, 3),
+                      "gpu_stream_s": round(e0.elapsed_time(e1) / 1e3, 3), "sequences_admitted": next_id,
+                      "host_allocator_us_per_step": round(alloc_s / args.steps * 1e6, 1),
+                      "enospc": enospc, "preempted": preempted, "reclaims": reclaims, "lent_fraction_every_50_steps": lent_frac,
+                      "device_status": st["device_status"], "plans_built": st.get("plans_built")}), flush=True)
+    s.slice_destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", choices=["copy", "reclaim", "all"], default="all")
+    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "all"], default="all")
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--arena-gb", type=float, default=48.0)
+    ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--blocks", type=int, nargs="*", default=[1_000, 10_000, 100_000, 400_000])
     ap.add_argument("--ctas", type=int, nargs="*", default=[0, 148, 592])
     ap.add_argument("--take", type=int, nargs="*", default=[954, 3815])
@@ -144,6 +274,8 @@ def main():
         copy_sweep(args)
     if args.what in ("reclaim", "all"):
         reclaim_bench(args)
+    if args.what == "growth":
+        growth_bench(args)
 
 
 if __name__ == "__main__":
