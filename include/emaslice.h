@@ -223,7 +223,11 @@ int slice_lend(slice_t* s, uint32_t n_blocks);
 /* One new token per sequence (the caller has already grown len and allocated a block where
  * needed): writes K and V rows of token len-1 for `layer` into the home block and, when the home is
  * lent and the layer is validly staged for this batch, into the staged copy too.
- *   k_new, v_new  device, [nseq][num_kv_heads][128] bf16. */
+ *   k_new, v_new  device, [nseq][num_kv_heads][128] bf16 (canonical order; the call applies the block
+ *                 format's swizzle).
+ *   layer == SLICE_ALL_LAYERS appends to every layer in one launch (at most 128 layers):
+ *                 k_new, v_new are then [num_layers][nseq][num_kv_heads][128]. */
+#define SLICE_ALL_LAYERS 0xFFFFFFFFu
 int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* k_new,
                     const void* v_new, void* stream);
 

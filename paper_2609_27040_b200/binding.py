@@ -148,6 +148,9 @@ def kv_block_swizzle(x):
     return out.reshape(shape)
 
 
+ALL_LAYERS = 0xFFFFFFFF
+
+
 class Slice:
     """Owner of one ``slice_t`` handle. Methods are named after the C entry points and return the
     status code (plus outputs); ``check=True`` turns a non-zero status into SliceError."""

@@ -124,11 +124,16 @@ size_t static_scratch_needed(uint32_t slots, uint32_t Hq, uint32_t nseq, uint32_
 cudaError_t launch_layer_static(LayerParams p, uint32_t slots, cudaStream_t stream);
 
 struct AppendParams {
-  uint8_t* local_layer;        // this layer's local arena
+  uint8_t* local_layer;        // local arena of the first layer appended to
   uint64_t local_block_stride;
-  uint8_t* lent_layer;         // this layer's lent arena
+  uint8_t* lent_layer;         // lent arena of the first layer appended to
   uint64_t lent_block_stride;
-  uint8_t* slot_base;          // ring slot holding the layer, or NULL when not staged
+  uint8_t* slot_base;          // one layer: ring slot holding the layer, or NULL when not staged
+  // several layers in one launch (grid.y = layer): strides to the next layer, and which layers are staged
+  uint32_t num_layers, first_layer, ring_slots;
+  uint64_t local_layer_stride, lent_layer_stride, io_layer_stride, slot_bytes;
+  uint8_t* staging_base;
+  uint32_t staged_mask[4];     // bit l: layer first_layer + l is validly staged for this batch
   uint64_t block_bytes;
   const int32_t* home_entry;   // [nseq] table entry of the block holding token len-1
   const int32_t* stage_pos;    // [nseq] staging position of that block, or -1

@@ -1042,7 +1042,7 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
   }
 }
 
-// One CTA per sequence: the new token's K and V rows go to the home block and the staged copy.
+// One CTA per (sequence, layer): the new token's K and V rows go to the home block and the staged copy.
 __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   const uint32_t i = blockIdx.x;
   if (i >= p.nseq) return;
@@ -1050,14 +1050,18 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   if (len == 0) return;
   const uint32_t r = (len - 1) % p.block_tokens;
   const int32_t e = p.home_entry[i];
-  uint8_t* home = e >= 0 ? p.local_layer + static_cast<uint64_t>(e) * p.local_block_stride
-                         : p.lent_layer + static_cast<uint64_t>(~e) * p.lent_block_stride;
+  const uint32_t y = blockIdx.y;  // layer within the launch
+  uint8_t* home = e >= 0 ? p.local_layer + y * p.local_layer_stride + static_cast<uint64_t>(e) * p.local_block_stride
+                         : p.lent_layer + y * p.lent_layer_stride + static_cast<uint64_t>(~e) * p.lent_block_stride;
   const int32_t sp = p.stage_pos[i];
-  uint8_t* staged = (p.slot_base && sp >= 0) ? p.slot_base + static_cast<uint64_t>(sp) * p.block_bytes : nullptr;
+  uint8_t* slot = p.slot_base;
+  if (p.num_layers > 1)
+    slot = (p.staged_mask[y >> 5] >> (y & 31u)) & 1u ? p.staging_base + ((p.first_layer + y) % p.ring_slots) * p.slot_bytes : nullptr;
+  uint8_t* staged = (slot && sp >= 0) ? slot + static_cast<uint64_t>(sp) * p.block_bytes : nullptr;
   const uint32_t plane = p.block_tokens * p.row_bytes;
   const uint32_t vecs = p.row_bytes >> 4;
-  const uint4* ks = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(p.k_new) + static_cast<uint64_t>(i) * p.row_bytes);
-  const uint4* vs = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(p.v_new) + static_cast<uint64_t>(i) * p.row_bytes);
+  const uint4* ks = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(p.k_new) + y * p.io_layer_stride + static_cast<uint64_t>(i) * p.row_bytes);
+  const uint4* vs = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(p.v_new) + y * p.io_layer_stride + static_cast<uint64_t>(i) * p.row_bytes);
   for (uint32_t v = threadIdx.x; v < vecs; v += blockDim.x) {
     const uint4 kv = ks[v], vv = vs[v];
     const uint32_t w = (v & ~7u) | ((v & 7u) ^ (r & 7u));  // the block format's swizzle of 16-byte units
@@ -1103,7 +1107,7 @@ cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t stream) {
   if (p.nseq == 0) return cudaSuccess;
-  append_kv_kernel<<<p.nseq, 128, 0, stream>>>(p);
+  append_kv_kernel<<<dim3(p.nseq, p.num_layers ? p.num_layers : 1), 128, 0, stream>>>(p);
   return cudaGetLastError();
 }
 

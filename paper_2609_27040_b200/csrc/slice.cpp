@@ -1113,7 +1113,9 @@ int slice_lend(slice_t* s, uint32_t n) {
 
 int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* k_new,
                     const void* v_new, void* stream_v) {
-  if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
+  const bool all = layer == SLICE_ALL_LAYERS;
+  if (!s || (!all && layer >= s->cfg.num_layers)) return SLICE_EINVAL;
+  if (all && s->cfg.num_layers > 128) return SLICE_EINVAL;
   if (!s->null_dev && (!k_new || !v_new)) return SLICE_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   Plan* p = nullptr;
@@ -1127,16 +1129,29 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   if (rc) return rc;
   rc = plan_on_stream(s, p, stream);
   if (rc) return rc;
-  const uint32_t slot = layer % s->cfg.ring_slots;
-  SlotState& sl = s->slots[slot];
-  const bool is_staged = staged(s, layer, p);
-  if (is_staged && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  const uint32_t first = all ? 0 : layer, count = all ? s->cfg.num_layers : 1;
   ema::AppendParams a{};
-  a.local_layer = static_cast<uint8_t*>(s->cfg.local_base) + layer * s->local_ls;
+  bool one_staged = false;
+  for (uint32_t l = first; l < first + count; ++l) {
+    SlotState& sl = s->slots[l % s->cfg.ring_slots];
+    if (!staged(s, l, p)) continue;
+    if (sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    a.staged_mask[(l - first) >> 5] |= 1u << ((l - first) & 31u);
+    one_staged = true;
+  }
+  a.local_layer = static_cast<uint8_t*>(s->cfg.local_base) + first * s->local_ls;
   a.local_block_stride = s->local_bs;
-  a.lent_layer = static_cast<uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  a.lent_layer = static_cast<uint8_t*>(s->cfg.lent_base) + first * s->lent_ls;
   a.lent_block_stride = s->lent_bs;
-  a.slot_base = is_staged ? static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes : nullptr;
+  a.slot_base = (count == 1 && one_staged) ? static_cast<uint8_t*>(s->cfg.staging_base) + (first % s->cfg.ring_slots) * s->slot_bytes : nullptr;
+  a.num_layers = count;
+  a.first_layer = first;
+  a.ring_slots = s->cfg.ring_slots;
+  a.local_layer_stride = s->local_ls;
+  a.lent_layer_stride = s->lent_ls;
+  a.io_layer_stride = static_cast<uint64_t>(nseq) * s->cfg.num_kv_heads * kHeadDim * 2;
+  a.slot_bytes = s->slot_bytes;
+  a.staging_base = static_cast<uint8_t*>(s->cfg.staging_base);
   a.block_bytes = s->block_bytes;
   a.home_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_home);
   a.stage_pos = reinterpret_cast<const int32_t*>(p->dev + p->off_stage_pos);

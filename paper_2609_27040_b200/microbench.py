@@ -135,7 +135,7 @@ def growth_bench(args):
     """Bursty KV growth at serving size: Poisson arrivals, one token per sequence per step, blocks
     allocated as sequences grow (local first, then lent), finished sequences freed, the lender taking
     2-8 GB back every 200 steps and lending it again 100 steps later; on ENOSPC the most recently
-    admitted sequence is preempted. Every step = one append per layer + one decode pass (one launch).
+    admitted sequence is preempted. Every step = one append launch (all layers) + one decode launch.
     KV contents are whatever the arenas hold (random): only shapes and placement matter for timing."""
     import time
     import torch
@@ -157,7 +157,7 @@ def growth_bench(args):
     main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
     q = torch.empty((Lr, max_batch, Hq, 128), dtype=torch.bfloat16, device="cuda").normal_()
     out = torch.zeros_like(q)
-    knew = torch.empty((max_batch, Hkv, 128), dtype=torch.bfloat16, device="cuda").normal_()
+    knew = torch.empty((Lr, max_batch, Hkv, 128), dtype=torch.bfloat16, device="cuda").normal_()
     rng = np.random.default_rng(args.seed)
     arrivals = synth.bursty_arrivals(args.seed, args.steps)
     by_step = {}
@@ -231,8 +231,8 @@ def growth_bench(args):
             continue
         seqs = np.array(active, np.int32)
         n = len(active)
-        for layer in range(Lr):
-            assert s.slice_append_kv(layer, seqs, knew[:n], knew[:n], main) == 0
+        kn = knew if n == max_batch else knew[:, :n].contiguous()
+        assert s.slice_append_kv(B.ALL_LAYERS, seqs, kn, kn, main) == 0
         assert s.slice_decode_step(seqs, q[:, :n].contiguous() if n != max_batch else q, Hq, scale, out[:, :n].contiguous() if n != max_batch else out,
                                    False, True, main, side) == 0
         tokens += n

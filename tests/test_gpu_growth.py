@@ -135,11 +135,15 @@ def test_bursty_growth_replica_matches_oracle(pipeline_mode, static_split):
         _tables_equal(s, orc, active)
         seqs = np.array(active, np.int32)
         n = len(active)
+        k_new = synth.normal_bf16_bits(rng, (L, n, HKV, D))
+        v_new = synth.normal_bf16_bits(rng, (L, n, HKV, D))
         for layer in range(L):
-            k_new = synth.normal_bf16_bits(rng, (n, HKV, D))
-            v_new = synth.normal_bf16_bits(rng, (n, HKV, D))
-            assert orc.append_kv(layer, seqs, k_new, v_new, HKV, D, local, lent, None) == 0
-            assert s.slice_append_kv(layer, seqs, to_dev(k_new), to_dev(v_new), main) == B.OK
+            assert orc.append_kv(layer, seqs, k_new[layer], v_new[layer], HKV, D, local, lent, None) == 0
+        if static_split:        # every layer in one launch
+            assert s.slice_append_kv(B.ALL_LAYERS, seqs, to_dev(k_new), to_dev(v_new), main) == B.OK
+        else:
+            for layer in range(L):
+                assert s.slice_append_kv(layer, seqs, to_dev(k_new[layer]), to_dev(v_new[layer]), main) == B.OK
         q = synth.normal_bf16_bits(rng, (L, n, HQ, D))
         gq = to_dev(q)
         gout = torch.zeros_like(gq)

@@ -330,6 +330,30 @@ def test_append_kv_writes_home_and_staged_copy():
             assert (kv_to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
             _check_layer(sc, g, layer)       # re-prefetches (already staged plan) and attends
         assert (kv_to_host(g.local) == sc.local).all() and (kv_to_host(g.lent) == sc.lent).all()
+    # every layer in one launch, with both ring slots validly staged (layers 0 and 1): the staged
+    # copies get the rows too
+    for i in sc.seq_ids:
+        _, tab, ln = sc.orc.block_table(i)
+        if ln % sc.T == 0:
+            assert sc.orc.alloc_blocks(i, 1, oracle.AUTO)[0] == 0 and g.s.slice_alloc_blocks(i, 1, B.TIER_AUTO)[0] == 0
+        assert sc.orc.set_seq_len(i, ln + 1) == 0 and g.s.slice_set_seq_len(i, ln + 1) == 0
+        sc.pl.lengths[i] = ln + 1
+    k_all = synth.normal_bf16_bits(rng, (sc.L, sc.nseq, sc.Hkv, sc.D))
+    v_all = synth.normal_bf16_bits(rng, (sc.L, sc.nseq, sc.Hkv, sc.D))
+    for layer in range(sc.L):
+        assert g.s.prefetch_layer(layer, sc.seq_ids, g.side) == B.OK
+        assert sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)[0] == 0
+        assert sc.orc.append_kv(layer, sc.seq_ids, k_all[layer], v_all[layer], sc.Hkv, sc.D, sc.local, sc.lent,
+                                sc.staging[layer % wl.ring_slots]) == 0
+    assert g.s.slice_append_kv(B.ALL_LAYERS, sc.seq_ids, to_dev(k_all), to_dev(v_all), g.main) == B.OK
+    torch.cuda.synchronize()
+    k = g.s.slice_get_resolved(sc.seq_ids)[2]
+    for layer in range(sc.L):
+        slot = layer % wl.ring_slots
+        assert (kv_to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all()
+    assert (kv_to_host(g.local) == sc.local).all() and (kv_to_host(g.lent) == sc.lent).all()
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer)
 
 
 def test_writeback_round_trip():
