@@ -206,6 +206,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   RingPos pos;
   bool ok = true;
 
+  // Every KV byte is read once per pass: its L2 lines are the first to go, which leaves the L2 to
+  // the staged blocks the gather has just written (they are read one layer later).
+  const uint64_t pol_stream = ptx::policy_evict_first();
   // What is the same in every layer of the launch: the own range, its resolved entries (copied to
   // shared memory as far as they fit) and the sequence its first block belongs to.
   const bool owner = blockIdx.x < p.used_cta;
@@ -336,7 +339,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
               ptx::mbar_arrive_expect_tx(full, plane_bytes);
               // One request per plane: an SM streams far faster through few large bulk copies than
               // through many small ones.
-              ptx::bulk_g2s(ring + stg * hsb, src + plane * plane_bytes, plane_bytes, full);
+              ptx::bulk_g2s_hint(ring + stg * hsb, src + plane * plane_bytes, plane_bytes, full, pol_stream);
             }
           }
         }
@@ -911,6 +914,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   const uint32_t pieces = static_cast<uint32_t>((p.block_bytes + kCopyChunk - 1) / kCopyChunk);
   const uint32_t ring = ptx::smem_u32(sm.copy_ring);
   const uint64_t pol = ptx::policy_evict_first();
+  const uint64_t pol_keep = ptx::policy_evict_last();  // staged lines: wanted again within a layer's time
   uint32_t issued = 0, done = 0;  // pieces over the whole launch: stages and barrier phases continue
   bool ok = true;
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
@@ -981,7 +985,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       const uint32_t stg = done % kNC;
       ok = ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[stg]), (done / kNC) & 1u, p.status, kDevTimeout);
       if (!ok) break;
-      ptx::bulk_s2g(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg]);
+      ptx::bulk_s2g_hint(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg], pol_keep);
       ptx::bulk_commit();
       ++done;
       // All but the newest kNC - kCopyLoadsAhead stores are complete after this wait: their stages
