@@ -24,7 +24,7 @@ constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must 
 constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a range, at least this
 constexpr uint32_t kStealFloorLast = 8; // default steal floor in the last layer of a launch
 constexpr uint32_t kInlineMergePer = 48; // ranges up to this many blocks: consumer warps merge in line
-constexpr uint32_t kMinPer = 8;          // least blocks per CTA range: fewer CTAs rather than more partials
+constexpr uint32_t kMinPer = 12;          // least blocks per CTA range: fewer CTAs rather than more partials
 constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
