@@ -84,7 +84,8 @@ class DeviceWorkload:
     """Arenas, tables and query tensors of one workload on the current CUDA device."""
 
     def __init__(self, wl: synth.Workload, seed: int, flags: int = 0, copy_kind: int = 0, copy_ctas: int = 0,
-                 decode_ctas: int = 0, pipeline_mode: int = 0, static_split: int = 0, steal_floor: int = 0):
+                 decode_ctas: int = 0, pipeline_mode: int = 0, static_split: int = 0, steal_floor: int = 0,
+                 prefetch_priority: int = 0):
         import torch
         from paper_2609_27040_b200 import binding as B
         self.wl, self.B = wl, B
@@ -114,7 +115,8 @@ class DeviceWorkload:
                          max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks, flags=flags,
                          local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order,
                          copy_kind=copy_kind, copy_ctas=copy_ctas, decode_ctas=decode_ctas,
-                         pipeline_mode=pipeline_mode, static_split=static_split, steal_floor=steal_floor)
+                         pipeline_mode=pipeline_mode, static_split=static_split, steal_floor=steal_floor,
+                         prefetch_priority=prefetch_priority)
         t0 = time.perf_counter()
         for i, hints in enumerate(pl.hints):
             for h in hints:
@@ -439,21 +441,25 @@ def run_ours(args, wl):
             abl["two_streams"]["event_stall_definition"] = "max(0, end of prefetch(l) - end of attention(l-1)) from CUDA events"
             del wt
             torch.cuda.empty_cache()
-            # Lock step: idle CTAs steal down to the last block of every layer, so all CTAs change layers
-            # together and (almost) none waits for prefetched data.
+            # Ways to keep attention from waiting for prefetched blocks, each at a price in tokens/s:
+            # lock step (idle CTAs steal down to the last block of every layer, so all CTAs change
+            # layers together), prefetch priority (the copy threads keep 4 instead of 3 loads in
+            # flight and win the bandwidth they need), and both.
             if args.pipeline_mode == 0:
-                wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, steal_floor=1, **kw)
-                for _ in range(3):
+                for label, opts in (("lock_step_stealing", {"steal_floor": 1}), ("prefetch_priority", {"prefetch_priority": 1}),
+                                    ("prefetch_priority_lock_step", {"steal_floor": 1, "prefetch_priority": 1})):
+                    wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **opts, **kw)
+                    for _ in range(3):
+                        wa.step(wrap)
+                    ta = wa.timed(reps, wrap)
                     wa.step(wrap)
-                ta = wa.timed(reps, wrap)
-                wa.step(wrap)
-                tr = wa.s.slice_cta_trace(0).astype(np.float64)
-                abl["lock_step_stealing"] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
-                                             "hbm_gbs_combined": step_bytes * reps / ta / 1e9,
-                                             "stall_us_per_layer": float((tr[1:, :, 1] / 1e3).mean()),
-                                             "note": "traced run (a few per cent slower than an untraced one)"}
-                del wa
-                torch.cuda.empty_cache()
+                    tr = wa.s.slice_cta_trace(0).astype(np.float64)
+                    abl[label] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
+                                  "hbm_gbs_combined": step_bytes * reps / ta / 1e9,
+                                  "stall_us_per_layer": float((tr[1:, :, 1] / 1e3).mean()),
+                                  "note": "traced run (a few per cent slower than an untraced one)"}
+                    del wa
+                    torch.cuda.empty_cache()
             ws = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, pipeline_mode=1, **kw)
             for _ in range(2):
                 assert ws.s.slice_decode_step(ws.seqs, ws.q, wl.num_q_heads, ws.scale, ws.out, False, wrap, ws.main, ws.main) == 0
@@ -474,18 +480,25 @@ def run_ours(args, wl):
             abl["serialised_prefetch"] = {"tokens_per_s": wl.batch * n_ser / t_serial, "ms_per_step": t_serial / n_ser * 1e3,
                                           "note": "on-demand variant: prefetch not overlapped with attention"}
             extra["ablations"] = abl
-            if "lock_step_stealing" in abl:
-                ls = abl["lock_step_stealing"]
+            alts = {k: v for k, v in abl.items() if "stall_us_per_layer" in v}
+            if alts:
+                def frac(v):
+                    return v["stall_us_per_layer"] / (v["ms_per_step"] * 1e3 / L)
+                ok = [k for k, v in alts.items() if frac(v) < 0.05 and v["hbm_gbs_combined"] / NOMINAL_HBM_GBS >= 0.70]
+                pick = max(ok, key=lambda k: alts[k]["tokens_per_s"]) if ok else min(alts, key=lambda k: frac(alts[k]))
                 extra["targets"] = {
                     "hbm_frac_of_nominal_8TBs": {"target": 0.70, "default_pipeline": combined / NOMINAL_HBM_GBS,
-                                                 "lock_step_pipeline": ls["hbm_gbs_combined"] / NOMINAL_HBM_GBS},
+                                                 pick: alts[pick]["hbm_gbs_combined"] / NOMINAL_HBM_GBS},
                     "stall_frac_of_layer": {"target": 0.05, "default_pipeline": extra["stall_frac_of_layer"],
-                                            "lock_step_pipeline": ls["stall_us_per_layer"] / (ls["ms_per_step"] * 1e3 / L)},
-                    "note": "the default pipeline maximises tokens/s; steal_floor = 1 (lock step) meets both targets at once"}
+                                            pick: frac(alts[pick])},
+                    "both_met_by": pick if ok else None,
+                    "note": "the default pipeline maximises tokens/s (it is HBM-bound, the wait is slack of the faster "
+                            "stream); the named configuration trades tokens/s for a prefetch that is always ahead"}
             extra["kernels_alone"] = {
                 "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
-                                                "frac": attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak},
+                                                "frac": attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak,
+                                                "note": "one launch per layer, prefetch serialised before it"},
                 "copy_blocks_vector_gather": {"us_per_launch": iso_pref_us, "algorithmic_bytes": pref_bytes_layer,
                                               "achieved_gbs": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9,
                                               "frac": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9 / peak}}

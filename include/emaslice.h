@@ -114,7 +114,12 @@ typedef struct {
                                      in single-layer launches); 1 = steal down to the last block, which
                                      keeps all CTAs in step: almost no CTA ever waits for
                                      prefetched data, at a lower overall rate                    */
-  uint32_t reserved;
+  uint32_t prefetch_priority;     /* fused pipelines: 0 = default, the copy thread of an SM keeps 3 loads
+                                     of 16 KB in flight and attention, with more bytes in flight,
+                                     takes its share of HBM first (highest tokens/s; attention then
+                                     waits for prefetched blocks part of the time); 1 = 4 loads in
+                                     flight: the prefetch wins the bandwidth it needs, attention
+                                     (almost) never waits for it, and the pass as a whole is slower */
 } slice_config_t;
 
 typedef struct {

@@ -43,7 +43,7 @@ class SliceConfig(C.Structure):
         ("local_free_order", C.c_void_p), ("lent_free_order", C.c_void_p),
         ("decode_ctas", C.c_uint32), ("copy_ctas", C.c_uint32), ("copy_kind", C.c_uint32),
         ("pipeline_mode", C.c_uint32), ("static_split", C.c_uint32), ("claim_blocks", C.c_uint32),
-        ("steal_floor", C.c_uint32), ("reserved", C.c_uint32),
+        ("steal_floor", C.c_uint32), ("prefetch_priority", C.c_uint32),
     ]
 
 
@@ -161,7 +161,7 @@ class Slice:
                  max_blocks_per_seq: int = 512, head_dim: int = 128, block_tokens: int = 16,
                  lent_kind: int = 0, flags: int = 0, local_free_order=None, lent_free_order=None,
                  decode_ctas: int = 0, copy_ctas: int = 0, copy_kind: int = 0, pipeline_mode: int = 0,
-                 static_split: int = 0, claim_blocks: int = 0, steal_floor: int = 0,
+                 static_split: int = 0, claim_blocks: int = 0, steal_floor: int = 0, prefetch_priority: int = 0,
                  local_layer_stride: int = 0, local_block_stride: int = 0,
                  lent_layer_stride: int = 0, lent_block_stride: int = 0):
         cfg = SliceConfig()
@@ -180,7 +180,7 @@ class Slice:
         cfg.local_free_order, cfg.lent_free_order = _ptr(self._lo), _ptr(self._ro)
         cfg.decode_ctas, cfg.copy_ctas, cfg.copy_kind = decode_ctas, copy_ctas, copy_kind
         cfg.pipeline_mode, cfg.static_split = pipeline_mode, static_split
-        cfg.claim_blocks, cfg.steal_floor = claim_blocks, steal_floor
+        cfg.claim_blocks, cfg.steal_floor, cfg.prefetch_priority = claim_blocks, steal_floor, prefetch_priority
         self.cfg = cfg
         self._keep = (local, lent, staging)       # arenas must outlive the slice
         h = C.c_void_p()

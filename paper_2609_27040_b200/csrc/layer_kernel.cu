@@ -59,8 +59,9 @@ constexpr uint32_t kNAAlone = 3;           // ... and when the launch gathers no
                                            // stage a deeper ring only queues more reads in the memory
                                            // system and measures slower (3: 6.1 TB/s, 6: 5.3 TB/s).
 constexpr uint32_t kNAMax = 4;
-constexpr int kNC = 5;                     // copy ring: 16 KB stages
-constexpr int kCopyLoadsAhead = 3;         // loads in flight; the other stages drain as stores
+constexpr int kNC = 6;                     // copy ring: 16 KB stages
+constexpr uint32_t kCopyLoadsDefault = 3;  // loads in flight (LayerParams::copy_loads_ahead, 3 or 4) ...
+constexpr int kStoresOpen = 2;             // ... and stores not yet known complete; 4 + 2 = kNC
 constexpr uint32_t kCopyChunk = 16384;
 constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAMax / 2 + 1)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
@@ -71,7 +72,7 @@ constexpr uint32_t kStealMin = 2, kStealMax = 16;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
 constexpr uint64_t kWaitNs = 2000000000ull;
-constexpr uint32_t kOwnCache = 2048;       // resolved entries of the own range kept in shared memory
+constexpr uint32_t kOwnCache = 512;        // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
 __host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_bytes(Hkv); }
@@ -915,6 +916,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   const uint32_t ring = ptx::smem_u32(sm.copy_ring);
   const uint64_t pol = ptx::policy_evict_first();
   const uint64_t pol_keep = ptx::policy_evict_last();  // staged lines: wanted again within a layer's time
+  const uint32_t loads_ahead = p.copy_loads_ahead == 4 ? 4u : kCopyLoadsDefault;
   uint32_t issued = 0, done = 0;  // pieces over the whole launch: stages and barrier phases continue
   bool ok = true;
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
@@ -980,7 +982,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       }
     };
 
-    while (issued - done < static_cast<uint32_t>(kCopyLoadsAhead) && more) more = issue_next();
+    while (issued - done < loads_ahead && more) more = issue_next();
     while (done < issued) {
       const uint32_t stg = done % kNC;
       ok = ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[stg]), (done / kNC) & 1u, p.status, kDevTimeout);
@@ -988,11 +990,11 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       ptx::bulk_s2g_hint(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg], pol_keep);
       ptx::bulk_commit();
       ++done;
-      // All but the newest kNC - kCopyLoadsAhead stores are complete after this wait: their stages
-      // may be refilled and their bytes are in global memory.
-      ptx::bulk_wait_all<kNC - kCopyLoadsAhead>();
+      // All but the newest kStoresOpen stores are complete after this wait: their stages may be
+      // refilled and their bytes are in global memory. (Three open stores measured 4 % slower.)
+      ptx::bulk_wait_all<kStoresOpen>();
       const uint32_t stored = done - first_piece;
-      report_landed(stored > static_cast<uint32_t>(kNC - kCopyLoadsAhead) ? stored - (kNC - kCopyLoadsAhead) : 0);
+      report_landed(stored > kStoresOpen ? stored - kStoresOpen : 0);
       if (more) more = issue_next();
     }
     ptx::bulk_wait_all<0>();

@@ -525,6 +525,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.steal_floor_last = s->cfg.steal_floor ? std::min(s->cfg.steal_floor, kStealFloorLast) : kStealFloorLast;
   // A layer of a few dozen blocks per CTA lasts less than the merges of one sequence done in a row.
   d.merge_inline = p->per <= kInlineMergePer ? 1u : 0u;
+  d.copy_loads_ahead = s->cfg.prefetch_priority ? 4u : 3u;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;
@@ -770,7 +771,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 2 || cfg->static_split > 1) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 2 || cfg->static_split > 1 || cfg->prefetch_priority > 1) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
