@@ -219,6 +219,17 @@ def test_many_different_batches_rotate_the_plan_buffers():
             assert attention_close(got[layer], ref, ATOL, RTOL)[0], (bt, layer)
 
 
+@pytest.mark.parametrize("knobs", [{"steal_floor": 1}, {"prefetch_priority": 1}, {"claim_blocks": 4},
+                                   {"claim_blocks": 32, "steal_floor": 3}, {"prefetch_priority": 1, "steal_floor": 1, "static_split": 1}])
+def test_scheduling_knobs_do_not_change_results(knobs):
+    """Claim size, steal floor and the number of copy loads in flight decide who does what when,
+    never what is computed."""
+    wl = synth.Workload("knobs", 5, 32, 8, 7, 60, 1400, 0.45)
+    sc = Scenario(wl, 29)
+    g = _gpu(sc, decode_ctas=20, **knobs)
+    _step_matches_oracle(sc, g)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
