@@ -919,6 +919,9 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   const uint32_t loads_ahead = p.copy_loads_ahead == 4 ? 4u : kCopyLoadsDefault;
   uint32_t issued = 0, done = 0;  // pieces over the whole launch: stages and barrier phases continue
   bool ok = true;
+  // Over a slow link only a few SMs copy: a handful of them keeps the link full, and an SM whose
+  // copy engine is queued up with slow loads also delays its own attention loads.
+  if (p.copy_sms && blockIdx.x >= p.copy_sms) return;
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
     const int32_t target = p.gather_target[li];
     if (target < 0 || p.copy_n == 0) continue;

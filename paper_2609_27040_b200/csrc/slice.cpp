@@ -24,6 +24,7 @@ constexpr uint32_t kStealMin = 2;  // smallest unclipped steal, in blocks (must 
 constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a range, at least this
 constexpr uint32_t kStealFloorLast = 8; // default steal floor in the last layer of a launch
 constexpr uint32_t kInlineMergePer = 48; // ranges up to this many blocks: consumer warps merge in line
+constexpr uint32_t kSlowLinkCopySms = 8;  // copy threads that take part in the gather over a slow link
 constexpr uint32_t kMinPer = 12;          // least blocks per CTA range: fewer CTAs rather than more partials
 constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
@@ -526,6 +527,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   // A layer of a few dozen blocks per CTA lasts less than the merges of one sequence done in a row.
   d.merge_inline = p->per <= kInlineMergePer ? 1u : 0u;
   d.copy_loads_ahead = s->cfg.prefetch_priority ? 4u : 3u;
+  // Lent arena behind a slow link (pinned host memory): a few copy threads saturate it.
+  d.copy_sms = s->cfg.lent_kind == 1 ? (s->cfg.copy_ctas ? std::min(s->cfg.copy_ctas, s->ncta) : std::min(kSlowLinkCopySms, s->ncta)) : 0u;
   d.q = q;
   d.out = out;
   d.io_layer_stride = static_cast<uint64_t>(p->nseq) * Hq * kHeadDim * 2;

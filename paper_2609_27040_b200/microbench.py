@@ -258,12 +258,84 @@ def growth_bench(args):
     s.slice_destroy()
 
 
+def link_bench(args):
+    """The paper's transparency condition (Section 2.3 / 4: a transfer of m bytes over a link of
+    bandwidth B is hidden when it fits in the latency window L between two uses, B*L >= m) with a
+    real bandwidth-limited link: the lent arena lives in pinned host memory (lent_kind = 1), so the
+    prefetch crosses PCIe. For a sweep of lent fractions f: measured time per layer of the one-launch
+    pass against the model max(T0, m/B), T0 = time per layer with nothing lent, m = lent bytes per
+    layer, B = link rate measured with the stand-alone gather from the same arena."""
+    import dataclasses
+    import torch
+    from paper_2609_27040_b200 import binding as B, synth
+    Lr = 8
+    rows = []
+    for f in args.fractions:
+        wl = dataclasses.replace(synth.WORKLOADS["llama3_8b_decode"], num_layers=Lr, lent_fraction=f)
+        pl = synth.make_placement(wl, args.seed, slack_blocks=64)
+        shape = (2, 16, wl.num_kv_heads, 128)
+        local = torch.empty((Lr, pl.local_blocks) + shape, device="cuda", dtype=torch.bfloat16).normal_()
+        lent = torch.empty((Lr, max(pl.lent_blocks, 1)) + shape, dtype=torch.bfloat16).normal_().pin_memory()
+        staging = torch.zeros((2, max(pl.staging_blocks, 1)) + shape, device="cuda", dtype=torch.bfloat16)
+        q = torch.empty((Lr, wl.batch, wl.num_q_heads, 128), device="cuda", dtype=torch.bfloat16).normal_()
+        out = torch.zeros_like(q)
+        s = B.Slice(Lr, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks, local=local, lent=lent,
+                    staging=staging, max_seqs=wl.batch, max_blocks_per_seq=300, lent_kind=1,
+                    local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
+        for i, hints in enumerate(pl.hints):
+            for h in hints:
+                assert s.slice_alloc_blocks(i, 1, int(h))[0] == 0
+            assert s.slice_set_seq_len(i, int(pl.lengths[i])) == 0
+        seqs = np.arange(wl.batch, dtype=np.int32)
+        main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+        scale = 1.0 / float(np.sqrt(128))
+        m = pl.staging_blocks * BLOCK_BYTES
+        link_gbs = None
+        if m:
+            def gather():
+                assert s.prefetch_layer(3, seqs, main) == 0
+                assert s.prefetch_layer(5, seqs, main) == 0      # same slot, other layer: always a real copy
+            us = _time_us(gather, main, 5) / 2
+            link_gbs = m / us / 1e3
+        for _ in range(3):
+            assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 10
+        e0.record(main)
+        for _ in range(reps):
+            assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
+        e1.record(main)
+        e1.synchronize()
+        rows.append({"f": f, "lent_bytes_per_layer": m, "us_per_layer": e0.elapsed_time(e1) * 1e3 / reps / Lr,
+                     "link_gbs": link_gbs, "device_status": s.slice_stats()["device_status"]})
+        s.slice_destroy()
+        del local, lent, staging
+    t0 = min(r["us_per_layer"] for r in rows if r["lent_bytes_per_layer"] == 0) if any(r["lent_bytes_per_layer"] == 0 for r in rows) else None
+    rates = [r["link_gbs"] for r in rows if r["link_gbs"]]
+    link = max(rates) if rates else None
+    for r in rows:
+        if t0 is not None and link:
+            pred = max(t0, r["lent_bytes_per_layer"] / (link * 1e3))
+            r.update({"model_us_per_layer": round(pred, 1), "stall_us_measured": round(r["us_per_layer"] - t0, 1),
+                      "stall_us_model": round(pred - t0, 1), "measured_over_model": round(r["us_per_layer"] / pred, 3)})
+        r["us_per_layer"] = round(r["us_per_layer"], 1)
+        r["link_gbs"] = round(r["link_gbs"], 1) if r["link_gbs"] else None
+        print(json.dumps({"case": "link", **r}), flush=True)
+    if t0 is not None and link:
+        bytes_layer = 614.3e6
+        print(json.dumps({"case": "link_summary", "T0_us_per_layer": round(t0, 1), "link_gbs": round(link, 1),
+                          "knee_lent_bytes_per_layer": round(link * 1e3 * t0), "knee_fraction_of_kv": round(link * 1e3 * t0 / bytes_layer, 4),
+                          "model": "time per layer = max(T0, m / B_link): the transfer is hidden while B*L >= m"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "all"], default="all")
+    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "all"], default="all")
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--arena-gb", type=float, default=48.0)
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--fractions", type=float, nargs="*", default=[0.0, 0.002, 0.005, 0.01, 0.02, 0.05, 0.1, 0.2])
     ap.add_argument("--blocks", type=int, nargs="*", default=[1_000, 10_000, 100_000, 400_000])
     ap.add_argument("--ctas", type=int, nargs="*", default=[0, 148, 592])
     ap.add_argument("--take", type=int, nargs="*", default=[954, 3815])
@@ -276,6 +348,8 @@ def main():
         reclaim_bench(args)
     if args.what == "growth":
         growth_bench(args)
+    if args.what == "link":
+        link_bench(args)
 
 
 if __name__ == "__main__":

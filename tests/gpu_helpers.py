@@ -30,10 +30,14 @@ def kv_to_host(t: torch.Tensor) -> np.ndarray:
 
 
 class GpuScenario:
-    def __init__(self, sc: Scenario, **kw):
+    def __init__(self, sc: Scenario, host_lent: bool = False, **kw):
         self.sc = sc
         self.local = kv_to_dev(sc.local)
-        self.lent = kv_to_dev(sc.lent)
+        if host_lent:       # the lent arena behind a real link: mapped pinned host memory
+            self.lent = torch.from_numpy(B.kv_block_swizzle(sc.lent).view(np.int16)).pin_memory()
+            kw["lent_kind"] = 1
+        else:
+            self.lent = kv_to_dev(sc.lent)
         self.staging = kv_to_dev(sc.staging)
         self.q = to_dev(sc.q)
         self.out = torch.zeros_like(self.q)

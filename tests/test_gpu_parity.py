@@ -230,6 +230,44 @@ def test_scheduling_knobs_do_not_change_results(knobs):
     _step_matches_oracle(sc, g)
 
 
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_lent_arena_in_pinned_host_memory(mode):
+    """The lent part behind a real, slow link (PCIe): prefetch, one-launch pass, append to lent tail
+    blocks, write-back and reclaim all read or write the host arena and must give the same bytes and
+    the same attention as with the arena in HBM."""
+    wl = synth.Workload("hostlent", 4, 16, 4, 6, 40, 900, 0.35)
+    sc = Scenario(wl, 33, slack=64)
+    g = _gpu(sc, host_lent=True, pipeline_mode=mode, decode_ctas=16)
+    from tests.gpu_helpers import kv_to_host, to_dev
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer)
+    _step_matches_oracle(sc, g)
+    # grow every sequence by a token (all layers in one launch), attend again
+    rng = np.random.default_rng(8)
+    for i in sc.seq_ids:
+        _, tab, ln = sc.orc.block_table(i)
+        if ln % sc.T == 0:
+            assert sc.orc.alloc_blocks(i, 1, oracle.AUTO)[0] == 0 and g.s.slice_alloc_blocks(i, 1, B.TIER_AUTO)[0] == 0
+        assert sc.orc.set_seq_len(i, ln + 1) == 0 and g.s.slice_set_seq_len(i, ln + 1) == 0
+        sc.pl.lengths[i] = ln + 1
+    k_all = synth.normal_bf16_bits(rng, (sc.L, sc.nseq, sc.Hkv, sc.D))
+    v_all = synth.normal_bf16_bits(rng, (sc.L, sc.nseq, sc.Hkv, sc.D))
+    for layer in range(sc.L):
+        assert sc.orc.append_kv(layer, sc.seq_ids, k_all[layer], v_all[layer], sc.Hkv, sc.D, sc.local, sc.lent, None) == 0
+    assert g.s.slice_append_kv(B.ALL_LAYERS, sc.seq_ids, to_dev(k_all), to_dev(v_all), g.main) == B.OK
+    _step_matches_oracle(sc, g, passes=1)
+    torch.cuda.synchronize()
+    assert (kv_to_host(g.local) == sc.local).all() and (kv_to_host(g.lent) == sc.lent).all()
+    # the lender takes half of it back: blocks migrate out of the host arena
+    take = sc.orc.lent_capacity // 2
+    rc, mig = sc.orc.reclaim(take, sc.local, sc.lent)
+    rc2, mig2 = g.s.slice_reclaim(take, g.main)
+    assert rc == rc2 == 0 and mig == mig2 and mig > 0
+    torch.cuda.synchronize()
+    g.tables_equal_oracle()
+    _step_matches_oracle(sc, g, passes=1)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
