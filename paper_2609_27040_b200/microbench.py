@@ -267,7 +267,7 @@ def link_bench(args):
     layer, B = link rate measured with the stand-alone gather from the same arena."""
     import dataclasses
     import torch
-    from paper_2609_27040_b200 import binding as B, synth
+    from paper_2609_27040_b200 import binding as B, capacity, synth
     Lr = 8
     rows = []
     for f in args.fractions:
@@ -316,7 +316,7 @@ def link_bench(args):
     link = max(rates) if rates else None
     for r in rows:
         if t0 is not None and link:
-            pred = max(t0, r["lent_bytes_per_layer"] / (link * 1e3))
+            pred = capacity.layer_time(t0, r["lent_bytes_per_layer"], link * 1e3)   # us, bytes, bytes per us
             r.update({"model_us_per_layer": round(pred, 1), "stall_us_measured": round(r["us_per_layer"] - t0, 1),
                       "stall_us_model": round(pred - t0, 1), "measured_over_model": round(r["us_per_layer"] / pred, 3)})
         r["us_per_layer"] = round(r["us_per_layer"], 1)
