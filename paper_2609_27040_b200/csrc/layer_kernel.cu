@@ -10,23 +10,27 @@
 //
 // Work distribution. The batch's blocks, flattened in batch order, are cut into one contiguous range
 // per CTA (the same for every layer). A CTA claims blocks from the FRONT of its own range; a CTA
-// whose range is used up steals from the BACK of the range with the most unclaimed blocks. Both
-// kinds of claim are one atomicAdd on the range's packed 64-bit word (front count | back count), so
-// they can never overlap. SMs stream at visibly different rates (position on the die, mixed
-// read/write traffic); stealing keeps all of them busy. A CTA keeps one running softmax state per
-// "run" = consecutive claims within one sequence, so partial results stay few.
+// whose range is used up steals from the BACK of the range with the most unclaimed blocks, provided
+// that range is well behind (steal floor), and otherwise moves on to the next layer. Both kinds of
+// claim are one atomicAdd on the range's packed 64-bit word (front count | back count), so they can
+// never overlap. SMs stream at visibly different rates (position on the die, mixed read/write
+// traffic). A CTA keeps one running softmax state per "run" = consecutive claims within one
+// sequence, so partial results stay few.
 //
 // Roles inside a CTA (warps):
 //   * producer warp: claims work and streams KV blocks into a shared-memory ring of half blocks
-//     (K plane / V plane, 16 token rows of Hkv*256 B, each row padded by 16 B so ldmatrix is
-//     bank-conflict free) with untiled TMA bulk copies (cp.async.bulk, one row per lane), completion
-//     by mbarrier expect-tx; a small descriptor queue tells the consumers what each unit is.
+//     (K plane / V plane, 16 token rows of Hkv*256 B) with ONE untiled TMA bulk copy per plane
+//     (cp.async.bulk, 32 KB for 8 KV heads: small copies cap the rate an SM can stream at),
+//     completion by mbarrier expect-tx; the block format stores the 16-byte units of a row swizzled,
+//     so the linear copy leaves a layout that ldmatrix reads without bank conflicts. A small
+//     descriptor queue tells the consumers what each unit is.
 //   * one consumer warp per KV head: tile products on tensor cores when the GQA group is >= 2
 //     (mma.sync m16n8k16 bf16, swapped form), f32 FMAs when G == 1; online softmax with warp
 //     shuffles. A finished run writes (max, sums, unnormalised output) to a partial slot and adds its
 //     block count to the (sequence, KV head) counter; the warp whose addition completes the sequence
 //     queues a merge request (the ring is shared by all consumer warps, so a warp that stopped to
-//     merge would stall the whole CTA).
+//     merge would stall the whole CTA) or, when layers are short, merges in line (then the merges
+//     of a sequence's KV heads run side by side instead of one after the other).
 //   * merge warp: serves the CTA's merge requests; consumer warps join it once their streaming is
 //     over.
 //   * copy warp: one thread moves 16 KB pieces lent arena -> shared ring -> staging slot with TMA
@@ -34,12 +38,13 @@
 //     64 KB units from an atomic counter. No SM lane touches the copied bytes.
 //
 // Waits. Inside a CTA everything is mbarriers. Between CTAs there are three waits, only in launches
-// that span several layers (which are launched cooperatively, so every CTA is resident): staged
-// blocks of layer l are read only after all of l's gathered blocks have landed; a ring slot is
-// overwritten only after the attention of the layer that last used it is complete; a partial
+// that span several layers (which are launched cooperatively, so every CTA is resident): a staged
+// block of layer l is read only after its ready flag shows that the gather has landed it; a ring
+// slot is overwritten only after the attention of the layer that last used it is complete; a partial
 // buffer (two alternate) is reused only after the merges of the layer before last are done. They
-// wait on counters that earlier layers' work increments, never on later work, so they cannot form a
-// cycle. Every wait, mbarrier or counter, is bounded (about two seconds): on expiry the role records
+// wait on what earlier layers' work produces, never on later work, and a run left open at the end of
+// a layer is closed at once (a CTA may find nothing to claim in later layers), so they cannot form a
+// cycle. A fourth, optional wait is for queries that arrive from the host while the launch runs. Every wait, mbarrier or counter, is bounded (about two seconds): on expiry the role records
 // SLICE_ETIMEOUT in the status word, gives its own copies in flight a bounded chance to land and
 // returns.
 // HBM-bound: algorithmic bytes per layer = sum_s len_s * 2*Hkv*128*2 (+ q, out, table)
