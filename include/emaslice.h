@@ -70,7 +70,11 @@ enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
 enum {
   SLICE_FLAG_PROFILE = 1u,     /* record timing events around the kernels (slice_layer_times)     */
   SLICE_FLAG_TRACE = 2u,       /* per-CTA device-timer traces (slice_cta_trace)                    */
-  SLICE_FLAG_NULL_DEVICE = 4u  /* tables only: no CUDA call is made, no kernel is launched       */
+  SLICE_FLAG_NULL_DEVICE = 4u, /* tables only: no CUDA call is made, no kernel is launched       */
+  SLICE_FLAG_TEST_WITHHOLD_Q = 8u /* test hook for the bounded waits: queries streamed in from pinned
+                                     host memory arrive, their arrival flags are never written, so
+                                     the kernel's wait for them runs out (about two seconds) and it
+                                     returns with SLICE_ETIMEOUT in slice_stats().device_status     */
 };
 
 typedef struct {

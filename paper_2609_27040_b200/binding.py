@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libemaslice.so")
 
 OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
-FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE = 1, 2, 4
+FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE, FLAG_TEST_WITHHOLD_Q = 1, 2, 4, 8
 COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
 TAKE_ALL = 0xFFFFFFFF
 

@@ -1277,7 +1277,8 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
         const size_t bytes = per_layer * std::min(per_flag, L - l0);
         CU(s, cudaMemcpyAsync(static_cast<uint8_t*>(s->io_q) + l0 * per_layer, static_cast<const uint8_t*>(q) + l0 * per_layer, bytes,
                               cudaMemcpyHostToDevice, s->io_stream));
-        CU(s, cudaMemcpyAsync(s->q_flags_dev + l0 / per_flag, epoch_word, sizeof(uint32_t), cudaMemcpyHostToDevice, s->io_stream));
+        if (!(s->cfg.flags & SLICE_FLAG_TEST_WITHHOLD_Q))
+          CU(s, cudaMemcpyAsync(s->q_flags_dev + l0 / per_flag, epoch_word, sizeof(uint32_t), cudaMemcpyHostToDevice, s->io_stream));
       }
       s->step_q_ready = s->q_flags_dev;
       s->step_q_layers = per_flag;
