@@ -792,7 +792,7 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
       if (run_li >= q_upto) {  // q may still be on its way from the host: wait for this layer's chunk
-        if (p.q_ready && !wait_counter_eq(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
         q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
       }
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
@@ -877,7 +877,7 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
       if (run_li >= q_upto) {
-        if (p.q_ready && !wait_counter_eq(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
         q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
       }
       const __nv_bfloat16* qg =

@@ -1271,7 +1271,10 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       CU(s, cudaStreamWaitEvent(s->io_stream, s->ev_tmp, 0));
       const uint32_t per_flag = 4;
       ++s->q_epoch;
-      uint32_t* epoch_word = s->q_epoch_host + (s->q_epoch % 64);  // a slot of its own while copies of it are in flight
+      // The flag copies read this word when they execute; epochs only grow and the kernel waits for
+      // "at least its own", so a word overwritten by a later pass that is enqueued far ahead still
+      // says what it must: this pass's chunk has arrived (its copy precedes the flag copy).
+      uint32_t* epoch_word = s->q_epoch_host + (s->q_epoch % 64);
       *epoch_word = s->q_epoch;
       for (uint32_t l0 = 0; l0 < L; l0 += per_flag) {
         const size_t bytes = per_layer * std::min(per_flag, L - l0);
