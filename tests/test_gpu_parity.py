@@ -268,6 +268,18 @@ def test_lent_arena_in_pinned_host_memory(mode):
     _step_matches_oracle(sc, g, passes=1)
 
 
+@pytest.mark.parametrize("hq,hkv", [(12, 4), (6, 1), (40, 8), (7, 1), (10, 2)])
+def test_group_sizes_that_are_not_powers_of_two(hq, hkv):
+    """GQA groups of 3, 6, 5, 7 and 5 query heads per KV head: the MMA tile pads the group to 8
+    columns and the merge goes head by head."""
+    wl = synth.Workload("oddg", 3, hq, hkv, 5, 20, 800, 0.4)
+    sc = Scenario(wl, 37)
+    g = _gpu(sc, decode_ctas=16)
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer)
+    _step_matches_oracle(sc, g, passes=1)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
