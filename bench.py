@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--pipeline-mode", type=int, default=0,
                     help="0 one persistent launch per pass, 1 two streams with events, 2 one fused launch per layer")
     ap.add_argument("--static-split", type=int, default=0, help="1: no work stealing between CTAs")
+    ap.add_argument("--prefetch-priority", type=int, default=0,
+                    help="1: the copy threads keep 4 loads in flight (prefetch always ahead, slower pass)")
     ap.add_argument("--no-ablations", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
@@ -313,7 +315,7 @@ def run_ours(args, wl):
 
     # Replicas only: every rank runs the same workload shape on its own GPU with its own seed.
     kw = dict(copy_kind=args.copy_kind, copy_ctas=args.copy_ctas, decode_ctas=args.decode_ctas,
-              static_split=args.static_split)
+              static_split=args.static_split, prefetch_priority=args.prefetch_priority)
     w = DeviceWorkload(wl, args.seed + rank, pipeline_mode=args.pipeline_mode, **kw)
     wrap = not args.no_wrap
     for _ in range(max(args.warmup, 3)):
@@ -448,7 +450,7 @@ def run_ours(args, wl):
             if args.pipeline_mode == 0:
                 for label, opts in (("lock_step_stealing", {"steal_floor": 1}), ("prefetch_priority", {"prefetch_priority": 1}),
                                     ("prefetch_priority_lock_step", {"steal_floor": 1, "prefetch_priority": 1})):
-                    wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **opts, **kw)
+                    wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **{**kw, **opts})
                     for _ in range(3):
                         wa.step(wrap)
                     ta = wa.timed(reps, wrap)
