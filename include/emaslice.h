@@ -86,7 +86,9 @@ typedef struct {
   uint32_t ring_slots;            /* staging ring depth R >= 1; layer l uses slot l mod R        */
   uint32_t staging_blocks_per_slot;
   uint32_t max_seqs, max_blocks_per_seq;
-  uint32_t lent_kind;             /* 0 = device HBM arena, 1 = mapped pinned-host arena          */
+  uint32_t lent_kind;             /* 0 = device HBM arena, 1 = mapped pinned-host arena (a slow link:
+                                     in the fused pipelines only a few SMs then copy; copy_ctas, if
+                                     set, says how many)                                          */
   uint32_t flags;                 /* SLICE_FLAG_*                                                */
   void* local_base;               /* device pointers, caller-owned (may be NULL with NULL_DEVICE) */
   void* lent_base;
@@ -109,8 +111,8 @@ typedef struct {
                                      CTAs steal from the ranges with most left (default); 1 = static
                                      ranges only                                                  */
   uint32_t claim_blocks;          /* most KV blocks a CTA claims from its own range at a time
-                                     (0 = default); smaller claims leave more for idle CTAs to
-                                     steal, larger ones cost fewer atomics                       */
+                                     (0 = default 16, at most 32); smaller claims leave more for idle
+                                     CTAs to steal, larger ones cost fewer atomics               */
   uint32_t steal_floor;           /* persistent pass (pipeline_mode 0): before the last layer an idle
                                      CTA steals only from a range with at least this many blocks
                                      left, and otherwise starts on the next layer. 0 = default (a
@@ -119,11 +121,11 @@ typedef struct {
                                      keeps all CTAs in step: almost no CTA ever waits for
                                      prefetched data, at a lower overall rate                    */
   uint32_t prefetch_priority;     /* fused pipelines: 0 = default, the copy thread of an SM keeps 3 loads
-                                     of 16 KB in flight and attention, with more bytes in flight,
-                                     takes its share of HBM first (highest tokens/s; attention then
-                                     waits for prefetched blocks part of the time); 1 = 4 loads in
-                                     flight: the prefetch wins the bandwidth it needs, attention
-                                     (almost) never waits for it, and the pass as a whole is slower */
+                                     of 16 KB in flight; attention follows the prefetch closely,
+                                     waits for it part of the time and reads staged blocks out of L2
+                                     (highest tokens/s); 1 = 4 loads in flight: the prefetch stays
+                                     far ahead, attention (almost) never waits for it, staged blocks
+                                     come from DRAM and the pass as a whole is slower             */
 } slice_config_t;
 
 typedef struct {
