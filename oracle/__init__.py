@@ -19,7 +19,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ema_oracle.cpp")
 _LIB = os.path.join(_HERE, "libema_oracle.so")
 
-OK, E_INVAL, E_NOSPC, E_STAGING, E_STATE = 0, -1, -2, -3, -7
+OK, E_INVAL, E_NOSPC, E_STAGING, E_STATE, E_CAPPED = 0, -1, -2, -3, -7, -9
+PREEMPT_OOM, PREEMPT_RECLAIM = 1, 2
 AUTO, LOCAL, LENT = 0, 1, 2
 
 
@@ -62,6 +63,12 @@ def lib() -> C.CDLL:
         L.oracle_to_bf16.restype = None
         L.oracle_reclaim.argtypes = [vp, u32, vp, vp, vp]
         L.oracle_lend.argtypes = [vp, u32]
+        L.oracle_set_preempt_window.argtypes = [vp, u64]
+        L.oracle_set_time.argtypes = [vp, u64]
+        L.oracle_preempt_seq.argtypes = [vp, i32, i32]
+        L.oracle_reclaim_preempt.argtypes = [vp, u32, u32, vp, vp, vp, u32, vp, vp]
+        L.oracle_preempt_state.argtypes = [vp, vp]
+        L.oracle_preempt_state.restype = None
         L.oracle_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, u32, u32, vp, vp, vp]
         L.oracle_num_threads.restype = C.c_int
     return _lib
@@ -175,6 +182,32 @@ class OracleSlice:
 
     def lend(self, n: int) -> int:
         return lib().oracle_lend(self._h, n)
+
+    # -- preemption ---------------------------------------------------------------------------
+    def set_preempt_window(self, window: int) -> int:
+        return lib().oracle_set_preempt_window(self._h, window)
+
+    def set_time(self, now: int) -> int:
+        return lib().oracle_set_time(self._h, now)
+
+    def preempt_seq(self, seq: int, cause: int) -> int:
+        return lib().oracle_preempt_seq(self._h, seq, cause)
+
+    def reclaim_preempt(self, take: int, slab_blocks: int, local_arena: Optional[np.ndarray],
+                        lent_arena: Optional[np.ndarray], max_victims: Optional[int] = None):
+        """Returns (rc, evicted sequence ids in eviction order, migrated blocks)."""
+        cap = self.max_seqs if max_victims is None else max_victims
+        victims = np.zeros(max(cap, 1), np.int32)
+        n, mig = C.c_uint32(0), C.c_uint64(0)
+        rc = lib().oracle_reclaim_preempt(self._h, min(take, 0xFFFFFFFF), slab_blocks, _ptr(local_arena),
+                                          _ptr(lent_arena), _ptr(victims), cap, C.byref(n), C.byref(mig))
+        return rc, victims[:n.value].tolist(), mig.value
+
+    def preempt_state(self) -> dict:
+        out = np.zeros(6, np.uint64)
+        lib().oracle_preempt_state(self._h, _ptr(out))
+        keys = ("preempt_oom", "preempt_reclaim", "now", "window", "cap_until", "cap_level")
+        return {k: int(v) for k, v in zip(keys, out)}
 
     def append_kv(self, layer: int, seqs: Sequence[int], k_new: np.ndarray, v_new: np.ndarray,
                   num_kv_heads: int, head_dim: int, local_arena: np.ndarray, lent_arena: np.ndarray,

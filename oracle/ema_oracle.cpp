@@ -22,11 +22,20 @@
 //                 The paper does it by preempting the borrower; this build migrates the lent
 //                 blocks instead and rewrites the mapping tables (the variant the task fixes).
 //   * O-append  — one new token's K/V row written to its home block and to the staged copy.
+//   * O-preempt — the paper's own reclaim (Section 4.1): when the lender wants capacity back and
+//                 the borrower has no room to keep the data, requests of the borrower are evicted
+//                 until it has; the allocator picks "a slab ... that contains the fewest number
+//                 of active requests" (Section 4.2.1); after a preemption above the static share
+//                 the user's allocations are capped for a window T (Section 5.3, bursty workload
+//                 preemption control); preemptions are counted by cause (Section 6.6).
 //
 // Parity pins (tests/test_oracle_*.py): paged == dense brute force; softmax row sums; closed
 // forms (n=1, equal keys, constant V, dominant key, score shift, token permutation); fp64
 // library attention; NaN-poisoned tails; tag round trips for gather; byte/logical-order
-// preservation for migration; allocator invariants under random operation sequences.
+// preservation for migration; allocator invariants under random operation sequences; for
+// O-preempt hand-worked victim choices and cap time lines, twin states that reclaim without
+// preemption, a brute-force request count per slab, and the back-and-forth scenario of
+// Section 5.3 with and without the cap (tests/test_oracle_preempt.py).
 // Bit-level agreement of the GPU attention with this file is "parity unpinned" beyond the
 // stated tolerance, by design: any result within tolerance is correct.
 //
@@ -56,6 +65,7 @@ enum Status : int {
   E_NOSPC = -2,
   E_STAGING = -3,
   E_STATE = -7,
+  E_CAPPED = -9,
 };
 
 enum Tier : int { AUTO = 0, LOCAL = 1, LENT = 2 };
@@ -88,7 +98,20 @@ struct State {
   std::map<int32_t, Seq> seqs;
   std::vector<Owner> owner_local;
   std::vector<Owner> owner_lent;
+  // Preemption control (O-preempt). Time is a number the caller sets; the window is in its unit.
+  uint64_t now = 0;
+  uint64_t window = 0;      // T; 0 = no cap is ever set
+  uint64_t cap_until = 0;   // a cap holds while now < cap_until
+  uint32_t cap_level = 0;   // blocks the user may hold while the cap holds
+  uint64_t preempt_oom = 0, preempt_reclaim = 0;
 };
+
+inline uint32_t used_blocks(const State* s) {
+  uint32_t u = 0;
+  for (const auto& kv : s->seqs) u += static_cast<uint32_t>(kv.second.table.size());
+  return u;
+}
+inline bool cap_holds(const State* s) { return s->window > 0 && s->now < s->cap_until; }
 
 inline double bf16_to_double(uint16_t b) {
   uint32_t u = static_cast<uint32_t>(b) << 16;
@@ -162,6 +185,8 @@ int oracle_alloc_blocks(void* h, int32_t seq, uint32_t n, int32_t hint, int32_t*
   if (!exists && s->seqs.size() >= s->max_seqs) return E_INVAL;
   const size_t have = exists ? it->second.table.size() : 0;
   if (have + n > s->max_blocks_per_seq) return E_INVAL;
+  // Section 5.3: while a cap from an earlier preemption holds, the user may not grow past it.
+  if (n > 0 && cap_holds(s) && used_blocks(s) + n > s->cap_level) return E_CAPPED;
   const size_t fl = s->free_local.size(), fr = s->free_lent.size();
   if (hint == AUTO && n > fl + fr) return E_NOSPC;
   if (hint == LOCAL && n > fl) return E_NOSPC;
@@ -472,6 +497,132 @@ int oracle_reclaim(void* h, uint32_t take, uint8_t* local_arena, uint8_t* lent_a
   s->lent_cap = cut;
   if (out_migrated) *out_migrated = victims.size();
   return OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// O-preempt: reclaim by preemption, the cap that follows it, and the counters.
+// ------------------------------------------------------------------------------------------
+
+// Time and window T of the preemption cap (Section 5.3). The paper gives T no unit: the caller
+// chooses one and reports the time in it; time never runs backwards.
+int oracle_set_preempt_window(void* h, uint64_t window) {
+  static_cast<State*>(h)->window = window;
+  return OK;
+}
+
+int oracle_set_time(void* h, uint64_t now) {
+  State* s = static_cast<State*>(h);
+  if (now < s->now) return E_INVAL;
+  s->now = now;
+  return OK;
+}
+
+namespace {
+// Section 5.3: a user preempted while it holds more than its static share (its own, local part of
+// the slice: half of a symmetric slice) is limited to the level it was preempted to; a later
+// preemption inside the window can only lower the level, and every one restarts the window.
+void note_reclaim_preemption(State* s, uint32_t used_before, uint32_t used_after) {
+  if (s->window == 0 || used_before <= s->local_blocks) return;
+  s->cap_level = cap_holds(s) ? std::min(s->cap_level, used_after) : used_after;
+  s->cap_until = s->now + s->window;
+}
+}  // namespace
+
+// One request is preempted by the engine's own choice. cause: 1 = out of memory (the user's own
+// requests give way because capacity is exhausted), 2 = reclamation by the lender (Section 5.2
+// names the two causes, Section 6.6 counts them). Only cause 2 can set the cap.
+int oracle_preempt_seq(void* h, int32_t seq, int32_t cause) {
+  State* s = static_cast<State*>(h);
+  if (cause != 1 && cause != 2) return E_INVAL;
+  if (s->seqs.find(seq) == s->seqs.end()) return E_STATE;
+  const uint32_t before = used_blocks(s);
+  oracle_free_seq(h, seq);
+  if (cause == 1) {
+    ++s->preempt_oom;
+  } else {
+    ++s->preempt_reclaim;
+    note_reclaim_preemption(s, before, used_blocks(s));
+  }
+  return OK;
+}
+
+// The lender takes the top `take` ids back and the borrower may have no room for what is stored
+// there. Section 4.1: requests of the borrower are evicted "until" enough is reclaimed; Section
+// 4.2.1: the allocator takes the slab with the fewest active requests. Slabs are runs of
+// slab_blocks consecutive lent ids (the last one may be short). While the blocks that must leave
+// the reclaimed range outnumber the free places (local, or lent below the cut), the slab of the
+// lent range that holds blocks of the fewest distinct requests (at least one; ties: the highest
+// slab) loses all its requests, in ascending id order. What then remains in the range migrates as
+// in O-reclaim. victims (cap entries) receives the evicted ids in eviction order.
+// Returns E_INVAL, with nothing changed, when slab_blocks is 0 or cap is too small.
+int oracle_reclaim_preempt(void* h, uint32_t take, uint32_t slab_blocks, uint8_t* local_arena,
+                           uint8_t* lent_arena, int32_t* victims, uint32_t cap,
+                           uint32_t* n_victims, uint64_t* out_migrated) {
+  State* s = static_cast<State*>(h);
+  if (slab_blocks == 0) return E_INVAL;
+  if (take > s->lent_cap) take = s->lent_cap;
+  const uint32_t cut = s->lent_cap - take;
+  // Choose first (nothing changes if the caller's array is too small), on a copy of the owners.
+  std::vector<int32_t> chosen;
+  auto gone = [&](int32_t seq) {
+    return std::find(chosen.begin(), chosen.end(), seq) != chosen.end();
+  };
+  for (;;) {
+    size_t must_move = 0, room = s->free_local.size();
+    for (uint32_t id = cut; id < s->lent_cap; ++id)
+      if (s->owner_lent[id].seq >= 0 && !gone(s->owner_lent[id].seq)) ++must_move;
+    for (int32_t id : s->free_lent)
+      if (static_cast<uint32_t>(id) < cut) ++room;
+    for (uint32_t id = 0; id < s->local_blocks; ++id)
+      if (s->owner_local[id].seq >= 0 && gone(s->owner_local[id].seq)) ++room;
+    for (uint32_t id = 0; id < cut; ++id)
+      if (s->owner_lent[id].seq >= 0 && gone(s->owner_lent[id].seq)) ++room;
+    if (must_move <= room) break;
+    const uint32_t nslabs = (s->lent_cap + slab_blocks - 1) / slab_blocks;
+    int64_t best = -1;
+    size_t best_count = 0;
+    std::vector<int32_t> best_set;
+    for (uint32_t sl = 0; sl < nslabs; ++sl) {
+      std::vector<int32_t> in_slab;
+      const uint32_t hi = std::min(s->lent_cap, (sl + 1) * slab_blocks);
+      for (uint32_t id = sl * slab_blocks; id < hi; ++id) {
+        const int32_t q = s->owner_lent[id].seq;
+        if (q >= 0 && !gone(q) && std::find(in_slab.begin(), in_slab.end(), q) == in_slab.end())
+          in_slab.push_back(q);
+      }
+      if (in_slab.empty()) continue;
+      if (best < 0 || in_slab.size() <= best_count) {  // <= : the highest slab wins a tie
+        best = sl;
+        best_count = in_slab.size();
+        best_set = in_slab;
+      }
+    }
+    std::sort(best_set.begin(), best_set.end());
+    for (int32_t q : best_set) chosen.push_back(q);
+  }
+  if (chosen.size() > cap) return E_INVAL;
+  const uint32_t before = used_blocks(s);
+  for (size_t k = 0; k < chosen.size(); ++k) {
+    oracle_free_seq(h, chosen[k]);
+    if (victims) victims[k] = chosen[k];
+    ++s->preempt_reclaim;
+  }
+  if (n_victims) *n_victims = static_cast<uint32_t>(chosen.size());
+  const int rc = oracle_reclaim(h, take, local_arena, lent_arena, out_migrated);
+  if (!chosen.empty()) note_reclaim_preemption(s, before, used_blocks(s));
+  return rc;
+}
+
+// out[0..6) = preemptions by out-of-memory, preemptions by reclamation, now, window, cap_until,
+// cap level in blocks (0 when no cap holds).
+void oracle_preempt_state(void* h, uint64_t* out) {
+  State* s = static_cast<State*>(h);
+  out[0] = s->preempt_oom;
+  out[1] = s->preempt_reclaim;
+  out[2] = s->now;
+  out[3] = s->window;
+  out[4] = cap_holds(s) ? s->cap_until : 0;
+  out[5] = cap_holds(s) ? s->cap_level : 0;
 }
 
 // The lender offers n more block ids: capacity grows, new ids pop in ascending order.
