@@ -62,7 +62,9 @@ enum {
   SLICE_ECUDA = -5,    /* a CUDA call failed; slice_stats reports the code                       */
   SLICE_ETIMEOUT = -6, /* a bounded device-side wait expired (reported through slice_stats)      */
   SLICE_ESTATE = -7,   /* unknown sequence, double free                                          */
-  SLICE_ESCRATCH = -8  /* paged_decode_noalloc: the batch needs more than the static scratch array */
+  SLICE_ESCRATCH = -8, /* paged_decode_noalloc: the batch needs more than the static scratch array */
+  SLICE_ECAPPED = -9   /* slice_alloc_blocks: a cap set by an earlier preemption still holds
+                          (Section 5.3); the request waits, nobody is preempted for it          */
 };
 
 enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
@@ -153,7 +155,8 @@ int slice_destroy(slice_t* s);
  * sequence seq (created when absent). AUTO takes free local ids first and the lent part only when
  * local memory is exhausted; LOCAL / LENT force a tier (seeded placements). out_entries (host, n
  * entries, may be NULL) receives the new table entries. Errors: ENOSPC (nothing changes), EINVAL
- * (negative seq, bad hint, more than max_seqs sequences or max_blocks_per_seq blocks). */
+ * (negative seq, bad hint, more than max_seqs sequences or max_blocks_per_seq blocks), ECAPPED
+ * (n > 0 and a cap from an earlier preemption holds, see slice_preempt_seq; nothing changes). */
 int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t tier_hint, int32_t* out_entries);
 
 /* Sets the number of valid tokens of seq; len <= block_tokens * allocated blocks.
@@ -226,6 +229,50 @@ int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32
  * block ids moved. The copy is enqueued on stream after all outstanding work of the slice; later
  * calls on other streams wait for it. Errors: ENOSPC (no room; nothing changes), ECUDA. */
 int slice_reclaim(slice_t* s, uint32_t take_blocks, uint64_t* out_n_migrated, void* stream);
+
+/* Section 4.1 as the paper states it: where the migration of slice_reclaim has no room, requests of
+ * the borrower are preempted until it has. Section 4.2.1 gives the choice: the slab with the fewest
+ * active requests. Slabs are runs of slab_blocks consecutive lent ids (the paper's default is 10;
+ * the last slab may be short). While the in-use blocks of the reclaimed range outnumber the free
+ * places (local, or lent below the cut), the slab of the lent range that holds blocks of the
+ * fewest distinct requests (at least one; among equals the highest slab, which lies nearest the
+ * reclaimed range) loses all its requests, in ascending id order: they are freed as by
+ * slice_free_seq and the caller re-queues them. What then remains in the range migrates as in
+ * slice_reclaim (same stream ordering). The call never fails for lack of room.
+ *   victims     host, cap entries: the preempted sequence ids in eviction order; n_victims (host,
+ *               may be NULL) their number; out_n_migrated as in slice_reclaim.
+ * Every victim counts as a preemption by reclamation and, as in slice_preempt_seq, can set the cap.
+ * Errors: EINVAL (slab_blocks == 0, or cap smaller than the number of victims: nothing changes),
+ * ECUDA. */
+int slice_reclaim_preempt(slice_t* s, uint32_t take_blocks, uint32_t slab_blocks, int32_t* victims, uint32_t cap,
+                          uint32_t* n_victims, uint64_t* out_n_migrated, void* stream);
+
+/* A preemption the serving engine chose itself: frees seq like slice_free_seq and counts it by
+ * cause (Section 5.2 names the two, Section 6.6 reports them): SLICE_PREEMPT_OOM, the user's own
+ * requests give way because capacity is exhausted, or SLICE_PREEMPT_RECLAIM, the lender took
+ * memory back. Section 5.3, against back-and-forth preemption under bursty load: a user preempted
+ * by reclamation while it holds more than its static share (the local part of the slice, half of a
+ * symmetric slice) may afterwards not grow beyond the level it was preempted to, for a window of
+ * length T; a later such preemption inside the window can only lower the level and restarts the
+ * window; once T has passed without one the cap is lifted. While the cap holds,
+ * slice_alloc_blocks returns SLICE_ECAPPED for a request that would pass the level.
+ * Errors: EINVAL (cause), ESTATE (unknown seq). */
+enum { SLICE_PREEMPT_OOM = 1, SLICE_PREEMPT_RECLAIM = 2 };
+int slice_preempt_seq(slice_t* s, int32_t seq, int32_t cause);
+
+/* Section 5.3 leaves T and its unit open: the caller sets the window (0, the default, = no cap is
+ * ever set) and reports the time in the same unit (steps, milliseconds, ...); time must not run
+ * backwards (EINVAL). */
+int slice_set_preempt_window(slice_t* s, uint64_t window);
+int slice_set_time(slice_t* s, uint64_t now);
+
+typedef struct {
+  uint64_t preempt_oom, preempt_reclaim; /* requests preempted so far, by cause                    */
+  uint64_t now, window;
+  uint64_t cap_until;                    /* the cap holds while now < cap_until; 0 when none holds */
+  uint64_t cap_level;                    /* blocks the user may hold while it holds; 0 when none   */
+} slice_preempt_stats_t;
+int slice_preempt_stats(slice_t* s, slice_preempt_stats_t* out);
 
 /* The lender offers n more block ids (the share of a slice is renegotiated at run time,
  * Section 1 / 4.1). New ids are handed out in ascending order. Errors: EINVAL (beyond arena). */

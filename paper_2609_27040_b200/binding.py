@@ -16,7 +16,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libemaslice.so")
 
-OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH = 0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH, ECAPPED = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
+PREEMPT_OOM, PREEMPT_RECLAIM = 1, 2
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
 FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE, FLAG_TEST_WITHHOLD_Q = 1, 2, 4, 8
 COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
@@ -27,6 +28,7 @@ EXPORTS = [
     "slice_get_block_table", "slice_get_free_stack", "prefetch_layer", "paged_decode", "slice_reclaim",
     "slice_lend", "slice_append_kv", "slice_writeback_layer", "slice_decode_step", "slice_stats",
     "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc", "slice_cta_trace",
+    "slice_reclaim_preempt", "slice_preempt_seq", "slice_set_preempt_window", "slice_set_time", "slice_preempt_stats",
 ]
 
 
@@ -62,6 +64,16 @@ class SliceStats(C.Structure):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
 
 
+class SlicePreemptStats(C.Structure):
+    _fields_ = [
+        ("preempt_oom", C.c_uint64), ("preempt_reclaim", C.c_uint64), ("now", C.c_uint64),
+        ("window", C.c_uint64), ("cap_until", C.c_uint64), ("cap_level", C.c_uint64),
+    ]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
 _lib = None
 
 
@@ -86,6 +98,11 @@ def lib() -> C.CDLL:
         L.paged_decode_noalloc.argtypes = [vp, u32, vp, u32, vp, u32, C.c_float, vp, vp, vp]
         L.slice_reclaim.argtypes = [vp, u32, vp, vp]
         L.slice_lend.argtypes = [vp, u32]
+        L.slice_reclaim_preempt.argtypes = [vp, u32, u32, vp, u32, vp, vp, vp]
+        L.slice_preempt_seq.argtypes = [vp, C.c_int32, C.c_int32]
+        L.slice_set_preempt_window.argtypes = [vp, C.c_uint64]
+        L.slice_set_time.argtypes = [vp, C.c_uint64]
+        L.slice_preempt_stats.argtypes = [vp, vp]
         L.slice_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, vp]
         L.slice_writeback_layer.argtypes = [vp, u32, vp, u32, vp]
         L.slice_decode_step.argtypes = [vp, vp, u32, vp, u32, C.c_float, vp, i32, i32, vp, vp]
@@ -260,6 +277,32 @@ class Slice:
 
     def slice_lend(self, n_blocks: int) -> int:
         return lib().slice_lend(self._h, n_blocks)
+
+    def slice_reclaim_preempt(self, take_blocks: int = TAKE_ALL, slab_blocks: int = 10, stream=None,
+                              max_victims: int = None):
+        """Returns (rc, preempted sequence ids in eviction order, migrated blocks)."""
+        cap = int(self.cfg.max_seqs) if max_victims is None else max_victims
+        victims = np.zeros(max(cap, 1), np.int32)
+        n, mig = C.c_uint32(0), C.c_uint64(0)
+        rc = lib().slice_reclaim_preempt(self._h, take_blocks, slab_blocks, _ptr(victims), cap, C.byref(n),
+                                         C.byref(mig), _stream(stream))
+        return rc, victims[:n.value].tolist(), mig.value
+
+    def slice_preempt_seq(self, seq: int, cause: int) -> int:
+        return lib().slice_preempt_seq(self._h, seq, cause)
+
+    def slice_set_preempt_window(self, window: int) -> int:
+        return lib().slice_set_preempt_window(self._h, window)
+
+    def slice_set_time(self, now: int) -> int:
+        return lib().slice_set_time(self._h, now)
+
+    def slice_preempt_stats(self) -> dict:
+        st = SlicePreemptStats()
+        rc = lib().slice_preempt_stats(self._h, C.byref(st))
+        if rc != OK:
+            raise SliceError(rc, "slice_preempt_stats")
+        return st.as_dict()
 
     def slice_append_kv(self, layer: int, seqs, k_new, v_new, stream=None) -> int:
         sq = _seqs(seqs)

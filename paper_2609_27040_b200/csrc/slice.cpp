@@ -98,6 +98,10 @@ struct ema_slice {
   std::vector<Owner> owner_local, owner_lent;
   uint32_t lent_cap = 0;
   uint64_t version = 1;
+  // preemption control: caller's clock, window T, the cap in force while now < cap_until
+  uint64_t now = 0, preempt_window = 0, cap_until = 0;
+  uint32_t cap_level = 0;
+  uint64_t preempt_oom = 0, preempt_reclaim = 0;
   // plans and slots
   Plan plans[kNumPlans];
   int next_plan = 0;
@@ -160,6 +164,23 @@ namespace {
 inline uint32_t blocks_for(uint32_t len) { return (len + kBlockTokens - 1) / kBlockTokens; }
 
 inline bool multi_stream(const ema_slice* s) { return s->streams.size() > 1; }
+
+// Blocks the user holds in both parts of the slice.
+inline uint32_t blocks_held(const ema_slice* s) {
+  return static_cast<uint32_t>(s->cfg.local_blocks - s->free_local.size() + s->lent_cap - s->free_lent.size());
+}
+
+inline bool cap_in_force(const ema_slice* s) { return s->preempt_window != 0 && s->now < s->cap_until; }
+
+// Bursty-workload control: a preemption by reclamation above the static share (the local part)
+// limits the user to the level it fell to; inside the window the level only goes down, and every
+// such preemption restarts the window.
+inline void cap_after_reclaim_preemption(ema_slice* s, uint32_t held_before) {
+  if (s->preempt_window == 0 || held_before <= s->cfg.local_blocks) return;
+  const uint32_t level = blocks_held(s);
+  s->cap_level = cap_in_force(s) ? std::min(s->cap_level, level) : level;
+  s->cap_until = s->now + s->preempt_window;
+}
 
 // Registers a stream with the slice. A stream seen for the first time waits for everything the
 // slice has enqueued on the streams it already knows (from then on per-operation events order the
@@ -907,6 +928,7 @@ int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t hint, int32_
   if (!exists && s->seqs.size() >= s->cfg.max_seqs) return SLICE_EINVAL;
   const size_t have = exists ? it->second.table.size() : 0;
   if (have + n > s->cfg.max_blocks_per_seq) return SLICE_EINVAL;
+  if (n > 0 && cap_in_force(s) && static_cast<uint64_t>(blocks_held(s)) + n > s->cap_level) return SLICE_ECAPPED;
   const size_t fl = s->free_local.size(), fr = s->free_lent.size();
   if (hint == SLICE_TIER_AUTO && n > fl + fr) return SLICE_ENOSPC;
   if (hint == SLICE_TIER_LOCAL && n > fl) return SLICE_ENOSPC;
@@ -1104,6 +1126,118 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
   s->st.migrated_blocks += victims.size();
   s->st.migrated_bytes += static_cast<uint64_t>(victims.size()) * s->block_bytes * s->cfg.num_layers;
   if (out_n_migrated) *out_n_migrated = victims.size();
+  return SLICE_OK;
+}
+
+int slice_set_preempt_window(slice_t* s, uint64_t window) {
+  if (!s) return SLICE_EINVAL;
+  s->preempt_window = window;
+  return SLICE_OK;
+}
+
+int slice_set_time(slice_t* s, uint64_t now) {
+  if (!s || now < s->now) return SLICE_EINVAL;
+  s->now = now;
+  return SLICE_OK;
+}
+
+int slice_preempt_seq(slice_t* s, int32_t seq, int32_t cause) {
+  if (!s || (cause != SLICE_PREEMPT_OOM && cause != SLICE_PREEMPT_RECLAIM)) return SLICE_EINVAL;
+  const uint32_t held = blocks_held(s);
+  const int rc = slice_free_seq(s, seq);
+  if (rc) return rc;
+  if (cause == SLICE_PREEMPT_OOM) {
+    ++s->preempt_oom;
+  } else {
+    ++s->preempt_reclaim;
+    cap_after_reclaim_preemption(s, held);
+  }
+  return SLICE_OK;
+}
+
+int slice_reclaim_preempt(slice_t* s, uint32_t take, uint32_t slab_blocks, int32_t* victims, uint32_t cap,
+                          uint32_t* n_victims, uint64_t* out_n_migrated, void* stream) {
+  if (!s || slab_blocks == 0) return SLICE_EINVAL;
+  if (take > s->lent_cap) take = s->lent_cap;
+  const uint32_t cut = s->lent_cap - take;
+  // What has to leave the range and the places it can go to, kept up to date as requests are marked.
+  int64_t must_move = 0, room = static_cast<int64_t>(s->free_local.size());
+  for (uint32_t id = cut; id < s->lent_cap; ++id) must_move += s->owner_lent[id].seq >= 0;
+  for (int32_t id : s->free_lent) room += static_cast<uint32_t>(id) < cut;
+  std::vector<int32_t> order;  // marked requests, in eviction order
+  if (must_move > room) {
+    // Dense request numbers for the lent ids, so that the rounds below touch arrays only.
+    std::unordered_map<int32_t, uint32_t> number;
+    std::vector<int32_t> id_of;
+    std::vector<uint32_t> req(s->lent_cap, UINT32_MAX);
+    for (uint32_t id = 0; id < s->lent_cap; ++id) {
+      const int32_t q = s->owner_lent[id].seq;
+      if (q < 0) continue;
+      auto ins = number.emplace(q, static_cast<uint32_t>(id_of.size()));
+      if (ins.second) id_of.push_back(q);
+      req[id] = ins.first->second;
+    }
+    std::vector<uint32_t> stamp(id_of.size(), 0);  // 1 + slab a request was last counted in
+    std::vector<char> marked(id_of.size(), 0);
+    const uint32_t nslabs = (s->lent_cap + slab_blocks - 1) / slab_blocks;
+    while (must_move > room) {
+      // Requests per slab, each counted once per slab (the ids of a slab are consecutive).
+      uint32_t best = UINT32_MAX, best_n = UINT32_MAX;
+      std::fill(stamp.begin(), stamp.end(), 0u);
+      for (uint32_t sl = 0; sl < nslabs; ++sl) {
+        uint32_t n = 0;
+        const uint32_t end = std::min(s->lent_cap, (sl + 1) * slab_blocks);
+        for (uint32_t id = sl * slab_blocks; id < end; ++id) {
+          const uint32_t r = req[id];
+          if (r == UINT32_MAX || marked[r] || stamp[r] == sl + 1) continue;
+          stamp[r] = sl + 1;
+          ++n;
+        }
+        if (n && n <= best_n) {  // <=: among equals the highest slab
+          best_n = n;
+          best = sl;
+        }
+      }
+      if (best == UINT32_MAX) break;  // nothing in use: cannot happen while must_move > 0
+      std::vector<int32_t> grp;
+      const uint32_t end = std::min(s->lent_cap, (best + 1) * slab_blocks);
+      for (uint32_t id = best * slab_blocks; id < end; ++id) {
+        const uint32_t r = req[id];
+        if (r == UINT32_MAX || marked[r]) continue;
+        marked[r] = 1;
+        grp.push_back(id_of[r]);
+      }
+      std::sort(grp.begin(), grp.end());
+      for (int32_t q : grp) {
+        order.push_back(q);
+        for (int32_t e : s->seqs[q].table) {
+          if (e < 0 && static_cast<uint32_t>(~e) >= cut) --must_move;
+          else ++room;
+        }
+      }
+    }
+  }
+  if (order.size() > cap || (!order.empty() && !victims)) return SLICE_EINVAL;
+  const uint32_t held = blocks_held(s);
+  for (size_t k = 0; k < order.size(); ++k) {
+    slice_free_seq(s, order[k]);
+    victims[k] = order[k];
+    ++s->preempt_reclaim;
+  }
+  if (n_victims) *n_victims = static_cast<uint32_t>(order.size());
+  const int rc = slice_reclaim(s, take, out_n_migrated, stream);
+  if (!order.empty()) cap_after_reclaim_preemption(s, held);
+  return rc;
+}
+
+int slice_preempt_stats(slice_t* s, slice_preempt_stats_t* out) {
+  if (!s || !out) return SLICE_EINVAL;
+  out->preempt_oom = s->preempt_oom;
+  out->preempt_reclaim = s->preempt_reclaim;
+  out->now = s->now;
+  out->window = s->preempt_window;
+  out->cap_until = cap_in_force(s) ? s->cap_until : 0;
+  out->cap_level = cap_in_force(s) ? s->cap_level : 0;
   return SLICE_OK;
 }
 
@@ -1451,6 +1585,7 @@ const char* slice_strerror(int code) {
     case SLICE_ECUDA: return "CUDA call failed";
     case SLICE_ETIMEOUT: return "bounded device wait expired";
     case SLICE_ESTATE: return "unknown sequence or bad state";
+    case SLICE_ECAPPED: return "a cap set by an earlier preemption holds";
     case SLICE_ESCRATCH: return "request exceeds the static scratch array";
     default: return "unknown status";
   }

@@ -134,8 +134,13 @@ def reclaim_bench(args):
 def growth_bench(args):
     """Bursty KV growth at serving size: Poisson arrivals, one token per sequence per step, blocks
     allocated as sequences grow (local first, then lent), finished sequences freed, the lender taking
-    2-8 GB back every 200 steps and lending it again 100 steps later; on ENOSPC the most recently
-    admitted sequence is preempted. Every step = one append launch (all layers) + one decode launch.
+    2-8 GB back every 200 steps and lending it again 100 steps later. Where the lender's reclaim has
+    no room to migrate into, requests are preempted: by the library (--victims slab: the slab with
+    the fewest requests, slice_reclaim_preempt) or by the driver (--victims lifo: the most recently
+    admitted sequence, then a retry); a sequence that cannot grow preempts the most recently admitted
+    one (cause: out of memory). Preempted requests go back to the head of the queue with what they
+    had generated. --cap-window T (steps) turns on the cap after a preemption (Section 5.3).
+    Every step = one append launch (all layers) + one decode launch.
     KV contents are whatever the arenas hold (random): only shapes and placement matter for timing."""
     import time
     import torch
@@ -164,7 +169,12 @@ def growth_bench(args):
     for a in arrivals:
         by_step.setdefault(a.step, []).append(a)
     waiting, active, length, remaining = [], [], {}, {}
-    next_id = taken = tokens = preempted = enospc = 0
+    next_id = taken = tokens = preempted = enospc = capped = 0
+    assert s.slice_set_preempt_window(args.cap_window) == 0
+
+    def requeue(victim, t):
+        waiting.insert(0, synth.Arrival(t, length[victim], remaining[victim]))
+        del length[victim], remaining[victim]
     alloc_s = 0.0
     reclaims, lent_frac = [], []
     scale = 1.0 / float(np.sqrt(128))
@@ -175,11 +185,13 @@ def growth_bench(args):
     for t in range(args.steps):
         waiting += by_step.get(t, [])
         t_a = time.perf_counter()
+        assert s.slice_set_time(t) == 0
         while waiting and len(active) < max_batch:
             a = waiting[0]
             need = synth.blocks_for(a.prompt_len)
             rc, _ = s.slice_alloc_blocks(next_id, need, B.TIER_AUTO)
-            if rc == B.ENOSPC:               # a failing call changes nothing: the request keeps waiting
+            if rc in (B.ENOSPC, B.ECAPPED):  # a failing call changes nothing: the request keeps waiting
+                capped += rc == B.ECAPPED
                 break
             assert rc == 0, rc
             assert s.slice_set_seq_len(next_id, a.prompt_len) == 0
@@ -191,18 +203,30 @@ def growth_bench(args):
             take = int(rng.uniform(2, 8) * 2**30 / (Lr * BLOCK_BYTES))
             r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             r0.record(main)
-            rc, mig = s.slice_reclaim(take, main)
-            while rc == B.ENOSPC and active:  # no room for the blocks in use up there: preempt and retry
-                victim = active.pop()
-                assert s.slice_free_seq(victim) == 0
-                del length[victim], remaining[victim]
-                preempted += 1
+            h0 = time.perf_counter()
+            n_victims = 0
+            if args.victims == "slab":
+                rc, victims, mig = s.slice_reclaim_preempt(take, args.slab, main)
+                for victim in victims:
+                    active.remove(victim)
+                    requeue(victim, t)
+                n_victims = len(victims)
+            else:
                 rc, mig = s.slice_reclaim(take, main)
+                while rc == B.ENOSPC and active:  # no room for the blocks in use up there: preempt and retry
+                    victim = active.pop()
+                    assert s.slice_preempt_seq(victim, B.PREEMPT_RECLAIM) == 0
+                    requeue(victim, t)
+                    n_victims += 1
+                    rc, mig = s.slice_reclaim(take, main)
+            host_ms = (time.perf_counter() - h0) * 1e3
+            preempted += n_victims
             r1.record(main)
             r1.synchronize()
             if rc == 0:
                 taken = take
-                reclaims.append({"step": t, "take_ids": take, "migrated_ids": int(mig), "ms": round(r0.elapsed_time(r1), 3),
+                reclaims.append({"step": t, "take_ids": take, "migrated_ids": int(mig), "preempted": n_victims,
+                                 "host_ms": round(host_ms, 3), "ms": round(r0.elapsed_time(r1), 3),
                                  "gbs": round(2 * mig * Lr * BLOCK_BYTES / r0.elapsed_time(r1) / 1e6, 1)})
             else:
                 reclaims.append({"step": t, "take_ids": take, "rc": rc})
@@ -216,9 +240,9 @@ def growth_bench(args):
                 while s.slice_alloc_blocks(i, 1, B.TIER_AUTO)[0] != 0:
                     enospc += 1
                     victim = active[-1]
-                    assert s.slice_free_seq(victim) == 0
+                    assert s.slice_preempt_seq(victim, B.PREEMPT_OOM) == 0
                     active.remove(victim)
-                    del length[victim], remaining[victim]
+                    requeue(victim, t)
                     preempted += 1
                     if victim == i:
                         break
@@ -253,7 +277,10 @@ def growth_bench(args):
                       "decoded_tokens": tokens, "tokens_per_s": round(tokens / wall, 1), "wall_s": round(wall, 3),
                       "gpu_stream_s": round(e0.elapsed_time(e1) / 1e3, 3), "sequences_admitted": next_id,
                       "host_allocator_us_per_step": round(alloc_s / args.steps * 1e6, 1),
-                      "enospc": enospc, "preempted": preempted, "reclaims": reclaims, "lent_fraction_every_50_steps": lent_frac,
+                      "victims": args.victims, "slab_blocks": args.slab, "cap_window_steps": args.cap_window,
+                      "enospc": enospc, "capped_admissions": capped, "preempted": preempted,
+                      "preempted_by_cause": {k: v for k, v in s.slice_preempt_stats().items() if k.startswith("preempt_")},
+                      "reclaims": reclaims, "lent_fraction_every_50_steps": lent_frac,
                       "device_status": st["device_status"], "plans_built": st.get("plans_built")}), flush=True)
     s.slice_destroy()
 
@@ -339,6 +366,9 @@ def main():
     ap.add_argument("--blocks", type=int, nargs="*", default=[1_000, 10_000, 100_000, 400_000])
     ap.add_argument("--ctas", type=int, nargs="*", default=[0, 148, 592])
     ap.add_argument("--take", type=int, nargs="*", default=[954, 3815])
+    ap.add_argument("--victims", choices=["slab", "lifo"], default="slab")
+    ap.add_argument("--slab", type=int, default=10, help="blocks per slab for the victim rule (the paper's default)")
+    ap.add_argument("--cap-window", type=int, default=0, help="steps a cap holds after a preemption by reclamation")
     args = ap.parse_args()
     from paper_2609_27040_b200 import binding as B
     B.lib()                                    # fails loudly when the CUDA library is missing

@@ -1,5 +1,5 @@
 """Random interleavings of the public calls against the oracle: sequences come and go, grow, the
-lender takes and gives, and attention is asked for through every entry point (whole pass in one
+lender takes and gives (with and without preempting requests), and attention is asked for through every entry point (whole pass in one
 launch, per-layer prefetch + decode, write-back in between) on whatever state the earlier calls
 left. Return codes must agree with the oracle's state machine; every attention result and, at the
 end, every arena byte must agree with the oracle."""
@@ -38,7 +38,7 @@ def test_random_call_sequences_match_the_oracle(seed, mode):
                 static_split=int(seed % 2))
     main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
     scale = 1.0 / float(np.sqrt(D))
-    active, next_id, taken, attended = [], 0, 0, 0
+    active, next_id, taken, attended, preempted = [], 0, 0, 0, 0
 
     def tables_equal():
         for i in active:
@@ -63,7 +63,7 @@ def test_random_call_sequences_match_the_oracle(seed, mode):
 
     for step in range(90):
         op = rng.choice(["arrive", "grow", "free", "reclaim", "lend", "pass", "layers", "writeback"],
-                        p=[0.14, 0.22, 0.06, 0.06, 0.06, 0.22, 0.18, 0.06])
+                        p=[0.14, 0.22, 0.05, 0.09, 0.06, 0.22, 0.17, 0.05])
         if op == "arrive" and len(active) < MAXSEQ:
             n = int(rng.integers(1, 90))
             need = synth.blocks_for(n)
@@ -114,6 +114,14 @@ def test_random_call_sequences_match_the_oracle(seed, mode):
         elif op == "free" and active:
             i = active.pop(int(rng.integers(len(active))))
             assert s.slice_free_seq(i) == orc.free_seq(i) == 0
+        elif op == "reclaim" and rng.random() < 0.5:
+            take, slab = int(rng.integers(1, 16)), int(rng.integers(1, 6))
+            rc, victims, mig = orc.reclaim_preempt(take, slab, local, lent)      # evicts where there is no room
+            rc2, victims2, mig2 = s.slice_reclaim_preempt(take, slab, main)
+            assert rc == rc2 == 0 and victims == victims2 and mig == mig2
+            active = [i for i in active if i not in victims]
+            preempted += len(victims)
+            taken = LENT - orc.lent_capacity
         elif op == "reclaim":
             take = int(rng.integers(1, 10))
             rc, mig = orc.reclaim(take, local, lent)
@@ -156,6 +164,7 @@ def test_random_call_sequences_match_the_oracle(seed, mode):
         tables_equal()
         st = s.slice_stats()
         assert st["device_status"] == 0 and st["last_cuda_error"] == 0 and st["lent_capacity"] == orc.lent_capacity
+        assert s.slice_preempt_stats()["preempt_reclaim"] == orc.preempt_state()["preempt_reclaim"] == preempted
     torch.cuda.synchronize()
     assert attended >= 5
     assert (kv_to_host(g_local) == local).all() and (kv_to_host(g_lent) == lent).all()

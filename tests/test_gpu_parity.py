@@ -361,6 +361,53 @@ def test_reclaim_without_room_changes_nothing():
     _check_layer(sc, g, 0)
 
 
+@pytest.mark.parametrize("slab,window", [(1, 0), (4, 50), (10, 50)])
+def test_reclaim_by_preemption_matches_oracle_and_survivors_keep_their_bytes(slab, window):
+    """No free block anywhere: the lender's reclaim has to evict. The library and the oracle must
+    name the same victims in the same order, migrate the same blocks to the same places bit for
+    bit, count the same preemptions and set the same cap; attention over the survivors is right."""
+    wl = synth.Workload("full_gqa", 2, 32, 8, 6, 40, 200, 0.5)
+    sc = Scenario(wl, 2, slack=0)
+    g = _gpu(sc)
+    from tests.gpu_helpers import kv_to_host
+    assert g.s.slice_set_preempt_window(window) == sc.orc.set_preempt_window(window) == 0
+    assert g.s.slice_set_time(7) == sc.orc.set_time(7) == 0
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer)
+    take = sc.orc.lent_capacity // 2
+    assert g.s.slice_reclaim(take, g.main)[0] == B.ENOSPC
+    rc, victims, mig = sc.orc.reclaim_preempt(take, slab, sc.local, sc.lent)
+    rc2, victims2, mig2 = g.s.slice_reclaim_preempt(take, slab, g.main)
+    assert rc == rc2 == 0 and victims == victims2 and len(victims) > 0 and mig == mig2
+    torch.cuda.synchronize()
+    assert g.s.slice_preempt_stats() == sc.orc.preempt_state()
+    survivors = [i for i in sc.seq_ids if i not in victims]
+    assert survivors
+    for i in victims:
+        assert g.s.slice_get_block_table(i)[0] == B.ESTATE
+    local_gpu, lent_gpu = kv_to_host(g.local), kv_to_host(g.lent)
+    for i in survivors:
+        rc, t, ln = g.s.slice_get_block_table(i)
+        rc2, t2, ln2 = sc.orc.block_table(i)
+        assert rc == rc2 == 0 and ln == ln2 and t.tolist() == t2.tolist()
+        for l in range(sc.L):
+            for e in t2.tolist():
+                a = local_gpu[l, e] if e >= 0 else lent_gpu[l, ~e]
+                b = sc.local[l, e] if e >= 0 else sc.lent[l, ~e]
+                assert (a == b).all()
+    assert g.s.slice_get_free_stack(B.TIER_LOCAL).tolist() == sc.orc.free_stack(1).tolist()
+    assert g.s.slice_get_free_stack(B.TIER_LENT).tolist() == sc.orc.free_stack(2).tolist()
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer, seqs=survivors)
+    if window:                                                      # the user was above its share: capped
+        held = g.s.slice_stats()
+        assert g.s.slice_preempt_stats()["cap_level"] == held["local_used"] + held["lent_used"]
+        assert g.s.slice_alloc_blocks(victims[0], 1, B.TIER_AUTO)[0] == B.ECAPPED == sc.orc.alloc_blocks(victims[0], 1, oracle.AUTO)[0]
+        assert g.s.slice_set_time(57) == sc.orc.set_time(57) == 0
+        rc = g.s.slice_alloc_blocks(victims[0], 1, B.TIER_AUTO)[0]
+        assert rc == sc.orc.alloc_blocks(victims[0], 1, oracle.AUTO)[0] and rc != B.ECAPPED      # lifted
+
+
 def test_append_kv_writes_home_and_staged_copy():
     wl = synth.Workload("app", 2, 32, 8, 4, 17, 90, 0.5)
     sc = Scenario(wl, 5, slack=8)

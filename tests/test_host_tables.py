@@ -206,3 +206,78 @@ def test_decode_step_plans_prefetches_for_any_ring_depth(ring, calls):
             assert s.slice_decode_step(seqs, None, 16, 0.1, None, False, True, None, None) == B.OK
         assert s.slice_stats()["prefetch_calls"] == calls
         s.slice_destroy()
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_preemption_calls_match_oracle_state_machine(seed):
+    """Reclaim by preemption, engine-chosen preemptions, the clock and the cap: return codes, the
+    victims and their order, tables, free lists and the counters agree with the oracle over random
+    call sequences in which the lender's demand comes and goes."""
+    rng = np.random.default_rng(100 + seed)
+    LB, RB, PH, CAP = 10, 18, 24, 24
+    lo, ro = synth.free_order(rng, LB), synth.free_order(rng, PH)
+    s = _null_slice(2, 8, LB, RB, PH, CAP, 10, 9, lo, ro)
+    o = oracle.OracleSlice(2, 16, 65536, LB, RB, PH, 2, CAP, max_seqs=10, max_blocks_per_seq=9,
+                           local_free_order=lo, lent_free_order=ro)
+    window = int(rng.choice([0, 5, 40]))
+    assert s.slice_set_preempt_window(window) == o.set_preempt_window(window) == 0
+    live, now, evictions, capped = set(), 0, 0, 0
+    for step in range(3000):
+        op = int(rng.integers(0, 14))
+        if op < 6:
+            q, n, hint = int(rng.integers(0, 12)), int(rng.integers(0, 5)), int(rng.integers(0, 3))
+            rc1, e1 = s.slice_alloc_blocks(q, n, hint)
+            rc2, e2 = o.alloc_blocks(q, n, hint)
+            assert rc1 == rc2
+            capped += rc1 == B.ECAPPED
+            if rc1 == 0:
+                assert e1.tolist() == e2.tolist()
+                live.add(q)
+        elif op == 6:
+            q = int(rng.integers(0, 12))
+            assert s.slice_free_seq(q) == o.free_seq(q)
+            live.discard(q)
+        elif op == 7:
+            q, cause = int(rng.integers(0, 12)), int(rng.integers(0, 4))
+            rc1, rc2 = s.slice_preempt_seq(q, cause), o.preempt_seq(q, cause)
+            assert rc1 == rc2
+            if rc1 == 0:
+                live.discard(q)
+        elif op in (8, 9):
+            take, slab = int(rng.integers(0, 9)), int(rng.integers(0, 6))
+            cap = None if rng.random() < 0.8 else int(rng.integers(0, 3))
+            rc1, v1, m1 = s.slice_reclaim_preempt(take, slab, max_victims=cap)
+            rc2, v2, m2 = o.reclaim_preempt(take, slab, None, None, max_victims=cap)
+            assert rc1 == rc2 and v1 == v2 and (rc1 != 0 or m1 == m2), (rc1, rc2, v1, v2)
+            if rc1 == 0:
+                live -= set(v1)
+                evictions += len(v1)
+        elif op == 10:
+            take = int(rng.integers(0, 6))
+            rc1, m1 = s.slice_reclaim(take)
+            rc2, m2 = o.reclaim(take, None, None)
+            assert rc1 == rc2 and (rc1 != 0 or m1 == m2)
+        elif op == 11:
+            n = int(rng.integers(0, 6))
+            assert s.slice_lend(n) == o.lend(n)
+        elif op == 12:
+            now += int(rng.integers(0, 8))
+            assert s.slice_set_time(now) == o.set_time(now) == 0
+        else:
+            back = max(now - 1, 0)
+            assert s.slice_set_time(back) == o.set_time(back)          # refused unless equal
+        _same_state(s, o, live)
+        assert s.slice_preempt_stats() == o.preempt_state()
+    assert evictions > 0 and (window == 0 or capped > 0)
+    s.close()
+
+
+def test_preemption_bad_arguments():
+    s = _null_slice(2, 8, 4, 4, 4, 4, 4, 8)
+    assert s.slice_reclaim_preempt(2, 0)[0] == B.EINVAL
+    assert s.slice_preempt_seq(0, B.PREEMPT_OOM) == B.ESTATE
+    assert s.slice_alloc_blocks(0, 1, B.TIER_LENT)[0] == B.OK
+    assert s.slice_preempt_seq(0, 0) == B.EINVAL and s.slice_preempt_seq(0, 3) == B.EINVAL
+    assert s.slice_set_time(5) == B.OK and s.slice_set_time(4) == B.EINVAL
+    assert B.slice_strerror(B.ECAPPED).startswith("a cap")
+    s.close()
