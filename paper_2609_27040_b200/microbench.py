@@ -285,6 +285,45 @@ def growth_bench(args):
     s.slice_destroy()
 
 
+def transfer_size_sweep(args):
+    """Effective bandwidth of a gather against the size of its contiguous pieces (Section 4.2: small
+    fragments lower the effective bandwidth B, hence slabs and layer groups: pieces of S..mS, kS or
+    kS..mkS bytes). The same total is gathered as n scattered pieces of c bytes each, for c from 4 KB
+    to 16 MB (64 KB = one KV block of one layer; 640 KB = a slab of 10; 2.5 MB = a slab of 10 times a
+    group of 4 layers), out of an arena twice as large, over both links: HBM to HBM and pinned host
+    memory to HBM."""
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    stream = torch.cuda.Stream()
+    flush = torch.zeros(160 << 20, dtype=torch.uint8, device="cuda")
+    sizes = [4 << 10, 16 << 10, 64 << 10, 256 << 10, 640 << 10, 2560 << 10, 16 << 20]
+    for link, total in (("hbm", 1 << 30), ("pinned_host", 256 << 20)):
+        arena = torch.empty(2 * total // 2, dtype=torch.int16, device="cuda" if link == "hbm" else "cpu")
+        arena.random_(-30000, 30000)
+        if link != "hbm":
+            arena = arena.pin_memory()
+        dst = torch.zeros(total // 2, dtype=torch.int16, device="cuda")
+        for c in sizes:
+            n = total // c
+            rng = np.random.default_rng(c)
+            idx = torch.from_numpy(rng.permutation(2 * total // c)[:n].astype(np.int32)).cuda()
+            pos = torch.arange(n, dtype=torch.int32, device="cuda")
+            for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk")):
+                for ctas in ((0,) if link == "hbm" else (8, 0)):
+                    def run():
+                        assert B.slice_copy_blocks(dst, pos, arena, idx, n, c, kind, ctas, stream) == 0
+                    us = _time_us(run, stream, 10 if link == "hbm" else 3, flush)
+                    ok = None
+                    if c >= 64 << 10:
+                        got = dst[: n * c // 2].view(n, c // 2)
+                        want = arena[: (2 * total // c) * c // 2].view(-1, c // 2).index_select(0, idx.long().to(arena.device))
+                        ok = bool(torch.equal(got.cpu() if link != "hbm" else got, want))
+                    print(json.dumps({"case": "transfer_size", "link": link, "kernel": name, "ctas": ctas or "default",
+                                      "piece_bytes": c, "pieces": n, "us": round(us, 1),
+                                      "gbs_read": round(n * c / us / 1e3, 1), "matches_index_select": ok}), flush=True)
+        del arena, dst
+
+
 def link_bench(args):
     """The paper's transparency condition (Section 2.3 / 4: a transfer of m bytes over a link of
     bandwidth B is hidden when it fits in the latency window L between two uses, B*L >= m) with a
@@ -358,7 +397,7 @@ def link_bench(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "all"], default="all")
+    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "size", "all"], default="all")
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--arena-gb", type=float, default=48.0)
     ap.add_argument("--seed", type=int, default=0)
@@ -380,6 +419,8 @@ def main():
         growth_bench(args)
     if args.what == "link":
         link_bench(args)
+    if args.what == "size":
+        transfer_size_sweep(args)
 
 
 if __name__ == "__main__":
