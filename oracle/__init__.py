@@ -250,3 +250,19 @@ def to_bf16(x: np.ndarray) -> np.ndarray:
     y = np.zeros(x.shape, np.uint16)
     lib().oracle_to_bf16(_ptr(x), _ptr(y), x.size)
     return y
+
+
+# -- scheduling across slices (O-schedule) --------------------------------------------------------
+def gll_choose(own_blocks: Sequence[int], peer_blocks: Sequence[int], capacity_blocks: Sequence[int]) -> int:
+    """Section 5.2 / Appendix C, Greedy-Least-Loaded: a request goes to the incident slice k with the
+    smallest util_{k,i} + util_{k,j}, each utilisation being blocks held over the slice's capacity.
+    Exact rational arithmetic; among equals the first slice. Returns -1 for an empty list."""
+    from fractions import Fraction
+    best, best_u = -1, None
+    for k, (a, b, c) in enumerate(zip(own_blocks, peer_blocks, capacity_blocks)):
+        if c <= 0:
+            raise ValueError("slice without capacity")
+        u = Fraction(int(a), int(c)) + Fraction(int(b), int(c))
+        if best_u is None or u < best_u:
+            best, best_u = k, u
+    return best

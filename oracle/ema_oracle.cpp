@@ -28,6 +28,9 @@
 //                 of active requests" (Section 4.2.1); after a preemption above the static share
 //                 the user's allocations are capped for a window T (Section 5.3, bursty workload
 //                 preemption control); preemptions are counted by cause (Section 6.6).
+//   * O-schedule — the choice among several slices (Section 5.2, Greedy-Least-Loaded) is stated in
+//                 the Python front end (gll_choose, exact rationals); pins in
+//                 tests/test_oracle_schedule.py.
 //
 // Parity pins (tests/test_oracle_*.py): paged == dense brute force; softmax row sums; closed
 // forms (n=1, equal keys, constant V, dominant key, score shift, token permutation); fp64
