@@ -274,6 +274,20 @@ typedef struct {
 } slice_preempt_stats_t;
 int slice_preempt_stats(slice_t* s, slice_preempt_stats_t* out);
 
+/* Section 5.2: a process with several slices (one per peer, Section 5.1) sends each request to the
+ * slice k with the smallest util_{k,i} + util_{k,j} (Greedy-Least-Loaded; Appendix C bounds its peak
+ * utilisation by (m + 3) / 2 times the offline optimum for m GPUs). A slice's capacity is all its
+ * block ids, local part plus the peer's whole arena; util_{k,i} = blocks this user holds / capacity;
+ * util_{k,j} = blocks the peer itself holds / capacity, which only the peer knows: its side reports
+ * the number with slice_set_peer_used (0 until then). Errors: EINVAL (more than the peer's arena). */
+int slice_set_peer_used(slice_t* s, uint32_t peer_blocks);
+
+/* Picks among slices[0..n) (host array of handles) by the rule above, compared exactly (as
+ * fractions, not in floating point); among equals the first. out_index (host) receives the choice.
+ * Nothing is allocated: the caller then calls slice_alloc_blocks on that slice. Errors: EINVAL
+ * (n == 0, NULL handle). */
+int slice_schedule_gll(slice_t* const* slices, uint32_t n, uint32_t* out_index);
+
 /* The lender offers n more block ids (the share of a slice is renegotiated at run time,
  * Section 1 / 4.1). New ids are handed out in ascending order. Errors: EINVAL (beyond arena). */
 int slice_lend(slice_t* s, uint32_t n_blocks);

@@ -29,6 +29,7 @@ EXPORTS = [
     "slice_lend", "slice_append_kv", "slice_writeback_layer", "slice_decode_step", "slice_stats",
     "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc", "slice_cta_trace",
     "slice_reclaim_preempt", "slice_preempt_seq", "slice_set_preempt_window", "slice_set_time", "slice_preempt_stats",
+    "slice_set_peer_used", "slice_schedule_gll",
 ]
 
 
@@ -103,6 +104,8 @@ def lib() -> C.CDLL:
         L.slice_set_preempt_window.argtypes = [vp, C.c_uint64]
         L.slice_set_time.argtypes = [vp, C.c_uint64]
         L.slice_preempt_stats.argtypes = [vp, vp]
+        L.slice_set_peer_used.argtypes = [vp, u32]
+        L.slice_schedule_gll.argtypes = [vp, u32, vp]
         L.slice_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, vp]
         L.slice_writeback_layer.argtypes = [vp, u32, vp, u32, vp]
         L.slice_decode_step.argtypes = [vp, vp, u32, vp, u32, C.c_float, vp, i32, i32, vp, vp]
@@ -297,6 +300,9 @@ class Slice:
     def slice_set_time(self, now: int) -> int:
         return lib().slice_set_time(self._h, now)
 
+    def slice_set_peer_used(self, peer_blocks: int) -> int:
+        return lib().slice_set_peer_used(self._h, peer_blocks)
+
     def slice_preempt_stats(self) -> dict:
         st = SlicePreemptStats()
         rc = lib().slice_preempt_stats(self._h, C.byref(st))
@@ -362,3 +368,13 @@ def slice_copy_blocks(dst, dst_idx, src, src_idx, n: int, block_bytes: int, kind
                       stream=None) -> int:
     return lib().slice_copy_blocks(_ptr(dst), _ptr(dst_idx), _ptr(src), _ptr(src_idx), n, block_bytes, kind,
                                    ctas, _stream(stream))
+
+
+def slice_schedule_gll(slices) -> int:
+    """Index of the slice a new request goes to (Greedy-Least-Loaded over Slice objects)."""
+    arr = (C.c_void_p * len(slices))(*[sl._h for sl in slices])
+    out = C.c_uint32(0)
+    rc = lib().slice_schedule_gll(arr, len(slices), C.byref(out))
+    if rc != OK:
+        raise SliceError(rc, "slice_schedule_gll")
+    return int(out.value)

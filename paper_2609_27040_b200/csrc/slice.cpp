@@ -102,6 +102,7 @@ struct ema_slice {
   uint64_t now = 0, preempt_window = 0, cap_until = 0;
   uint32_t cap_level = 0;
   uint64_t preempt_oom = 0, preempt_reclaim = 0;
+  uint32_t peer_used = 0;  // blocks the peer holds in this slice, as last reported
   // plans and slots
   Plan plans[kNumPlans];
   int next_plan = 0;
@@ -1238,6 +1239,33 @@ int slice_preempt_stats(slice_t* s, slice_preempt_stats_t* out) {
   out->window = s->preempt_window;
   out->cap_until = cap_in_force(s) ? s->cap_until : 0;
   out->cap_level = cap_in_force(s) ? s->cap_level : 0;
+  return SLICE_OK;
+}
+
+int slice_set_peer_used(slice_t* s, uint32_t peer_blocks) {
+  if (!s || peer_blocks > s->cfg.lent_blocks_physical) return SLICE_EINVAL;
+  s->peer_used = peer_blocks;
+  return SLICE_OK;
+}
+
+int slice_schedule_gll(slice_t* const* slices, uint32_t n, uint32_t* out_index) {
+  if (!slices || !out_index || n == 0) return SLICE_EINVAL;
+  for (uint32_t k = 0; k < n; ++k)
+    if (!slices[k]) return SLICE_EINVAL;
+  // used_k / cap_k compared by cross-multiplication: both factors are below 2^33.
+  uint32_t best = 0;
+  uint64_t best_used = 0, best_cap = 1;
+  for (uint32_t k = 0; k < n; ++k) {
+    const ema_slice* s = slices[k];
+    const uint64_t used = static_cast<uint64_t>(blocks_held(s)) + s->peer_used;
+    const uint64_t cap = static_cast<uint64_t>(s->cfg.local_blocks) + s->cfg.lent_blocks_physical;
+    if (k == 0 || used * best_cap < best_used * cap) {
+      best = k;
+      best_used = used;
+      best_cap = cap;
+    }
+  }
+  *out_index = best;
   return SLICE_OK;
 }
 

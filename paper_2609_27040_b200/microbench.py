@@ -324,6 +324,134 @@ def transfer_size_sweep(args):
         del arena, dst
 
 
+def multislice_bench(args):
+    """One compute process with several slices (Section 5: one per peer) at serving size. Every
+    slice has a local half and a half in its peer's memory; each peer's own use of its half follows
+    a square wave with its own period (busy: it takes memory back, reclaim by preemption; idle: it
+    lends again) and is reported to the slice. Arriving requests are sent to a slice by --policy:
+    gll (Section 5.2, smallest combined utilisation), random, or round_robin; a request whose slice
+    has no room waits. Sequences grow on their slice; one that cannot grow preempts the most recently
+    admitted one of the same slice. Every step = per slice with work one append launch and one
+    decode launch. Reports tokens/s and the preemptions by cause, summed over the slices."""
+    import time
+    import torch
+    from paper_2609_27040_b200 import binding as B, synth
+    Lr, Hq, Hkv, max_batch, ns = 32, 32, 8, 256, args.slices
+    ids = int(args.arena_gb * 2**30 / (Lr * BLOCK_BYTES)) // ns
+    half = ids // 2
+    shape = (2, 16, Hkv, 128)
+    max_blocks = (2048 + 8192) // 16 + 2
+    slices, keep = [], []
+    for k in range(ns):
+        local = torch.empty((Lr, half) + shape, dtype=torch.bfloat16, device="cuda")
+        lent = torch.empty((Lr, half) + shape, dtype=torch.bfloat16, device="cuda")
+        for l in range(Lr):
+            local[l].normal_()
+            lent[l].normal_()
+        staging = torch.zeros((2, half) + shape, dtype=torch.bfloat16, device="cuda")
+        keep.append((local, lent, staging))
+        slices.append(B.Slice(Lr, Hkv, half, half, half, local=local, lent=lent, staging=staging, max_seqs=max_batch,
+                              max_blocks_per_seq=max_blocks))
+    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    q = torch.empty((Lr, max_batch, Hq, 128), dtype=torch.bfloat16, device="cuda").normal_()
+    out = torch.zeros_like(q)
+    knew = torch.empty((Lr, max_batch, Hkv, 128), dtype=torch.bfloat16, device="cuda").normal_()
+    rng = np.random.default_rng(args.seed)
+    by_step = {}
+    for a in synth.bursty_arrivals(args.seed, args.steps, rate=args.rate):
+        by_step.setdefault(a.step, []).append(a)
+    period = [240 + 90 * k for k in range(ns)]                 # peers are busy at different times
+    busy_frac = [0.9, 0.6, 0.75, 0.5, 0.8, 0.7, 0.65, 0.85][:ns]
+    peer_used = [int(0.1 * half)] * ns
+    for k in range(ns):                                          # what the peer uses it does not lend
+        assert slices[k].slice_reclaim(peer_used[k], main)[0] == 0
+        assert slices[k].slice_set_peer_used(peer_used[k]) == 0
+    waiting, active, home, length, remaining = [], [[] for _ in range(ns)], {}, {}, {}
+    next_id = tokens = enospc = waits = rr = 0
+    scale = 1.0 / float(np.sqrt(128))
+
+    def requeue(victim, t):
+        waiting.insert(0, synth.Arrival(t, length[victim], remaining[victim]))
+        active[home[victim]].remove(victim)
+        del length[victim], remaining[victim], home[victim]
+
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    for t in range(args.steps):
+        waiting += by_step.get(t, [])
+        for k in range(ns):                                      # the peers' own demand
+            want = int((busy_frac[k] if (t // period[k]) % 2 == 1 else 0.1) * half)
+            if want > peer_used[k]:
+                rc, victims, _ = slices[k].slice_reclaim_preempt(want - peer_used[k], args.slab, main)
+                assert rc == 0, rc
+                for v in victims:
+                    requeue(v, t)
+            elif want < peer_used[k]:
+                assert slices[k].slice_lend(peer_used[k] - want) == 0
+            peer_used[k] = want
+            assert slices[k].slice_set_peer_used(want) == 0
+        while waiting and sum(len(a) for a in active) < max_batch:
+            a = waiting[0]
+            if args.policy == "gll":
+                k = B.slice_schedule_gll(slices)
+            elif args.policy == "random":
+                k = int(rng.integers(ns))
+            else:
+                k, rr = rr % ns, rr + 1
+            rc, _ = slices[k].slice_alloc_blocks(next_id, synth.blocks_for(a.prompt_len), B.TIER_AUTO)
+            if rc != 0:
+                waits += 1
+                break
+            assert slices[k].slice_set_seq_len(next_id, a.prompt_len) == 0
+            waiting.pop(0)
+            active[k].append(next_id)
+            home[next_id], length[next_id], remaining[next_id] = k, a.prompt_len, a.output_len
+            next_id += 1
+        for k in range(ns):
+            for i in list(active[k]):
+                if i not in length:
+                    continue
+                if length[i] % 16 == 0:
+                    while slices[k].slice_alloc_blocks(i, 1, B.TIER_AUTO)[0] != 0:
+                        enospc += 1
+                        victim = active[k][-1]
+                        assert slices[k].slice_preempt_seq(victim, B.PREEMPT_OOM) == 0
+                        requeue(victim, t)
+                        if victim == i:
+                            break
+                    if i not in length:
+                        continue
+                length[i] += 1
+                assert slices[k].slice_set_seq_len(i, length[i]) == 0
+            n = len(active[k])
+            if not n:
+                continue
+            seqs = np.array(active[k], np.int32)
+            kn = knew if n == max_batch else knew[:, :n].contiguous()
+            assert slices[k].slice_append_kv(B.ALL_LAYERS, seqs, kn, kn, main) == 0
+            assert slices[k].slice_decode_step(seqs, q if n == max_batch else q[:, :n].contiguous(), Hq, scale,
+                                               out if n == max_batch else out[:, :n].contiguous(), False, True, main, side) == 0
+            tokens += n
+            for i in list(active[k]):
+                remaining[i] -= 1
+                if remaining[i] <= 0:
+                    assert slices[k].slice_free_seq(i) == 0
+                    active[k].remove(i)
+                    del length[i], remaining[i], home[i]
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    ps = [sl.slice_preempt_stats() for sl in slices]
+    st = [sl.slice_stats() for sl in slices]
+    print(json.dumps({"case": "multislice", "policy": args.policy, "arrivals_per_step": args.rate, "slices": ns, "steps": args.steps, "arena_gb": args.arena_gb,
+                      "block_ids_per_slice": ids, "decoded_tokens": tokens, "tokens_per_s": round(tokens / wall, 1),
+                      "wall_s": round(wall, 3), "sequences_admitted": next_id, "admission_waits": waits,
+                      "preempt_oom": sum(p["preempt_oom"] for p in ps), "preempt_reclaim": sum(p["preempt_reclaim"] for p in ps),
+                      "migrated_blocks": sum(x["migrated_blocks"] for x in st),
+                      "device_status": [x["device_status"] for x in st]}), flush=True)
+    for sl in slices:
+        sl.slice_destroy()
+
+
 def link_bench(args):
     """The paper's transparency condition (Section 2.3 / 4: a transfer of m bytes over a link of
     bandwidth B is hidden when it fits in the latency window L between two uses, B*L >= m) with a
@@ -397,7 +525,7 @@ def link_bench(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "size", "all"], default="all")
+    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "size", "multislice", "all"], default="all")
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--arena-gb", type=float, default=48.0)
     ap.add_argument("--seed", type=int, default=0)
@@ -407,6 +535,9 @@ def main():
     ap.add_argument("--take", type=int, nargs="*", default=[954, 3815])
     ap.add_argument("--victims", choices=["slab", "lifo"], default="slab")
     ap.add_argument("--slab", type=int, default=10, help="blocks per slab for the victim rule (the paper's default)")
+    ap.add_argument("--slices", type=int, default=3, help="multislice: slices of the one compute process (at most 8)")
+    ap.add_argument("--rate", type=float, default=0.5, help="multislice: mean arrivals per step (Poisson)")
+    ap.add_argument("--policy", choices=["gll", "random", "round_robin"], default="gll")
     ap.add_argument("--cap-window", type=int, default=0, help="steps a cap holds after a preemption by reclamation")
     args = ap.parse_args()
     from paper_2609_27040_b200 import binding as B
@@ -421,6 +552,8 @@ def main():
         link_bench(args)
     if args.what == "size":
         transfer_size_sweep(args)
+    if args.what == "multislice":
+        multislice_bench(args)
 
 
 if __name__ == "__main__":

@@ -281,3 +281,44 @@ def test_preemption_bad_arguments():
     assert s.slice_set_time(5) == B.OK and s.slice_set_time(4) == B.EINVAL
     assert B.slice_strerror(B.ECAPPED).startswith("a cap")
     s.close()
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_slice_choice_matches_oracle(seed):
+    """Greedy-Least-Loaded over several slices of different sizes, with requests coming and going
+    and the peers' own use changing: the library picks the slice the oracle picks, ties included."""
+    rng = np.random.default_rng(seed)
+    shapes = [(8, 8), (8, 8), (6, 10), (16, 16)]                    # (local, lent): equal and unequal capacities
+    slices = [_null_slice(1, 8, lb, rb, rb, rb, 64, 8) for lb, rb in shapes]
+    cap = [lb + rb for lb, rb in shapes]
+    own, peer, homes, next_id, ties = [0] * 4, [0] * 4, {}, 0, 0
+    for step in range(1500):
+        op = int(rng.integers(0, 4))
+        if op < 2:
+            k = B.slice_schedule_gll(slices)
+            assert k == oracle.gll_choose(own, peer, cap)
+            from fractions import Fraction
+            u = [Fraction(own[i] + peer[i], cap[i]) for i in range(4)]
+            ties += sum(x == min(u) for x in u) > 1
+            n = int(rng.integers(1, 3))
+            if slices[k].slice_alloc_blocks(next_id, n, B.TIER_AUTO)[0] == B.OK:
+                own[k] += n
+                homes[next_id] = (k, n)
+                next_id += 1
+        elif op == 2 and homes:
+            q = int(rng.choice(sorted(homes)))
+            k, n = homes.pop(q)
+            assert slices[k].slice_free_seq(q) == B.OK
+            own[k] -= n
+        else:
+            k = int(rng.integers(0, 4))
+            used = int(rng.integers(0, shapes[k][1] + 2))
+            rc = slices[k].slice_set_peer_used(used)
+            assert rc == (B.OK if used <= shapes[k][1] else B.EINVAL)
+            if rc == B.OK:
+                peer[k] = used
+    assert ties > 20
+    with pytest.raises(B.SliceError):
+        B.slice_schedule_gll([])
+    for sl in slices:
+        sl.close()
