@@ -408,6 +408,52 @@ def test_reclaim_by_preemption_matches_oracle_and_survivors_keep_their_bytes(sla
         assert rc == sc.orc.alloc_blocks(victims[0], 1, oracle.AUTO)[0] and rc != B.ECAPPED      # lifted
 
 
+def test_three_slices_one_process_choice_and_decode():
+    """Several slices on one GPU (one per peer): the library's Greedy-Least-Loaded choice equals the
+    oracle's as the peers report their use and requests leave; every slice decodes its own part of
+    the batch in one launch per pass, each against its own oracle state."""
+    wls = [synth.Workload("s0", 2, 32, 8, 5, 30, 150, 0.5), synth.Workload("s1", 2, 32, 8, 3, 60, 200, 0.3),
+           synth.Workload("s2", 2, 32, 8, 6, 17, 90, 0.7)]
+    scs = [Scenario(wl, 20 + k, slack=24) for k, wl in enumerate(wls)]
+    gs = [_gpu(sc) for sc in scs]
+    cap = [sc.pl.local_blocks + sc.lent_phys for sc in scs]
+    peer = [0, 0, 0]
+
+    def held(sc):
+        return sum(len(sc.orc.block_table(i)[1]) for i in sc.seq_ids)
+
+    rng = np.random.default_rng(5)
+    for step in range(12):
+        own = [held(sc) for sc in scs]
+        k = B.slice_schedule_gll([g.s for g in gs])
+        assert k == oracle.gll_choose(own, peer, cap)
+        j = int(rng.integers(3))
+        if step % 3 == 2 and len(scs[j].seq_ids) > 1:              # a request of slice j finishes
+            i = scs[j].seq_ids.pop()
+            assert gs[j].s.slice_free_seq(i) == scs[j].orc.free_seq(i) == 0
+        else:                                                       # peer j reports another use of its half
+            peer[j] = int(rng.integers(0, scs[j].lent_phys + 1))
+            assert gs[j].s.slice_set_peer_used(peer[j]) == B.OK
+    for sc, g in zip(scs, gs):
+        g.tables_equal_oracle()
+        pos = [sc.pl.seq_ids.index(i) for i in sc.seq_ids]
+        q = g.q[:, pos].contiguous()
+        out = torch.zeros_like(q)
+        assert g.s.slice_decode_step(sc.seq_ids, q, sc.Hq, float(sc.sm_scale), out, False, True, g.main, g.side) == B.OK
+        torch.cuda.synchronize()
+        g.device_ok()
+        got = _bf16_to_f64(out)
+        lens = np.asarray([int(sc.pl.lengths[i]) for i in sc.seq_ids], np.uint32)
+        for layer in range(sc.L):
+            rc, resolved, _ = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+            assert rc == oracle.OK
+            rc, ref, _ = oracle.paged_attention(sc.q[layer][pos], sc.local[layer], sc.staging[layer % sc.wl.ring_slots],
+                                                resolved, lens, sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+            assert rc == oracle.OK
+            ok, max_abs, max_rel = attention_close(got[layer], ref, ATOL, RTOL)
+            assert ok, (layer, max_abs, max_rel)
+
+
 def test_append_kv_writes_home_and_staged_copy():
     wl = synth.Workload("app", 2, 32, 8, 4, 17, 90, 0.5)
     sc = Scenario(wl, 5, slack=8)
