@@ -207,7 +207,7 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
  * library until the process exits. It calls no cudaMalloc, cudaFree or other allocating routine.
  *   Limit: this entry point splits the work statically (no stealing between CTAs), which needs one
  *   partial slot per (sequence, CTA range it touches) plus one per sequence, i.e. at most
- *   2 * nseq + CTAs slots; slots * num_q_heads * 528 bytes plus about 4 bytes per (sequence, KV head)
+ *   2 * nseq + CTAs slots; slots * num_q_heads * 528 bytes plus about 8 bytes per (sequence, KV head)
  *   and 8 per CTA must fit in 8 MiB; larger requests return SLICE_ESCRATCH
  *   and change nothing.
  *   First call on a device: looks up the array's device address (one-time set-up for that device,

@@ -37,17 +37,24 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
 
 // Device counters of ONE layer inside a layer-kernel launch; the whole block must be zero when the
 // kernel starts. Layout in uint32 words:
-//   [0, 16)                 launch words: [1] next copy unit of the gather issued during this layer,
-//                           [2] attention work finished (blocks x KV heads), [4] merges finished
-//   [16, 16 + 2*ncta)       one 64-bit claim word per CTA range: blocks claimed from the front (low
+//   [0, 32)                 launch words: [1] next copy unit of the gather issued during this layer,
+//                           [2] attention work finished (blocks x KV heads); in a cache line of
+//                           their own, which idle merge warps poll, [16] merge requests published,
+//                           [17] merge requests taken, [18] query heads merged
+//   [32, 32 + 2*ncta)       one 64-bit claim word per CTA range: blocks claimed from the front (low
 //                           half, by the owner) and from the back (high half, by thieves)
 //   [.., + nseq)            partial slots handed out per sequence
 //   [.., + nseq*Hkv)        blocks finished per (sequence, KV head)
-constexpr uint32_t kLaunchCounters = 16;
-constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntMerged = 4;
+//   [.., + 8*nseq*Hkv)      merge requests in the order they were published:
+//                           1 + 16*(sequence*Hkv + KV head) + (8 + query head of the group, for a
+//                           request that covers one query head only, else 0)
+constexpr uint32_t kLaunchCounters = 32;
+constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntMergePub = 16, kCntMergeTaken = 17, kCntMerged = 18;
 constexpr uint32_t kMaxStepLayers = 128;
+constexpr uint32_t kSharedMergeMin = 12;  // partials from which a merge is offered to every CTA
+constexpr uint32_t kSplitMergeMin = 48;   // partials from which it is offered one query head at a time
 inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
-  return kLaunchCounters + 2 * static_cast<size_t>(ncta) + nseq + static_cast<size_t>(nseq) * Hkv;
+  return kLaunchCounters + 2 * static_cast<size_t>(ncta) + nseq + 9 * static_cast<size_t>(nseq) * Hkv;
 }
 
 // Parameters of one launch of the layer kernel. It covers layers first_layer .. first_layer +
@@ -74,6 +81,7 @@ struct LayerParams {
   uint32_t steal_floor;         // before the launch's last layer: least a range must have left to be stolen from
   uint32_t steal_floor_last;    // the same in the launch's last layer
   uint32_t merge_inline;        // 1: the warp that completes a (sequence, KV head) merges it itself
+  uint32_t shared_merges;       // 1: merges of kSharedMergeMin partials or more are published for every CTA to take
   uint32_t copy_loads_ahead;    // 16 KB loads the copy thread keeps in flight: 3 (default) or 4
   uint32_t copy_sms;            // 0: every CTA's copy thread takes part in the gather; else only the first copy_sms
   const void* q;                // first_layer's [nseq][Hq][128] bf16

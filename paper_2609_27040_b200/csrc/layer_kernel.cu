@@ -31,8 +31,12 @@
 //     queues a merge request (the ring is shared by all consumer warps, so a warp that stopped to
 //     merge would stall the whole CTA) or, when layers are short, merges in line (then the merges
 //     of a sequence's KV heads run side by side instead of one after the other).
-//   * merge warp: serves the CTA's merge requests; consumer warps join it once their streaming is
-//     over.
+//   * merge warp: serves the CTA's merge queue, then merge requests that any CTA has published for
+//     all: the KV heads of a sequence finish together in one CTA, and with few long sequences their
+//     merges, of a hundred and more partials each, would queue up behind one warp (a layer of one
+//     128k-token sequence took 155 us that way and takes 87 us now). Consumer warps join once their
+//     streaming is over. Nobody waits for a request that is not yet published, so a CTA never stays
+//     behind for work of CTAs that are not resident yet.
 //   * copy warp: one thread moves 16 KB pieces lent arena -> shared ring -> staging slot with TMA
 //     bulk copies (global->shared on an mbarrier, shared->global in bulk async-groups), pulling
 //     64 KB units from an atomic counter. No SM lane touches the copied bytes.
@@ -74,9 +78,10 @@ constexpr uint32_t kFlush = 0xFFFFFFFEu;   // descriptor without data: close the
 constexpr uint32_t kNewRun = 0x80000000u;
 constexpr uint32_t kRingAlign = 128;
 constexpr uint32_t kStealMin = 2, kStealMax = 16;
+constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
-constexpr uint64_t kWaitNs = 2000000000ull;
+constexpr uint32_t kMqTail = kMq, kMqHead = kMq + 1, kMqDone = kMq + 2;
 constexpr uint32_t kOwnCache = 512;        // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
@@ -120,7 +125,7 @@ struct Smem {
   UnitDesc* queue;      // [kQueue]
   uint8_t** copy_dst;   // [kNC]
   uint32_t* copy_len;   // [kNC]
-  uint32_t* mq;         // merge queue: [kMq] entries, then tail, head, consumer warps done
+  uint32_t* mq;         // merge queue of the CTA: [kMq] entries, then tail, head, consumer warps done
   int32_t* own_res;     // [kOwnCache] resolved entries of the CTA's own range
 };
 
@@ -168,6 +173,9 @@ __device__ __forceinline__ uint32_t* seq_counts(const LayerParams& p, uint32_t l
   return layer_counters(p, li) + kLaunchCounters + 2 * p.ncta;
 }
 __device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p, uint32_t li) { return seq_counts(p, li) + p.nseq; }
+__device__ __forceinline__ uint32_t* merge_requests(const LayerParams& p, uint32_t li) {
+  return merge_counts(p, li) + p.nseq * p.Hkv;
+}
 __device__ __forceinline__ float* part_o_of(const LayerParams& p, uint32_t li) { return p.part_o + (li & 1u) * p.part_o_stride; }
 __device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) { return p.part_ml + (li & 1u) * p.part_ml_stride; }
 
@@ -253,7 +261,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     }
     // The partial buffer of this layer's parity was last used two layers ago: its merges must be done.
     if (li >= 2) {
-      ok = wait_counter(layer_counters(p, li - 2) + kCntMerged, p.nseq * Hkv, p.status);
+      ok = wait_counter(layer_counters(p, li - 2) + kCntMerged, p.nseq * p.Hq, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
     }
@@ -625,7 +633,8 @@ __device__ __forceinline__ void merge_heads_serial(const LayerParams& p, const M
   }
 }
 
-__device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uint32_t seq, uint32_t g) {
+// sub = 0: all query heads of KV head g; sub = 8 + hh: query head hh of the group only.
+__device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uint32_t seq, uint32_t g, uint32_t sub = 0) {
   MergeCtx c;
   c.part_o = part_o_of(p, li);
   c.part_ml = part_ml_of(p, li);
@@ -634,7 +643,8 @@ __device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uin
   const uint32_t s0 = p.seq_slot_base[seq];
   const uint32_t n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
                                    : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
-  switch (p.G) {
+  switch (sub ? 0u : p.G) {
+    case 0: merge_heads<1>(p, c, seq, g * p.G + (sub & 7u), s0, n); break;  // one head: 16 partials in flight
     case 1: merge_heads<1>(p, c, seq, g, s0, n); break;
     case 2: merge_heads<2>(p, c, seq, g, s0, n); break;
     case 4: merge_heads<4>(p, c, seq, g, s0, n); break;
@@ -644,7 +654,7 @@ __device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uin
   __syncwarp();
   if ((threadIdx.x & 31u) == 0) {
     __threadfence();
-    atomicAdd(layer_counters(p, li) + kCntMerged, 1u);
+    atomicAdd(layer_counters(p, li) + kCntMerged, sub ? 1u : p.G);
   }
 }
 
@@ -663,14 +673,32 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
   old = __shfl_sync(0xffffffffu, old, 0);
   if (old + blocks != p.blk_off[seq + 1] - p.blk_off[seq]) return;
   __threadfence();
+  // A sequence cut into many partials (few, long sequences) has long merges, and those of its KV
+  // heads all become due in this CTA at the same time: they are published for any CTA's merge warp
+  // to take. Other merges are done in line when a layer is short (they are the critical path then:
+  // the Hkv warps that finish a sequence together merge side by side), else they go to the CTA's
+  // own queue, which costs no global atomics and does not hold up the ring.
+  const uint32_t n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
+                                   : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
+  const bool shared = p.shared_merges && n >= kSharedMergeMin;
+  if (p.merge_inline && !shared) {
+    merge_one(p, li, seq, g);
+    return;
+  }
   volatile uint32_t* mq = sm.mq;
   uint32_t queued = 0;
   if (lane == 0) {
-    // Up to Hkv warps may pass this check at once, hence the margin. When a layer is short
-    // (merge_inline) the merges are the critical path: the Hkv warps that finish a sequence together
-    // merge side by side instead of leaving Hkv merges in a row to the merge warp.
-    if (!p.merge_inline && static_cast<int32_t>(mq[kMq] - mq[kMq + 1]) < static_cast<int32_t>(kMq - 8)) {
-      const uint32_t t = atomicAdd(&sm.mq[kMq], 1u);
+    if (shared) {
+      // A very long merge goes out one query head at a time: more warps, and each keeps four times
+      // as many partials in flight.
+      const uint32_t parts = n >= kSplitMergeMin && p.G > 1 ? p.G : 1u;
+      const uint32_t slot = atomicAdd(layer_counters(p, li) + kCntMergePub, parts);
+      for (uint32_t hh = 0; hh < parts; ++hh)
+        ptx::st_release_gpu(merge_requests(p, li) + slot + hh, 1u + 16u * (seq * p.Hkv + g) + (parts > 1 ? 8u + hh : 0u));
+      queued = 1;
+    } else if (static_cast<int32_t>(mq[kMqTail] - mq[kMqHead]) < static_cast<int32_t>(kMq - 8)) {
+      // Up to Hkv warps may pass this check at once, hence the margin.
+      const uint32_t t = atomicAdd(&sm.mq[kMqTail], 1u);
       const uint64_t t0 = ptx::global_timer_ns();
       while (mq[t % kMq] != kMqEmpty && ptx::global_timer_ns() - t0 < kWaitNs) __nanosleep(64);
       mq[t % kMq] = (li << 24) | (seq << 4) | g;
@@ -681,32 +709,108 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
   if (!queued) merge_one(p, li, seq, g);
 }
 
-// Serves the merge queue until every consumer warp of the CTA has finished and no request is left.
-// Run by the merge warp from the start and by each consumer warp once its streaming is over.
-__device__ void merge_role(const LayerParams& p, const Smem& sm) {
+// Serves merge requests: first those of the CTA's own queue, then requests that any CTA has
+// published for all. Run by the merge warp from the start and by each consumer warp once its
+// streaming is over. A warp leaves when its CTA queues nothing more (a consumer warp: at once), its
+// queue is empty and nothing published is left untaken; a published request is therefore taken at
+// the latest by the warp that published it. Nobody waits for a request that is not yet published, so
+// a CTA never stays behind for work of CTAs that are not resident yet.
+__device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consumer) {
+  if (p.merge_inline && !p.shared_merges) return;
   const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t total = p.nseq * p.Hq;  // query heads to merge per layer
   volatile uint32_t* mq = sm.mq;
+  uint32_t gli = 0, nap = 64;
   for (;;) {
-    uint32_t v = kMqEmpty;
+    uint32_t v = kMqEmpty, sub = 0;  // a request in the CTA queue's format; one query head only?
+    bool leave = false;
     if (lane == 0) {
-      const uint32_t h = atomicAdd(&sm.mq[kMq + 1], 1u);
-      const uint64_t t0 = ptx::global_timer_ns();
       for (;;) {
-        v = mq[h % kMq];
-        if (v != kMqEmpty) {
-          mq[h % kMq] = kMqEmpty;
+        // 1. the CTA's own queue
+        const uint32_t hd = mq[kMqHead];
+        if (static_cast<int32_t>(mq[kMqTail] - hd) > 0) {
+          if (atomicCAS(&sm.mq[kMqHead], hd, hd + 1) != hd) continue;
+          const uint64_t t0 = ptx::global_timer_ns();
+          while ((v = mq[hd % kMq]) == kMqEmpty) {  // its writer holds the ticket already
+            if (ptx::global_timer_ns() - t0 > kWaitNs) {
+              if (p.status) atomicExch(p.status, kDevTimeout);
+              leave = true;
+              break;
+            }
+          }
+          if (!leave) mq[hd % kMq] = kMqEmpty;
           break;
         }
-        // No request will ever get this ticket once all consumers are done and the tail is behind it.
-        if (mq[kMq + 2] == p.Hkv && static_cast<int32_t>(mq[kMq] - h) <= 0) break;
-        if (ptx::global_timer_ns() - t0 > 2 * kWaitNs) break;  // a consumer that gave up never reports in
-        __nanosleep(128);
+        // 2. requests published for all: the oldest layer not yet merged completely, and the next
+        if (p.shared_merges)
+          while (gli < p.num_layers && __ldcg(layer_counters(p, gli) + kCntMerged) >= total) ++gli;
+        for (uint32_t l = gli; p.shared_merges && l < p.num_layers && l < gli + 2 && v == kMqEmpty && !leave; ++l) {
+          uint32_t* cnt = layer_counters(p, l);
+          uint32_t pub = __ldcg(cnt + kCntMergePub);
+          uint32_t taken = __ldcg(cnt + kCntMergeTaken);
+          if (taken < pub) {
+            // Every idle merge warp of the GPU sees a new request within a microsecond or two. They
+            // come forward in sixteen groups, 128 ns apart, so that a handful of them compete for
+            // it and the rest find it gone without touching the counter.
+            const uint32_t turn = (blockIdx.x + taken) & 15u;
+            if (turn) {
+              __nanosleep(turn * 128);
+              pub = __ldcg(cnt + kCntMergePub);
+              taken = __ldcg(cnt + kCntMergeTaken);
+            }
+          }
+          while (taken < pub) {
+            const uint32_t old = atomicCAS(cnt + kCntMergeTaken, taken, taken + 1);
+            if (old != taken) {
+              taken = old;
+              continue;
+            }
+            // The publisher bumps the count before it writes the entry: a short, bounded wait.
+            const uint32_t* e = merge_requests(p, l) + taken;
+            uint32_t job;
+            const uint64_t t0 = ptx::global_timer_ns();
+            while ((job = ptx::ld_acquire_gpu(e)) == 0) {
+              if (ptx::global_timer_ns() - t0 > kWaitNs) {
+                if (p.status) atomicExch(p.status, kDevTimeout);
+                leave = true;
+                break;
+              }
+            }
+            if (!leave) {
+              const uint32_t sg = (job - 1) >> 4;
+              v = (l << 24) | ((sg / p.Hkv) << 4) | (sg % p.Hkv);
+              sub = (job - 1) & 15u;
+            }
+            break;
+          }
+        }
+        if (v != kMqEmpty || leave) break;
+        // 3. nothing to do: leave, or look again a little later
+        if (is_consumer || mq[kMqDone] == p.Hkv) {
+          bool pending = static_cast<int32_t>(mq[kMqTail] - mq[kMqHead]) > 0;
+          for (uint32_t l = gli; p.shared_merges && l < p.num_layers && !pending; ++l) {
+            const uint32_t* cnt = layer_counters(p, l);
+            pending = __ldcg(cnt + kCntMergeTaken) < __ldcg(cnt + kCntMergePub);
+          }
+          if (!pending) {
+            leave = true;
+            break;
+          }
+          continue;
+        }
+        __nanosleep(nap);
+        nap = min(nap * 2, 2048u);
       }
     }
+    leave = __shfl_sync(0xffffffffu, leave, 0);
     v = __shfl_sync(0xffffffffu, v, 0);
-    if (v == kMqEmpty) return;
-    __threadfence();
-    merge_one(p, v >> 24, (v >> 4) & 0xFFFFFu, v & 15u);
+    sub = __shfl_sync(0xffffffffu, sub, 0);
+    if (v != kMqEmpty) {
+      nap = 64;
+      __threadfence();
+      merge_one(p, v >> 24, (v >> 4) & 0xFFFFFu, v & 15u, sub);
+    }
+    if (leave) return;
   }
 }
 
@@ -1031,7 +1135,7 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     }
     for (int s = 0; s < kNC; ++s) ptx::mbar_init(ptx::smem_u32(&sm.copy_full[s]), 1);
     for (uint32_t s = 0; s < kMq; ++s) sm.mq[s] = kMqEmpty;
-    sm.mq[kMq] = sm.mq[kMq + 1] = sm.mq[kMq + 2] = 0;
+    sm.mq[kMqTail] = sm.mq[kMqHead] = sm.mq[kMqDone] = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
@@ -1043,16 +1147,16 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     __syncwarp();
     if (lane == 0) {
       __threadfence_block();
-      atomicAdd(&sm.mq[kMq + 2], 1u);  // this consumer warp queues no more merges
+      atomicAdd(&sm.mq[kMqDone], 1u);  // this consumer warp queues no more merges
     }
     __syncwarp();
-    merge_role(p, sm);
+    merge_role(p, sm, true);
   } else if (warp == p.Hkv) {
     producer_role(p, sm);
   } else if (warp == p.Hkv + 1) {
     if (lane == 0) copy_role(p, sm);
   } else if (warp == p.Hkv + 2) {
-    merge_role(p, sm);
+    merge_role(p, sm, false);
   }
 }
 

@@ -548,6 +548,11 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.steal_floor_last = s->cfg.steal_floor ? std::min(s->cfg.steal_floor, kStealFloorLast) : kStealFloorLast;
   // A layer of a few dozen blocks per CTA lasts less than the merges of one sequence done in a row.
   d.merge_inline = p->per <= kInlineMergePer ? 1u : 0u;
+  // Few, long sequences: a sequence is cut into many partials and its merges are worth sharing
+  // between the CTAs (stealing adds a few partials to the count the even split gives).
+  uint32_t longest = 0;
+  for (uint32_t i = 0; i < p->nseq; ++i) longest = std::max(longest, p->blk_off[i + 1] - p->blk_off[i]);
+  d.shared_merges = longest / p->per + 4 >= ema::kSharedMergeMin ? 1u : 0u;
   d.copy_loads_ahead = s->cfg.prefetch_priority ? 4u : 3u;
   // Lent arena behind a slow link (pinned host memory): a few copy threads saturate it.
   d.copy_sms = s->cfg.lent_kind == 1 ? (s->cfg.copy_ctas ? std::min(s->cfg.copy_ctas, s->ncta) : std::min(kSlowLinkCopySms, s->ncta)) : 0u;

@@ -184,6 +184,30 @@ def test_decode_step_corner_shapes(case):
     _step_matches_oracle(sc, g)
 
 
+@pytest.mark.parametrize("case", ["split_inline", "shared_queue", "split_queue", "static_long"])
+@pytest.mark.parametrize("mode", [0, 2])
+def test_few_long_sequences_share_their_merges(case, mode):
+    """A long sequence is cut into many partials; its merges are published for every CTA's merge
+    warp (one query head at a time from 48 partials up) instead of being done by the CTA that
+    finished it. Short layers (merges otherwise in line), long layers (otherwise the CTA's queue),
+    a short sequence beside the long one (its merge stays local), and the static split."""
+    kw = {"pipeline_mode": mode}
+    if case == "split_inline":        # 148 ranges of 17 blocks: a layer is short, 148 partials
+        lengths = np.array([40000])
+    elif case == "shared_queue":      # 30 ranges of 85 blocks: about 30 partials, and a short neighbour
+        lengths, kw["decode_ctas"] = np.array([40000, 700]), 30
+    elif case == "split_queue":       # 60 ranges of 50 blocks: 60 partials each split by query head
+        lengths, kw["decode_ctas"] = np.array([48000]), 60
+    else:
+        lengths, kw["decode_ctas"], kw["static_split"] = np.array([30000, 9000]), 50, 1
+    wl = synth.Workload(case, 3, 8, 2, len(lengths), int(lengths.min()), int(lengths.max()), 0.4)
+    sc = Scenario(wl, 31, lengths=lengths)
+    g = _gpu(sc, **kw)
+    _step_matches_oracle(sc, g)
+    for layer in (0, 2):                                   # and through the per-layer entry points
+        _check_layer(sc, g, layer, check_bytes=False)
+
+
 def test_many_different_batches_rotate_the_plan_buffers():
     """More distinct batches (subsets and orders of the sequences) than the library has plan buffers,
     enqueued back to back without synchronising, then each result checked: a plan buffer must not
