@@ -67,12 +67,14 @@ constexpr uint32_t kNAFused = 4;           // attention ring (half-block stages)
 constexpr uint32_t kNAAlone = 3;           // ... and when the launch gathers nothing. With one 32 KB request per
                                            // stage a deeper ring only queues more reads in the memory
                                            // system and measures slower (3: 6.1 TB/s, 6: 5.3 TB/s).
-constexpr uint32_t kNAMax = 4;
+                                           // With fewer KV heads a stage is smaller (4 KB per head): the
+                                           // ring then has 8 / Hkv times as many stages, the same bytes.
+constexpr uint32_t kNAMax = 32;
 constexpr int kNC = 6;                     // copy ring: 16 KB stages
 constexpr uint32_t kCopyLoadsDefault = 3;  // loads in flight (LayerParams::copy_loads_ahead, 3 or 4) ...
 constexpr int kStoresOpen = 2;             // ... and stores not yet known complete; 4 + 2 = kNC
 constexpr uint32_t kCopyChunk = 16384;
-constexpr int kQueue = 8;                  // unit descriptors in flight (> kNAMax / 2 + 1)
+constexpr int kQueue = 20;                 // unit descriptors in flight (> kNAMax / 2 + 1)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kFlush = 0xFFFFFFFEu;   // descriptor without data: close the open run now
 constexpr uint32_t kNewRun = 0x80000000u;
@@ -82,7 +84,7 @@ constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
 constexpr uint32_t kMqTail = kMq, kMqHead = kMq + 1, kMqDone = kMq + 2;
-constexpr uint32_t kOwnCache = 512;        // resolved entries of the own range kept in shared memory
+constexpr uint32_t kOwnCache = 352;        // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
 __host__ __device__ constexpr uint32_t half_stage_bytes(uint32_t Hkv) { return kT * row_bytes(Hkv); }
@@ -130,26 +132,33 @@ struct Smem {
 };
 
 // Bookkeeping area behind the two rings; every part 16-byte aligned.
-constexpr size_t kBarBytes = 24 * sizeof(uint64_t);
+constexpr size_t kBarBytes = 70 * sizeof(uint64_t);
 constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
 constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
 constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
 constexpr size_t kOwnBytes = kOwnCache * sizeof(int32_t);
-static_assert(2 * kNAMax + kNC <= 24 && kNC <= 8, "bookkeeping area too small");
+static_assert(2 * kNAMax + kNC <= 70 && kNC <= 8 && kQueue > kNAMax / 2 + 1, "bookkeeping area too small");
 static_assert(kNAFused * 32768 + kNC * 16384 >= kNAAlone * 32768, "the deeper ring must fit in the fused layout");
 
+// Stages per 32 KB of ring: 1 for 5..8 KV heads, 2 for 3 or 4, 4 for 2, 8 for 1.
+__host__ __device__ constexpr uint32_t ring_scale(uint32_t Hkv) { return 8u / Hkv; }
+
+static_assert(kRingAlign + kNAFused * 32768 + kNC * kCopyChunk + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes +
+                      kOwnBytes <= 232448,
+              "more shared memory than a CTA can have (227 KB)");
+
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
-  return kRingAlign + static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
+  return kRingAlign + static_cast<size_t>(kNAFused) * ring_scale(Hkv) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
   Smem s;
-  s.na = gathers ? kNAFused : kNAAlone;
+  s.na = (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
   base += (kRingAlign - (ptx::smem_u32(base) & (kRingAlign - 1))) & (kRingAlign - 1);
   s.att_ring = base;
-  s.copy_ring = base + static_cast<size_t>(kNAFused) * half_stage_bytes(Hkv);
+  s.copy_ring = base + static_cast<size_t>(kNAFused) * ring_scale(Hkv) * half_stage_bytes(Hkv);
   uint8_t* p = s.copy_ring + static_cast<size_t>(kNC) * kCopyChunk;
   s.att_full = reinterpret_cast<uint64_t*>(p);
   s.att_empty = s.att_full + kNAMax;

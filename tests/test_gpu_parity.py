@@ -99,7 +99,7 @@ def test_small_decode_grid_and_many_segments():
 
 
 def test_ranges_longer_than_the_cached_table_and_multi_layer_pass():
-    """One or two CTAs over ~2 500 blocks: a range is longer than the 2 048 table entries a CTA keeps
+    """One or two CTAs over ~2 500 blocks: a range is longer than the few hundred table entries a CTA keeps
     in shared memory, so the tail of the range reads its entries from global memory; claims of 16
     blocks cross the boundary. Checked per layer and as one launch over both layers."""
     wl = synth.Workload("long", 2, 4, 2, 5, 7000, 8200, 0.45)
