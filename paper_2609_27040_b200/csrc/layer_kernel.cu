@@ -687,9 +687,10 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
   // to take. Other merges are done in line when a layer is short (they are the critical path then:
   // the Hkv warps that finish a sequence together merge side by side), else they go to the CTA's
   // own queue, which costs no global atomics and does not hold up the ring.
-  const uint32_t n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
-                                   : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
-  const bool shared = p.shared_merges && n >= kSharedMergeMin;
+  uint32_t n = 0;  // partials of the sequence; only looked up where merges can be shared at all
+  if (p.shared_merges)
+    n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq]) : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
+  const bool shared = n >= kSharedMergeMin;
   if (p.merge_inline && !shared) {
     merge_one(p, li, seq, g);
     return;
@@ -724,12 +725,44 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
 // queue is empty and nothing published is left untaken; a published request is therefore taken at
 // the latest by the warp that published it. Nobody waits for a request that is not yet published, so
 // a CTA never stays behind for work of CTAs that are not resident yet.
+// The CTA's own queue only (launches in which no merge is shared): every warp draws a ticket and
+// waits for the request that gets it, or until no request can get it any more.
+__device__ void merge_role_local(const LayerParams& p, const Smem& sm) {
+  const uint32_t lane = threadIdx.x & 31u;
+  volatile uint32_t* mq = sm.mq;
+  for (;;) {
+    uint32_t v = kMqEmpty;
+    if (lane == 0) {
+      const uint32_t h = atomicAdd(&sm.mq[kMqHead], 1u);
+      const uint64_t t0 = ptx::global_timer_ns();
+      for (;;) {
+        v = mq[h % kMq];
+        if (v != kMqEmpty) {
+          mq[h % kMq] = kMqEmpty;
+          break;
+        }
+        // No request will ever get this ticket once all consumers are done and the tail is behind it.
+        if (mq[kMqDone] == p.Hkv && static_cast<int32_t>(mq[kMqTail] - h) <= 0) break;
+        if (ptx::global_timer_ns() - t0 > 2 * kWaitNs) break;  // a consumer that gave up never reports in
+        __nanosleep(128);
+      }
+    }
+    v = __shfl_sync(0xffffffffu, v, 0);
+    if (v == kMqEmpty) return;
+    __threadfence();
+    merge_one(p, v >> 24, (v >> 4) & 0xFFFFFu, v & 15u);
+  }
+}
+
 __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consumer) {
-  if (p.merge_inline && !p.shared_merges) return;
+  if (!p.shared_merges) {
+    if (!p.merge_inline) merge_role_local(p, sm);
+    return;
+  }
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t total = p.nseq * p.Hq;  // query heads to merge per layer
   volatile uint32_t* mq = sm.mq;
-  uint32_t gli = 0, nap = 64;
+  uint32_t gli = 0, idle = 0;  // idle: looks at the own queue since the last request
   for (;;) {
     uint32_t v = kMqEmpty, sub = 0;  // a request in the CTA queue's format; one query head only?
     bool leave = false;
@@ -750,10 +783,14 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
           if (!leave) mq[hd % kMq] = kMqEmpty;
           break;
         }
-        // 2. requests published for all: the oldest layer not yet merged completely, and the next
-        if (p.shared_merges)
+        // 2. requests published for all: the oldest layer not yet merged completely, and the next.
+        // The own queue (shared memory) is looked at every 128 ns, the list in device memory at
+        // once when the warp falls idle and then every eighth time, about once a microsecond.
+        const bool look = (idle & 7u) == 0;
+        ++idle;
+        if (look)
           while (gli < p.num_layers && __ldcg(layer_counters(p, gli) + kCntMerged) >= total) ++gli;
-        for (uint32_t l = gli; p.shared_merges && l < p.num_layers && l < gli + 2 && v == kMqEmpty && !leave; ++l) {
+        for (uint32_t l = gli; look && l < p.num_layers && l < gli + 2 && v == kMqEmpty && !leave; ++l) {
           uint32_t* cnt = layer_counters(p, l);
           uint32_t pub = __ldcg(cnt + kCntMergePub);
           uint32_t taken = __ldcg(cnt + kCntMergeTaken);
@@ -797,7 +834,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
         // 3. nothing to do: leave, or look again a little later
         if (is_consumer || mq[kMqDone] == p.Hkv) {
           bool pending = static_cast<int32_t>(mq[kMqTail] - mq[kMqHead]) > 0;
-          for (uint32_t l = gli; p.shared_merges && l < p.num_layers && !pending; ++l) {
+          for (uint32_t l = gli; l < p.num_layers && !pending; ++l) {
             const uint32_t* cnt = layer_counters(p, l);
             pending = __ldcg(cnt + kCntMergeTaken) < __ldcg(cnt + kCntMergePub);
           }
@@ -807,15 +844,14 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
           }
           continue;
         }
-        __nanosleep(nap);
-        nap = min(nap * 2, 2048u);
+        __nanosleep(128);
       }
     }
     leave = __shfl_sync(0xffffffffu, leave, 0);
     v = __shfl_sync(0xffffffffu, v, 0);
     sub = __shfl_sync(0xffffffffu, sub, 0);
     if (v != kMqEmpty) {
-      nap = 64;
+      idle = 0;
       __threadfence();
       merge_one(p, v >> 24, (v >> 4) & 0xFFFFFu, v & 15u, sub);
     }
@@ -1138,7 +1174,7 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
   const Smem sm = carve(smem_raw, p.Hkv, gathers);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
   if (threadIdx.x == 0) {
-    for (uint32_t s = 0; s < kNAMax; ++s) {
+    for (uint32_t s = 0; s < sm.na; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sm.att_full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), p.Hkv);
     }
