@@ -25,7 +25,7 @@ constexpr uint32_t kStealFloorMin = 4;  // default steal floor: a third of a ran
 constexpr uint32_t kStealFloorLast = 8; // default steal floor in the last layer of a launch
 constexpr uint32_t kInlineMergePer = 48; // ranges up to this many blocks: consumer warps merge in line
 constexpr uint32_t kSlowLinkCopySms = 8;  // copy threads that take part in the gather over a slow link
-constexpr uint32_t kMinPer = 12;          // least blocks per CTA range: fewer CTAs rather than more partials
+constexpr uint32_t kMinPer = 8;           // least blocks per CTA range: fewer CTAs rather than more partials
 constexpr uint32_t kOwnChunk = 16;  // most blocks a CTA claims from its own range at a time
 
 struct Seq {
