@@ -92,8 +92,9 @@ struct LayerParams {
   uint32_t q_ready_layers;
   float* lse;                   // [nseq][Hq] or NULL (single-layer launches only)
   float* part_o;                // [slots][Hq][128] unnormalised partial outputs; layers alternate
-  float* part_ml;               // [slots][Hq][4]   between two such buffers (stride below)
-  uint64_t part_o_stride, part_ml_stride;  // floats between the two buffers (0: single layer)
+  float* part_ml;               // [slots][Hq][4]   between part_buffers such buffers (stride below)
+  uint64_t part_o_stride, part_ml_stride;  // floats between the buffers (0: single layer)
+  uint32_t part_buffers;        // buffers the layers of a launch take turns with (1, 2 or 4)
   uint32_t* counters;           // first_layer's layer_counter_words(), all zeroed before the launch
   uint64_t counters_stride;     // words from one layer's counters to the next
   uint32_t nseq, ncta;

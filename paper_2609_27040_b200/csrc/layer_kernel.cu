@@ -45,7 +45,7 @@
 // that span several layers (which are launched cooperatively, so every CTA is resident): a staged
 // block of layer l is read only after its ready flag shows that the gather has landed it; a ring
 // slot is overwritten only after the attention of the layer that last used it is complete; a partial
-// buffer (two alternate) is reused only after the merges of the layer before last are done. They
+// buffer (four take turns) is reused only after the merges of the layer that used it last are done. They
 // wait on what earlier layers' work produces, never on later work, and a run left open at the end of
 // a layer is closed at once (a CTA may find nothing to claim in later layers), so they cannot form a
 // cycle. A fourth, optional wait is for queries that arrive from the host while the launch runs. Every wait, mbarrier or counter, is bounded (about two seconds): on expiry the role records
@@ -185,8 +185,12 @@ __device__ __forceinline__ uint32_t* merge_counts(const LayerParams& p, uint32_t
 __device__ __forceinline__ uint32_t* merge_requests(const LayerParams& p, uint32_t li) {
   return merge_counts(p, li) + p.nseq * p.Hkv;
 }
-__device__ __forceinline__ float* part_o_of(const LayerParams& p, uint32_t li) { return p.part_o + (li & 1u) * p.part_o_stride; }
-__device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) { return p.part_ml + (li & 1u) * p.part_ml_stride; }
+__device__ __forceinline__ float* part_o_of(const LayerParams& p, uint32_t li) {
+  return p.part_o + (li & (p.part_buffers - 1u)) * p.part_o_stride;
+}
+__device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) {
+  return p.part_ml + (li & (p.part_buffers - 1u)) * p.part_ml_stride;
+}
 
 // Bounded wait until a device word written by another CTA equals `value`.
 __device__ __forceinline__ bool wait_counter_eq(const uint32_t* word, uint32_t value, int* status) {
@@ -268,9 +272,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       p.trace[li * p.trace_stride + 4 * blockIdx.x] = ptx::global_timer_ns();
       p.trace[li * p.trace_stride + 4 * blockIdx.x + 1] = 0;
     }
-    // The partial buffer of this layer's parity was last used two layers ago: its merges must be done.
-    if (li >= 2) {
-      ok = wait_counter(layer_counters(p, li - 2) + kCntMerged, p.nseq * p.Hq, p.status);
+    // The partial buffer of this layer was last used part_buffers layers ago: its merges must be done.
+    if (li >= p.part_buffers) {
+      ok = wait_counter(layer_counters(p, li - p.part_buffers) + kCntMerged, p.nseq * p.Hq, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
     }
