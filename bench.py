@@ -496,9 +496,9 @@ def run_ours(args, wl):
                     "both_met_by": pick if ok else None,
                     "default_step_time_over_nominal_hbm_floor": 1.0 - combined / NOMINAL_HBM_GBS,
                     "note": "the default pipeline maximises tokens/s: it is HBM-bound (its step takes the stated fraction "
-                            "longer than the same bytes at the nominal 8 TB/s), so the wait is slack of CTAs that are "
-                            "ahead, not time the step loses; the named configuration trades tokens/s for a prefetch "
-                            "that is always ahead of every CTA"}
+                            "longer than the same bytes at the nominal 8 TB/s), so the wait is not time the step loses: "
+                            "attention takes its share of HBM first and then waits while the copy threads use the "
+                            "rest; the named configuration trades tokens/s for a prefetch that is always ahead"}
             extra["kernels_alone"] = {
                 "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
