@@ -48,7 +48,7 @@ def parse_args():
                     help="0 one persistent launch per pass, 1 two streams with events, 2 one fused launch per layer")
     ap.add_argument("--static-split", type=int, default=0, help="1: no work stealing between CTAs")
     ap.add_argument("--prefetch-priority", type=int, default=0,
-                    help="1: the copy threads keep 4 loads in flight (prefetch always ahead, slower pass)")
+                    help="1: two partial buffers instead of four (CTAs in step, prefetch always ahead, slower pass)")
     ap.add_argument("--no-ablations", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")

@@ -122,12 +122,14 @@ typedef struct {
                                      in single-layer launches); 1 = steal down to the last block, which
                                      keeps all CTAs in step: almost no CTA ever waits for
                                      prefetched data, at a lower overall rate                    */
-  uint32_t prefetch_priority;     /* fused pipelines: 0 = default, the copy thread of an SM keeps 3 loads
-                                     of 16 KB in flight; attention follows the prefetch closely,
-                                     waits for it part of the time and reads staged blocks out of L2
-                                     (highest tokens/s); 1 = 4 loads in flight: the prefetch stays
-                                     far ahead, attention (almost) never waits for it, staged blocks
-                                     come from DRAM and the pass as a whole is slower             */
+  uint32_t prefetch_priority;     /* one launch per pass: 0 = default, the layers take turns with four
+                                     buffers of split-KV partials, so a CTA may run up to three
+                                     layers ahead of the slowest merge; attention follows the
+                                     prefetch closely, waits for it part of the time and reads
+                                     staged blocks out of L2 (highest tokens/s); 1 = two buffers:
+                                     the CTAs stay within a layer of one another, the prefetch is
+                                     far ahead of all of them, attention (almost) never waits for
+                                     it, staged blocks come from DRAM and the pass is slower     */
 } slice_config_t;
 
 typedef struct {

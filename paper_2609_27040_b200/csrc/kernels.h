@@ -82,7 +82,7 @@ struct LayerParams {
   uint32_t steal_floor_last;    // the same in the launch's last layer
   uint32_t merge_inline;        // 1: the warp that completes a (sequence, KV head) merges it itself
   uint32_t shared_merges;       // 1: merges of kSharedMergeMin partials or more are published for every CTA to take
-  uint32_t copy_loads_ahead;    // 16 KB loads the copy thread keeps in flight: 3 (default) or 4
+  uint32_t copy_loads_ahead;    // 16 KB loads the copy thread keeps in flight: 3 or 4 (the host sets 4)
   uint32_t copy_sms;            // 0: every CTA's copy thread takes part in the gather; else only the first copy_sms
   const void* q;                // first_layer's [nseq][Hq][128] bf16
   void* out;
