@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=None, help="default 200 (reference arm: 5)")
+    ap.add_argument("--warmup", type=int, default=None, help="default 10 (reference arm: 1)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_8b_decode", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--seed", type=int, default=0)
@@ -51,24 +51,35 @@ def parse_args():
                     help="1: two partial buffers instead of four (CTAs in step, prefetch always ahead, slower pass)")
     ap.add_argument("--no-ablations", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parity-check", action="store_true", help="skip the oracle check of the last timed pass")
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (debugging)")
-    return ap.parse_args()
+    args = ap.parse_args()
+    # The reference arm really spends what it reports (about four seconds per step): fewer steps by default.
+    if args.steps is None:
+        args.steps = 5 if args.impl == "reference" else 200
+    if args.warmup is None:
+        args.warmup = 1 if args.impl == "reference" else 10
+    return args
 
 
-def profile_traffic(wl, mode):
-    """DRAM bytes per launch of the layer kernel from the committed ncu summary. The capture ran the
-    full batch on 2 layers; traffic grows in proportion to the layers a launch spans, so it is scaled
-    by layers. None for other workloads or pipelines."""
-    path = os.path.join(ROOT, "profiles", "slice_layer_kernel_llama3_8b_batch64_ncu.md")
-    if wl.name != "llama3_8b_decode" or wl.batch != 64 or mode != 0 or not os.path.exists(path):
-        return None
+def profile_traffic(wl, mode, prefetch_priority=0):
+    """DRAM bytes per launch of the layer kernel as ncu counted them (dram__bytes_read.sum +
+    dram__bytes_write.sum) in the capture recorded in profiles/ncu_traffic.json: the full batch on
+    fewer layers than the bench runs (a full-size launch is too large to capture), scaled by the
+    layers a launch spans, to which the traffic is proportional. A figure from that capture, not a
+    measurement of this run; None for workloads, pipelines or knobs that were not captured."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None, None
     with open(path) as f:
-        for line in f:
-            if line.strip().startswith("traffic_bytes_per_layer:"):
-                return int(line.split(":")[1]) * wl.num_layers
-    return None
+        table = json.load(f)
+    key = f"{wl.name}/batch{wl.batch}/pipeline{mode}/prefetch_priority{prefetch_priority}"
+    rec = table.get("captures", {}).get(key)
+    if not rec:
+        return None, None
+    return int(rec["dram_bytes_per_layer"] * wl.num_layers), rec
 
 
 def measured_peaks():
@@ -205,13 +216,13 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ---------------------------------------------------------------------------------------------
-def oracle_layer_sample(wl: synth.Workload, seed: int, nseq: int, repeats: int):
-    """Times the oracle (gather + fp64 paged attention) on one layer of the first `nseq` sequences
-    of the workload, host data drawn with the same placement rule. Returns (seconds per repeat,
-    sample tokens, threads)."""
+def oracle_layer_runner(wl: synth.Workload, seed: int):
+    """Host data of ONE layer of the full batch (same placement rule as the device workload) and a
+    function that runs the oracle on it once: gather of the lent blocks into a host staging slot, then
+    fp64 paged attention of every sequence through the resolved table. Returns (run, tokens, threads)."""
     import oracle
     pl = synth.make_placement(wl, seed, slack_blocks=64)
-    sub = list(range(min(nseq, wl.batch)))
+    sub = list(range(wl.batch))
     n_local = sum(int((pl.hints[i] == synth.LOCAL).sum()) for i in sub)
     n_lent = sum(int((pl.hints[i] == synth.LENT).sum()) for i in sub)
     max_blocks = int(max(len(pl.hints[i]) for i in sub)) + 1
@@ -228,49 +239,106 @@ def oracle_layer_sample(wl: synth.Workload, seed: int, nseq: int, repeats: int):
     staging = np.zeros((1, max(n_lent, 1)) + shape, np.uint16)
     q = synth.normal_bf16_bits(rng, (len(sub), wl.num_q_heads, wl.head_dim))
     lens = np.asarray([pl.lengths[i] for i in sub], np.uint32)
-    times = []
-    for _ in range(repeats):
-        t0 = time.perf_counter()
+
+    def run():
         rc, resolved, k = orc.gather(0, sub, lent, staging)
         assert rc == 0
         rc, out, _ = oracle.paged_attention(q, local[0], staging[0], resolved, lens, wl.num_q_heads, wl.num_kv_heads,
                                             wl.head_dim, wl.block_tokens, 1.0 / np.sqrt(wl.head_dim), want_lse=False)
         assert rc == 0
-        times.append(time.perf_counter() - t0)
-    return times, int(lens.sum()), oracle.num_threads()
+
+    return run, int(lens.sum()), oracle.num_threads()
 
 
-def oracle_tokens_per_s(wl, seconds_per_layer_sample, sample_tokens, total_tokens):
-    """Scales one sampled layer to a full step: time grows with tokens and with layers."""
-    step_s = seconds_per_layer_sample * (total_tokens / sample_tokens) * wl.num_layers
-    return wl.batch / step_s
+def oracle_step_seconds(run, layers: int) -> float:
+    """One step of the oracle: the whole batch, `layers` times (every layer has the same shape; the
+    oracle is run on one layer's host data again and again, so that a step costs 0.6 GB of host
+    memory instead of 19 GB). The time is the time spent, nothing is extrapolated."""
+    t0 = time.perf_counter()
+    for _ in range(layers):
+        run()
+    return time.perf_counter() - t0
 
 
 def run_reference(args, wl):
+    """The reference arm: there is no reference implementation, so the CPU oracle is timed as it
+    stands, on the same workload and metric. Every step runs what it reports."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
     oracle.build()
-    nseq = min(8, wl.batch)
-    pl = synth.make_placement(wl, args.seed, slack_blocks=64)
-    total_tokens = int(pl.lengths.sum())
-    times, sample_tokens, threads = oracle_layer_sample(wl, args.seed, nseq, args.warmup + args.steps)
-    timed = times[args.warmup:]
-    per = sum(timed) / len(timed)
-    value = oracle_tokens_per_s(wl, per, sample_tokens, total_tokens)
-    sample = (f"each step = oracle gather + fp64 paged attention of 1 layer over the first {nseq} of {wl.batch} "
-              f"sequences ({sample_tokens} of {total_tokens} tokens), scaled by tokens and by {wl.num_layers} layers")
+    run, tokens, threads = oracle_layer_runner(wl, args.seed)
+    for _ in range(args.warmup):
+        oracle_step_seconds(run, wl.num_layers)
+    t = sum(oracle_step_seconds(run, wl.num_layers) for _ in range(args.steps))
+    value = wl.batch * args.steps / t
+    sample = (f"each step = {wl.num_layers} x (oracle gather + fp64 paged attention of all {wl.batch} sequences, "
+              f"{tokens} tokens, on one layer's host data); time as spent, nothing extrapolated")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": per * (total_tokens / sample_tokens) * wl.num_layers * 1e3,
+        "warmup": args.warmup, "ms_per_step": t / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.num_layers, "sample": sample},
+        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.num_layers, "q_heads": wl.num_q_heads,
+                   "kv_heads": wl.num_kv_heads, "lent_fraction": wl.lent_fraction, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def parity_check(wl, pl, local, lent, q, outs, scale, seed):
+    """Outside every timed region: sampled outputs of the last timed pass against the CPU oracle.
+    The oracle replays the placement on its own allocator (so the tables do not come from the CUDA
+    library), the blocks of a sampled (layer, sequence) are copied back from the device arenas and
+    its dense fp64 attention is compared with what the pass wrote, all query heads, within the stated
+    bf16 tolerance. `outs` maps a label to an output tensor [layers][batch][Hq][128]. Raises when a
+    sampled output is outside the tolerance: a throughput of wrong results is no result."""
+    import oracle
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    oracle.build()
+    orc = oracle.OracleSlice(1, wl.block_tokens, wl.block_bytes, pl.local_blocks, pl.lent_blocks, pl.lent_blocks, 1,
+                             max(pl.staging_blocks, 1), max_seqs=wl.batch, max_blocks_per_seq=int(max(len(h) for h in pl.hints)) + 4,
+                             local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
+    for i, hints in enumerate(pl.hints):
+        for h in hints:
+            assert orc.alloc_blocks(i, 1, int(h))[0] == 0
+    L = wl.num_layers
+    layers = sorted({0, min(4, L - 1), min(5, L - 1), L // 2, L - 1})
+    order = np.argsort(pl.lengths)
+    rng = np.random.default_rng(seed)
+    seqs = sorted({int(order[0]), int(order[-1])} | {int(x) for x in rng.choice(wl.batch, min(2, wl.batch), replace=False)})
+    worst = {k: 0.0 for k in outs}
+    worst_rel = {k: 0.0 for k in outs}
+
+    def bits(t):
+        return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+    for layer in layers:
+        for i in seqs:
+            n = int(pl.lengths[i])
+            tab = orc.block_table(i)[1][: synth.blocks_for(n)]
+            blocks = torch.stack([local[layer, e] if e >= 0 else lent[layer, ~e] for e in tab.tolist()])
+            blocks = B.kv_block_swizzle(blocks)              # block format -> canonical token rows
+            K = blocks[:, 0].reshape(-1, wl.num_kv_heads, wl.head_dim)[:n]
+            V = blocks[:, 1].reshape(-1, wl.num_kv_heads, wl.head_dim)[:n]
+            rc, ref, _, _ = oracle.dense_attention(bits(q[layer, i]), bits(K), bits(V), wl.num_q_heads, wl.num_kv_heads,
+                                                   wl.head_dim, scale)
+            assert rc == 0
+            for label, out in outs.items():
+                got = out[layer, i].double().cpu().numpy()
+                err = np.abs(got - ref)
+                if not (np.isfinite(got).all() and (err <= 1e-2 + 1e-2 * np.abs(ref)).all()):
+                    raise RuntimeError(f"parity check failed: {label}, layer {layer}, sequence {i}, max |err| {err.max():.3e}")
+                worst[label] = max(worst[label], float(err.max()))
+                big = np.abs(ref) >= 2.0 ** -6
+                if big.any():
+                    worst_rel[label] = max(worst_rel[label], float((err[big] / np.abs(ref[big])).max()))
+    return {"layers": layers, "seqs": seqs, "heads": "all", "checked": sorted(outs), "against": "oracle.dense_attention (fp64)",
+            "tolerance": "|err| <= 1e-2 + 1e-2*|ref|", "max_abs_err": max(worst.values()),
+            "max_abs_err_by_pass": worst, "max_rel_err": max(worst_rel.values()), "ok": True}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -351,10 +419,16 @@ def run_ours(args, wl):
 
     # ---- the dominant kernel inside the pipelined pass (profile events + per-CTA trace), rank 0 ----
     roof = None
+    parity = None
     extra = {}
     if rank == 0:
         step_bytes, tokens, pl_blocks, k_blocks = w.step_bytes, w.tokens, w.pl.total_blocks, w.pl.staging_blocks
         attn_bytes_layer, pref_bytes_layer = w.attn_bytes_layer, w.pref_bytes_layer
+        if not args.no_parity_check:
+            # what the last timed pass left in `out` (device-resident run) and in the pinned host
+            # buffer (end-to-end run), against the oracle
+            parity = parity_check(wl, w.pl, w.local, w.lent, w.q, {"resident": w.out, "e2e_host": oh.view(torch.bfloat16)},
+                                  w.scale, args.seed)
         del w
         torch.cuda.empty_cache()
         peak, peak_src = measured_peaks()
@@ -392,8 +466,16 @@ def run_ours(args, wl):
         name = {0: "slice_layer_kernel (one launch per pass: attention + gather of every layer)",
                 1: "slice_layer_kernel (attention only; gather in copy_blocks_vector on a second stream)",
                 2: "slice_layer_kernel (one launch per layer: attention + gather of the next layer)"}[args.pipeline_mode]
+        traffic, traffic_rec = profile_traffic(wl, args.pipeline_mode, args.prefetch_priority)
         roof = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": profile_traffic(wl, args.pipeline_mode),
+                "frac": achieved / peak, "traffic": traffic,
+                # DRAM bytes (ncu, scaled by layers) over this run's launch time: what HBM actually moved
+                "achieved_dram": traffic / kernel_s / 1e9 if traffic else None,
+                "frac_dram": traffic / kernel_s / 1e9 / peak if traffic else None,
+                "frac_dram_of_nominal_8TBs": traffic / kernel_s / 1e9 / NOMINAL_HBM_GBS if traffic else None,
+                "traffic_source": ({"file": "profiles/ncu_traffic.json", **{k: traffic_rec[k] for k in
+                                    ("layers_captured", "dram_bytes_per_layer", "l2_hit_rate_pct", "dram_over_algorithmic")
+                                    if k in traffic_rec}} if traffic_rec else None),
                 "peak_source": f"of {peak_src}", "launches_per_step": launches_per_step,
                 "launch_us": kernel_s * 1e6 / max(launches_per_step, 1) if args.pipeline_mode != 1 else None,
                 "algorithmic_bytes_per_launch": algo // max(launches_per_step, 1) if args.pipeline_mode != 1 else attn_bytes_layer,
@@ -484,21 +566,40 @@ def run_ours(args, wl):
             extra["ablations"] = abl
             alts = {k: v for k, v in abl.items() if "stall_us_per_layer" in v}
             if alts:
+                # The 70 % gate is about what HBM moves: algorithmic bytes times the DRAM-to-algorithmic
+                # ratio of the ncu capture of the same configuration (L2 serves part of the staged
+                # blocks), where one was captured; the algorithmic figure is kept beside it.
+                def dram_ratio(prio):
+                    rec = profile_traffic(wl, 0, prio)[1]
+                    return rec.get("dram_over_algorithmic") if rec else None
+
                 def frac(v):
                     return v["stall_us_per_layer"] / (v["ms_per_step"] * 1e3 / L)
-                ok = [k for k, v in alts.items() if frac(v) < 0.05 and v["hbm_gbs_combined"] / NOMINAL_HBM_GBS >= 0.70]
+
+                def hbm(gbs, prio):
+                    r = dram_ratio(prio)
+                    return {"algorithmic_bytes": gbs / NOMINAL_HBM_GBS,
+                            "dram_bytes": gbs * r / NOMINAL_HBM_GBS if r else None,
+                            "dram_bytes_source": "ncu capture, profiles/ncu_traffic.json" if r else "unmeasured"}
+
+                def gate(gbs, prio):
+                    h = hbm(gbs, prio)
+                    return (h["dram_bytes"] if h["dram_bytes"] is not None else h["algorithmic_bytes"]) >= 0.70
+
+                prio_of = {"lock_step_stealing": 0, "prefetch_priority": 1, "prefetch_priority_lock_step": 1}
+                ok = [k for k, v in alts.items() if frac(v) < 0.05 and gate(v["hbm_gbs_combined"], prio_of.get(k, 0))]
                 pick = max(ok, key=lambda k: alts[k]["tokens_per_s"]) if ok else min(alts, key=lambda k: frac(alts[k]))
+                default_stall = extra["stall_frac_of_layer"]
                 extra["targets"] = {
-                    "hbm_frac_of_nominal_8TBs": {"target": 0.70, "default_pipeline": combined / NOMINAL_HBM_GBS,
-                                                 pick: alts[pick]["hbm_gbs_combined"] / NOMINAL_HBM_GBS},
-                    "stall_frac_of_layer": {"target": 0.05, "default_pipeline": extra["stall_frac_of_layer"],
-                                            pick: frac(alts[pick])},
+                    "hbm_frac_of_nominal_8TBs": {"target": 0.70, "default_pipeline": hbm(combined, args.prefetch_priority),
+                                                 pick: hbm(alts[pick]["hbm_gbs_combined"], prio_of.get(pick, 0))},
+                    "stall_frac_of_layer": {"target": 0.05, "default_pipeline": default_stall, pick: frac(alts[pick])},
+                    "default_pipeline_meets": {"hbm": gate(combined, args.prefetch_priority), "stall": default_stall < 0.05},
                     "both_met_by": pick if ok else None,
-                    "default_step_time_over_nominal_hbm_floor": 1.0 - combined / NOMINAL_HBM_GBS,
-                    "note": "the default pipeline maximises tokens/s: it is HBM-bound (its step takes the stated fraction "
-                            "longer than the same bytes at the nominal 8 TB/s), so the wait is not time the step loses: "
-                            "attention takes its share of HBM first and then waits while the copy threads use the "
-                            "rest; the named configuration trades tokens/s for a prefetch that is always ahead"}
+                    "default_tokens_per_s": wl.batch * args.steps / t, "both_met_tokens_per_s": alts[pick]["tokens_per_s"] if ok else None,
+                    "note": "the default pipeline maximises tokens/s and misses the stall target: attention and prefetch "
+                            "share one HBM, attention takes its share first and then waits while the copy threads use "
+                            "the rest; the named configuration meets both targets at the lower tokens/s stated"}
             extra["kernels_alone"] = {
                 "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
@@ -520,13 +621,12 @@ def run_ours(args, wl):
     if not args.no_cpu_baseline and world == 1:
         import oracle
         oracle.build()
-        nseq = wl.batch
-        times, sample_tokens, threads = oracle_layer_sample(wl, args.seed, nseq, 3)
-        per = min(times)
-        cpu = {"value": oracle_tokens_per_s(wl, per, sample_tokens, tokens), "unit": UNIT, "cores": threads,
-               "kind": "oracle",
-               "sample": f"oracle gather + fp64 paged attention of 1 layer over the first {nseq} of {wl.batch} sequences "
-                         f"({sample_tokens} of {tokens} tokens, best of 3), scaled by tokens and by {wl.num_layers} layers"}
+        run, sample_tokens, threads = oracle_layer_runner(wl, args.seed)
+        run()                                                   # page the data in
+        step_s = min(oracle_step_seconds(run, wl.num_layers) for _ in range(2))
+        cpu = {"value": wl.batch / step_s, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"one whole step, best of 2: {wl.num_layers} x (oracle gather + fp64 paged attention of all "
+                         f"{wl.batch} sequences, {sample_tokens} tokens, on one layer's host data); {step_s:.2f} s per step"}
 
     value = job_value(wl.batch, world, args.steps, t)
     line = {
@@ -540,7 +640,7 @@ def run_ours(args, wl):
                    "parallelism": "replicas" if world > 1 else "single", "pipeline_mode": args.pipeline_mode,
                    "l2": "inputs larger than L2: every step streams %.1f GB of KV" % (step_bytes / 1e9)},
         "hbm_gbs_combined": step_bytes * world * args.steps / t / 1e9,
-        "roofline": roof, "cpu_baseline": cpu,
+        "roofline": roof, "cpu_baseline": cpu, "parity_checked": parity,
         "e2e": {"value": wl.batch * world / t_e2e_step, "unit": UNIT, "h2d_bytes_per_step": io_bytes,
                 "d2h_bytes_per_step": io_bytes, "ms_per_step": t_e2e_step * 1e3},
         "gpu_launches": int(launches), "clocks": clocks,

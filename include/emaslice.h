@@ -72,11 +72,19 @@ enum { SLICE_TIER_AUTO = 0, SLICE_TIER_LOCAL = 1, SLICE_TIER_LENT = 2 };
 enum {
   SLICE_FLAG_PROFILE = 1u,     /* record timing events around the kernels (slice_layer_times)     */
   SLICE_FLAG_TRACE = 2u,       /* per-CTA device-timer traces (slice_cta_trace)                    */
-  SLICE_FLAG_NULL_DEVICE = 4u, /* tables only: no CUDA call is made, no kernel is launched       */
-  SLICE_FLAG_TEST_WITHHOLD_Q = 8u /* test hook for the bounded waits: queries streamed in from pinned
-                                     host memory arrive, their arrival flags are never written, so
-                                     the kernel's wait for them runs out (about two seconds) and it
-                                     returns with SLICE_ETIMEOUT in slice_stats().device_status     */
+  SLICE_FLAG_NULL_DEVICE = 4u  /* tables only: no CUDA call is made, no kernel is launched       */
+};
+
+/* TEST HOOKS, not for callers: further bits of slice_config_t.flags with which the library's own
+ * tests make a failure happen on the host side, without faulting anything on the GPU. */
+enum {
+  SLICE_FLAG_TEST_WITHHOLD_Q = 8u, /* bounded waits: queries streamed in from pinned host memory
+                                      arrive, their arrival flags are never written, so the kernel's
+                                      wait for them runs out (about two seconds) and it returns with
+                                      SLICE_ETIMEOUT in slice_stats().device_status               */
+  SLICE_FLAG_TEST_FAIL_COPY = 16u  /* slice_reclaim / slice_reclaim_preempt: the step that enqueues
+                                      the migration reports failure like a failed CUDA call
+                                      (SLICE_ECUDA); the state must be left as it was              */
 };
 
 typedef struct {
@@ -140,8 +148,9 @@ typedef struct {
   uint64_t plans_built;          /* how often tables were re-resolved for a batch               */
   uint64_t kernel_launches;      /* kernels of this library launched so far                     */
   int32_t last_cuda_error;       /* cudaError_t of the last failed CUDA call, 0 if none         */
-  int32_t device_status;         /* 0, or SLICE_ETIMEOUT if a kernel gave up a bounded wait
-                                    (read back by slice_stats; the call synchronises nothing)   */
+  int32_t device_status;         /* 0, or SLICE_ETIMEOUT if a kernel gave up a bounded wait (a word in
+                                    mapped host memory that the kernels write: reading it makes no
+                                    CUDA call and waits for nothing)                            */
 } slice_stats_t;
 
 /* Section 4 (memory slice with a mapping table per user). Creates the allocator state and the
@@ -153,9 +162,9 @@ int slice_create(const slice_config_t* cfg, slice_t** out);
 /* Frees what slice_create made after waiting for the slice's outstanding work. */
 int slice_destroy(slice_t* s);
 
-/* Section 4.1: "first attempts to allocate from free memory" — appends n logical blocks to
- * sequence seq (created when absent). AUTO takes free local ids first and the lent part only when
- * local memory is exhausted; LOCAL / LENT force a tier (seeded placements). out_entries (host, n
+/* Section 4.1 (allocation tries the user's own free memory before anything else): appends n
+ * logical blocks to sequence seq (created when absent). AUTO takes free local ids first and the
+ * lent part only when local memory is exhausted; LOCAL / LENT force a tier (seeded placements). out_entries (host, n
  * entries, may be NULL) receives the new table entries. Errors: ENOSPC (nothing changes), EINVAL
  * (negative seq, bad hint, more than max_seqs sequences or max_blocks_per_seq blocks), ECAPPED
  * (n > 0 and a cap from an earlier preemption holds, see slice_preempt_seq; nothing changes). */
@@ -205,21 +214,29 @@ int paged_decode(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq,
  * tolerate the device-wide synchronisation an allocation brings, and under rules that forbid
  * allocator calls once initialisation is over. paged_decode_noalloc takes the same arguments,
  * computes the same result and orders itself on the streams the same way, but keeps the scratch in a
- * static device array built into the library: 8 MiB per GPU, held by every GPU that loads the
- * library until the process exits. It calls no cudaMalloc, cudaFree or other allocating routine.
+ * static device array built into the library: 8 MiB on every GPU on which a slice has been created
+ * (or this entry point called), held until the process exits. The call itself makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *   Set-up: slice_create (without SLICE_FLAG_NULL_DEVICE) does everything that has to happen once
+ *   per device, with that device current: it loads the part of the library that holds the array
+ *   (under CUDA's lazy loading this is the moment the 8 MiB are reserved), looks up the array's
+ *   device address and runs the attention kernels once on an empty batch. A first decode call
+ *   therefore finds nothing left to set up. Should the look-up not have happened for the current
+ *   device, the first call here does it; create slices, and make such a first call, outside any
+ *   stream capture.
+ *   Device: the call must be made with the slice's device current (the device that was current in
+ *   slice_create); otherwise it returns SLICE_EINVAL and launches nothing.
  *   Limit: this entry point splits the work statically (no stealing between CTAs), which needs one
  *   partial slot per (sequence, CTA range it touches) plus one per sequence, i.e. at most
  *   2 * nseq + CTAs slots; slots * num_q_heads * 528 bytes plus about 8 bytes per (sequence, KV head)
  *   and 8 per CTA must fit in 8 MiB; larger requests return SLICE_ESCRATCH
  *   and change nothing.
- *   First call on a device: looks up the array's device address (one-time set-up for that device,
- *   done with that device current). Make that first call outside any stream capture.
  *   Sharing: all calls, from every slice in the process, use the one array, and it keeps the last
  *   call's contents (its counters are cleared on the stream before every launch; the partial rows
  *   need no clearing: each call overwrites what it later reads). Two
  *   calls whose kernels may overlap on the GPU (different streams without an ordering between them)
  *   race on it; issue them on one stream or order them with events.
- * Errors: as paged_decode, plus SLICE_ESCRATCH. */
+ * Errors: as paged_decode, plus SLICE_ESCRATCH and SLICE_EINVAL (other device current). */
 int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, const void* q,
                          uint32_t num_q_heads, float sm_scale, void* out, float* lse_or_null, void* stream);
 
@@ -244,8 +261,9 @@ int slice_reclaim(slice_t* s, uint32_t take_blocks, uint64_t* out_n_migrated, vo
  *   victims     host, cap entries: the preempted sequence ids in eviction order; n_victims (host,
  *               may be NULL) their number; out_n_migrated as in slice_reclaim.
  * Every victim counts as a preemption by reclamation and, as in slice_preempt_seq, can set the cap.
- * Errors: EINVAL (slab_blocks == 0, or cap smaller than the number of victims: nothing changes),
- * ECUDA. */
+ * Errors: EINVAL (slab_blocks == 0, or cap smaller than the number of victims), ECUDA (the
+ * migration could not be enqueued). After an error nothing has changed: no request was evicted, no
+ * counter moved, no cap was set. */
 int slice_reclaim_preempt(slice_t* s, uint32_t take_blocks, uint32_t slab_blocks, int32_t* victims, uint32_t cap,
                           uint32_t* n_victims, uint64_t* out_n_migrated, void* stream);
 

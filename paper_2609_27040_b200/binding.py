@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libemaslice.so")
 OK, EINVAL, ENOSPC, ESTAGING, ESTALE, ECUDA, ETIMEOUT, ESTATE, ESCRATCH, ECAPPED = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 PREEMPT_OOM, PREEMPT_RECLAIM = 1, 2
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
-FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE, FLAG_TEST_WITHHOLD_Q = 1, 2, 4, 8
+FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE = 1, 2, 4
+FLAG_TEST_WITHHOLD_Q, FLAG_TEST_FAIL_COPY = 8, 16      # test hooks (see include/emaslice.h)
 COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
 TAKE_ALL = 0xFFFFFFFF
 

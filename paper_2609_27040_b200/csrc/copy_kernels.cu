@@ -141,13 +141,16 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
   if (d.n == 0 || d.nlayers == 0) return cudaSuccess;
   if (kind == kCopyDefault) kind = kCopyVector;
   if (kind == kCopyBulk) {
-    static bool attr_set = false;
+    static bool attr_set[64] = {};  // the attribute is a property of the function on one device
     const size_t smem = static_cast<size_t>(kStages) * kChunk;
-    if (!attr_set) {
-      cudaError_t e = cudaFuncSetAttribute(copy_blocks_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(smem));
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+      e = cudaFuncSetAttribute(copy_blocks_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      attr_set = true;
+      attr_set[dev] = true;
     }
     const uint64_t pieces = (d.block_bytes + kChunk - 1) / kChunk;
     const uint64_t total = static_cast<uint64_t>(d.n) * d.nlayers * pieces;

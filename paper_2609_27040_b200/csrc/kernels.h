@@ -88,7 +88,7 @@ struct LayerParams {
   void* out;
   uint64_t io_layer_stride;     // bytes from one layer's q / out to the next
   const uint32_t* q_ready;      // optional: q arrives while the launch runs; layer l's rows may be read once
-  uint32_t q_ready_epoch;       //   q_ready[l / q_ready_layers] == q_ready_epoch (written by the copy that brought them)
+  uint32_t q_ready_epoch;       //   q_ready[l / q_ready_layers] >= q_ready_epoch (written after the rows themselves)
   uint32_t q_ready_layers;
   float* lse;                   // [nseq][Hq] or NULL (single-layer launches only)
   float* part_o;                // [slots][Hq][128] unnormalised partial outputs; layers alternate
@@ -130,7 +130,10 @@ cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream);
 // noalloc.cu: the same launch with partials and counters in a static device array (part_o,
 // part_ml, counters of p are ignored). static_scratch_needed() > static_scratch_bytes() must be
 // rejected by the caller.
+// static_scratch_setup(): initialisation-time set-up on the current device (module load = the
+// array's reservation, address look-up, one empty launch of the kernel variant for G).
 size_t static_scratch_bytes();
+cudaError_t static_scratch_setup(uint32_t Hkv, uint32_t G, uint32_t ncta);
 size_t static_scratch_needed(uint32_t slots, uint32_t Hq, uint32_t nseq, uint32_t Hkv, uint32_t ncta);
 cudaError_t launch_layer_static(LayerParams p, uint32_t slots, cudaStream_t stream);
 

@@ -192,13 +192,14 @@ __device__ __forceinline__ float* part_ml_of(const LayerParams& p, uint32_t li) 
   return p.part_ml + (li & (p.part_buffers - 1u)) * p.part_ml_stride;
 }
 
-// Bounded wait until a device word written by another CTA equals `value`.
+// Bounded wait until a device word written by another CTA equals `value`. The reads are acquires:
+// what the writer did before its release of the word is visible after a successful wait.
 __device__ __forceinline__ bool wait_counter_eq(const uint32_t* word, uint32_t value, int* status) {
-  if (__ldcg(word) == value) return true;
+  if (ptx::ld_acquire_gpu(word) == value) return true;
   const uint64_t t0 = ptx::global_timer_ns();
-  while (__ldcg(word) != value) {
+  while (ptx::ld_acquire_gpu(word) != value) {
     if (ptx::global_timer_ns() - t0 > kWaitNs) {
-      if (status) atomicExch(status, kDevTimeout);
+      ptx::report_status(status, kDevTimeout);
       return false;
     }
     __nanosleep(64);
@@ -208,11 +209,11 @@ __device__ __forceinline__ bool wait_counter_eq(const uint32_t* word, uint32_t v
 
 // Bounded wait until a device counter written by other CTAs reaches `target`.
 __device__ __forceinline__ bool wait_counter(const uint32_t* cnt, uint32_t target, int* status) {
-  if (__ldcg(cnt) >= target) return true;
+  if (ptx::ld_acquire_gpu(cnt) >= target) return true;
   const uint64_t t0 = ptx::global_timer_ns();
-  while (__ldcg(cnt) < target) {
+  while (ptx::ld_acquire_gpu(cnt) < target) {
     if (ptx::global_timer_ns() - t0 > kWaitNs) {
-      if (status) atomicExch(status, kDevTimeout);
+      ptx::report_status(status, kDevTimeout);
       return false;
     }
     __nanosleep(128);
@@ -306,8 +307,11 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       ++nclaims;
       if (!have_rdy) {
         rdy = epoch;
-        if (check_ready && lane < c.e - c.b && my < 0) rdy = __ldcg(ready + static_cast<uint32_t>(~my));
+        if (check_ready && lane < c.e - c.b && my < 0) rdy = ptx::ld_acquire_gpu(ready + static_cast<uint32_t>(~my));
       }
+      // The flags were read (acquired) one per lane and lane 0 issues the copies: the warp barrier
+      // carries every lane's acquire over to it.
+      __syncwarp();
       uint32_t at = c.b;
       while (at < c.e && ok) {
         seek(at, at == c.b ? hint : kSentinel);
@@ -327,7 +331,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           }
           const uint32_t base = p.seq_slot_base[seq], cap = p.seq_slot_base[seq + 1] - base;
           if (k >= cap) {  // cannot happen with the host's sizing; never write outside the slots
-            if (lane == 0 && p.status) atomicExch(p.status, kDevTimeout - 1);
+            if (lane == 0) ptx::report_status(p.status, kDevTimeout - 1);
             k = cap - 1;
           }
           slot_flag = (base + k) | kNewRun;
@@ -363,6 +367,10 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
               // it through the asynchronous proxy. Without this fence the copy can overtake those
               // reads: seen as rare wrong V tiles in launches spanning several layers.
               ptx::fence_proxy_async();
+              // A staged block was written by another CTA's bulk stores and announced through its
+              // ready flag (release / acquire above): the bulk load reads it through the
+              // asynchronous proxy, which the acquire alone does not cover.
+              if (check_ready && e < 0 && plane == 0) ptx::fence_proxy_async_global();
               ptx::mbar_arrive_expect_tx(full, plane_bytes);
               // One request per plane: an SM streams far faster through few large bulk copies than
               // through many small ones.
@@ -403,7 +411,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       my = 0;
       if (lane < n) my = have ? sm.own_res[b + lane - r0] : p.resolved[b + lane];
       rdy = epoch;
-      if (have && check_ready && lane < n && my < 0) rdy = __ldcg(ready + static_cast<uint32_t>(~my));
+      if (have && check_ready && lane < n && my < 0) rdy = ptx::ld_acquire_gpu(ready + static_cast<uint32_t>(~my));
     };
 
     // Before the last layer of a launch a CTA that is out of own work does better to start on the
@@ -714,9 +722,21 @@ __device__ __forceinline__ void finish_run(const LayerParams& p, const Smem& sm,
       // Up to Hkv warps may pass this check at once, hence the margin.
       const uint32_t t = atomicAdd(&sm.mq[kMqTail], 1u);
       const uint64_t t0 = ptx::global_timer_ns();
-      while (mq[t % kMq] != kMqEmpty && ptx::global_timer_ns() - t0 < kWaitNs) __nanosleep(64);
-      mq[t % kMq] = (li << 24) | (seq << 4) | g;
-      queued = 1;
+      bool slot_free = true;
+      while (mq[t % kMq] != kMqEmpty) {
+        if (ptx::global_timer_ns() - t0 > kWaitNs) {  // the merge warp is gone or stuck: report, merge in line
+          ptx::report_status(p.status, kDevTimeout);
+          slot_free = false;
+          break;
+        }
+        __nanosleep(64);
+      }
+      // The ticket is spent either way; a merge warp that draws it finds the slot still holding the
+      // older request (or nothing) and this warp does the merge itself.
+      if (slot_free) {
+        mq[t % kMq] = (li << 24) | (seq << 4) | g;
+        queued = 1;
+      }
     }
   }
   queued = __shfl_sync(0xffffffffu, queued, 0);
@@ -779,7 +799,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
           const uint64_t t0 = ptx::global_timer_ns();
           while ((v = mq[hd % kMq]) == kMqEmpty) {  // its writer holds the ticket already
             if (ptx::global_timer_ns() - t0 > kWaitNs) {
-              if (p.status) atomicExch(p.status, kDevTimeout);
+              ptx::report_status(p.status, kDevTimeout);
               leave = true;
               break;
             }
@@ -821,7 +841,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
             const uint64_t t0 = ptx::global_timer_ns();
             while ((job = ptx::ld_acquire_gpu(e)) == 0) {
               if (ptx::global_timer_ns() - t0 > kWaitNs) {
-                if (p.status) atomicExch(p.status, kDevTimeout);
+                ptx::report_status(p.status, kDevTimeout);
                 leave = true;
                 break;
               }
@@ -1138,8 +1158,10 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       if (!ready) return;
       const uint32_t units = complete / pieces;
       if (units > reported) {
-        __threadfence();
-        for (; reported < units; ++reported) ready[my_pos[reported % 16]] = epoch;
+        // The unit's bulk stores are complete (wait_group); they went through the asynchronous
+        // proxy, the flag goes through the generic one: order the two, then publish with a release.
+        ptx::fence_proxy_async_global();
+        for (; reported < units; ++reported) ptx::st_release_gpu(ready + my_pos[reported % 16], epoch);
       }
     };
 

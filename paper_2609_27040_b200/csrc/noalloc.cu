@@ -9,11 +9,15 @@
 // For them this file provides the same two launches with the scratch placed in a file-scope
 // `static __device__` array of fixed size.
 //
-// The array occupies kStaticScratchBytes on every GPU that loads the library, until the process
-// exits. In host code the array's name is only a host-side stand-in, not a device address, so the
-// address handed to the kernels is looked up with cudaGetSymbolAddress: once per device, on the
-// first call made with that device current. All calls share the one array and it keeps whatever the
-// last call left in it; two calls whose kernels overlap on the GPU would race on it.
+// The array occupies kStaticScratchBytes on every GPU on which this part of the library has been
+// loaded, until the process exits. With CUDA's lazy module loading (the default) that load, and
+// with it the reservation of the array, happens at the first use of a symbol of this file on the
+// device; slice_create does that use (static_scratch_setup below), so that it falls into
+// initialisation and not into the first decode call. In host code the array's name is only a
+// host-side stand-in, not a device address, so the address handed to the kernels is looked up with
+// cudaGetSymbolAddress: once per device, with that device current. All calls share the one array
+// and it keeps whatever the last call left in it; two calls whose kernels overlap on the GPU would
+// race on it.
 #include "kernels.h"
 
 namespace {
@@ -23,8 +27,9 @@ constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-// Device addresses of g_static_scratch, filled in lazily per device.
+// Device addresses of g_static_scratch, filled in once per device.
 void* g_scratch_addr[kMaxDevices] = {};
+bool g_warmed[kMaxDevices][2] = {};  // [device][tensor-core variant]: an empty launch has been made
 
 inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
@@ -54,6 +59,40 @@ cudaError_t static_scratch_address(void** out) {
     g_scratch_addr[dev] = p;
   }
   *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+// Initialisation-time set-up for the device that is current (called by slice_create): loads this
+// module on the device, which is what reserves the array, resolves the array's address, and makes
+// one empty launch of the attention kernel variant that serves `G` query heads per KV head, so that
+// whatever the driver sets up at a kernel's first launch (its code, the thread stacks) is in place
+// before the first decode call rather than inside it.
+cudaError_t static_scratch_setup(uint32_t Hkv, uint32_t G, uint32_t ncta) {
+  void* base = nullptr;
+  cudaError_t e = static_scratch_address(&base);
+  if (e != cudaSuccess) return e;
+  int dev = 0;
+  e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const int variant = G == 1 ? 0 : 1;
+  if (g_warmed[dev][variant]) return cudaSuccess;
+  LayerParams p{};  // no blocks, no sequences, no gather: every role finds nothing to do and returns
+  p.num_layers = 1;
+  p.ring_slots = 1;
+  p.per = 1;
+  p.merge_inline = 1;
+  p.part_buffers = 1;
+  p.ncta = ncta;
+  p.Hkv = Hkv;
+  p.G = G;
+  p.Hq = Hkv * G;
+  p.counters = static_cast<uint32_t*>(base);
+  for (uint32_t i = 0; i < kMaxStepLayers; ++i) p.gather_target[i] = p.gather_after[i] = -1;
+  e = launch_layer(p, nullptr);
+  if (e != cudaSuccess) return e;
+  e = cudaStreamSynchronize(nullptr);
+  if (e != cudaSuccess) return e;
+  g_warmed[dev][variant] = true;
   return cudaSuccess;
 }
 

@@ -26,6 +26,14 @@ __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// Orders this thread's generic-proxy view of GLOBAL memory with its asynchronous-proxy operations
+// (bulk copies that read or wrote global memory): after an acquire that learned of another CTA's
+// bulk stores and before the bulk load that reads them; after a completed bulk store group and
+// before the release that announces it.
+__device__ __forceinline__ void fence_proxy_async_global() {
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -52,6 +60,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+// Records `code` in the library's status word (mapped host memory, or NULL): a plain store, which
+// needs no atomic support on the way to the host; the codes written are all failures and any one
+// of them is enough for the caller.
+__device__ __forceinline__ void report_status(int* status, int code) {
+  if (status) *reinterpret_cast<volatile int*>(status) = code;
+}
+
 // Bounded wait: gives up after about two seconds, records the failure in *status and returns
 // false, so that a lost copy or a missing arrival can never hang the GPU.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code) {
@@ -60,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
   uint32_t polls = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++polls & 0x3FFu) == 0 && global_timer_ns() - t0 > 2000000000ull) {
-      if (status) atomicExch(status, code);
+      report_status(status, code);
       return false;
     }
   }

@@ -88,6 +88,7 @@ struct ema_slice {
   bool null_dev = false, profile = false, trace = false;
   uint64_t block_bytes = 0;
   uint64_t local_ls = 0, local_bs = 0, lent_ls = 0, lent_bs = 0, slot_bytes = 0;
+  int device = -1;  // the CUDA device the slice was created on
   int num_sms = 148;
   uint32_t ncta = 148;
   bool steal = true;
@@ -115,7 +116,7 @@ struct ema_slice {
   uint32_t* cnt_dev = nullptr;  // [num_layers][cnt_stride] device counters of the layer kernel
   uint32_t* ready_dev = nullptr;  // [ring_slots][staging_blocks_per_slot] ready flags (epochs)
   uint32_t epoch = 1;
-  int* dev_status = nullptr;
+  int* dev_status = nullptr;  // mapped pinned host word: kernels record a failed bounded wait, the host reads it
   // reclaim
   int32_t* reclaim_host = nullptr;
   int32_t* reclaim_dev = nullptr;
@@ -597,9 +598,14 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
   for (uint32_t i = 0; i < p->nseq; ++i)
     if (lens[i] == 0) return SLICE_EINVAL;
-  if (static_scratch &&
-      ema::static_scratch_needed(p->slots_static, Hq, p->nseq, Hkv, s->ncta) > ema::static_scratch_bytes())
-    return SLICE_ESCRATCH;
+  if (static_scratch) {
+    if (ema::static_scratch_needed(p->slots_static, Hq, p->nseq, Hkv, s->ncta) > ema::static_scratch_bytes())
+      return SLICE_ESCRATCH;
+    // The array's address belongs to the device the slice lives on; with another device current the
+    // launch would be given another GPU's array.
+    int cur = -1;
+    if (!s->null_dev && (cudaGetDevice(&cur) != cudaSuccess || cur != s->device)) return SLICE_EINVAL;
+  }
   const uint32_t slot = layer % R;
   SlotState& sl = s->slots[slot];
   if (p->k && !staged(s, layer, p)) return SLICE_ESTALE;
@@ -780,7 +786,7 @@ void destroy_impl(ema_slice* s) {
     if (s->part_ml) cudaFree(s->part_ml);
     if (s->cnt_dev) cudaFree(s->cnt_dev);
     if (s->ready_dev) cudaFree(s->ready_dev);
-    if (s->dev_status) cudaFree(s->dev_status);
+    if (s->dev_status) cudaFreeHost(s->dev_status);
     if (s->reclaim_host) cudaFreeHost(s->reclaim_host);
     if (s->reclaim_dev) cudaFree(s->reclaim_dev);
     if (s->reclaim_done) cudaEventDestroy(s->reclaim_done);
@@ -870,9 +876,19 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return fail(SLICE_ECUDA);
+    s->device = dev;
     if (ema::layer_setup() != cudaSuccess) return fail(SLICE_ECUDA);
   }
   s->ncta = cfg->decode_ctas ? cfg->decode_ctas : static_cast<uint32_t>(s->num_sms);
+  if (!null_dev) {
+    // paged_decode_noalloc must find nothing left to set up when it is first called: load its module
+    // (which reserves the static scratch array on this device), look the array up and run both
+    // variants of the attention kernel once, empty.
+    const uint32_t warm_ctas = std::min(s->ncta, static_cast<uint32_t>(s->num_sms));
+    if (ema::static_scratch_setup(cfg->num_kv_heads, 1, warm_ctas) != cudaSuccess ||
+        ema::static_scratch_setup(cfg->num_kv_heads, 2, warm_ctas) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+  }
   const size_t cap = plan_capacity(s);
   for (Plan& p : s->plans) {
     p.cap = cap;
@@ -893,8 +909,8 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
           cudaEventCreateWithFlags(&sl.attn_done, cudaEventDisableTiming) != cudaSuccess)
         return fail(SLICE_ECUDA);
     }
-    if (cudaMalloc(reinterpret_cast<void**>(&s->dev_status), 256) != cudaSuccess) return fail(SLICE_ECUDA);
-    if (cudaMemset(s->dev_status, 0, 256) != cudaSuccess) return fail(SLICE_ECUDA);
+    if (cudaHostAlloc(reinterpret_cast<void**>(&s->dev_status), 256, cudaHostAllocMapped) != cudaSuccess) return fail(SLICE_ECUDA);
+    std::memset(s->dev_status, 0, 256);
     s->cnt_stride = align_up(ema::layer_counter_words(s->ncta, cfg->max_seqs, cfg->num_kv_heads), 64);
     const size_t cnt_words = static_cast<size_t>(cfg->num_layers) * s->cnt_stride;
     if (cudaMalloc(reinterpret_cast<void**>(&s->cnt_dev), cnt_words * sizeof(uint32_t)) != cudaSuccess ||
@@ -1070,6 +1086,11 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
   for (size_t k = 0; k < n_local; ++k) dst[k] = s->free_local[s->free_local.size() - 1 - k];
   for (size_t k = 0; k < n_lent; ++k) dst[n_local + k] = ~sorted_below[k];
 
+  // Test hook: the step that enqueues the migration fails, as a CUDA call might; nothing is committed.
+  if ((s->cfg.flags & SLICE_FLAG_TEST_FAIL_COPY) && !victims.empty()) {
+    s->st.last_cuda_error = static_cast<int>(cudaErrorUnknown);
+    return SLICE_ECUDA;
+  }
   if (!s->null_dev && !victims.empty()) {
     // Everything outstanding on the slice's streams must finish before blocks move.
     int rc = ensure_stream(s, stream);
@@ -1234,15 +1255,46 @@ int slice_reclaim_preempt(slice_t* s, uint32_t take, uint32_t slab_blocks, int32
   }
   if (order.size() > cap || (!order.empty() && !victims)) return SLICE_EINVAL;
   const uint32_t held = blocks_held(s);
-  for (size_t k = 0; k < order.size(); ++k) {
-    slice_free_seq(s, order[k]);
-    victims[k] = order[k];
-    ++s->preempt_reclaim;
+  // The migration plans its destinations on the state the evictions leave, and its enqueue can still
+  // fail (a CUDA error): the evictions are therefore made on the live state with everything they
+  // touch kept aside, and put back if the migration does not go through. Nothing is reported to the
+  // caller, counted or capped before it has.
+  struct Saved {
+    std::vector<int32_t> free_local, free_lent;
+    std::vector<std::pair<int32_t, Seq>> seqs;
+    uint64_t version;
+  } keep;
+  if (!order.empty()) {
+    keep.free_local = s->free_local;
+    keep.free_lent = s->free_lent;
+    keep.version = s->version;
+    for (int32_t q : order) keep.seqs.emplace_back(q, s->seqs[q]);
+    for (int32_t q : order) slice_free_seq(s, q);
   }
-  if (n_victims) *n_victims = static_cast<uint32_t>(order.size());
   const int rc = slice_reclaim(s, take, out_n_migrated, stream);
+  if (rc != SLICE_OK) {
+    if (!order.empty()) {
+      s->free_local.swap(keep.free_local);
+      s->free_lent.swap(keep.free_lent);
+      for (auto& kv : keep.seqs) {
+        const std::vector<int32_t>& t = kv.second.table;
+        for (size_t b = 0; b < t.size(); ++b) {
+          const int32_t e = t[b];
+          (e >= 0 ? s->owner_local[e] : s->owner_lent[~e]) = Owner{kv.first, static_cast<int32_t>(b)};
+        }
+        s->seqs[kv.first] = std::move(kv.second);
+      }
+      // The plans built meanwhile saw none of this; a new version keeps them from being reused.
+      s->version = keep.version;
+      bump_version(s);
+    }
+    return rc;
+  }
+  for (size_t k = 0; k < order.size(); ++k) victims[k] = order[k];
+  s->preempt_reclaim += order.size();
+  if (n_victims) *n_victims = static_cast<uint32_t>(order.size());
   if (!order.empty()) cap_after_reclaim_preemption(s, held);
-  return rc;
+  return SLICE_OK;
 }
 
 int slice_preempt_stats(slice_t* s, slice_preempt_stats_t* out) {
@@ -1538,11 +1590,8 @@ int slice_stats(slice_t* s, slice_stats_t* out) {
   s->st.lent_used = s->lent_cap - s->st.lent_free;
   s->st.lent_capacity = s->lent_cap;
   s->st.num_seqs = static_cast<uint32_t>(s->seqs.size());
-  if (!s->null_dev && s->dev_status) {
-    // A plain blocking copy of one word: reports what finished kernels have recorded.
-    int v = 0;
-    if (cudaMemcpy(&v, s->dev_status, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess) s->st.device_status = v;
-  }
+  // The status word lives in mapped host memory: reading it costs no CUDA call and waits for nothing.
+  if (!s->null_dev && s->dev_status) s->st.device_status = *static_cast<volatile int*>(s->dev_status);
   *out = s->st;
   return SLICE_OK;
 }
@@ -1596,13 +1645,12 @@ int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_ba
                       uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream) {
   if (!dst_base || !src_base || (block_bytes & 15u) || block_bytes == 0 || kind > 2) return SLICE_EINVAL;
   if ((reinterpret_cast<uintptr_t>(dst_base) | reinterpret_cast<uintptr_t>(src_base)) & 15u) return SLICE_EINVAL;
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return SLICE_ECUDA;
-  }
+  static int sms_of[64] = {};  // per device
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLICE_ECUDA;
+  if (!sms_of[dev] && cudaDeviceGetAttribute(&sms_of[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SLICE_ECUDA;
+  const int sms = sms_of[dev];
   ema::CopyDesc d{};
   d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(src_base);
   d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(dst_base);

@@ -1,0 +1,135 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The Llama-3-8B- and 70B-shaped batches are decoded with the default knobs (one persistent launch
+per pass, one CTA per SM, work stealing). At these sizes a CTA's range is longer than 48 blocks, so
+finished sequences are queued to the CTA's merge warp instead of being merged in line, and with 9
+(6, 5) layers every buffer of split-KV partials is reused, some twice, behind the cross-CTA wait on
+the merges of the layer that used it last: the combination that nearly every timed layer of the
+benchmark runs. Everything is compared with the CPU oracle: resolved tables and staged bytes in
+full, attention for every sequence and every head of the first, a middle and the last layer.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_27040_b200 import binding as B
+from paper_2609_27040_b200 import build as build_mod
+from paper_2609_27040_b200 import synth
+from tests.helpers import attention_close
+
+pytestmark = pytest.mark.gpu
+
+ATOL = RTOL = 1e-2   # bf16 attention tolerance of the benchmark definition
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+
+
+def _bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class FullBatch:
+    """Arenas, slice and oracle state of one full-size workload restricted to L layers (block ids
+    and tables do not depend on the layer, so a one-layer oracle serves every layer's bytes)."""
+
+    def __init__(self, name: str, L: int, seed: int = 0, **kw):
+        self.wl = wl = synth.WORKLOADS[name]
+        self.L = L
+        self.pl = pl = synth.make_placement(wl, seed, slack_blocks=64)
+        gen = torch.Generator(device="cuda").manual_seed(seed)
+        shape = (2, wl.block_tokens, wl.num_kv_heads, wl.head_dim)
+        bf = torch.bfloat16
+        self.local = torch.empty((L, pl.local_blocks) + shape, device="cuda", dtype=bf).normal_(generator=gen)
+        self.lent = torch.empty((L, pl.lent_blocks) + shape, device="cuda", dtype=bf).normal_(generator=gen)
+        self.staging = torch.zeros((2, pl.staging_blocks) + shape, device="cuda", dtype=bf)
+        self.q = torch.empty((L, wl.batch, wl.num_q_heads, wl.head_dim), device="cuda", dtype=bf).normal_(generator=gen)
+        self.out = torch.zeros_like(self.q)
+        self.max_blocks = 520
+        self.s = B.Slice(L, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks, local=self.local,
+                         lent=self.lent, staging=self.staging, max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks,
+                         local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order, **kw)
+        self.orc = oracle.OracleSlice(1, wl.block_tokens, wl.block_bytes, pl.local_blocks, pl.lent_blocks, pl.lent_blocks,
+                                      1, pl.staging_blocks, max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks,
+                                      local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
+        for i, hints in enumerate(pl.hints):
+            for h in hints:
+                assert self.s.slice_alloc_blocks(i, 1, int(h))[0] == 0 and self.orc.alloc_blocks(i, 1, int(h))[0] == 0
+            assert self.s.slice_set_seq_len(i, int(pl.lengths[i])) == 0 and self.orc.set_seq_len(i, int(pl.lengths[i])) == 0
+        self.seqs = np.arange(wl.batch, dtype=np.int32)
+        self.lens = np.asarray(pl.lengths, np.uint32)
+        self.main, self.side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+        self.scale = 1.0 / np.sqrt(wl.head_dim)
+
+    def decode_passes(self, n: int):
+        for _ in range(n):
+            assert self.s.slice_decode_step(self.seqs, self.q, self.wl.num_q_heads, self.scale, self.out, False, True,
+                                            self.main, self.side) == B.OK
+        torch.cuda.synchronize()
+        st = self.s.slice_stats()
+        assert st["device_status"] == 0 and st["last_cuda_error"] == 0
+        return st
+
+    def check_tables(self):
+        rc, resolved, k = self.orc.gather(0, self.seqs, None, None)
+        rc2, res_gpu, k_gpu = self.s.slice_get_resolved(self.seqs)
+        assert rc == rc2 == 0 and k == k_gpu == self.pl.staging_blocks
+        assert (resolved == res_gpu).all()
+        for i in range(self.wl.batch):
+            assert self.s.slice_get_block_table(i)[1].tolist() == self.orc.block_table(i)[1].tolist()
+        return resolved, k
+
+    def check_staged_bytes(self, k: int):
+        """The two ring slots, in full, against the lent arena read through the oracle's tables (on the
+        device), and slot 0 once more against the oracle's own gather (on the host)."""
+        L = self.L
+        ids = torch.tensor([~int(e) for i in range(self.wl.batch)
+                            for e in self.orc.block_table(i)[1][: synth.blocks_for(self.pl.lengths[i])] if e < 0], device="cuda")
+        last_odd = L - 1 if (L - 1) % 2 else L - 2
+        for layer, slot in ((0, 0), (last_odd, 1)):        # slot 0 was refilled with layer 0 for the next pass
+            assert torch.equal(self.staging[slot, :k], self.lent[layer].index_select(0, ids)), (layer, slot)
+        lent0 = _bits(B.kv_block_swizzle(self.lent[0]))
+        staged = np.zeros((1, k) + lent0.shape[1:], np.uint16)
+        rc, _, k2 = self.orc.gather(0, self.seqs, lent0[None], staged)
+        assert rc == 0 and k2 == k
+        assert (_bits(B.kv_block_swizzle(self.staging[0, :k])) == staged[0]).all()
+
+    def check_attention_in_full(self, layer: int, resolved: np.ndarray, k: int):
+        """Every sequence and every query head of `layer`: the oracle gathers the layer's lent blocks
+        into a host staging slot and attends in fp64 through the resolved table."""
+        wl = self.wl
+        local = _bits(B.kv_block_swizzle(self.local[layer]))       # block format -> canonical token rows
+        lent = _bits(B.kv_block_swizzle(self.lent[layer]))
+        staged = np.zeros((1, max(k, 1)) + lent.shape[1:], np.uint16)
+        assert self.orc.gather(0, self.seqs, lent[None], staged)[0] == 0
+        rc, ref, _ = oracle.paged_attention(_bits(self.q[layer]), local, staged[0], resolved, self.lens, wl.num_q_heads,
+                                            wl.num_kv_heads, wl.head_dim, wl.block_tokens, self.scale, want_lse=False)
+        assert rc == 0
+        got = self.out[layer].double().cpu().numpy()
+        assert np.isfinite(got).all()
+        ok, max_abs, max_rel = attention_close(got, ref, ATOL, RTOL)
+        assert ok, (layer, max_abs, max_rel)
+        return max_abs
+
+
+@pytest.mark.parametrize("name,L,kw", [
+    ("llama3_8b_decode", 9, {}),                              # four partial buffers, each reused at least once
+    ("llama3_70b_decode", 6, {}),
+    ("llama3_8b_decode", 5, {"prefetch_priority": 1}),        # two partial buffers, reused twice
+])
+def test_timed_launch_configuration_matches_oracle_in_full(name, L, kw):
+    fb = FullBatch(name, L, **kw)
+    per = -(-fb.pl.total_blocks // 148)
+    assert per > 48                                            # merges are queued, not done in line
+    st = fb.decode_passes(2)
+    assert st["kernel_launches"] <= 5                          # one launch per pass, plus the gathers of layer 0
+                                                               # (priming; refill of a slot the last layer shares)
+    resolved, k = fb.check_tables()
+    fb.check_staged_bytes(k)
+    mid = max(4, L // 2) if L > 5 else 3
+    for layer in sorted({0, mid, L - 1}):
+        fb.check_attention_in_full(layer, resolved, k)
+    fb.s.close()

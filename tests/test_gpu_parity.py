@@ -210,14 +210,13 @@ def test_few_long_sequences_share_their_merges(case, mode):
     layer = 2
     rc, resolved, _ = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
     out = torch.zeros_like(g.q[layer])
-    rc = g.s.paged_decode_noalloc(layer, sc.seq_ids, g.q[layer], sc.Hq, float(sc.sm_scale), out, None, g.main)
-    assert rc in (B.OK, B.ESCRATCH)
-    if rc == B.OK:
-        torch.cuda.synchronize()
-        g.device_ok()
-        _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % sc.wl.ring_slots], resolved,
-                                           sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
-        assert attention_close(_bf16_to_f64(out), ref, ATOL, RTOL)[0]
+    # at most 150 partial slots x 8 query heads x 528 B: far inside the 8 MiB array
+    assert g.s.paged_decode_noalloc(layer, sc.seq_ids, g.q[layer], sc.Hq, float(sc.sm_scale), out, None, g.main) == B.OK
+    torch.cuda.synchronize()
+    g.device_ok()
+    _, ref, _ = oracle.paged_attention(sc.q[layer], sc.local[layer], sc.staging[layer % sc.wl.ring_slots], resolved,
+                                       sc.lengths(), sc.Hq, sc.Hkv, sc.D, sc.T, sc.sm_scale)
+    assert attention_close(_bf16_to_f64(out), ref, ATOL, RTOL)[0]
 
 
 def test_many_different_batches_rotate_the_plan_buffers():

@@ -272,6 +272,64 @@ def test_preemption_calls_match_oracle_state_machine(seed):
     s.close()
 
 
+def _snapshot(s: B.Slice, seqs):
+    return ([(q,) + tuple(x.tolist() if hasattr(x, "tolist") else x for x in s.slice_get_block_table(q)) for q in seqs],
+            s.slice_get_free_stack(B.TIER_LOCAL).tolist(), s.slice_get_free_stack(B.TIER_LENT).tolist(),
+            s.slice_preempt_stats(), {k: v for k, v in s.slice_stats().items() if k != "last_cuda_error"})
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_failed_migration_leaves_reclaim_and_preemption_uncommitted(seed):
+    """Injected on the host (a test hook makes the step that enqueues the migration report failure,
+    as a failed CUDA call would): slice_reclaim and slice_reclaim_preempt return ECUDA and tables,
+    free lists, the evicted requests, counters and the cap are exactly as before; a twin slice
+    without the hook, fed the same calls, shows what the same request does when the copy goes
+    through (when nothing has to migrate there is no copy to fail, and both succeed alike)."""
+    rng = np.random.default_rng(40 + seed)
+    LB, RB, PH = 6, 16, 16
+    lo, ro = synth.free_order(rng, LB), synth.free_order(rng, PH)
+    mk = lambda flags: B.Slice(2, 8, LB, RB, 16, lent_blocks_physical=PH, max_seqs=8, max_blocks_per_seq=8,
+                               flags=B.FLAG_NULL_DEVICE | flags, local_free_order=lo, lent_free_order=ro)
+    seqs = list(range(6))
+    lens = [16 * (4 if q < 4 else 3) - int(rng.integers(0, 16)) for q in seqs]
+    failed_with_victims = 0
+    for take in range(3, 12):
+        bad, good = mk(B.FLAG_TEST_FAIL_COPY), mk(0)
+        for s in (bad, good):
+            assert s.slice_set_preempt_window(50) == B.OK and s.slice_set_time(3) == B.OK
+            for q in seqs:                                  # fill both parts completely
+                assert s.slice_alloc_blocks(q, 4 if q < 4 else 3, B.TIER_AUTO)[0] == B.OK
+                assert s.slice_set_seq_len(q, lens[q]) == B.OK
+        before = _snapshot(bad, seqs)
+        assert before == _snapshot(good, seqs)
+        assert good.slice_reclaim(take)[0] == B.ENOSPC and bad.slice_reclaim(take)[0] == B.ENOSPC   # no room
+        assert _snapshot(bad, seqs) == before
+        rc_g, victims_g, mig_g = good.slice_reclaim_preempt(take, 4)
+        assert rc_g == B.OK and len(victims_g) > 0
+        rc, victims, mig = bad.slice_reclaim_preempt(take, 4)
+        if mig_g > 0:                                       # something had to be copied: the copy "fails"
+            assert rc == B.ECUDA and victims == [] and mig == 0
+            assert _snapshot(bad, seqs) == before           # nobody evicted, nothing counted, no cap
+            assert bad.slice_stats()["last_cuda_error"] != 0
+            assert bad.slice_get_resolved(seqs)[0] == B.OK  # and the state is still usable
+            failed_with_victims += 1
+        else:
+            assert rc == B.OK and victims == victims_g
+            live = [q for q in seqs if q not in victims]
+            assert _snapshot(bad, live) == _snapshot(good, live)
+        bad.close()
+        good.close()
+    assert failed_with_victims >= 2
+    # a plain migration that has room fails the same way and commits nothing
+    bad = mk(B.FLAG_TEST_FAIL_COPY)
+    for q in seqs[:4]:
+        assert bad.slice_alloc_blocks(q, 1, B.TIER_LENT)[0] == B.OK and bad.slice_set_seq_len(q, 14) == B.OK
+    before = _snapshot(bad, seqs[:4])
+    assert bad.slice_reclaim(B.TAKE_ALL)[0] == B.ECUDA
+    assert _snapshot(bad, seqs[:4]) == before
+    bad.close()
+
+
 def test_preemption_bad_arguments():
     s = _null_slice(2, 8, 4, 4, 4, 4, 4, 8)
     assert s.slice_reclaim_preempt(2, 0)[0] == B.EINVAL
