@@ -544,6 +544,66 @@ def run_ours(args, wl):
                                   "note": "traced run (a few per cent slower than an untraced one)"}
                     del wa
                     torch.cuda.empty_cache()
+            # The same one-launch pass as a decoder can drive it: the queries of layer l+1 are released
+            # only when the output of layer l is complete (here they ARE that output, aliased in
+            # memory: q = X[l], out = X[l+1]); the caller's stream only waits and releases, through
+            # stream-ordered memory operations, so no kernel has to fit beside the persistent one.
+            # A second form leaves 8 SMs free and has a kernel of the caller (an elementwise negation)
+            # compute q[l+1] from out[l] on them.
+            for label, alias in ((("layer_dependent_q", True), ("layer_dependent_q_caller_kernel", False))
+                                 if args.pipeline_mode == 0 else ()):
+                kwa = dict(kw) if alias else {**kw, "decode_ctas": max(1, torch.cuda.get_device_properties(0).multi_processor_count - 8)}
+                try:
+                    wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **kwa)
+                    X = torch.zeros((L + 1,) + tuple(wa.q.shape[1:]), device="cuda", dtype=torch.bfloat16)
+                    X[0].copy_(wa.q[0])
+                    caller = torch.cuda.Stream()
+                    if not alias:
+                        torch.neg(wa.out[0], out=wa.q[1])        # loads the kernel's code before any pass runs
+                    torch.cuda.synchronize()
+
+                    def dependent_step():
+                        rc = wa.s.slice_step_begin(wa.seqs, X[:L] if alias else wa.q, wl.num_q_heads, wa.scale,
+                                                   X[1:] if alias else wa.out, wrap, wa.main)
+                        if rc != 0:
+                            raise RuntimeError(f"slice_step_begin: {B.slice_strerror(rc)}")
+                        assert wa.s.slice_step_submit_q(0, caller) == 0
+                        for l in range(L - 1):
+                            assert wa.s.slice_step_wait_out(l, caller) == 0
+                            if not alias:
+                                with torch.cuda.stream(caller):
+                                    torch.neg(wa.out[l], out=wa.q[l + 1])
+                            assert wa.s.slice_step_submit_q(l + 1, caller) == 0
+
+                    for _ in range(3):
+                        dependent_step()
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(wa.main)
+                    for _ in range(reps):
+                        dependent_step()
+                    e1.record(wa.main)
+                    torch.cuda.synchronize()
+                    ta = e0.elapsed_time(e1) / 1e3
+                    if wa.s.slice_stats()["device_status"] != 0:
+                        raise RuntimeError("layer-dependent pass: a bounded device wait expired")
+                    tr = wa.s.slice_cta_trace(0).astype(np.float64)
+                    abl[label] = {
+                        "tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
+                        "hbm_gbs_combined": step_bytes * reps / ta / 1e9,
+                        "stall_us_per_layer": float((tr[1:, :wa.s.cfg.decode_ctas or None, 1] / 1e3).mean()),
+                        "decode_ctas": int(wa.s.cfg.decode_ctas) or "one per SM",
+                        "note": "slice_step_begin: every layer's attention waits for its queries, which are released only "
+                                "after the previous layer's output is complete (" +
+                                ("q[l+1] = out[l], aliased in memory: the caller's stream only waits and releases"
+                                 if alias else "q[l+1] = -out[l], computed by a kernel of the caller on the 8 SMs left free"
+                                               ) + "); traced run"}
+                    del wa, X
+                    torch.cuda.empty_cache()
+                except RuntimeError as err:      # an ablation must not cost the bench line
+                    abl[label] = {"error": str(err)}
+                    torch.cuda.synchronize()
+                    torch.cuda.empty_cache()
             ws = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, pipeline_mode=1, **kw)
             for _ in range(2):
                 assert ws.s.slice_decode_step(ws.seqs, ws.q, wl.num_q_heads, ws.scale, ws.out, False, wrap, ws.main, ws.main) == 0
@@ -586,7 +646,8 @@ def run_ours(args, wl):
                     h = hbm(gbs, prio)
                     return (h["dram_bytes"] if h["dram_bytes"] is not None else h["algorithmic_bytes"]) >= 0.70
 
-                prio_of = {"lock_step_stealing": 0, "prefetch_priority": 1, "prefetch_priority_lock_step": 1}
+                prio_of = {"lock_step_stealing": 0, "prefetch_priority": 1, "prefetch_priority_lock_step": 1,
+                           "layer_dependent_q": -1, "layer_dependent_q_caller_kernel": -1}     # DRAM traffic of that mode: not captured
                 ok = [k for k, v in alts.items() if frac(v) < 0.05 and gate(v["hbm_gbs_combined"], prio_of.get(k, 0))]
                 pick = max(ok, key=lambda k: alts[k]["tokens_per_s"]) if ok else min(alts, key=lambda k: frac(alts[k]))
                 default_stall = extra["stall_frac_of_layer"]

@@ -347,6 +347,40 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
                       float sm_scale, void* out, int32_t io_on_host, int32_t wrap_prefetch,
                       void* stream, void* side_stream);
 
+/* Sections 2.3 and 5.1: the layer-dependent form of the one-launch pass. In a decoder the queries of
+ * layer l+1 exist only after layer l's output has gone through the rest of the block; the latency
+ * window in which the prefetch of a layer hides is exactly that time. slice_step_begin enqueues
+ * the same persistent launch as slice_decode_step (pipeline_mode 0, device q and out, same layout),
+ * except that the attention of EVERY layer l first waits, bounded, for the arrival of q[l], and that
+ * the merge which completes out[l] announces it. The gathers do not wait for queries: while a
+ * layer's attention waits for its q, the copy threads go on prefetching.
+ *   slice_step_begin      enqueues the pass on `stream` and returns. No layer's queries count as
+ *                         arrived yet, layer 0 included.
+ *   slice_step_submit_q   enqueues on caller_stream, behind the work already enqueued there (which
+ *                         wrote q[layer]), a write of layer's arrival word.
+ *   slice_step_wait_out   makes caller_stream wait until out[layer] is complete.
+ *   slice_step_flags      for callers whose own kernels do the signalling instead: device addresses
+ *                         of the two arrays of 32-bit words (one word per layer) and the epoch of
+ *                         the pass. q[l] has arrived when q_ready[l] >= epoch (write q, fence, then
+ *                         the word); out[l] is complete once out_ready[l] >= epoch (acquire).
+ * submit / wait / flags refer to the pass begun last; begin the next pass only after all of them
+ * have been enqueued for this one. caller_stream must differ from `stream` (which the running
+ * launch occupies). The launch holds every SM it runs on for the whole pass, with nearly all of
+ * their shared memory: kernels of the caller that are to run meanwhile (device-to-device copies are
+ * kernels in this sense) need SMs of their own, i.e. decode_ctas below the SM count, and must have
+ * run once before the pass begins (a kernel's first launch loads its code, which does not finish
+ * while the pass runs); the two calls above need neither. A q that does not
+ * arrive within the kernel's bounded wait (about two seconds) ends the launch with SLICE_ETIMEOUT in
+ * slice_stats().device_status.
+ * Errors: EINVAL (pipeline_mode other than 0, a ring of one slot, fewer than 2 or more than 128
+ * layers, more CTAs than SMs; submit / wait / flags without a pass begun by slice_step_begin),
+ * ECUDA (the driver offers no stream memory operations), and those of slice_decode_step. */
+int slice_step_begin(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t num_q_heads,
+                     float sm_scale, void* out, int32_t wrap_prefetch, void* stream);
+int slice_step_submit_q(slice_t* s, uint32_t layer, void* caller_stream);
+int slice_step_wait_out(slice_t* s, uint32_t layer, void* caller_stream);
+int slice_step_flags(slice_t* s, uint32_t** q_ready, uint32_t** out_ready, uint32_t* epoch);
+
 /* Counters and capacities (host struct). */
 int slice_stats(slice_t* s, slice_stats_t* out);
 

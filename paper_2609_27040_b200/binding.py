@@ -31,6 +31,7 @@ EXPORTS = [
     "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc", "slice_cta_trace",
     "slice_reclaim_preempt", "slice_preempt_seq", "slice_set_preempt_window", "slice_set_time", "slice_preempt_stats",
     "slice_set_peer_used", "slice_schedule_gll",
+    "slice_step_begin", "slice_step_submit_q", "slice_step_wait_out", "slice_step_flags",
 ]
 
 
@@ -110,6 +111,10 @@ def lib() -> C.CDLL:
         L.slice_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, vp]
         L.slice_writeback_layer.argtypes = [vp, u32, vp, u32, vp]
         L.slice_decode_step.argtypes = [vp, vp, u32, vp, u32, C.c_float, vp, i32, i32, vp, vp]
+        L.slice_step_begin.argtypes = [vp, vp, u32, vp, u32, C.c_float, vp, i32, vp]
+        L.slice_step_submit_q.argtypes = [vp, u32, vp]
+        L.slice_step_wait_out.argtypes = [vp, u32, vp]
+        L.slice_step_flags.argtypes = [vp, vp, vp, vp]
         L.slice_stats.argtypes = [vp, C.POINTER(SliceStats)]
         L.slice_get_resolved.argtypes = [vp, vp, u32, vp, u32, vp]
         L.slice_layer_times.argtypes = [vp, vp, u32]
@@ -326,6 +331,24 @@ class Slice:
         return lib().slice_decode_step(self._h, _ptr(sq), len(sq), _ptr(q), num_q_heads, sm_scale, _ptr(out),
                                        int(io_on_host), int(wrap_prefetch), _stream(stream),
                                        _stream(side_stream))
+
+    def slice_step_begin(self, seqs, q, num_q_heads: int, sm_scale: float, out, wrap_prefetch: bool = True,
+                         stream=None) -> int:
+        sq = seqs if isinstance(seqs, np.ndarray) and seqs.dtype == np.int32 else _seqs(seqs)
+        return lib().slice_step_begin(self._h, _ptr(sq), len(sq), _ptr(q), num_q_heads, sm_scale, _ptr(out),
+                                      int(wrap_prefetch), _stream(stream))
+
+    def slice_step_submit_q(self, layer: int, caller_stream) -> int:
+        return lib().slice_step_submit_q(self._h, layer, _stream(caller_stream))
+
+    def slice_step_wait_out(self, layer: int, caller_stream) -> int:
+        return lib().slice_step_wait_out(self._h, layer, _stream(caller_stream))
+
+    def slice_step_flags(self):
+        """(rc, device address of q_ready[], device address of out_ready[], epoch of the pass begun last)."""
+        qr, orr, ep = C.c_void_p(), C.c_void_p(), C.c_uint32(0)
+        rc = lib().slice_step_flags(self._h, C.byref(qr), C.byref(orr), C.byref(ep))
+        return rc, qr.value, orr.value, ep.value
 
     # -- introspection ----------------------------------------------------------------------
     def slice_stats(self) -> dict:

@@ -90,6 +90,8 @@ struct LayerParams {
   const uint32_t* q_ready;      // optional: q arrives while the launch runs; layer l's rows may be read once
   uint32_t q_ready_epoch;       //   q_ready[l / q_ready_layers] >= q_ready_epoch (written after the rows themselves)
   uint32_t q_ready_layers;
+  uint32_t* out_ready;          // optional: out_ready[l] = out_ready_epoch once every row of layer l's output is written
+  uint32_t out_ready_epoch;
   float* lse;                   // [nseq][Hq] or NULL (single-layer launches only)
   float* part_o;                // [slots][Hq][128] unnormalised partial outputs; layers alternate
   float* part_ml;               // [slots][Hq][4]   between part_buffers such buffers (stride below)

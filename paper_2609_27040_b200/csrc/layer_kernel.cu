@@ -675,7 +675,15 @@ __device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uin
   __syncwarp();
   if ((threadIdx.x & 31u) == 0) {
     __threadfence();
-    atomicAdd(layer_counters(p, li) + kCntMerged, sub ? 1u : p.G);
+    const uint32_t add = sub ? 1u : p.G;
+    const uint32_t old = atomicAdd(layer_counters(p, li) + kCntMerged, add);
+    // The merge that completes the layer announces its output to whoever computes the next layer's
+    // queries from it (another stream of the caller, waiting on this word). Every merging warp
+    // fenced before its addition and this one fences after it, so all rows are visible first.
+    if (p.out_ready && old + add == p.nseq * p.Hq) {
+      __threadfence_system();
+      *reinterpret_cast<volatile uint32_t*>(p.out_ready + li) = p.out_ready_epoch;
+    }
   }
 }
 

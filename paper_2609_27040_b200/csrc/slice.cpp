@@ -142,6 +142,17 @@ struct ema_slice {
   bool io_q_busy = false;
   const uint32_t* step_q_ready = nullptr;  // set for the pass being enqueued
   uint32_t step_q_layers = 0;
+  // layer-dependent passes (slice_step_begin): out_flags_dev[l] = epoch once layer l's output is complete
+  uint32_t* out_flags_dev = nullptr;
+  uint32_t* step_out_ready = nullptr;      // set for the pass being enqueued
+  // After the launch of a layer-dependent pass, in stream order, every out-ready word is set once
+  // more from pinned host memory: whatever happened inside the kernel (a bounded wait that ran out),
+  // a caller's stream that waits for an output is released when the launch has ended.
+  static constexpr int kFillSlots = 8;
+  uint32_t* out_fill_host = nullptr;       // [kFillSlots][kMaxStepLayers]
+  cudaEvent_t fill_done[kFillSlots] = {};
+  bool fill_busy[kFillSlots] = {};
+  bool dependent_pass = false;             // a pass begun by slice_step_begin is the most recent one
   // profiling
   std::vector<cudaEvent_t> prof;  // [layer][5]
   std::vector<uint8_t> prof_set;
@@ -722,6 +733,11 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     d.q_ready = s->step_q_ready;
     d.q_ready_epoch = s->q_epoch;
     d.q_ready_layers = s->step_q_layers ? s->step_q_layers : 1;
+    d.out_ready = s->step_out_ready;
+    d.out_ready_epoch = s->q_epoch;
+    // A layer-dependent pass has a hard boundary after every layer: a CTA that is out of work cannot
+    // start on the next layer, so it steals as it would in the last layer of a launch.
+    if (s->step_out_ready && !s->cfg.steal_floor) d.steal_floor = d.steal_floor_last;
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / nbuf;
@@ -795,6 +811,10 @@ void destroy_impl(ema_slice* s) {
     if (s->io_q) cudaFree(s->io_q);
     if (s->io_out) cudaFree(s->io_out);
     if (s->q_flags_dev) cudaFree(s->q_flags_dev);
+    if (s->out_flags_dev) cudaFree(s->out_flags_dev);
+    if (s->out_fill_host) cudaFreeHost(s->out_fill_host);
+    for (auto e : s->fill_done)
+      if (e) cudaEventDestroy(e);
     if (s->q_epoch_host) cudaFreeHost(s->q_epoch_host);
     if (s->io_q_free) cudaEventDestroy(s->io_q_free);
     if (s->io_stream) cudaStreamDestroy(s->io_stream);
@@ -919,6 +939,16 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     const size_t rd = static_cast<size_t>(cfg->ring_slots) * std::max(cfg->staging_blocks_per_slot, 1u) * sizeof(uint32_t);
     if (cudaMalloc(reinterpret_cast<void**>(&s->ready_dev), rd) != cudaSuccess || cudaMemset(s->ready_dev, 0, rd) != cudaSuccess)
       return fail(SLICE_ECUDA);
+    if (cudaMalloc(reinterpret_cast<void**>(&s->q_flags_dev), ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&s->out_flags_dev), ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(s->q_flags_dev, 0, ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(s->out_flags_dev, 0, ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+    if (cudaMallocHost(reinterpret_cast<void**>(&s->out_fill_host),
+                       ema_slice::kFillSlots * ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess)
+      return fail(SLICE_ECUDA);
+    for (auto& e : s->fill_done)
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return fail(SLICE_ECUDA);
     const size_t rl = static_cast<size_t>(std::max(cfg->lent_blocks_physical, 1u)) * 2 * sizeof(int32_t);
     if (cudaMallocHost(reinterpret_cast<void**>(&s->reclaim_host), rl) != cudaSuccess) return fail(SLICE_ECUDA);
     if (cudaMalloc(reinterpret_cast<void**>(&s->reclaim_dev), rl) != cudaSuccess) return fail(SLICE_ECUDA);
@@ -1437,8 +1467,41 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   return SLICE_OK;
 }
 
-int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
-                      void* out, int32_t io_on_host, int32_t wrap, void* stream_v, void* side_v) {
+}  // extern "C"
+
+namespace {
+
+// Stream memory operations of the driver (a stream-ordered 32-bit write; a stream-ordered wait until
+// a 32-bit word has reached a value), looked up through the runtime so that the library does not
+// link against the driver library. Both take (stream, device address, value, flags).
+typedef int (*StreamValue32Fn)(cudaStream_t, unsigned long long, unsigned int, unsigned int);
+struct StreamOps {
+  StreamValue32Fn write = nullptr, wait = nullptr;
+  bool tried = false;
+};
+StreamOps g_stream_ops;
+
+bool stream_ops_ready() {
+  if (!g_stream_ops.tried) {
+    g_stream_ops.tried = true;
+    void *w = nullptr, *v = nullptr;
+    cudaDriverEntryPointQueryResult qw, qv;
+    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &w, cudaEnableDefault, &qw) == cudaSuccess &&
+        cudaGetDriverEntryPoint("cuStreamWaitValue32", &v, cudaEnableDefault, &qv) == cudaSuccess &&
+        qw == cudaDriverEntryPointSuccess && qv == cudaDriverEntryPointSuccess) {
+      g_stream_ops.write = reinterpret_cast<StreamValue32Fn>(w);
+      g_stream_ops.wait = reinterpret_cast<StreamValue32Fn>(v);
+    } else {
+      cudaGetLastError();
+    }
+  }
+  return g_stream_ops.write && g_stream_ops.wait;
+}
+
+// One pass over all layers (slice_decode_step), or the same pass in its layer-dependent form
+// (slice_step_begin): every layer's queries are waited for and every layer's output is announced.
+int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
+                     void* out, int32_t io_on_host, int32_t wrap, void* stream_v, void* side_v, bool dependent) {
   if (!s) return SLICE_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v), side = static_cast<cudaStream_t>(side_v);
   Plan* p = nullptr;
@@ -1453,8 +1516,24 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
   const uint8_t* qd = static_cast<const uint8_t*>(q);
   uint8_t* od = static_cast<uint8_t*>(out);
-  bool out_mapped = false;
+  bool out_mapped = false, streamed_q = false;
   s->step_q_ready = nullptr;
+  s->step_out_ready = nullptr;
+  if (dependent) {
+    // Only the one-launch pass has anything to feed: with the other pipelines the caller drives the
+    // layers itself and the stream already orders a layer's attention after its queries.
+    if (io_on_host || !step) return SLICE_EINVAL;
+    for (uint32_t i = 0; i < nseq; ++i)
+      if (s->seqs[seqs[i]].len == 0) return SLICE_EINVAL;  // before the epoch moves
+    if (!s->null_dev && !stream_ops_ready()) {
+      s->st.last_cuda_error = static_cast<int>(cudaErrorNotSupported);
+      return SLICE_ECUDA;
+    }
+    ++s->q_epoch;
+    s->step_q_ready = s->q_flags_dev;
+    s->step_q_layers = 1;
+    s->step_out_ready = s->out_flags_dev;
+  }
   if (!s->null_dev) {
     rc = ensure_stream(s, stream);
     if (rc) return rc;
@@ -1488,8 +1567,6 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       // reads a layer's rows only after its flag shows this pass's epoch (bounded wait).
       if (!s->io_stream) {
         CU(s, cudaStreamCreateWithFlags(&s->io_stream, cudaStreamNonBlocking));
-        CU(s, cudaMalloc(reinterpret_cast<void**>(&s->q_flags_dev), ema::kMaxStepLayers * sizeof(uint32_t)));
-        CU(s, cudaMemset(s->q_flags_dev, 0, ema::kMaxStepLayers * sizeof(uint32_t)));
         CU(s, cudaMallocHost(reinterpret_cast<void**>(&s->q_epoch_host), 64 * sizeof(uint32_t)));
         CU(s, cudaEventCreateWithFlags(&s->io_q_free, cudaEventDisableTiming));
       }
@@ -1513,6 +1590,7 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
       }
       s->step_q_ready = s->q_flags_dev;
       s->step_q_layers = per_flag;
+      streamed_q = true;
     } else {
       CU(s, cudaMemcpyAsync(s->io_q, q, need, cudaMemcpyHostToDevice, stream));
     }
@@ -1535,6 +1613,15 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
   if (step) {
     rc = do_step(s, p, qd, Hq, sm_scale, od, stream, wrap != 0);
     if (rc) return rc;
+    if (dependent && !s->null_dev) {
+      const int slot = static_cast<int>(s->q_epoch % ema_slice::kFillSlots);
+      if (s->fill_busy[slot]) CU(s, cudaEventSynchronize(s->fill_done[slot]));  // the words of 8 passes ago
+      uint32_t* words = s->out_fill_host + static_cast<size_t>(slot) * ema::kMaxStepLayers;
+      for (uint32_t l = 0; l < L; ++l) words[l] = s->q_epoch;
+      CU(s, cudaMemcpyAsync(s->out_flags_dev, words, L * sizeof(uint32_t), cudaMemcpyHostToDevice, stream));
+      CU(s, cudaEventRecord(s->fill_done[slot], stream));
+      s->fill_busy[slot] = true;
+    }
   }
   for (uint32_t l = 0; l < L && !step; ++l) {
     // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.
@@ -1570,15 +1657,66 @@ int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void
     rc = do_prefetch(s, 0, p, side);
     if (rc) return rc;
   }
-  if (s->step_q_ready) {
+  if (streamed_q) {
     // io_q may be overwritten once this pass is done; a later non-streamed use of io_q on `stream`
     // is ordered by the stream itself.
     CU(s, cudaEventRecord(s->io_q_free, stream));
     s->io_q_busy = true;
-    s->step_q_ready = nullptr;
   }
+  s->step_q_ready = nullptr;
+  s->step_out_ready = nullptr;
+  s->dependent_pass = dependent;
   if (io_on_host && !s->null_dev && !out_mapped)
     CU(s, cudaMemcpyAsync(out, s->io_out, per_layer * L, cudaMemcpyDeviceToHost, stream));
+  return SLICE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int slice_decode_step(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
+                      void* out, int32_t io_on_host, int32_t wrap, void* stream_v, void* side_v) {
+  return decode_step_impl(s, seqs, nseq, q, Hq, sm_scale, out, io_on_host, wrap, stream_v, side_v, false);
+}
+
+int slice_step_begin(slice_t* s, const int32_t* seqs, uint32_t nseq, const void* q, uint32_t Hq, float sm_scale,
+                     void* out, int32_t wrap, void* stream_v) {
+  return decode_step_impl(s, seqs, nseq, q, Hq, sm_scale, out, 0, wrap, stream_v, stream_v, true);
+}
+
+int slice_step_submit_q(slice_t* s, uint32_t layer, void* caller_stream) {
+  if (!s || layer >= s->cfg.num_layers || !s->dependent_pass) return SLICE_EINVAL;
+  if (s->null_dev) return SLICE_OK;
+  if (!stream_ops_ready()) return SLICE_ECUDA;
+  const int r = g_stream_ops.write(static_cast<cudaStream_t>(caller_stream),
+                                   reinterpret_cast<unsigned long long>(s->q_flags_dev + layer), s->q_epoch, 0u);
+  if (r != 0) {
+    s->st.last_cuda_error = r;
+    return SLICE_ECUDA;
+  }
+  return SLICE_OK;
+}
+
+int slice_step_wait_out(slice_t* s, uint32_t layer, void* caller_stream) {
+  if (!s || layer >= s->cfg.num_layers || !s->dependent_pass) return SLICE_EINVAL;
+  if (s->null_dev) return SLICE_OK;
+  if (!stream_ops_ready()) return SLICE_ECUDA;
+  const int r = g_stream_ops.wait(static_cast<cudaStream_t>(caller_stream),
+                                  reinterpret_cast<unsigned long long>(s->out_flags_dev + layer), s->q_epoch,
+                                  0u /* wait until the word is >= the value (epochs only grow) */);
+  if (r != 0) {
+    s->st.last_cuda_error = r;
+    return SLICE_ECUDA;
+  }
+  return SLICE_OK;
+}
+
+int slice_step_flags(slice_t* s, uint32_t** q_ready, uint32_t** out_ready, uint32_t* epoch) {
+  if (!s || !s->dependent_pass) return SLICE_EINVAL;
+  if (q_ready) *q_ready = s->q_flags_dev;
+  if (out_ready) *out_ready = s->out_flags_dev;
+  if (epoch) *epoch = s->q_epoch;
   return SLICE_OK;
 }
 

@@ -97,18 +97,21 @@ class FullBatch:
         assert rc == 0 and k2 == k
         assert (_bits(B.kv_block_swizzle(self.staging[0, :k])) == staged[0]).all()
 
-    def check_attention_in_full(self, layer: int, resolved: np.ndarray, k: int):
+    def check_attention_in_full(self, layer: int, resolved: np.ndarray, k: int, q_layer=None, out_layer=None):
         """Every sequence and every query head of `layer`: the oracle gathers the layer's lent blocks
-        into a host staging slot and attends in fp64 through the resolved table."""
+        into a host staging slot and attends in fp64 through the resolved table. q_layer / out_layer
+        (device tensors) replace self.q[layer] / self.out[layer] where the pass used other buffers."""
         wl = self.wl
+        q_layer = self.q[layer] if q_layer is None else q_layer
+        out_layer = self.out[layer] if out_layer is None else out_layer
         local = _bits(B.kv_block_swizzle(self.local[layer]))       # block format -> canonical token rows
         lent = _bits(B.kv_block_swizzle(self.lent[layer]))
         staged = np.zeros((1, max(k, 1)) + lent.shape[1:], np.uint16)
         assert self.orc.gather(0, self.seqs, lent[None], staged)[0] == 0
-        rc, ref, _ = oracle.paged_attention(_bits(self.q[layer]), local, staged[0], resolved, self.lens, wl.num_q_heads,
+        rc, ref, _ = oracle.paged_attention(_bits(q_layer), local, staged[0], resolved, self.lens, wl.num_q_heads,
                                             wl.num_kv_heads, wl.head_dim, wl.block_tokens, self.scale, want_lse=False)
         assert rc == 0
-        got = self.out[layer].double().cpu().numpy()
+        got = out_layer.double().cpu().numpy()
         assert np.isfinite(got).all()
         ok, max_abs, max_rel = attention_close(got, ref, ATOL, RTOL)
         assert ok, (layer, max_abs, max_rel)

@@ -39,7 +39,7 @@ def test_library_exports_every_declared_entry_point():
 
 
 def test_config_struct_matches_header_size():
-    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 6 uint32
+    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 8 uint32
     assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 8 * 4
 
 
@@ -155,6 +155,37 @@ def test_decode_step_drives_the_layer_pipeline_in_tables_only_mode():
     st = s.slice_stats()
     assert st["prefetch_calls"] == 8 and st["decode_calls"] == 8   # layer 0 was already staged
     s.close()
+
+
+def test_layer_dependent_pass_bookkeeping_in_tables_only_mode():
+    """slice_step_begin does the same bookkeeping as slice_decode_step; the calls that feed and follow
+    the running pass need a pass begun by it, and only the one-launch pipeline has one."""
+    s = _null_slice(4, 8, 8, 8, 8, 4, 4, 8)
+    s.slice_alloc_blocks(0, 2, B.TIER_LENT)
+    s.slice_alloc_blocks(0, 1, B.TIER_LOCAL)
+    s.slice_set_seq_len(0, 40)
+    assert s.slice_step_submit_q(0, None) == B.EINVAL and s.slice_step_wait_out(0, None) == B.EINVAL
+    assert s.slice_step_flags()[0] == B.EINVAL
+    assert s.slice_step_begin([0], None, 8, 1.0, None) == B.OK
+    st = s.slice_stats()
+    assert st["prefetch_calls"] == 5 and st["decode_calls"] == 4
+    for layer in range(4):
+        assert s.slice_step_submit_q(layer, None) == B.OK and s.slice_step_wait_out(layer, None) == B.OK
+    assert s.slice_step_submit_q(4, None) == B.EINVAL
+    rc, _, _, epoch = s.slice_step_flags()
+    assert rc == B.OK and epoch == 1
+    assert s.slice_decode_step([0], None, 8, 1.0, None) == B.OK       # a free-running pass ends the dependent one
+    assert s.slice_step_submit_q(0, None) == B.EINVAL
+    assert s.slice_step_begin([0], None, 12, 1.0, None) == B.EINVAL   # bad head count
+    assert s.slice_set_seq_len(0, 0) == B.OK
+    assert s.slice_step_begin([0], None, 8, 1.0, None) == B.EINVAL    # empty sequence
+    s.close()
+    for kw in ({"pipeline_mode": 1}, {"pipeline_mode": 2}, {"ring_slots": 1}):
+        s = B.Slice(4, 8, 8, 8, 4, lent_blocks_physical=8, max_seqs=4, max_blocks_per_seq=8, flags=B.FLAG_NULL_DEVICE, **kw)
+        s.slice_alloc_blocks(0, 2, B.TIER_LENT)
+        s.slice_set_seq_len(0, 20)
+        assert s.slice_step_begin([0], None, 8, 1.0, None) == B.EINVAL
+        s.close()
 
 
 def test_decode_step_with_a_shared_ring_slot_for_first_and_last_layer():
