@@ -381,6 +381,16 @@ int slice_step_submit_q(slice_t* s, uint32_t layer, void* caller_stream);
 int slice_step_wait_out(slice_t* s, uint32_t layer, void* caller_stream);
 int slice_step_flags(slice_t* s, uint32_t** q_ready, uint32_t** out_ready, uint32_t* epoch);
 
+/* Measurement and test utility for the calls above (the paper has no counterpart): enqueues on
+ * caller_stream a one-thread kernel that plays the rest of a decoder whose work between two
+ * attention layers takes no time. It releases q[0] at once and q[l+1] as soon as out[l] is announced,
+ * through the device words of slice_step_flags (about a microsecond per hand-over; the stream-ordered
+ * slice_step_wait_out + slice_step_submit_q pair costs tens of microseconds per layer). The caller
+ * must have put q[l+1] where out[l] is written (q = X, out = X + one layer) or not care what the
+ * later layers attend to. Needs an SM the pass leaves free: EINVAL unless decode_ctas is below the
+ * SM count, or without a pass begun by slice_step_begin. Bounded waits as everywhere. */
+int slice_step_relay(slice_t* s, void* caller_stream);
+
 /* Counters and capacities (host struct). */
 int slice_stats(slice_t* s, slice_stats_t* out);
 
@@ -397,9 +407,12 @@ int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers);
 
 /* With SLICE_FLAG_PROFILE: per-CTA times (GPU nanosecond timer) of the most recent launch of each
  * layer's kernel, as [num_layers][ctas_per_layer][words_per_cta] uint64 on the host; unused entries
- * are 0. which = 0: layer kernel, 4 words (time the CTA started on the layer, nanoseconds its
+ * are 0. which = 0: layer kernel, 8 words (time the CTA started on the layer, nanoseconds its
  * attention waited for the layer's prefetched blocks, end of the copy work it did during the layer,
- * SM id | runs << 16 | claims << 32); which = 1: stand-alone gather kernel, 2 words (start, end). out may be NULL to query
+ * SM id | runs << 16 | claims << 32, time its producer had issued the layer's last block, time its
+ * first consumer warp finished its last run of the layer, nanoseconds that warp waited for the
+ * layer's queries, time it first had them: the last two only where queries arrive while the launch
+ * runs); which = 1: stand-alone gather kernel, 2 words (start, end). out may be NULL to query
  * the two sizes. Synchronises the device. */
 int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entries, uint32_t* ctas_per_layer,
                     uint32_t* words_per_cta);

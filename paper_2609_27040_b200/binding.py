@@ -31,7 +31,7 @@ EXPORTS = [
     "slice_get_resolved", "slice_layer_times", "slice_copy_blocks", "slice_strerror", "paged_decode_noalloc", "slice_cta_trace",
     "slice_reclaim_preempt", "slice_preempt_seq", "slice_set_preempt_window", "slice_set_time", "slice_preempt_stats",
     "slice_set_peer_used", "slice_schedule_gll",
-    "slice_step_begin", "slice_step_submit_q", "slice_step_wait_out", "slice_step_flags",
+    "slice_step_begin", "slice_step_submit_q", "slice_step_wait_out", "slice_step_flags", "slice_step_relay",
 ]
 
 
@@ -115,6 +115,7 @@ def lib() -> C.CDLL:
         L.slice_step_submit_q.argtypes = [vp, u32, vp]
         L.slice_step_wait_out.argtypes = [vp, u32, vp]
         L.slice_step_flags.argtypes = [vp, vp, vp, vp]
+        L.slice_step_relay.argtypes = [vp, vp]
         L.slice_stats.argtypes = [vp, C.POINTER(SliceStats)]
         L.slice_get_resolved.argtypes = [vp, vp, u32, vp, u32, vp]
         L.slice_layer_times.argtypes = [vp, vp, u32]
@@ -343,6 +344,9 @@ class Slice:
 
     def slice_step_wait_out(self, layer: int, caller_stream) -> int:
         return lib().slice_step_wait_out(self._h, layer, _stream(caller_stream))
+
+    def slice_step_relay(self, caller_stream) -> int:
+        return lib().slice_step_relay(self._h, _stream(caller_stream))
 
     def slice_step_flags(self):
         """(rc, device address of q_ready[], device address of out_ready[], epoch of the pass begun last)."""

@@ -51,6 +51,12 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
 constexpr uint32_t kLaunchCounters = 32;
 constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntMergePub = 16, kCntMergeTaken = 17, kCntMerged = 18;
 constexpr uint32_t kMaxStepLayers = 128;
+// Words of the per-CTA, per-layer trace of the layer kernel: [0] time the CTA started on the layer,
+// [1] ns its attention waited for prefetched blocks, [2] end of the copy work it did during the
+// layer, [3] SM id | runs << 16 | claims << 32, [4] time its producer had issued the layer's last
+// block, [5] time the first consumer warp finished its last run of the layer, [6] ns that warp
+// waited for the layer's queries, [7] time it first had them.
+constexpr uint32_t kTraceWords = 8;
 constexpr uint32_t kSharedMergeMin = 12;  // partials from which a merge is offered to every CTA
 constexpr uint32_t kSplitMergeMin = 48;   // partials from which it is offered one query head at a time
 inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
@@ -116,7 +122,7 @@ struct LayerParams {
   int16_t gather_target[kMaxStepLayers];
   int16_t gather_after[kMaxStepLayers];
   int* status;
-  unsigned long long* trace;    // optional, per layer [ncta][4]: start, ns waited for the gather, copy end, info
+  unsigned long long* trace;    // optional, per layer [ncta][kTraceWords]
   uint64_t trace_stride;        // words from one layer's trace to the next
 };
 
@@ -128,6 +134,11 @@ cudaError_t layer_setup();
 // layers contain bounded waits between CTAs and are therefore launched cooperatively (all CTAs
 // resident).
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream);
+
+// A one-thread kernel that releases q_ready[l + 1] as soon as out_ready[l] shows `epoch` (and
+// q_ready[0] at once): the rest of a decoder, taking no time (measurements and tests).
+cudaError_t launch_step_relay(const uint32_t* out_ready, uint32_t* q_ready, uint32_t layers, uint32_t epoch, int* status,
+                              cudaStream_t stream);
 
 // noalloc.cu: the same launch with partials and counters in a static device array (part_o,
 // part_ml, counters of p are ignored). static_scratch_needed() > static_scratch_bytes() must be

@@ -270,8 +270,8 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     const uint32_t epoch = p.epoch_base + li;
     uint64_t waited_ns = 0;
     if (p.trace && lane == 0) {
-      p.trace[li * p.trace_stride + 4 * blockIdx.x] = ptx::global_timer_ns();
-      p.trace[li * p.trace_stride + 4 * blockIdx.x + 1] = 0;
+      p.trace[li * p.trace_stride + kTraceWords * blockIdx.x] = ptx::global_timer_ns();
+      p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 1] = 0;
     }
     // The partial buffer of this layer was last used part_buffers layers ago: its merges must be done.
     if (li >= p.part_buffers) {
@@ -514,10 +514,11 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
       }
     }
     if (p.trace && lane == 0) {
+      p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 4] = ptx::global_timer_ns();
       uint32_t smid;
       asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      p.trace[li * p.trace_stride + 4 * blockIdx.x + 1] = waited_ns;
-      p.trace[li * p.trace_stride + 4 * blockIdx.x + 3] =
+      p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 1] = waited_ns;
+      p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 3] =
           smid | (static_cast<unsigned long long>(nruns) << 16) | (static_cast<unsigned long long>(nclaims) << 32);
     }
   }
@@ -947,6 +948,8 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       if (h0 < G) *reinterpret_cast<float4*>(pml + h0 * 4) = make_float4(st.m0, st.l0, st.e0, 0.f);
       if (h1 < G) *reinterpret_cast<float4*>(pml + h1 * 4) = make_float4(st.m1, st.l1, st.e1, 0.f);
     }
+    if (p.trace && g == 0 && lane == 0)
+      p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 5] = ptx::global_timer_ns();
     finish_run(p, sm, run_li, run_seq, g, run_blocks);
   };
 
@@ -972,9 +975,15 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
-      if (run_li >= q_upto) {  // q may still be on its way from the host: wait for this layer's chunk
+      if (run_li >= q_upto) {  // q may still be on its way: wait for this layer's rows (or chunk of layers)
+        const uint64_t w0 = p.trace && p.q_ready ? ptx::global_timer_ns() : 0;
         if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
         q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+        if (p.trace && p.q_ready && g == 0 && lane == 0) {
+          const uint64_t w1 = ptx::global_timer_ns();
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 6] = w1 - w0;
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 7] = w1;
+        }
       }
       // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
       const __nv_bfloat16* qg =
@@ -1032,6 +1041,8 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
     if (lane == 0)
       *reinterpret_cast<float4*>(part_ml_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g) * 4) =
           make_float4(st.m0, st.l0, st.l0, 0.f);
+    if (p.trace && g == 0 && lane == 0)
+      p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 5] = ptx::global_timer_ns();
     finish_run(p, sm, run_li, run_seq, g, run_blocks);
   };
 
@@ -1057,9 +1068,15 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
       run_blocks = 0;
       len = p.lens[run_seq];
       st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
-      if (run_li >= q_upto) {
+      if (run_li >= q_upto) {  // q may still be on its way: wait for this layer's rows (or chunk of layers)
+        const uint64_t w0 = p.trace && p.q_ready ? ptx::global_timer_ns() : 0;
         if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
         q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+        if (p.trace && p.q_ready && g == 0 && lane == 0) {
+          const uint64_t w1 = ptx::global_timer_ns();
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 6] = w1 - w0;
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 7] = w1;
+        }
       }
       const __nv_bfloat16* qg =
           reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
@@ -1190,7 +1207,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     }
     ptx::bulk_wait_all<0>();
     if (ok) report_landed(done - first_piece);
-    if (p.trace) p.trace[li * p.trace_stride + 4 * blockIdx.x + 2] = ptx::global_timer_ns();
+    if (p.trace) p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 2] = ptx::global_timer_ns();
   }
   if (!ok) {
     for (uint32_t k = done; k < issued; ++k)
@@ -1271,7 +1288,26 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   }
 }
 
+// One thread stands in for the rest of a decoder whose work between two attention layers takes no
+// time: it releases the queries of layer 0 and then, as soon as the output of layer l is announced,
+// those of layer l+1. It gives up at the first bounded wait that runs out.
+__global__ void __launch_bounds__(32) step_relay_kernel(const uint32_t* out_ready, uint32_t* q_ready, uint32_t layers,
+                                                        uint32_t epoch, int* status) {
+  if (threadIdx.x != 0) return;
+  ptx::st_release_gpu(q_ready, epoch);
+  for (uint32_t l = 0; l + 1 < layers; ++l) {
+    if (!wait_counter(out_ready + l, epoch, status)) return;
+    ptx::st_release_gpu(q_ready + l + 1, epoch);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_step_relay(const uint32_t* out_ready, uint32_t* q_ready, uint32_t layers, uint32_t epoch, int* status,
+                              cudaStream_t stream) {
+  step_relay_kernel<<<1, 32, 0, stream>>>(out_ready, q_ready, layers, epoch, status);
+  return cudaGetLastError();
+}
 
 size_t layer_smem_bytes(uint32_t Hkv) {
   if (Hkv == 0 || Hkv > 8) return 0;

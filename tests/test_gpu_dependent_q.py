@@ -108,19 +108,21 @@ def test_queries_released_layer_by_layer_small(static):
         assert attention_close(got[layer], ref, ATOL, RTOL)[0]
 
 
-@pytest.mark.parametrize("ctas,how", [(0, "alias"), (140, "kernel")])
+@pytest.mark.parametrize("ctas,how", [(0, "alias"), (140, "kernel"), (147, "relay")])
 def test_queries_released_layer_by_layer_full_batch(ctas, how):
     """The benchmark's batch on 6 layers. 'alias': one CTA per SM (no room for any other kernel), the
     next layer's queries are the previous layer's output in place (q = X[l], out = X[l+1]), so the
     caller only waits and releases. 'kernel': 140 CTAs, the caller's own kernel (an elementwise
     negation, launched once beforehand so that its code is loaded) computes the next queries on the
-    SMs left free while the pass runs."""
+    SMs left free while the pass runs. 'relay': 147 CTAs and the library's one-thread relay kernel on
+    the SM left free, which hands every layer's output over as the next layer's queries (aliased as
+    in 'alias') through the device words themselves instead of stream-ordered operations."""
     from tests.test_gpu_full_batch import FullBatch
     L = 6
     fb = FullBatch("llama3_8b_decode", L, decode_ctas=ctas)
     wl = fb.wl
     caller = torch.cuda.Stream()
-    if how == "alias":
+    if how in ("alias", "relay"):
         X = torch.zeros((L + 1,) + tuple(fb.q.shape[1:]), device="cuda", dtype=torch.bfloat16)
         X[0].copy_(fb.q[0])
         q, out, make_q = X[:L], X[1:], None
@@ -134,7 +136,10 @@ def test_queries_released_layer_by_layer_full_batch(ctas, how):
     torch.cuda.synchronize()
     for rep in range(2):
         assert fb.s.slice_step_begin(fb.seqs, q, wl.num_q_heads, fb.scale, out, True, fb.main) == B.OK
-        _feed(fb.s, L, caller, make_q)
+        if how == "relay":
+            assert fb.s.slice_step_relay(caller) == B.OK
+        else:
+            _feed(fb.s, L, caller, make_q)
         torch.cuda.synchronize()
         st = fb.s.slice_stats()
         assert st["device_status"] == 0 and st["last_cuda_error"] == 0

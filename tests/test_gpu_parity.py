@@ -613,7 +613,7 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
     else:
         assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
     trace = g.s.slice_cta_trace(0)
-    assert trace.shape == (sc.L, 12, 4) and (trace[:, :, 0] > 0).all()      # every CTA visited every layer
+    assert trace.shape == (sc.L, 12, 8) and (trace[:, :, 0] > 0).all()      # every CTA visited every layer
     # the staged bytes left in the ring are the oracle's
     from tests.gpu_helpers import kv_to_host, to_host
     for slot in range(wl.ring_slots):

@@ -171,7 +171,7 @@ def test_layer_dependent_pass_bookkeeping_in_tables_only_mode():
     assert st["prefetch_calls"] == 5 and st["decode_calls"] == 4
     for layer in range(4):
         assert s.slice_step_submit_q(layer, None) == B.OK and s.slice_step_wait_out(layer, None) == B.OK
-    assert s.slice_step_submit_q(4, None) == B.EINVAL
+    assert s.slice_step_submit_q(4, None) == B.EINVAL and s.slice_step_relay(None) == B.OK
     rc, _, _, epoch = s.slice_step_flags()
     assert rc == B.OK and epoch == 1
     assert s.slice_decode_step([0], None, 8, 1.0, None) == B.OK       # a free-running pass ends the dependent one
