@@ -71,6 +71,11 @@ def lib() -> C.CDLL:
         L.oracle_preempt_state.restype = None
         L.oracle_append_kv.argtypes = [vp, u32, vp, u32, vp, vp, u32, u32, vp, vp, vp]
         L.oracle_num_threads.restype = C.c_int
+        L.oracle_set_slab_blocks.argtypes = [vp, u32]
+        L.oracle_layout_offset.argtypes = [u32, u32, u32, u32, u32, u64, u32, u32]
+        L.oracle_layout_offset.restype = u64
+        L.oracle_swap_pieces.argtypes = [u32, u32, u32, u32, u32, u64, u32, vp, u32, vp, u32]
+        L.oracle_swap_pieces.restype = u32
     return _lib
 
 
@@ -131,6 +136,10 @@ class OracleSlice:
 
     def set_seq_len(self, seq: int, length: int) -> int:
         return lib().oracle_set_seq_len(self._h, seq, length)
+
+    def set_slab_blocks(self, slab_blocks: int) -> int:
+        """Slab allocator of Section 4.2.1 (0 = off). Before the first allocation."""
+        return lib().oracle_set_slab_blocks(self._h, slab_blocks)
 
     def free_seq(self, seq: int) -> int:
         return lib().oracle_free_seq(self._h, seq)
@@ -266,3 +275,32 @@ def gll_choose(own_blocks: Sequence[int], peer_blocks: Sequence[int], capacity_b
         if best_u is None or u < best_u:
             best, best_u = k, u
     return best
+
+
+# -- memory layouts (O-slab) ------------------------------------------------------------------------
+LAYER_MAJOR, SLAB_MAJOR, LAYER_GROUP_MAJOR = 0, 1, 2
+
+
+def layout_offset(layout: int, num_layers: int, n_blocks: int, slab_blocks: int, layer_group: int,
+                  block_bytes: int, layer: int, block_id: int) -> int:
+    """Byte offset of a block in an arena laid out as Section 4.2.1 / 4.2.2 / 4.2.3 describes."""
+    return int(lib().oracle_layout_offset(layout, num_layers, n_blocks, slab_blocks, layer_group, block_bytes,
+                                          layer, block_id))
+
+
+def swap_pieces(layout: int, num_layers: int, n_blocks: int, slab_blocks: int, layer_group: int,
+                block_bytes: int, group: int, slabs: Sequence[int]) -> list:
+    """Lengths in bytes of the contiguous pieces one swap of `group` moves for the owner of `slabs`."""
+    sl = np.ascontiguousarray(slabs, np.uint32)
+    n = lib().oracle_swap_pieces(layout, num_layers, n_blocks, slab_blocks, layer_group, block_bytes, group,
+                                 _ptr(sl), len(sl), None, 0)
+    out = np.zeros(max(n, 1), np.uint64)
+    lib().oracle_swap_pieces(layout, num_layers, n_blocks, slab_blocks, layer_group, block_bytes, group,
+                             _ptr(sl), len(sl), _ptr(out), n)
+    return [int(x) for x in out[:n]]
+
+
+def group_layers(layer_group: int, group: int) -> range:
+    """Section 4.2.2: a layer group is a set of logically consecutive layers; group g of size k holds
+    layers g*k .. g*k + k - 1, and is handled like one big layer."""
+    return range(group * layer_group, (group + 1) * layer_group)

@@ -28,6 +28,12 @@
 //                 of active requests" (Section 4.2.1); after a preemption above the static share
 //                 the user's allocations are capped for a window T (Section 5.3, bursty workload
 //                 preemption control); preemptions are counted by cause (Section 6.6).
+//   * O-slab    — Section 4.2.1: the slice hands out slabs, runs of consecutive block ids that belong
+//                 to one user as a whole (a slab returns to the slice only when its last block is
+//                 freed); Sections 4.2.1-4.2.3: the three memory layouts (layer-major, slab-major,
+//                 layer-group-major) as address maps, the layer group as the unit of a swap, and
+//                 the sizes of the contiguous pieces a swap of one layer group moves (S..mS, kS,
+//                 kS..mkS), found by brute force over the address map.
 //   * O-schedule — the choice among several slices (Section 5.2, Greedy-Least-Loaded) is stated in
 //                 the Python front end (gll_choose, exact rationals); pins in
 //                 tests/test_oracle_schedule.py.
@@ -107,6 +113,8 @@ struct State {
   uint64_t cap_until = 0;   // a cap holds while now < cap_until
   uint32_t cap_level = 0;   // blocks the user may hold while the cap holds
   uint64_t preempt_oom = 0, preempt_reclaim = 0;
+  // O-slab: blocks per slab; 0 = block-granular free stacks (the seeded orders), no slabs.
+  uint32_t slab = 0;
 };
 
 inline uint32_t used_blocks(const State* s) {
@@ -136,6 +144,32 @@ inline uint16_t double_to_bf16_rne(double x) {
 
 inline uint32_t blocks_for(uint32_t len, uint32_t block_tokens) {
   return (len + block_tokens - 1) / block_tokens;
+}
+
+// The next free id of a part of the slice. Without slabs: the top of the free stack. With slabs
+// (Section 4.2.1): a slab belongs to the user as long as one of its blocks is in use, and the
+// user fills the slabs it already has before it asks the slice for another one: the lowest free
+// id that lies in a slab holding a block in use; failing that the lowest free id of all, which
+// opens the lowest free slab. The caller has checked that a free id exists.
+int32_t take_free(State* s, bool local) {
+  std::vector<int32_t>& fr = local ? s->free_local : s->free_lent;
+  if (s->slab == 0) {
+    const int32_t id = fr.back();
+    fr.pop_back();
+    return id;
+  }
+  const std::vector<Owner>& own = local ? s->owner_local : s->owner_lent;
+  int32_t in_open_slab = -1, any = -1;
+  for (int32_t f : fr) {
+    if (any < 0 || f < any) any = f;
+    const uint32_t first = static_cast<uint32_t>(f) / s->slab * s->slab;
+    bool in_use = false;
+    for (uint32_t id = first; id < first + s->slab && id < own.size(); ++id) in_use = in_use || own[id].seq >= 0;
+    if (in_use && (in_open_slab < 0 || f < in_open_slab)) in_open_slab = f;
+  }
+  const int32_t id = in_open_slab >= 0 ? in_open_slab : any;
+  fr.erase(std::find(fr.begin(), fr.end(), id));
+  return id;
 }
 
 }  // namespace
@@ -180,6 +214,16 @@ void* oracle_create(uint32_t num_layers, uint32_t block_tokens, uint64_t block_b
 
 void oracle_destroy(void* h) { delete static_cast<State*>(h); }
 
+// O-slab: turns the slab allocator on (blocks per slab; the paper's default is 10, Section 6.6).
+// To be called before the first allocation; capacities need not be multiples of the slab (the
+// last slab of a part is then short).
+int oracle_set_slab_blocks(void* h, uint32_t slab_blocks) {
+  State* s = static_cast<State*>(h);
+  if (!s->seqs.empty()) return E_STATE;
+  s->slab = slab_blocks;
+  return OK;
+}
+
 int oracle_alloc_blocks(void* h, int32_t seq, uint32_t n, int32_t hint, int32_t* out_entries) {
   State* s = static_cast<State*>(h);
   if (seq < 0 || hint < AUTO || hint > LENT) return E_INVAL;
@@ -199,13 +243,11 @@ int oracle_alloc_blocks(void* h, int32_t seq, uint32_t n, int32_t hint, int32_t*
     bool take_local = hint == LOCAL || (hint == AUTO && !s->free_local.empty());
     int32_t entry;
     if (take_local) {
-      int32_t id = s->free_local.back();
-      s->free_local.pop_back();
+      int32_t id = take_free(s, true);
       s->owner_local[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
       entry = id;
     } else {
-      int32_t id = s->free_lent.back();
-      s->free_lent.pop_back();
+      int32_t id = take_free(s, false);
       s->owner_lent[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
       entry = ~id;
     }
@@ -478,8 +520,9 @@ int oracle_reclaim(void* h, uint32_t take, uint8_t* local_arena, uint8_t* lent_a
     bool to_local = !s->free_local.empty();
     int32_t dst;
     if (to_local) {
-      dst = s->free_local.back();
-      s->free_local.pop_back();
+      dst = take_free(s, true);
+    } else if (s->slab) {
+      dst = take_free(s, false);  // what is left of the lent list lies below the cut
     } else {
       auto mn = std::min_element(s->free_lent.begin(), s->free_lent.end());
       dst = *mn;
@@ -688,6 +731,61 @@ int oracle_num_threads(void) {
 #else
   return 1;
 #endif
+}
+
+// ------------------------------------------------------------------------------------------
+// O-slab: memory layouts of Section 4.2 as address maps. An arena holds n_blocks block ids (a
+// whole number of slabs of S ids) for each of L layers; a layer group is k consecutive layers
+// (group g = layers g*k .. g*k + k - 1; L a multiple of k). The byte offset of block `id` of
+// `layer` is the position of that block in the nested array the figure of each layout draws:
+//   0 layer-major        [layer][id]                              (Section 4.2.1)
+//   1 slab-major         [slab][layer][block in slab]             (Section 4.2.2: all layers of a
+//                                                                  slab together)
+//   2 layer-group-major  [group][slab][layer in group][block in slab]   (Section 4.2.3: slab i+1
+//                                                                  of the same group follows slab i)
+// ------------------------------------------------------------------------------------------
+uint64_t oracle_layout_offset(uint32_t layout, uint32_t L, uint32_t n_blocks, uint32_t S, uint32_t k,
+                              uint64_t block_bytes, uint32_t layer, uint32_t id) {
+  const uint64_t slabs = n_blocks / S, slab = id / S, in_slab = id % S;
+  uint64_t index = 0;  // in blocks
+  if (layout == 0) {
+    index = static_cast<uint64_t>(layer) * n_blocks + id;
+  } else if (layout == 1) {
+    index = (slab * L + layer) * S + in_slab;
+  } else {
+    const uint64_t group = layer / k, in_group = layer % k;
+    index = ((group * slabs + slab) * k + in_group) * S + in_slab;
+  }
+  return index * block_bytes;
+}
+
+// The contiguous pieces that a swap of layer group `group` moves for a user who owns the listed
+// slabs (Section 4.2.3 compares their sizes across the layouts), by brute force: the byte interval
+// of every block of every listed slab in every layer of the group is laid on the address line,
+// touching intervals are joined, and the lengths of the joined pieces are returned in ascending
+// address order. Returns the number of pieces (out may be NULL to count).
+uint32_t oracle_swap_pieces(uint32_t layout, uint32_t L, uint32_t n_blocks, uint32_t S, uint32_t k,
+                            uint64_t block_bytes, uint32_t group, const uint32_t* slabs, uint32_t nslabs,
+                            uint64_t* out_bytes, uint32_t cap) {
+  std::vector<std::pair<uint64_t, uint64_t>> iv;
+  for (uint32_t layer = group * k; layer < (group + 1) * k && layer < L; ++layer)
+    for (uint32_t j = 0; j < nslabs; ++j)
+      for (uint32_t b = 0; b < S; ++b) {
+        const uint64_t off = oracle_layout_offset(layout, L, n_blocks, S, k, block_bytes, layer, slabs[j] * S + b);
+        iv.emplace_back(off, off + block_bytes);
+      }
+  std::sort(iv.begin(), iv.end());
+  uint32_t n = 0;
+  size_t i = 0;
+  while (i < iv.size()) {
+    uint64_t lo = iv[i].first, hi = iv[i].second;
+    size_t j = i + 1;
+    while (j < iv.size() && iv[j].first <= hi) hi = std::max(hi, iv[j++].second);
+    if (out_bytes && n < cap) out_bytes[n] = hi - lo;
+    ++n;
+    i = j;
+  }
+  return n;
 }
 
 }  // extern "C"
