@@ -138,6 +138,28 @@ typedef struct {
                                      the CTAs stay within a layer of one another, the prefetch is
                                      far ahead of all of them, attention (almost) never waits for
                                      it, staged blocks come from DRAM and the pass is slower     */
+  uint32_t slab_blocks;           /* Section 4.2.1: 0 = blocks are handed out one by one from free stacks
+                                     (the seeded orders); S > 0 = slab allocator: the ids of each part
+                                     form slabs of S consecutive ids (the paper's default is 10,
+                                     Section 6.6), a slab belongs to the user while one of its blocks
+                                     is in use, and the next id is the lowest free id in a slab the
+                                     user holds, else the lowest free id of all (a new slab). The
+                                     free orders must then be NULL                                 */
+  uint32_t layer_group;           /* Section 4.2.2: layers per layer group, the unit of a swap (0 or 1 =
+                                     single layers; the paper's default is 4). A ring slot holds one
+                                     group: staging is [ring_slots][layer_group][staging_blocks_per_slot]
+                                     blocks, layer l is staged in layer slot l mod (ring_slots *
+                                     layer_group), and the pipelines fetch layer l + layer_group
+                                     while layer l is attended to (a group's transfer is issued as
+                                     one piece per layer, at the start of each layer of the group
+                                     before; buffer and latency window are those of a group)       */
+  uint32_t layout;                /* Sections 4.2.1-4.2.3, order of the blocks in BOTH arenas (bytes;
+                                     bb = block bytes, S = slab_blocks, k = layer_group, N = ids of
+                                     the arena, L = layers): 0 layer-major [layer][id] (strides may
+                                     override it); 1 slab-major [slab][layer][block in slab];
+                                     2 layer-group-major [group][slab][layer in group][block in slab].
+                                     1 and 2 need S > 0, N a multiple of S for both arenas, L a
+                                     multiple of k, and zero strides                               */
 } slice_config_t;
 
 typedef struct {

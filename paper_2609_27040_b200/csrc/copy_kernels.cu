@@ -21,14 +21,18 @@ __device__ __forceinline__ const uint8_t* src_addr(const CopyDesc& d, uint32_t i
   int32_t e = d.src_entry ? d.src_entry[i] : static_cast<int32_t>(i);
   int t = e < 0;
   uint32_t id = t ? static_cast<uint32_t>(~e) : static_cast<uint32_t>(e);
-  return d.src_base[t] + layer * d.src_layer_stride[t] + id * d.src_block_stride[t];
+  const uint64_t lo = d.layer_group > 1 ? layer_offset(layer, d.layer_group, d.src_group_stride[t], d.src_layer_stride[t])
+                                        : layer * d.src_layer_stride[t];
+  return d.src_base[t] + lo + id * d.src_block_stride[t];
 }
 
 __device__ __forceinline__ uint8_t* dst_addr(const CopyDesc& d, uint32_t i, uint32_t layer) {
   int32_t e = d.dst_entry ? d.dst_entry[i] : static_cast<int32_t>(i);
   int t = e < 0;
   uint32_t id = t ? static_cast<uint32_t>(~e) : static_cast<uint32_t>(e);
-  return d.dst_base[t] + layer * d.dst_layer_stride[t] + id * d.dst_block_stride[t];
+  const uint64_t lo = d.layer_group > 1 ? layer_offset(layer, d.layer_group, d.dst_group_stride[t], d.dst_layer_stride[t])
+                                        : layer * d.dst_layer_stride[t];
+  return d.dst_base[t] + lo + id * d.dst_block_stride[t];
 }
 
 __global__ void __launch_bounds__(kVecThreads) copy_blocks_vector(const CopyDesc d) {

@@ -14,6 +14,13 @@ constexpr int kDevTimeout = -6;
 // One batched block copy: item i moves block_bytes from src(entry src_entry[i]) to
 // dst(entry dst_entry[i]) for each of nlayers layers. An entry e >= 0 addresses id e of base[0],
 // e < 0 addresses id ~e of base[1]. A NULL entry array means entry i = i.
+// Byte offset of layer l in an arena whose layers come in groups of k: group l / k starts at a
+// multiple of group_stride, layer l % k of the group at a multiple of layer_stride (k = 1 and
+// group_stride = layer_stride give the plain [layer] order).
+__host__ __device__ inline uint64_t layer_offset(uint32_t l, uint32_t k, uint64_t group_stride, uint64_t layer_stride) {
+  return static_cast<uint64_t>(l / k) * group_stride + static_cast<uint64_t>(l % k) * layer_stride;
+}
+
 struct CopyDesc {
   const uint8_t* src_base[2];
   uint8_t* dst_base[2];
@@ -21,6 +28,9 @@ struct CopyDesc {
   uint64_t dst_block_stride[2];
   uint64_t src_layer_stride[2];
   uint64_t dst_layer_stride[2];
+  uint64_t src_group_stride[2];  // used when layer_group > 1 (see layer_offset)
+  uint64_t dst_group_stride[2];
+  uint32_t layer_group;          // 0 or 1: layers are src/dst_layer_stride apart
   const int32_t* src_entry;
   const int32_t* dst_entry;
   uint32_t n;
@@ -66,9 +76,12 @@ inline size_t layer_counter_words(uint32_t ncta, uint32_t nseq, uint32_t Hkv) {
 // Parameters of one launch of the layer kernel. It covers layers first_layer .. first_layer +
 // num_layers - 1 of one batch; pointers refer to first_layer and the strides lead to the next layer.
 struct LayerParams {
-  const uint8_t* local_layer;   // local arena of first_layer
-  uint64_t local_layer_stride;
+  const uint8_t* local_base;    // local arena; layer l starts at layer_offset(l, layer_group, local_group_stride,
+  uint64_t local_group_stride;  //   local_layer_stride), and an entry e >= 0 addresses e * local_block_stride
+  uint64_t local_layer_stride;  //   from there (entries are physical indices: the host has applied the layout)
   uint64_t local_block_stride;
+  uint32_t layer_group;         // layers per group of the arenas' layout (>= 1)
+  uint32_t prefetch_distance;   // the gather issued during launch layer i fetches layer i + prefetch_distance
   const uint8_t* staging_base;  // ring: layer l is staged in slot l % ring_slots
   uint64_t slot_bytes;
   uint32_t ring_slots;
@@ -111,8 +124,8 @@ struct LayerParams {
   // Gather issued while layer first_layer + i is attended to: target layer (or -1), and the layer of
   // this launch whose attention must be complete before the target's ring slot may be overwritten
   // (-1: ordered by the stream already).
-  const uint8_t* lent_base;     // lent arena of layer 0
-  uint64_t lent_layer_stride, lent_block_stride;
+  const uint8_t* lent_base;     // lent arena (same addressing as the local one)
+  uint64_t lent_group_stride, lent_layer_stride, lent_block_stride;
   const int32_t* copy_src;      // [copy_n] lent entries in staging order
   const uint32_t* copy_order;   // [copy_n] staging positions in the order they are gathered
   uint32_t copy_n;
@@ -151,10 +164,12 @@ size_t static_scratch_needed(uint32_t slots, uint32_t Hq, uint32_t nseq, uint32_
 cudaError_t launch_layer_static(LayerParams p, uint32_t slots, cudaStream_t stream);
 
 struct AppendParams {
-  uint8_t* local_layer;        // local arena of the first layer appended to
+  uint8_t* local_base;         // arenas; layer first_layer + y of the launch at layer_offset(...) from there
   uint64_t local_block_stride;
-  uint8_t* lent_layer;         // lent arena of the first layer appended to
+  uint8_t* lent_base;
   uint64_t lent_block_stride;
+  uint32_t layer_group;
+  uint64_t local_group_stride, lent_group_stride;
   uint8_t* slot_base;          // one layer: ring slot holding the layer, or NULL when not staged
   // several layers in one launch (grid.y = layer): strides to the next layer, and which layers are staged
   uint32_t num_layers, first_layer, ring_slots;
@@ -162,7 +177,7 @@ struct AppendParams {
   uint8_t* staging_base;
   uint32_t staged_mask[4];     // bit l: layer first_layer + l is validly staged for this batch
   uint64_t block_bytes;
-  const int32_t* home_entry;   // [nseq] table entry of the block holding token len-1
+  const int32_t* home_entry;   // [nseq] entry (physical index) of the block holding token len-1
   const int32_t* stage_pos;    // [nseq] staging position of that block, or -1
   const uint32_t* lens;        // [nseq]
   const void* k_new;           // [nseq][Hkv][128] bf16

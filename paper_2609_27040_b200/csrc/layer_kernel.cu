@@ -256,16 +256,17 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
 
   for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
     const uint32_t layer = p.first_layer + li;
-    const uint8_t* local_layer = p.local_layer + li * p.local_layer_stride;
+    const uint8_t* local_layer = p.local_base + layer_offset(layer, p.layer_group, p.local_group_stride, p.local_layer_stride);
     const uint8_t* slot_base = p.staging_base + (layer % p.ring_slots) * p.slot_bytes;
     unsigned long long* rw = range_words(p, li);
     uint32_t* seq_count = seq_counts(p, li);
     uint32_t cur_seq = kSentinel, nruns = 0, nclaims = 0;
     Cursor cur = first;
     // A staged block of this layer may be read once the gather issued during the previous layer of
-    // this launch has landed it (per-position ready flags carrying the layer's epoch); the first
-    // layer's gather precedes the launch in stream order, as does any gather the host skipped.
-    const bool check_ready = li > 0 && p.gather_target[li - 1] == static_cast<int16_t>(layer);
+    // this launch (prefetch_distance layers ahead of it) has landed it (per-position ready flags
+    // carrying the layer's epoch); the first layers' gathers precede the launch in stream order, as
+    // does any gather the host skipped.
+    const bool check_ready = li >= p.prefetch_distance && p.gather_target[li - p.prefetch_distance] == static_cast<int16_t>(layer);
     const uint32_t* ready = p.ready + static_cast<size_t>(layer % p.ring_slots) * p.ready_stride;
     const uint32_t epoch = p.epoch_base + li;
     uint64_t waited_ns = 0;
@@ -1135,12 +1136,12 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
                         p.total_blocks * p.Hkv, p.status);
       if (!ok) break;
     }
-    const uint8_t* src_layer = p.lent_base + static_cast<uint64_t>(target) * p.lent_layer_stride;
+    const uint8_t* src_layer = p.lent_base + layer_offset(static_cast<uint32_t>(target), p.layer_group, p.lent_group_stride, p.lent_layer_stride);
     uint8_t* dst_slot = const_cast<uint8_t*>(p.staging_base) + (static_cast<uint32_t>(target) % p.ring_slots) * p.slot_bytes;
     uint32_t* ticket = layer_counters(p, li) + kCntCopyTicket;
     // A landed block is announced by writing the target layer's epoch to its position's ready flag
     // (only when the target is attended to later in this launch).
-    const bool report = static_cast<uint32_t>(target) > p.first_layer && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
+    const bool report = static_cast<uint32_t>(target) > p.first_layer + li && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
     uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
     const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
     uint32_t my_pos[16];                  // positions of this thread's most recent units
@@ -1265,8 +1266,11 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   const uint32_t r = (len - 1) % p.block_tokens;
   const int32_t e = p.home_entry[i];
   const uint32_t y = blockIdx.y;  // layer within the launch
-  uint8_t* home = e >= 0 ? p.local_layer + y * p.local_layer_stride + static_cast<uint64_t>(e) * p.local_block_stride
-                         : p.lent_layer + y * p.lent_layer_stride + static_cast<uint64_t>(~e) * p.lent_block_stride;
+  const uint32_t layer = p.first_layer + y;
+  uint8_t* home = e >= 0 ? p.local_base + layer_offset(layer, p.layer_group, p.local_group_stride, p.local_layer_stride) +
+                               static_cast<uint64_t>(e) * p.local_block_stride
+                         : p.lent_base + layer_offset(layer, p.layer_group, p.lent_group_stride, p.lent_layer_stride) +
+                               static_cast<uint64_t>(~e) * p.lent_block_stride;
   const int32_t sp = p.stage_pos[i];
   uint8_t* slot = p.slot_base;
   if (p.num_layers > 1)

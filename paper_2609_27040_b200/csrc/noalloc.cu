@@ -79,6 +79,8 @@ cudaError_t static_scratch_setup(uint32_t Hkv, uint32_t G, uint32_t ncta) {
   LayerParams p{};  // no blocks, no sequences, no gather: every role finds nothing to do and returns
   p.num_layers = 1;
   p.ring_slots = 1;
+  p.layer_group = 1;
+  p.prefetch_distance = 1;
   p.per = 1;
   p.merge_inline = 1;
   p.part_buffers = 1;

@@ -54,6 +54,7 @@ struct Plan {
   size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_blk_off = 0, off_slot_base = 0,
          off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
+  std::vector<int32_t> resolved_ids;  // resolved table in block ids (the device copy holds physical indices)
   uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
   uint8_t* dev = nullptr;
   size_t cap = 0;
@@ -88,6 +89,14 @@ struct ema_slice {
   bool null_dev = false, profile = false, trace = false;
   uint64_t block_bytes = 0;
   uint64_t local_ls = 0, local_bs = 0, lent_ls = 0, lent_bs = 0, slot_bytes = 0;
+  // Layout of the arenas (Section 4.2): layers in groups of `group` (layer l of an arena starts at
+  // (l / group) * gs + (l % group) * ls), block ids in slabs of `slab` (physical index of id b within
+  // a layer: (b / slab) * W + b % slab; W = slab for the layer-major order, where it equals b).
+  uint32_t group = 1, slab = 0, layout = 0;
+  uint64_t local_gs = 0, lent_gs = 0;
+  uint32_t local_W = 0, lent_W = 0;
+  uint32_t layer_slots = 1;  // ring slots in layers: ring_slots groups of `group` layers
+  std::vector<uint32_t> slab_used_local, slab_used_lent;  // blocks in use per slab (slab allocator)
   int device = -1;  // the CUDA device the slice was created on
   int num_sms = 148;
   uint32_t ncta = 148;
@@ -177,6 +186,64 @@ namespace {
 inline uint32_t blocks_for(uint32_t len) { return (len + kBlockTokens - 1) / kBlockTokens; }
 
 inline bool multi_stream(const ema_slice* s) { return s->streams.size() > 1; }
+
+inline uint64_t local_off(const ema_slice* s, uint32_t l) { return ema::layer_offset(l, s->group, s->local_gs, s->local_ls); }
+inline uint64_t lent_off(const ema_slice* s, uint32_t l) { return ema::layer_offset(l, s->group, s->lent_gs, s->lent_ls); }
+
+// Table entry -> what the kernels index with: the block's physical index inside a layer of its
+// arena (the id itself in the layer-major order), lent entries staying negative (~index).
+inline int32_t phys_entry(const ema_slice* s, int32_t e) {
+  if (!s->layout) return e;
+  const uint32_t id = e >= 0 ? static_cast<uint32_t>(e) : static_cast<uint32_t>(~e);
+  const uint32_t W = e >= 0 ? s->local_W : s->lent_W;
+  const int32_t ph = static_cast<int32_t>(id / s->slab * W + id % s->slab);
+  return e >= 0 ? ph : ~ph;
+}
+
+// Slab allocator (Section 4.2.1): the next id of a part of the slice among the ids below `cap` that
+// are neither in use nor marked in `taken`: the lowest one lying in a slab of which `used` says
+// that it holds blocks already (the user fills the slabs it has), else the lowest one of all (it
+// opens the lowest free slab). -1 when there is none. `used` counts blocks per slab, those marked
+// taken included.
+int32_t slab_choose(const std::vector<Owner>& own, const std::vector<uint32_t>& used, const std::vector<char>* taken,
+                    uint32_t S, uint32_t cap) {
+  const uint32_t nslabs = (cap + S - 1) / S;
+  int32_t fresh = -1;
+  for (uint32_t sl = 0; sl < nslabs; ++sl) {
+    const uint32_t first = sl * S, avail = std::min(S, cap - first);
+    if (used[sl] >= S) continue;                // full
+    if (used[sl] == 0) {                        // a free slab: remembered, taken only if no slab in use has room
+      if (fresh < 0) fresh = static_cast<int32_t>(first);
+      continue;
+    }
+    // In use (possibly only by ids at or above cap, which count but cannot be handed out).
+    for (uint32_t id = first; id < first + avail; ++id)
+      if (own[id].seq < 0 && !(taken && (*taken)[id])) return static_cast<int32_t>(id);
+  }
+  return fresh;
+}
+
+void recount_slabs(ema_slice* s) {
+  if (!s->slab) return;
+  std::fill(s->slab_used_local.begin(), s->slab_used_local.end(), 0u);
+  std::fill(s->slab_used_lent.begin(), s->slab_used_lent.end(), 0u);
+  for (size_t id = 0; id < s->owner_local.size(); ++id) s->slab_used_local[id / s->slab] += s->owner_local[id].seq >= 0;
+  for (size_t id = 0; id < s->owner_lent.size(); ++id) s->slab_used_lent[id / s->slab] += s->owner_lent[id].seq >= 0;
+}
+
+// Takes the next free id of a tier: the top of the free stack, or the slab rule's choice.
+int32_t take_free(ema_slice* s, bool local) {
+  std::vector<int32_t>& stack = local ? s->free_local : s->free_lent;
+  if (!s->slab) {
+    const int32_t id = stack.back();
+    stack.pop_back();
+    return id;
+  }
+  const int32_t id = slab_choose(local ? s->owner_local : s->owner_lent, local ? s->slab_used_local : s->slab_used_lent,
+                                 nullptr, s->slab, local ? s->cfg.local_blocks : s->lent_cap);
+  stack.erase(std::find(stack.begin(), stack.end(), id));
+  return id;
+}
 
 // Blocks the user holds in both parts of the slice.
 inline uint32_t blocks_held(const ema_slice* s) {
@@ -353,6 +420,7 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   int32_t* stage_pos = reinterpret_cast<int32_t*>(p.host + p.off_stage_pos);
 
   p.blk_off.resize(nseq + 1);
+  p.resolved_ids.resize(total);
   uint32_t flat = 0, kk = 0, slots = 0, slots_static = 0;
   for (uint32_t i = 0; i < nseq; ++i) {
     const Seq& q = s->seqs[seqs[i]];
@@ -371,10 +439,12 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
     const uint32_t last_b = q.len ? (q.len - 1) / kBlockTokens : 0;
     for (uint32_t b = 0; b < nb; ++b) {
       const int32_t e = q.table[b];
-      int32_t r = e;
+      int32_t r = phys_entry(s, e);
+      p.resolved_ids[flat] = e;
       if (e < 0) {
-        copy_src[kk] = e;  // negative entry: tier 1 (lent arena), id ~e
+        copy_src[kk] = r;  // negative entry: tier 1 (lent arena), physical index ~r
         r = ~static_cast<int32_t>(kk);
+        p.resolved_ids[flat] = r;
         pos_range[kk] = flat / per;
         pos_rank[kk] = range_staged[flat / per]++;
         ++kk;
@@ -382,7 +452,7 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
       resolved[flat] = r;
       blk_seq[flat] = i;
       if (b == last_b) {
-        home[i] = e;
+        home[i] = phys_entry(s, e);
         stage_pos[i] = e < 0 ? ~r : -1;
       }
       ++flat;
@@ -441,15 +511,15 @@ int prof_record(ema_slice* s, uint32_t layer, int which, cudaStream_t stream) {
 }
 
 bool staged(const ema_slice* s, uint32_t layer, const Plan* p) {
-  const SlotState& sl = s->slots[layer % s->cfg.ring_slots];
+  const SlotState& sl = s->slots[layer % s->layer_slots];
   return sl.valid && sl.layer == layer && sl.plan_serial == p->serial;
 }
 
 // Describes the gather of `layer`'s lent blocks into its ring slot.
 void fill_gather(const ema_slice* s, uint32_t layer, const Plan* p, ema::CopyDesc& d) {
-  const uint32_t slot = layer % s->cfg.ring_slots;
+  const uint32_t slot = layer % s->layer_slots;
   d = ema::CopyDesc{};
-  d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.lent_base) + lent_off(s, layer);
   d.src_block_stride[0] = d.src_block_stride[1] = s->lent_bs;
   d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
   d.dst_block_stride[0] = d.dst_block_stride[1] = s->block_bytes;
@@ -492,7 +562,7 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
   if (rc) return rc;
   rc = plan_on_stream(s, p, side);
   if (rc) return rc;
-  SlotState& sl = s->slots[layer % s->cfg.ring_slots];
+  SlotState& sl = s->slots[layer % s->layer_slots];
   if (!s->null_dev) {
     rc = order_before_slot_write(s, sl, side);
     if (rc) return rc;
@@ -536,12 +606,15 @@ int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots, uint32_t buffers 
 void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_t first_layer, uint32_t num_layers,
                  const void* q, void* out, uint32_t Hq, float sm_scale, bool steal) {
   const uint32_t Hkv = s->cfg.num_kv_heads;
-  d.local_layer = static_cast<const uint8_t*>(s->cfg.local_base) + first_layer * s->local_ls;
+  d.local_base = static_cast<const uint8_t*>(s->cfg.local_base);
+  d.local_group_stride = s->local_gs;
   d.local_layer_stride = s->local_ls;
   d.local_block_stride = s->local_bs;
+  d.layer_group = s->group;
+  d.prefetch_distance = s->group;
   d.staging_base = static_cast<const uint8_t*>(s->cfg.staging_base);
   d.slot_bytes = s->slot_bytes;
-  d.ring_slots = s->cfg.ring_slots;
+  d.ring_slots = s->layer_slots;
   d.first_layer = first_layer;
   d.num_layers = num_layers;
   d.block_bytes = s->block_bytes;
@@ -584,6 +657,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.G = Hq / Hkv;
   d.scale_log2 = sm_scale * 1.4426950408889634f;
   d.lent_base = static_cast<const uint8_t*>(s->cfg.lent_base);
+  d.lent_group_stride = s->lent_gs;
   d.lent_layer_stride = s->lent_ls;
   d.lent_block_stride = s->lent_bs;
   d.copy_src = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
@@ -603,7 +677,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
 int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out, float* lse,
              cudaStream_t stream, int next_layer, bool static_scratch, bool counters_zeroed) {
   const uint32_t Hkv = s->cfg.num_kv_heads;
-  const uint32_t R = s->cfg.ring_slots;
+  const uint32_t R = s->layer_slots;
   if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
   if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
   const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
@@ -677,13 +751,16 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
 // layer's lent blocks, layer boundaries soft (see layer_kernel.cu). The caller has primed layer 0.
 int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, void* out, cudaStream_t stream,
             bool wrap) {
-  const uint32_t Hkv = s->cfg.num_kv_heads, L = s->cfg.num_layers, R = s->cfg.ring_slots;
+  const uint32_t Hkv = s->cfg.num_kv_heads, L = s->cfg.num_layers, R = s->layer_slots, K = s->group;
   if (Hq == 0 || Hq % Hkv != 0 || Hq / Hkv > 8) return SLICE_EINVAL;
   if (!s->null_dev && (!q || !out)) return SLICE_EINVAL;
   const uint32_t* lens = reinterpret_cast<const uint32_t*>(p->host + p->off_lens);
   for (uint32_t i = 0; i < p->nseq; ++i)
     if (lens[i] == 0) return SLICE_EINVAL;
-  if (p->k && !staged(s, 0, p)) return SLICE_ESTALE;
+  // The first layer group is staged before the launch; inside it, the gather issued during layer l
+  // fetches layer l + K (the same layer of the next group).
+  for (uint32_t l = 0; p->k && l < std::min(K, L); ++l)
+    if (!staged(s, l, p)) return SLICE_ESTALE;
   // Plan the gathers by following what each ring slot will hold.
   std::vector<int64_t> holds(R, -1);
   for (uint32_t r = 0; r < R; ++r)
@@ -694,10 +771,14 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     target[l] = after[l] = -1;
     if (!p->k) continue;
     int64_t t = -1;
-    if (l + 1 < L)
-      t = l + 1;
-    else if (wrap && L > 1 && (L - 1) % R != 0)
-      t = 0;
+    if (l + K < L) {
+      t = l + K;
+    } else if (wrap && L > 1) {
+      // A layer of the next pass's first group, unless its slot still serves a layer of this pass.
+      t = static_cast<int64_t>(l) + K - L;
+      for (uint32_t j = l; j < L; ++j)
+        if (j % R == t % R) t = -1;
+    }
     if (t < 0 || holds[t % R] == t) continue;  // nothing to fetch, or the slot still holds that layer
     target[l] = static_cast<int16_t>(t);
     for (int64_t j = static_cast<int64_t>(l) - 1; j >= 0; --j)
@@ -843,6 +924,18 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
   if (cfg->pipeline_mode > 2 || cfg->static_split > 1 || cfg->prefetch_priority > 1) return SLICE_EINVAL;
+  // Section 4.2: slabs, layer groups, layouts.
+  const uint32_t group = cfg->layer_group ? cfg->layer_group : 1u, slab = cfg->slab_blocks;
+  if (cfg->layout > 2 || group > cfg->num_layers) return SLICE_EINVAL;
+  if (slab && (cfg->local_free_order || cfg->lent_free_order)) return SLICE_EINVAL;  // the slab rule fixes the order
+  if (cfg->layout != 0) {
+    // The slab-major and layer-group-major orders are defined over whole slabs and whole groups,
+    // and exclude caller-chosen strides.
+    if (!slab || cfg->local_blocks % slab || cfg->lent_blocks_physical % slab || cfg->num_layers % group) return SLICE_EINVAL;
+    if (cfg->local_layer_stride || cfg->local_block_stride || cfg->lent_layer_stride || cfg->lent_block_stride)
+      return SLICE_EINVAL;
+  }
+  if (static_cast<uint64_t>(cfg->ring_slots) * group > 4096) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
@@ -882,6 +975,28 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   s->lent_bs = cfg->lent_block_stride ? cfg->lent_block_stride : bb;
   s->lent_ls = cfg->lent_layer_stride ? cfg->lent_layer_stride : bb * cfg->lent_blocks_physical;
   s->slot_bytes = bb * cfg->staging_blocks_per_slot;
+  s->group = group;
+  s->slab = slab;
+  s->layout = cfg->layout;
+  s->layer_slots = cfg->ring_slots * group;
+  if (cfg->layout == 0) {          // [layer][id]: groups are just runs of layers
+    s->local_gs = group * s->local_ls;
+    s->lent_gs = group * s->lent_ls;
+    s->local_W = s->lent_W = slab;
+  } else if (cfg->layout == 1) {   // slab-major [slab][layer][block in slab]
+    s->local_ls = s->lent_ls = bb * slab;
+    s->local_gs = s->lent_gs = bb * slab * group;
+    s->local_W = s->lent_W = cfg->num_layers * slab;
+  } else {                         // layer-group-major [group][slab][layer in group][block in slab]
+    s->local_ls = s->lent_ls = bb * slab;
+    s->local_gs = bb * slab * group * (cfg->local_blocks / slab);
+    s->lent_gs = bb * slab * group * (cfg->lent_blocks_physical / slab);
+    s->local_W = s->lent_W = group * slab;
+  }
+  if (slab) {
+    s->slab_used_local.assign((cfg->local_blocks + slab - 1) / slab, 0u);
+    s->slab_used_lent.assign((cfg->lent_blocks_physical + slab - 1) / slab, 0u);
+  }
   s->lent_cap = cfg->lent_blocks;
   s->owner_local.assign(cfg->local_blocks, Owner());
   s->owner_lent.assign(cfg->lent_blocks_physical, Owner());
@@ -891,7 +1006,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     const uint32_t id = cfg->lent_free_order ? cfg->lent_free_order[k] : k;
     if (id < cfg->lent_blocks) s->free_lent.push_back(static_cast<int32_t>(id));
   }
-  s->slots.resize(cfg->ring_slots);
+  s->slots.resize(s->layer_slots);
 
   auto fail = [&](int code) {
     destroy_impl(s);
@@ -942,7 +1057,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     if (cudaMalloc(reinterpret_cast<void**>(&s->cnt_dev), cnt_words * sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(s->cnt_dev, 0, cnt_words * sizeof(uint32_t)) != cudaSuccess)
       return fail(SLICE_ECUDA);
-    const size_t rd = static_cast<size_t>(cfg->ring_slots) * std::max(cfg->staging_blocks_per_slot, 1u) * sizeof(uint32_t);
+    const size_t rd = static_cast<size_t>(s->layer_slots) * std::max(cfg->staging_blocks_per_slot, 1u) * sizeof(uint32_t);
     if (cudaMalloc(reinterpret_cast<void**>(&s->ready_dev), rd) != cudaSuccess || cudaMemset(s->ready_dev, 0, rd) != cudaSuccess)
       return fail(SLICE_ECUDA);
     if (cudaMalloc(reinterpret_cast<void**>(&s->q_flags_dev), ema::kMaxStepLayers * sizeof(uint32_t)) != cudaSuccess ||
@@ -1008,10 +1123,9 @@ int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t hint, int32_
   Seq& q = s->seqs[seq];
   for (uint32_t k = 0; k < n; ++k) {
     const bool local = hint == SLICE_TIER_LOCAL || (hint == SLICE_TIER_AUTO && !s->free_local.empty());
-    std::vector<int32_t>& stack = local ? s->free_local : s->free_lent;
-    const int32_t id = stack.back();
-    stack.pop_back();
+    const int32_t id = take_free(s, local);
     (local ? s->owner_local : s->owner_lent)[id] = Owner{seq, static_cast<int32_t>(q.table.size())};
+    if (s->slab) ++(local ? s->slab_used_local : s->slab_used_lent)[id / s->slab];
     const int32_t entry = local ? id : ~id;
     q.table.push_back(entry);
     if (out_entries) out_entries[k] = entry;
@@ -1042,9 +1156,11 @@ int slice_free_seq(slice_t* s, int32_t seq) {
     if (e >= 0) {
       s->free_local.push_back(e);
       s->owner_local[e] = Owner();
+      if (s->slab) --s->slab_used_local[e / s->slab];
     } else {
       s->free_lent.push_back(~e);
       s->owner_lent[~e] = Owner();
+      if (s->slab) --s->slab_used_lent[~e / s->slab];
     }
   }
   s->seqs.erase(it);
@@ -1121,11 +1237,32 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
   // Plan first: destinations in ascending victim order, local ids before lent ids.
   const size_t n_local = std::min(victims.size(), s->free_local.size());
   const size_t n_lent = victims.size() - n_local;
-  std::vector<int32_t> sorted_below(below);
-  std::sort(sorted_below.begin(), sorted_below.end());
   std::vector<int32_t> dst(victims.size());
-  for (size_t k = 0; k < n_local; ++k) dst[k] = s->free_local[s->free_local.size() - 1 - k];
-  for (size_t k = 0; k < n_lent; ++k) dst[n_local + k] = ~sorted_below[k];
+  if (!s->slab) {
+    std::vector<int32_t> sorted_below(below);
+    std::sort(sorted_below.begin(), sorted_below.end());
+    for (size_t k = 0; k < n_local; ++k) dst[k] = s->free_local[s->free_local.size() - 1 - k];
+    for (size_t k = 0; k < n_lent; ++k) dst[n_local + k] = ~sorted_below[k];
+  } else {
+    // Slab allocator: every victim goes where the next allocation would go, each choice seeing the
+    // ones before it (scratch copies; nothing is committed yet).
+    std::vector<uint32_t> used_l(s->slab_used_local), used_r(s->slab_used_lent);
+    std::vector<char> taken_l(s->owner_local.size(), 0), taken_r(s->owner_lent.size(), 0);
+    for (size_t k = 0; k < victims.size(); ++k) {
+      if (k < n_local) {
+        const int32_t id = slab_choose(s->owner_local, used_l, &taken_l, s->slab, s->cfg.local_blocks);
+        taken_l[id] = 1;
+        ++used_l[id / s->slab];
+        dst[k] = id;
+      } else {
+        const int32_t id = slab_choose(s->owner_lent, used_r, &taken_r, s->slab, cut);
+        taken_r[id] = 1;
+        ++used_r[id / s->slab];
+        dst[k] = ~id;
+      }
+      --used_r[victims[k] / s->slab];  // this victim has left its slab before the next one is placed
+    }
+  }
 
   // Test hook: the step that enqueues the migration fails, as a CUDA call might; nothing is committed.
   if ((s->cfg.flags & SLICE_FLAG_TEST_FAIL_COPY) && !victims.empty()) {
@@ -1143,9 +1280,9 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
       CU(s, cudaStreamWaitEvent(stream, s->ev_tmp, 0));
     }
     const size_t n = victims.size();
-    for (size_t k = 0; k < n; ++k) {
-      s->reclaim_host[k] = ~victims[k];
-      s->reclaim_host[n + k] = dst[k];
+    for (size_t k = 0; k < n; ++k) {  // physical indices for the kernel
+      s->reclaim_host[k] = phys_entry(s, ~victims[k]);
+      s->reclaim_host[n + k] = phys_entry(s, dst[k]);
     }
     CU(s, cudaMemcpyAsync(s->reclaim_dev, s->reclaim_host, 2 * n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
     ema::CopyDesc d{};
@@ -1158,6 +1295,9 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
     d.dst_base[1] = static_cast<uint8_t*>(s->cfg.lent_base);
     d.dst_block_stride[1] = s->lent_bs;
     d.dst_layer_stride[1] = s->lent_ls;
+    d.layer_group = s->group;
+    d.src_group_stride[0] = d.src_group_stride[1] = d.dst_group_stride[1] = s->lent_gs;
+    d.dst_group_stride[0] = s->local_gs;
     d.src_entry = s->reclaim_dev;
     d.dst_entry = s->reclaim_dev + n;
     d.n = static_cast<uint32_t>(n);
@@ -1186,7 +1326,10 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
     const int32_t v = victims[k];
     const Owner own = s->owner_lent[v];
     if (k < n_local) {
-      s->free_local.pop_back();
+      if (s->slab)
+        s->free_local.erase(std::find(s->free_local.begin(), s->free_local.end(), dst[k]));
+      else
+        s->free_local.pop_back();
       s->owner_local[dst[k]] = own;
     } else {
       const int32_t id = ~dst[k];
@@ -1196,6 +1339,7 @@ int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* str
     s->seqs[own.seq].table[own.logical] = dst[k];
     s->owner_lent[v] = Owner();
   }
+  recount_slabs(s);
   s->lent_cap = cut;
   bump_version(s);
   invalidate_staged(s);
@@ -1325,6 +1469,7 @@ int slice_reclaim_preempt(slice_t* s, uint32_t take, uint32_t slab_blocks, int32
         }
         s->seqs[kv.first] = std::move(kv.second);
       }
+      recount_slabs(s);
       // The plans built meanwhile saw none of this; a new version keeps them from being reused.
       s->version = keep.version;
       bump_version(s);
@@ -1406,20 +1551,23 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   ema::AppendParams a{};
   bool one_staged = false;
   for (uint32_t l = first; l < first + count; ++l) {
-    SlotState& sl = s->slots[l % s->cfg.ring_slots];
+    SlotState& sl = s->slots[l % s->layer_slots];
     if (!staged(s, l, p)) continue;
     if (sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
     a.staged_mask[(l - first) >> 5] |= 1u << ((l - first) & 31u);
     one_staged = true;
   }
-  a.local_layer = static_cast<uint8_t*>(s->cfg.local_base) + first * s->local_ls;
+  a.local_base = static_cast<uint8_t*>(s->cfg.local_base);
   a.local_block_stride = s->local_bs;
-  a.lent_layer = static_cast<uint8_t*>(s->cfg.lent_base) + first * s->lent_ls;
+  a.lent_base = static_cast<uint8_t*>(s->cfg.lent_base);
   a.lent_block_stride = s->lent_bs;
-  a.slot_base = (count == 1 && one_staged) ? static_cast<uint8_t*>(s->cfg.staging_base) + (first % s->cfg.ring_slots) * s->slot_bytes : nullptr;
+  a.layer_group = s->group;
+  a.local_group_stride = s->local_gs;
+  a.lent_group_stride = s->lent_gs;
+  a.slot_base = (count == 1 && one_staged) ? static_cast<uint8_t*>(s->cfg.staging_base) + (first % s->layer_slots) * s->slot_bytes : nullptr;
   a.num_layers = count;
   a.first_layer = first;
-  a.ring_slots = s->cfg.ring_slots;
+  a.ring_slots = s->layer_slots;
   a.local_layer_stride = s->local_ls;
   a.lent_layer_stride = s->lent_ls;
   a.io_layer_stride = static_cast<uint64_t>(nseq) * s->cfg.num_kv_heads * kHeadDim * 2;
@@ -1448,7 +1596,7 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   Plan* p = nullptr;
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
-  const uint32_t slot = layer % s->cfg.ring_slots;
+  const uint32_t slot = layer % s->layer_slots;
   SlotState& sl = s->slots[slot];
   if (!staged(s, layer, p)) return SLICE_ESTALE;
   if (s->null_dev || p->k == 0) return SLICE_OK;
@@ -1460,7 +1608,7 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   ema::CopyDesc d{};
   d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
   d.src_block_stride[0] = d.src_block_stride[1] = s->block_bytes;
-  d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.lent_base) + layer * s->lent_ls;
+  d.dst_base[0] = d.dst_base[1] = static_cast<uint8_t*>(s->cfg.lent_base) + lent_off(s, layer);
   d.dst_block_stride[0] = d.dst_block_stride[1] = s->lent_bs;
   d.src_entry = nullptr;
   d.dst_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
@@ -1518,11 +1666,11 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   Plan* p = nullptr;
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
-  const uint32_t L = s->cfg.num_layers, R = s->cfg.ring_slots;
+  const uint32_t L = s->cfg.num_layers, R = s->layer_slots, K = s->group;
   // Mode 0: one launch for the whole pass when the shape allows it, else one launch per layer.
-  const bool step = s->cfg.pipeline_mode == 0 && R >= 2 && L >= 2 && L <= ema::kMaxStepLayers &&
+  const bool step = s->cfg.pipeline_mode == 0 && s->cfg.ring_slots >= 2 && L >= 2 && L <= ema::kMaxStepLayers &&
                     s->ncta <= static_cast<uint32_t>(s->num_sms);
-  const bool fused = s->cfg.pipeline_mode != 1 && R >= 2;
+  const bool fused = s->cfg.pipeline_mode != 1 && s->cfg.ring_slots >= 2;
   if (fused) side = stream;
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
   const uint8_t* qd = static_cast<const uint8_t*>(q);
@@ -1617,8 +1765,9 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   }
   if (!s->null_dev)  // the work counters of all layers, cleared once per pass
     CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * s->cnt_stride * sizeof(uint32_t), stream));
-  if (p->k && !staged(s, 0, p)) {
-    rc = do_prefetch(s, 0, p, side);
+  for (uint32_t l = 0; p->k && l < std::min(K, L); ++l) {  // the first layer group
+    if (staged(s, l, p)) continue;
+    rc = do_prefetch(s, l, p, side);
     if (rc) return rc;
   }
   if (step) {
@@ -1638,10 +1787,13 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
     // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.
     int next = -1;
     if (p->k) {
-      if (l + 1 < L)
-        next = static_cast<int>(l + 1);
-      else if (wrap && L > 1 && (L - 1) % R != 0)
-        next = 0;
+      if (l + K < L) {
+        next = static_cast<int>(l + K);
+      } else if (wrap && L > 1) {
+        next = static_cast<int>(l + K - L);
+        for (uint32_t j = l; j < L; ++j)
+          if (j % R == static_cast<uint32_t>(next) % R) next = -1;  // its slot still serves this pass
+      }
       if (next >= 0 && staged(s, static_cast<uint32_t>(next), p)) next = -1;
     }
     if (fused) {
@@ -1663,9 +1815,11 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
       }
     }
   }
-  if (p->k && wrap && L > 1 && (L - 1) % R == 0 && !staged(s, 0, p)) {
-    // The last layer shares its ring slot with layer 0: refill it only after that attention.
-    rc = do_prefetch(s, 0, p, side);
+  for (uint32_t l = 0; p->k && wrap && L > 1 && l < std::min(K, L); ++l) {
+    // Layers of the next pass's first group whose ring slot served a layer of this pass to the end:
+    // refilled only after that attention.
+    if (staged(s, l, p)) continue;
+    rc = do_prefetch(s, l, p, side);
     if (rc) return rc;
   }
   if (streamed_q) {
@@ -1765,10 +1919,9 @@ int slice_get_resolved(slice_t* s, const int32_t* seqs, uint32_t nseq, int32_t* 
   if (out) {
     const uint32_t stride = s->cfg.max_blocks_per_seq;
     if (static_cast<uint64_t>(cap) < static_cast<uint64_t>(nseq) * stride) return SLICE_EINVAL;
-    const int32_t* resolved = reinterpret_cast<const int32_t*>(p->host + p->off_resolved);
     for (uint32_t i = 0; i < nseq; ++i)
       for (uint32_t f = p->blk_off[i]; f < p->blk_off[i + 1]; ++f)
-        out[static_cast<size_t>(i) * stride + (f - p->blk_off[i])] = resolved[f];
+        out[static_cast<size_t>(i) * stride + (f - p->blk_off[i])] = p->resolved_ids[f];
   }
   return SLICE_OK;
 }

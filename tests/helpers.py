@@ -17,13 +17,17 @@ class Scenario:
     def __init__(self, wl: synth.Workload, seed: int, poison: bool = False, slack: int = 16,
                  num_layers: int | None = None, lent_extra_physical: int = 0,
                  lengths: np.ndarray | None = None, permute: bool = True,
-                 max_blocks_per_seq: int | None = None):
+                 max_blocks_per_seq: int | None = None, slab_blocks: int = 0):
         self.wl = wl
         self.seed = seed
         self.L = wl.num_layers if num_layers is None else num_layers
         self.T, self.Hkv, self.Hq, self.D = wl.block_tokens, wl.num_kv_heads, wl.num_q_heads, wl.head_dim
-        self.pl = synth.make_placement(wl, seed, slack_blocks=slack, permute=permute, lengths=lengths)
+        self.slab = slab_blocks
+        self.pl = synth.make_placement(wl, seed, slack_blocks=slack, permute=permute and not slab_blocks, lengths=lengths)
         pl = self.pl
+        if slab_blocks:          # slab allocator: whole slabs, ids in the order the slab rule gives (no seeded order)
+            pl.local_blocks = -(-pl.local_blocks // slab_blocks) * slab_blocks
+            pl.lent_blocks = -(-(pl.lent_blocks + lent_extra_physical) // slab_blocks) * slab_blocks - lent_extra_physical
         self.nseq = len(pl.lengths)
         self.lent_phys = pl.lent_blocks + lent_extra_physical
         self.staging_cap = max(pl.staging_blocks, 1)
@@ -39,6 +43,8 @@ class Scenario:
                                       self.lent_phys, wl.ring_slots, self.staging_cap,
                                       max_seqs=max(self.nseq, 1) + 4, max_blocks_per_seq=self.max_blocks,
                                       local_free_order=self.local_order, lent_free_order=self.lent_order)
+        if slab_blocks:
+            assert self.orc.set_slab_blocks(slab_blocks) == oracle.OK
         self.seq_ids = list(pl.seq_ids)
         # one allocation call per block, in logical order, with the drawn tier hint
         for i, hints in zip(self.seq_ids, pl.hints):

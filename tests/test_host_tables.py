@@ -39,8 +39,8 @@ def test_library_exports_every_declared_entry_point():
 
 
 def test_config_struct_matches_header_size():
-    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 8 uint32
-    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 8 * 4
+    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 11 uint32 (+ 4 bytes of tail padding)
+    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 11 * 4 + 4
 
 
 def test_create_rejects_bad_configs():
@@ -411,3 +411,102 @@ def test_slice_choice_matches_oracle(seed):
         B.slice_schedule_gll([])
     for sl in slices:
         sl.close()
+
+
+@pytest.mark.parametrize("seed,slab", [(0, 4), (1, 3), (2, 10), (3, 1)])
+def test_slab_allocator_matches_oracle_state_machine(seed, slab):
+    """Slab allocator (Section 4.2.1) in the library and in the oracle over random allocations,
+    frees, reclaims (plain and by preemption) and lends: the same ids in the same order, the same
+    migration destinations, the same free ids (as sets: in slab mode the rule, not a stack, orders
+    them), capacities not multiples of the slab."""
+    rng = np.random.default_rng(300 + seed)
+    LB, RB, PH, CAP = 23, 17, 26, 26
+    s = B.Slice(2, 8, LB, RB, CAP, lent_blocks_physical=PH, max_seqs=10, max_blocks_per_seq=9,
+                flags=B.FLAG_NULL_DEVICE, slab_blocks=slab)
+    o = oracle.OracleSlice(2, 16, 65536, LB, RB, PH, 2, CAP, max_seqs=10, max_blocks_per_seq=9)
+    assert o.set_slab_blocks(slab) == 0
+    live = set()
+    moved = evicted = 0
+    for step in range(2500):
+        op = int(rng.integers(0, 12))
+        if op < 6:
+            q, n, hint = int(rng.integers(0, 12)), int(rng.integers(0, 5)), int(rng.integers(0, 3))
+            rc1, e1 = s.slice_alloc_blocks(q, n, hint)
+            rc2, e2 = o.alloc_blocks(q, n, hint)
+            assert rc1 == rc2
+            if rc1 == 0:
+                assert e1.tolist() == e2.tolist()
+                live.add(q)
+        elif op == 6:
+            q = int(rng.integers(0, 12))
+            assert s.slice_free_seq(q) == o.free_seq(q)
+            live.discard(q)
+        elif op == 7:
+            take = int(rng.integers(0, 7))
+            rc1, m1 = s.slice_reclaim(take)
+            rc2, m2 = o.reclaim(take, None, None)
+            assert rc1 == rc2 and (rc1 != 0 or m1 == m2)
+            moved += m1 if rc1 == 0 else 0
+        elif op == 8:
+            take, sb = int(rng.integers(0, 9)), int(rng.integers(1, 6))
+            rc1, v1, m1 = s.slice_reclaim_preempt(take, sb)
+            rc2, v2, m2 = o.reclaim_preempt(take, sb, None, None)
+            assert rc1 == rc2 and v1 == v2 and (rc1 != 0 or m1 == m2)
+            if rc1 == 0:
+                live -= set(v1)
+                evicted += len(v1)
+        elif op == 9:
+            n = int(rng.integers(0, 6))
+            assert s.slice_lend(n) == o.lend(n)
+        elif live:
+            batch = [int(x) for x in rng.permutation(sorted(live))[: int(rng.integers(1, len(live) + 1))]]
+            rc2, r2, k2 = o.gather(0, batch, None, None)
+            rc1, r1, k1 = s.slice_get_resolved(batch)
+            assert rc1 == rc2 and (rc1 != 0 or (k1 == k2 and (r1 == r2).all()))
+        for q in live:
+            assert s.slice_get_block_table(q)[1].tolist() == o.block_table(q)[1].tolist()
+        assert sorted(s.slice_get_free_stack(B.TIER_LOCAL).tolist()) == sorted(o.free_stack(oracle.LOCAL).tolist())
+        assert sorted(s.slice_get_free_stack(B.TIER_LENT).tolist()) == sorted(o.free_stack(oracle.LENT).tolist())
+        assert s.slice_stats()["lent_capacity"] == o.lent_capacity
+    assert moved > 0 and evicted > 0
+    s.close()
+
+
+def test_layout_and_group_configurations_are_validated():
+    ok = dict(lent_blocks_physical=20, max_seqs=4, max_blocks_per_seq=8, flags=B.FLAG_NULL_DEVICE)
+    B.Slice(8, 8, 20, 20, 8, slab_blocks=10, layer_group=4, layout=B.LAYOUT_LAYER_GROUP_MAJOR, **ok).close()
+    B.Slice(8, 8, 20, 20, 8, slab_blocks=5, layer_group=2, layout=B.LAYOUT_SLAB_MAJOR, **ok).close()
+    B.Slice(8, 8, 23, 20, 8, slab_blocks=10, layer_group=3, **ok).close()       # layer-major: no divisibility needed
+    for bad in (dict(layout=3), dict(layout=1), dict(layout=2, slab_blocks=10, layer_group=3),
+                dict(layout=1, slab_blocks=7), dict(layer_group=9), dict(layout=1, slab_blocks=10, lent_block_stride=65536),
+                dict(slab_blocks=4, local_free_order=np.arange(20, dtype=np.uint32))):
+        with pytest.raises(B.SliceError):
+            B.Slice(8, 8, 20, 20, 8, **{**ok, **bad})
+
+
+@pytest.mark.parametrize("group,ring,layers,first,second", [(1, 2, 8, 9, 8), (4, 2, 8, 8, 0), (2, 2, 8, 10, 8), (2, 3, 7, 8, 2),
+                                                            (4, 1, 8, 12, 8), (3, 2, 5, 5, 0)])
+def test_decode_step_prefetches_one_layer_group_ahead(group, ring, layers, first, second):
+    """Layer groups (Section 4.2.2): a ring slot holds one group, the pass fetches layer l + k while
+    layer l runs and the first group of the next pass at its end. Tables-only mode, every pipeline:
+    the counts are worked out by hand. (1,2,8): layer 0, then 1..7 inside the pass, then layer 0 again
+    = 9, later passes 8. (4,2,8) and (3,2,5): the ring holds the whole model, every layer is fetched
+    once and stays. (2,2,8): 0,1 then 2..7 then 0,1 = 10, later 8. (2,3,7): six layer slots for
+    seven layers: 0,1 then 2..6, layer 6 displacing layer 0, which is fetched again once layer 6 has
+    been attended to = 8; later passes fetch only those two.
+    (4,1,8): a ring of one group: every fetch follows the attention that frees its slot: 12, later 8."""
+    for mode in (0, 1, 2):
+        s = B.Slice(layers, 4, 64, 64, 64, lent_blocks_physical=64, ring_slots=ring, max_seqs=8, max_blocks_per_seq=64,
+                    flags=B.FLAG_NULL_DEVICE, pipeline_mode=mode, layer_group=group)
+        for i in range(3):
+            for b in range(10):
+                assert s.slice_alloc_blocks(i, 1, B.TIER_LENT if b % 2 else B.TIER_LOCAL)[0] == B.OK
+            assert s.slice_set_seq_len(i, 150) == B.OK
+        seqs = np.arange(3, dtype=np.int32)
+        assert s.slice_decode_step(seqs, None, 16, 0.1, None, False, True, None, None) == B.OK
+        st1 = s.slice_stats()
+        assert st1["prefetch_calls"] == first and st1["decode_calls"] == layers, (mode, st1["prefetch_calls"])
+        assert s.slice_decode_step(seqs, None, 16, 0.1, None, False, True, None, None) == B.OK
+        st2 = s.slice_stats()
+        assert st2["prefetch_calls"] - first == second and st2["decode_calls"] == 2 * layers, (mode, st2["prefetch_calls"])
+        s.slice_destroy()
