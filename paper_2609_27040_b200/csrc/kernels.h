@@ -126,8 +126,10 @@ struct LayerParams {
   // (-1: ordered by the stream already).
   const uint8_t* lent_base;     // lent arena (same addressing as the local one)
   uint64_t lent_group_stride, lent_layer_stride, lent_block_stride;
-  const int32_t* copy_src;      // [copy_n] lent entries in staging order
-  const uint32_t* copy_order;   // [copy_n] staging positions in the order they are gathered
+  const int32_t* copy_src;      // lent entries (~physical index) by staging position
+  const uint32_t* copy_order;   // [copy_n] copy units in the order they are gathered: first staging position
+                                //   (low 24 bits) and blocks - 1 (high 8 bits) of a run of blocks that
+                                //   are neighbours in the lent arena and in the slot
   uint32_t copy_n;
   uint32_t* ready;              // [ring_slots][ready_stride] per staged position: epoch of the layer
   uint32_t ready_stride;        //   whose block has landed there (multi-layer launches)

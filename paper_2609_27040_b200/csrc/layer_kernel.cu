@@ -1116,7 +1116,6 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
 // copy warp (one thread): the gathers issued during each layer of the launch
 // ---------------------------------------------------------------------------------------------
 __device__ void copy_role(const LayerParams& p, const Smem& sm) {
-  const uint32_t pieces = static_cast<uint32_t>((p.block_bytes + kCopyChunk - 1) / kCopyChunk);
   const uint32_t ring = ptx::smem_u32(sm.copy_ring);
   const uint64_t pol = ptx::policy_evict_first();
   const uint64_t pol_keep = ptx::policy_evict_last();  // staged lines: wanted again within a layer's time
@@ -1144,30 +1143,39 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     const bool report = static_cast<uint32_t>(target) > p.first_layer + li && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
     uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
     const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
-    uint32_t my_pos[16];                  // positions of this thread's most recent units
+    // A unit is a run of blocks that are neighbours both in the lent arena and in the slot (one block
+    // when blocks are 64 KB; up to 64 KB worth of smaller blocks that the slab allocator kept together).
+    uint32_t my_pos[16], my_n[16], my_end[16];  // this thread's most recent units: first position, blocks,
+                                                // and this layer's piece count once the unit is fully issued
     uint32_t my_units = 0;                // units of this layer taken by this thread
-    uint32_t piece = pieces;  // forces a unit fetch
+    uint32_t piece = 0, pieces = 0;       // equal: forces a unit fetch
+    uint64_t unit_bytes = 0;
     const uint8_t* src_blk = nullptr;
     uint8_t* dst_blk = nullptr;
     const uint32_t first_piece = issued;  // this layer's pieces are [first_piece, issued)
     uint32_t reported = 0;                // units of this layer already reported as landed
     bool more = true;
 
-    // Issues the load of the next 16 KB piece, pulling a new 64 KB unit when the current one is used up.
+    // Issues the load of the next 16 KB piece, pulling a new unit when the current one is used up.
     auto issue_next = [&]() -> bool {
       if (piece == pieces) {
         const uint32_t unit = atomicAdd(ticket, 1u);
         if (unit >= p.copy_n) return false;
-        const uint32_t pos = p.copy_order[unit];
+        const uint32_t v = p.copy_order[unit];
+        const uint32_t pos = v & 0xFFFFFFu, n = (v >> 24) + 1u;
         const int32_t e = p.copy_src[pos];
         src_blk = src_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
         dst_blk = dst_slot + static_cast<uint64_t>(pos) * p.block_bytes;
+        unit_bytes = static_cast<uint64_t>(n) * p.block_bytes;
+        pieces = static_cast<uint32_t>((unit_bytes + kCopyChunk - 1) / kCopyChunk);
         my_pos[my_units % 16] = pos;
+        my_n[my_units % 16] = n;
+        my_end[my_units % 16] = issued - first_piece + pieces;
         ++my_units;
         piece = 0;
       }
       const uint64_t off = static_cast<uint64_t>(piece) * kCopyChunk;
-      const uint64_t left = p.block_bytes - off;
+      const uint64_t left = unit_bytes - off;
       const uint32_t bytes = left < kCopyChunk ? static_cast<uint32_t>(left) : kCopyChunk;
       const uint32_t stg = issued % kNC;
       sm.copy_dst[stg] = dst_blk + off;
@@ -1181,14 +1189,12 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     };
     // Reports the units all of whose pieces are among the first `complete` stored pieces of this layer.
     auto report_landed = [&](uint32_t complete) {
-      if (!ready) return;
-      const uint32_t units = complete / pieces;
-      if (units > reported) {
-        // The unit's bulk stores are complete (wait_group); they went through the asynchronous
-        // proxy, the flag goes through the generic one: order the two, then publish with a release.
-        ptx::fence_proxy_async_global();
-        for (; reported < units; ++reported) ptx::st_release_gpu(ready + my_pos[reported % 16], epoch);
-      }
+      if (!ready || reported == my_units || my_end[reported % 16] > complete) return;
+      // The units' bulk stores are complete (wait_group); they went through the asynchronous proxy,
+      // the flags go through the generic one: order the two, then publish with a release.
+      ptx::fence_proxy_async_global();
+      for (; reported < my_units && my_end[reported % 16] <= complete; ++reported)
+        for (uint32_t i = 0; i < my_n[reported % 16]; ++i) ptx::st_release_gpu(ready + my_pos[reported % 16] + i, epoch);
     };
 
     while (issued - done < loads_ahead && more) more = issue_next();

@@ -47,6 +47,7 @@ struct Plan {
   uint64_t version = 0;  // table version it was built from
   std::vector<int32_t> seqs;
   uint32_t nseq = 0, total_blocks = 0, k = 0;
+  uint32_t units = 0;                    // copy units of the fused gather (runs of neighbouring staged blocks)
   uint32_t per = 1, used_cta = 0;        // attention ranges: range c = [c*per, min((c+1)*per, total))
   uint32_t slots = 0, slots_static = 0;  // partial slots with / without work stealing
   uint64_t tokens = 0;
@@ -466,13 +467,31 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   // Order in which the fused kernel gathers the staged positions: the first staged block of every
   // CTA range, then the second of every range, ... A CTA reads its range front to back, so what it
   // needs first lands first and what lands last is needed last.
+  // Blocks smaller than 64 KB (fewer KV heads) are gathered several at a time where they are
+  // neighbours both in the lent arena and in the slot, which the slab allocator brings about
+  // (Section 4.2: transfers in large pieces): a unit is such a run within one CTA range, at most
+  // 64 KB and 8 blocks. With 64 KB blocks every unit is one block.
   {
+    const uint32_t max_n = s->lent_bs == s->block_bytes ? static_cast<uint32_t>(std::min<uint64_t>(8, std::max<uint64_t>(1, 65536 / s->block_bytes))) : 1u;
+    std::vector<uint32_t> unit_first, unit_len;
+    for (uint32_t j = 0; j < kk; ++j) {
+      const bool joins = j > 0 && unit_len.back() < max_n && pos_range[j] == pos_range[j - 1] &&
+                         ~copy_src[j] == ~copy_src[j - 1] + 1;
+      if (joins) {
+        ++unit_len.back();
+      } else {
+        unit_first.push_back(j);
+        unit_len.push_back(1);
+      }
+    }
+    p.units = static_cast<uint32_t>(unit_first.size());
     uint32_t max_rank = 0;
     for (uint32_t c = 0; c < p.used_cta; ++c) max_rank = std::max(max_rank, range_staged[c]);
     std::vector<uint32_t> start(max_rank + 1, 0);
-    for (uint32_t j = 0; j < kk; ++j) ++start[pos_rank[j] + 1];
+    for (uint32_t u = 0; u < p.units; ++u) ++start[pos_rank[unit_first[u]] + 1];
     for (uint32_t r = 0; r < max_rank; ++r) start[r + 1] += start[r];
-    for (uint32_t j = 0; j < kk; ++j) copy_order[start[pos_rank[j]]++] = j;  // positions ascend within a rank
+    for (uint32_t u = 0; u < p.units; ++u)  // positions ascend within a rank
+      copy_order[start[pos_rank[unit_first[u]]]++] = unit_first[u] | ((unit_len[u] - 1) << 24);
   }
   p.guarded = false;
   p.valid = true;
@@ -662,7 +681,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.lent_block_stride = s->lent_bs;
   d.copy_src = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
   d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order);
-  d.copy_n = p->k;
+  d.copy_n = p->units;
   d.ready = s->ready_dev;
   d.ready_stride = s->cfg.staging_blocks_per_slot;
   d.epoch_base = 0;
@@ -935,7 +954,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
     if (cfg->local_layer_stride || cfg->local_block_stride || cfg->lent_layer_stride || cfg->lent_block_stride)
       return SLICE_EINVAL;
   }
-  if (static_cast<uint64_t>(cfg->ring_slots) * group > 4096) return SLICE_EINVAL;
+  if (static_cast<uint64_t>(cfg->ring_slots) * group > 4096 || cfg->staging_blocks_per_slot >= (1u << 24)) return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;

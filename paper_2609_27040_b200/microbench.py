@@ -523,9 +523,94 @@ def link_bench(args):
                           "model": "time per layer = max(T0, m / B_link): the transfer is hidden while B*L >= m"}), flush=True)
 
 
+def layout_sweep(args):
+    """Section 4.2 / Figure "Throughput under Different Group and Slab Size", on this machine: the
+    one-launch pass over 16 layers of the Llama-3-8B-shaped batch with the slab allocator (slab sizes
+    1..100, and the block-granular free stack with a seeded order as the scattered extreme), layer
+    groups of 1 and 4, the layer-major and layer-group-major orders, 8 / 2 / 1 KV heads (64 / 16 /
+    8 KB blocks), the lent arena in HBM and behind PCIe (pinned host memory). Blocks are allocated
+    either request by request (a prompt's blocks at once) or interleaved over the requests (growth
+    during decoding). Reports time per layer, the algorithmic rate and the mean length of the runs
+    the fused gather could copy as one unit (neighbours in the arena and in the slot, <= 64 KB)."""
+    import dataclasses
+    import torch
+    from paper_2609_27040_b200 import binding as B, synth
+    Lr = 16      # more layers than the ring has layer slots (2 groups of up to 4), so every layer is fetched in every pass
+    for link in args.links:
+        for hkv in args.kv_heads:
+            base = dataclasses.replace(synth.WORKLOADS["llama3_8b_decode"], num_layers=Lr, num_kv_heads=hkv,
+                                       num_q_heads=4 * hkv, lent_fraction=0.4 if link == "hbm" else 0.02)
+            bb = base.block_bytes
+            for order in ("per_request", "interleaved"):
+                for slab, group, layout in [(0, 1, 0), (1, 1, 0), (10, 1, 0), (10, 4, 0), (10, 4, 2), (10, 4, 1), (100, 4, 2), (100, 1, 0)]:
+                    pl = synth.make_placement(base, args.seed, slack_blocks=64, permute=slab == 0)
+                    nl, nr = pl.local_blocks, pl.lent_blocks
+                    if slab:
+                        nl, nr = -(-nl // slab) * slab, -(-nr // slab) * slab
+                    shape = (2, 16, hkv, 128)
+                    local = torch.empty((Lr, nl) + shape, device="cuda", dtype=torch.bfloat16).normal_()
+                    if link == "hbm":
+                        lent = torch.empty((Lr, nr) + shape, device="cuda", dtype=torch.bfloat16).normal_()
+                    else:
+                        lent = torch.empty((Lr, nr) + shape, dtype=torch.bfloat16).normal_().pin_memory()
+                    staging = torch.zeros((2 * group, max(pl.staging_blocks, 1)) + shape, device="cuda", dtype=torch.bfloat16)
+                    q = torch.empty((Lr, base.batch, base.num_q_heads, 128), device="cuda", dtype=torch.bfloat16).normal_()
+                    out = torch.zeros_like(q)
+                    s = B.Slice(Lr, hkv, nl, nr, pl.staging_blocks, local=local, lent=lent, staging=staging, max_seqs=base.batch,
+                                max_blocks_per_seq=300, lent_kind=int(link != "hbm"), slab_blocks=slab, layer_group=group,
+                                layout=layout, local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
+                    if order == "per_request":
+                        for i, hints in enumerate(pl.hints):
+                            for h in hints:
+                                assert s.slice_alloc_blocks(i, 1, int(h))[0] == 0
+                    else:
+                        for b in range(max(len(h) for h in pl.hints)):
+                            for i, hints in enumerate(pl.hints):
+                                if b < len(hints):
+                                    assert s.slice_alloc_blocks(i, 1, int(hints[b]))[0] == 0
+                    for i in range(base.batch):
+                        assert s.slice_set_seq_len(i, int(pl.lengths[i])) == 0
+                    # runs of lent blocks that are neighbours by id and in the staging order
+                    ids = [~int(e) for i in range(base.batch) for e in s.slice_get_block_table(i)[1] if e < 0]
+                    runs, cap = [], max(1, min(8, 65536 // bb))
+                    for a, b2 in zip([None] + ids[:-1], ids):
+                        if a is not None and b2 == a + 1 and runs[-1] < cap:
+                            runs[-1] += 1
+                        else:
+                            runs.append(1)
+                    seqs = np.arange(base.batch, dtype=np.int32)
+                    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+                    scale = 1.0 / float(np.sqrt(128))
+                    for _ in range(3):
+                        assert s.slice_decode_step(seqs, q, base.num_q_heads, scale, out, False, True, main, side) == 0
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    reps = 10
+                    fetched0 = s.slice_stats()["prefetched_bytes"]
+                    e0.record(main)
+                    for _ in range(reps):
+                        assert s.slice_decode_step(seqs, q, base.num_q_heads, scale, out, False, True, main, side) == 0
+                    e1.record(main)
+                    e1.synchronize()
+                    us = e0.elapsed_time(e1) * 1e3 / reps / Lr
+                    tokens = int(pl.lengths.sum())
+                    fetched = (s.slice_stats()["prefetched_bytes"] - fetched0) / reps / Lr      # gathered per layer, as counted by the library
+                    algo = tokens * base.kv_bytes_per_token + 2 * fetched
+                    print(json.dumps({"case": "layouts", "link": link, "kv_heads": hkv, "block_kb": bb // 1024, "alloc": order,
+                                      "slab": slab or "stack, seeded order", "group": group,
+                                      "layout": ["layer-major", "slab-major", "layer-group-major"][layout],
+                                      "us_per_layer": round(us, 1), "algorithmic_gbs": round(algo / us / 1e3, 1),
+                                      "lent_mb_per_layer": round(pl.staging_blocks * bb / 1e6, 1), "gathered_mb_per_layer": round(fetched / 1e6, 1),
+                                      "mean_blocks_per_copy_unit": round(float(np.mean(runs)), 2) if runs else None,
+                                      "device_status": s.slice_stats()["device_status"]}), flush=True)
+                    s.slice_destroy()
+                    del local, lent, staging, q, out
+                    torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "size", "multislice", "all"], default="all")
+    ap.add_argument("--what", choices=["copy", "reclaim", "growth", "link", "size", "multislice", "layouts", "all"], default="all")
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--arena-gb", type=float, default=48.0)
     ap.add_argument("--seed", type=int, default=0)
@@ -539,6 +624,8 @@ def main():
     ap.add_argument("--rate", type=float, default=0.5, help="multislice: mean arrivals per step (Poisson)")
     ap.add_argument("--policy", choices=["gll", "random", "round_robin"], default="gll")
     ap.add_argument("--cap-window", type=int, default=0, help="steps a cap holds after a preemption by reclamation")
+    ap.add_argument("--links", nargs="*", default=["hbm", "host"], help="layouts: where the lent arena lives")
+    ap.add_argument("--kv-heads", type=int, nargs="*", default=[8, 2, 1], help="layouts: KV heads (block = 8 KB per head)")
     args = ap.parse_args()
     from paper_2609_27040_b200 import binding as B
     B.lib()                                    # fails loudly when the CUDA library is missing
@@ -554,6 +641,8 @@ def main():
         transfer_size_sweep(args)
     if args.what == "multislice":
         multislice_bench(args)
+    if args.what == "layouts":
+        layout_sweep(args)
 
 
 if __name__ == "__main__":

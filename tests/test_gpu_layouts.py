@@ -145,3 +145,32 @@ def test_append_and_reclaim_move_the_right_bytes_in_every_layout(layout, slab, g
     for layer in range(sc.L):
         _, _, ref, _ = _oracle_layer(sc, layer)
         assert attention_close(got[layer], ref, ATOL, RTOL)[0], layer
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 1), (8, 2), (2, 2)])
+@pytest.mark.parametrize("layout,slab,group", [(0, 10, 1), (2, 10, 4), (0, 0, 1)])
+def test_small_blocks_are_gathered_in_runs(hq, hkv, layout, slab, group):
+    """With 1 or 2 KV heads a block is 8 or 16 KB; where the slab allocator has kept a sequence's lent
+    blocks together, the fused gather moves up to 64 KB of neighbouring blocks per copy unit. The
+    staged bytes and the attention must not depend on how the units were cut (slab 0: seeded free
+    order, hardly any neighbours; slabs: long runs)."""
+    from tests.gpu_helpers import kv_to_host
+    sc, g = _make(layout, slab, group, layers=8, hq=hq, hkv=hkv, decode_ctas=10)
+    seqs = np.asarray(sc.seq_ids, np.int32)
+    for rep in range(2):
+        g.out.zero_()
+        assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
+        torch.cuda.synchronize()
+        g.device_ok()
+        got = _f64(g.out)
+        for layer in range(sc.L):
+            _, _, ref, _ = _oracle_layer(sc, layer)
+            ok, max_abs, _ = attention_close(got[layer], ref, ATOL, RTOL)
+            assert ok, (rep, layer, max_abs)
+    LS = sc.wl.ring_slots
+    holder = {}
+    for l in list(range(sc.L)) + list(range(min(max(group, 1), sc.L))):
+        holder[l % LS] = l
+    for slot, layer in holder.items():
+        rc, _, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
+        assert (kv_to_host(g.staging[slot, :k]) == sc.staging[slot, :k]).all(), (slot, layer)
