@@ -160,6 +160,18 @@ typedef struct {
                                      2 layer-group-major [group][slab][layer in group][block in slab].
                                      1 and 2 need S > 0, N a multiple of S for both arenas, L a
                                      multiple of k, and zero strides                               */
+  uint32_t split_layer;           /* Section 4.1, the paper's own placement (expansion ratio 2 when it is
+                                     half the layers): 0 = off, blocks are placed local or lent one
+                                     by one; s in 1..L-1 = every block keeps layers 0..s-1 in the
+                                     local arena and layers s..L-1 in the lent arena, under the same
+                                     block id. The local arena then holds s layers, the lent arena
+                                     L - s (its first layer is layer s) with at least local_blocks
+                                     ids, ids come from the local list only (hint LENT is EINVAL),
+                                     layers below s are attended to in place, layers from s on are
+                                     prefetched whole (every block of the batch, staging position =
+                                     position of the block in the batch), and slice_reclaim does not
+                                     apply (EINVAL): the lender regains memory by preemption. Needs
+                                     layout 0                                                       */
 } slice_config_t;
 
 typedef struct {

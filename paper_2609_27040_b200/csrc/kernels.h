@@ -82,6 +82,9 @@ struct LayerParams {
   uint64_t local_block_stride;
   uint32_t layer_group;         // layers per group of the arenas' layout (>= 1)
   uint32_t prefetch_distance;   // the gather issued during launch layer i fetches layer i + prefetch_distance
+  uint32_t split_layer;         // layer-split placement: from this layer on EVERY block of the batch is read from
+                                //   the ring slot, at the position equal to its flat index (0xFFFFFFFF: no split;
+                                //   then the resolved table says where each block is)
   const uint8_t* staging_base;  // ring: layer l is staged in slot l % ring_slots
   uint64_t slot_bytes;
   uint32_t ring_slots;
@@ -172,6 +175,8 @@ struct AppendParams {
   uint64_t lent_block_stride;
   uint32_t layer_group;
   uint64_t local_group_stride, lent_group_stride;
+  uint32_t split_layer;        // layers from here on have their home in the lent arena, at the id the entry names
+                               //   (0xFFFFFFFF: no split; the entry's sign names the arena)
   uint8_t* slot_base;          // one layer: ring slot holding the layer, or NULL when not staged
   // several layers in one launch (grid.y = layer): strides to the next layer, and which layers are staged
   uint32_t num_layers, first_layer, ring_slots;

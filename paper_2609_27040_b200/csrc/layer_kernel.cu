@@ -269,6 +269,8 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     const bool check_ready = li >= p.prefetch_distance && p.gather_target[li - p.prefetch_distance] == static_cast<int16_t>(layer);
     const uint32_t* ready = p.ready + static_cast<size_t>(layer % p.ring_slots) * p.ready_stride;
     const uint32_t epoch = p.epoch_base + li;
+    // Layer-split placement: this layer's blocks all come from the ring slot, in flat order.
+    const bool all_staged = layer >= p.split_layer;
     uint64_t waited_ns = 0;
     if (p.trace && lane == 0) {
       p.trace[li * p.trace_stride + kTraceWords * blockIdx.x] = ptx::global_timer_ns();
@@ -408,9 +410,9 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     // Entries of n own blocks from flat block b on and, when they come from the shared-memory copy
     // (no load to wait for), their ready flags as well.
     auto prefetch_own = [&](uint32_t b, uint32_t n, int32_t& my, uint32_t& rdy, bool& have) {
-      have = b + n - r0 <= ncache;
+      have = all_staged || b + n - r0 <= ncache;
       my = 0;
-      if (lane < n) my = have ? sm.own_res[b + lane - r0] : p.resolved[b + lane];
+      if (lane < n) my = all_staged ? ~static_cast<int32_t>(b + lane) : have ? sm.own_res[b + lane - r0] : p.resolved[b + lane];
       rdy = epoch;
       if (have && check_ready && lane < n && my < 0) rdy = ptx::ld_acquire_gpu(ready + static_cast<uint32_t>(~my));
     };
@@ -490,7 +492,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     if (ok && p.allow_steal) {
       Claim c = steal();
       while (c.b < c.e && ok) {
-        const int32_t my = lane < c.e - c.b ? p.resolved[c.b + lane] : 0;
+        const int32_t my = lane >= c.e - c.b ? 0 : all_staged ? ~static_cast<int32_t>(c.b + lane) : p.resolved[c.b + lane];
         const uint32_t hint = p.blk_seq[c.b];
         const Claim nxt = steal();
         stream_claim(c, my, 0, false, hint);
@@ -1273,10 +1275,12 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   const int32_t e = p.home_entry[i];
   const uint32_t y = blockIdx.y;  // layer within the launch
   const uint32_t layer = p.first_layer + y;
-  uint8_t* home = e >= 0 ? p.local_base + layer_offset(layer, p.layer_group, p.local_group_stride, p.local_layer_stride) +
-                               static_cast<uint64_t>(e) * p.local_block_stride
+  const bool lent_home = p.split_layer == 0xFFFFFFFFu ? e < 0 : layer >= p.split_layer;
+  const uint32_t id = e >= 0 ? static_cast<uint32_t>(e) : static_cast<uint32_t>(~e);
+  uint8_t* home = !lent_home ? p.local_base + layer_offset(layer, p.layer_group, p.local_group_stride, p.local_layer_stride) +
+                               static_cast<uint64_t>(id) * p.local_block_stride
                          : p.lent_base + layer_offset(layer, p.layer_group, p.lent_group_stride, p.lent_layer_stride) +
-                               static_cast<uint64_t>(~e) * p.lent_block_stride;
+                               static_cast<uint64_t>(id) * p.lent_block_stride;
   const int32_t sp = p.stage_pos[i];
   uint8_t* slot = p.slot_base;
   if (p.num_layers > 1)

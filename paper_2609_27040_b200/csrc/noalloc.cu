@@ -81,6 +81,7 @@ cudaError_t static_scratch_setup(uint32_t Hkv, uint32_t G, uint32_t ncta) {
   p.ring_slots = 1;
   p.layer_group = 1;
   p.prefetch_distance = 1;
+  p.split_layer = 0xFFFFFFFFu;
   p.per = 1;
   p.merge_inline = 1;
   p.part_buffers = 1;

@@ -97,6 +97,9 @@ struct ema_slice {
   uint64_t local_gs = 0, lent_gs = 0;
   uint32_t local_W = 0, lent_W = 0;
   uint32_t layer_slots = 1;  // ring slots in layers: ring_slots groups of `group` layers
+  // Layer-split placement (Section 4.1): layers [0, split) of every block live in the local arena,
+  // layers [split, L) in the lent arena under the same block id; 0 = blocks are split instead.
+  uint32_t split = 0;
   std::vector<uint32_t> slab_used_local, slab_used_lent;  // blocks in use per slab (slab allocator)
   int device = -1;  // the CUDA device the slice was created on
   int num_sms = 148;
@@ -189,7 +192,11 @@ inline uint32_t blocks_for(uint32_t len) { return (len + kBlockTokens - 1) / kBl
 inline bool multi_stream(const ema_slice* s) { return s->streams.size() > 1; }
 
 inline uint64_t local_off(const ema_slice* s, uint32_t l) { return ema::layer_offset(l, s->group, s->local_gs, s->local_ls); }
-inline uint64_t lent_off(const ema_slice* s, uint32_t l) { return ema::layer_offset(l, s->group, s->lent_gs, s->lent_ls); }
+// With the layer split the lent arena holds layers split .. L-1 only (layer-major, so the offset is linear).
+inline uint64_t lent_off(const ema_slice* s, uint32_t l) { return ema::layer_offset(l - s->split, s->group, s->lent_gs, s->lent_ls); }
+
+// Does `layer` read from its ring slot for this batch?
+inline bool needs_staging(const ema_slice* s, uint32_t layer, uint32_t k) { return k > 0 && (!s->split || layer >= s->split); }
 
 // Table entry -> what the kernels index with: the block's physical index inside a layer of its
 // arena (the id itself in the layer-major order), lent entries staying negative (~index).
@@ -349,6 +356,7 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
     for (uint32_t b = 0; b < nb; ++b)
       if (q.table[b] < 0) ++k;
   }
+  if (s->split) k = total_blocks;  // layer split: the layers of the lent half stage every block
   if (k > s->cfg.staging_blocks_per_slot) return SLICE_ESTAGING;
 
   // Plans of older table versions can never be used again: guard their buffers now.
@@ -442,7 +450,14 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
       const int32_t e = q.table[b];
       int32_t r = phys_entry(s, e);
       p.resolved_ids[flat] = e;
-      if (e < 0) {
+      if (s->split) {
+        // Layer split: the resolved table serves the local half; for the lent half the kernel reads
+        // block `flat` at staging position `flat`, and the gather brings it there from the same id.
+        copy_src[kk] = ~e;
+        pos_range[kk] = flat / per;
+        pos_rank[kk] = range_staged[flat / per]++;
+        ++kk;
+      } else if (e < 0) {
         copy_src[kk] = r;  // negative entry: tier 1 (lent arena), physical index ~r
         r = ~static_cast<int32_t>(kk);
         p.resolved_ids[flat] = r;
@@ -454,7 +469,7 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
       blk_seq[flat] = i;
       if (b == last_b) {
         home[i] = phys_entry(s, e);
-        stage_pos[i] = e < 0 ? ~r : -1;
+        stage_pos[i] = s->split ? static_cast<int32_t>(flat) : e < 0 ? ~r : -1;
       }
       ++flat;
     }
@@ -577,6 +592,7 @@ int note_slot_written(ema_slice* s, SlotState& sl, uint32_t layer, const Plan* p
 
 // Stand-alone gather of one layer (the copy kernel), used by prefetch_layer and to prime the ring.
 int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
+  if (s->split && layer < s->split) return SLICE_OK;  // a layer of the local half: read in place, nothing to fetch
   int rc = ensure_stream(s, side);
   if (rc) return rc;
   rc = plan_on_stream(s, p, side);
@@ -631,6 +647,7 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.local_block_stride = s->local_bs;
   d.layer_group = s->group;
   d.prefetch_distance = s->group;
+  d.split_layer = s->split ? s->split : 0xFFFFFFFFu;
   d.staging_base = static_cast<const uint8_t*>(s->cfg.staging_base);
   d.slot_bytes = s->slot_bytes;
   d.ring_slots = s->layer_slots;
@@ -675,7 +692,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.Hkv = Hkv;
   d.G = Hq / Hkv;
   d.scale_log2 = sm_scale * 1.4426950408889634f;
-  d.lent_base = static_cast<const uint8_t*>(s->cfg.lent_base);
+  // (with the layer split the lent arena starts at layer `split`: the kernel indexes it by layer)
+  d.lent_base = static_cast<const uint8_t*>(s->cfg.lent_base) - ema::layer_offset(s->split, s->group, s->lent_gs, s->lent_ls);
   d.lent_group_stride = s->lent_gs;
   d.lent_layer_stride = s->lent_ls;
   d.lent_block_stride = s->lent_bs;
@@ -712,8 +730,8 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   }
   const uint32_t slot = layer % R;
   SlotState& sl = s->slots[slot];
-  if (p->k && !staged(s, layer, p)) return SLICE_ESTALE;
-  const bool gather = next_layer >= 0 && p->k > 0;
+  if (needs_staging(s, layer, p->k) && !staged(s, layer, p)) return SLICE_ESTALE;
+  const bool gather = next_layer >= 0 && needs_staging(s, static_cast<uint32_t>(next_layer), p->k);
   if (next_layer >= 0 && static_cast<uint32_t>(next_layer) % R == slot) return SLICE_EINVAL;
   int rc = ensure_stream(s, stream);
   if (rc) return rc;
@@ -725,7 +743,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   if (rc) return rc;
   SlotState* nsl = next_layer >= 0 ? &s->slots[static_cast<uint32_t>(next_layer) % R] : nullptr;
   if (!s->null_dev) {
-    if (p->k && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+    if (needs_staging(s, layer, p->k) && sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
     if (gather) {
       rc = order_before_slot_write(s, *nsl, stream);
       if (rc) return rc;
@@ -762,7 +780,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   }
   s->st.decode_calls++;
   s->st.decode_tokens += p->tokens;
-  if (next_layer >= 0) return note_slot_written(s, *nsl, static_cast<uint32_t>(next_layer), p, stream);
+  if (gather) return note_slot_written(s, *nsl, static_cast<uint32_t>(next_layer), p, stream);
   return SLICE_OK;
 }
 
@@ -778,8 +796,8 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     if (lens[i] == 0) return SLICE_EINVAL;
   // The first layer group is staged before the launch; inside it, the gather issued during layer l
   // fetches layer l + K (the same layer of the next group).
-  for (uint32_t l = 0; p->k && l < std::min(K, L); ++l)
-    if (!staged(s, l, p)) return SLICE_ESTALE;
+  for (uint32_t l = 0; l < std::min(K, L); ++l)
+    if (needs_staging(s, l, p->k) && !staged(s, l, p)) return SLICE_ESTALE;
   // Plan the gathers by following what each ring slot will hold.
   std::vector<int64_t> holds(R, -1);
   for (uint32_t r = 0; r < R; ++r)
@@ -798,6 +816,7 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
       for (uint32_t j = l; j < L; ++j)
         if (j % R == t % R) t = -1;
     }
+    if (t >= 0 && !needs_staging(s, static_cast<uint32_t>(t), p->k)) t = -1;  // a layer of the local half
     if (t < 0 || holds[t % R] == t) continue;  // nothing to fetch, or the slot still holds that layer
     target[l] = static_cast<int16_t>(t);
     for (int64_t j = static_cast<int64_t>(l) - 1; j >= 0; --j)
@@ -955,6 +974,10 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
       return SLICE_EINVAL;
   }
   if (static_cast<uint64_t>(cfg->ring_slots) * group > 4096 || cfg->staging_blocks_per_slot >= (1u << 24)) return SLICE_EINVAL;
+  // Layer split: the same ids in both arenas, plain layer-major order, no block-level lending.
+  if (cfg->split_layer && (cfg->split_layer >= cfg->num_layers || cfg->layout != 0 || cfg->lent_blocks_physical < cfg->local_blocks ||
+                           cfg->lent_layer_stride || cfg->lent_block_stride))
+    return SLICE_EINVAL;
   if (!null_dev && (!cfg->local_base || !cfg->staging_base || (cfg->lent_blocks_physical && !cfg->lent_base)))
     return SLICE_EINVAL;
   const uint64_t bb = 2ull * kBlockTokens * cfg->num_kv_heads * kHeadDim * 2;
@@ -995,6 +1018,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   s->lent_ls = cfg->lent_layer_stride ? cfg->lent_layer_stride : bb * cfg->lent_blocks_physical;
   s->slot_bytes = bb * cfg->staging_blocks_per_slot;
   s->group = group;
+  s->split = cfg->split_layer;
   s->slab = slab;
   s->layout = cfg->layout;
   s->layer_slots = cfg->ring_slots * group;
@@ -1129,6 +1153,10 @@ int slice_destroy(slice_t* s) {
 
 int slice_alloc_blocks(slice_t* s, int32_t seq, uint32_t n, int32_t hint, int32_t* out_entries) {
   if (!s || seq < 0 || hint < SLICE_TIER_AUTO || hint > SLICE_TIER_LENT) return SLICE_EINVAL;
+  if (s->split) {  // layer split: an id names a block's place in both arenas; ids come from the local list only
+    if (hint == SLICE_TIER_LENT) return SLICE_EINVAL;
+    hint = SLICE_TIER_LOCAL;
+  }
   auto it = s->seqs.find(seq);
   const bool exists = it != s->seqs.end();
   if (!exists && s->seqs.size() >= s->cfg.max_seqs) return SLICE_EINVAL;
@@ -1242,6 +1270,9 @@ int paged_decode_noalloc(slice_t* s, uint32_t layer, const int32_t* seqs, uint32
 
 int slice_reclaim(slice_t* s, uint32_t take, uint64_t* out_n_migrated, void* stream_v) {
   if (!s) return SLICE_EINVAL;
+  // With the layer split a request's layers sit half here, half there: nothing can migrate; the
+  // lender gets memory back by preemption (slice_preempt_seq), as in Section 4.1.
+  if (s->split) return SLICE_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   if (take > s->lent_cap) take = s->lent_cap;
   const uint32_t cut = s->lent_cap - take;
@@ -1571,15 +1602,16 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   bool one_staged = false;
   for (uint32_t l = first; l < first + count; ++l) {
     SlotState& sl = s->slots[l % s->layer_slots];
-    if (!staged(s, l, p)) continue;
+    if (!needs_staging(s, l, p->k) || !staged(s, l, p)) continue;
     if (sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
     a.staged_mask[(l - first) >> 5] |= 1u << ((l - first) & 31u);
     one_staged = true;
   }
   a.local_base = static_cast<uint8_t*>(s->cfg.local_base);
   a.local_block_stride = s->local_bs;
-  a.lent_base = static_cast<uint8_t*>(s->cfg.lent_base);
+  a.lent_base = static_cast<uint8_t*>(s->cfg.lent_base) - ema::layer_offset(s->split, s->group, s->lent_gs, s->lent_ls);
   a.lent_block_stride = s->lent_bs;
+  a.split_layer = s->split ? s->split : 0xFFFFFFFFu;
   a.layer_group = s->group;
   a.local_group_stride = s->local_gs;
   a.lent_group_stride = s->lent_gs;
@@ -1617,6 +1649,7 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   if (rc) return rc;
   const uint32_t slot = layer % s->layer_slots;
   SlotState& sl = s->slots[slot];
+  if (s->split && layer < s->split) return SLICE_EINVAL;  // a layer of the local half is never staged
   if (!staged(s, layer, p)) return SLICE_ESTALE;
   if (s->null_dev || p->k == 0) return SLICE_OK;
   rc = ensure_stream(s, stream);
@@ -1784,8 +1817,8 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   }
   if (!s->null_dev)  // the work counters of all layers, cleared once per pass
     CU(s, cudaMemsetAsync(s->cnt_dev, 0, static_cast<size_t>(L) * s->cnt_stride * sizeof(uint32_t), stream));
-  for (uint32_t l = 0; p->k && l < std::min(K, L); ++l) {  // the first layer group
-    if (staged(s, l, p)) continue;
+  for (uint32_t l = 0; l < std::min(K, L); ++l) {  // the first layer group
+    if (!needs_staging(s, l, p->k) || staged(s, l, p)) continue;
     rc = do_prefetch(s, l, p, side);
     if (rc) return rc;
   }
@@ -1813,7 +1846,7 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
         for (uint32_t j = l; j < L; ++j)
           if (j % R == static_cast<uint32_t>(next) % R) next = -1;  // its slot still serves this pass
       }
-      if (next >= 0 && staged(s, static_cast<uint32_t>(next), p)) next = -1;
+      if (next >= 0 && (!needs_staging(s, static_cast<uint32_t>(next), p->k) || staged(s, static_cast<uint32_t>(next), p))) next = -1;
     }
     if (fused) {
       rc = do_layer(s, l, p, qd + l * per_layer, Hq, sm_scale, od + l * per_layer, nullptr, stream, next, false, true);
@@ -1834,10 +1867,10 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
       }
     }
   }
-  for (uint32_t l = 0; p->k && wrap && L > 1 && l < std::min(K, L); ++l) {
+  for (uint32_t l = 0; wrap && L > 1 && l < std::min(K, L); ++l) {
     // Layers of the next pass's first group whose ring slot served a layer of this pass to the end:
     // refilled only after that attention.
-    if (staged(s, l, p)) continue;
+    if (!needs_staging(s, l, p->k) || staged(s, l, p)) continue;
     rc = do_prefetch(s, l, p, side);
     if (rc) return rc;
   }

@@ -452,6 +452,59 @@ def multislice_bench(args):
         sl.slice_destroy()
 
 
+def link_point(f: float, seed: int = 0, layers: int = 8, reps: int = 10) -> dict:
+    """One point of the link measurement: the Llama-3-8B-shaped batch on `layers` layers with a
+    fraction f of every sequence's blocks in a lent arena in pinned host memory (lent_kind = 1, the
+    prefetch crosses PCIe). Returns the lent bytes per layer, the time per layer of the one-launch
+    pass and the link rate measured with the stand-alone gather from the same arena."""
+    import dataclasses
+    import torch
+    from paper_2609_27040_b200 import binding as B, synth
+    Lr = layers
+    wl = dataclasses.replace(synth.WORKLOADS["llama3_8b_decode"], num_layers=Lr, lent_fraction=f)
+    pl = synth.make_placement(wl, seed, slack_blocks=64)
+    shape = (2, 16, wl.num_kv_heads, 128)
+    local = torch.empty((Lr, pl.local_blocks) + shape, device="cuda", dtype=torch.bfloat16).normal_()
+    lent = torch.empty((Lr, max(pl.lent_blocks, 1)) + shape, dtype=torch.bfloat16).normal_().pin_memory()
+    staging = torch.zeros((2, max(pl.staging_blocks, 1)) + shape, device="cuda", dtype=torch.bfloat16)
+    q = torch.empty((Lr, wl.batch, wl.num_q_heads, 128), device="cuda", dtype=torch.bfloat16).normal_()
+    out = torch.zeros_like(q)
+    s = B.Slice(Lr, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks, local=local, lent=lent,
+                staging=staging, max_seqs=wl.batch, max_blocks_per_seq=300, lent_kind=1,
+                local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
+    for i, hints in enumerate(pl.hints):
+        for h in hints:
+            assert s.slice_alloc_blocks(i, 1, int(h))[0] == 0
+        assert s.slice_set_seq_len(i, int(pl.lengths[i])) == 0
+    seqs = np.arange(wl.batch, dtype=np.int32)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    scale = 1.0 / float(np.sqrt(128))
+    m = pl.staging_blocks * BLOCK_BYTES
+    link_gbs = None
+    if m:
+        def gather():
+            assert s.prefetch_layer(3, seqs, main) == 0
+            assert s.prefetch_layer(5, seqs, main) == 0      # same slot, other layer: always a real copy
+        us = _time_us(gather, main, 5) / 2
+        link_gbs = m / us / 1e3
+    for _ in range(3):
+        assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(main)
+    for _ in range(reps):
+        assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
+    e1.record(main)
+    e1.synchronize()
+    row = {"f": f, "lent_bytes_per_layer": m, "us_per_layer": e0.elapsed_time(e1) * 1e3 / reps / Lr,
+           "link_gbs": link_gbs, "device_status": s.slice_stats()["device_status"],
+           "kv_bytes_per_layer": int(pl.lengths.sum()) * wl.kv_bytes_per_token}
+    s.slice_destroy()
+    del local, lent, staging
+    torch.cuda.empty_cache()
+    return row
+
+
 def link_bench(args):
     """The paper's transparency condition (Section 2.3 / 4: a transfer of m bytes over a link of
     bandwidth B is hidden when it fits in the latency window L between two uses, B*L >= m) with a
@@ -459,52 +512,8 @@ def link_bench(args):
     prefetch crosses PCIe. For a sweep of lent fractions f: measured time per layer of the one-launch
     pass against the model max(T0, m/B), T0 = time per layer with nothing lent, m = lent bytes per
     layer, B = link rate measured with the stand-alone gather from the same arena."""
-    import dataclasses
-    import torch
-    from paper_2609_27040_b200 import binding as B, capacity, synth
-    Lr = 8
-    rows = []
-    for f in args.fractions:
-        wl = dataclasses.replace(synth.WORKLOADS["llama3_8b_decode"], num_layers=Lr, lent_fraction=f)
-        pl = synth.make_placement(wl, args.seed, slack_blocks=64)
-        shape = (2, 16, wl.num_kv_heads, 128)
-        local = torch.empty((Lr, pl.local_blocks) + shape, device="cuda", dtype=torch.bfloat16).normal_()
-        lent = torch.empty((Lr, max(pl.lent_blocks, 1)) + shape, dtype=torch.bfloat16).normal_().pin_memory()
-        staging = torch.zeros((2, max(pl.staging_blocks, 1)) + shape, device="cuda", dtype=torch.bfloat16)
-        q = torch.empty((Lr, wl.batch, wl.num_q_heads, 128), device="cuda", dtype=torch.bfloat16).normal_()
-        out = torch.zeros_like(q)
-        s = B.Slice(Lr, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks, local=local, lent=lent,
-                    staging=staging, max_seqs=wl.batch, max_blocks_per_seq=300, lent_kind=1,
-                    local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order)
-        for i, hints in enumerate(pl.hints):
-            for h in hints:
-                assert s.slice_alloc_blocks(i, 1, int(h))[0] == 0
-            assert s.slice_set_seq_len(i, int(pl.lengths[i])) == 0
-        seqs = np.arange(wl.batch, dtype=np.int32)
-        main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
-        scale = 1.0 / float(np.sqrt(128))
-        m = pl.staging_blocks * BLOCK_BYTES
-        link_gbs = None
-        if m:
-            def gather():
-                assert s.prefetch_layer(3, seqs, main) == 0
-                assert s.prefetch_layer(5, seqs, main) == 0      # same slot, other layer: always a real copy
-            us = _time_us(gather, main, 5) / 2
-            link_gbs = m / us / 1e3
-        for _ in range(3):
-            assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 10
-        e0.record(main)
-        for _ in range(reps):
-            assert s.slice_decode_step(seqs, q, wl.num_q_heads, scale, out, False, True, main, side) == 0
-        e1.record(main)
-        e1.synchronize()
-        rows.append({"f": f, "lent_bytes_per_layer": m, "us_per_layer": e0.elapsed_time(e1) * 1e3 / reps / Lr,
-                     "link_gbs": link_gbs, "device_status": s.slice_stats()["device_status"]})
-        s.slice_destroy()
-        del local, lent, staging
+    from paper_2609_27040_b200 import capacity
+    rows = [link_point(f, args.seed) for f in args.fractions]
     t0 = min(r["us_per_layer"] for r in rows if r["lent_bytes_per_layer"] == 0) if any(r["lent_bytes_per_layer"] == 0 for r in rows) else None
     rates = [r["link_gbs"] for r in rows if r["link_gbs"]]
     link = max(rates) if rates else None
