@@ -172,6 +172,18 @@ typedef struct {
                                      position of the block in the batch), and slice_reclaim does not
                                      apply (EINVAL): the lender regains memory by preemption. Needs
                                      layout 0                                                       */
+  uint32_t swap_out;              /* Section 2.3 (layers are swapped in AND out, cyclically; what comes in
+                                     must be matched by what goes out): 0 = the ring holds read-only
+                                     copies and slice_append_kv writes a new row to the home block and
+                                     to the staged copy; 1 = write-back: slice_append_kv writes a row
+                                     whose block is staged to the staged copy only, and every pass of
+                                     slice_decode_step writes each staged layer back to the lent
+                                     arena (all its staged blocks), on a stream of the library's own,
+                                     while that layer is attended to and the next transfer comes in;
+                                     a slot is refilled only after its write-back. Passes then run one
+                                     launch per layer. After an append, run a pass (or
+                                     slice_writeback_layer for the staged layers) before the tables
+                                     change again, or the appended rows of staged blocks are lost   */
 } slice_config_t;
 
 typedef struct {

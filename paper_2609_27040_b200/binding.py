@@ -51,7 +51,7 @@ class SliceConfig(C.Structure):
         ("pipeline_mode", C.c_uint32), ("static_split", C.c_uint32), ("claim_blocks", C.c_uint32),
         ("steal_floor", C.c_uint32), ("prefetch_priority", C.c_uint32),
         ("slab_blocks", C.c_uint32), ("layer_group", C.c_uint32), ("layout", C.c_uint32),
-        ("split_layer", C.c_uint32),
+        ("split_layer", C.c_uint32), ("swap_out", C.c_uint32),
     ]
 
 
@@ -192,7 +192,7 @@ class Slice:
                  lent_kind: int = 0, flags: int = 0, local_free_order=None, lent_free_order=None,
                  decode_ctas: int = 0, copy_ctas: int = 0, copy_kind: int = 0, pipeline_mode: int = 0,
                  static_split: int = 0, claim_blocks: int = 0, steal_floor: int = 0, prefetch_priority: int = 0,
-                 slab_blocks: int = 0, layer_group: int = 0, layout: int = 0, split_layer: int = 0,
+                 slab_blocks: int = 0, layer_group: int = 0, layout: int = 0, split_layer: int = 0, swap_out: int = 0,
                  local_layer_stride: int = 0, local_block_stride: int = 0,
                  lent_layer_stride: int = 0, lent_block_stride: int = 0):
         cfg = SliceConfig()
@@ -213,7 +213,7 @@ class Slice:
         cfg.pipeline_mode, cfg.static_split = pipeline_mode, static_split
         cfg.claim_blocks, cfg.steal_floor, cfg.prefetch_priority = claim_blocks, steal_floor, prefetch_priority
         cfg.slab_blocks, cfg.layer_group, cfg.layout = slab_blocks, layer_group, layout
-        cfg.split_layer = split_layer
+        cfg.split_layer, cfg.swap_out = split_layer, swap_out
         self.cfg = cfg
         self._keep = (local, lent, staging)       # arenas must outlive the slice
         h = C.c_void_p()

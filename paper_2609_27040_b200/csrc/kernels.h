@@ -175,6 +175,7 @@ struct AppendParams {
   uint64_t lent_block_stride;
   uint32_t layer_group;
   uint64_t local_group_stride, lent_group_stride;
+  uint32_t staged_only;        // 1: a row whose block is staged goes to the staged copy only (it is written back later)
   uint32_t split_layer;        // layers from here on have their home in the lent arena, at the id the entry names
                                //   (0xFFFFFFFF: no split; the entry's sign names the arena)
   uint8_t* slot_base;          // one layer: ring slot holding the layer, or NULL when not staged

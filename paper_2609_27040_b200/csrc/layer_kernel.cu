@@ -1293,8 +1293,10 @@ __global__ void __launch_bounds__(128) append_kv_kernel(const AppendParams p) {
   for (uint32_t v = threadIdx.x; v < vecs; v += blockDim.x) {
     const uint4 kv = ks[v], vv = vs[v];
     const uint32_t w = (v & ~7u) | ((v & 7u) ^ (r & 7u));  // the block format's swizzle of 16-byte units
-    reinterpret_cast<uint4*>(home + r * p.row_bytes)[w] = kv;
-    reinterpret_cast<uint4*>(home + plane + r * p.row_bytes)[w] = vv;
+    if (!(staged && p.staged_only)) {
+      reinterpret_cast<uint4*>(home + r * p.row_bytes)[w] = kv;
+      reinterpret_cast<uint4*>(home + plane + r * p.row_bytes)[w] = vv;
+    }
     if (staged) {
       reinterpret_cast<uint4*>(staged + r * p.row_bytes)[w] = kv;
       reinterpret_cast<uint4*>(staged + plane + r * p.row_bytes)[w] = vv;

@@ -73,9 +73,10 @@ struct SlotState {
   bool valid = false;
   uint32_t layer = 0;
   uint64_t plan_serial = 0;
-  bool pref_recorded = false, attn_recorded = false;
-  cudaStream_t pref_stream = nullptr, attn_stream = nullptr;
+  bool pref_recorded = false, attn_recorded = false, wb_recorded = false;
+  cudaStream_t pref_stream = nullptr, attn_stream = nullptr, wb_stream = nullptr;
   cudaEvent_t pref_done = nullptr, attn_done = nullptr;
+  cudaEvent_t wb_done = nullptr;  // swap-out passes: the slot's last write-back to the lent arena
 };
 
 struct StreamEpoch {
@@ -148,6 +149,7 @@ struct ema_slice {
   // q streamed in behind a running pass: copy stream, per-chunk arrival flags, their epoch (pinned
   // host word the flag copies read), and the event after which io_q may be overwritten.
   cudaStream_t io_stream = nullptr;
+  cudaStream_t swap_stream = nullptr;  // swap-out passes: the write-backs run here, beside gather and attention
   uint32_t* q_flags_dev = nullptr;
   uint32_t* q_epoch_host = nullptr;
   uint32_t q_epoch = 0;
@@ -531,6 +533,8 @@ int plan_on_stream(ema_slice* s, Plan* p, cudaStream_t stream) {
   return SLICE_OK;
 }
 
+int do_writeback(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t stream);
+
 void invalidate_staged(ema_slice* s) {
   for (auto& sl : s->slots) sl.valid = false;
 }
@@ -570,6 +574,9 @@ void fill_gather(const ema_slice* s, uint32_t layer, const Plan* p, ema::CopyDes
 int order_before_slot_write(ema_slice* s, SlotState& sl, cudaStream_t stream) {
   if (sl.attn_recorded && sl.attn_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.attn_done, 0));
   if (s->append_pending && s->append_stream != stream) CU(s, cudaStreamWaitEvent(stream, s->append_done, 0));
+  // Swap-out: the slot is refilled only when its content has been written back, and a gather of the
+  // same layer later on reads the lent arena only after that write.
+  if (sl.wb_recorded && sl.wb_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.wb_done, 0));
   return SLICE_OK;
 }
 
@@ -917,6 +924,7 @@ void destroy_impl(ema_slice* s) {
     for (auto& sl : s->slots) {
       if (sl.pref_done) cudaEventDestroy(sl.pref_done);
       if (sl.attn_done) cudaEventDestroy(sl.attn_done);
+      if (sl.wb_done) cudaEventDestroy(sl.wb_done);
     }
     for (auto e : s->prof)
       if (e) cudaEventDestroy(e);
@@ -943,6 +951,7 @@ void destroy_impl(ema_slice* s) {
     if (s->q_epoch_host) cudaFreeHost(s->q_epoch_host);
     if (s->io_q_free) cudaEventDestroy(s->io_q_free);
     if (s->io_stream) cudaStreamDestroy(s->io_stream);
+    if (s->swap_stream) cudaStreamDestroy(s->swap_stream);
   } else {
     for (Plan& p : s->plans) delete[] p.host;
   }
@@ -961,7 +970,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 2 || cfg->static_split > 1 || cfg->prefetch_priority > 1) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 2 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 1) return SLICE_EINVAL;
   // Section 4.2: slabs, layer groups, layouts.
   const uint32_t group = cfg->layer_group ? cfg->layer_group : 1u, slab = cfg->slab_blocks;
   if (cfg->layout > 2 || group > cfg->num_layers) return SLICE_EINVAL;
@@ -1090,7 +1099,8 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (!null_dev) {
     for (auto& sl : s->slots) {
       if (cudaEventCreateWithFlags(&sl.pref_done, cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&sl.attn_done, cudaEventDisableTiming) != cudaSuccess)
+          cudaEventCreateWithFlags(&sl.attn_done, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&sl.wb_done, cudaEventDisableTiming) != cudaSuccess)
         return fail(SLICE_ECUDA);
     }
     if (cudaHostAlloc(reinterpret_cast<void**>(&s->dev_status), 256, cudaHostAllocMapped) != cudaSuccess) return fail(SLICE_ECUDA);
@@ -1612,6 +1622,7 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
   a.lent_base = static_cast<uint8_t*>(s->cfg.lent_base) - ema::layer_offset(s->split, s->group, s->lent_gs, s->lent_ls);
   a.lent_block_stride = s->lent_bs;
   a.split_layer = s->split ? s->split : 0xFFFFFFFFu;
+  a.staged_only = s->cfg.swap_out;
   a.layer_group = s->group;
   a.local_group_stride = s->local_gs;
   a.lent_group_stride = s->lent_gs;
@@ -1643,10 +1654,19 @@ int slice_append_kv(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t ns
 
 int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint32_t nseq, void* stream_v) {
   if (!s || layer >= s->cfg.num_layers) return SLICE_EINVAL;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   Plan* p = nullptr;
   int rc = get_plan(s, seqs, nseq, &p);
   if (rc) return rc;
+  return do_writeback(s, layer, p, static_cast<cudaStream_t>(stream_v));
+}
+
+}  // extern "C"
+
+namespace {
+
+// Every staged block of `layer` goes from its ring slot back to its home in the lent arena.
+int do_writeback(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t stream) {
+  int rc = SLICE_OK;
   const uint32_t slot = layer % s->layer_slots;
   SlotState& sl = s->slots[slot];
   if (s->split && layer < s->split) return SLICE_EINVAL;  // a layer of the local half is never staged
@@ -1657,6 +1677,8 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   rc = plan_on_stream(s, p, stream);
   if (rc) return rc;
   if (sl.pref_recorded && sl.pref_stream != stream) CU(s, cudaStreamWaitEvent(stream, sl.pref_done, 0));
+  // rows appended to the staged copy (on the caller's stream) must be in it
+  if (s->append_pending && s->append_stream != stream) CU(s, cudaStreamWaitEvent(stream, s->append_done, 0));
   ema::CopyDesc d{};
   d.src_base[0] = d.src_base[1] = static_cast<const uint8_t*>(s->cfg.staging_base) + slot * s->slot_bytes;
   d.src_block_stride[0] = d.src_block_stride[1] = s->block_bytes;
@@ -1671,16 +1693,15 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
   const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
   CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, stream));
   s->st.kernel_launches++;
-  // A later prefetch of this layer reads the lent arena: it must see the written blocks.
-  if (multi_stream(s)) CU(s, cudaEventRecord(s->append_done, stream));
-  s->append_pending = multi_stream(s);
-  s->append_stream = stream;
+  // A later prefetch into this slot (of this layer again, which reads the lent arena, or of another
+  // layer, which overwrites the slot) must come after the written blocks.
+  if (multi_stream(s)) {
+    CU(s, cudaEventRecord(sl.wb_done, stream));
+    sl.wb_recorded = true;
+  }
+  sl.wb_stream = stream;
   return SLICE_OK;
 }
-
-}  // extern "C"
-
-namespace {
 
 // Stream memory operations of the driver (a stream-ordered 32-bit write; a stream-ordered wait until
 // a 32-bit word has reached a value), looked up through the runtime so that the library does not
@@ -1720,8 +1741,9 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   if (rc) return rc;
   const uint32_t L = s->cfg.num_layers, R = s->layer_slots, K = s->group;
   // Mode 0: one launch for the whole pass when the shape allows it, else one launch per layer.
+  // (Swap-out passes run layer by layer: the write-back of a layer goes on a stream of its own.)
   const bool step = s->cfg.pipeline_mode == 0 && s->cfg.ring_slots >= 2 && L >= 2 && L <= ema::kMaxStepLayers &&
-                    s->ncta <= static_cast<uint32_t>(s->num_sms);
+                    s->ncta <= static_cast<uint32_t>(s->num_sms) && !s->cfg.swap_out;
   const bool fused = s->cfg.pipeline_mode != 1 && s->cfg.ring_slots >= 2;
   if (fused) side = stream;
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;
@@ -1835,7 +1857,16 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
       s->fill_busy[slot] = true;
     }
   }
+  if (s->cfg.swap_out && !s->null_dev && !s->swap_stream)
+    CU(s, cudaStreamCreateWithFlags(&s->swap_stream, cudaStreamNonBlocking));
   for (uint32_t l = 0; l < L && !step; ++l) {
+    // Swap-out (Section 2.3: layers are swapped in and out cyclically; as much leaves as comes in):
+    // the layer's staged blocks go back to the lent arena, on a third stream, while the layer is
+    // attended to and the next transfer comes in. The slot is refilled only after that write.
+    if (s->cfg.swap_out && needs_staging(s, l, p->k) && staged(s, l, p)) {
+      rc = do_writeback(s, l, p, s->swap_stream);
+      if (rc) return rc;
+    }
     // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.
     int next = -1;
     if (p->k) {

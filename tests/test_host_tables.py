@@ -39,8 +39,8 @@ def test_library_exports_every_declared_entry_point():
 
 
 def test_config_struct_matches_header_size():
-    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 12 uint32
-    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 12 * 4
+    # 14 uint32, 3 pointers, 4 uint64, 2 pointers, 13 uint32 (+ 4 bytes of tail padding)
+    assert C.sizeof(B.SliceConfig) == 14 * 4 + 3 * 8 + 4 * 8 + 2 * 8 + 13 * 4 + 4
 
 
 def test_create_rejects_bad_configs():
