@@ -39,7 +39,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=None, help="default 200 (reference arm: 5)")
     ap.add_argument("--warmup", type=int, default=None, help="default 10 (reference arm: 1)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama3_8b_decode", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="llama3_8b_decode", choices=sorted(synth.WORKLOADS) + ["prefetch_microbench"],
+                    help="a decode workload, or prefetch_microbench: the gather / scatter sweep over launch sizes")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--copy-kind", type=int, default=0)
     ap.add_argument("--copy-ctas", type=int, default=0)
@@ -339,6 +340,108 @@ def parity_check(wl, pl, local, lent, q, outs, scale, seed):
     return {"layers": layers, "seqs": seqs, "heads": "all", "checked": sorted(outs), "against": "oracle.dense_attention (fp64)",
             "tolerance": "|err| <= 1e-2 + 1e-2*|ref|", "max_abs_err": max(worst.values()),
             "max_abs_err_by_pass": worst, "max_rel_err": max(worst_rel.values()), "ok": True}
+
+
+# ---------------------------------------------------------------------------------------------
+# Prefetch / migration microbenchmark (gather of randomly indexed 64 KB blocks into a ring, and back)
+# ---------------------------------------------------------------------------------------------
+def prefetch_microbench(totals=(1_000, 10_000, 100_000, 1_000_000), batches=(1, 8, 64, 512, 4096, 32768),
+                        arena_blocks=262_144, max_launches=2048, seed=0, reference_line=True):
+    """Gather of N randomly indexed KV blocks (16 tokens x 8 heads x 128 x bf16, K and V: 64 KB) from a
+    lent arena into a ring of two staging slots, in launches of b blocks, and the scatter of the same
+    blocks back to their ids. The arena holds min(N, arena_blocks) ids; the indices are seeded
+    permutations of it (fresh ones concatenated when N is larger). Up to max_launches launches of a
+    case are timed (CUDA events on the launching stream; the rate of a launch does not depend on how
+    many follow). GB/s counts bytes read plus bytes written. Returns a list of rows."""
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    BB = 65536
+    rows = []
+    stream = torch.cuda.Stream()
+    free, _ = torch.cuda.mem_get_info()
+    cap_blocks = int(min(arena_blocks, 0.6 * free // BB))
+    bmax = max(batches)
+    ring = torch.zeros((2, bmax, BB // 2), dtype=torch.int16, device="cuda")
+    arena = None
+    for N in totals:
+        A = min(N, cap_blocks)
+        if arena is None or arena.shape[0] != A:
+            del arena
+            torch.cuda.empty_cache()
+            arena = torch.empty((A, BB // 2), dtype=torch.int16, device="cuda")
+            arena.random_(-30000, 30000)
+        rng = np.random.default_rng(seed + N)
+        idx_h = np.concatenate([rng.permutation(A) for _ in range(-(-N // A))])[:N].astype(np.int32)
+        idx = torch.from_numpy(idx_h).cuda()
+        for b in batches:
+            if b > N:
+                continue
+            launches = min(N // b, max_launches)
+            for direction in ("gather", "scatter"):
+                def run(n_launch):          # the launches are issued by the library (one call), not one by one from here
+                    rc = B.slice_copy_blocks_series(ring, 2, bmax * BB, arena, idx, n_launch * b, b, BB, direction == "scatter",
+                                                    B.COPY_DEFAULT if b < 64 else B.COPY_BULK, 0, stream)
+                    assert rc == 0
+                run(min(launches, 8))
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                run(launches)
+                e1.record(stream)
+                e1.synchronize()
+                sec = e0.elapsed_time(e1) / 1e3
+                moved = 2 * launches * b * BB
+                row = {"blocks_total": N, "blocks_per_launch": b, "direction": direction, "launches_timed": launches,
+                       "us_per_launch": round(sec / launches * 1e6, 2), "gbs": round(moved / sec / 1e9, 1),
+                       "arena_blocks": A, "l2": "arena fits in L2" if A * BB <= 126 << 20 else "larger than L2"}
+                if direction == "gather" and b * launches <= 20000:      # byte check of what the last launches left in the ring
+                    torch.cuda.synchronize()
+                    j = launches - 1
+                    row["ring_matches_index_select"] = bool(torch.equal(ring[j & 1][:b], arena.index_select(0, idx[j * b:(j + 1) * b].long())))
+                rows.append(row)
+        if reference_line and N >= 10_000:
+            b = min(4096, N)
+            launches = min(N // b, 64)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                for j in range(launches):
+                    torch.index_select(arena, 0, idx[j * b:(j + 1) * b], out=ring[j & 1][:b])
+                e1.record(stream)
+            e1.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3
+            rows.append({"blocks_total": N, "blocks_per_launch": b, "direction": "gather",
+                         "kernel": "torch.index_select (a reference line, not product code)",
+                         "gbs": round(2 * launches * b * BB / sec / 1e9, 1)})
+    del arena, ring
+    torch.cuda.empty_cache()
+    return rows
+
+
+def run_prefetch_microbench(args):
+    """`--workload prefetch_microbench`: the whole sweep, one JSON line."""
+    import torch
+    from paper_2609_27040_b200 import binding as B
+    from paper_2609_27040_b200 import build as build_mod
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    build_mod.build()
+    B.lib()
+    peak, peak_src = measured_peaks()
+    rows = prefetch_microbench(seed=args.seed)
+    best = max(r["gbs"] for r in rows if "kernel" not in r)
+    line = {"metric": "prefetch_gather_scatter_gbs", "value": best, "unit": "GB/s", "n_gpus": 1, "steps": 1, "warmup": 1,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": "prefetch_microbench", "block_bytes": 65536, "ring_slots": 2,
+                       "note": "value = best rate of the sweep; rows = every case"},
+            "roofline": {"bound": "hbm", "achieved": best, "peak": peak, "unit": "GB/s", "frac": best / peak,
+                         "peak_source": f"of {peak_src}", "traffic": None},
+            "rows": rows}
+    print(json.dumps(line), flush=True)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -661,6 +764,9 @@ def run_ours(args, wl):
                     "note": "the default pipeline maximises tokens/s and misses the stall target: attention and prefetch "
                             "share one HBM, attention takes its share first and then waits while the copy threads use "
                             "the rest; the named configuration meets both targets at the lower tokens/s stated"}
+            # The prefetch / migration microbenchmark in short (the whole sweep: --workload prefetch_microbench).
+            extra["prefetch_microbench"] = prefetch_microbench(totals=(100_000,), batches=(1, 8, 64, 512, 4096, 32768),
+                                                               arena_blocks=100_000, max_launches=512, seed=args.seed)
             extra["kernels_alone"] = {
                 "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
@@ -714,6 +820,9 @@ def run_ours(args, wl):
 
 def main():
     args = parse_args()
+    if args.workload == "prefetch_microbench":
+        run_prefetch_microbench(args)
+        return
     wl = synth.WORKLOADS[args.workload]
     if args.layers or args.batch:
         import dataclasses

@@ -470,6 +470,16 @@ int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entri
 int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_base, const int32_t* src_idx,
                       uint32_t n, uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream);
 
+/* The prefetch / migration microbenchmark's inner loop, so that launches of a few blocks are not
+ * timed through a scripting language: blocks idx[0 .. n_total) (device array of ids into arena_base)
+ * are gathered in launches of per_launch blocks into a ring of ring_slots staging slots of
+ * slot_bytes each (launch j fills slot j mod ring_slots from position 0), or, with scatter != 0,
+ * written from the slots back to those ids. n_total / per_launch launches are enqueued on stream;
+ * a remainder is left out. Same kinds and alignment rules as slice_copy_blocks. */
+int slice_copy_blocks_series(void* ring_base, uint32_t ring_slots, uint64_t slot_bytes, void* arena_base, const int32_t* idx,
+                             uint64_t n_total, uint32_t per_launch, uint64_t block_bytes, int32_t scatter, uint32_t kind,
+                             uint32_t ctas, void* stream);
+
 const char* slice_strerror(int code);
 
 #ifdef __cplusplus

@@ -33,6 +33,7 @@ EXPORTS = [
     "slice_reclaim_preempt", "slice_preempt_seq", "slice_set_preempt_window", "slice_set_time", "slice_preempt_stats",
     "slice_set_peer_used", "slice_schedule_gll",
     "slice_step_begin", "slice_step_submit_q", "slice_step_wait_out", "slice_step_flags", "slice_step_relay",
+    "slice_copy_blocks_series",
 ]
 
 
@@ -124,6 +125,7 @@ def lib() -> C.CDLL:
         L.slice_layer_times.argtypes = [vp, vp, u32]
         L.slice_cta_trace.argtypes = [vp, i32, vp, u64, vp, vp]
         L.slice_copy_blocks.argtypes = [vp, vp, vp, vp, u32, u64, u32, u32, vp]
+        L.slice_copy_blocks_series.argtypes = [vp, u32, u64, vp, vp, u64, u32, u64, i32, u32, u32, vp]
         L.slice_strerror.argtypes = [C.c_int]
         L.slice_strerror.restype = C.c_char_p
         _lib = L
@@ -402,6 +404,12 @@ def slice_copy_blocks(dst, dst_idx, src, src_idx, n: int, block_bytes: int, kind
                       stream=None) -> int:
     return lib().slice_copy_blocks(_ptr(dst), _ptr(dst_idx), _ptr(src), _ptr(src_idx), n, block_bytes, kind,
                                    ctas, _stream(stream))
+
+
+def slice_copy_blocks_series(ring, ring_slots: int, slot_bytes: int, arena, idx, n_total: int, per_launch: int,
+                             block_bytes: int, scatter: bool = False, kind: int = 0, ctas: int = 0, stream=None) -> int:
+    return lib().slice_copy_blocks_series(_ptr(ring), ring_slots, slot_bytes, _ptr(arena), _ptr(idx), n_total, per_launch,
+                                          block_bytes, int(scatter), kind, ctas, _stream(stream))
 
 
 def slice_schedule_gll(slices) -> int:

@@ -2061,6 +2061,24 @@ int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_ba
   return ema::launch_copy(d, kind, ctas, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SLICE_OK : SLICE_ECUDA;
 }
 
+int slice_copy_blocks_series(void* ring_base, uint32_t ring_slots, uint64_t slot_bytes, void* arena_base, const int32_t* idx,
+                             uint64_t n_total, uint32_t per_launch, uint64_t block_bytes, int32_t scatter, uint32_t kind,
+                             uint32_t ctas, void* stream) {
+  if (!ring_base || !arena_base || !idx || ring_slots == 0 || per_launch == 0 || (block_bytes & 15u) || block_bytes == 0 || kind > 2)
+    return SLICE_EINVAL;
+  if (static_cast<uint64_t>(per_launch) * block_bytes > slot_bytes) return SLICE_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(ring_base) | reinterpret_cast<uintptr_t>(arena_base) | slot_bytes) & 15u) return SLICE_EINVAL;
+  const uint64_t launches = n_total / per_launch;
+  for (uint64_t j = 0; j < launches; ++j) {
+    uint8_t* slot = static_cast<uint8_t*>(ring_base) + (j % ring_slots) * slot_bytes;
+    const int32_t* sel = idx + j * per_launch;
+    const int rc = scatter ? slice_copy_blocks(arena_base, sel, slot, nullptr, per_launch, block_bytes, kind, ctas, stream)
+                           : slice_copy_blocks(slot, nullptr, arena_base, sel, per_launch, block_bytes, kind, ctas, stream);
+    if (rc) return rc;
+  }
+  return SLICE_OK;
+}
+
 const char* slice_strerror(int code) {
   switch (code) {
     case SLICE_OK: return "ok";

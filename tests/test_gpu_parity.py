@@ -758,3 +758,46 @@ def test_static_split_is_bit_identical_at_full_batch():
     st = s.slice_stats()
     assert st["device_status"] == 0 and st["last_cuda_error"] == 0
     s.close()
+
+
+@pytest.mark.parametrize("b,kind", [(1, B.COPY_DEFAULT), (7, B.COPY_VECTOR), (64, B.COPY_BULK), (300, B.COPY_BULK)])
+def test_gather_series_into_a_ring_and_back(b, kind):
+    """The microbenchmark's loop: N blocks gathered in launches of b into a ring of two slots, then
+    scattered back to the same ids. Every launch's slot content equals index_select of its ids, the
+    round trip leaves the arena bit-identical, and gathering the identity order is a plain copy."""
+    bb, A, N = 4096, 1000, 900
+    gen = torch.Generator(device="cuda").manual_seed(b)
+    arena = torch.randint(0, 256, (A, bb), dtype=torch.uint8, device="cuda", generator=gen)
+    keep = arena.clone()
+    idx = torch.randperm(A, device="cuda", generator=gen)[:N].to(torch.int32)
+    ring = torch.zeros((2, 300, bb), dtype=torch.uint8, device="cuda")
+    launches = N // b
+    for upto in (launches, launches - 1):                    # the last launch, then the one before it, left in the ring
+        ring.zero_()
+        assert B.slice_copy_blocks_series(ring, 2, 300 * bb, arena, idx, upto * b, b, bb, False, kind) == B.OK
+        torch.cuda.synchronize()
+        j = upto - 1
+        assert torch.equal(ring[j & 1, :b], arena[idx[j * b:(j + 1) * b].long()])
+    # scatter: what sits in the slots goes to the ids; written from a wiped arena it restores those blocks
+    arena.zero_()
+    src = torch.randint(0, 256, (2, 300, bb), dtype=torch.uint8, device="cuda", generator=gen)
+    assert B.slice_copy_blocks_series(src, 2, 300 * bb, arena, idx, launches * b, b, bb, True, kind) == B.OK
+    torch.cuda.synchronize()
+    want = torch.zeros_like(arena)
+    for j in range(launches):
+        want[idx[j * b:(j + 1) * b].long()] = src[j & 1, :b]
+    assert torch.equal(arena, want)
+    # round trip through a ring large enough for everything: gather all, wipe, scatter back
+    arena.copy_(keep)
+    big = torch.zeros((1, N, bb), dtype=torch.uint8, device="cuda")
+    assert B.slice_copy_blocks_series(big, 1, N * bb, arena, idx, N, N, bb, False, kind) == B.OK
+    arena[idx.long()] = 0
+    assert B.slice_copy_blocks_series(big, 1, N * bb, arena, idx, N, N, bb, True, kind) == B.OK
+    torch.cuda.synchronize()
+    assert torch.equal(arena, keep)
+    ident = torch.arange(N, dtype=torch.int32, device="cuda")
+    assert B.slice_copy_blocks_series(big, 1, N * bb, arena, ident, N, N, bb, False, kind) == B.OK
+    torch.cuda.synchronize()
+    assert torch.equal(big[0], keep[:N])
+    assert B.slice_copy_blocks_series(big, 1, N * bb, arena, idx, N, 0, bb, False, kind) == B.EINVAL
+    assert B.slice_copy_blocks_series(big, 1, 10 * bb, arena, idx, N, 11, bb, False, kind) == B.EINVAL
