@@ -53,6 +53,7 @@ def parse_args():
     ap.add_argument("--no-ablations", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parity-check", action="store_true", help="skip the oracle check of the last timed pass")
+    ap.add_argument("--no-microbench", action="store_true", help="skip the short prefetch / migration microbenchmark table")
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (debugging)")
@@ -765,8 +766,9 @@ def run_ours(args, wl):
                             "share one HBM, attention takes its share first and then waits while the copy threads use "
                             "the rest; the named configuration meets both targets at the lower tokens/s stated"}
             # The prefetch / migration microbenchmark in short (the whole sweep: --workload prefetch_microbench).
-            extra["prefetch_microbench"] = prefetch_microbench(totals=(100_000,), batches=(1, 8, 64, 512, 4096, 32768),
-                                                               arena_blocks=100_000, max_launches=512, seed=args.seed)
+            if not args.no_microbench:
+                extra["prefetch_microbench"] = prefetch_microbench(totals=(100_000,), batches=(1, 8, 64, 512, 4096, 32768),
+                                                                   arena_blocks=100_000, max_launches=512, seed=args.seed)
             extra["kernels_alone"] = {
                 "attention_only_layer_kernel": {"us_per_launch": iso_us, "algorithmic_bytes": attn_bytes_layer,
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
