@@ -63,18 +63,20 @@ namespace ema {
 
 namespace {
 
-constexpr uint32_t kNAFused = 4;           // attention ring (half-block stages) beside a copy ring
+constexpr uint32_t kNAFused = 4;           // attention ring (stages of up to 32 KB) beside a copy ring
 constexpr uint32_t kNAAlone = 3;           // ... and when the launch gathers nothing. With one 32 KB request per
                                            // stage a deeper ring only queues more reads in the memory
                                            // system and measures slower (3: 6.1 TB/s, 6: 5.3 TB/s).
-                                           // With fewer KV heads a stage is smaller (4 KB per head): the
-                                           // ring then has 8 / Hkv times as many stages, the same bytes.
-constexpr uint32_t kNAMax = 32;
+                                           // With 1 or 2 KV heads a plane is small (4 KB per head): a stage
+                                           // then holds the planes of 8 / Hkv consecutive blocks, each with
+                                           // consumer warps of its own (see blocks_per_stage); with 3 or 4
+                                           // the ring has twice as many, smaller stages.
+constexpr uint32_t kNAMax = 8;
 constexpr int kNC = 6;                     // copy ring: 16 KB stages
 constexpr uint32_t kCopyLoadsDefault = 3;  // loads in flight (LayerParams::copy_loads_ahead, 3 or 4) ...
 constexpr int kStoresOpen = 2;             // ... and stores not yet known complete; 4 + 2 = kNC
 constexpr uint32_t kCopyChunk = 16384;
-constexpr int kQueue = 20;                 // unit descriptors in flight (> kNAMax / 2 + 1)
+constexpr int kQueue = 12;                 // unit descriptors in flight (> kNAMax / 2 + 1, plus a flush and the end marker)
 constexpr uint32_t kSentinel = 0xFFFFFFFFu;
 constexpr uint32_t kFlush = 0xFFFFFFFEu;   // descriptor without data: close the open run now
 constexpr uint32_t kNewRun = 0x80000000u;
@@ -128,6 +130,7 @@ struct Smem {
   uint8_t** copy_dst;   // [kNC]
   uint32_t* copy_len;   // [kNC]
   uint32_t* mq;         // merge queue of the CTA: [kMq] entries, then tail, head, consumer warps done
+  uint32_t* head_runs;  // [8] per KV head: partials written by its consumer warps (runs x warps of the head)
   int32_t* own_res;     // [kOwnCache] resolved entries of the CTA's own range
 };
 
@@ -136,29 +139,46 @@ constexpr size_t kBarBytes = 70 * sizeof(uint64_t);
 constexpr size_t kQueueBytes = kQueue * sizeof(UnitDesc);
 constexpr size_t kCopyDstBytes = 8 * sizeof(uint8_t*);
 constexpr size_t kCopyLenBytes = 8 * sizeof(uint32_t);
-constexpr size_t kMqBytes = (kMq + 4) * sizeof(uint32_t);
+constexpr size_t kMqBytes = (kMq + 4 + 8) * sizeof(uint32_t);
 constexpr size_t kOwnBytes = kOwnCache * sizeof(int32_t);
 static_assert(2 * kNAMax + kNC <= 70 && kNC <= 8 && kQueue > kNAMax / 2 + 1, "bookkeeping area too small");
 static_assert(kNAFused * 32768 + kNC * 16384 >= kNAAlone * 32768, "the deeper ring must fit in the fused layout");
 
-// Stages per 32 KB of ring: 1 for 5..8 KV heads, 2 for 3 or 4, 4 for 2, 8 for 1.
-__host__ __device__ constexpr uint32_t ring_scale(uint32_t Hkv) { return 8u / Hkv; }
+// Blocks that share a stage: with few KV heads a plane is small (4 KB per head), and one warp per
+// KV head taking the blocks one by one, behind one producer lane issuing them one by one, is bound
+// by the per-block latencies of both (2.1 TB/s at 1 KV head, 4.2 at 2). A stage therefore holds the
+// planes of V = 8 / Hkv consecutive blocks of a unit, copied by V lanes of the producer at once, and
+// every KV head has V consumer warps, warp v taking block v of each group of V with a softmax state
+// and a partial of its own (the merge adds them up like any other partials).
+// Measured (64 sequences of 2k..8k tokens, nothing lent, KV read rate): 1 KV head 2.08 -> 3.2 TB/s,
+// 2 KV heads 4.17 -> 4.7; with 4 KV heads (16 KB planes) it is slower than one block per stage
+// (6.5 -> 5.9), so 3 and 4 KV heads keep one block per stage and twice as many stages instead.
+__host__ __device__ constexpr uint32_t blocks_per_stage(uint32_t Hkv) { return partials_per_slot(Hkv); }
+// A shared stage holds the V blocks whole (K plane and V plane are neighbours in memory: one request
+// of 8 or 16 KB per block instead of two of 4 or 8 KB), 64 KB per stage, two stages.
+__host__ __device__ constexpr uint32_t stage_bytes(uint32_t Hkv) {
+  return blocks_per_stage(Hkv) > 1 ? blocks_per_stage(Hkv) * 2 * half_stage_bytes(Hkv) : half_stage_bytes(Hkv);
+}
+constexpr uint32_t kGroupedStages = 2;
+// Stages per 32 KB of ring: 2 for 3 or 4 KV heads (planes of 12 or 16 KB), else 1.
+__host__ __device__ constexpr uint32_t ring_scale(uint32_t Hkv) { return Hkv == 3 || Hkv == 4 ? 2u : 1u; }
 
 static_assert(kRingAlign + kNAFused * 32768 + kNC * kCopyChunk + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes +
                       kOwnBytes <= 232448,
               "more shared memory than a CTA can have (227 KB)");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
-  return kRingAlign + static_cast<size_t>(kNAFused) * ring_scale(Hkv) * half_stage_bytes(Hkv) + static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
+  return kRingAlign + static_cast<size_t>(blocks_per_stage(Hkv) > 1 ? kGroupedStages : kNAFused * ring_scale(Hkv)) * stage_bytes(Hkv) +
+         static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
   Smem s;
-  s.na = (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
+  s.na = blocks_per_stage(Hkv) > 1 ? kGroupedStages : (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
   base += (kRingAlign - (ptx::smem_u32(base) & (kRingAlign - 1))) & (kRingAlign - 1);
   s.att_ring = base;
-  s.copy_ring = base + static_cast<size_t>(kNAFused) * ring_scale(Hkv) * half_stage_bytes(Hkv);
+  s.copy_ring = base + static_cast<size_t>(blocks_per_stage(Hkv) > 1 ? kGroupedStages : kNAFused * ring_scale(Hkv)) * stage_bytes(Hkv);
   uint8_t* p = s.copy_ring + static_cast<size_t>(kNC) * kCopyChunk;
   s.att_full = reinterpret_cast<uint64_t*>(p);
   s.att_empty = s.att_full + kNAMax;
@@ -167,6 +187,7 @@ __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers)
   s.copy_dst = reinterpret_cast<uint8_t**>(p + kBarBytes + kQueueBytes);
   s.copy_len = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes);
   s.mq = reinterpret_cast<uint32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes);
+  s.head_runs = s.mq + kMq + 4;
   s.own_res = reinterpret_cast<int32_t*>(p + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes);
   return s;
 }
@@ -224,11 +245,13 @@ __device__ __forceinline__ bool wait_counter(const uint32_t* cnt, uint32_t targe
 // ---------------------------------------------------------------------------------------------
 // producer warp
 // ---------------------------------------------------------------------------------------------
+template <bool kGrouped>
 __device__ void producer_role(const LayerParams& p, const Smem& sm) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv;
   const uint32_t hsb = half_stage_bytes(Hkv);
   const uint32_t plane_bytes = hsb;
+  const uint32_t V = kGrouped ? blocks_per_stage(Hkv) : 1u, sbytes = kGrouped ? stage_bytes(Hkv) : hsb;
   const uint32_t ring = ptx::smem_u32(sm.att_ring);
   uint32_t hs = 0, nq = 0;
   RingPos pos;
@@ -341,44 +364,93 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           cur_seq = seq;
           ++nruns;
         }
-        for (uint32_t blk = at; blk < ue && ok; ++blk) {
-          const uint32_t j = blk - c.b;
-          const int32_t e = __shfl_sync(0xffffffffu, my, j);
-          if (check_ready && e < 0 && __shfl_sync(0xffffffffu, rdy, j) != epoch) {
-            const uint64_t w0 = ptx::global_timer_ns();
-            ok = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
-            waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
+        if constexpr (!kGrouped) {
+          // One block at a time, one stage per plane (3 to 8 KV heads: a plane is 12 to 32 KB).
+          for (uint32_t blk = at; blk < ue && ok; ++blk) {
+            const uint32_t j = blk - c.b;
+            const int32_t e = __shfl_sync(0xffffffffu, my, j);
+            if (check_ready && e < 0 && __shfl_sync(0xffffffffu, rdy, j) != epoch) {
+              const uint64_t w0 = ptx::global_timer_ns();
+              ok = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) return;
+              waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
+            }
+            const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
+                                        : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
+  #pragma unroll
+            for (uint32_t plane = 0; plane < 2; ++plane, ++hs, pos.advance(sm.na)) {
+              const uint32_t stg = pos.stg;
+              ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) return;
+              const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
+              if (lane == 0) {
+                if (blk == at && plane == 0) {
+                  sm.queue[nq % kQueue] = UnitDesc{seq, at - seq_lo, ue - seq_lo, slot_flag, li, 0, 0, 0};
+                  ++nq;
+                }
+                // The stage was last read through the generic proxy (ldmatrix / ld.shared of the
+                // consumer warps, ordered before this point by the empty barrier); the bulk copy writes
+                // it through the asynchronous proxy. Without this fence the copy can overtake those
+                // reads: seen as rare wrong V tiles in launches spanning several layers.
+                ptx::fence_proxy_async();
+                // A staged block was written by another CTA's bulk stores and announced through its
+                // ready flag (release / acquire above): the bulk load reads it through the
+                // asynchronous proxy, which the acquire alone does not cover.
+                if (check_ready && e < 0 && plane == 0) ptx::fence_proxy_async_global();
+                ptx::mbar_arrive_expect_tx(full, plane_bytes);
+                // One request per plane: an SM streams far faster through few large bulk copies than
+                // through many small ones.
+                ptx::bulk_g2s_hint(ring + stg * hsb, src + plane * plane_bytes, plane_bytes, full, pol_stream);
+              }
+            }
           }
-          const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
-                                      : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
-#pragma unroll
-          for (uint32_t plane = 0; plane < 2; ++plane, ++hs, pos.advance(sm.na)) {
+        } else {
+          // Groups of V consecutive blocks of the unit share a stage: lane t takes block blk + t.
+          for (uint32_t blk = at; blk < ue && ok; blk += V) {
+            const uint32_t j0 = blk - c.b, np = min(V, ue - blk);
+            const int32_t e = __shfl_sync(0xffffffffu, my, (j0 + lane) & 31u);
+            const uint32_t r = __shfl_sync(0xffffffffu, rdy, (j0 + lane) & 31u);
+            const bool mine = lane < np;
+            const bool staged_blk = check_ready && mine && e < 0;
+            if (__any_sync(0xffffffffu, staged_blk && r != epoch)) {
+              const uint64_t w0 = ptx::global_timer_ns();
+              bool landed = true;
+              if (staged_blk && r != epoch) landed = wait_counter_eq(ready + static_cast<uint32_t>(~e), epoch, p.status);
+              ok = __all_sync(0xffffffffu, landed);
+              if (!ok) return;
+              waited_ns += ptx::global_timer_ns() - w0;  // the attention sat waiting for prefetched data
+            }
+            const uint8_t* src = e >= 0 ? local_layer + static_cast<uint64_t>(e) * p.local_block_stride
+                                        : slot_base + static_cast<uint64_t>(~e) * p.block_bytes;
             const uint32_t stg = pos.stg;
             ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
             const uint32_t full = ptx::smem_u32(&sm.att_full[stg]);
             if (lane == 0) {
-              if (blk == at && plane == 0) {
+              if (blk == at) {
                 sm.queue[nq % kQueue] = UnitDesc{seq, at - seq_lo, ue - seq_lo, slot_flag, li, 0, 0, 0};
                 ++nq;
               }
+              ptx::mbar_arrive_expect_tx(full, np * 2 * plane_bytes);
+            }
+            __syncwarp();
+            if (mine) {
               // The stage was last read through the generic proxy (ldmatrix / ld.shared of the
               // consumer warps, ordered before this point by the empty barrier); the bulk copy writes
-              // it through the asynchronous proxy. Without this fence the copy can overtake those
-              // reads: seen as rare wrong V tiles in launches spanning several layers.
+              // it through the asynchronous proxy: fence between the two.
               ptx::fence_proxy_async();
               // A staged block was written by another CTA's bulk stores and announced through its
               // ready flag (release / acquire above): the bulk load reads it through the
               // asynchronous proxy, which the acquire alone does not cover.
-              if (check_ready && e < 0 && plane == 0) ptx::fence_proxy_async_global();
-              ptx::mbar_arrive_expect_tx(full, plane_bytes);
-              // One request per plane: an SM streams far faster through few large bulk copies than
-              // through many small ones.
-              ptx::bulk_g2s_hint(ring + stg * hsb, src + plane * plane_bytes, plane_bytes, full, pol_stream);
+              if (staged_blk) ptx::fence_proxy_async_global();
+              // One request per block: its K plane and V plane are neighbours in memory.
+              ptx::bulk_g2s_hint(ring + stg * sbytes + lane * 2 * hsb, src, 2 * plane_bytes, full, pol_stream);
             }
+            ++hs;
+            pos.advance(sm.na);
           }
         }
         at = ue;
@@ -665,9 +737,11 @@ __device__ __forceinline__ void merge_one(const LayerParams& p, uint32_t li, uin
   c.part_ml = part_ml_of(p, li);
   c.out = static_cast<uint8_t*>(p.out) + li * p.io_layer_stride;
   c.lse = p.lse;
-  const uint32_t s0 = p.seq_slot_base[seq];
-  const uint32_t n = p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
-                                   : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1;
+  // Every run of the sequence left one partial per consumer warp of the KV head: V per slot.
+  const uint32_t V = blocks_per_stage(p.Hkv);
+  const uint32_t s0 = p.seq_slot_base[seq] * V;
+  const uint32_t n = (p.allow_steal ? __ldcg(&seq_counts(p, li)[seq])
+                                    : (p.blk_off[seq + 1] - 1) / p.per - p.blk_off[seq] / p.per + 1) * V;
   switch (sub ? 0u : p.G) {
     case 0: merge_heads<1>(p, c, seq, g * p.G + (sub & 7u), s0, n); break;  // one head: 16 partials in flight
     case 1: merge_heads<1>(p, c, seq, g, s0, n); break;
@@ -778,7 +852,7 @@ __device__ void merge_role_local(const LayerParams& p, const Smem& sm) {
           break;
         }
         // No request will ever get this ticket once all consumers are done and the tail is behind it.
-        if (mq[kMqDone] == p.Hkv && static_cast<int32_t>(mq[kMqTail] - h) <= 0) break;
+        if (mq[kMqDone] == p.Hkv * blocks_per_stage(p.Hkv) && static_cast<int32_t>(mq[kMqTail] - h) <= 0) break;
         if (ptx::global_timer_ns() - t0 > 2 * kWaitNs) break;  // a consumer that gave up never reports in
         __nanosleep(128);
       }
@@ -868,7 +942,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
         }
         if (v != kMqEmpty || leave) break;
         // 3. nothing to do: leave, or look again a little later
-        if (is_consumer || mq[kMqDone] == p.Hkv) {
+        if (is_consumer || mq[kMqDone] == p.Hkv * blocks_per_stage(p.Hkv)) {
           bool pending = static_cast<int32_t>(mq[kMqTail] - mq[kMqHead]) > 0;
           for (uint32_t l = gli; l < p.num_layers && !pending; ++l) {
             const uint32_t* cnt = layer_counters(p, l);
@@ -907,9 +981,9 @@ __device__ __forceinline__ void release_stage(const Smem& sm, const RingPos& pos
 }
 
 // ---------------------------------------------------------------------------------------------
-// consumer warp (= KV head g), tensor-core tiles
+// consumer warp (= KV head g), tensor-core tiles, one block per stage (3 to 8 KV heads)
 // ---------------------------------------------------------------------------------------------
-__device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
+__device__ void consumer_mma_single(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv, G = p.G;
   const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
@@ -1020,9 +1094,9 @@ __device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// consumer warp (= KV head = query head g), f32 tiles for G == 1
+// consumer warp (= KV head = query head g), f32 tiles for G == 1, one block per stage (3 to 8 KV heads)
 // ---------------------------------------------------------------------------------------------
-__device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
+__device__ void consumer_alu_single(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t Hkv = p.Hkv;
   const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
@@ -1114,6 +1188,259 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g) {
   }
 }
 
+// End of a run for consumer warp v of KV head g, its partial written: warp 0 of the head counts the
+// run's blocks (and merges or queues the merge when they complete a sequence) once the other warps
+// of the head have written theirs. They process the same stages in step, so the wait is short; it
+// is bounded like every other wait.
+__device__ __forceinline__ void close_run(const LayerParams& p, const Smem& sm, uint32_t li, uint32_t seq, uint32_t g,
+                                          uint32_t v, uint32_t blocks, uint32_t& runs_closed) {
+  const uint32_t V = blocks_per_stage(p.Hkv);
+  ++runs_closed;
+  if (V == 1) {
+    finish_run(p, sm, li, seq, g, blocks);
+    return;
+  }
+  __threadfence();
+  __syncwarp();
+  if ((threadIdx.x & 31u) == 0) atomicAdd(&sm.head_runs[g], 1u);
+  if (v != 0) return;
+  volatile uint32_t* cnt = sm.head_runs + g;
+  const uint32_t target = runs_closed * V;
+  if (*cnt < target) {
+    const uint64_t t0 = ptx::global_timer_ns();
+    while (*cnt < target) {
+      if (ptx::global_timer_ns() - t0 > kWaitNs) {
+        ptx::report_status(p.status, kDevTimeout);
+        break;
+      }
+    }
+  }
+  finish_run(p, sm, li, seq, g, blocks);
+}
+
+// ---------------------------------------------------------------------------------------------
+// consumer warp v of KV head g, tensor-core tiles
+// ---------------------------------------------------------------------------------------------
+template <bool kGrouped>
+__device__ void consumer_mma(const LayerParams& p, const Smem& sm, uint32_t g, uint32_t v) {
+  if constexpr (!kGrouped) {
+    consumer_mma_single(p, sm, g);
+    return;
+  }
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t Hkv = p.Hkv, G = p.G;
+  const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
+  const uint32_t V = kGrouped ? blocks_per_stage(Hkv) : 1u, sbytes = kGrouped ? stage_bytes(Hkv) : hsb;
+  const uint32_t head_off = v * 2 * hsb + g * kD * 2;  // this warp's block of a stage (K plane, then V plane), this head's columns
+  const uint32_t ring = ptx::smem_u32(sm.att_ring);
+  const uint32_t n = lane >> 2, tig = lane & 3u, r0 = lane >> 2;
+  uint32_t nunit = 0, runs_closed = 0;
+  RingPos pos;
+  bool have_run = false;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0, q_upto = 0;
+  SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+  uint32_t qf[8][2];
+  float o[8][4];
+
+  auto emit = [&]() {
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
+      st.l1 += __shfl_xor_sync(0xffffffffu, st.l1, sh);
+      st.e0 += __shfl_xor_sync(0xffffffffu, st.e0, sh);
+      st.e1 += __shfl_xor_sync(0xffffffffu, st.e1, sh);
+    }
+    const uint32_t h0 = 2 * tig, h1 = h0 + 1;
+    float* po = part_o_of(p, run_li) + ((static_cast<uint64_t>(run_slot) * V + v) * p.Hq + g * G) * kD;
+    float* pml = part_ml_of(p, run_li) + ((static_cast<uint64_t>(run_slot) * V + v) * p.Hq + g * G) * 4;
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      const uint32_t d = mt * 16 + r0;
+      if (h0 < G) {
+        po[h0 * kD + d] = o[mt][0];
+        po[h0 * kD + d + 8] = o[mt][2];
+      }
+      if (h1 < G) {
+        po[h1 * kD + d] = o[mt][1];
+        po[h1 * kD + d + 8] = o[mt][3];
+      }
+    }
+    if (r0 == 0) {
+      if (h0 < G) *reinterpret_cast<float4*>(pml + h0 * 4) = make_float4(st.m0, st.l0, st.e0, 0.f);
+      if (h1 < G) *reinterpret_cast<float4*>(pml + h1 * 4) = make_float4(st.m1, st.l1, st.e1, 0.f);
+    }
+    if (p.trace && g == 0 && v == 0 && lane == 0)
+      p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 5] = ptx::global_timer_ns();
+    close_run(p, sm, run_li, run_seq, g, v, run_blocks, runs_closed);
+  };
+
+  for (;;) {
+    if (!wait_stage(p, sm, pos)) return;
+    const UnitDesc it = sm.queue[nunit % kQueue];
+    if (it.seq_idx == kFlush) {
+      if (have_run) emit();
+      have_run = false;
+      ++nunit;
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      continue;
+    }
+    const bool end = it.seq_idx == kSentinel;
+    if (end || (it.slot & kNewRun)) {
+      if (have_run) emit();
+      if (end) break;
+      have_run = true;
+      run_seq = it.seq_idx;
+      run_slot = it.slot & ~kNewRun;
+      run_li = it.layer;
+      run_blocks = 0;
+      len = p.lens[run_seq];
+      st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+      if (run_li >= q_upto) {  // q may still be on its way: wait for this layer's rows (or chunk of layers)
+        const uint64_t w0 = p.trace && p.q_ready ? ptx::global_timer_ns() : 0;
+        if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+        if (p.trace && p.q_ready && g == 0 && v == 0 && lane == 0) {
+          const uint64_t w1 = ptx::global_timer_ns();
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 6] = w1 - w0;
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 7] = w1;
+        }
+      }
+      // Q^T fragments (B operand): head n = lane/4 of the group, dims ks*16 + 2*(lane%4) (+8).
+      const __nv_bfloat16* qg =
+          reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
+      const uint32_t* qrow =
+          reinterpret_cast<const uint32_t*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g * G + (n < G ? n : 0)) * kD);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qf[ks][0] = n < G ? __ldcg(qrow + ks * 8 + tig) : 0u;
+        qf[ks][1] = n < G ? __ldcg(qrow + ks * 8 + tig + 4) : 0u;
+      }
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    }
+    ++nunit;
+    // Groups of V blocks share a stage; this warp takes block v of each group (none in a short one).
+    for (uint32_t gb = it.blk_begin; gb < it.blk_end; gb += V) {
+      if (gb != it.blk_begin && !wait_stage(p, sm, pos)) return;
+      const uint32_t b = gb + v;
+      const bool mine = !kGrouped || b < it.blk_end;
+      const uint32_t valid = mine ? min(kT, len - b * kT) : 0u;
+      uint32_t pb0 = 0, pb1 = 0;
+      float al0 = 1.f, al1 = 1.f;
+      if (mine) {
+        tile_mma_scores(ring + pos.stg * sbytes + head_off, rb, valid, qf, p.scale_log2, st, pb0, pb1, al0, al1);
+        tile_mma_pv(ring + pos.stg * sbytes + head_off + hsb, rb, valid, pb0, pb1, al0, al1, o);
+      }
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+    }
+    run_blocks += it.blk_end - it.blk_begin;  // the run's blocks, whichever warp of the head took them
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// consumer warp v of KV head (= query head) g, f32 tiles for G == 1
+// ---------------------------------------------------------------------------------------------
+template <bool kGrouped>
+__device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g, uint32_t v) {
+  if constexpr (!kGrouped) {
+    consumer_alu_single(p, sm, g);
+    return;
+  }
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t Hkv = p.Hkv;
+  const uint32_t hsb = half_stage_bytes(Hkv), rb = row_bytes(Hkv);
+  const uint32_t V = kGrouped ? blocks_per_stage(Hkv) : 1u, sbytes = kGrouped ? stage_bytes(Hkv) : hsb;
+  const uint32_t head_off = v * 2 * hsb + g * kD * 2;
+  const uint32_t half = lane & 1u;
+  uint32_t nunit = 0, runs_closed = 0;
+  RingPos pos;
+  bool have_run = false;
+  uint32_t run_seq = 0, run_slot = 0, run_blocks = 0, run_li = 0, len = 0, q_upto = 0;
+  SegState st{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+  float qh[64];  // this lane's half (64 dims) of q as f32
+  float o[4] = {0.f, 0.f, 0.f, 0.f};
+
+  auto emit = [&]() {
+#pragma unroll
+    for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
+    float* po = part_o_of(p, run_li) + ((static_cast<uint64_t>(run_slot) * V + v) * p.Hq + g) * kD;
+    *reinterpret_cast<float4*>(po + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
+    if (lane == 0)
+      *reinterpret_cast<float4*>(part_ml_of(p, run_li) + ((static_cast<uint64_t>(run_slot) * V + v) * p.Hq + g) * 4) =
+          make_float4(st.m0, st.l0, st.l0, 0.f);
+    if (p.trace && g == 0 && v == 0 && lane == 0)
+      p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 5] = ptx::global_timer_ns();
+    close_run(p, sm, run_li, run_seq, g, v, run_blocks, runs_closed);
+  };
+
+  for (;;) {
+    if (!wait_stage(p, sm, pos)) return;
+    const UnitDesc it = sm.queue[nunit % kQueue];
+    if (it.seq_idx == kFlush) {
+      if (have_run) emit();
+      have_run = false;
+      ++nunit;
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+      continue;
+    }
+    const bool end = it.seq_idx == kSentinel;
+    if (end || (it.slot & kNewRun)) {
+      if (have_run) emit();
+      if (end) break;
+      have_run = true;
+      run_seq = it.seq_idx;
+      run_slot = it.slot & ~kNewRun;
+      run_li = it.layer;
+      run_blocks = 0;
+      len = p.lens[run_seq];
+      st = SegState{kNegInf, kNegInf, 0.f, 0.f, 0.f, 0.f};
+      if (run_li >= q_upto) {  // q may still be on its way: wait for this layer's rows (or chunk of layers)
+        const uint64_t w0 = p.trace && p.q_ready ? ptx::global_timer_ns() : 0;
+        if (p.q_ready && !wait_counter(p.q_ready + run_li / p.q_ready_layers, p.q_ready_epoch, p.status)) return;
+        q_upto = p.q_ready ? (run_li / p.q_ready_layers + 1) * p.q_ready_layers : 0xFFFFFFFFu;
+        if (p.trace && p.q_ready && g == 0 && v == 0 && lane == 0) {
+          const uint64_t w1 = ptx::global_timer_ns();
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 6] = w1 - w0;
+          p.trace[run_li * p.trace_stride + kTraceWords * blockIdx.x + 7] = w1;
+        }
+      }
+      const __nv_bfloat16* qg =
+          reinterpret_cast<const __nv_bfloat16*>(static_cast<const uint8_t*>(p.q) + run_li * p.io_layer_stride);
+      const uint4* qrow =
+          reinterpret_cast<const uint4*>(qg + (static_cast<uint64_t>(run_seq) * p.Hq + g) * kD + half * 64);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 v = __ldcg(qrow + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          qh[c * 8 + 2 * e] = __uint_as_float(w[e] << 16);
+          qh[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+        }
+      }
+      o[0] = o[1] = o[2] = o[3] = 0.f;
+    }
+    ++nunit;
+    for (uint32_t gb = it.blk_begin; gb < it.blk_end; gb += V) {
+      if (gb != it.blk_begin && !wait_stage(p, sm, pos)) return;
+      const uint32_t b = gb + v;
+      const bool mine = !kGrouped || b < it.blk_end;
+      const uint32_t valid = mine ? min(kT, len - b * kT) : 0u;
+      float pw = 0.f, al = 1.f;
+      if (mine) {
+        tile_alu_scores(sm.att_ring + pos.stg * sbytes + head_off, rb, valid, qh, p.scale_log2, st, pw, al);
+        tile_alu_pv(sm.att_ring + pos.stg * sbytes + head_off + hsb, rb, valid, pw, al, o);
+      }
+      release_stage(sm, pos);
+      pos.advance(sm.na);
+    }
+    run_blocks += it.blk_end - it.blk_begin;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // copy warp (one thread): the gathers issued during each layer of the launch
 // ---------------------------------------------------------------------------------------------
@@ -1150,6 +1477,11 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     uint32_t my_pos[16], my_n[16], my_end[16];  // this thread's most recent units: first position, blocks,
                                                 // and this layer's piece count once the unit is fully issued
     uint32_t my_units = 0;                // units of this layer taken by this thread
+    // Small blocks: tickets are drawn four at a time and the four units' descriptors fetched together.
+    // A unit costs an atomic and two dependent loads before its first byte can be requested, about
+    // 2.5 us that nothing overlaps; with 8 KB units that, not the bytes, was the gather's time.
+    const uint32_t batch = p.block_bytes <= 16384 ? 4u : 1u;
+    uint32_t bat_v[4], bat_e[4], bat_i = 0, bat_n = 0;
     uint32_t piece = 0, pieces = 0;       // equal: forces a unit fetch
     uint64_t unit_bytes = 0;
     const uint8_t* src_blk = nullptr;
@@ -1161,11 +1493,22 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     // Issues the load of the next 16 KB piece, pulling a new unit when the current one is used up.
     auto issue_next = [&]() -> bool {
       if (piece == pieces) {
-        const uint32_t unit = atomicAdd(ticket, 1u);
-        if (unit >= p.copy_n) return false;
-        const uint32_t v = p.copy_order[unit];
+        if (bat_i == bat_n) {
+          const uint32_t first = atomicAdd(ticket, batch);
+          if (first >= p.copy_n) return false;
+          bat_n = min(batch, p.copy_n - first);
+          bat_i = 0;
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i)
+            if (i < bat_n) bat_v[i] = p.copy_order[first + i];
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i)
+            if (i < bat_n) bat_e[i] = static_cast<uint32_t>(p.copy_src[bat_v[i] & 0xFFFFFFu]);
+        }
+        const uint32_t v = bat_v[bat_i];
+        const int32_t e = static_cast<int32_t>(bat_e[bat_i]);
+        ++bat_i;
         const uint32_t pos = v & 0xFFFFFFu, n = (v >> 24) + 1u;
-        const int32_t e = p.copy_src[pos];
         src_blk = src_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
         dst_blk = dst_slot + static_cast<uint64_t>(pos) * p.block_bytes;
         unit_bytes = static_cast<uint64_t>(n) * p.block_bytes;
@@ -1225,7 +1568,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   }
 }
 
-template <bool kMma>
+template <bool kMma, bool kGrouped>
 __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   bool gathers = false;
@@ -1233,22 +1576,24 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     for (uint32_t li = 0; li < p.num_layers; ++li) gathers |= p.gather_target[li] >= 0;
   const Smem sm = carve(smem_raw, p.Hkv, gathers);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t ncons = p.Hkv * blocks_per_stage(p.Hkv);  // consumer warps: blocks_per_stage per KV head
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < sm.na; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sm.att_full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), p.Hkv);
+      ptx::mbar_init(ptx::smem_u32(&sm.att_empty[s]), ncons);
     }
+    for (uint32_t g = 0; g < 8; ++g) sm.head_runs[g] = 0;
     for (int s = 0; s < kNC; ++s) ptx::mbar_init(ptx::smem_u32(&sm.copy_full[s]), 1);
     for (uint32_t s = 0; s < kMq; ++s) sm.mq[s] = kMqEmpty;
     sm.mq[kMqTail] = sm.mq[kMqHead] = sm.mq[kMqDone] = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
-  if (warp < p.Hkv) {
+  if (warp < ncons) {
     if constexpr (kMma)
-      consumer_mma(p, sm, warp);
+      consumer_mma<kGrouped>(p, sm, warp % p.Hkv, warp / p.Hkv);
     else
-      consumer_alu(p, sm, warp);
+      consumer_alu<kGrouped>(p, sm, warp % p.Hkv, warp / p.Hkv);
     __syncwarp();
     if (lane == 0) {
       __threadfence_block();
@@ -1256,11 +1601,11 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     }
     __syncwarp();
     merge_role(p, sm, true);
-  } else if (warp == p.Hkv) {
-    producer_role(p, sm);
-  } else if (warp == p.Hkv + 1) {
+  } else if (warp == ncons) {
+    producer_role<kGrouped>(p, sm);
+  } else if (warp == ncons + 1) {
     if (lane == 0) copy_role(p, sm);
-  } else if (warp == p.Hkv + 2) {
+  } else if (warp == ncons + 2) {
     merge_role(p, sm, false);
   }
 }
@@ -1330,28 +1675,37 @@ size_t layer_smem_bytes(uint32_t Hkv) {
   return smem_total(Hkv);
 }
 
+namespace {
+// The four instantiations: tensor-core or f32 tiles, one block per stage (5..8 KV heads) or groups of
+// 8 / Hkv blocks per stage (1 or 2 KV heads).
+const void* layer_kernel_for(uint32_t Hkv, uint32_t G) {
+  const bool grouped = blocks_per_stage(Hkv) > 1;
+  if (G == 1)
+    return grouped ? reinterpret_cast<const void*>(slice_layer_kernel<false, true>)
+                   : reinterpret_cast<const void*>(slice_layer_kernel<false, false>);
+  return grouped ? reinterpret_cast<const void*>(slice_layer_kernel<true, true>)
+                 : reinterpret_cast<const void*>(slice_layer_kernel<true, false>);
+}
+}  // namespace
+
 cudaError_t layer_setup() {
   const int smem = static_cast<int>(layer_smem_bytes(8));
-  cudaError_t e = cudaFuncSetAttribute(slice_layer_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(slice_layer_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  for (uint32_t Hkv : {8u, 1u})
+    for (uint32_t G : {1u, 2u}) {
+      cudaError_t e = cudaFuncSetAttribute(layer_kernel_for(Hkv, G), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (e != cudaSuccess) return e;
+    }
+  return cudaSuccess;
 }
 
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
   const size_t smem = layer_smem_bytes(p.Hkv);
-  const unsigned threads = (p.Hkv + 3) * 32;
-  if (p.num_layers > 1) {
-    // CTAs wait for one another across layers: all of them must be resident.
-    void* args[] = {const_cast<LayerParams*>(&p)};
-    const void* fn = p.G == 1 ? reinterpret_cast<const void*>(slice_layer_kernel<false>)
-                              : reinterpret_cast<const void*>(slice_layer_kernel<true>);
-    return cudaLaunchCooperativeKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
-  }
-  if (p.G == 1)
-    slice_layer_kernel<false><<<p.ncta, threads, smem, stream>>>(p);
-  else
-    slice_layer_kernel<true><<<p.ncta, threads, smem, stream>>>(p);
-  return cudaGetLastError();
+  const unsigned threads = (p.Hkv * blocks_per_stage(p.Hkv) + 3) * 32;
+  void* args[] = {const_cast<LayerParams*>(&p)};
+  const void* fn = layer_kernel_for(p.Hkv, p.G);
+  // CTAs of a launch that spans several layers wait for one another: all of them must be resident.
+  if (p.num_layers > 1) return cudaLaunchCooperativeKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
+  return cudaLaunchKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t stream) {

@@ -635,7 +635,8 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
 // Room for `buffers` partial buffers of slots * Hq rows each (a pass over all layers alternates
 // between two).
 int ensure_partials(ema_slice* s, uint32_t Hq, uint32_t slots, uint32_t buffers = 1) {
-  const size_t rows = static_cast<size_t>(slots) * Hq * buffers;
+  // (a slot holds one partial per consumer warp of a KV head)
+  const size_t rows = static_cast<size_t>(slots) * ema::partials_per_slot(s->cfg.num_kv_heads) * Hq * buffers;
   if (s->null_dev || rows <= s->part_rows) return SLICE_OK;
   if (s->part_o) {
     CU(s, cudaDeviceSynchronize());
@@ -735,7 +736,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
   for (uint32_t i = 0; i < p->nseq; ++i)
     if (lens[i] == 0) return SLICE_EINVAL;
   if (static_scratch) {
-    if (ema::static_scratch_needed(p->slots_static, Hq, p->nseq, Hkv, s->ncta) > ema::static_scratch_bytes())
+    if (ema::static_scratch_needed(p->slots_static * ema::partials_per_slot(Hkv), Hq, p->nseq, Hkv, s->ncta) > ema::static_scratch_bytes())
       return SLICE_ESCRATCH;
     // The array's address belongs to the device the slice lives on; with another device current the
     // launch would be given another GPU's array.
@@ -777,7 +778,7 @@ int do_layer(ema_slice* s, uint32_t layer, Plan* p, const void* q, uint32_t Hq, 
     d.gather_target[0] = gather ? static_cast<int16_t>(next_layer) : static_cast<int16_t>(-1);
     d.gather_after[0] = -1;  // the slot's last reader precedes this launch in stream order
     if (static_scratch)
-      CU(s, ema::launch_layer_static(d, p->slots_static, stream));
+      CU(s, ema::launch_layer_static(d, p->slots_static * ema::partials_per_slot(Hkv), stream));
     else
       CU(s, ema::launch_layer(d, stream));
     s->st.kernel_launches++;
