@@ -654,9 +654,15 @@ def run_ours(args, wl):
             # stream-ordered memory operations, so no kernel has to fit beside the persistent one.
             # A second form leaves 8 SMs free and has a kernel of the caller (an elementwise negation)
             # compute q[l+1] from out[l] on them.
-            for label, alias in ((("layer_dependent_q", True), ("layer_dependent_q_caller_kernel", False))
-                                 if args.pipeline_mode == 0 else ()):
-                kwa = dict(kw) if alias else {**kw, "decode_ctas": max(1, torch.cuda.get_device_properties(0).multi_processor_count - 8)}
+            for label, alias, prio in ((("layer_dependent_q", True, args.prefetch_priority),
+                                        ("layer_dependent_q_prefetch_priority", True, 1),
+                                        ("layer_dependent_q_caller_kernel", False, args.prefetch_priority))
+                                       if args.pipeline_mode == 0 else ()):
+                if label == "layer_dependent_q_prefetch_priority" and args.prefetch_priority:
+                    continue
+                kwa = {**kw, "prefetch_priority": prio}
+                if not alias:
+                    kwa["decode_ctas"] = max(1, torch.cuda.get_device_properties(0).multi_processor_count - 8)
                 try:
                     wa = DeviceWorkload(wl, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **kwa)
                     X = torch.zeros((L + 1,) + tuple(wa.q.shape[1:]), device="cuda", dtype=torch.bfloat16)
@@ -696,7 +702,7 @@ def run_ours(args, wl):
                         "tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
                         "hbm_gbs_combined": step_bytes * reps / ta / 1e9,
                         "stall_us_per_layer": float((tr[1:, :wa.s.cfg.decode_ctas or None, 1] / 1e3).mean()),
-                        "decode_ctas": int(wa.s.cfg.decode_ctas) or "one per SM",
+                        "decode_ctas": int(wa.s.cfg.decode_ctas) or "one per SM", "prefetch_priority": prio,
                         "note": "slice_step_begin: every layer's attention waits for its queries, which are released only "
                                 "after the previous layer's output is complete (" +
                                 ("q[l+1] = out[l], aliased in memory: the caller's stream only waits and releases"
@@ -751,7 +757,8 @@ def run_ours(args, wl):
                     return (h["dram_bytes"] if h["dram_bytes"] is not None else h["algorithmic_bytes"]) >= 0.70
 
                 prio_of = {"lock_step_stealing": 0, "prefetch_priority": 1, "prefetch_priority_lock_step": 1,
-                           "layer_dependent_q": -1, "layer_dependent_q_caller_kernel": -1}     # DRAM traffic of that mode: not captured
+                           "layer_dependent_q": -1, "layer_dependent_q_caller_kernel": -1,
+                           "layer_dependent_q_prefetch_priority": -1}     # DRAM traffic of these modes: not captured
                 ok = [k for k, v in alts.items() if frac(v) < 0.05 and gate(v["hbm_gbs_combined"], prio_of.get(k, 0))]
                 pick = max(ok, key=lambda k: alts[k]["tokens_per_s"]) if ok else min(alts, key=lambda k: frac(alts[k]))
                 default_stall = extra["stall_frac_of_layer"]

@@ -878,7 +878,12 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     // the last block to the announcement of the output); in line, the warps that finish a sequence
     // together merge side by side, and the ring they stall has nothing to stream for long anyway.
     if (s->step_out_ready) d.merge_inline = 1;
-    if (s->step_out_ready) d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order_rev);
+    // Layer-dependent passes gather in reverse order by default: what a CTA reads first lands last and
+    // is still in the L2 when the layer starts (5.5 -> 5.3 ms per pass on the 8B shapes); the price is
+    // that the start of a layer may wait for those last blocks. prefetch_priority keeps the forward
+    // order: no wait, the slower pass.
+    if (s->step_out_ready && !s->cfg.prefetch_priority)
+      d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order_rev);
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / nbuf;
