@@ -145,7 +145,7 @@ typedef struct {
   uint32_t slab_blocks;           /* Section 4.2.1: 0 = blocks are handed out one by one from free stacks
                                      (the seeded orders); S > 0 = slab allocator: the ids of each part
                                      form slabs of S consecutive ids (the paper's default is 10,
-                                     Section 6.6), a slab belongs to the user while one of its blocks
+                                     Section 6.7), a slab belongs to the user while one of its blocks
                                      is in use, and the next id is the lowest free id in a slab the
                                      user holds, else the lowest free id of all (a new slab). The
                                      free orders must then be NULL                                 */

@@ -214,7 +214,7 @@ void* oracle_create(uint32_t num_layers, uint32_t block_tokens, uint64_t block_b
 
 void oracle_destroy(void* h) { delete static_cast<State*>(h); }
 
-// O-slab: turns the slab allocator on (blocks per slab; the paper's default is 10, Section 6.6).
+// O-slab: turns the slab allocator on (blocks per slab; the paper's default is 10, Section 6.7).
 // To be called before the first allocation; capacities need not be multiples of the slab (the
 // last slab of a part is then short).
 int oracle_set_slab_blocks(void* h, uint32_t slab_blocks) {

@@ -1,5 +1,5 @@
 """Pins of the oracle's slab allocator and memory layouts (Sections 4.2.1 - 4.2.3, defaults of
-Section 6.6): a hand-worked allocation sequence, the rule checked by brute force over random
+Section 6.7): a hand-worked allocation sequence, the rule checked by brute force over random
 operation sequences, the layouts as nested arrays, the paper's layer-group index example, and the
 sizes of the contiguous pieces one swap moves in each layout. CPU only."""
 import json
