@@ -46,7 +46,8 @@ def parse_args():
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--decode-ctas", type=int, default=0)
     ap.add_argument("--pipeline-mode", type=int, default=0,
-                    help="0 one persistent launch per pass, 1 two streams with events, 2 one fused launch per layer")
+                    help="0 one persistent launch per pass, 1 two streams with events, 2 one fused launch per layer, "
+                         "3 a chain of launches, one per layer, each starting while the one before it runs")
     ap.add_argument("--static-split", type=int, default=0, help="1: no work stealing between CTAs")
     ap.add_argument("--prefetch-priority", type=int, default=0,
                     help="1: two partial buffers instead of four (CTAs in step, prefetch always ahead, slower pass)")
@@ -547,8 +548,8 @@ def run_ours(args, wl):
             wp.step(wrap)
             tm = wp.s.slice_layer_times().astype(np.float64)         # synchronises
             launches_per_step = wp.s.slice_stats()["kernel_launches"] - k0
-            if args.pipeline_mode == 0:
-                kernel_us.append(float(tm[L - 1, 3] - tm[0, 2]))     # one launch spans the pass
+            if args.pipeline_mode in (0, 3):
+                kernel_us.append(float(tm[L - 1, 3] - tm[0, 2]))     # one launch (or one chain) spans the pass
             else:
                 kernel_us.append(float(np.nansum(tm[:, 4] - tm[:, 2])))
         del wp
@@ -569,7 +570,9 @@ def run_ours(args, wl):
         combined = step_bytes * args.steps / t / 1e9
         name = {0: "slice_layer_kernel (one launch per pass: attention + gather of every layer)",
                 1: "slice_layer_kernel (attention only; gather in copy_blocks_vector on a second stream)",
-                2: "slice_layer_kernel (one launch per layer: attention + gather of the next layer)"}[args.pipeline_mode]
+                2: "slice_layer_kernel (one launch per layer: attention + gather of the next layer)",
+                3: "slice_layer_kernel (a chain of launches, one per layer, each starting while the one before it runs)"
+                }[args.pipeline_mode]
         traffic, traffic_rec = profile_traffic(wl, args.pipeline_mode, args.prefetch_priority)
         roof = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic,
@@ -600,11 +603,12 @@ def run_ours(args, wl):
         del wp
         torch.cuda.empty_cache()
         if not args.no_ablations:
-            # Other pipelines on the same workload: one fused launch per layer; two kernels on two
+            # Other pipelines on the same workload: one fused launch per layer; the same launches as a
+            # chain in which each starts while the one before it runs; two kernels on two
             # streams; and the on-demand variant (gather and attention serialised on one stream), whose
             # profile events also give each kernel's duration with nothing running beside it.
             abl = {}
-            for label, mode in (("fused_launch_per_layer", 2), ("two_streams", 1)):
+            for label, mode in (("fused_launch_per_layer", 2), ("chained_launch_per_layer", 3), ("two_streams", 1)):
                 if mode == args.pipeline_mode:
                     continue
                 wa = DeviceWorkload(wl, args.seed, pipeline_mode=mode, **kw)

@@ -116,7 +116,15 @@ typedef struct {
                                      (attention of layer l overlapped with the gather of layer l+1,
                                      soft layer boundaries; falls back to 2 when the shape does not
                                      allow it), 1 = two kernels on two streams ordered by events,
-                                     2 = one fused launch per layer                              */
+                                     2 = one fused launch per layer, the stream ordering the layers,
+                                     3 = a chain of fused launches, one per layer, in which each
+                                     launch starts while the one before it still runs (programmatic
+                                     dependent launch): its CTAs take the SMs that the earlier
+                                     launch's CTAs leave and the layers order themselves through the
+                                     same flags and counters as inside the single launch of mode 0.
+                                     Same fall-back as mode 0. Nothing else may be enqueued on
+                                     `stream` by other threads while slice_decode_step enqueues a
+                                     chain                                                        */
   uint32_t static_split;          /* attention work split: 0 = each CTA owns a range of blocks and idle
                                      CTAs steal from the ranges with most left (default); 1 = static
                                      ranges only                                                  */

@@ -92,6 +92,14 @@ struct LayerParams {
   uint64_t slot_bytes;
   uint32_t ring_slots;
   uint32_t first_layer, num_layers;
+  uint32_t li_begin, li_end;    // the layers first_layer + [li_begin, li_end) are what THIS launch runs. A pass may be
+                                //   one launch (0, num_layers) or a chain of launches over the same parameter
+                                //   block, each taking a slice of the layers (see `chained`)
+  uint32_t chained;             // 0: a launch of its own. 1, 2: a link of a chain of launches in one stream, every
+                                //   link lets its successor start as soon as all its own CTAs have started
+                                //   (programmatic dependent launch; 2 = launched as such a successor). The
+                                //   links order themselves through the same flags and counters as the layers
+                                //   of a single launch, and a link ends only after its predecessor has ended
   uint64_t block_bytes;
   const int32_t* resolved;      // flat resolved table of the batch (batch order, then block order)
   const uint32_t* lens;         // [nseq] tokens
@@ -151,9 +159,10 @@ struct LayerParams {
 size_t layer_smem_bytes(uint32_t Hkv);
 // One-time per-process opt-in to large dynamic shared memory.
 cudaError_t layer_setup();
-// Attention (+ fused gather, + merges) of num_layers layers: ONE launch. Launches that span several
-// layers contain bounded waits between CTAs and are therefore launched cooperatively (all CTAs
-// resident).
+// Attention (+ fused gather, + merges) of the layers [li_begin, li_end) of p: ONE launch. A launch
+// that spans several layers contains bounded waits between its CTAs and is therefore launched
+// cooperatively (all CTAs resident); a link of a chain spans one layer and waits only for CTAs of
+// earlier links, which have all started before its first CTA does.
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream);
 
 // A one-thread kernel that releases q_ready[l + 1] as soon as out_ready[l] shows `epoch` (and

@@ -86,6 +86,7 @@ constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kMq = 32;               // merge requests queued per CTA
 constexpr uint32_t kMqEmpty = 0xFFFFFFFFu;
 constexpr uint32_t kMqTail = kMq, kMqHead = kMq + 1, kMqDone = kMq + 2;
+constexpr uint32_t kMqWind = kMq + 3;      // set by the producer when it streams the launch's last claim
 constexpr uint32_t kOwnCache = 352;        // resolved entries of the own range kept in shared memory
 
 __host__ __device__ constexpr uint32_t row_bytes(uint32_t Hkv) { return Hkv * kD * 2; }
@@ -277,7 +278,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
     first.nhi = p.blk_off[min(first.seq + 2, p.nseq)];
   }
 
-  for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
+  for (uint32_t li = p.li_begin; li < p.li_end && ok; ++li) {
     const uint32_t layer = p.first_layer + li;
     const uint8_t* local_layer = p.local_base + layer_offset(layer, p.layer_group, p.local_group_stride, p.local_layer_stride);
     const uint8_t* slot_base = p.staging_base + (layer % p.ring_slots) * p.slot_bytes;
@@ -567,14 +568,18 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
         const int32_t my = lane >= c.e - c.b ? 0 : all_staged ? ~static_cast<int32_t>(c.b + lane) : p.resolved[c.b + lane];
         const uint32_t hint = p.blk_seq[c.b];
         const Claim nxt = steal();
+        // The last claim of a link of a chain: its copy thread takes no more units from here on, so
+        // that its last copies land while the last blocks are attended to, not after them.
+        if (nxt.b >= nxt.e && li + 1 == p.li_end && lane == 0) *reinterpret_cast<volatile uint32_t*>(sm.mq + kMqWind) = 1u;
         stream_claim(c, my, 0, false, hint);
         c = nxt;
       }
     }
+    if (li + 1 == p.li_end && lane == 0) *reinterpret_cast<volatile uint32_t*>(sm.mq + kMqWind) = 1u;
     // A run left open at the end of a layer would be closed only by this CTA's next unit, and a CTA
     // may find nothing to claim in the following layers while every CTA waits for this layer's
     // merges: close it now with a descriptor that has no data behind it.
-    if (ok && cur_seq != kSentinel && li + 1 < p.num_layers) {
+    if (ok && cur_seq != kSentinel && li + 1 < p.li_end) {
       const uint32_t stg = pos.stg;
       ok = ptx::mbar_wait(ptx::smem_u32(&sm.att_empty[stg]), pos.phase ^ 1u, p.status, kDevTimeout);
       ok = __all_sync(0xffffffffu, ok);
@@ -864,7 +869,7 @@ __device__ void merge_role_local(const LayerParams& p, const Smem& sm) {
   }
 }
 
-__device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consumer) {
+__device__ __forceinline__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consumer) {
   if (!p.shared_merges) {
     if (!p.merge_inline) merge_role_local(p, sm);
     return;
@@ -872,7 +877,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t total = p.nseq * p.Hq;  // query heads to merge per layer
   volatile uint32_t* mq = sm.mq;
-  uint32_t gli = 0, idle = 0;  // idle: looks at the own queue since the last request
+  uint32_t gli = p.li_begin, idle = 0;  // idle: looks at the own queue since the last request
   for (;;) {
     uint32_t v = kMqEmpty, sub = 0;  // a request in the CTA queue's format; one query head only?
     bool leave = false;
@@ -899,8 +904,8 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
         const bool look = (idle & 7u) == 0;
         ++idle;
         if (look)
-          while (gli < p.num_layers && __ldcg(layer_counters(p, gli) + kCntMerged) >= total) ++gli;
-        for (uint32_t l = gli; look && l < p.num_layers && l < gli + 2 && v == kMqEmpty && !leave; ++l) {
+          while (gli < p.li_end && __ldcg(layer_counters(p, gli) + kCntMerged) >= total) ++gli;
+        for (uint32_t l = gli; look && l < p.li_end && l < gli + 2 && v == kMqEmpty && !leave; ++l) {
           uint32_t* cnt = layer_counters(p, l);
           uint32_t pub = __ldcg(cnt + kCntMergePub);
           uint32_t taken = __ldcg(cnt + kCntMergeTaken);
@@ -944,7 +949,7 @@ __device__ void merge_role(const LayerParams& p, const Smem& sm, bool is_consume
         // 3. nothing to do: leave, or look again a little later
         if (is_consumer || mq[kMqDone] == p.Hkv * blocks_per_stage(p.Hkv)) {
           bool pending = static_cast<int32_t>(mq[kMqTail] - mq[kMqHead]) > 0;
-          for (uint32_t l = gli; l < p.num_layers && !pending; ++l) {
+          for (uint32_t l = gli; l < p.li_end && !pending; ++l) {
             const uint32_t* cnt = layer_counters(p, l);
             pending = __ldcg(cnt + kCntMergeTaken) < __ldcg(cnt + kCntMergePub);
           }
@@ -1110,7 +1115,7 @@ __device__ void consumer_alu_single(const LayerParams& p, const Smem& sm, uint32
   float qh[64];  // this lane's half (64 dims) of q as f32
   float o[4] = {0.f, 0.f, 0.f, 0.f};
 
-  auto emit = [&]() {
+  auto emit = [&]() __attribute__((always_inline)) {
 #pragma unroll
     for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
     float* po = part_o_of(p, run_li) + (static_cast<uint64_t>(run_slot) * p.Hq + g) * kD;
@@ -1362,7 +1367,7 @@ __device__ void consumer_alu(const LayerParams& p, const Smem& sm, uint32_t g, u
   float qh[64];  // this lane's half (64 dims) of q as f32
   float o[4] = {0.f, 0.f, 0.f, 0.f};
 
-  auto emit = [&]() {
+  auto emit = [&]() __attribute__((always_inline)) {
 #pragma unroll
     for (int sh = 1; sh <= 16; sh <<= 1) st.l0 += __shfl_xor_sync(0xffffffffu, st.l0, sh);
     float* po = part_o_of(p, run_li) + ((static_cast<uint64_t>(run_slot) * V + v) * p.Hq + g) * kD;
@@ -1454,9 +1459,16 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   // Over a slow link only a few SMs copy: a handful of them keeps the link full, and an SM whose
   // copy engine is queued up with slow loads also delays its own attention loads.
   if (p.copy_sms && blockIdx.x >= p.copy_sms) return;
-  for (uint32_t li = 0; li < p.num_layers && ok; ++li) {
+  // A link of a chain of launches must not keep its SM until the last unit of its layer's gather has
+  // landed: its successor's CTA is waiting for that SM. Once the CTA's attention is done the copy
+  // thread takes no more units (before the pass's last layer), and the copy thread of a link
+  // starts with what is left of the gather of the layer before.
+  const uint32_t li_first = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin;
+  volatile uint32_t* winding_down = sm.mq + kMqWind;
+  for (uint32_t li = li_first; li < p.li_end && ok; ++li) {
     const int32_t target = p.gather_target[li];
     if (target < 0 || p.copy_n == 0) continue;
+    const bool may_leave = p.chained && li >= p.li_begin && li + 1 < p.num_layers;
     // The target's ring slot was last read by an earlier layer of this launch: wait for its attention.
     const int32_t after = p.gather_after[li];
     if (after >= 0) {
@@ -1494,6 +1506,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     auto issue_next = [&]() -> bool {
       if (piece == pieces) {
         if (bat_i == bat_n) {
+          if (may_leave && *winding_down) return false;
           const uint32_t first = atomicAdd(ticket, batch);
           if (first >= p.copy_n) return false;
           bat_n = min(batch, p.copy_n - first);
@@ -1573,7 +1586,11 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
   extern __shared__ __align__(128) uint8_t smem_raw[];
   bool gathers = false;
   if (p.copy_n)
-    for (uint32_t li = 0; li < p.num_layers; ++li) gathers |= p.gather_target[li] >= 0;
+    for (uint32_t li = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin; li < p.li_end; ++li)
+      gathers |= p.gather_target[li] >= 0;
+  // A link of a chain of launches: the next link may start as soon as every CTA of this one has (it
+  // takes the SMs that CTAs of this link leave, and waits for nothing but flags and counters).
+  if (p.chained) ptx::launch_dependents();
   const Smem sm = carve(smem_raw, p.Hkv, gathers);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
   const uint32_t ncons = p.Hkv * blocks_per_stage(p.Hkv);  // consumer warps: blocks_per_stage per KV head
@@ -1585,7 +1602,7 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
     for (uint32_t g = 0; g < 8; ++g) sm.head_runs[g] = 0;
     for (int s = 0; s < kNC; ++s) ptx::mbar_init(ptx::smem_u32(&sm.copy_full[s]), 1);
     for (uint32_t s = 0; s < kMq; ++s) sm.mq[s] = kMqEmpty;
-    sm.mq[kMqTail] = sm.mq[kMqHead] = sm.mq[kMqDone] = 0;
+    sm.mq[kMqTail] = sm.mq[kMqHead] = sm.mq[kMqDone] = sm.mq[kMqWind] = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
@@ -1604,7 +1621,12 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
   } else if (warp == ncons) {
     producer_role<kGrouped>(p, sm);
   } else if (warp == ncons + 1) {
-    if (lane == 0) copy_role(p, sm);
+    if (lane == 0) {
+      copy_role(p, sm);
+      // Links end in order: the stream's next operation, which waits for the last link only, then
+      // finds the whole chain complete (no wait at all in a kernel that is no dependent).
+      if (p.chained) ptx::grid_dependency_wait();
+    }
   } else if (warp == ncons + 2) {
     merge_role(p, sm, false);
   }
@@ -1704,7 +1726,21 @@ cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
   void* args[] = {const_cast<LayerParams*>(&p)};
   const void* fn = layer_kernel_for(p.Hkv, p.G);
   // CTAs of a launch that spans several layers wait for one another: all of them must be resident.
-  if (p.num_layers > 1) return cudaLaunchCooperativeKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
+  if (p.li_end - p.li_begin > 1) return cudaLaunchCooperativeKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
+  if (p.chained == 2) {
+    // A later link of a chain: it may start while its predecessor still runs.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(p.ncta);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, fn, args);
+  }
   return cudaLaunchKernel(fn, dim3(p.ncta), dim3(threads), args, smem, stream);
 }
 

@@ -78,6 +78,7 @@ cudaError_t static_scratch_setup(uint32_t Hkv, uint32_t G, uint32_t ncta) {
   if (g_warmed[dev][variant]) return cudaSuccess;
   LayerParams p{};  // no blocks, no sequences, no gather: every role finds nothing to do and returns
   p.num_layers = 1;
+  p.li_end = 1;
   p.ring_slots = 1;
   p.layer_group = 1;
   p.prefetch_distance = 1;

@@ -26,6 +26,14 @@ __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// Programmatic dependent launch. launch_dependents: this CTA no longer holds back the start of the next
+// kernel in the stream (when that kernel was launched with programmatic stream serialisation; it
+// starts once every CTA of this grid has said so or exited). grid_dependency_wait: returns when the
+// preceding kernel of the stream has completed and its writes are visible (at once when this kernel
+// was not launched as such a dependent).
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Orders this thread's generic-proxy view of GLOBAL memory with its asynchronous-proxy operations
 // (bulk copies that read or wrote global memory): after an acquire that learned of another CTA's
 // bulk stores and before the bulk load that reads them; after a completed bulk store group and

@@ -668,6 +668,9 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.ring_slots = s->layer_slots;
   d.first_layer = first_layer;
   d.num_layers = num_layers;
+  d.li_begin = 0;
+  d.li_end = num_layers;
+  d.chained = 0;
   d.block_bytes = s->block_bytes;
   d.resolved = reinterpret_cast<const int32_t*>(p->dev + p->off_resolved);
   d.lens = reinterpret_cast<const uint32_t*>(p->dev + p->off_lens);
@@ -894,8 +897,23 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
       d.gather_target[l] = target[l];
       d.gather_after[l] = after[l];
     }
-    CU(s, ema::launch_layer(d, stream));
-    s->st.kernel_launches++;
+    if (s->cfg.pipeline_mode == 3) {
+      // A chain of launches, one per layer, over the one parameter block: each link starts as soon as
+      // every CTA of the link before it has started, on the SMs that link's CTAs leave, and the links
+      // order themselves through the flags and counters that order the layers of a single launch.
+      // Nothing else may be enqueued between two links.
+      d.merge_inline = 1;  // a link's CTA leaves when its merges are done: side by side, not queued
+      for (uint32_t l = 0; l < L; ++l) {
+        d.li_begin = l;
+        d.li_end = l + 1;
+        d.chained = l == 0 ? 1u : 2u;
+        CU(s, ema::launch_layer(d, stream));
+        s->st.kernel_launches++;
+      }
+    } else {
+      CU(s, ema::launch_layer(d, stream));
+      s->st.kernel_launches++;
+    }
     rc = prof_record(s, L - 1, 4, stream);  // ... and end of the last layer
     if (rc) return rc;
     rc = prof_record(s, L - 1, 3, stream);
@@ -984,7 +1002,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 2 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 1) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 3 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 1) return SLICE_EINVAL;
   // Section 4.2: slabs, layer groups, layouts.
   const uint32_t group = cfg->layer_group ? cfg->layer_group : 1u, slab = cfg->slab_blocks;
   if (cfg->layout > 2 || group > cfg->num_layers) return SLICE_EINVAL;
@@ -1756,7 +1774,8 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   const uint32_t L = s->cfg.num_layers, R = s->layer_slots, K = s->group;
   // Mode 0: one launch for the whole pass when the shape allows it, else one launch per layer.
   // (Swap-out passes run layer by layer: the write-back of a layer goes on a stream of its own.)
-  const bool step = s->cfg.pipeline_mode == 0 && s->cfg.ring_slots >= 2 && L >= 2 && L <= ema::kMaxStepLayers &&
+  const bool step = (s->cfg.pipeline_mode == 0 || s->cfg.pipeline_mode == 3) && s->cfg.ring_slots >= 2 && L >= 2 &&
+                    L <= ema::kMaxStepLayers &&
                     s->ncta <= static_cast<uint32_t>(s->num_sms) && !s->cfg.swap_out;
   const bool fused = s->cfg.pipeline_mode != 1 && s->cfg.ring_slots >= 2;
   if (fused) side = stream;
@@ -1769,7 +1788,7 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   if (dependent) {
     // Only the one-launch pass has anything to feed: with the other pipelines the caller drives the
     // layers itself and the stream already orders a layer's attention after its queries.
-    if (io_on_host || !step) return SLICE_EINVAL;
+    if (io_on_host || !step || s->cfg.pipeline_mode != 0) return SLICE_EINVAL;
     for (uint32_t i = 0; i < nseq; ++i)
       if (s->seqs[seqs[i]].len == 0) return SLICE_EINVAL;  // before the epoch moves
     if (!s->null_dev && !stream_ops_ready()) {

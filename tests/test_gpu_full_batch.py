@@ -122,14 +122,17 @@ class FullBatch:
     ("llama3_8b_decode", 9, {}),                              # four partial buffers, each reused at least once
     ("llama3_70b_decode", 6, {}),
     ("llama3_8b_decode", 5, {"prefetch_priority": 1}),        # two partial buffers, reused twice
+    ("llama3_8b_decode", 9, {"pipeline_mode": 3}),            # the same pass as a chain of one launch per layer
 ])
 def test_timed_launch_configuration_matches_oracle_in_full(name, L, kw):
     fb = FullBatch(name, L, **kw)
     per = -(-fb.pl.total_blocks // 148)
     assert per > 48                                            # merges are queued, not done in line
     st = fb.decode_passes(2)
-    assert st["kernel_launches"] <= 5                          # one launch per pass, plus the gathers of layer 0
-                                                               # (priming; refill of a slot the last layer shares)
+    per_pass = L if kw.get("pipeline_mode") == 3 else 1
+    assert st["kernel_launches"] <= 2 * per_pass + 3           # one launch per pass (per layer in a chain), plus the
+                                                               # gathers of layer 0 (priming; refill of a slot the
+                                                               # last layer shares)
     resolved, k = fb.check_tables()
     fb.check_staged_bytes(k)
     mid = max(4, L // 2) if L > 5 else 3

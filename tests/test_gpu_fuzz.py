@@ -19,7 +19,7 @@ L, HQ, HKV, D, T = 3, 8, 2, 128, 16
 LOCAL, LENT, MAXSEQ, MAXBLK = 28, 30, 6, 12
 
 
-@pytest.mark.parametrize("seed,mode", [(1, 0), (2, 1), (3, 2), (4, 0)])
+@pytest.mark.parametrize("seed,mode", [(1, 0), (2, 1), (3, 2), (4, 0), (5, 3)])
 def test_random_call_sequences_match_the_oracle(seed, mode):
     import torch
     from tests.gpu_helpers import kv_to_dev, kv_to_host, to_dev

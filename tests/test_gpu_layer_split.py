@@ -93,7 +93,7 @@ class SplitScenario:
             assert (kv_to_host(self.staging[slot, :k]) == staged[:k]).all(), slot
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
 @pytest.mark.parametrize("L,split,group", [(6, 3, 0), (8, 4, 2), (5, 1, 0), (5, 4, 0)])
 def test_layer_split_matches_oracle_in_every_pipeline(mode, L, split, group):
     sp = SplitScenario(L, split, 11, group=group, pipeline_mode=mode, decode_ctas=12)

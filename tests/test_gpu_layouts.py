@@ -68,7 +68,7 @@ def test_per_layer_calls_in_every_layout(layout, slab, group):
         assert np.abs(lse.double().cpu().numpy() - ref_lse).max() <= 1e-3
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
 @pytest.mark.parametrize("layout,slab,group,layers,ring", [(2, 10, 4, 8, 2), (1, 10, 2, 8, 2), (0, 4, 3, 7, 2), (2, 4, 2, 6, 3),
                                                            (2, 10, 4, 12, 2), (1, 5, 4, 8, 1)])
 def test_pipelines_fetch_one_group_ahead(mode, layout, slab, group, layers, ring):

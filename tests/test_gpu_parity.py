@@ -123,7 +123,7 @@ def test_ranges_longer_than_the_cached_table_and_multi_layer_pass():
             assert attention_close(got[layer], ref, ATOL, RTOL)[0]
 
 
-@pytest.mark.parametrize("ring,mode", [(1, 0), (1, 1), (3, 0), (3, 1), (3, 2), (4, 0)])
+@pytest.mark.parametrize("ring,mode", [(1, 0), (1, 1), (3, 0), (3, 1), (3, 2), (4, 0), (1, 3), (3, 3), (4, 3)])
 def test_other_ring_depths(ring, mode):
     """A ring of one slot cannot overlap anything (every prefetch waits for the attention that reads
     the slot); rings of three and four slots change which layer a slot holds and which attention a
@@ -586,10 +586,12 @@ def test_copy_blocks_matches_index_select(kind, n, bb):
     assert torch.equal(dst2, src[src_idx.long()])
 
 
-@pytest.mark.parametrize("mode,layers,static", [(0, 5, 0), (0, 4, 1), (0, 4, 0), (1, 5, 0), (1, 4, 1), (2, 5, 0), (2, 4, 1)])
+@pytest.mark.parametrize("mode,layers,static", [(0, 5, 0), (0, 4, 1), (0, 4, 0), (1, 5, 0), (1, 4, 1), (2, 5, 0), (2, 4, 1),
+                                                (3, 5, 0), (3, 4, 1), (3, 9, 0)])
 def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, static):
-    """All three pipelines (0: one persistent launch per pass; 1: two streams with events; 2: one
-    fused launch per layer), odd and even layer counts on a ring of two, three passes each."""
+    """All four pipelines (0: one persistent launch per pass; 1: two streams with events; 2: one
+    fused launch per layer; 3: a chain of launches, one per layer, each starting while the one before
+    it runs), odd and even layer counts on a ring of two, three passes each."""
     wl = synth.Workload("pipe", layers, 32, 8, 7, 100, 1200, 0.4)
     sc = Scenario(wl, 9)
     g = _gpu(sc, flags=B.FLAG_PROFILE | B.FLAG_TRACE, pipeline_mode=mode, static_split=static, decode_ctas=12)
@@ -608,8 +610,8 @@ def test_decode_step_pipeline_matches_oracle_for_every_layer(mode, layers, stati
         ok, max_abs, _ = attention_close(out[layer], ref, ATOL, RTOL)
         assert ok, (layer, max_abs)
     times = g.s.slice_layer_times()
-    if mode == 0:
-        assert np.isfinite(times[0, 2]) and times[-1, 3] >= times[0, 2]      # one launch spans the pass
+    if mode in (0, 3):
+        assert np.isfinite(times[0, 2]) and times[-1, 3] >= times[0, 2]      # one launch (or chain) spans the pass
     else:
         assert np.isfinite(times[:, 2:]).all() and (times[:, 3] >= times[:, 2]).all()
     trace = g.s.slice_cta_trace(0)

@@ -23,7 +23,7 @@ def _built():
     build_mod.build()
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
 @pytest.mark.parametrize("ring", [2, 3])
 def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, ring):
     from tests.gpu_helpers import GpuScenario, kv_to_host, to_dev

@@ -225,7 +225,7 @@ def test_decode_step_plans_prefetches_for_any_ring_depth(ring, calls):
     """Tables-only mode: two passes over 5 layers succeed for every pipeline and ring depth (a ring
     of one slot prefetches after the attention that reads the slot), and the number of prefetches
     follows from which layers are still staged when the second pass starts."""
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 3):
         s = B.Slice(5, 4, 64, 64, 64, lent_blocks_physical=64, ring_slots=ring, max_seqs=8, max_blocks_per_seq=64,
                     flags=B.FLAG_NULL_DEVICE, pipeline_mode=mode)
         for i in range(3):
@@ -495,7 +495,7 @@ def test_decode_step_prefetches_one_layer_group_ahead(group, ring, layers, first
     seven layers: 0,1 then 2..6, layer 6 displacing layer 0, which is fetched again once layer 6 has
     been attended to = 8; later passes fetch only those two.
     (4,1,8): a ring of one group: every fetch follows the attention that frees its slot: 12, later 8."""
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 3):
         s = B.Slice(layers, 4, 64, 64, 64, lent_blocks_physical=64, ring_slots=ring, max_seqs=8, max_blocks_per_seq=64,
                     flags=B.FLAG_NULL_DEVICE, pipeline_mode=mode, layer_group=group)
         for i in range(3):
