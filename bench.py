@@ -569,7 +569,7 @@ def run_ours(args, wl):
         achieved = algo / kernel_s / 1e9
         combined = step_bytes * args.steps / t / 1e9
         name = {0: "slice_layer_kernel (one launch per pass: attention + gather of every layer)",
-                1: "slice_layer_kernel (attention only; gather in copy_blocks_vector on a second stream)",
+                1: "slice_layer_kernel (attention only; gather in copy_blocks_bulk<6> on a second stream, sharing the SMs)",
                 2: "slice_layer_kernel (one launch per layer: attention + gather of the next layer)",
                 3: "slice_layer_kernel (a chain of launches, one per layer, each starting while the one before it runs)"
                 }[args.pipeline_mode]
@@ -785,7 +785,7 @@ def run_ours(args, wl):
                                                 "achieved_gbs": attn_bytes_layer / (iso_us * 1e-6) / 1e9,
                                                 "frac": attn_bytes_layer / (iso_us * 1e-6) / 1e9 / peak,
                                                 "note": "one launch per layer, prefetch serialised before it"},
-                "copy_blocks_vector_gather": {"us_per_launch": iso_pref_us, "algorithmic_bytes": pref_bytes_layer,
+                "copy_blocks_bulk_gather": {"us_per_launch": iso_pref_us, "kernel": "copy_blocks_bulk<6> (6 x 16 KB ring per CTA, one CTA per SM)", "algorithmic_bytes": pref_bytes_layer,
                                               "achieved_gbs": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9,
                                               "frac": pref_bytes_layer / (iso_pref_us * 1e-6) / 1e9 / peak}}
             del ws

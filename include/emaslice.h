@@ -111,7 +111,12 @@ typedef struct {
                                        ids >= lent_blocks are skipped at creation                */
   uint32_t decode_ctas;           /* 0 = one per SM; CTAs of the layer (attention) kernel        */
   uint32_t copy_ctas;             /* 0 = default; CTAs of the stand-alone gather / migration kernel */
-  uint32_t copy_kind;             /* 0 = default, 1 = vector load/store kernel, 2 = bulk-copy ring */
+  uint32_t copy_kind;             /* stand-alone gather, write-back and migration kernel: 0 = default (gather
+                                     and write-back: 3; migration: 2), 1 = vector load/store kernel, 2 =
+                                     bulk-copy ring of 8 x 16 KB per CTA (fastest alone), 3 = the same
+                                     with 6 stages: a CTA of it fits on an SM beside a CTA of the
+                                     attention kernel, so a gather on a second stream runs WHILE the
+                                     attention does instead of taking turns with it                 */
   uint32_t pipeline_mode;         /* slice_decode_step: 0 = one persistent launch for the whole pass
                                      (attention of layer l overlapped with the gather of layer l+1,
                                      soft layer boundaries; falls back to 2 when the shape does not
@@ -478,7 +483,8 @@ int slice_cta_trace(slice_t* s, int32_t which, uint64_t* out, uint64_t cap_entri
 /* Low-level copy used by the prefetch microbenchmark: n blocks of block_bytes (a multiple of 16
  * bytes, 16-byte aligned addresses) are copied dst_base + dst_idx[i]*block_bytes <-
  * src_base + src_idx[i]*block_bytes. Index arrays and bases are device pointers; dst_idx or src_idx
- * may be NULL for the identity. kind: 0 default, 1 vector load/store, 2 bulk-copy ring. */
+ * may be NULL for the identity. kind: 0 default (vector), 1 vector load/store, 2 bulk-copy ring,
+ * 3 bulk-copy ring of 6 stages. */
 int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_base, const int32_t* src_idx,
                       uint32_t n, uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream);
 

@@ -66,8 +66,9 @@ __global__ void __launch_bounds__(kVecThreads) copy_blocks_vector(const CopyDesc
 // Bulk ring: stage = 16 KB; kLoadsAhead loads in flight, the remaining stages drain as stores.
 // Measured on 100 000 blocks: 8 stages with 4 loads ahead 6.40 TB/s; 12 with 8 ahead 6.00; 6 with 3
 // ahead 6.04; 32 KB stages 6.27-6.35: more bytes in flight only queue in the memory system.
+// With 6 stages (kCopyBulkShared) a CTA needs 96 KB and fits beside a CTA of the layer kernel that
+// only attends, so that a gather on a second stream really runs while the attention does.
 constexpr uint32_t kChunk = 16384;
-constexpr int kStages = 8;
 constexpr int kLoadsAhead = 4;
 
 struct ChunkRef {
@@ -90,6 +91,7 @@ __device__ __forceinline__ ChunkRef chunk_ref(const CopyDesc& d, uint64_t w, uin
   return c;
 }
 
+template <int kStages>
 __global__ void __launch_bounds__(32) copy_blocks_bulk(const CopyDesc d) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t bars[kStages];
@@ -105,6 +107,7 @@ __global__ void __launch_bounds__(32) copy_blocks_bulk(const CopyDesc d) {
   ptx::fence_barrier_init();
   const uint32_t base = ptx::smem_u32(smem);
   const uint64_t pol = ptx::policy_evict_first();
+  const uint64_t pol_keep = ptx::policy_evict_last();  // the shared form gathers: staged blocks are read within a layer's time
   uint32_t issued = 0;
   for (; issued < cnt && issued < static_cast<uint32_t>(kLoadsAhead); ++issued) {
     ChunkRef c = chunk_ref(d, w0 + issued, pieces);
@@ -119,7 +122,10 @@ __global__ void __launch_bounds__(32) copy_blocks_bulk(const CopyDesc d) {
     ok = ptx::mbar_wait(ptx::smem_u32(&bars[st]), (j / kStages) & 1u, d.status, kDevTimeout);
     if (!ok) break;
     ChunkRef c = chunk_ref(d, w0 + j, pieces);
-    ptx::bulk_s2g(c.dst, base + st * kChunk, c.bytes);
+    if constexpr (kStages == 6)
+      ptx::bulk_s2g_hint(c.dst, base + st * kChunk, c.bytes, pol_keep);
+    else
+      ptx::bulk_s2g(c.dst, base + st * kChunk, c.bytes);
     ptx::bulk_commit();
     if (issued < cnt) {
       // The stage about to be refilled was last read by the store of chunk issued - kStages.
@@ -144,15 +150,22 @@ __global__ void __launch_bounds__(32) copy_blocks_bulk(const CopyDesc d) {
 cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num_sms, cudaStream_t stream) {
   if (d.n == 0 || d.nlayers == 0) return cudaSuccess;
   if (kind == kCopyDefault) kind = kCopyVector;
-  if (kind == kCopyBulk) {
+  if (kind == kCopyBulk || kind == kCopyBulkShared) {
     static bool attr_set[64] = {};  // the attribute is a property of the function on one device
-    const size_t smem = static_cast<size_t>(kStages) * kChunk;
+    const int stages = kind == kCopyBulk ? 8 : 6;
+    const size_t smem = static_cast<size_t>(stages) * kChunk;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-      e = cudaFuncSetAttribute(copy_blocks_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      e = cudaFuncSetAttribute(copy_blocks_bulk<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * static_cast<int>(kChunk));
+      if (e != cudaSuccess) return e;
+      e = cudaFuncSetAttribute(copy_blocks_bulk<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, 6 * static_cast<int>(kChunk));
+      if (e != cudaSuccess) return e;
+      // Two kernels share an SM only under one split of its L1 / shared memory: both ask for the
+      // largest shared part (as does the layer kernel), whatever they need themselves.
+      e = cudaFuncSetAttribute(copy_blocks_bulk<6>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
       if (e != cudaSuccess) return e;
       attr_set[dev] = true;
     }
@@ -160,7 +173,10 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
     const uint64_t total = static_cast<uint64_t>(d.n) * d.nlayers * pieces;
     uint64_t grid = ctas ? ctas : static_cast<uint64_t>(num_sms);
     if (grid > total) grid = total;
-    copy_blocks_bulk<<<static_cast<unsigned>(grid), 32, smem, stream>>>(d);
+    if (kind == kCopyBulk)
+      copy_blocks_bulk<8><<<static_cast<unsigned>(grid), 32, smem, stream>>>(d);
+    else
+      copy_blocks_bulk<6><<<static_cast<unsigned>(grid), 32, smem, stream>>>(d);
   } else {
     const uint64_t vecs = d.block_bytes >> 4;
     const uint64_t pieces = (vecs + kPieceVecs - 1) / kPieceVecs;

@@ -40,7 +40,9 @@ struct CopyDesc {
   unsigned long long* trace;  // optional [grid][2] start/end %globaltimer per CTA (profiling)
 };
 
-enum CopyKind : uint32_t { kCopyDefault = 0, kCopyVector = 1, kCopyBulk = 2 };
+// kCopyBulkShared: the bulk-copy ring with 6 instead of 8 stages (96 KB), small enough for a CTA of it
+// to share an SM with a CTA of the layer kernel that gathers nothing itself.
+enum CopyKind : uint32_t { kCopyDefault = 0, kCopyVector = 1, kCopyBulk = 2, kCopyBulkShared = 3 };
 
 // Launches one copy kernel on `stream`. ctas == 0 picks a default grid. Returns the CUDA error.
 cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num_sms, cudaStream_t stream);

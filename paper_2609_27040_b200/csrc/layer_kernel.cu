@@ -174,13 +174,26 @@ __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
+// Attention stages of a launch: beside a copy ring, or alone (the launch gathers nothing).
+__host__ __device__ constexpr uint32_t attention_stages(uint32_t Hkv, bool gathers) {
+  return blocks_per_stage(Hkv) > 1 ? (gathers ? kGroupedStages : 3u) : (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
+}
+// A launch that gathers nothing has no copy ring: the bookkeeping follows the attention ring, and with
+// 3 to 8 KV heads the CTA takes 100 KB, which leaves room on its SM for a CTA of the shared form of
+// the gather kernel (a gather on a second stream then really runs beside the attention).
+__host__ __device__ constexpr size_t smem_needed(uint32_t Hkv, bool gathers) {
+  return kRingAlign + static_cast<size_t>(attention_stages(Hkv, gathers)) * stage_bytes(Hkv) +
+         (gathers ? static_cast<size_t>(kNC) * kCopyChunk : 0) + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes +
+         kOwnBytes;
+}
+
 __device__ __forceinline__ Smem carve(uint8_t* base, uint32_t Hkv, bool gathers) {
   Smem s;
-  s.na = blocks_per_stage(Hkv) > 1 ? (gathers ? kGroupedStages : 3u) : (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
+  s.na = attention_stages(Hkv, gathers);
   base += (kRingAlign - (ptx::smem_u32(base) & (kRingAlign - 1))) & (kRingAlign - 1);
   s.att_ring = base;
-  s.copy_ring = base + static_cast<size_t>(blocks_per_stage(Hkv) > 1 ? kGroupedStages : kNAFused * ring_scale(Hkv)) * stage_bytes(Hkv);
-  uint8_t* p = s.copy_ring + static_cast<size_t>(kNC) * kCopyChunk;
+  s.copy_ring = base + static_cast<size_t>(s.na) * stage_bytes(Hkv);
+  uint8_t* p = s.copy_ring + (gathers ? static_cast<size_t>(kNC) * kCopyChunk : 0);
   s.att_full = reinterpret_cast<uint64_t*>(p);
   s.att_empty = s.att_full + kNAMax;
   s.copy_full = s.att_empty + kNAMax;
@@ -1716,12 +1729,21 @@ cudaError_t layer_setup() {
     for (uint32_t G : {1u, 2u}) {
       cudaError_t e = cudaFuncSetAttribute(layer_kernel_for(Hkv, G), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e != cudaSuccess) return e;
+      // A launch that gathers nothing takes 100 KB; the SM keeps its largest shared-memory split all
+      // the same, so that a CTA of the gather kernel can join it (and leave) without the split changing.
+      e = cudaFuncSetAttribute(layer_kernel_for(Hkv, G), cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+      if (e != cudaSuccess) return e;
     }
   return cudaSuccess;
 }
 
 cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
-  const size_t smem = layer_smem_bytes(p.Hkv);
+  // The same test as in the kernel: does any layer this launch works on gather?
+  bool gathers = false;
+  if (p.copy_n)
+    for (uint32_t li = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin; li < p.li_end; ++li)
+      gathers |= p.gather_target[li] >= 0;
+  const size_t smem = smem_needed(p.Hkv, gathers);
   const unsigned threads = (p.Hkv * blocks_per_stage(p.Hkv) + 3) * 32;
   void* args[] = {const_cast<LayerParams*>(&p)};
   const void* fn = layer_kernel_for(p.Hkv, p.G);

@@ -622,7 +622,12 @@ int do_prefetch(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t side) {
       fill_gather(s, layer, p, d);
       if (s->trace_copy && (s->cfg.copy_ctas ? s->cfg.copy_ctas : s->num_sms * 8u) <= kTraceCopyCtas)
         d.trace = s->trace_copy + static_cast<size_t>(layer) * kTraceCopyCtas * 2;
-      const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+      // Default: the bulk-copy ring in the form that shares an SM with an attention CTA, so that a
+      // gather on a second stream runs while the attention does (the vector kernel needs no shared
+      // memory, but beside the layer kernel's 352 threads there are not the registers for its CTAs:
+      // the two took turns instead of overlapping).
+      uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+      if (kind == ema::kCopyDefault) kind = ema::kCopyBulkShared;
       CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, side));
       s->st.kernel_launches++;
     }
@@ -1001,7 +1006,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->head_dim != kHeadDim || cfg->block_tokens != kBlockTokens || cfg->dtype != 0) return SLICE_EINVAL;
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
-  if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 2) return SLICE_EINVAL;
+  if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 3) return SLICE_EINVAL;
   if (cfg->pipeline_mode > 3 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 1) return SLICE_EINVAL;
   // Section 4.2: slabs, layer groups, layouts.
   const uint32_t group = cfg->layer_group ? cfg->layer_group : 1u, slab = cfg->slab_blocks;
@@ -1722,7 +1727,8 @@ int do_writeback(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t stream) {
   d.nlayers = 1;
   d.block_bytes = s->block_bytes;
   d.status = s->dev_status;
-  const uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+  uint32_t kind = s->cfg.lent_kind == 1 ? ema::kCopyVector : s->cfg.copy_kind;
+  if (kind == ema::kCopyDefault) kind = ema::kCopyBulkShared;  // runs beside the attention, like the gather
   CU(s, ema::launch_copy(d, kind, s->cfg.copy_ctas, s->num_sms, stream));
   s->st.kernel_launches++;
   // A later prefetch into this slot (of this layer again, which reads the lent arena, or of another
@@ -2072,7 +2078,7 @@ int slice_layer_times(slice_t* s, float* out, uint32_t cap_layers) {
 
 int slice_copy_blocks(void* dst_base, const int32_t* dst_idx, const void* src_base, const int32_t* src_idx, uint32_t n,
                       uint64_t block_bytes, uint32_t kind, uint32_t ctas, void* stream) {
-  if (!dst_base || !src_base || (block_bytes & 15u) || block_bytes == 0 || kind > 2) return SLICE_EINVAL;
+  if (!dst_base || !src_base || (block_bytes & 15u) || block_bytes == 0 || kind > 3) return SLICE_EINVAL;
   if ((reinterpret_cast<uintptr_t>(dst_base) | reinterpret_cast<uintptr_t>(src_base)) & 15u) return SLICE_EINVAL;
   static int sms_of[64] = {};  // per device
   int dev = 0;

@@ -63,7 +63,7 @@ def copy_sweep(args):
         moved = 2 * n * BLOCK_BYTES
         use_flush = flush if moved < 4 * L2_BYTES else None
         reps = 20 if n <= 100_000 else 5
-        for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk")):
+        for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk"), (3, "copy_blocks_bulk, 6 stages")):
             for ctas in args.ctas:
                 def run():
                     assert B.slice_copy_blocks(dst, pos, src, idx, n, BLOCK_BYTES, kind, ctas, stream) == 0
@@ -308,7 +308,7 @@ def transfer_size_sweep(args):
             rng = np.random.default_rng(c)
             idx = torch.from_numpy(rng.permutation(2 * total // c)[:n].astype(np.int32)).cuda()
             pos = torch.arange(n, dtype=torch.int32, device="cuda")
-            for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk")):
+            for kind, name in ((1, "copy_blocks_vector"), (2, "copy_blocks_bulk"), (3, "copy_blocks_bulk, 6 stages")):
                 for ctas in ((0,) if link == "hbm" else (8, 0)):
                     def run():
                         assert B.slice_copy_blocks(dst, pos, arena, idx, n, c, kind, ctas, stream) == 0
