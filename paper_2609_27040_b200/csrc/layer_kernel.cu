@@ -151,9 +151,9 @@ static_assert(kNAFused * 32768 + kNC * 16384 >= kNAAlone * 32768, "the deeper ri
 // planes of V = 8 / Hkv consecutive blocks of a unit, copied by V lanes of the producer at once, and
 // every KV head has V consumer warps, warp v taking block v of each group of V with a softmax state
 // and a partial of its own (the merge adds them up like any other partials).
-// Measured (64 sequences of 2k..8k tokens, nothing lent, KV read rate): 1 KV head 2.08 -> 3.2 TB/s,
-// 2 KV heads 4.17 -> 4.7; with 4 KV heads (16 KB planes) it is slower than one block per stage
-// (6.5 -> 5.9), so 3 and 4 KV heads keep one block per stage and twice as many stages instead.
+// Measured (64 sequences of 2k..8k tokens, nothing lent, KV read rate): 1 KV head 2.08 -> 4.46 TB/s,
+// 2 KV heads 4.17 -> 6.02, 4 KV heads 6.49 -> 6.79 (the same as one block per stage when the launch
+// also gathers); 3 KV heads (8 is no multiple) keep one block per stage and twice as many stages.
 __host__ __device__ constexpr uint32_t blocks_per_stage(uint32_t Hkv) { return partials_per_slot(Hkv); }
 // A shared stage holds the V blocks whole (K plane and V plane are neighbours in memory: one request
 // of 8 or 16 KB per block instead of two of 4 or 8 KB), 64 KB per stage, two stages.
