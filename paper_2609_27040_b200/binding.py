@@ -21,7 +21,7 @@ PREEMPT_OOM, PREEMPT_RECLAIM = 1, 2
 TIER_AUTO, TIER_LOCAL, TIER_LENT = 0, 1, 2
 FLAG_PROFILE, FLAG_TRACE, FLAG_NULL_DEVICE = 1, 2, 4
 FLAG_TEST_WITHHOLD_Q, FLAG_TEST_FAIL_COPY = 8, 16      # test hooks (see include/emaslice.h)
-COPY_DEFAULT, COPY_VECTOR, COPY_BULK = 0, 1, 2
+COPY_DEFAULT, COPY_VECTOR, COPY_BULK, COPY_BULK_SHARED = 0, 1, 2, 3
 LAYOUT_LAYER_MAJOR, LAYOUT_SLAB_MAJOR, LAYOUT_LAYER_GROUP_MAJOR = 0, 1, 2
 TAKE_ALL = 0xFFFFFFFF
 

@@ -80,7 +80,7 @@ def test_prefetch_and_decode_match_oracle(wl, seed):
         _check_layer(sc, g, 0, seqs=[sc.seq_ids[2], sc.seq_ids[0]])
 
 
-@pytest.mark.parametrize("kind", [B.COPY_VECTOR, B.COPY_BULK])
+@pytest.mark.parametrize("kind", [B.COPY_VECTOR, B.COPY_BULK, B.COPY_BULK_SHARED])
 def test_both_gather_kernels_are_bit_exact(kind):
     sc = Scenario(GQA4, 5)
     g = _gpu(sc, copy_kind=kind)
@@ -566,7 +566,7 @@ def test_writeback_round_trip():
     assert g.s.slice_writeback_layer(0, sc.seq_ids[:2], g.main) == B.ESTALE
 
 
-@pytest.mark.parametrize("kind", [B.COPY_VECTOR, B.COPY_BULK])
+@pytest.mark.parametrize("kind", [B.COPY_VECTOR, B.COPY_BULK, B.COPY_BULK_SHARED])
 @pytest.mark.parametrize("n,bb", [(1, 65536), (37, 65536), (300, 4096), (5, 48), (2000, 65536)])
 def test_copy_blocks_matches_index_select(kind, n, bb):
     gen = torch.Generator(device="cuda").manual_seed(n + bb)

@@ -54,6 +54,11 @@ def test_create_rejects_bad_configs():
         _null_slice(1, 8, 4, 4, 4, 4, 4, 4, lo=np.array([0, 0, 1, 2], np.uint32))   # not a permutation
     with pytest.raises(B.SliceError):
         B.Slice(1, 8, 4, 4, 4)                                     # device mode needs arenas
+    for kw in ({"pipeline_mode": 4}, {"copy_kind": 4}, {"prefetch_priority": 2}, {"swap_out": 2}):
+        with pytest.raises(B.SliceError):
+            B.Slice(2, 8, 4, 4, 4, max_seqs=4, max_blocks_per_seq=4, flags=B.FLAG_NULL_DEVICE, **kw)
+    for kw in ({"pipeline_mode": 3}, {"copy_kind": 3}):                # the chain of launches; the SM-sharing gather
+        B.Slice(2, 8, 4, 4, 4, max_seqs=4, max_blocks_per_seq=4, flags=B.FLAG_NULL_DEVICE, **kw).close()
 
 
 def _same_state(s: B.Slice, o: oracle.OracleSlice, live):
@@ -180,7 +185,7 @@ def test_layer_dependent_pass_bookkeeping_in_tables_only_mode():
     assert s.slice_set_seq_len(0, 0) == B.OK
     assert s.slice_step_begin([0], None, 8, 1.0, None) == B.EINVAL    # empty sequence
     s.close()
-    for kw in ({"pipeline_mode": 1}, {"pipeline_mode": 2}, {"ring_slots": 1}):
+    for kw in ({"pipeline_mode": 1}, {"pipeline_mode": 2}, {"pipeline_mode": 3}, {"ring_slots": 1}):
         s = B.Slice(4, 8, 8, 8, 4, lent_blocks_physical=8, max_seqs=4, max_blocks_per_seq=8, flags=B.FLAG_NULL_DEVICE, **kw)
         s.slice_alloc_blocks(0, 2, B.TIER_LENT)
         s.slice_set_seq_len(0, 20)
