@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--no-wrap", action="store_true", help="do not prefetch layer 0 of the next pass")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (debugging)")
+    ap.add_argument("--kv-heads", type=int, default=0,
+                    help="override the KV heads, same query heads per KV head (profiling the few-KV-head kernel variants)")
     args = ap.parse_args()
     # The reference arm really spends what it reports (about four seconds per step): fewer steps by default.
     if args.steps is None:
@@ -837,9 +839,11 @@ def main():
         run_prefetch_microbench(args)
         return
     wl = synth.WORKLOADS[args.workload]
-    if args.layers or args.batch:
+    if args.layers or args.batch or args.kv_heads:
         import dataclasses
-        wl = dataclasses.replace(wl, num_layers=args.layers or wl.num_layers, batch=args.batch or wl.batch)
+        hkv = args.kv_heads or wl.num_kv_heads
+        wl = dataclasses.replace(wl, num_layers=args.layers or wl.num_layers, batch=args.batch or wl.batch, num_kv_heads=hkv,
+                                 num_q_heads=wl.num_q_heads // wl.num_kv_heads * hkv)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
