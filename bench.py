@@ -128,7 +128,7 @@ class DeviceWorkload:
         self.side = torch.cuda.Stream(priority=-1)
         torch.cuda.synchronize()
         self.max_blocks = int(max(len(h) for h in pl.hints)) + 4
-        self.s = B.Slice(wl.num_layers, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, pl.staging_blocks,
+        self.s = B.Slice(wl.num_layers, wl.num_kv_heads, pl.local_blocks, pl.lent_blocks, max(pl.staging_blocks, 1),
                          local=self.local, lent=self.lent, staging=self.staging, ring_slots=wl.ring_slots,
                          max_seqs=wl.batch, max_blocks_per_seq=self.max_blocks, flags=flags,
                          local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order,
@@ -718,6 +718,77 @@ def run_ours(args, wl):
                     torch.cuda.empty_cache()
                 except RuntimeError as err:      # an ablation must not cost the bench line
                     abl[label] = {"error": str(err)}
+                    torch.cuda.synchronize()
+                    torch.cuda.empty_cache()
+            # Performance transparency (Sections 2.3, 4): a layer's lent data comes in during the latency
+            # window before the layer is used. A decoder leaves such a window by itself: between out[l]
+            # and q[l+1] lie the projections and the MLP of the block. Here a spinning kernel of the
+            # caller stands for them (window_us per layer, on an SM the pass leaves free), and the time
+            # from a layer's queries to its output is compared with the same batch with nothing lent.
+            if args.pipeline_mode == 0 and wl.lent_fraction > 0:
+                try:
+                    import dataclasses
+                    windows_us = (0.0, 50.0, 100.0, 150.0)
+                    props = torch.cuda.get_device_properties(0)
+                    sms = props.multi_processor_count
+                    cycles_per_us = getattr(props, "clock_rate", 1965000) * 1e-3                 # SM cycles
+                    res = {}
+                    for name, wlx in (("lent", wl), ("all_local", dataclasses.replace(wl, lent_fraction=0.0))):
+                        wa = DeviceWorkload(wlx, args.seed, flags=B.FLAG_TRACE, pipeline_mode=0, **{**kw, "decode_ctas": sms - 1})
+                        X = torch.zeros((L + 1,) + tuple(wa.q.shape[1:]), device="cuda", dtype=torch.bfloat16)
+                        X[0].copy_(wa.q[0])
+                        caller = torch.cuda.Stream()
+                        with torch.cuda.stream(caller):
+                            torch.cuda._sleep(1000)                 # loads the spinning kernel before any pass runs
+                        torch.cuda.synchronize()
+
+                        def windowed_step(spin):
+                            rc = wa.s.slice_step_begin(wa.seqs, X[:L], wl.num_q_heads, wa.scale, X[1:], wrap, wa.main)
+                            if rc != 0:
+                                raise RuntimeError(f"slice_step_begin: {B.slice_strerror(rc)}")
+                            assert wa.s.slice_step_submit_q(0, caller) == 0
+                            for l in range(L - 1):
+                                assert wa.s.slice_step_wait_out(l, caller) == 0
+                                if spin:
+                                    with torch.cuda.stream(caller):
+                                        torch.cuda._sleep(spin)
+                                assert wa.s.slice_step_submit_q(l + 1, caller) == 0
+
+                        for w_us in windows_us:
+                            spin = int(w_us * cycles_per_us)
+                            for _ in range(2):
+                                windowed_step(spin)
+                            torch.cuda.synchronize()
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            n_w = max(3, reps // 2)
+                            e0.record(wa.main)
+                            for _ in range(n_w):
+                                windowed_step(spin)
+                            e1.record(wa.main)
+                            torch.cuda.synchronize()
+                            if wa.s.slice_stats()["device_status"] != 0:
+                                raise RuntimeError("windowed layer-dependent pass: a bounded device wait expired")
+                            tr = wa.s.slice_cta_trace(0).astype(np.float64)[:, :sms - 1]
+                            seen = np.where(tr[:, :, 7] > 0, tr[:, :, 7], np.inf).min(axis=1)  # first CTA to have the layer's q
+                            done = tr[:, :, 5].max(axis=1)                                       # last CTA to finish its last run
+                            res[(name, w_us)] = {"ms_per_step": e0.elapsed_time(e1) / n_w,
+                                                 "q_to_last_block_us_per_layer": float(np.mean((done - seen)[1:-1]) / 1e3),
+                                                 "stall_us_per_layer": float((tr[1:, :, 1] / 1e3).mean())}
+                        del wa, X
+                        torch.cuda.empty_cache()
+                    abl["transparency_with_a_window"] = {
+                        "decode_ctas": sms - 1, "lent_fraction": wl.lent_fraction,
+                        "windows": [{"window_us_per_layer": w_us, "lent": res[("lent", w_us)], "all_local": res[("all_local", w_us)],
+                                     "layer_time_ratio_lent_over_all_local":
+                                         res[("lent", w_us)]["q_to_last_block_us_per_layer"] / res[("all_local", w_us)]["q_to_last_block_us_per_layer"],
+                                     "step_time_ratio_lent_over_all_local":
+                                         res[("lent", w_us)]["ms_per_step"] / res[("all_local", w_us)]["ms_per_step"]} for w_us in windows_us],
+                        "note": "slice_step_begin with a spinning kernel of the caller between out[l] and q[l+1] (the rest of a "
+                                "decoder block); q_to_last_block = from the first CTA seeing a layer's queries to the last CTA "
+                                "finishing its last run of the layer (device timer, mean over the inner layers); a ratio of 1 "
+                                "means the lent part of the KV cost the layer nothing: the prefetch fitted in the window"}
+                except RuntimeError as err:
+                    abl["transparency_with_a_window"] = {"error": str(err)}
                     torch.cuda.synchronize()
                     torch.cuda.empty_cache()
             ws = DeviceWorkload(wl, args.seed, flags=B.FLAG_PROFILE, pipeline_mode=1, **kw)
