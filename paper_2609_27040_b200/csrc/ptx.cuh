@@ -1,5 +1,5 @@
 // ptx.cuh — thin inline-PTX wrappers for sm_100a: mbarriers, bulk asynchronous copies (TMA,
-// untiled, never the cluster-multicast form), ldmatrix / movmatrix / mma.sync fragments.
+// untiled, always to the issuing CTA's own shared memory), ldmatrix / movmatrix / mma.sync fragments.
 #pragma once
 
 #include <cuda_runtime.h>
