@@ -393,10 +393,11 @@ int slice_writeback_layer(slice_t* s, uint32_t layer, const int32_t* seqs, uint3
 
 /* One pass of the whole path over a batch: for every layer, the prefetch of layer l+1 overlapped
  * with the attention of layer l (cyclic: the last layer's attention overlaps the prefetch of layer 0
- * for the next pass when wrap_prefetch != 0). With pipeline_mode 0 or 2 and a ring of at least two
+ * for the next pass when wrap_prefetch != 0). With pipeline_mode 0, 2 or 3 and a ring of at least two
  * slots both run inside the same kernel on `stream` (side_stream is not used): one launch for the
- * whole pass (mode 0) or one per layer (mode 2); with pipeline_mode 1 the gather kernel runs on
- * side_stream and the attention kernel on stream, ordered by events.
+ * whole pass (mode 0) or one per layer (mode 2; mode 3, in which the launches overlap); with
+ * pipeline_mode 1 the gather kernel runs on side_stream and the attention kernel on stream, ordered
+ * by events, the two sharing the SMs.
  *   q, out: [num_layers][nseq][num_q_heads][128] bf16; device pointers when io_on_host == 0.
  *   With io_on_host != 0 they are host pointers. Pageable memory: q is copied to the device and out
  *   back to the host on `stream`, inside the call's enqueued work, through device buffers the
