@@ -315,6 +315,20 @@ def test_group_sizes_that_are_not_powers_of_two(hq, hkv):
     _step_matches_oracle(sc, g, passes=1)
 
 
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (32, 4), (2, 2), (16, 2), (1, 1), (8, 1)])
+@pytest.mark.parametrize("mode", [0, 3])
+def test_few_kv_heads_with_the_smallest_and_the_largest_group(hq, hkv, mode):
+    """1, 2 and 4 KV heads run the kernel variants in which several whole blocks share a stage and
+    every KV head has 8 / Hkv consumer warps: with one query head per KV head (f32 tiles) and with
+    eight (all columns of the tensor-core tile), ragged lengths, per-layer calls and whole passes."""
+    wl = synth.Workload("fewkv", 4, hq, hkv, 6, 1, 900, 0.4)
+    sc = Scenario(wl, 41 + hq)
+    g = _gpu(sc, decode_ctas=16, pipeline_mode=mode)
+    for layer in range(sc.L):
+        _check_layer(sc, g, layer)
+    _step_matches_oracle(sc, g, passes=2)
+
+
 def test_nan_poisoned_tails_do_not_leak_on_gpu():
     for wl in (WL1, GQA4):
         sc = Scenario(wl, 4, poison=True)
