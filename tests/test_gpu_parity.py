@@ -185,7 +185,7 @@ def test_decode_step_corner_shapes(case):
 
 
 @pytest.mark.parametrize("case", ["split_inline", "shared_queue", "split_queue", "static_long"])
-@pytest.mark.parametrize("mode", [0, 2])
+@pytest.mark.parametrize("mode", [0, 2, 3])
 def test_few_long_sequences_share_their_merges(case, mode):
     """A long sequence is cut into many partials; its merges are published for every CTA's merge
     warp (one query head at a time from 48 partials up) instead of being done by the CTA that
