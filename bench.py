@@ -661,11 +661,8 @@ def run_ours(args, wl):
             # A second form leaves 8 SMs free and has a kernel of the caller (an elementwise negation)
             # compute q[l+1] from out[l] on them.
             for label, alias, prio in ((("layer_dependent_q", True, args.prefetch_priority),
-                                        ("layer_dependent_q_prefetch_priority", True, 1),
                                         ("layer_dependent_q_caller_kernel", False, args.prefetch_priority))
                                        if args.pipeline_mode == 0 else ()):
-                if label == "layer_dependent_q_prefetch_priority" and args.prefetch_priority:
-                    continue
                 kwa = {**kw, "prefetch_priority": prio}
                 if not alias:
                     kwa["decode_ctas"] = max(1, torch.cuda.get_device_properties(0).multi_processor_count - 8)
@@ -834,8 +831,7 @@ def run_ours(args, wl):
                     return (h["dram_bytes"] if h["dram_bytes"] is not None else h["algorithmic_bytes"]) >= 0.70
 
                 prio_of = {"lock_step_stealing": 0, "prefetch_priority": 1, "prefetch_priority_lock_step": 1,
-                           "layer_dependent_q": -1, "layer_dependent_q_caller_kernel": -1,
-                           "layer_dependent_q_prefetch_priority": -1}     # DRAM traffic of these modes: not captured
+                           "layer_dependent_q": -1, "layer_dependent_q_caller_kernel": -1}  # DRAM traffic of these: not captured
                 ok = [k for k, v in alts.items() if frac(v) < 0.05 and gate(v["hbm_gbs_combined"], prio_of.get(k, 0))]
                 pick = max(ok, key=lambda k: alts[k]["tokens_per_s"]) if ok else min(alts, key=lambda k: frac(alts[k]))
                 default_stall = extra["stall_frac_of_layer"]

@@ -151,10 +151,8 @@ typedef struct {
                                      the CTAs stay within a layer of one another, the prefetch is
                                      far ahead of all of them, attention (almost) never waits for
                                      it, staged blocks come from DRAM and the pass is slower.
-                                     Layer-dependent passes (slice_step_begin): 0 = the gather fills a
-                                     slot in reverse, what a CTA reads first landing last (still in
-                                     L2 when the layer starts, which may wait for it); 1 = in
-                                     reading order: no wait, slower                              */
+                                     (Layer-dependent passes, slice_step_begin, have a hard boundary
+                                     after every layer: the setting changes little there)          */
   uint32_t slab_blocks;           /* Section 4.2.1: 0 = blocks are handed out one by one from free stacks
                                      (the seeded orders); S > 0 = slab allocator: the ids of each part
                                      form slabs of S consecutive ids (the paper's default is 10,

@@ -52,7 +52,7 @@ struct Plan {
   uint32_t slots = 0, slots_static = 0;  // partial slots with / without work stealing
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
-  size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_copy_order_rev = 0, off_blk_off = 0, off_slot_base = 0,
+  size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_blk_off = 0, off_slot_base = 0,
          off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
   std::vector<int32_t> resolved_ids;  // resolved table in block ids (the device copy holds physical indices)
@@ -300,7 +300,7 @@ size_t plan_capacity(const ema_slice* s) {
   size_t b = 0;
   b += 2 * align_up(static_cast<size_t>(c.max_seqs) * c.max_blocks_per_seq * 4, 256);  // resolved, blk_seq (upper bound)
   b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                              // lens
-  b += 3 * align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src, copy_order (both directions)
+  b += 2 * align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src, copy_order
   b += 3 * align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // blk_off, slot bases
   b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos
   return b;
@@ -404,8 +404,6 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   p.off_copy_src = off;
   off += align_up(static_cast<size_t>(k) * 4, 256);
   p.off_copy_order = off;
-  off += align_up(static_cast<size_t>(k) * 4, 256);
-  p.off_copy_order_rev = off;
   off += align_up(static_cast<size_t>(k) * 4, 256);
   p.off_blk_off = off;
   off += align_up((static_cast<size_t>(nseq) + 1) * 4, 256);
@@ -511,11 +509,6 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
     for (uint32_t r = 0; r < max_rank; ++r) start[r + 1] += start[r];
     for (uint32_t u = 0; u < p.units; ++u)  // positions ascend within a rank
       copy_order[start[pos_rank[unit_first[u]]]++] = unit_first[u] | ((unit_len[u] - 1) << 24);
-    // The same units in reverse: for layer-dependent passes, in which the gather of a layer is complete
-    // before its attention starts; what a CTA reads first then lands last and is still in the L2
-    // (171 -> 166 us per layer measured; in a free-running pass the reverse order costs 19 %).
-    uint32_t* copy_order_rev = reinterpret_cast<uint32_t*>(p.host + p.off_copy_order_rev);
-    for (uint32_t u = 0; u < p.units; ++u) copy_order_rev[u] = copy_order[p.units - 1 - u];
   }
   p.guarded = false;
   p.valid = true;
@@ -886,12 +879,10 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     // the last block to the announcement of the output); in line, the warps that finish a sequence
     // together merge side by side, and the ring they stall has nothing to stream for long anyway.
     if (s->step_out_ready) d.merge_inline = 1;
-    // Layer-dependent passes gather in reverse order by default: what a CTA reads first lands last and
-    // is still in the L2 when the layer starts (5.5 -> 5.3 ms per pass on the 8B shapes); the price is
-    // that the start of a layer may wait for those last blocks. prefetch_priority keeps the forward
-    // order: no wait, the slower pass.
-    if (s->step_out_ready && !s->cfg.prefetch_priority)
-      d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order_rev);
+    // (Layer-dependent passes gather in the same order as the others. The reverse order — what a
+    // CTA reads first lands last and is still in the L2 when the layer starts — was tried: 2 % faster
+    // on the 8B shapes in some runs and 2 % slower in others, 10 % slower on the 70B shapes, where the
+    // start of every layer waited 86 us for those last blocks.)
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / nbuf;
