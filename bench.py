@@ -103,7 +103,7 @@ class DeviceWorkload:
 
     def __init__(self, wl: synth.Workload, seed: int, flags: int = 0, copy_kind: int = 0, copy_ctas: int = 0,
                  decode_ctas: int = 0, pipeline_mode: int = 0, static_split: int = 0, steal_floor: int = 0,
-                 prefetch_priority: int = 0):
+                 prefetch_priority: int = 0, swap_out: int = 0):
         import torch
         from paper_2609_27040_b200 import binding as B
         self.wl, self.B = wl, B
@@ -134,7 +134,7 @@ class DeviceWorkload:
                          local_free_order=pl.local_free_order, lent_free_order=pl.lent_free_order,
                          copy_kind=copy_kind, copy_ctas=copy_ctas, decode_ctas=decode_ctas,
                          pipeline_mode=pipeline_mode, static_split=static_split, steal_floor=steal_floor,
-                         prefetch_priority=prefetch_priority)
+                         prefetch_priority=prefetch_priority, swap_out=swap_out)
         t0 = time.perf_counter()
         for i, hints in enumerate(pl.hints):
             for h in hints:
@@ -619,6 +619,20 @@ def run_ours(args, wl):
                 ta = wa.timed(reps, wrap)
                 abl[label] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
                               "hbm_gbs_combined": step_bytes * reps / ta / 1e9}
+                del wa
+                torch.cuda.empty_cache()
+            # Swap-out beside swap-in (Section 2.3): the ring as a write-back cache, every staged layer written
+            # back to the lent arena by the copy threads of the same launch while it is attended to.
+            if args.pipeline_mode == 0:
+                wa = DeviceWorkload(wl, args.seed, pipeline_mode=0, swap_out=1, **kw)
+                for _ in range(3):
+                    wa.step(wrap)
+                ta = wa.timed(reps, wrap)
+                swap_bytes = step_bytes + L * wa.pref_bytes_layer
+                abl["swap_out_write_back"] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
+                                              "hbm_gbs_combined": swap_bytes * reps / ta / 1e9,
+                                              "note": "swap_out = 1: attention + gather + write-back of every staged layer "
+                                                      "(algorithmic bytes: attention + 4 x the lent bytes), one launch per pass"}
                 del wa
                 torch.cuda.empty_cache()
             # Two kernels on two streams with events, the pipeline the paper's description maps to most

@@ -193,10 +193,12 @@ typedef struct {
                                      to the staged copy; 1 = write-back: slice_append_kv writes a row
                                      whose block is staged to the staged copy only, and every pass of
                                      slice_decode_step writes each staged layer back to the lent
-                                     arena (all its staged blocks), on a stream of the library's own,
-                                     while that layer is attended to and the next transfer comes in;
-                                     a slot is refilled only after its write-back. Passes then run one
-                                     launch per layer. After an append, run a pass (or
+                                     arena (all its staged blocks) while that layer is attended to and
+                                     the next transfer comes in; a slot is refilled only after its
+                                     write-back. With pipeline_mode 0 the copy threads of the pass's
+                                     one launch do it; with the other pipelines the pass runs one
+                                     launch per layer and the write-back goes on a stream of the
+                                     library's own. After an append, run a pass (or
                                      slice_writeback_layer for the staged layers) before the tables
                                      change again, or the appended rows of staged blocks are lost   */
 } slice_config_t;

@@ -61,7 +61,8 @@ cudaError_t launch_copy(const CopyDesc& d, uint32_t kind, uint32_t ctas, int num
 //                           1 + 16*(sequence*Hkv + KV head) + (8 + query head of the group, for a
 //                           request that covers one query head only, else 0)
 constexpr uint32_t kLaunchCounters = 32;
-constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntMergePub = 16, kCntMergeTaken = 17, kCntMerged = 18;
+constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntWbTicket = 3, kCntWbDone = 4, kCntMergePub = 16, kCntMergeTaken = 17,
+                   kCntMerged = 18;
 constexpr uint32_t kMaxStepLayers = 128;
 // Consumer warps per KV head in the layer kernel, each leaving a partial of its own in every partial
 // slot: with 1, 2 or 4 KV heads the blocks of a unit are dealt to 8 / Hkv warps per head.
@@ -147,6 +148,9 @@ struct LayerParams {
                                 //   (low 24 bits) and blocks - 1 (high 8 bits) of a run of blocks that
                                 //   are neighbours in the lent arena and in the slot
   uint32_t copy_n;
+  uint32_t writeback;           // swap-out pass: while layer l >= writeback_from is attended to, the copy threads
+  uint32_t writeback_from;      //   also write its copy_n units back from the ring slot to the lent arena, and
+                                //   a slot is refilled only after the write-back of the layer it held
   uint32_t* ready;              // [ring_slots][ready_stride] per staged position: epoch of the layer
   uint32_t ready_stride;        //   whose block has landed there (multi-layer launches)
   uint32_t epoch_base;          // epoch of first_layer; layer l has epoch_base + (l - first_layer)

@@ -1478,27 +1478,17 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   // starts with what is left of the gather of the layer before.
   const uint32_t li_first = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin;
   volatile uint32_t* winding_down = sm.mq + kMqWind;
-  for (uint32_t li = li_first; li < p.li_end && ok; ++li) {
-    const int32_t target = p.gather_target[li];
-    if (target < 0 || p.copy_n == 0) continue;
-    const bool may_leave = p.chained && li >= p.li_begin && li + 1 < p.num_layers;
-    // The target's ring slot was last read by an earlier layer of this launch: wait for its attention.
-    const int32_t after = p.gather_after[li];
-    if (after >= 0) {
-      ok = wait_counter(layer_counters(p, static_cast<uint32_t>(after) - p.first_layer) + kCntAttnDone,
-                        p.total_blocks * p.Hkv, p.status);
-      if (!ok) break;
-    }
-    const uint8_t* src_layer = p.lent_base + layer_offset(static_cast<uint32_t>(target), p.layer_group, p.lent_group_stride, p.lent_layer_stride);
-    uint8_t* dst_slot = const_cast<uint8_t*>(p.staging_base) + (static_cast<uint32_t>(target) % p.ring_slots) * p.slot_bytes;
-    uint32_t* ticket = layer_counters(p, li) + kCntCopyTicket;
-    // A landed block is announced by writing the target layer's epoch to its position's ready flag
-    // (only when the target is attended to later in this launch).
-    const bool report = static_cast<uint32_t>(target) > p.first_layer + li && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
-    uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
-    const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
-    // A unit is a run of blocks that are neighbours both in the lent arena and in the slot (one block
-    // when blocks are 64 KB; up to 64 KB worth of smaller blocks that the slab allocator kept together).
+
+  // Moves the copy units of one layer between the lent arena and the layer's ring slot, in one
+  // direction: in (the gather: lent arena -> slot, landed positions announced through `ready`) or
+  // out (the write-back of a swap-out pass: slot -> lent arena). Units are drawn by ticket from
+  // `ticket`; returns the number of units this thread moved, all of them complete in global memory.
+  // A unit is a run of blocks that are neighbours both in the lent arena and in the slot (one block
+  // when blocks are 64 KB; up to 64 KB worth of smaller blocks that the slab allocator kept together).
+  auto transfer = [&](uint32_t layer, bool out, uint32_t* ticket, uint32_t* ready, uint32_t epoch, bool may_leave,
+                      uint32_t li_trace) -> uint32_t {
+    uint8_t* lent_layer = const_cast<uint8_t*>(p.lent_base) + layer_offset(layer, p.layer_group, p.lent_group_stride, p.lent_layer_stride);
+    uint8_t* slot = const_cast<uint8_t*>(p.staging_base) + (layer % p.ring_slots) * p.slot_bytes;
     uint32_t my_pos[16], my_n[16], my_end[16];  // this thread's most recent units: first position, blocks,
                                                 // and this layer's piece count once the unit is fully issued
     uint32_t my_units = 0;                // units of this layer taken by this thread
@@ -1535,8 +1525,10 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
         const int32_t e = static_cast<int32_t>(bat_e[bat_i]);
         ++bat_i;
         const uint32_t pos = v & 0xFFFFFFu, n = (v >> 24) + 1u;
-        src_blk = src_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
-        dst_blk = dst_slot + static_cast<uint64_t>(pos) * p.block_bytes;
+        uint8_t* in_arena = lent_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
+        uint8_t* in_slot = slot + static_cast<uint64_t>(pos) * p.block_bytes;
+        src_blk = out ? in_slot : in_arena;
+        dst_blk = out ? in_arena : in_slot;
         unit_bytes = static_cast<uint64_t>(n) * p.block_bytes;
         pieces = static_cast<uint32_t>((unit_bytes + kCopyChunk - 1) / kCopyChunk);
         my_pos[my_units % 16] = pos;
@@ -1573,7 +1565,8 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       const uint32_t stg = done % kNC;
       ok = ptx::mbar_wait(ptx::smem_u32(&sm.copy_full[stg]), (done / kNC) & 1u, p.status, kDevTimeout);
       if (!ok) break;
-      ptx::bulk_s2g_hint(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg], pol_keep);
+      // (what goes out to the lent arena is not read again before the next pass)
+      ptx::bulk_s2g_hint(sm.copy_dst[stg], ring + stg * kCopyChunk, sm.copy_len[stg], out ? pol : pol_keep);
       ptx::bulk_commit();
       ++done;
       // All but the newest kStoresOpen stores are complete after this wait: their stages may be
@@ -1585,7 +1578,55 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     }
     ptx::bulk_wait_all<0>();
     if (ok) report_landed(done - first_piece);
-    if (p.trace) p.trace[li * p.trace_stride + kTraceWords * blockIdx.x + 2] = ptx::global_timer_ns();
+    if (p.trace && !out) p.trace[li_trace * p.trace_stride + kTraceWords * blockIdx.x + 2] = ptx::global_timer_ns();
+    return my_units;
+  };
+
+  for (uint32_t li = li_first; li < p.li_end && ok; ++li) {
+    const uint32_t layer = p.first_layer + li;
+    const int32_t target = p.gather_target[li];
+    if (target >= 0 && p.copy_n != 0) {
+      const bool may_leave = p.chained && li >= p.li_begin && li + 1 < p.num_layers;
+      // The target's ring slot was last read by an earlier layer of this launch: wait for its attention
+      // and, in a swap-out pass, for its write-back (the slot's content is then safe in the lent arena).
+      const int32_t after = p.gather_after[li];
+      if (after >= 0) {
+        uint32_t* cnt = layer_counters(p, static_cast<uint32_t>(after) - p.first_layer);
+        ok = wait_counter(cnt + kCntAttnDone, p.total_blocks * p.Hkv, p.status);
+        if (ok && p.writeback && static_cast<uint32_t>(after) >= p.writeback_from) ok = wait_counter(cnt + kCntWbDone, p.copy_n, p.status);
+        if (!ok) break;
+      }
+      // A layer of the next pass (gathered at the end of this one) is read from the lent arena only
+      // after this pass has written it back.
+      if (p.writeback && static_cast<uint32_t>(target) < layer && static_cast<uint32_t>(target) >= p.writeback_from &&
+          static_cast<uint32_t>(target) >= p.first_layer) {
+        ok = wait_counter(layer_counters(p, static_cast<uint32_t>(target) - p.first_layer) + kCntWbDone, p.copy_n, p.status);
+        if (!ok) break;
+      }
+      // (the waits above were acquires of counters that bulk copies' completions were released to)
+      if (p.writeback) ptx::fence_proxy_async_global();
+      // A landed block is announced by writing the target layer's epoch to its position's ready flag
+      // (only when the target is attended to later in this launch).
+      const bool report = static_cast<uint32_t>(target) > layer && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
+      uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
+      const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
+      transfer(static_cast<uint32_t>(target), false, layer_counters(p, li) + kCntCopyTicket, ready, epoch, may_leave, li);
+      if (!ok) break;
+    }
+    // Swap-out pass (Section 2.3: what comes in is matched by what goes out): while this layer is attended
+    // to, its staged blocks, rows appended since they were fetched included, go back to the lent
+    // arena. The attention only reads the slot; nothing writes it before the gather that waits above.
+    if (p.writeback && p.copy_n != 0 && li >= p.li_begin && layer >= p.writeback_from) {
+      const uint32_t moved = transfer(layer, true, layer_counters(p, li) + kCntWbTicket, nullptr, 0, false, li);
+      if (!ok) break;
+      if (moved) {
+        // every store of this thread is complete (bulk_wait_all<0>); they went through the
+        // asynchronous proxy, the counter goes through the generic one
+        ptx::fence_proxy_async_global();
+        __threadfence();
+        atomicAdd(layer_counters(p, li) + kCntWbDone, moved);
+      }
+    }
   }
   if (!ok) {
     for (uint32_t k = done; k < issued; ++k)
@@ -1600,7 +1641,7 @@ __global__ void __launch_bounds__(352, 1) slice_layer_kernel(const LayerParams p
   bool gathers = false;
   if (p.copy_n)
     for (uint32_t li = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin; li < p.li_end; ++li)
-      gathers |= p.gather_target[li] >= 0;
+      gathers |= p.gather_target[li] >= 0 || p.writeback != 0;
   // A link of a chain of launches: the next link may start as soon as every CTA of this one has (it
   // takes the SMs that CTAs of this link leave, and waits for nothing but flags and counters).
   if (p.chained) ptx::launch_dependents();
@@ -1742,7 +1783,7 @@ cudaError_t launch_layer(const LayerParams& p, cudaStream_t stream) {
   bool gathers = false;
   if (p.copy_n)
     for (uint32_t li = p.chained && p.li_begin > 0 ? p.li_begin - 1 : p.li_begin; li < p.li_end; ++li)
-      gathers |= p.gather_target[li] >= 0;
+      gathers |= p.gather_target[li] >= 0 || p.writeback != 0;
   const size_t smem = smem_needed(p.Hkv, gathers);
   const unsigned threads = (p.Hkv * blocks_per_stage(p.Hkv) + 3) * 32;
   void* args[] = {const_cast<LayerParams*>(&p)};

@@ -716,6 +716,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.copy_src = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
   d.copy_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_copy_order);
   d.copy_n = p->units;
+  d.writeback = 0;
+  d.writeback_from = s->split;
   d.ready = s->ready_dev;
   d.ready_stride = s->cfg.staging_blocks_per_slot;
   d.epoch_base = 0;
@@ -883,6 +885,9 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     // CTA reads first lands last and is still in the L2 when the layer starts — was tried: 2 % faster
     // on the 8B shapes in some runs and 2 % slower in others, 10 % slower on the 70B shapes, where the
     // start of every layer waited 86 us for those last blocks.)
+    // Swap-out pass: the write-back of every staged layer is part of the launch (the copy threads do it
+    // while the layer is attended to; the gathers wait for it where they must).
+    d.writeback = s->cfg.swap_out && p->k ? 1u : 0u;
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / nbuf;
@@ -922,8 +927,13 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
         CU(s, cudaEventRecord(sl.attn_done, stream));
         CU(s, cudaEventRecord(sl.pref_done, stream));
         sl.attn_recorded = sl.pref_recorded = true;
+        if (s->cfg.swap_out) {
+          CU(s, cudaEventRecord(sl.wb_done, stream));
+          sl.wb_recorded = true;
+        }
       }
       sl.attn_stream = sl.pref_stream = stream;
+      if (s->cfg.swap_out) sl.wb_stream = stream;
     }
     if (holds[r] >= 0) {
       sl.valid = true;
@@ -1773,7 +1783,7 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
   // (Swap-out passes run layer by layer: the write-back of a layer goes on a stream of its own.)
   const bool step = (s->cfg.pipeline_mode == 0 || s->cfg.pipeline_mode == 3) && s->cfg.ring_slots >= 2 && L >= 2 &&
                     L <= ema::kMaxStepLayers &&
-                    s->ncta <= static_cast<uint32_t>(s->num_sms) && !s->cfg.swap_out;
+                    s->ncta <= static_cast<uint32_t>(s->num_sms) && !(s->cfg.swap_out && s->cfg.pipeline_mode == 3);
   const bool fused = s->cfg.pipeline_mode != 1 && s->cfg.ring_slots >= 2;
   if (fused) side = stream;
   const size_t per_layer = static_cast<size_t>(nseq) * Hq * kHeadDim * 2;

@@ -139,3 +139,33 @@ def test_timed_launch_configuration_matches_oracle_in_full(name, L, kw):
     for layer in sorted({0, mid, L - 1}):
         fb.check_attention_in_full(layer, resolved, k)
     fb.s.close()
+
+
+def test_swap_out_pass_at_full_batch_writes_the_ring_back_inside_its_one_launch():
+    """swap_out = 1 at the benchmark's size: the write-back of every staged layer is done by the copy
+    threads of the one launch that is the pass. A block of layer 0 is changed in its STAGED copy
+    only (as an appended row would); after the next pass the lent arena must hold the change, the
+    pass must have attended to it, and every other byte of the lent arena must be as it was."""
+    L = 6
+    fb = FullBatch("llama3_8b_decode", L, swap_out=1)
+    fb.decode_passes(1)                                        # leaves layer 0 staged in slot 0 for the next pass
+    before = fb.lent.clone()
+    rc, resolved, k = fb.orc.gather(0, fb.seqs, None, None)
+    assert rc == 0 and k == fb.pl.staging_blocks
+    # staging position 7 of the batch: which lent id is it?
+    ids = [~int(e) for i in range(fb.wl.batch) for e in fb.orc.block_table(i)[1][: synth.blocks_for(fb.pl.lengths[i])] if e < 0]
+    pos, lent_id = 7, ids[7]
+    assert torch.equal(fb.staging[0, pos], fb.lent[0, lent_id])
+    fb.staging[0, pos].mul_(-1.0)                              # the change exists in the ring only
+    changed = fb.staging[0, pos].clone()
+    assert not torch.equal(changed, fb.lent[0, lent_id])
+    k0 = fb.s.slice_stats()["kernel_launches"]
+    st = fb.decode_passes(1)
+    assert st["kernel_launches"] - k0 <= 3                     # one launch for the pass (+ at most the gathers of layer 0)
+    assert torch.equal(fb.lent[0, lent_id], changed)           # written back
+    before[0, lent_id] = changed
+    assert torch.equal(fb.lent, before)                        # and nothing else moved
+    resolved, k = fb.check_tables()
+    for layer in (0, 3, L - 1):                                # layer 0 was attended to with the change in place
+        fb.check_attention_in_full(layer, resolved, k)
+    fb.s.close()

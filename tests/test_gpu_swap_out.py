@@ -35,9 +35,12 @@ def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, ring):
 
     def check_pass():
         g.out.zero_()
+        k0 = g.s.slice_stats()["kernel_launches"]
         assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
         torch.cuda.synchronize()
         g.device_ok()
+        if mode == 0:      # the write-backs are part of the pass's one launch (plus, at most, gathers of the first layers)
+            assert g.s.slice_stats()["kernel_launches"] - k0 <= 1 + ring
         got = g.out.view(torch.bfloat16).double().cpu().numpy()
         for layer in range(sc.L):
             rc, resolved, k = sc.orc.gather(layer, sc.seq_ids, sc.lent, sc.staging)
