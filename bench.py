@@ -623,16 +623,18 @@ def run_ours(args, wl):
                 torch.cuda.empty_cache()
             # Swap-out beside swap-in (Section 2.3): the ring as a write-back cache, every staged layer written
             # back to the lent arena by the copy threads of the same launch while it is attended to.
-            if args.pipeline_mode == 0:
-                wa = DeviceWorkload(wl, args.seed, pipeline_mode=0, swap_out=1, **kw)
+            for label, swap in ((("swap_out_write_back", 1), ("swap_out_tail_blocks_only", 2)) if args.pipeline_mode == 0 else ()):
+                wa = DeviceWorkload(wl, args.seed, pipeline_mode=0, swap_out=swap, **kw)
                 for _ in range(3):
                     wa.step(wrap)
                 ta = wa.timed(reps, wrap)
-                swap_bytes = step_bytes + L * wa.pref_bytes_layer
-                abl["swap_out_write_back"] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
-                                              "hbm_gbs_combined": swap_bytes * reps / ta / 1e9,
-                                              "note": "swap_out = 1: attention + gather + write-back of every staged layer "
-                                                      "(algorithmic bytes: attention + 4 x the lent bytes), one launch per pass"}
+                swap_bytes = step_bytes + L * (wa.pref_bytes_layer if swap == 1 else 2 * wl.batch * wl.block_bytes)
+                abl[label] = {"tokens_per_s": wl.batch * reps / ta, "ms_per_step": ta / reps * 1e3,
+                              "hbm_gbs_combined": swap_bytes * reps / ta / 1e9,
+                              "note": ("swap_out = 1: attention + gather + write-back of every staged layer (algorithmic "
+                                       "bytes: attention + 4 x the lent bytes), one launch per pass" if swap == 1 else
+                                       "swap_out = 2: the write-back takes only the staged tail blocks, the ones an append "
+                                       "can have changed (at most one block per sequence and layer), one launch per pass")}
                 del wa
                 torch.cuda.empty_cache()
             # Two kernels on two streams with events, the pipeline the paper's description maps to most

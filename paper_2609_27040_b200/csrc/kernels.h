@@ -148,9 +148,11 @@ struct LayerParams {
                                 //   (low 24 bits) and blocks - 1 (high 8 bits) of a run of blocks that
                                 //   are neighbours in the lent arena and in the slot
   uint32_t copy_n;
-  uint32_t writeback;           // swap-out pass: while layer l >= writeback_from is attended to, the copy threads
-  uint32_t writeback_from;      //   also write its copy_n units back from the ring slot to the lent arena, and
-                                //   a slot is refilled only after the write-back of the layer it held
+  uint32_t writeback;           // swap-out pass (0 when wb_n is 0): while layer l >= writeback_from is attended to,
+  uint32_t writeback_from;      //   the copy threads also write the units wb_order[0 .. wb_n) back from its ring
+  const uint32_t* wb_order;     //   slot to the lent arena (units as in copy_order: all of them, or only the
+  uint32_t wb_n;                //   blocks that can have changed), and a slot is refilled only after the
+                                //   write-back of the layer it held
   uint32_t* ready;              // [ring_slots][ready_stride] per staged position: epoch of the layer
   uint32_t ready_stride;        //   whose block has landed there (multi-layer launches)
   uint32_t epoch_base;          // epoch of first_layer; layer l has epoch_base + (l - first_layer)

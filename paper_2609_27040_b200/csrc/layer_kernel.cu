@@ -1485,8 +1485,11 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
   // `ticket`; returns the number of units this thread moved, all of them complete in global memory.
   // A unit is a run of blocks that are neighbours both in the lent arena and in the slot (one block
   // when blocks are 64 KB; up to 64 KB worth of smaller blocks that the slab allocator kept together).
-  auto transfer = [&](uint32_t layer, bool out, uint32_t* ticket, uint32_t* ready, uint32_t epoch, bool may_leave,
-                      uint32_t li_trace) -> uint32_t {
+  // `ready` / `epoch`: on the way in, the flags to set for what has landed (or null); on the way out,
+  // the flags to wait for before a position is read (or null when the layer was staged before the
+  // launch): the slot may still be filling, by other CTAs' copy threads, when a write-back starts.
+  auto transfer = [&](uint32_t layer, bool out, uint32_t* ticket, const uint32_t* order, uint32_t count, uint32_t* ready,
+                      uint32_t epoch, bool may_leave, uint32_t li_trace) -> uint32_t {
     uint8_t* lent_layer = const_cast<uint8_t*>(p.lent_base) + layer_offset(layer, p.layer_group, p.lent_group_stride, p.lent_layer_stride);
     uint8_t* slot = const_cast<uint8_t*>(p.staging_base) + (layer % p.ring_slots) * p.slot_bytes;
     uint32_t my_pos[16], my_n[16], my_end[16];  // this thread's most recent units: first position, blocks,
@@ -1511,12 +1514,12 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
         if (bat_i == bat_n) {
           if (may_leave && *winding_down) return false;
           const uint32_t first = atomicAdd(ticket, batch);
-          if (first >= p.copy_n) return false;
-          bat_n = min(batch, p.copy_n - first);
+          if (first >= count) return false;
+          bat_n = min(batch, count - first);
           bat_i = 0;
 #pragma unroll
           for (uint32_t i = 0; i < 4; ++i)
-            if (i < bat_n) bat_v[i] = p.copy_order[first + i];
+            if (i < bat_n) bat_v[i] = order[first + i];
 #pragma unroll
           for (uint32_t i = 0; i < 4; ++i)
             if (i < bat_n) bat_e[i] = static_cast<uint32_t>(p.copy_src[bat_v[i] & 0xFFFFFFu]);
@@ -1525,6 +1528,11 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
         const int32_t e = static_cast<int32_t>(bat_e[bat_i]);
         ++bat_i;
         const uint32_t pos = v & 0xFFFFFFu, n = (v >> 24) + 1u;
+        if (out && ready) {
+          for (uint32_t i = 0; i < n && ok; ++i) ok = wait_counter_eq(ready + pos + i, epoch, p.status);
+          if (!ok) return false;
+          ptx::fence_proxy_async_global();  // the flags were acquired; the bulk loads read through the asynchronous proxy
+        }
         uint8_t* in_arena = lent_layer + static_cast<uint64_t>(static_cast<uint32_t>(~e)) * p.lent_block_stride;
         uint8_t* in_slot = slot + static_cast<uint64_t>(pos) * p.block_bytes;
         src_blk = out ? in_slot : in_arena;
@@ -1552,7 +1560,7 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
     };
     // Reports the units all of whose pieces are among the first `complete` stored pieces of this layer.
     auto report_landed = [&](uint32_t complete) {
-      if (!ready || reported == my_units || my_end[reported % 16] > complete) return;
+      if (out || !ready || reported == my_units || my_end[reported % 16] > complete) return;
       // The units' bulk stores are complete (wait_group); they went through the asynchronous proxy,
       // the flags go through the generic one: order the two, then publish with a release.
       ptx::fence_proxy_async_global();
@@ -1593,14 +1601,14 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       if (after >= 0) {
         uint32_t* cnt = layer_counters(p, static_cast<uint32_t>(after) - p.first_layer);
         ok = wait_counter(cnt + kCntAttnDone, p.total_blocks * p.Hkv, p.status);
-        if (ok && p.writeback && static_cast<uint32_t>(after) >= p.writeback_from) ok = wait_counter(cnt + kCntWbDone, p.copy_n, p.status);
+        if (ok && p.writeback && static_cast<uint32_t>(after) >= p.writeback_from) ok = wait_counter(cnt + kCntWbDone, p.wb_n, p.status);
         if (!ok) break;
       }
       // A layer of the next pass (gathered at the end of this one) is read from the lent arena only
       // after this pass has written it back.
       if (p.writeback && static_cast<uint32_t>(target) < layer && static_cast<uint32_t>(target) >= p.writeback_from &&
           static_cast<uint32_t>(target) >= p.first_layer) {
-        ok = wait_counter(layer_counters(p, static_cast<uint32_t>(target) - p.first_layer) + kCntWbDone, p.copy_n, p.status);
+        ok = wait_counter(layer_counters(p, static_cast<uint32_t>(target) - p.first_layer) + kCntWbDone, p.wb_n, p.status);
         if (!ok) break;
       }
       // (the waits above were acquires of counters that bulk copies' completions were released to)
@@ -1610,14 +1618,19 @@ __device__ void copy_role(const LayerParams& p, const Smem& sm) {
       const bool report = static_cast<uint32_t>(target) > layer && static_cast<uint32_t>(target) < p.first_layer + p.num_layers;
       uint32_t* ready = report ? p.ready + static_cast<size_t>(static_cast<uint32_t>(target) % p.ring_slots) * p.ready_stride : nullptr;
       const uint32_t epoch = p.epoch_base + (static_cast<uint32_t>(target) - p.first_layer);
-      transfer(static_cast<uint32_t>(target), false, layer_counters(p, li) + kCntCopyTicket, ready, epoch, may_leave, li);
+      transfer(static_cast<uint32_t>(target), false, layer_counters(p, li) + kCntCopyTicket, p.copy_order, p.copy_n, ready, epoch,
+               may_leave, li);
       if (!ok) break;
     }
     // Swap-out pass (Section 2.3: what comes in is matched by what goes out): while this layer is attended
     // to, its staged blocks, rows appended since they were fetched included, go back to the lent
     // arena. The attention only reads the slot; nothing writes it before the gather that waits above.
-    if (p.writeback && p.copy_n != 0 && li >= p.li_begin && layer >= p.writeback_from) {
-      const uint32_t moved = transfer(layer, true, layer_counters(p, li) + kCntWbTicket, nullptr, 0, false, li);
+    if (p.writeback && li >= p.li_begin && layer >= p.writeback_from) {
+      // (the same test as the attention's: was this layer gathered inside this launch?)
+      const bool filling = li >= p.prefetch_distance && p.gather_target[li - p.prefetch_distance] == static_cast<int16_t>(layer);
+      uint32_t* landed = filling ? p.ready + static_cast<size_t>(layer % p.ring_slots) * p.ready_stride : nullptr;
+      const uint32_t moved = transfer(layer, true, layer_counters(p, li) + kCntWbTicket, p.wb_order, p.wb_n, landed,
+                                      p.epoch_base + li, false, li);
       if (!ok) break;
       if (moved) {
         // every store of this thread is complete (bulk_wait_all<0>); they went through the

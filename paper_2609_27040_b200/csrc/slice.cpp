@@ -48,12 +48,13 @@ struct Plan {
   std::vector<int32_t> seqs;
   uint32_t nseq = 0, total_blocks = 0, k = 0;
   uint32_t units = 0;                    // copy units of the fused gather (runs of neighbouring staged blocks)
+  uint32_t tail_units = 0;               // staged tail blocks of the batch (the only staged blocks an append changes)
   uint32_t per = 1, used_cta = 0;        // attention ranges: range c = [c*per, min((c+1)*per, total))
   uint32_t slots = 0, slots_static = 0;  // partial slots with / without work stealing
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
   size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_blk_off = 0, off_slot_base = 0,
-         off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, bytes = 0;
+         off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, off_tail_order = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
   std::vector<int32_t> resolved_ids;  // resolved table in block ids (the device copy holds physical indices)
   uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
@@ -302,7 +303,7 @@ size_t plan_capacity(const ema_slice* s) {
   b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                              // lens
   b += 2 * align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src, copy_order
   b += 3 * align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // blk_off, slot bases
-  b += 2 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos
+  b += 3 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos, staged tail blocks
   return b;
 }
 
@@ -415,6 +416,8 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.off_stage_pos = off;
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
+  p.off_tail_order = off;
+  off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.bytes = off;
   if (off > p.cap) return SLICE_EINVAL;  // cannot happen: capacity is sized from the maxima
 
@@ -509,6 +512,14 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
     for (uint32_t r = 0; r < max_rank; ++r) start[r + 1] += start[r];
     for (uint32_t u = 0; u < p.units; ++u)  // positions ascend within a rank
       copy_order[start[pos_rank[unit_first[u]]]++] = unit_first[u] | ((unit_len[u] - 1) << 24);
+  }
+  // The staged tail blocks, as copy units of one block each: what a swap-out pass that writes back
+  // only what can have changed has to move (rows are appended to tail blocks and nowhere else).
+  {
+    uint32_t* tail_order = reinterpret_cast<uint32_t*>(p.host + p.off_tail_order);
+    p.tail_units = 0;
+    for (uint32_t i = 0; i < nseq; ++i)
+      if (stage_pos[i] >= 0) tail_order[p.tail_units++] = static_cast<uint32_t>(stage_pos[i]);
   }
   p.guarded = false;
   p.valid = true;
@@ -718,6 +729,8 @@ void fill_common(const ema_slice* s, const Plan* p, ema::LayerParams& d, uint32_
   d.copy_n = p->units;
   d.writeback = 0;
   d.writeback_from = s->split;
+  d.wb_order = nullptr;
+  d.wb_n = 0;
   d.ready = s->ready_dev;
   d.ready_stride = s->cfg.staging_blocks_per_slot;
   d.epoch_base = 0;
@@ -887,7 +900,14 @@ int do_step(ema_slice* s, Plan* p, const void* q, uint32_t Hq, float sm_scale, v
     // start of every layer waited 86 us for those last blocks.)
     // Swap-out pass: the write-back of every staged layer is part of the launch (the copy threads do it
     // while the layer is attended to; the gathers wait for it where they must).
-    d.writeback = s->cfg.swap_out && p->k ? 1u : 0u;
+    if (s->cfg.swap_out == 2) {  // only the blocks that can have changed
+      d.wb_order = reinterpret_cast<const uint32_t*>(p->dev + p->off_tail_order);
+      d.wb_n = p->tail_units;
+    } else if (s->cfg.swap_out) {
+      d.wb_order = d.copy_order;
+      d.wb_n = p->units;
+    }
+    d.writeback = d.wb_n ? 1u : 0u;
     d.epoch_base = s->epoch;
     s->epoch += L;  // one epoch per layer of every pass: a ready flag never matches a later layer
     const size_t rows = s->part_rows / nbuf;
@@ -1008,7 +1028,7 @@ int slice_create(const slice_config_t* cfg, slice_t** out) {
   if (cfg->num_kv_heads == 0 || cfg->num_kv_heads > 8 || cfg->num_layers == 0) return SLICE_EINVAL;
   if (cfg->ring_slots == 0 || cfg->lent_blocks > cfg->lent_blocks_physical) return SLICE_EINVAL;
   if (cfg->max_seqs == 0 || cfg->max_blocks_per_seq == 0 || cfg->lent_kind > 1 || cfg->copy_kind > 3) return SLICE_EINVAL;
-  if (cfg->pipeline_mode > 3 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 1) return SLICE_EINVAL;
+  if (cfg->pipeline_mode > 3 || cfg->static_split > 1 || cfg->prefetch_priority > 1 || cfg->swap_out > 2) return SLICE_EINVAL;
   // Section 4.2: slabs, layer groups, layouts.
   const uint32_t group = cfg->layer_group ? cfg->layer_group : 1u, slab = cfg->slab_blocks;
   if (cfg->layout > 2 || group > cfg->num_layers) return SLICE_EINVAL;

@@ -141,20 +141,28 @@ def test_timed_launch_configuration_matches_oracle_in_full(name, L, kw):
     fb.s.close()
 
 
-def test_swap_out_pass_at_full_batch_writes_the_ring_back_inside_its_one_launch():
-    """swap_out = 1 at the benchmark's size: the write-back of every staged layer is done by the copy
-    threads of the one launch that is the pass. A block of layer 0 is changed in its STAGED copy
-    only (as an appended row would); after the next pass the lent arena must hold the change, the
-    pass must have attended to it, and every other byte of the lent arena must be as it was."""
+@pytest.mark.parametrize("swap", [1, 2])
+def test_swap_out_pass_at_full_batch_writes_the_ring_back_inside_its_one_launch(swap):
+    """swap_out at the benchmark's size: the write-back of every staged layer (1), or of its staged
+    tail blocks only (2), is done by the copy threads of the one launch that is the pass. A block of
+    layer 0 is changed in its STAGED copy only (as an appended row would: a tail block); after the
+    next pass the lent arena must hold the change, the pass must have attended to it, and every
+    other byte of the lent arena must be as it was."""
     L = 6
-    fb = FullBatch("llama3_8b_decode", L, swap_out=1)
+    fb = FullBatch("llama3_8b_decode", L, swap_out=swap)
     fb.decode_passes(1)                                        # leaves layer 0 staged in slot 0 for the next pass
     before = fb.lent.clone()
     rc, resolved, k = fb.orc.gather(0, fb.seqs, None, None)
     assert rc == 0 and k == fb.pl.staging_blocks
-    # staging position 7 of the batch: which lent id is it?
-    ids = [~int(e) for i in range(fb.wl.batch) for e in fb.orc.block_table(i)[1][: synth.blocks_for(fb.pl.lengths[i])] if e < 0]
-    pos, lent_id = 7, ids[7]
+    # the first sequence whose tail block is lent: its staging position and its lent id
+    pos, lent_id, at = None, None, 0
+    for i in range(fb.wl.batch):
+        entries = fb.orc.block_table(i)[1][: synth.blocks_for(fb.pl.lengths[i])]
+        staged = [int(e) for e in entries if e < 0]
+        if pos is None and entries[-1] < 0:
+            pos, lent_id = at + len(staged) - 1, ~int(entries[-1])
+        at += len(staged)
+    assert pos is not None
     assert torch.equal(fb.staging[0, pos], fb.lent[0, lent_id])
     fb.staging[0, pos].mul_(-1.0)                              # the change exists in the ring only
     changed = fb.staging[0, pos].clone()

@@ -23,13 +23,15 @@ def _built():
     build_mod.build()
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("mode,swap", [(0, 1), (0, 2), (1, 1), (2, 1), (3, 1), (2, 2)])
 @pytest.mark.parametrize("ring", [2, 3])
-def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, ring):
+def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, swap, ring):
+    """swap = 1: every staged block of a layer is written back; swap = 2: only the blocks that can have
+    changed, the tail blocks (in the one-launch pass; the other pipelines write whole layers)."""
     from tests.gpu_helpers import GpuScenario, kv_to_host, to_dev
     wl = synth.Workload("swap", 5, 32, 8, 5, 17, 300, 0.5, ring_slots=ring)
     sc = Scenario(wl, 9, slack=16)
-    g = GpuScenario(sc, pipeline_mode=mode, swap_out=1, decode_ctas=12)
+    g = GpuScenario(sc, pipeline_mode=mode, swap_out=swap, decode_ctas=12)
     seqs = np.asarray(sc.seq_ids, np.int32)
     rng = np.random.default_rng(3)
 

@@ -54,7 +54,7 @@ def test_create_rejects_bad_configs():
         _null_slice(1, 8, 4, 4, 4, 4, 4, 4, lo=np.array([0, 0, 1, 2], np.uint32))   # not a permutation
     with pytest.raises(B.SliceError):
         B.Slice(1, 8, 4, 4, 4)                                     # device mode needs arenas
-    for kw in ({"pipeline_mode": 4}, {"copy_kind": 4}, {"prefetch_priority": 2}, {"swap_out": 2}):
+    for kw in ({"pipeline_mode": 4}, {"copy_kind": 4}, {"prefetch_priority": 2}, {"swap_out": 3}):
         with pytest.raises(B.SliceError):
             B.Slice(2, 8, 4, 4, 4, max_seqs=4, max_blocks_per_seq=4, flags=B.FLAG_NULL_DEVICE, **kw)
     for kw in ({"pipeline_mode": 3}, {"copy_kind": 3}):                # the chain of launches; the SM-sharing gather
