@@ -23,9 +23,10 @@ def _built():
     build_mod.build()
 
 
-@pytest.mark.parametrize("mode,swap", [(0, 1), (0, 2), (1, 1), (2, 1), (3, 1), (2, 2)])
+@pytest.mark.parametrize("mode,swap,dependent", [(0, 1, False), (0, 2, False), (1, 1, False), (2, 1, False), (3, 1, False),
+                                                 (2, 2, False), (0, 1, True), (0, 2, True)])
 @pytest.mark.parametrize("ring", [2, 3])
-def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, swap, ring):
+def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, swap, dependent, ring):
     """swap = 1: every staged block of a layer is written back; swap = 2: only the blocks that can have
     changed, the tail blocks (in the one-launch pass; the other pipelines write whole layers)."""
     from tests.gpu_helpers import GpuScenario, kv_to_host, to_dev
@@ -38,7 +39,13 @@ def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, swap, ring):
     def check_pass():
         g.out.zero_()
         k0 = g.s.slice_stats()["kernel_launches"]
-        assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
+        if dependent:      # the layer-dependent form of the pass: its queries released by the caller's stream
+            caller = torch.cuda.Stream()
+            assert g.s.slice_step_begin(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, True, g.main) == B.OK
+            for layer in range(sc.L):
+                assert g.s.slice_step_submit_q(layer, caller) == B.OK
+        else:
+            assert g.s.slice_decode_step(seqs, g.q, sc.Hq, float(sc.sm_scale), g.out, False, True, g.main, g.side) == B.OK
         torch.cuda.synchronize()
         g.device_ok()
         if mode == 0:      # the write-backs are part of the pass's one launch (plus, at most, gathers of the first layers)
