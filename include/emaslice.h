@@ -198,11 +198,12 @@ typedef struct {
                                      write-back. With pipeline_mode 0 the copy threads of the pass's
                                      one launch do it; with the other pipelines the pass runs one
                                      launch per layer and the write-back goes on a stream of the
-                                     library's own. 2 = the same, but a one-launch pass writes back
-                                     only the blocks that can have changed since they were fetched:
-                                     the staged tail block of every sequence of the batch (rows are
-                                     appended nowhere else), a few MB per layer instead of the
-                                     layer's whole lent part. After an append, run a pass (or
+                                     library's own. 2 = the same, but a pass writes back only the
+                                     blocks that can have changed since they were fetched: the staged
+                                     tail block of every sequence of the batch (rows are appended
+                                     nowhere else), a few MB per layer instead of the layer's whole
+                                     lent part (slice_writeback_layer still writes the whole layer).
+                                     After an append, run a pass (or
                                      slice_writeback_layer for the staged layers) before the tables
                                      change again, or the appended rows of staged blocks are lost   */
 } slice_config_t;

@@ -54,7 +54,7 @@ struct Plan {
   uint64_t tokens = 0;
   // byte offsets inside the plan buffer
   size_t off_resolved = 0, off_blk_seq = 0, off_lens = 0, off_copy_src = 0, off_copy_order = 0, off_blk_off = 0, off_slot_base = 0,
-         off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, off_tail_order = 0, bytes = 0;
+         off_slot_base_static = 0, off_home = 0, off_stage_pos = 0, off_tail_order = 0, off_tail_dst = 0, bytes = 0;
   std::vector<uint32_t> blk_off;  // host copy for the test hook
   std::vector<int32_t> resolved_ids;  // resolved table in block ids (the device copy holds physical indices)
   uint8_t* host = nullptr;        // pinned (plain memory in tables-only mode)
@@ -141,6 +141,7 @@ struct ema_slice {
   std::vector<StreamEpoch> streams;
   cudaEvent_t append_done = nullptr;
   bool append_pending = false;
+  bool in_pass = false;  // a write-back is being enqueued by slice_decode_step, not by slice_writeback_layer
   cudaStream_t append_stream = nullptr;
   cudaEvent_t ev_tmp = nullptr;
   // host io staging for slice_decode_step
@@ -303,7 +304,7 @@ size_t plan_capacity(const ema_slice* s) {
   b += align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                              // lens
   b += 2 * align_up(static_cast<size_t>(c.staging_blocks_per_slot) * 4, 256);           // copy_src, copy_order
   b += 3 * align_up((static_cast<size_t>(c.max_seqs) + 1) * 4, 256);                    // blk_off, slot bases
-  b += 3 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos, staged tail blocks
+  b += 4 * align_up(static_cast<size_t>(c.max_seqs) * 4, 256);                          // home, stage_pos, staged tail blocks (positions, homes)
   return b;
 }
 
@@ -418,6 +419,8 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.off_tail_order = off;
   off += align_up(static_cast<size_t>(nseq) * 4, 256);
+  p.off_tail_dst = off;
+  off += align_up(static_cast<size_t>(nseq) * 4, 256);
   p.bytes = off;
   if (off > p.cap) return SLICE_EINVAL;  // cannot happen: capacity is sized from the maxima
 
@@ -517,9 +520,13 @@ int get_plan(ema_slice* s, const int32_t* seqs, uint32_t nseq, Plan** out) {
   // only what can have changed has to move (rows are appended to tail blocks and nowhere else).
   {
     uint32_t* tail_order = reinterpret_cast<uint32_t*>(p.host + p.off_tail_order);
+    int32_t* tail_dst = reinterpret_cast<int32_t*>(p.host + p.off_tail_dst);  // their homes, for the stand-alone copy kernel
     p.tail_units = 0;
     for (uint32_t i = 0; i < nseq; ++i)
-      if (stage_pos[i] >= 0) tail_order[p.tail_units++] = static_cast<uint32_t>(stage_pos[i]);
+      if (stage_pos[i] >= 0) {
+        tail_dst[p.tail_units] = copy_src[stage_pos[i]];
+        tail_order[p.tail_units++] = static_cast<uint32_t>(stage_pos[i]);
+      }
   }
   p.guarded = false;
   p.valid = true;
@@ -1745,6 +1752,14 @@ int do_writeback(ema_slice* s, uint32_t layer, Plan* p, cudaStream_t stream) {
   d.src_entry = nullptr;
   d.dst_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_copy_src);
   d.n = p->k;
+  if (s->cfg.swap_out == 2 && s->in_pass) {
+    // Inside a pass only the staged tail blocks can differ from their homes (the explicit
+    // slice_writeback_layer call still writes the whole layer).
+    if (p->tail_units == 0) return SLICE_OK;
+    d.src_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_tail_order);
+    d.dst_entry = reinterpret_cast<const int32_t*>(p->dev + p->off_tail_dst);
+    d.n = p->tail_units;
+  }
   d.nlayers = 1;
   d.block_bytes = s->block_bytes;
   d.status = s->dev_status;
@@ -1924,7 +1939,9 @@ int decode_step_impl(ema_slice* s, const int32_t* seqs, uint32_t nseq, const voi
     // the layer's staged blocks go back to the lent arena, on a third stream, while the layer is
     // attended to and the next transfer comes in. The slot is refilled only after that write.
     if (s->cfg.swap_out && needs_staging(s, l, p->k) && staged(s, l, p)) {
+      s->in_pass = true;
       rc = do_writeback(s, l, p, s->swap_stream);
+      s->in_pass = false;
       if (rc) return rc;
     }
     // Layer-boundary check (Section 4.2.2): decide the next transfer before computing this layer.

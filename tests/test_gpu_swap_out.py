@@ -24,11 +24,11 @@ def _built():
 
 
 @pytest.mark.parametrize("mode,swap,dependent", [(0, 1, False), (0, 2, False), (1, 1, False), (2, 1, False), (3, 1, False),
-                                                 (2, 2, False), (0, 1, True), (0, 2, True)])
+                                                 (1, 2, False), (2, 2, False), (3, 2, False), (0, 1, True), (0, 2, True)])
 @pytest.mark.parametrize("ring", [2, 3])
 def test_appended_rows_reach_the_lent_arena_through_the_ring(mode, swap, dependent, ring):
     """swap = 1: every staged block of a layer is written back; swap = 2: only the blocks that can have
-    changed, the tail blocks (in the one-launch pass; the other pipelines write whole layers)."""
+    changed, the tail blocks."""
     from tests.gpu_helpers import GpuScenario, kv_to_host, to_dev
     wl = synth.Workload("swap", 5, 32, 8, 5, 17, 300, 0.5, ring_slots=ring)
     sc = Scenario(wl, 9, slack=16)
