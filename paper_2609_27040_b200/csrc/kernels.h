@@ -65,8 +65,8 @@ constexpr uint32_t kCntCopyTicket = 1, kCntAttnDone = 2, kCntWbTicket = 3, kCntW
                    kCntMerged = 18;
 constexpr uint32_t kMaxStepLayers = 128;
 // Consumer warps per KV head in the layer kernel, each leaving a partial of its own in every partial
-// slot: with 1, 2 or 4 KV heads the blocks of a unit are dealt to 8 / Hkv warps per head.
-__host__ __device__ constexpr uint32_t partials_per_slot(uint32_t Hkv) { return Hkv <= 2 || Hkv == 4 ? 8u / Hkv : 1u; }
+// slot: with 1 to 4 KV heads the blocks of a unit are dealt to 8 / Hkv (8, 4, 2, 2) warps per head.
+__host__ __device__ constexpr uint32_t partials_per_slot(uint32_t Hkv) { return Hkv <= 4 ? 8u / Hkv : 1u; }
 // Words of the per-CTA, per-layer trace of the layer kernel: [0] time the CTA started on the layer,
 // [1] ns its attention waited for prefetched blocks, [2] end of the copy work it did during the
 // layer, [3] SM id | runs << 16 | claims << 32, [4] time its producer had issued the layer's last

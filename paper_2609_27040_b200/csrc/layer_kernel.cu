@@ -152,8 +152,8 @@ static_assert(kNAFused * 32768 + kNC * 16384 >= kNAAlone * 32768, "the deeper ri
 // every KV head has V consumer warps, warp v taking block v of each group of V with a softmax state
 // and a partial of its own (the merge adds them up like any other partials).
 // Measured (64 sequences of 2k..8k tokens, nothing lent, KV read rate): 1 KV head 2.08 -> 4.46 TB/s,
-// 2 KV heads 4.17 -> 6.02, 4 KV heads 6.49 -> 6.79 (the same as one block per stage when the launch
-// also gathers); 3 KV heads (8 is no multiple) keep one block per stage and twice as many stages.
+// 2 KV heads 4.17 -> 6.02, 3 KV heads (two warps per head, six in all) 5.80 -> 6.52, 4 KV heads
+// 6.49 -> 6.79 (3 and 4 heads: the same as one block per stage when the launch also gathers).
 __host__ __device__ constexpr uint32_t blocks_per_stage(uint32_t Hkv) { return partials_per_slot(Hkv); }
 // A shared stage holds the V blocks whole (K plane and V plane are neighbours in memory: one request
 // of 8 or 16 KB per block instead of two of 4 or 8 KB), 64 KB per stage, two stages.
@@ -161,22 +161,20 @@ __host__ __device__ constexpr uint32_t stage_bytes(uint32_t Hkv) {
   return blocks_per_stage(Hkv) > 1 ? blocks_per_stage(Hkv) * 2 * half_stage_bytes(Hkv) : half_stage_bytes(Hkv);
 }
 constexpr uint32_t kGroupedStages = 2;     // beside a copy ring; 3 when the launch gathers nothing (4-5 % faster there)
-// Stages per 32 KB of ring: 2 for 3 or 4 KV heads (planes of 12 or 16 KB), else 1.
-__host__ __device__ constexpr uint32_t ring_scale(uint32_t Hkv) { return Hkv == 3 || Hkv == 4 ? 2u : 1u; }
 
 static_assert(kRingAlign + kNAFused * 32768 + kNC * kCopyChunk + kBarBytes + kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes +
                       kOwnBytes <= 232448,
               "more shared memory than a CTA can have (227 KB)");
 
 __host__ __device__ constexpr size_t smem_total(uint32_t Hkv) {
-  return kRingAlign + static_cast<size_t>(blocks_per_stage(Hkv) > 1 ? kGroupedStages : kNAFused * ring_scale(Hkv)) * stage_bytes(Hkv) +
+  return kRingAlign + static_cast<size_t>(blocks_per_stage(Hkv) > 1 ? kGroupedStages : kNAFused) * stage_bytes(Hkv) +
          static_cast<size_t>(kNC) * kCopyChunk + kBarBytes +
          kQueueBytes + kCopyDstBytes + kCopyLenBytes + kMqBytes + kOwnBytes;
 }
 
 // Attention stages of a launch: beside a copy ring, or alone (the launch gathers nothing).
 __host__ __device__ constexpr uint32_t attention_stages(uint32_t Hkv, bool gathers) {
-  return blocks_per_stage(Hkv) > 1 ? (gathers ? kGroupedStages : 3u) : (gathers ? kNAFused : kNAAlone) * ring_scale(Hkv);
+  return blocks_per_stage(Hkv) > 1 ? (gathers ? kGroupedStages : 3u) : (gathers ? kNAFused : kNAAlone);
 }
 // A launch that gathers nothing has no copy ring: the bookkeeping follows the attention ring, and with
 // 3 to 8 KV heads the CTA takes 100 KB, which leaves room on its SM for a CTA of the shared form of
