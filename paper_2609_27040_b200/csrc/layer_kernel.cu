@@ -177,7 +177,7 @@ __host__ __device__ constexpr uint32_t attention_stages(uint32_t Hkv, bool gathe
   return blocks_per_stage(Hkv) > 1 ? (gathers ? kGroupedStages : 3u) : (gathers ? kNAFused : kNAAlone);
 }
 // A launch that gathers nothing has no copy ring: the bookkeeping follows the attention ring, and with
-// 3 to 8 KV heads the CTA takes 100 KB, which leaves room on its SM for a CTA of the shared form of
+// 5 to 8 KV heads the CTA takes 100 KB, which leaves room on its SM for a CTA of the shared form of
 // the gather kernel (a gather on a second stream then really runs beside the attention).
 __host__ __device__ constexpr size_t smem_needed(uint32_t Hkv, bool gathers) {
   return kRingAlign + static_cast<size_t>(attention_stages(Hkv, gathers)) * stage_bytes(Hkv) +
@@ -377,7 +377,7 @@ __device__ void producer_role(const LayerParams& p, const Smem& sm) {
           ++nruns;
         }
         if constexpr (!kGrouped) {
-          // One block at a time, one stage per plane (3 to 8 KV heads: a plane is 12 to 32 KB).
+          // One block at a time, one stage per plane (5 to 8 KV heads: a plane is 20 to 32 KB).
           for (uint32_t blk = at; blk < ue && ok; ++blk) {
             const uint32_t j = blk - c.b;
             const int32_t e = __shfl_sync(0xffffffffu, my, j);
@@ -997,7 +997,7 @@ __device__ __forceinline__ void release_stage(const Smem& sm, const RingPos& pos
 }
 
 // ---------------------------------------------------------------------------------------------
-// consumer warp (= KV head g), tensor-core tiles, one block per stage (3 to 8 KV heads)
+// consumer warp (= KV head g), tensor-core tiles, one block per stage (5 to 8 KV heads)
 // ---------------------------------------------------------------------------------------------
 __device__ void consumer_mma_single(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
@@ -1110,7 +1110,7 @@ __device__ void consumer_mma_single(const LayerParams& p, const Smem& sm, uint32
 }
 
 // ---------------------------------------------------------------------------------------------
-// consumer warp (= KV head = query head g), f32 tiles for G == 1, one block per stage (3 to 8 KV heads)
+// consumer warp (= KV head = query head g), f32 tiles for G == 1, one block per stage (5 to 8 KV heads)
 // ---------------------------------------------------------------------------------------------
 __device__ void consumer_alu_single(const LayerParams& p, const Smem& sm, uint32_t g) {
   const uint32_t lane = threadIdx.x & 31u;
