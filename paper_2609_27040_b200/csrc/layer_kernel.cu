@@ -1764,7 +1764,7 @@ size_t layer_smem_bytes(uint32_t Hkv) {
 
 namespace {
 // The four instantiations: tensor-core or f32 tiles, one block per stage (5..8 KV heads) or groups of
-// 8 / Hkv blocks per stage (1 or 2 KV heads).
+// 8 / Hkv blocks per stage (1 to 4 KV heads).
 const void* layer_kernel_for(uint32_t Hkv, uint32_t G) {
   const bool grouped = blocks_per_stage(Hkv) > 1;
   if (G == 1)
